@@ -1,0 +1,360 @@
+"""Pins for the CPU oracle: what the paper's definitions and plain mathematics fix, checked without a GPU.
+
+Each test is chosen so that a plausible slip in the oracle (dropped term, wrong sign or index, transposed
+operand, wrong head grouping, wrong tie order) makes it fail.
+"""
+import itertools
+import json
+import math
+import os
+from fractions import Fraction
+
+import pytest
+import torch
+
+import oracle
+from helpers import random_cache
+
+GOLD = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "closed_forms.json")))
+
+
+def _scale(L, val):
+    return torch.full((L,), val, dtype=torch.float32)
+
+
+# --------------------------------------------------------------------------- attention (Sec. 4.2, Eq. 3)
+
+def test_golden_attention_and_relevance():
+    g = GOLD["attention"]
+    k = torch.tensor([[math.log(a), c] for a, c in zip(g["k_ln_of"], g["k_second_col"])], dtype=torch.float32)
+    v = torch.tensor(g["v"], dtype=torch.float32)
+    cap = 4
+    K = torch.zeros((1, 1, 1, cap, 2)); V = torch.zeros((1, 1, 1, cap, 2))
+    K[0, 0, 0, :3] = k; V[0, 0, 0, :3] = v
+    c = oracle.OracleCache(1, 1, 2, 1, 2, cap, K, V, torch.zeros((1, 1, 1, cap)),
+                           torch.zeros((1, 1, 1, cap), dtype=torch.int32), torch.tensor([[[3]]], dtype=torch.int32))
+    q = torch.tensor(g["q"], dtype=torch.float32).reshape(1, 1, 2, 2)
+    st, out, lse, probs = oracle.decode_attend(c, 0, 1, q, None, None, None, _scale(1, g["scale"]), 0.9,
+                                               want_lse=True, want_probs=True)
+    assert st == oracle.OK
+    assert torch.allclose(probs[0, 0, :, :3], torch.tensor(g["p"], dtype=torch.float64), atol=1e-7)
+    assert torch.allclose(out[0, 0].double(), torch.tensor(g["o"], dtype=torch.float64), atol=1e-5)
+    assert torch.allclose(c.rel[0, 0, 0, :3].double(), torch.tensor(g["rel_step1"], dtype=torch.float64), atol=1e-6)
+    assert abs(lse[0, 0, 0].item() - math.log(7.0)) < 1e-6 and abs(lse[0, 0, 1].item() - math.log(3.0)) < 1e-6
+    st, _, _, _ = oracle.decode_attend(c, 0, 1, q, None, None, None, _scale(1, g["scale"]), g["gamma2"])
+    assert torch.allclose(c.rel[0, 0, 0, :3].double(), torch.tensor(g["rel_step2"], dtype=torch.float64), atol=1e-6)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("Hq,Hkv", [(8, 2), (7, 1), (4, 4)])
+def test_attention_matches_library_sdpa(dtype, Hq, Hkv):
+    """Special case that reduces to a library routine: fp64 SDPA on K/V expanded per query head (Eq. 3's
+    `repeat`), with a different length for every item."""
+    L, B, D, cap = 2, 3, 16, 40
+    lens = torch.randint(1, cap + 1, (L, B, Hkv), generator=torch.Generator().manual_seed(5))
+    c = random_cache(L, B, Hq, Hkv, D, cap, lens, dtype=dtype, seed=11)
+    g = torch.Generator().manual_seed(3)
+    q = torch.randn((L, B, Hq, D), generator=g).to(dtype)
+    scale = torch.tensor([0.37, 0.11], dtype=torch.float32)
+    st, out, lse, probs = oracle.decode_attend(c, 0, L, q, None, None, None, scale, 0.5, want_lse=True,
+                                               want_probs=True)
+    assert st == oracle.OK
+    G = Hq // Hkv
+    for l in range(L):
+        for b in range(B):
+            for h in range(Hq):
+                n = int(lens[l, b, h // G])
+                kk = c.k[l, b, h // G, :n].double(); vv = c.v[l, b, h // G, :n].double()
+                ref = torch.nn.functional.scaled_dot_product_attention(
+                    q[l, b, h].double()[None, None, None, :], kk[None, None], vv[None, None],
+                    scale=float(scale[l]))[0, 0, 0]
+                tol = 1e-6 if dtype == torch.float32 else 1.6e-2   # bf16: one rounding of |o| < 4 is <= 2^-7
+                assert torch.allclose(out[l, b, h].double(), ref, atol=tol), (l, b, h)
+                s = (kk @ q[l, b, h].double()) * float(scale[l])
+                assert abs(lse[l, b, h].item() - torch.logsumexp(s, 0).item()) < 1e-5
+                assert abs(probs[l, b, h, :n].sum().item() - 1.0) < 1e-12          # softmax rows sum to one
+                assert torch.all(probs[l, b, h, n:] == 0)
+                # relevance from zero equals the group's summed library softmax (Eq. 5 with s_0 = 0)
+    for l in range(L):
+        for b in range(B):
+            for hk in range(Hkv):
+                n = int(lens[l, b, hk])
+                kk = c.k[l, b, hk, :n].double()
+                mass = torch.zeros(n, dtype=torch.float64)
+                for g_ in range(G):
+                    mass += torch.softmax((kk @ q[l, b, hk * G + g_].double()) * float(scale[l]), 0)
+                assert torch.allclose(c.rel[l, b, hk, :n].double(), mass, rtol=1e-6, atol=1e-8)
+                assert torch.all(c.rel[l, b, hk, n:] == 0)
+
+
+def test_uniform_attention_closed_forms():
+    """q = 0 gives p = 1/n and o = column mean of V; n = 1 gives o = V[0]."""
+    c = random_cache(1, 1, 4, 2, 8, 16, torch.tensor([[[9, 1]]]), seed=2)
+    q = torch.zeros((1, 1, 4, 8))
+    q[0, 0, 2:] = torch.randn((2, 8), generator=torch.Generator().manual_seed(1))   # heads of the n = 1 item
+    st, out, _, probs = oracle.decode_attend(c, 0, 1, q, None, None, None, _scale(1, 0.3), 0.9, want_probs=True)
+    assert torch.allclose(probs[0, 0, 0, :9], torch.full((9,), 1 / 9, dtype=torch.float64), atol=1e-15)
+    assert torch.allclose(out[0, 0, 0], c.v[0, 0, 0, :9].mean(0), atol=1e-6)
+    assert torch.equal(out[0, 0, 2], c.v[0, 0, 1, 0]) and torch.equal(out[0, 0, 3], c.v[0, 0, 1, 0])
+
+
+def test_append_semantics():
+    """The new token is written at slot len, gets pos = token_pos, starts at zero relevance and attends to
+    itself in the same step (Sec. 4.1)."""
+    c = random_cache(1, 2, 4, 2, 8, 8, 5, seed=4, rel_init="rand")
+    before = c.clone()
+    g = torch.Generator().manual_seed(9)
+    q = torch.randn((1, 2, 4, 8), generator=g); kn = torch.randn((1, 2, 2, 8), generator=g)
+    vn = torch.randn((1, 2, 2, 8), generator=g)
+    tp = torch.tensor([100, 200], dtype=torch.int32)
+    st, out, _, probs = oracle.decode_attend(c, 0, 1, q, kn, vn, tp, _scale(1, 0.35), 0.75, want_probs=True)
+    assert st == oracle.OK
+    assert torch.all(c.len == 6)
+    assert torch.equal(c.k[0, :, :, 5], kn[0]) and torch.equal(c.v[0, :, :, 5], vn[0])
+    assert torch.equal(c.k[0, :, :, :5], before.k[0, :, :, :5])
+    assert torch.all(c.pos[0, 0, :, 5] == 100) and torch.all(c.pos[0, 1, :, 5] == 200)
+    for b in range(2):
+        for hk in range(2):
+            mass = probs[0, b, 2 * hk:2 * hk + 2, :6].sum(0)
+            want = 0.75 * before.rel[0, b, hk, :6].double() + mass
+            want[5] = mass[5]                       # new token: zero history
+            assert torch.allclose(c.rel[0, b, hk, :6].double(), want, rtol=1e-6)
+            assert mass[5] > 0
+    # a full cache refuses the append and changes nothing
+    full = random_cache(1, 1, 2, 1, 4, 3, 3, seed=1)
+    snap = full.clone()
+    st, *_ = oracle.decode_attend(full, 0, 1, torch.zeros((1, 1, 2, 4)), torch.ones((1, 1, 1, 4)),
+                                  torch.ones((1, 1, 1, 4)), torch.tensor([7], dtype=torch.int32), _scale(1, 1.0), 0.9)
+    assert st == oracle.ERR_CAPACITY
+    assert torch.equal(full.k, snap.k) and torch.equal(full.len, snap.len)
+
+
+# --------------------------------------------------------------------------- relevance recurrence (Eq. 5)
+
+@pytest.mark.parametrize("gamma", [0.5, 0.9, 1.0])
+def test_relevance_mass_conservation(gamma):
+    """Without pruning every step adds exactly G (one unit of attention per query head), so from zero
+    sum_j rel_t = G (1 - gamma^t)/(1 - gamma), or G t when gamma = 1."""
+    L, B, Hq, Hkv, D, cap = 1, 2, 6, 2, 8, 24
+    G = Hq // Hkv
+    c = random_cache(L, B, Hq, Hkv, D, cap, 4, seed=8)
+    g = torch.Generator().manual_seed(21)
+    for t in range(1, 13):
+        q = torch.randn((L, B, Hq, D), generator=g); kn = torch.randn((L, B, Hkv, D), generator=g)
+        vn = torch.randn((L, B, Hkv, D), generator=g)
+        st, *_ = oracle.decode_attend(c, 0, L, q, kn, vn, torch.full((B,), t, dtype=torch.int32), _scale(L, 0.4),
+                                      gamma)
+        assert st == oracle.OK
+        want = G * t if gamma == 1.0 else G * (1 - gamma ** t) / (1 - gamma)
+        tot = c.rel.double().sum(-1)
+        assert torch.allclose(tot, torch.full_like(tot, want), rtol=1e-5)
+
+
+def test_relevance_linearity_in_history():
+    """rel after a block of steps = gamma^steps * (history) + (the same block run from zero history)."""
+    mk = lambda init: random_cache(1, 1, 4, 2, 8, 12, 12, seed=3, rel_init=init)
+    a, z = mk("rand"), mk("zero")
+    hist = a.rel.clone()
+    g = torch.Generator().manual_seed(2)
+    gamma, steps = 0.8, 5
+    for _ in range(steps):
+        q = torch.randn((1, 1, 4, 8), generator=g)
+        oracle.decode_attend(a, 0, 1, q, None, None, None, _scale(1, 0.5), gamma)
+        oracle.decode_attend(z, 0, 1, q, None, None, None, _scale(1, 0.5), gamma)
+    assert torch.allclose(a.rel.double(), gamma ** steps * hist.double() + z.rel.double(), rtol=2e-6, atol=1e-7)
+
+
+# --------------------------------------------------------------------------- Hoyer sparsity (Eq. 1)
+
+def _hoyer_cache(vectors, cap=None):
+    """One layer, one sequence, one KV head per vector."""
+    H = len(vectors)
+    cap = cap or max(len(v) for v in vectors)
+    rel = torch.zeros((1, 1, H, cap))
+    ln = torch.zeros((1, 1, H), dtype=torch.int32)
+    for i, v in enumerate(vectors):
+        rel[0, 0, i, :len(v)] = torch.tensor(v, dtype=torch.float32)
+        ln[0, 0, i] = len(v)
+    z = torch.zeros((1, 1, H, cap, 2))
+    return oracle.OracleCache(1, 1, H, H, 2, cap, z, z.clone(), rel, torch.zeros((1, 1, H, cap), dtype=torch.int32), ln)
+
+
+def test_golden_hoyer():
+    for case in GOLD["hoyer"]:
+        st, s = oracle.estimate_sparsity(_hoyer_cache([case["a"]]))
+        assert st == oracle.OK and abs(s.item() - case["expect"]) < 1e-6, case
+
+
+def test_hoyer_properties():
+    g = torch.Generator().manual_seed(0)
+    for n in (2, 3, 17, 100):
+        a = torch.rand(n, generator=g).tolist()
+        s1 = oracle.estimate_sparsity(_hoyer_cache([a]))[1].item()
+        s2 = oracle.estimate_sparsity(_hoyer_cache([[x * 37.5 for x in a]]))[1].item()
+        assert 0.0 <= s1 <= 1.0 and abs(s1 - s2) < 1e-6                      # range, scale invariance
+        for m in range(1, n + 1):                                            # m equal non-zeros of n
+            vec = [2.5] * m + [0.0] * (n - m)
+            want = (math.sqrt(n) - math.sqrt(m)) / (math.sqrt(n) - 1)
+            assert abs(oracle.estimate_sparsity(_hoyer_cache([vec]))[1].item() - want) < 1e-6
+    # degenerate: length 0 or 1, zero vector -> 0; slots beyond len are ignored
+    c = _hoyer_cache([[5.0], [0.0, 0.0, 0.0], [1.0, 1.0]], cap=6)
+    c.rel[0, 0, 2, 2:] = 99.0
+    assert abs(oracle.estimate_sparsity(c)[1].item()) < 1e-12
+    # layer value = mean over the KV heads
+    c = _hoyer_cache([[1.0, 0, 0, 0], [1.0, 1, 1, 1], [1.0, 1, 0, 0]])
+    assert abs(oracle.estimate_sparsity(c)[1].item() - (1 + 0 + (2 - math.sqrt(2))) / 3) < 1e-6
+
+
+# --------------------------------------------------------------------------- budgets (Sec. 4.2)
+
+def _lr_fraction(S, T, k_min):
+    """Exact-rational largest-remainder apportionment of the weights the rule defines."""
+    w = []
+    for s in S:
+        s32 = torch.tensor(s, dtype=torch.float32)
+        s32 = torch.where(s32 >= 0, s32, torch.zeros(())).clamp(max=1.0) if not math.isnan(s) else torch.zeros(())
+        d = (torch.tensor(1.0, dtype=torch.float32) - s32)
+        w.append(max(1, int(torch.round(d * 1048576.0).item())))
+    F = T - len(S) * k_min
+    W = sum(w)
+    quota = [Fraction(wi * F, W) for wi in w]
+    base = [q.numerator // q.denominator for q in quota]
+    order = sorted(range(len(S)), key=lambda i: (-(quota[i] - base[i]), i))
+    for i in order[:F - sum(base)]:
+        base[i] += 1
+    return [k_min + x for x in base]
+
+
+def test_golden_budgets():
+    for case in GOLD["budgets"]:
+        S = torch.tensor(case["sparsity"], dtype=torch.float32)[:, None]
+        st, k = oracle.alloc_budgets(S, torch.tensor([case["total"]], dtype=torch.int64), case["k_min"])
+        assert st == oracle.OK and k[:, 0].tolist() == case["expect"], case
+
+
+def test_budget_invariants_and_exact_rationals():
+    g = torch.Generator().manual_seed(7)
+    for trial in range(60):
+        L = int(torch.randint(1, 40, (1,), generator=g)); B = int(torch.randint(1, 5, (1,), generator=g))
+        S = torch.rand((L, B), generator=g)
+        if trial % 5 == 0:
+            S[0] = float("nan"); S[-1] = 1.0
+        if trial % 7 == 0:
+            S[:] = S[0, 0]                                       # all equal
+        k_min = int(torch.randint(0, 70, (1,), generator=g))
+        T = torch.randint(L * k_min, L * k_min + 5000, (B,), generator=g, dtype=torch.int64)
+        st, k = oracle.alloc_budgets(S, T, k_min)
+        assert st == oracle.OK
+        assert torch.equal(k.long().sum(0), T)                   # layer budgets sum to the global budget
+        assert torch.all(k >= k_min)
+        for b in range(B):
+            assert k[:, b].tolist() == _lr_fraction(S[:, b].tolist(), int(T[b]), k_min)
+            Sb = torch.nan_to_num(S[:, b], nan=0.0)
+            for i in range(L):                                   # sparser layer never gets more
+                for j in range(L):
+                    if Sb[i] > Sb[j]:
+                        assert k[i, b] <= k[j, b]
+        if trial % 7 == 0:
+            F = T - L * k_min
+            for b in range(B):
+                want = [k_min + int(F[b]) // L + (1 if l < int(F[b]) % L else 0) for l in range(L)]
+                assert k[:, b].tolist() == want
+    st, _ = oracle.alloc_budgets(torch.zeros((4, 1)), torch.tensor([39], dtype=torch.int64), 10)
+    assert st == oracle.ERR_BUDGET
+
+
+# --------------------------------------------------------------------------- selection and compaction
+
+def _prune_one(rel, k, recent, sink, D=4, seed=0):
+    n = len(rel)
+    c = random_cache(1, 1, 1, 1, D, n + 3, n, seed=seed)
+    c.rel[0, 0, 0, :n] = torch.tensor(rel, dtype=torch.float32)
+    before = c.clone()
+    st, keep = oracle.rasr_prune(c, torch.tensor([[k]], dtype=torch.int32), recent, sink, max_k=n + 3)
+    kept = [i for i in keep[0, 0, 0].tolist() if i >= 0]
+    return st, kept, c, before
+
+
+def test_golden_select():
+    g = GOLD["select"]
+    st, kept, c, before = _prune_one(g["rel"], g["budget"], g["recent"], g["sink"])
+    assert st == oracle.OK and kept == g["expect"]
+
+
+def test_select_brute_force_tiny():
+    """n <= 11: among all size-k supersets of the protected set, the kept set has the largest score sum and,
+    among those, the lexicographically smallest index tuple."""
+    g = torch.Generator().manual_seed(13)
+    for trial in range(120):
+        n = int(torch.randint(2, 12, (1,), generator=g))
+        sink = int(torch.randint(0, 3, (1,), generator=g)); recent = int(torch.randint(0, 4, (1,), generator=g))
+        # few distinct values -> many ties
+        rel = (torch.randint(0, 4, (n,), generator=g).float() * 0.25).tolist()
+        prot = set(range(min(sink, n))) | set(range(n - min(recent, n), n))
+        if len(prot) >= n:
+            continue
+        k = int(torch.randint(len(prot), n, (1,), generator=g))
+        st, kept, _, _ = _prune_one(rel, k, recent, sink, seed=trial)
+        assert st == oracle.OK and len(kept) == k and prot <= set(kept)
+        rest = [j for j in range(n) if j not in prot]
+        best = None
+        for extra in itertools.combinations(rest, k - len(prot)):
+            key = (-sum(rel[j] for j in extra), tuple(sorted(extra)))
+            if best is None or key < best:
+                best = key
+        assert tuple(sorted(set(kept) - prot)) == best[1], (rel, k, sink, recent, kept)
+
+
+def test_select_matches_stable_sort_and_compaction_is_a_gather():
+    g = torch.Generator().manual_seed(17)
+    for n, k, recent, sink in [(300, 100, 32, 4), (4096, 1000, 64, 4), (1000, 999, 0, 0), (513, 36, 32, 4),
+                               (200, 50, 0, 7), (200, 50, 9, 0)]:
+        rel = torch.rand(n, generator=g)
+        rel[torch.randint(0, n, (n // 3,), generator=g)] = 0.5           # ties
+        st, kept, c, before = _prune_one(rel.tolist(), k, recent, sink, D=8, seed=n)
+        assert st == oracle.OK and len(kept) == k == int(c.len[0, 0, 0])
+        cand = torch.arange(sink, n - recent)
+        order = torch.sort(rel[cand], descending=True, stable=True).indices
+        want = sorted(list(range(sink)) + list(range(n - recent, n)) + cand[order[:k - sink - recent]].tolist())
+        assert kept == want
+        idx = torch.tensor(kept)
+        assert torch.equal(c.k[0, 0, 0, :k], before.k[0, 0, 0, idx]) and torch.equal(c.v[0, 0, 0, :k], before.v[0, 0, 0, idx])
+        assert torch.equal(c.rel[0, 0, 0, :k], before.rel[0, 0, 0, idx]) and torch.equal(c.pos[0, 0, 0, :k], before.pos[0, 0, 0, idx])
+        assert torch.all(c.pos[0, 0, 0, 1:k] > c.pos[0, 0, 0, :k - 1])
+
+
+def test_select_special_cases():
+    rel = torch.rand(50, generator=torch.Generator().manual_seed(1)).tolist()
+    # budget >= length: bitwise identity (FullKV)
+    for k in (50, 51, 1000):
+        st, kept, c, before = _prune_one(rel, k, 8, 2)
+        assert st == oracle.OK and kept == list(range(50))
+        for name in ("k", "v", "rel", "pos", "len"):
+            assert torch.equal(getattr(c, name), getattr(before, name))
+    # budget = sink + recent: sinks plus window whatever the scores (StreamingLLM)
+    st, kept, _, _ = _prune_one(rel, 10, 8, 2)
+    assert kept == [0, 1] + list(range(42, 50))
+    # all scores equal: the oldest candidates survive (tie order made visible)
+    st, kept, _, _ = _prune_one([0.0] * 50, 15, 8, 2)
+    assert kept == list(range(7)) + list(range(42, 50))
+    # protected set larger than the budget: exactly the protected set, flagged
+    st, kept, c, _ = _prune_one(rel, 5, 8, 2)
+    assert st == oracle.ERR_BUDGET and kept == [0, 1] + list(range(42, 50)) and int(c.len[0, 0, 0]) == 10
+    # sink and recent overlap (n < sink + recent): nothing to drop beyond the union
+    st, kept, _, _ = _prune_one(rel[:6], 3, 4, 4)
+    assert st == oracle.ERR_BUDGET and kept == list(range(6))
+
+
+def test_multi_item_budgets_are_per_layer_and_sequence():
+    L, B, Hkv = 3, 2, 2
+    lens = torch.tensor([[[20, 25], [30, 18]], [[22, 22], [9, 40]], [[40, 40], [40, 40]]])
+    c = random_cache(L, B, 4, Hkv, 4, 48, lens, seed=5, rel_init="rand")
+    budgets = torch.tensor([[10, 20], [22, 12], [39, 40]], dtype=torch.int32)
+    st, keep = oracle.rasr_prune(c, budgets, 3, 1, max_k=48)
+    assert st == oracle.OK
+    for l in range(L):
+        for b in range(B):
+            for h in range(Hkv):
+                assert int(c.len[l, b, h]) == min(int(lens[l, b, h]), int(budgets[l, b]))
+                kk = [i for i in keep[l, b, h].tolist() if i >= 0]
+                assert len(kk) == int(c.len[l, b, h]) and kk == sorted(kk)
