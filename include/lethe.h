@@ -1,0 +1,186 @@
+/*
+ * lethe.h — C ABI of the B200 (sm_100a) Lethe hot path.
+ *
+ * Lethe (arXiv 2511.06029) keeps the KV cache of a decoding LLM small by pruning it
+ * repeatedly during generation: per layer, guided by measured attention sparsity
+ * (Sec. 4.2), and per token, guided by a decayed record of the attention each cached
+ * token has received (RASR, Sec. 4.3, Eq. 5).  This library is the data-parallel part
+ * of that loop:
+ *
+ *   lethe_decode_attend      one decode step: append the new token's k/v, softmax
+ *                            attention of the new query over the retained tokens, and
+ *                            the Eq. 5 relevance update, in one pass over K and V
+ *   lethe_estimate_sparsity  Eq. 1 (Hoyer) on the relevance vectors -> one value per
+ *                            (layer, sequence)
+ *   lethe_alloc_budgets      per-layer token budgets from those sparsities (Sec. 4.2)
+ *   lethe_rasr_prune         protected top-k retention + in-place stable compaction
+ *                            (Sec. 4.3; sink / recent sets of Algorithm 1)
+ *
+ * General conventions
+ *   - Unless marked HOST, every pointer is a DEVICE pointer to memory owned by the
+ *     caller; the library owns only the scratch inside lethe_ctx.
+ *   - All arrays are dense row-major in the index order written beside them.
+ *   - The four calls enqueue work on `stream` (a cudaStream_t passed as void*, NULL =
+ *     the legacy default stream) and return without synchronising.
+ *   - Errors detectable on the host return a status and enqueue nothing.  Conditions
+ *     only the device can see (a full cache on append, a budget below the protected
+ *     count, a page id outside the pool) never trap: the kernel skips or clamps the
+ *     item as documented, and records the first such event in a status word that
+ *     lethe_poll_status reads.
+ *   - Same inputs and same tuning give bitwise-identical results.  budgets, keep_idx,
+ *     len and the moved rows have exactly one correct value; out, rel and sparsity are
+ *     floating-point results.
+ *
+ * Notation: L layers, B sequences, Hq / Hkv query / KV heads, G = Hq / Hkv query heads
+ * per KV head (head h reads KV head h / G — the contiguous grouping that Eq. 3's
+ * `repeat` would produce), D head dimension.  An "item" is one (layer, sequence, KV
+ * head); n = len[item] is its number of retained tokens; slot j < n of an item is its
+ * j-th retained token in original order.
+ */
+#ifndef LETHE_H
+#define LETHE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lethe_ctx lethe_ctx; /* opaque: device id, scratch, status word, tuning */
+
+typedef enum {
+    LETHE_OK = 0,
+    LETHE_ERR_INVALID_ARG = 1, /* null pointer, bad shape / dtype / range */
+    LETHE_ERR_CAPACITY = 2,    /* device-side: append on an item with len == capacity */
+    LETHE_ERR_BUDGET = 3,      /* budget below the protected (sink + recent) count, or total < L * k_min */
+    LETHE_ERR_CUDA = 4,        /* a CUDA runtime call failed; see lethe_last_error */
+    LETHE_ERR_TIMEOUT = 5,     /* reserved: a bounded device-side wait ran out */
+    LETHE_ERR_UNSUPPORTED = 6, /* valid request outside what the kernels cover */
+    LETHE_ERR_PAGE = 7         /* device-side: page id outside [0, n_pages) */
+} lethe_status;
+
+enum { LETHE_F32 = 0, LETHE_BF16 = 1 };
+enum { LETHE_CONTIG = 0, LETHE_PAGED = 1 };
+
+/* Cache state of all layers (Sec. 4.1: per-layer K, V; Sec. 4.3: the score vector s_t). */
+typedef struct {
+    int32_t n_layers, batch, n_q_heads, n_kv_heads;
+    int32_t head_dim;    /* 64 or 128 */
+    int32_t dtype;       /* LETHE_F32 or LETHE_BF16: type of k, v, q, k_new, v_new, out */
+    int32_t layout;      /* LETHE_CONTIG or LETHE_PAGED */
+    int32_t capacity;    /* CONTIG: token slots per item.  PAGED: page-table entries per item */
+    int32_t page_tokens; /* PAGED: tokens per page (16); CONTIG: ignored */
+    void *k, *v;         /* CONTIG: [L][B][Hkv][capacity][D].  PAGED: pools [n_pages][page_tokens][D] */
+    float *rel;          /* [L][B][Hkv][cap_tokens]  Eq. 5 state s_t, indexed by logical slot           */
+    int32_t *pos;        /* [L][B][Hkv][cap_tokens]  original position of the token in each slot        */
+    int32_t *len;        /* [L][B][Hkv]              retained tokens per item                           */
+    int32_t *page_table; /* PAGED: [L][B][Hkv][capacity] page ids (never written by the library)       */
+    int64_t n_pages;     /* PAGED: pages in each pool                                                    */
+} lethe_cache;
+/* cap_tokens = capacity (CONTIG) or capacity * page_tokens (PAGED).  k, v and rel must be 16-byte aligned. */
+
+/* Create a context on CUDA device `device`.  scratch_bytes_hint (0 = default) sizes the
+ * device scratch the calls may use; it grows on demand (growth synchronises the device).
+ * Returns LETHE_ERR_CUDA if no usable sm_100 device / runtime is present. */
+lethe_status lethe_create(lethe_ctx **ctx, int device, size_t scratch_bytes_hint);
+void lethe_destroy(lethe_ctx *ctx);
+
+/* HOST string describing the last host-side error of this context (never NULL). */
+const char *lethe_last_error(const lethe_ctx *ctx);
+
+/* Synchronise `stream`, then return and clear the device status word: LETHE_OK or the first
+ * device-side error since the last poll.  info (HOST, optional, int32[2]) receives
+ * {status, flat item index l*B*Hkv + b*Hkv + h of the first offender}. */
+lethe_status lethe_poll_status(lethe_ctx *ctx, void *stream, int32_t *info);
+
+/* Tuning knobs (HOST values).  variant: 0 = automatic, 1 = CUDA-core kernel, 2 = tensor-core
+ * (mma) kernel (bf16 only).  splits: 0 = automatic, else CTAs per item (1, 2, 4, 8 or 16; they
+ * form one thread-block cluster).  Returns LETHE_ERR_INVALID_ARG for other values. */
+lethe_status lethe_set_tuning(lethe_ctx *ctx, int variant, int splits);
+
+/*
+ * One decode step for layers [layer_begin, layer_end)  (Sec. 4.1; Eq. 3; Eq. 5).
+ * With li = layer - layer_begin and nl = layer_end - layer_begin:
+ *   q      [nl][B][Hq][D]   query of the token being generated
+ *   k_new  [nl][B][Hkv][D]  its key and value; both NULL = attend without appending
+ *   v_new  [nl][B][Hkv][D]
+ *   token_pos [B] int32     original position of that token (written to pos[]); may be NULL
+ *                           when k_new is NULL
+ *   scale  HOST float[L]    softmax scale per layer, indexed by absolute layer (1/sqrt(D),
+ *                           or 1/(sqrt(D) T_l) for a layer temperature T_l)
+ *   gamma                   decay of Eq. 5, 0 < gamma <= 1
+ *   out    [nl][B][Hq][D]   attention output, cache dtype (bf16: round to nearest even)
+ *   lse    [nl][B][Hq] fp32 optional (NULL to skip): log-sum-exp of the scaled logits
+ * Per item: the new k/v row is written to slot n = len, rel[n] = 0, pos[n] = token_pos[b],
+ * len = n + 1; every query head h of the group attends over slots 0..n (the new token
+ * included): p_h = softmax_j(scale * q_h . K_j), out_h = sum_j p_hj V_j; then
+ * rel[j] = gamma * rel[j] + sum_{h in group} p_hj for every slot j.
+ * An item with len == cap_tokens cannot append: it is left untouched, its out rows are
+ * zero-filled, and LETHE_ERR_CAPACITY is recorded in the status word.
+ * An empty item (no append, len == 0) gives out = 0 and lse = -inf.
+ * Calls on the same items must be ordered (same stream or events): the call reads and
+ * writes k, v (the appended row), rel, pos and len.
+ */
+lethe_status lethe_decode_attend(lethe_ctx *ctx, const lethe_cache *cache, int layer_begin, int layer_end,
+                                 const void *q, const void *k_new, const void *v_new, const int32_t *token_pos,
+                                 const float *scale, float gamma, void *out, float *lse, void *stream);
+
+/*
+ * The same step with HOST-resident per-step tensors: q, k_new, v_new, token_pos and
+ * out (and lse if not NULL) are HOST pointers (pinned memory makes the copies
+ * asynchronous).  The call copies the inputs to context-owned device staging, runs
+ * lethe_decode_attend, and copies out (and lse) back, all on `stream`; the results are
+ * valid in host memory once `stream` has been synchronised.  The cache stays on the device.
+ */
+lethe_status lethe_decode_attend_host(lethe_ctx *ctx, const lethe_cache *cache, int layer_begin, int layer_end,
+                                      const void *q_host, const void *k_new_host, const void *v_new_host,
+                                      const int32_t *token_pos_host, const float *scale, float gamma, void *out_host,
+                                      float *lse_host, void *stream);
+
+/*
+ * Layer sparsity estimate (Eq. 1, Sec. 3.1; used per layer in Sec. 4.2).
+ * For every item, a = rel[0..n): S_item = (sqrt(n) - |a|_1 / |a|_2) / (sqrt(n) - 1), taken
+ * as 0 when n <= 1 or |a|_2 == 0 and clamped to [0, 1];
+ * sparsity[l][b] = mean over the Hkv items of (l, b).     sparsity: [L][B] fp32.
+ */
+lethe_status lethe_estimate_sparsity(lethe_ctx *ctx, const lethe_cache *cache, float *sparsity, void *stream);
+
+/*
+ * Per-layer budgets from sparsity (Sec. 4.2: sparse layers are given fewer tokens, dense
+ * layers more).  Integer arithmetic after one fp32 subtraction, so results are exact:
+ *   w_l = max(1, rint((1 - clamp(S_l, 0, 1)) * 2^20))   (NaN reads as S = 0)
+ *   F   = total_budget[b] - L * k_min
+ *   k_l = k_min + floor(w_l F / W) + [l among the F - sum floor(..) largest remainders
+ *                                      (w_l F) mod W, ties to the lower layer],  W = sum_l w_l
+ * so sum_l k_l == total_budget[b] and k_l >= k_min.
+ *   sparsity [L][B] fp32; total_budget [B] int64; budgets [L][B] int32 (output); L <= 1024.
+ * A sequence with total_budget[b] < L * k_min gets k_l = k_min for all l and records
+ * LETHE_ERR_BUDGET in the status word.
+ */
+lethe_status lethe_alloc_budgets(lethe_ctx *ctx, int n_layers, int batch, const float *sparsity,
+                                 const int64_t *total_budget, int32_t k_min, int32_t *budgets, void *stream);
+
+/*
+ * RASR retention for every item (Sec. 4.3; Algorithm 1's sink and recent sets), in place.
+ * With n = len[item], k = budgets[l][b]:
+ *   k >= n: the item is not touched.
+ *   else  : keep slots j < min(sink, n), slots j >= n - min(recent, n), and of the
+ *           remaining slots those with the largest rel (equal values: lower slot first)
+ *           until k slots are kept; if the protected slots alone outnumber k, exactly
+ *           they are kept and LETHE_ERR_BUDGET is recorded.  Survivors' rows of k, v, rel
+ *           and pos move to slots 0..k-1 in their old order (PAGED: logical slot i lives
+ *           in page page_table[i / page_tokens], offset i % page_tokens; pages from index
+ *           ceil(len / page_tokens) on are free for the caller to reuse); len = k.
+ *   budgets  [L][B] int32
+ *   keep_idx optional (NULL to skip) [L][B][Hkv][max_k] int32: the old slot of each
+ *            survivor in ascending order, -1 padded; an untouched item lists 0..n-1
+ *            (the first max_k of them).
+ */
+lethe_status lethe_rasr_prune(lethe_ctx *ctx, const lethe_cache *cache, const int32_t *budgets, int32_t recent,
+                              int32_t sink, int32_t *keep_idx, int32_t max_k, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LETHE_H */

@@ -1,0 +1,356 @@
+// C ABI of the Lethe hot path: argument checking, launch geometry, context-owned scratch and status word.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "common.cuh"
+
+namespace lethe {
+cudaError_t launch_attend_simt(const AttendArgs& a, int dtype, int D, bool paged, cudaStream_t stream);
+size_t simt_smem_bytes(int D, int chunk_tokens, int GP);
+cudaError_t launch_attend_mma(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream);
+size_t mma_smem_bytes(int D, int shape, int chunk_tokens, int GP);
+cudaError_t launch_sparsity(const CacheView& c, float* sparsity, cudaStream_t stream);
+cudaError_t launch_budgets(int L, int B, const float* sparsity, const long long* total, int k_min, int32_t* budgets,
+                           int32_t* status, cudaStream_t stream);
+cudaError_t launch_rasr_prune(const CacheView& c, const int32_t* budgets, int recent, int sink, int32_t* keep_idx,
+                              int max_k, int smem_tokens, int32_t* list_scratch, int32_t* status,
+                              cudaStream_t stream);
+}  // namespace lethe
+
+using namespace lethe;
+
+struct lethe_ctx {
+    int device;
+    int sm_count;
+    size_t max_smem;  // opt-in dynamic shared memory per CTA
+    int32_t* status;  // device: {code, item}
+    void* scratch;
+    size_t scratch_bytes;
+    void* staging;  // device staging of lethe_decode_attend_host
+    size_t staging_bytes;
+    int variant, splits;
+    char err[256];
+};
+
+static lethe_status fail(lethe_ctx* ctx, lethe_status st, const char* fmt, const char* detail = "") {
+    if (ctx) snprintf(ctx->err, sizeof(ctx->err), fmt, detail);
+    return st;
+}
+
+static lethe_status cuda_fail(lethe_ctx* ctx, cudaError_t e, const char* where) {
+    if (ctx) snprintf(ctx->err, sizeof(ctx->err), "%s: %s", where, cudaGetErrorString(e));
+    return LETHE_ERR_CUDA;
+}
+
+namespace {
+struct DeviceGuard {
+    int prev = -1;
+    bool ok;
+    explicit DeviceGuard(int dev) {
+        ok = cudaGetDevice(&prev) == cudaSuccess && (prev == dev || cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+lethe_status ensure(lethe_ctx* ctx, void** buf, size_t* have, size_t need, const char* what) {
+    if (need <= *have) return LETHE_OK;
+    cudaError_t e = cudaDeviceSynchronize();  // the old buffer may still be in use
+    if (e != cudaSuccess) return cuda_fail(ctx, e, what);
+    if (*buf) cudaFree(*buf);
+    *buf = nullptr;
+    *have = 0;
+    size_t sz = need + need / 4;
+    e = cudaMalloc(buf, sz);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, what);
+    *have = sz;
+    return LETHE_OK;
+}
+
+lethe_status check_cache(lethe_ctx* ctx, const lethe_cache* c) {
+    if (!ctx) return LETHE_ERR_INVALID_ARG;
+    if (!c) return fail(ctx, LETHE_ERR_INVALID_ARG, "cache is NULL");
+    if (!c->k || !c->v || !c->rel || !c->pos || !c->len) return fail(ctx, LETHE_ERR_INVALID_ARG, "cache has a NULL tensor");
+    if (c->n_layers < 1 || c->batch < 1 || c->n_kv_heads < 1 || c->n_q_heads < 1)
+        return fail(ctx, LETHE_ERR_INVALID_ARG, "cache dimensions must be positive");
+    if (c->n_q_heads % c->n_kv_heads) return fail(ctx, LETHE_ERR_INVALID_ARG, "n_q_heads must be a multiple of n_kv_heads");
+    if (c->head_dim != 64 && c->head_dim != 128) return fail(ctx, LETHE_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+    if (c->dtype != LETHE_F32 && c->dtype != LETHE_BF16) return fail(ctx, LETHE_ERR_INVALID_ARG, "unknown dtype");
+    if (c->layout != LETHE_CONTIG && c->layout != LETHE_PAGED) return fail(ctx, LETHE_ERR_INVALID_ARG, "unknown layout");
+    if (c->capacity < 1) return fail(ctx, LETHE_ERR_INVALID_ARG, "capacity must be positive");
+    if (c->layout == LETHE_PAGED) {
+        if (!c->page_table || c->page_tokens < 1 || c->n_pages < 1)
+            return fail(ctx, LETHE_ERR_INVALID_ARG, "paged layout needs page_table, page_tokens and n_pages");
+        if ((long long)c->capacity * c->page_tokens > 0x7fffffffLL) return fail(ctx, LETHE_ERR_INVALID_ARG, "capacity too large");
+    }
+    if (((uintptr_t)c->k | (uintptr_t)c->v | (uintptr_t)c->rel) & 15) return fail(ctx, LETHE_ERR_INVALID_ARG, "k, v, rel must be 16-byte aligned");
+    const long long items = (long long)c->n_layers * c->batch * c->n_kv_heads;
+    if (items > 0x7fffffffLL / 16) return fail(ctx, LETHE_ERR_UNSUPPORTED, "too many (layer, sequence, head) items");
+    return LETHE_OK;
+}
+
+int cap_tokens_of(const lethe_cache* c) { return c->layout == LETHE_PAGED ? c->capacity * c->page_tokens : c->capacity; }
+
+CacheView view_of(const lethe_cache* c) {
+    CacheView v;
+    v.k = c->k; v.v = c->v; v.rel = c->rel; v.pos = c->pos; v.len = c->len; v.page_table = c->page_table;
+    v.n_pages = c->n_pages;
+    v.L = c->n_layers; v.B = c->batch; v.Hkv = c->n_kv_heads; v.D = c->head_dim;
+    v.elt_bytes = c->dtype == LETHE_BF16 ? 2 : 4;
+    v.capacity = c->capacity; v.cap_tokens = cap_tokens_of(c);
+    v.page_tokens = c->layout == LETHE_PAGED ? c->page_tokens : 1;
+    v.paged = c->layout == LETHE_PAGED;
+    return v;
+}
+}  // namespace
+
+extern "C" {
+
+lethe_status lethe_create(lethe_ctx** out, int device, size_t scratch_bytes_hint) {
+    if (!out) return LETHE_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return LETHE_ERR_CUDA;
+    DeviceGuard guard(device);
+    if (!guard.ok) return LETHE_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return LETHE_ERR_CUDA;
+    if (prop.major != 10) return LETHE_ERR_CUDA;  // built for sm_100a only
+    lethe_ctx* ctx = new (std::nothrow) lethe_ctx();
+    if (!ctx) return LETHE_ERR_CUDA;
+    memset(ctx, 0, sizeof(*ctx));
+    ctx->device = device;
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->max_smem = prop.sharedMemPerBlockOptin;
+    strcpy(ctx->err, "no error");
+    if (cudaMalloc((void**)&ctx->status, 2 * sizeof(int32_t)) != cudaSuccess ||
+        cudaMemset(ctx->status, 0, 2 * sizeof(int32_t)) != cudaSuccess) {
+        delete ctx;
+        return LETHE_ERR_CUDA;
+    }
+    if (scratch_bytes_hint) {
+        if (ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, scratch_bytes_hint, "scratch") != LETHE_OK) {
+            cudaFree(ctx->status);
+            delete ctx;
+            return LETHE_ERR_CUDA;
+        }
+    }
+    *out = ctx;
+    return LETHE_OK;
+}
+
+void lethe_destroy(lethe_ctx* ctx) {
+    if (!ctx) return;
+    DeviceGuard guard(ctx->device);
+    cudaDeviceSynchronize();
+    if (ctx->status) cudaFree(ctx->status);
+    if (ctx->scratch) cudaFree(ctx->scratch);
+    if (ctx->staging) cudaFree(ctx->staging);
+    delete ctx;
+}
+
+const char* lethe_last_error(const lethe_ctx* ctx) { return ctx ? ctx->err : "context is NULL"; }
+
+lethe_status lethe_poll_status(lethe_ctx* ctx, void* stream, int32_t* info) {
+    if (!ctx) return LETHE_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "poll_status: synchronize");
+    int32_t h[2] = {0, 0};
+    e = cudaMemcpyAsync(h, ctx->status, sizeof(h), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "poll_status: read");
+    if (h[0] != 0) {
+        e = cudaMemsetAsync(ctx->status, 0, sizeof(h), s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "poll_status: clear");
+        snprintf(ctx->err, sizeof(ctx->err), "device-side status %d at item %d", h[0], h[1]);
+    }
+    if (info) {
+        info[0] = h[0];
+        info[1] = h[1];
+    }
+    return (lethe_status)h[0];
+}
+
+lethe_status lethe_set_tuning(lethe_ctx* ctx, int variant, int splits) {
+    if (!ctx) return LETHE_ERR_INVALID_ARG;
+    if (variant < 0 || variant > 3) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..3");
+    if (!(splits == 0 || splits == 1 || splits == 2 || splits == 4 || splits == 8 || splits == 16))
+        return fail(ctx, LETHE_ERR_INVALID_ARG, "splits must be 0, 1, 2, 4, 8 or 16");
+    ctx->variant = variant;
+    ctx->splits = splits;
+    return LETHE_OK;
+}
+
+lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer_begin, int layer_end, const void* q,
+                                 const void* k_new, const void* v_new, const int32_t* token_pos, const float* scale,
+                                 float gamma, void* out, float* lse, void* stream) {
+    lethe_status st = check_cache(ctx, c);
+    if (st != LETHE_OK) return st;
+    if (!q || !out || !scale) return fail(ctx, LETHE_ERR_INVALID_ARG, "q, out and scale are required");
+    if (layer_begin < 0 || layer_end > c->n_layers || layer_begin >= layer_end)
+        return fail(ctx, LETHE_ERR_INVALID_ARG, "bad layer range");
+    if ((k_new == nullptr) != (v_new == nullptr)) return fail(ctx, LETHE_ERR_INVALID_ARG, "k_new and v_new go together");
+    if (k_new && !token_pos) return fail(ctx, LETHE_ERR_INVALID_ARG, "token_pos is required when appending");
+    if (!(gamma > 0.f && gamma <= 1.f)) return fail(ctx, LETHE_ERR_INVALID_ARG, "gamma must be in (0, 1]");
+    if (c->n_layers > kMaxLayers) return fail(ctx, LETHE_ERR_UNSUPPORTED, "more than 128 layers");
+    const int G = c->n_q_heads / c->n_kv_heads;
+    if (G > kMaxGroup) return fail(ctx, LETHE_ERR_UNSUPPORTED, "more than 8 query heads per KV head");
+    if (((uintptr_t)q | (uintptr_t)out | (uintptr_t)k_new | (uintptr_t)v_new) & 15)
+        return fail(ctx, LETHE_ERR_INVALID_ARG, "q, k_new, v_new, out must be 16-byte aligned");
+    for (int l = layer_begin; l < layer_end; ++l)
+        if (!(scale[l] == scale[l]) || fabsf(scale[l]) > 1e30f) return fail(ctx, LETHE_ERR_INVALID_ARG, "scale must be finite");
+
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, LETHE_ERR_CUDA, "cannot select the context's device");
+
+    AttendArgs a;
+    memset(&a, 0, sizeof(a));
+    a.k = c->k; a.v = c->v; a.rel = c->rel; a.pos = c->pos; a.len = c->len; a.page_table = c->page_table;
+    a.q = q; a.k_new = k_new; a.v_new = v_new; a.token_pos = token_pos; a.out = out; a.lse = lse;
+    a.status = ctx->status;
+    a.n_pages = c->n_pages;
+    a.B = c->batch; a.Hq = c->n_q_heads; a.Hkv = c->n_kv_heads; a.G = G; a.GP = (G + 1) & ~1;
+    a.capacity = c->capacity; a.cap_tokens = cap_tokens_of(c);
+    a.page_tokens = c->layout == LETHE_PAGED ? c->page_tokens : 1;
+    a.layer_begin = layer_begin;
+    a.n_items = (layer_end - layer_begin) * c->batch * c->n_kv_heads;
+    a.gamma = gamma;
+    for (int l = 0; l < c->n_layers; ++l) a.scale_log2[l] = scale[l] * 1.4426950408889634f;
+
+    const bool paged = c->layout == LETHE_PAGED;
+    const bool mma_ok = c->dtype == LETHE_BF16 && (!paged || c->page_tokens == kGroupTokens);
+    int variant = ctx->variant;
+    if (variant == 0) variant = mma_ok ? 2 : 1;
+    if (variant >= 2 && !mma_ok) return fail(ctx, LETHE_ERR_UNSUPPORTED, "tensor-core variant needs bf16 and 16-token pages");
+
+    // CTAs per item: the smallest cluster whose logit buffer fits, grown until the grid covers the SMs twice.
+    const int cap_groups = (a.cap_tokens + kGroupTokens - 1) / kGroupTokens;
+    auto smem_for = [&](int S) -> size_t {
+        const int chunk = ((cap_groups + S - 1) / S) * kGroupTokens;
+        return variant == 1 ? simt_smem_bytes(c->head_dim, chunk, a.GP) : mma_smem_bytes(c->head_dim, variant - 2, chunk, a.GP);
+    };
+    int S = ctx->splits;
+    if (S == 0) {
+        S = 1;
+        while (S < 16 && smem_for(S) > ctx->max_smem) S *= 2;
+        while (S < 8 && (long long)a.n_items * S < 2LL * ctx->sm_count && cap_groups / (2 * S) >= 4) S *= 2;
+    }
+    if (smem_for(S) > ctx->max_smem)
+        return fail(ctx, LETHE_ERR_UNSUPPORTED, "capacity too large for the on-chip logit buffer at this split count");
+    a.splits = S;
+    a.chunk_tokens = ((cap_groups + S - 1) / S) * kGroupTokens;
+
+    cudaError_t e = variant == 1 ? launch_attend_simt(a, c->dtype, c->head_dim, paged, (cudaStream_t)stream)
+                                 : launch_attend_mma(a, c->head_dim, variant - 2, paged, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attend launch");
+    return LETHE_OK;
+}
+
+lethe_status lethe_decode_attend_host(lethe_ctx* ctx, const lethe_cache* c, int layer_begin, int layer_end,
+                                      const void* q_host, const void* k_new_host, const void* v_new_host,
+                                      const int32_t* token_pos_host, const float* scale, float gamma, void* out_host,
+                                      float* lse_host, void* stream) {
+    lethe_status st = check_cache(ctx, c);
+    if (st != LETHE_OK) return st;
+    if (!q_host || !out_host) return fail(ctx, LETHE_ERR_INVALID_ARG, "q and out are required");
+    if (layer_begin < 0 || layer_end > c->n_layers || layer_begin >= layer_end)
+        return fail(ctx, LETHE_ERR_INVALID_ARG, "bad layer range");
+    if ((k_new_host == nullptr) != (v_new_host == nullptr)) return fail(ctx, LETHE_ERR_INVALID_ARG, "k_new and v_new go together");
+    if (k_new_host && !token_pos_host) return fail(ctx, LETHE_ERR_INVALID_ARG, "token_pos is required when appending");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, LETHE_ERR_CUDA, "cannot select the context's device");
+    const size_t nl = (size_t)(layer_end - layer_begin);
+    const size_t eb = c->dtype == LETHE_BF16 ? 2 : 4;
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    const size_t q_bytes = nl * c->batch * c->n_q_heads * c->head_dim * eb;
+    const size_t kv_bytes = nl * c->batch * c->n_kv_heads * c->head_dim * eb;
+    const size_t pos_bytes = (size_t)c->batch * 4;
+    const size_t lse_bytes = nl * c->batch * c->n_q_heads * 4;
+    const size_t total = 2 * up(q_bytes) + 2 * up(kv_bytes) + up(pos_bytes) + up(lse_bytes);
+    st = ensure(ctx, &ctx->staging, &ctx->staging_bytes, total, "staging");
+    if (st != LETHE_OK) return st;
+    char* p = (char*)ctx->staging;
+    void* dq = p; p += up(q_bytes);
+    void* dout = p; p += up(q_bytes);
+    void* dk = p; p += up(kv_bytes);
+    void* dv = p; p += up(kv_bytes);
+    int32_t* dpos = (int32_t*)p; p += up(pos_bytes);
+    float* dlse = (float*)p;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess && k_new_host) {
+        e = cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dpos, token_pos_host, pos_bytes, cudaMemcpyHostToDevice, s);
+    }
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attend_host: upload");
+    st = lethe_decode_attend(ctx, c, layer_begin, layer_end, dq, k_new_host ? dk : nullptr, k_new_host ? dv : nullptr,
+                             k_new_host ? dpos : nullptr, scale, gamma, dout, lse_host ? dlse : nullptr, stream);
+    if (st != LETHE_OK) return st;
+    e = cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && lse_host) e = cudaMemcpyAsync(lse_host, dlse, lse_bytes, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attend_host: download");
+    return LETHE_OK;
+}
+
+lethe_status lethe_estimate_sparsity(lethe_ctx* ctx, const lethe_cache* c, float* sparsity, void* stream) {
+    lethe_status st = check_cache(ctx, c);
+    if (st != LETHE_OK) return st;
+    if (!sparsity) return fail(ctx, LETHE_ERR_INVALID_ARG, "sparsity is NULL");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, LETHE_ERR_CUDA, "cannot select the context's device");
+    cudaError_t e = launch_sparsity(view_of(c), sparsity, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "estimate_sparsity launch");
+    return LETHE_OK;
+}
+
+lethe_status lethe_alloc_budgets(lethe_ctx* ctx, int n_layers, int batch, const float* sparsity,
+                                 const int64_t* total_budget, int32_t k_min, int32_t* budgets, void* stream) {
+    if (!ctx) return LETHE_ERR_INVALID_ARG;
+    if (!sparsity || !total_budget || !budgets) return fail(ctx, LETHE_ERR_INVALID_ARG, "NULL argument");
+    if (n_layers < 1 || batch < 1 || k_min < 0) return fail(ctx, LETHE_ERR_INVALID_ARG, "bad sizes");
+    if (n_layers > 1024) return fail(ctx, LETHE_ERR_UNSUPPORTED, "more than 1024 layers");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, LETHE_ERR_CUDA, "cannot select the context's device");
+    cudaError_t e = launch_budgets(n_layers, batch, sparsity, (const long long*)total_budget, k_min, budgets,
+                                   ctx->status, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "alloc_budgets launch");
+    return LETHE_OK;
+}
+
+lethe_status lethe_rasr_prune(lethe_ctx* ctx, const lethe_cache* c, const int32_t* budgets, int32_t recent,
+                              int32_t sink, int32_t* keep_idx, int32_t max_k, void* stream) {
+    lethe_status st = check_cache(ctx, c);
+    if (st != LETHE_OK) return st;
+    if (!budgets) return fail(ctx, LETHE_ERR_INVALID_ARG, "budgets is NULL");
+    if (recent < 0 || sink < 0) return fail(ctx, LETHE_ERR_INVALID_ARG, "recent and sink must be >= 0");
+    if (keep_idx && max_k < 1) return fail(ctx, LETHE_ERR_INVALID_ARG, "max_k must be positive with keep_idx");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, LETHE_ERR_CUDA, "cannot select the context's device");
+    const CacheView v = view_of(c);
+    // keys / source list live in shared memory when an item fits; otherwise the list goes to global scratch
+    const size_t budget_smem = ctx->max_smem - 8 * 1024;
+    int smem_tokens = v.cap_tokens;
+    int32_t* list_scratch = nullptr;
+    if ((size_t)smem_tokens * 4 > budget_smem) {
+        smem_tokens = (int)(budget_smem / 4);
+        const size_t need = (size_t)v.L * v.B * v.Hkv * v.cap_tokens * sizeof(int32_t);
+        st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "prune scratch");
+        if (st != LETHE_OK) return st;
+        list_scratch = (int32_t*)ctx->scratch;
+    }
+    cudaError_t e = launch_rasr_prune(v, budgets, recent, sink, keep_idx, keep_idx ? max_k : 0, smem_tokens,
+                                      list_scratch, ctx->status, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "rasr_prune launch");
+    return LETHE_OK;
+}
+
+}  // extern "C"

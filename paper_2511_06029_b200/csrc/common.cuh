@@ -1,0 +1,236 @@
+// Shared device-side definitions of the Lethe kernels (sm_100a).
+#pragma once
+
+#include <cooperative_groups.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/lethe.h"
+
+namespace cg = cooperative_groups;
+
+namespace lethe {
+
+constexpr int kMaxLayers = 128;  // layers addressable by one decode call (scale table travels by value)
+constexpr int kMaxGroup = 8;     // query heads per KV head the attend kernels hold at once
+constexpr int kGroupTokens = 16; // tokens per streaming group (= one page in the paged layout)
+
+// Arguments of one lethe_decode_attend launch.
+struct AttendArgs {
+    const void* k;
+    const void* v;
+    float* rel;
+    int32_t* pos;
+    int32_t* len;
+    const int32_t* page_table;
+    const void* q;
+    const void* k_new;
+    const void* v_new;
+    const int32_t* token_pos;
+    void* out;
+    float* lse;
+    int32_t* status;  // device status word: {code, item}
+    long long n_pages;
+    int B, Hq, Hkv, G, GP;  // GP = G rounded up to even: row pitch of the logit buffer
+    int capacity, cap_tokens, page_tokens;
+    int layer_begin, n_items;  // items of this call: nl * B * Hkv
+    int splits;                // CTAs per item (cluster size)
+    int chunk_tokens;          // logit-buffer capacity of one CTA, in tokens
+    float gamma;
+    float scale_log2[kMaxLayers];  // scale[l] * log2(e), by absolute layer
+};
+
+// Cache state as the prune-round kernels see it.
+struct CacheView {
+    void* k;
+    void* v;
+    float* rel;
+    int32_t* pos;
+    int32_t* len;
+    const int32_t* page_table;
+    long long n_pages;
+    int L, B, Hkv, D, elt_bytes, capacity, cap_tokens, page_tokens, paged;
+};
+
+__device__ __forceinline__ void record_error(int32_t* status, int code, int item) {
+    if (atomicCAS(status, 0, code) == 0) status[1] = item;
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// exp2(a - b) that reads (-inf) - (-inf) as 0 rather than NaN
+__device__ __forceinline__ float exp2_diff(float a, float b) { return (a == -INFINITY) ? 0.f : fast_exp2(a - b); }
+
+template <typename T>
+__device__ __forceinline__ float to_float(T x);
+template <>
+__device__ __forceinline__ float to_float<float>(float x) {
+    return x;
+}
+template <>
+__device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 x) {
+    return __bfloat162float(x);
+}
+template <typename T>
+__device__ __forceinline__ T from_float(float x);
+template <>
+__device__ __forceinline__ float from_float<float>(float x) {
+    return x;
+}
+template <>
+__device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(float x) {
+    return __float2bfloat16_rn(x);
+}
+
+// Decoded position of a CTA inside the launch.
+struct ItemCoord {
+    int item_call;  // item index within the call
+    int item;       // absolute flat item (l * B + b) * Hkv + hkv
+    int li, l, b, hkv;
+    int rank;  // CTA rank among the item's splits
+};
+
+__device__ __forceinline__ ItemCoord decode_item(const AttendArgs& a) {
+    ItemCoord c;
+    c.item_call = blockIdx.x / a.splits;
+    c.rank = blockIdx.x % a.splits;
+    c.hkv = c.item_call % a.Hkv;
+    c.b = (c.item_call / a.Hkv) % a.B;
+    c.li = c.item_call / (a.Hkv * a.B);
+    c.l = a.layer_begin + c.li;
+    c.item = (c.l * a.B + c.b) * a.Hkv + c.hkv;
+    return c;
+}
+
+// Token range of this CTA: whole 16-token groups [g_begin, g_end) of the item's ceil(n/16) groups.
+__device__ __forceinline__ void split_range(int n, int splits, int rank, int& g_begin, int& g_end) {
+    const int ng = (n + kGroupTokens - 1) / kGroupTokens;
+    const int per = (ng + splits - 1) / splits;
+    g_begin = min(ng, rank * per);
+    g_end = min(ng, g_begin + per);
+}
+
+// Byte address of row `slot` of an item in K or V.  PAGED returns nullptr for a page id outside the pool.
+template <bool PAGED>
+__device__ __forceinline__ const char* row_ptr(const AttendArgs& a, const void* base, int item, int slot, int row_bytes,
+                                               bool* bad_page) {
+    if (!PAGED) return (const char*)base + ((size_t)item * a.capacity + slot) * row_bytes;
+    const int page = a.page_table[(size_t)item * a.capacity + slot / a.page_tokens];
+    if (page < 0 || page >= a.n_pages) {
+        *bad_page = true;
+        return nullptr;
+    }
+    return (const char*)base + ((size_t)page * a.page_tokens + slot % a.page_tokens) * row_bytes;
+}
+
+// Shared-memory bookkeeping used by the common epilogue.
+struct EpilogueSmem {
+    float2 wstat[16][kMaxGroup];  // per warp, per head: (running max in log2 units, partial sum)
+    float wscale[16][kMaxGroup];  // per warp rescale factor to the CTA max
+    float2 cta_stat[kMaxGroup];   // per head: (CTA max, CTA sum)
+    float2 fin[kMaxGroup];        // per head: (global max, 1 / global sum)
+    float rscale[16][kMaxGroup];  // per cluster rank: exp2(m_r - m) / l
+    int flags[4];
+};
+
+/*
+ * Common tail of both attend kernels.  On entry every warp has written, for the tokens it streamed,
+ *   es.wstat[w][h]   = (m, l): running max (log2 units) and sum of exp2(s - m) of head h
+ *   wo[w*wo_stride + h*D + d] = sum_j exp2(s_hj - m) V_j[d]
+ *   lg[(j - t0)*GP + h] = s_hj in log2 units for every token j of the CTA's range [t0, t1)
+ * The function merges warps, then the CTAs of the cluster (distributed shared memory), writes out / lse, and
+ * applies Eq. 5 to rel[t0..t1) with the exact global normaliser.
+ */
+template <typename T, int D, int NW>
+__device__ void combine_and_finish(const AttendArgs& a, const ItemCoord& ic, EpilogueSmem& es, float* wo, int wo_stride,
+                                   float* cta_o /*[kMaxGroup][D]*/, const float* lg, int t0, int t1, int append_slot,
+                                   int n) {
+    const int tid = threadIdx.x;
+    const int G = a.G;
+    constexpr int NT = NW * 32;
+    __syncthreads();
+    if (tid < kMaxGroup) {
+        const int h = tid;
+        float m = -INFINITY;
+        for (int w = 0; w < NW; ++w) m = fmaxf(m, es.wstat[w][h].x);
+        float l = 0.f;
+        for (int w = 0; w < NW; ++w) {
+            const float sc = exp2_diff(es.wstat[w][h].x, m);
+            es.wscale[w][h] = sc;
+            l += es.wstat[w][h].y * sc;
+        }
+        es.cta_stat[h] = make_float2(m, l);
+    }
+    __syncthreads();
+    for (int idx = tid; idx < G * D; idx += NT) {
+        const int h = idx / D;
+        float acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) acc += wo[w * wo_stride + idx] * es.wscale[w][h];
+        cta_o[idx] = acc;
+    }
+
+    const int S = a.splits;
+    T* out = (T*)a.out + ((size_t)(ic.li * a.B + ic.b) * a.Hq + ic.hkv * G) * D;
+    float* lse = a.lse ? a.lse + (size_t)(ic.li * a.B + ic.b) * a.Hq + ic.hkv * G : nullptr;
+    if (S == 1) {
+        __syncthreads();
+        if (tid < kMaxGroup) {
+            const float2 st = es.cta_stat[tid];
+            es.fin[tid] = make_float2(st.x, st.y > 0.f ? 1.f / st.y : 0.f);
+            if (lse && tid < G) lse[tid] = st.y > 0.f ? (st.x + log2f(st.y)) * 0.6931471805599453f : -INFINITY;
+        }
+        __syncthreads();
+        for (int idx = tid; idx < G * D; idx += NT) out[idx] = from_float<T>(cta_o[idx] * es.fin[idx / D].y);
+    } else {
+        cg::cluster_group cluster = cg::this_cluster();
+        cluster.sync();  // every CTA's cta_o / cta_stat is complete and visible cluster-wide
+        if (tid < kMaxGroup) {
+            const int h = tid;
+            float m = -INFINITY;
+            for (int r = 0; r < S; ++r) m = fmaxf(m, cluster.map_shared_rank(&es.cta_stat[0], r)[h].x);
+            float l = 0.f;
+            for (int r = 0; r < S; ++r) {
+                const float2 st = cluster.map_shared_rank(&es.cta_stat[0], r)[h];
+                l += st.y * exp2_diff(st.x, m);
+            }
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+            for (int r = 0; r < S; ++r)
+                es.rscale[r][h] = exp2_diff(cluster.map_shared_rank(&es.cta_stat[0], r)[h].x, m) * inv;
+            es.fin[h] = make_float2(m, inv);
+            if (lse && ic.rank == 0 && h < G) lse[h] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+        }
+        __syncthreads();
+        // each rank finishes an equal slice of the G*D outputs
+        const int total = G * D;
+        const int per = (total + S - 1) / S;
+        const int lo = ic.rank * per, hi = min(total, lo + per);
+        for (int idx = lo + tid; idx < hi; idx += NT) {
+            const int h = idx / D;
+            float acc = 0.f;
+            for (int r = 0; r < S; ++r) acc += cluster.map_shared_rank(cta_o, r)[idx] * es.rscale[r][h];
+            out[idx] = from_float<T>(acc);
+        }
+    }
+
+    // Eq. 5: rel[j] = gamma * rel[j] + sum over the group's heads of p_hj, with the global (m, 1/l).
+    float* rel = a.rel + (size_t)ic.item * a.cap_tokens;
+    const int GP = a.GP;
+    const int hi_tok = min(t1, n);
+    for (int j = t0 + tid; j < hi_tok; j += NT) {
+        const float* row = lg + (size_t)(j - t0) * GP;
+        float mass = 0.f;
+        for (int h = 0; h < G; ++h) mass += fast_exp2(row[h] - es.fin[h].x) * es.fin[h].y;
+        const float old = (j == append_slot) ? 0.f : rel[j];
+        rel[j] = fmaf(a.gamma, old, mass);
+    }
+    if (S > 1) cg::this_cluster().sync();  // peers may still be reading this CTA's shared memory
+    if (append_slot >= 0 && ic.rank == 0 && tid == 0) a.len[ic.item] = n;
+}
+
+}  // namespace lethe

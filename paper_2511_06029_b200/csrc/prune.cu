@@ -1,0 +1,347 @@
+// Prune-round kernels: Hoyer sparsity per (layer, sequence), integer budget allocation, and the RASR
+// retention step (protected top-k by radix select on the fp32 bit pattern + in-place stable compaction).
+#include "common.cuh"
+
+namespace lethe {
+
+
+// ------------------------------------------------------------------------------------------------ Eq. 1
+// One CTA per (layer, sequence); loops over the KV heads; deterministic tree reductions in double.
+__global__ void __launch_bounds__(256) sparsity_kernel(CacheView c, float* __restrict__ sparsity) {
+    __shared__ double s1[256], s2[256];
+    const int lb = blockIdx.x;
+    const int tid = threadIdx.x;
+    double acc = 0.0;
+    for (int h = 0; h < c.Hkv; ++h) {
+        const size_t item = (size_t)lb * c.Hkv + h;
+        const int n = c.len[item];
+        const float* r = c.rel + item * c.cap_tokens;
+        double a1 = 0.0, a2 = 0.0;
+        for (int j = tid; j < n; j += 256) {
+            const double x = (double)r[j];
+            a1 += fabs(x);
+            a2 += x * x;
+        }
+        s1[tid] = a1;
+        s2[tid] = a2;
+        __syncthreads();
+        for (int off = 128; off > 0; off >>= 1) {
+            if (tid < off) {
+                s1[tid] += s1[tid + off];
+                s2[tid] += s2[tid + off];
+            }
+            __syncthreads();
+        }
+        if (tid == 0) {
+            double s = 0.0;
+            if (n > 1 && s2[0] > 0.0) {
+                const double rn = sqrt((double)n);
+                s = (rn - s1[0] / sqrt(s2[0])) / (rn - 1.0);
+                s = fmin(fmax(s, 0.0), 1.0);
+            }
+            acc += s;
+        }
+        __syncthreads();
+    }
+    if (tid == 0) sparsity[lb] = (float)(acc / (double)c.Hkv);
+}
+
+cudaError_t launch_sparsity(const CacheView& c, float* sparsity, cudaStream_t stream) {
+    sparsity_kernel<<<c.L * c.B, 256, 0, stream>>>(c, sparsity);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------- budget allocation
+// One CTA per sequence.  w_l from one fp32 subtraction and an exact power-of-two scaling; everything after
+// is 64-bit integer arithmetic (largest-remainder apportionment, ties to the lower layer).
+constexpr int kBudgetMaxLayers = 1024;
+
+__global__ void __launch_bounds__(128) budgets_kernel(int L, int B, const float* __restrict__ sparsity,
+                                                      const long long* __restrict__ total, int k_min,
+                                                      int32_t* __restrict__ budgets, int32_t* status) {
+    __shared__ long long w[kBudgetMaxLayers], rem[kBudgetMaxLayers];
+    __shared__ long long red[128];
+    __shared__ long long W_sh, R_sh;
+    const int b = blockIdx.x, tid = threadIdx.x;
+    long long part = 0;
+    for (int l = tid; l < L; l += 128) {
+        float s = sparsity[(size_t)l * B + b];
+        if (!(s >= 0.0f)) s = 0.0f;
+        if (s > 1.0f) s = 1.0f;
+        const float d = __fsub_rn(1.0f, s);
+        long long wl = (long long)rintf(__fmul_rn(d, 1048576.0f));
+        if (wl < 1) wl = 1;
+        w[l] = wl;
+        part += wl;
+    }
+    red[tid] = part;
+    __syncthreads();
+    for (int off = 64; off > 0; off >>= 1) {
+        if (tid < off) red[tid] += red[tid + off];
+        __syncthreads();
+    }
+    if (tid == 0) W_sh = red[0];
+    __syncthreads();
+    const long long W = W_sh;
+    long long F = total[b] - (long long)L * k_min;
+    if (F < 0) {
+        for (int l = tid; l < L; l += 128) budgets[(size_t)l * B + b] = k_min;
+        if (tid == 0) record_error(status, LETHE_ERR_BUDGET, b);
+        return;
+    }
+    part = 0;
+    for (int l = tid; l < L; l += 128) {
+        const long long prod = w[l] * F;
+        const long long base = prod / W;
+        rem[l] = prod - base * W;
+        w[l] = base;  // reuse: floor share
+        part += base;
+    }
+    __syncthreads();
+    red[tid] = part;
+    __syncthreads();
+    for (int off = 64; off > 0; off >>= 1) {
+        if (tid < off) red[tid] += red[tid + off];
+        __syncthreads();
+    }
+    if (tid == 0) R_sh = F - red[0];
+    __syncthreads();
+    const long long R = R_sh;  // 0 <= R < L
+    for (int l = tid; l < L; l += 128) {
+        // rank of layer l by (remainder desc, layer asc)
+        long long rank = 0;
+        const long long rl = rem[l];
+        for (int o = 0; o < L; ++o) rank += (rem[o] > rl) || (rem[o] == rl && o < l);
+        budgets[(size_t)l * B + b] = (int32_t)((long long)k_min + w[l] + (rank < R ? 1 : 0));
+    }
+}
+
+cudaError_t launch_budgets(int L, int B, const float* sparsity, const long long* total, int k_min, int32_t* budgets,
+                           int32_t* status, cudaStream_t stream) {
+    budgets_kernel<<<B, 128, 0, stream>>>(L, B, sparsity, total, k_min, budgets, status);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------- RASR retention + compaction
+// Order-preserving map from fp32 to uint32 (zero of either sign maps to the same key).
+__device__ __forceinline__ uint32_t score_key(float x) {
+    uint32_t u = __float_as_uint(x);
+    if ((u << 1) == 0u) u = 0u;
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+constexpr int kPruneThreads = 512;
+
+__device__ __forceinline__ char* prune_row_ptr(const CacheView& c, void* base, size_t item, int slot, int row_bytes,
+                                               bool* bad) {
+    if (!c.paged) return (char*)base + (item * c.capacity + slot) * row_bytes;
+    const int page = c.page_table[item * c.capacity + slot / c.page_tokens];
+    if (page < 0 || page >= c.n_pages) {
+        *bad = true;
+        return nullptr;
+    }
+    return (char*)base + ((size_t)page * c.page_tokens + slot % c.page_tokens) * row_bytes;
+}
+
+// Block-wide exclusive scan of one counter per thread (kPruneThreads threads): returns this thread's
+// exclusive prefix and the block total.  Ends with a barrier, so warp_buf may be reused at once.
+__device__ __forceinline__ void block_scan(int v, int* warp_buf, int& ex, int& tot) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, inc, off);
+        if (lane >= off) inc += t;
+    }
+    if (lane == 31) warp_buf[warp] = inc;
+    __syncthreads();
+    int base = 0;
+    tot = 0;
+#pragma unroll
+    for (int w = 0; w < kPruneThreads / 32; ++w) {
+        const int x = warp_buf[w];
+        if (w < warp) base += x;
+        tot += x;
+    }
+    ex = base + inc - v;
+    __syncthreads();
+}
+
+/*
+ * One CTA per item.
+ *  1. keys: score_key(rel[j]) into shared memory (or re-read from global when the item is too long).
+ *  2. 4-pass, 8-bit radix select of the `take`-th largest candidate key -> threshold T, count above it.
+ *  3. ascending sweep: keep = protected | key > T | (key == T and among the first need_eq such slots);
+ *     block scans turn the keep flags into destination slots; the source slot of every destination is
+ *     written to a list (shared memory, in place over the keys; global scratch for items longer than
+ *     smem_tokens, whose keys are then re-read from rel).
+ *  4. rows move in waves of ascending destinations: load wave -> barrier -> store wave.  Because the
+ *     destination of a survivor never exceeds its source and waves ascend, no unread source is overwritten.
+ */
+__global__ void __launch_bounds__(kPruneThreads) rasr_prune_kernel(CacheView c, const int32_t* __restrict__ budgets,
+                                                                   int recent, int sink, int32_t* keep_idx, int max_k,
+                                                                   int smem_tokens, int32_t* list_scratch,
+                                                                   int32_t* status) {
+    extern __shared__ __align__(16) uint32_t dyn[];  // keys, later the source list  [smem_tokens]
+    __shared__ int hist[256];
+    __shared__ int warp_buf[kPruneThreads / 32];
+    __shared__ uint32_t sel_prefix;
+    __shared__ int sel_remaining;
+
+    const size_t item = blockIdx.x;
+    const int tid = threadIdx.x;
+    const int l = (int)(item / ((size_t)c.B * c.Hkv));
+    const int b = (int)((item / c.Hkv) % c.B);
+    const int n = c.len[item];
+    long long k = budgets[(size_t)l * c.B + b];
+    if (k < 0) k = 0;
+    int32_t* kout = keep_idx ? keep_idx + item * max_k : nullptr;
+    if (k >= n) {  // identity
+        if (kout)
+            for (int i = tid; i < max_k; i += kPruneThreads) kout[i] = (i < n) ? i : -1;
+        return;
+    }
+    const int n_sink = min(sink, n), n_recent = min(recent, n);
+    const int cand_lo = n_sink;
+    const int cand_hi = max(n - n_recent, cand_lo);
+    const int n_prot = n - (cand_hi - cand_lo);
+    if (n_prot > k) {
+        k = n_prot;
+        if (tid == 0) record_error(status, LETHE_ERR_BUDGET, (int)item);
+    }
+    const int keep_n = (int)k;
+    const int take = keep_n - n_prot;
+    float* rel = c.rel + item * c.cap_tokens;
+    int32_t* pos = c.pos + item * c.cap_tokens;
+    const bool in_smem = n <= smem_tokens;
+
+    if (in_smem)
+        for (int j = tid; j < n; j += kPruneThreads) dyn[j] = score_key(rel[j]);
+    __syncthreads();
+    auto key_at = [&](int j) -> uint32_t { return in_smem ? dyn[j] : score_key(rel[j]); };
+
+    // ---- radix select: T = take-th largest candidate key (take >= 1), n_gt = candidates above T
+    uint32_t T = 0xffffffffu;
+    int need_eq = 0;
+    if (take > 0) {
+        if (tid == 0) {
+            sel_prefix = 0u;
+            sel_remaining = take;
+        }
+        for (int pass = 0; pass < 4; ++pass) {
+            const int shift = 24 - 8 * pass;
+            const uint32_t mask_hi = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+            if (tid < 256) hist[tid] = 0;
+            __syncthreads();
+            const uint32_t prefix = sel_prefix;
+            for (int j = cand_lo + tid; j < cand_hi; j += kPruneThreads) {
+                const uint32_t key = key_at(j);
+                if ((key & mask_hi) == prefix) atomicAdd(&hist[(key >> shift) & 0xffu], 1);
+            }
+            __syncthreads();
+            if (tid == 0) {
+                int remaining = sel_remaining;
+                int d = 255;
+                for (; d > 0; --d) {
+                    if (hist[d] >= remaining) break;
+                    remaining -= hist[d];
+                }
+                sel_prefix = prefix | ((uint32_t)d << shift);
+                sel_remaining = remaining;
+            }
+            __syncthreads();
+        }
+        T = sel_prefix;
+        need_eq = sel_remaining;  // how many slots equal to T are kept (the oldest ones)
+    }
+
+    // ---- ascending sweep: destinations by prefix sums; source list written over consumed keys
+    int32_t* src_list = in_smem ? reinterpret_cast<int32_t*>(dyn) : list_scratch + item * c.cap_tokens;
+    int run_keep = 0, run_eq = 0;
+    for (int base = 0; base < n; base += kPruneThreads) {
+        const int j = base + tid;
+        int is_keep = 0, is_eq = 0;
+        uint32_t key = 0;
+        if (j < n) {
+            if (j < cand_lo || j >= cand_hi) is_keep = 1;
+            else if (take > 0) {
+                key = key_at(j);
+                if (key > T) is_keep = 1;
+                else if (key == T) is_eq = 1;
+            }
+        }
+        int ex_keep, ex_eq, tot_keep, tot_eq;
+        // first the rank among slots equal to the threshold (slot order), then the keep scan that depends on it
+        block_scan(is_eq, warp_buf, ex_eq, tot_eq);
+        if (is_eq && run_eq + ex_eq < need_eq) is_keep = 1;
+        block_scan(is_keep, warp_buf, ex_keep, tot_keep);
+        if (is_keep) {
+            const int dst = run_keep + ex_keep;
+            src_list[dst] = j;  // dst <= j, and every key of this chunk was read before the scans' barriers
+            if (kout && dst < max_k) kout[dst] = j;
+        }
+        run_keep += tot_keep;
+        run_eq += tot_eq;
+    }
+    __syncthreads();
+    if (kout)
+        for (int i = keep_n + tid; i < max_k; i += kPruneThreads) kout[i] = -1;
+
+    // ---- move rows in ascending waves
+    const int row_bytes = c.D * c.elt_bytes;
+    const int lanes_per_row = row_bytes / 16;            // 16-byte pieces per row (8, 16 or 32)
+    const int rows_per_wave = kPruneThreads / lanes_per_row;
+    const int piece = tid % lanes_per_row, rslot = tid / lanes_per_row;
+    bool bad = false;
+    // skip the unmoved prefix: destinations whose source is themselves
+    for (int w0 = 0; w0 < keep_n; w0 += rows_per_wave) {
+        const int dst = w0 + rslot;
+        int src = -1;
+        if (dst < keep_n) src = src_list[dst];
+        uint4 kv = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
+        float rv = 0.f;
+        int pv = 0;
+        const bool moves = src >= 0 && src != dst;
+        if (moves) {
+            const char* ks = prune_row_ptr(c, c.k, item, src, row_bytes, &bad);
+            const char* vs = prune_row_ptr(c, c.v, item, src, row_bytes, &bad);
+            if (ks && vs) {
+                kv = *reinterpret_cast<const uint4*>(ks + piece * 16);
+                vv = *reinterpret_cast<const uint4*>(vs + piece * 16);
+            }
+            if (piece == 0) {
+                rv = rel[src];
+                pv = pos[src];
+            }
+        }
+        __syncthreads();
+        if (moves) {
+            char* kd = prune_row_ptr(c, c.k, item, dst, row_bytes, &bad);
+            char* vd = prune_row_ptr(c, c.v, item, dst, row_bytes, &bad);
+            if (kd && vd) {
+                *reinterpret_cast<uint4*>(kd + piece * 16) = kv;
+                *reinterpret_cast<uint4*>(vd + piece * 16) = vv;
+            }
+            if (piece == 0) {
+                rel[dst] = rv;
+                pos[dst] = pv;
+            }
+        }
+        // no barrier needed here: the next wave's sources lie above every destination written so far
+    }
+    if (bad && tid == 0) record_error(status, LETHE_ERR_PAGE, (int)item);
+    if (tid == 0) c.len[item] = keep_n;
+}
+
+cudaError_t launch_rasr_prune(const CacheView& c, const int32_t* budgets, int recent, int sink, int32_t* keep_idx,
+                              int max_k, int smem_tokens, int32_t* list_scratch, int32_t* status,
+                              cudaStream_t stream) {
+    const size_t smem = (size_t)smem_tokens * 4;
+    cudaError_t e = cudaFuncSetAttribute(rasr_prune_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    rasr_prune_kernel<<<c.L * c.B * c.Hkv, kPruneThreads, smem, stream>>>(c, budgets, recent, sink, keep_idx, max_k,
+                                                                         smem_tokens, list_scratch, status);
+    return cudaGetLastError();
+}
+
+}  // namespace lethe

@@ -1,0 +1,270 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element, on the same
+seeded inputs.  Tolerances: integer / index / moved-row results bit-exact; attention output max-abs 2e-2 for
+bf16 caches and 1e-4 for fp32; relevance and sparsity |d| <= 1e-3 |ref| + 1e-6.
+"""
+import pytest
+import torch
+
+import oracle
+from helpers import (assert_state_matches, cache_from_state, gpu_context, oracle_prune_round, random_cache, sync_state,
+                     to_device)
+from paper_2511_06029_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+OUT_TOL = {torch.float32: 1e-4, torch.bfloat16: 2e-2}
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = gpu_context()
+    yield c
+    c.close()
+
+
+def _lens(L, B, Hkv, cap, seed, special=()):
+    g = torch.Generator().manual_seed(seed)
+    ln = torch.randint(1, cap, (L, B, Hkv), generator=g)
+    flat = ln.view(-1)
+    for i, val in enumerate(special):
+        flat[i % flat.numel()] = val
+    return ln
+
+
+def _step(ctx, oc, gc, q, kn, vn, tp, scale, gamma, l0, l1, want_lse=True):
+    """Run one decode call on both sides and compare everything it produces."""
+    dev = gc.device
+    st, o_out, o_lse, _ = oracle.decode_attend(oc, l0, l1, q, kn, vn, tp, scale, gamma, want_lse=True)
+    assert st == oracle.OK
+    out = torch.full_like(q, float("nan"), device=dev)
+    lse = torch.full((l1 - l0, oc.batch, oc.n_q_heads), float("nan"), device=dev) if want_lse else None
+    ctx.decode_attend(gc, l0, l1, q.to(dev), None if kn is None else kn.to(dev), None if vn is None else vn.to(dev),
+                      None if tp is None else tp.to(dev), scale.tolist(), gamma, out, lse)
+    st, item = ctx.poll_status()
+    assert st == 0, (st, item)
+    tol = OUT_TOL[q.dtype]
+    err = (out.cpu().double() - o_out.double()).abs().max().item()
+    assert err <= tol, f"out max-abs error {err}"
+    if want_lse:
+        fin = torch.isfinite(o_lse)
+        assert torch.equal(torch.isfinite(lse.cpu()), fin)
+        assert torch.allclose(lse.cpu()[fin], o_lse[fin], rtol=1e-4, atol=1e-4)
+    assert_state_matches(gc, oc)
+    return out
+
+
+CASES = [
+    # dtype, D, Hq, Hkv, cap, variant, splits
+    (torch.float32, 64, 8, 2, 200, 1, 1),
+    (torch.float32, 64, 8, 2, 200, 1, 4),
+    (torch.float32, 128, 4, 4, 150, 1, 2),
+    (torch.bfloat16, 128, 32, 8, 300, 1, 1),
+    (torch.bfloat16, 64, 14, 2, 300, 1, 8),
+    (torch.bfloat16, 128, 32, 8, 300, 2, 1),
+    (torch.bfloat16, 128, 32, 8, 300, 2, 2),
+    (torch.bfloat16, 128, 28, 4, 300, 2, 4),
+    (torch.bfloat16, 128, 28, 4, 700, 3, 1),
+    (torch.bfloat16, 128, 8, 1, 700, 3, 8),
+    (torch.bfloat16, 128, 6, 2, 1000, 3, 16),
+    (torch.bfloat16, 64, 8, 2, 300, 2, 2),
+    (torch.bfloat16, 64, 10, 2, 500, 3, 4),
+    (torch.bfloat16, 128, 8, 8, 260, 0, 0),
+    (torch.float32, 128, 16, 2, 260, 0, 0),
+]
+
+
+@pytest.mark.parametrize("dtype,D,Hq,Hkv,cap,variant,splits", CASES)
+def test_decode_attend_parity(ctx, dtype, D, Hq, Hkv, cap, variant, splits):
+    """Ragged lengths spanning several 16-token groups and ragged tails; append and attend-only steps; a layer
+    sub-range; every kernel variant and cluster size."""
+    L, B = 3, 2
+    lens = _lens(L, B, Hkv, cap - 4, seed=cap + D, special=(1, 15, 16, 17, cap - 5, 33))
+    oc = random_cache(L, B, Hq, Hkv, D, cap, lens, dtype=dtype, seed=D + Hq, rel_init="rand")
+    gc = to_device(oc)
+    ctx.set_tuning(variant, splits)
+    try:
+        g = torch.Generator().manual_seed(99)
+        scale = torch.tensor([0.09, 0.2, 0.05], dtype=torch.float32) * (128 / D) ** 0.5
+        for step, (l0, l1, app) in enumerate([(0, 3, True), (1, 2, False), (0, 3, True), (2, 3, True)]):
+            nl = l1 - l0
+            q = torch.randn((nl, B, Hq, D), generator=g).to(dtype)
+            kn = torch.randn((nl, B, Hkv, D), generator=g).to(dtype) if app else None
+            vn = torch.randn((nl, B, Hkv, D), generator=g).to(dtype) if app else None
+            tp = torch.tensor([1000 + step, 2000 + step], dtype=torch.int32) if app else None
+            _step(ctx, oc, gc, q, kn, vn, tp, scale, 0.9, l0, l1)
+    finally:
+        ctx.set_tuning(0, 0)
+
+
+def test_empty_and_full_items(ctx):
+    """len == 0 without append gives zeros and -inf; a full item refuses the append, is left untouched and
+    reports LETHE_ERR_CAPACITY."""
+    from paper_2511_06029_b200 import binding
+    L, B, Hq, Hkv, D, cap = 1, 2, 8, 2, 128, 32
+    lens = torch.tensor([[[0, 5], [32, 31]]])
+    oc = random_cache(L, B, Hq, Hkv, D, cap, lens, dtype=torch.bfloat16, seed=3, rel_init="rand")
+    gc = to_device(oc)
+    g = torch.Generator().manual_seed(1)
+    q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+    scale = torch.tensor([0.1])
+    _step(ctx, oc, gc, q, None, None, None, scale, 0.9, 0, 1)           # empty item: out 0, lse -inf
+    before = gc.k.clone(), gc.rel.clone(), gc.len.clone()
+    kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16).cuda()
+    out = torch.full((L, B, Hq, D), 7.0, dtype=torch.bfloat16, device="cuda")
+    ctx.decode_attend(gc, 0, 1, q.cuda(), kn, kn, torch.tensor([9, 9], dtype=torch.int32).cuda(), [0.1], 0.9, out)
+    st, item = ctx.poll_status()
+    assert st == binding.ERR_CAPACITY and item == 2                    # (l0, b1, h0) is the full one
+    assert torch.equal(gc.len.cpu(), torch.tensor([[[1, 6], [32, 32]]], dtype=torch.int32))
+    assert torch.equal(gc.k[0, 1, 0], before[0][0, 1, 0]) and torch.equal(gc.rel[0, 1, 0], before[1][0, 1, 0])
+    assert torch.all(out[0, 1, :4] == 0)
+    assert ctx.poll_status()[0] == 0                                     # the status word was cleared
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+def test_paged_decode_and_prune_parity(ctx, variant):
+    """16-token pages behind a shuffled page table: decode steps and prune rounds, call by call."""
+    w = synth.shrink(synth.WORKLOADS["ragged"], n_layers=2, batch=3, prompt_len=200)
+    cap = 256
+    st_c = synth.initial_kv(w, 200, cap)
+    st_c["len"][0, 0, 0] = 33; st_c["len"][1, 1, 1] = 16; st_c["len"][1, 0, 0] = 1; st_c["len"][0, 2, 3] = 177
+    st_p = synth.to_paged(st_c, 16, seed=3, spare_pages=7)
+    oc = cache_from_state(w, st_p, cap)
+    gc = to_device(oc)
+    scale = synth.layer_scales(w)
+    T = torch.tensor([150 * 2, 90 * 2, 400 * 2], dtype=torch.int64)
+    ctx.set_tuning(variant, 2)
+    try:
+        for step in range(6):
+            x = synth.step_inputs(w, step)
+            _step(ctx, oc, gc, x["q"], x["k_new"], x["v_new"], x["token_pos"], scale, 0.95, 0, 2)
+            if step in (2, 5):
+                _prune_both(ctx, oc, gc, T, 12, 8, 4, cap)
+    finally:
+        ctx.set_tuning(0, 0)
+
+
+def _prune_both(ctx, oc, gc, T, k_min, recent, sink, max_k):
+    """One prune round on both sides from identical state; integer results must be bit-exact."""
+    dev = gc.device
+    sync_state(gc, oc)                                   # selection runs on the oracle's fp32 scores
+    S_g = torch.zeros((oc.n_layers, oc.batch), dtype=torch.float32, device=dev)
+    ctx.estimate_sparsity(gc, S_g)
+    st, S_o = oracle.estimate_sparsity(oc)
+    assert torch.allclose(S_g.cpu(), S_o, rtol=1e-3, atol=1e-6)
+    bud_g = torch.zeros((oc.n_layers, oc.batch), dtype=torch.int32, device=dev)
+    ctx.alloc_budgets(S_o.to(dev), T.to(dev), k_min, bud_g)          # budgets bit-exact given the oracle's S
+    st, bud_o = oracle.alloc_budgets(S_o, T, k_min)
+    assert st == oracle.OK and torch.equal(bud_g.cpu(), bud_o)
+    keep_g = torch.full((oc.n_layers, oc.batch, oc.n_kv_heads, max_k), -7, dtype=torch.int32, device=dev)
+    ctx.rasr_prune(gc, bud_g, recent, sink, keep_g)
+    st_o, keep_o = oracle.rasr_prune(oc, bud_o, recent, sink, max_k=max_k)
+    st_g, _ = ctx.poll_status()
+    assert st_g == (3 if st_o == oracle.ERR_BUDGET else 0)
+    assert torch.equal(keep_g.cpu(), keep_o)                           # retained index sets bit-exact
+    assert_state_matches(gc, oc, exact_rel=True)
+    return bud_o, keep_o
+
+
+@pytest.mark.parametrize("dtype,D", [(torch.float32, 64), (torch.bfloat16, 128), (torch.bfloat16, 64), (torch.float32, 128)])
+def test_prune_round_parity(ctx, dtype, D):
+    """Sparsity within tolerance; budgets, keep_idx, len and moved rows bit-exact, with ties, items that are not
+    pruned, items whose protected set exceeds the budget, and lengths around the block size."""
+    L, B, Hq, Hkv, cap = 4, 3, 8, 2, 1500
+    lens = _lens(L, B, Hkv, cap, seed=D, special=(1, 2, 511, 512, 513, 1024, 1499, 40, 7))
+    oc = random_cache(L, B, Hq, Hkv, D, cap, lens, dtype=dtype, seed=5, rel_init="rand")
+    oc.rel[oc.rel > 0.8] = 0.5                                         # many ties at the top
+    oc.rel[0, 0, 0] = 0.0                                              # an all-equal item
+    gc = to_device(oc)
+    T = torch.tensor([4 * 300, 4 * 40, 4 * 1400], dtype=torch.int64)
+    _prune_both(ctx, oc, gc, T, 36, 32, 4, cap)
+    # second round on the survivors (multi-round pruning), tighter
+    T2 = torch.tensor([4 * 100, 4 * 38, 4 * 600], dtype=torch.int64)
+    _prune_both(ctx, oc, gc, T2, 36, 32, 4, cap)
+
+
+def test_budget_edge_cases(ctx):
+    from paper_2511_06029_b200 import binding
+    dev = torch.device("cuda")
+    for case in [([0.0, 0.5, 0.5, 0.75], 103, 2), ([0.25, 0.25, 0.25], 17, 5), ([float("nan"), 1.0, 2.0, -1.0], 1000, 0)]:
+        S = torch.tensor(case[0], dtype=torch.float32)[:, None]
+        T = torch.tensor([case[1]], dtype=torch.int64)
+        out = torch.zeros((len(case[0]), 1), dtype=torch.int32, device=dev)
+        ctx.alloc_budgets(S.to(dev), T.to(dev), case[2], out)
+        st, ref = oracle.alloc_budgets(S, T, case[2])
+        assert st == oracle.OK and torch.equal(out.cpu(), ref) and int(out.sum()) == case[1]
+    g = torch.Generator().manual_seed(3)
+    S = torch.rand((64, 5), generator=g); T = torch.randint(64 * 70, 64 * 3000, (5,), generator=g, dtype=torch.int64)
+    out = torch.zeros((64, 5), dtype=torch.int32, device=dev)
+    ctx.alloc_budgets(S.to(dev), T.to(dev), 68, out)
+    assert torch.equal(out.cpu(), oracle.alloc_budgets(S, T, 68)[1])
+    # total below the floor: every layer gets k_min and the status word says so
+    ctx.alloc_budgets(S.to(dev), torch.full((5,), 10, dtype=torch.int64, device=dev), 68, out)
+    st, _ = ctx.poll_status()
+    assert st == binding.ERR_BUDGET and torch.all(out == 68)
+
+
+def test_invalid_arguments_touch_nothing(ctx):
+    from paper_2511_06029_b200 import binding
+    oc = random_cache(1, 1, 8, 2, 128, 32, 8, dtype=torch.bfloat16, seed=0)
+    gc = to_device(oc)
+    q = torch.zeros((1, 1, 8, 128), dtype=torch.bfloat16, device="cuda")
+    out = torch.full_like(q, 3.0)
+    for kwargs in [dict(gamma=0.0), dict(gamma=1.5), dict(l1=2), dict(scale=[float("nan")])]:
+        with pytest.raises(binding.LetheError) as e:
+            ctx.decode_attend(gc, 0, kwargs.get("l1", 1), q, None, None, None, kwargs.get("scale", [0.1]),
+                              kwargs.get("gamma", 0.9), out)
+        assert e.value.status == binding.ERR_INVALID_ARG
+    with pytest.raises(binding.LetheError):
+        ctx.decode_attend(gc, 0, 1, q, q, None, None, [0.1], 0.9, out)       # k_new without v_new
+    assert torch.all(out == 3.0) and torch.equal(gc.len.cpu(), oc.len)
+    assert ctx.poll_status()[0] == 0
+
+
+def test_tiny_workload_trajectory(ctx):
+    """The Tiny configuration end to end: every call compared from identical state (call-by-call), and a
+    free-running GPU trajectory whose retained sets are compared with the oracle's at the end."""
+    w = synth.WORKLOADS["tiny"]
+    cap = w.prompt_len + w.prune_interval
+    scale = synth.layer_scales(w)
+    T = torch.tensor([w.total_budget], dtype=torch.int64)
+    oc = cache_from_state(w, synth.initial_kv(w, w.prompt_len, cap), cap)
+    gc = to_device(oc)
+    free = to_device(oc)
+    dev = gc.device
+    for step in range(w.gen_steps):
+        x = synth.step_inputs(w, step)
+        _step(ctx, oc, gc, x["q"], x["k_new"], x["v_new"], x["token_pos"], scale, w.gamma, 0, 1)
+        out = torch.empty_like(x["q"], device=dev)
+        ctx.decode_attend(free, 0, 1, x["q"].to(dev), x["k_new"].to(dev), x["v_new"].to(dev), x["token_pos"].to(dev),
+                          scale.tolist(), w.gamma, out)
+        if (step + 1) % w.prune_interval == 0:
+            _prune_both(ctx, oc, gc, T, w.k_min, w.recent, w.sink, cap)
+            S = torch.zeros((1, 1), dtype=torch.float32, device=dev); bud = torch.zeros((1, 1), dtype=torch.int32, device=dev)
+            ctx.estimate_sparsity(free, S); ctx.alloc_budgets(S, T.to(dev), w.k_min, bud)
+            ctx.rasr_prune(free, bud, w.recent, w.sink)
+    assert ctx.poll_status()[0] == 0
+    assert torch.equal(free.len.cpu(), oc.len)
+    for h in range(w.n_kv_heads):
+        a = set(free.pos[0, 0, h, :int(oc.len[0, 0, h])].cpu().tolist()); b = set(oc.pos[0, 0, h, :int(oc.len[0, 0, h])].tolist())
+        jac = len(a & b) / len(a | b)
+        print(f"tiny free-running retained-set Jaccard, head {h}: {jac:.4f}")
+        assert jac > 0.95
+
+
+@pytest.mark.parametrize("name,batch,steps", [("llama8b", 2, 10), ("qwen7b", 2, 6)])
+def test_model_shaped_workloads_call_by_call(ctx, name, batch, steps):
+    """Model-shaped geometry (all layers, full head counts, bf16) on a sub-batch of sequences, warm-started at
+    the mean budget; decode steps with the default tuning plus two prune rounds."""
+    w = synth.shrink(synth.WORKLOADS[name], batch=batch, prune_interval=steps // 2)
+    n0 = 300
+    cap = n0 + steps + 16
+    oc = cache_from_state(w, synth.initial_kv(w, n0, cap), cap)
+    gc = to_device(oc)
+    scale = synth.layer_scales(w)
+    T = torch.full((batch,), w.n_layers * 200, dtype=torch.int64)
+    for step in range(steps):
+        x = synth.step_inputs(w, step)
+        _step(ctx, oc, gc, x["q"], x["k_new"], x["v_new"], x["token_pos"], scale, w.gamma, 0, w.n_layers, want_lse=False)
+        if (step + 1) % w.prune_interval == 0:
+            bud, _ = _prune_both(ctx, oc, gc, T, w.k_min, w.recent, w.sink, cap)
+            assert int(bud.sum()) == int(T.sum())
