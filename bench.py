@@ -1,0 +1,414 @@
+#!/usr/bin/env python
+"""Benchmark of the Lethe hot path on B200: decode-step attention over the pruned KV cache (with the fused
+relevance update) plus the prune round every `prune_interval` steps, on the Llama-8B-shaped workload.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" = one decode step of the whole model shape (all layers, one lethe_decode_attend call) and, when the
+step index hits the prune interval, one prune round (estimate_sparsity -> alloc_budgets -> rasr_prune).  The
+printed JSON line follows the driver's contract; `value` is KV token-heads attended per second with the cache
+and the step inputs resident in HBM, `e2e` is the same through lethe_decode_attend_host (per-step q / k_new /
+v_new from pinned host memory, out read back to the host, a stream synchronise every step).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2511_06029_b200 import synth  # noqa: E402
+
+METRIC = "kv_token_heads_attended_per_s"
+UNIT = "token-heads/s"
+BYTES_PER_TOKEN_HEAD = 520          # K row 256 B + V row 256 B + relevance read 4 B + write 4 B (D=128, bf16)
+FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes per token-head of the attend kernel from the ncu capture summarised under profiles/ (None until
+# a capture exists for the kernel in use).
+NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = None
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples of one GPU while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def make_state(w, device, capacity, n0, seed):
+    """Device-resident cache at n0 tokens per item, values drawn on the device (throughput-only tensors)."""
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    L, B, H, D = w.n_layers, w.batch, w.n_kv_heads, w.head_dim
+    k = torch.empty((L, B, H, capacity, D), dtype=w.dtype, device=device)
+    v = torch.empty((L, B, H, capacity, D), dtype=w.dtype, device=device)
+    flags = synth.anchor_flags(w, torch.arange(capacity, device=device), torch.arange(B))   # [L][B][cap]
+    for l in range(L):
+        kk = torch.randn((B, H, capacity, D), generator=g, device=device, dtype=torch.float32)
+        kk *= torch.where(flags[l], w.anchor_gain, 1.0).to(torch.float32)[:, None, :, None]
+        k[l] = kk.to(w.dtype)
+        v[l] = torch.randn((B, H, capacity, D), generator=g, device=device, dtype=torch.float32).to(w.dtype)
+    rel = torch.zeros((L, B, H, capacity), dtype=torch.float32, device=device)
+    pos = torch.arange(capacity, dtype=torch.int32, device=device).expand(L, B, H, capacity).contiguous()
+    ln = torch.full((L, B, H), n0, dtype=torch.int32, device=device)
+    return k, v, rel, pos, ln
+
+
+class Runner:
+    """The decode / prune loop around the C ABI (host logic of the harness: when to prune)."""
+
+    def __init__(self, w, device, rank, capacity, variant, splits, pool=8):
+        from paper_2511_06029_b200 import binding
+        self.w, self.dev, self.binding = w, device, binding
+        self.ctx = binding.Context(device.index)
+        self.ctx.set_tuning(variant, splits)
+        k, v, rel, pos, ln = make_state(w, device, capacity, w.mean_budget, 1234 + 77 * rank)
+        self.cache = binding.Cache(w.n_q_heads, k, v, rel, pos, ln)
+        self.scale = synth.layer_scales(w).tolist()
+        self.scale_c = self.ctx._scale(self.scale)
+        L, B = w.n_layers, w.batch
+        g = torch.Generator(device=device); g.manual_seed(4321 + rank)
+        self.pool = []
+        for i in range(pool):
+            q = torch.randn((L, B, w.n_q_heads, w.head_dim), generator=g, device=device).to(w.dtype)
+            kn = torch.randn((L, B, w.n_kv_heads, w.head_dim), generator=g, device=device).to(w.dtype)
+            vn = torch.randn((L, B, w.n_kv_heads, w.head_dim), generator=g, device=device).to(w.dtype)
+            self.pool.append((q, kn, vn))
+        self.host_pool = [tuple(t.cpu().pin_memory() for t in p) for p in self.pool[:4]]
+        self.out = torch.empty((L, B, w.n_q_heads, w.head_dim), dtype=w.dtype, device=device)
+        self.out_host = torch.empty((L, B, w.n_q_heads, w.head_dim), dtype=w.dtype).pin_memory()
+        self.token_pos = torch.zeros((B,), dtype=torch.int32, device=device)
+        self.token_pos_host = torch.zeros((B,), dtype=torch.int32).pin_memory()
+        self.S = torch.zeros((L, B), dtype=torch.float32, device=device)
+        self.budgets = torch.zeros((L, B), dtype=torch.int32, device=device)
+        self.T = torch.full((B,), w.total_budget, dtype=torch.int64, device=device)
+        self.step_no = 0
+        self.launches = 0
+
+    def decode(self, host=False):
+        w = self.w
+        i = self.step_no
+        if host:
+            q, kn, vn = self.host_pool[i % len(self.host_pool)]
+            self.ctx.decode_attend_host(self.cache, 0, w.n_layers, q, kn, vn, self.token_pos_host, self.scale, w.gamma,
+                                        self.out_host, None, scale_c=self.scale_c)
+        else:
+            q, kn, vn = self.pool[i % len(self.pool)]
+            self.ctx.decode_attend(self.cache, 0, w.n_layers, q, kn, vn, self.token_pos, self.scale, w.gamma, self.out,
+                                   None, scale_c=self.scale_c)
+        self.launches += 1
+        self.step_no += 1
+
+    def prune_due(self):
+        return self.step_no % self.w.prune_interval == 0
+
+    def prune(self):
+        w = self.w
+        self.ctx.estimate_sparsity(self.cache, self.S)
+        self.ctx.alloc_budgets(self.S, self.T, w.k_min, self.budgets)
+        self.ctx.rasr_prune(self.cache, self.budgets, w.recent, w.sink)
+        self.launches += 3
+
+    def check(self):
+        st, item = self.ctx.poll_status()
+        if st != 0:
+            raise RuntimeError(f"device-side status {st} at item {item}")
+
+
+def timed_loop(r: Runner, steps: int, host: bool):
+    """Run `steps` steps; returns (total_ms, attend_ms list, prune_ms list, token_heads list)."""
+    dev = r.dev
+    stream = torch.cuda.current_stream(dev)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * steps)]
+    prune_ev = []
+    len_snap = [(0, r.cache.len.clone())]
+    t_begin = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    t_begin.record(stream)
+    for s in range(steps):
+        ev[2 * s].record(stream)
+        r.decode(host=host)
+        ev[2 * s + 1].record(stream)
+        if host:
+            stream.synchronize()               # the caller reads out before producing the next token
+        if r.prune_due():
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            r.prune()
+            b.record(stream)
+            prune_ev.append((a, b))
+            snap = torch.empty_like(r.cache.len)
+            snap.copy_(r.cache.len, non_blocking=True)
+            len_snap.append((s + 1, snap))
+    t_end.record(stream)
+    torch.cuda.synchronize(dev)
+    total_ms = t_begin.elapsed_time(t_end)
+    attend_ms = [ev[2 * s].elapsed_time(ev[2 * s + 1]) for s in range(steps)]
+    prune_ms = [a.elapsed_time(b) for a, b in prune_ev]
+    # token-heads attended at step s = sum of len after that step's append
+    items = r.cache.len.numel()
+    th = []
+    snaps = [(s0, int(t.sum().item())) for s0, t in len_snap]
+    for s in range(steps):
+        base_step, base_sum = max((x for x in snaps if x[0] <= s), key=lambda x: x[0])
+        th.append(base_sum + items * (s - base_step + 1))
+    return total_ms, attend_ms, prune_ms, th
+
+
+def cpu_baseline(w, r: Runner | None, seconds=12.0, layers=4, seqs=4):
+    """The oracle, as it stands, on a bounded sample of the workload on the host cores."""
+    import oracle
+    threads = oracle.max_threads()
+    oracle.set_threads(threads)
+    ws = synth.shrink(w, n_layers=layers, batch=seqs)
+    cap = w.mean_budget + 256
+    st = synth.initial_kv(ws, w.mean_budget, cap)
+    oc = oracle.OracleCache(ws.n_layers, seqs, ws.n_q_heads, ws.n_kv_heads, ws.head_dim, cap, st["k"], st["v"],
+                            st["rel"], st["pos"], st["len"])
+    scale = synth.layer_scales(w)[:layers].contiguous()
+    th = 0
+    t0 = time.perf_counter()
+    steps = 0
+    while True:
+        x = synth.step_inputs(ws, steps)
+        t1 = time.perf_counter()
+        s, *_ = oracle.decode_attend(oc, 0, layers, x["q"], x["k_new"], x["v_new"], x["token_pos"], scale, w.gamma)
+        dt = time.perf_counter() - t1
+        assert s == oracle.OK
+        th += int(oc.len.sum())
+        steps += 1
+        if steps == 1:
+            first = dt
+        if time.perf_counter() - t0 > seconds or steps >= 2000:
+            break
+    attend_s = time.perf_counter() - t0
+    # one prune round on the sample, amortised like the GPU loop
+    t1 = time.perf_counter()
+    _, S = oracle.estimate_sparsity(oc)
+    _, bud = oracle.alloc_budgets(S, torch.full((seqs,), layers * w.mean_budget, dtype=torch.int64), w.k_min)
+    oracle.rasr_prune(oc, bud, w.recent, w.sink)
+    prune_s = time.perf_counter() - t1
+    per_step = attend_s / steps + prune_s / w.prune_interval
+    return {"value": th / steps / per_step, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"{layers} layers x {seqs} sequences x {w.n_kv_heads} KV heads at ~{w.mean_budget} tokens, "
+                      f"{steps} decode steps in {attend_s:.1f} s plus one prune round ({prune_s * 1e3:.0f} ms) "
+                      f"amortised over {w.prune_interval} steps",
+            "ms_per_sample_step": per_step * 1e3, "token_heads_per_sample_step": th / steps}
+
+
+def run_reference(args, w):
+    """--impl reference: the oracle on the host cores, same metric / config keys."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    base = cpu_baseline(w, None, seconds=max(5.0, min(60.0, 0.5 * (args.steps + args.warmup))))
+    line = {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": base["ms_per_sample_step"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(w, args, extra={"note": "oracle timed on a bounded sample per step"}),
+            "cpu_baseline": base,
+            "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def workload_config(w, args, extra=None):
+    c = {"workload": f"{w.name}: L{w.n_layers} B{w.batch} Hq{w.n_q_heads}/Hkv{w.n_kv_heads} D{w.head_dim} bf16, "
+                     f"mean budget {w.mean_budget}/layer, recent {w.recent}, sink {w.sink}, prune every "
+                     f"{w.prune_interval} steps, gamma {w.gamma}",
+         "global_batch": w.batch * args.gpus, "l2": "inputs larger than L2 (>=1.1 GB of K/V streamed per step)",
+         "parallelism": f"dp{args.gpus} (sequences sharded, no data-path collective)"}
+    if extra:
+        c.update(extra)
+    return c
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama8b")
+    ap.add_argument("--variant", type=int, default=0)
+    ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--capacity", type=int, default=0)
+    ap.add_argument("--prep-rounds", type=int, default=6,
+                    help="untimed prune intervals run before warm-up so that lengths reach their budgets")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    w = synth.WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    from paper_2511_06029_b200 import build
+    if rank == 0 or world == 1:
+        build.build()
+    if dist is not None:
+        dist.barrier()
+
+    capacity = args.capacity or (2 * w.mean_budget)
+    r = Runner(w, dev, rank, capacity, args.variant, args.splits)
+    # state preparation (untimed): a few full prune intervals so that relevance, sparsity-driven budgets and
+    # lengths are those of a steady-state trajectory (dense layers need several rounds to grow to their budget)
+    for _ in range(max(1, args.prep_rounds)):
+        for _ in range(w.prune_interval):
+            r.decode()
+        r.prune()
+    r.check()
+    max_budget = int(r.budgets.max().item())
+    if max_budget + w.prune_interval > capacity:
+        raise SystemExit(f"capacity {capacity} too small for budget {max_budget} + interval {w.prune_interval}")
+    for _ in range(max(args.warmup, 3)):
+        r.decode()
+        if r.prune_due():
+            r.prune()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    r.launches = 0
+    total_ms, attend_ms, prune_ms, th = timed_loop(r, args.steps, host=False)
+    launches = r.launches
+    barrier()
+    r.check()
+    e2e = None
+    if not args.no_e2e:
+        barrier()
+        e_total_ms, _, _, e_th = timed_loop(r, args.steps, host=True)
+        barrier()
+        r.check()
+    clocks = sampler.stop() if sampler else None
+
+    units = float(sum(th))
+    t_ms = total_ms
+    if dist is not None:
+        t = torch.tensor([total_ms, e_total_ms if not args.no_e2e else 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        u = torch.tensor([units, float(sum(e_th)) if not args.no_e2e else 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(u, op=dist.ReduceOp.SUM)
+        t_ms, units = float(t[0]), float(u[0])
+        if not args.no_e2e:
+            e_total_ms, e_units = float(t[1]), float(u[1])
+    elif not args.no_e2e:
+        e_units = float(sum(e_th))
+
+    if rank == 0:
+        peak, which = measured_peak()
+        th_per_launch = sum(th) / len(th)
+        avg_attend_ms = sum(attend_ms) / len(attend_ms)
+        achieved = th_per_launch * BYTES_PER_TOKEN_HEAD / (avg_attend_ms * 1e-3) / 1e9
+        wq = w
+        h2d = (wq.n_layers * wq.batch * (wq.n_q_heads + 2 * wq.n_kv_heads) * wq.head_dim * 2 + wq.batch * 4)
+        d2h = wq.n_layers * wq.batch * wq.n_q_heads * wq.head_dim * 2
+        line = {
+            "metric": METRIC, "value": units / (t_ms * 1e-3), "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": t_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": workload_config(w, args, extra={
+                "capacity": capacity, "variant": args.variant, "splits": args.splits,
+                "launch_mode": "all layers in one lethe_decode_attend call per step",
+                "token_heads_per_step": th_per_launch,
+                "prune_rounds_timed": len(prune_ms),
+                "prune_round_ms": (sum(prune_ms) / len(prune_ms)) if prune_ms else None,
+                "attend_ms_per_step": avg_attend_ms,
+                "attend_ms_median": statistics.median(attend_ms)}),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_source": f"of {which}", "frac_of_8TBs_nominal": achieved / 8000.0,
+                         "kernel": "attend (dominant kernel; one launch per step)",
+                         "traffic": (NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD * th_per_launch
+                                     if NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD else None)},
+            "gpu_launches": launches, "clocks": clocks,
+        }
+        if not args.no_e2e:
+            line["e2e"] = {"value": e_units / (e_total_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                           "d2h_bytes_per_step": d2h, "ms_per_step": e_total_ms / args.steps}
+        if not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(w, r)
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

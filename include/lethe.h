@@ -94,9 +94,10 @@ const char *lethe_last_error(const lethe_ctx *ctx);
  * {status, flat item index l*B*Hkv + b*Hkv + h of the first offender}. */
 lethe_status lethe_poll_status(lethe_ctx *ctx, void *stream, int32_t *info);
 
-/* Tuning knobs (HOST values).  variant: 0 = automatic, 1 = CUDA-core kernel, 2 = tensor-core
- * (mma) kernel (bf16 only).  splits: 0 = automatic, else CTAs per item (1, 2, 4, 8 or 16; they
- * form one thread-block cluster).  Returns LETHE_ERR_INVALID_ARG for other values. */
+/* Tuning knobs (HOST values).  variant: 0 = automatic, 1 = CUDA-core kernel, 2..7 = tensor-core (mma)
+ * kernel (bf16 only) with (warps per CTA, pipeline stages per warp) = (4,3) (8,3) (4,2) (8,2) (4,4) (2,4).
+ * splits: 0 = automatic, else CTAs per item (1, 2, 4, 8 or 16; they form one thread-block cluster).
+ * Returns LETHE_ERR_INVALID_ARG for other values. */
 lethe_status lethe_set_tuning(lethe_ctx *ctx, int variant, int splits);
 
 /*

@@ -13,7 +13,7 @@ from typing import Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "liblethe.so")
+LIB_PATH = os.environ.get("LETHE_LIB", os.path.join(_HERE, "liblethe.so"))   # LETHE_LIB: an alternative build
 
 OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_BUDGET, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED, ERR_PAGE = range(8)
 F32, BF16 = 0, 1

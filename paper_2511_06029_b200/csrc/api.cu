@@ -22,6 +22,36 @@ cudaError_t launch_rasr_prune(const CacheView& c, const int32_t* budgets, int re
 
 using namespace lethe;
 
+#include <map>
+#include <mutex>
+#include <utility>
+
+namespace lethe {
+cudaError_t prepare_kernel(const void* func, size_t smem_needed) {
+    static std::mutex mu;
+    static std::map<std::pair<const void*, int>, size_t> done;  // (function, device) -> opted-in bytes
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = done.find({func, dev});
+    if (it != done.end()) return smem_needed <= it->second ? cudaSuccess : cudaErrorInvalidValue;
+    int max_optin = 0;
+    e = cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) return e;
+    cudaFuncAttributes fa;
+    e = cudaFuncGetAttributes(&fa, func);
+    if (e != cudaSuccess) return e;
+    const int max_dyn = max_optin - (int)fa.sharedSizeBytes;  // static shared memory counts against the limit
+    e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(func, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e != cudaSuccess) return e;
+    done[{func, dev}] = (size_t)max_dyn;
+    return smem_needed <= (size_t)max_dyn ? cudaSuccess : cudaErrorInvalidValue;
+}
+}  // namespace lethe
+
 struct lethe_ctx {
     int device;
     int sm_count;
@@ -32,6 +62,9 @@ struct lethe_ctx {
     void* staging;  // device staging of lethe_decode_attend_host
     size_t staging_bytes;
     int variant, splits;
+#ifdef LETHE_TIMELINE
+    unsigned long long* timeline;
+#endif
     char err[256];
 };
 
@@ -179,9 +212,18 @@ lethe_status lethe_poll_status(lethe_ctx* ctx, void* stream, int32_t* info) {
     return (lethe_status)h[0];
 }
 
+#ifdef LETHE_TIMELINE
+// Debug builds only: per-CTA timestamps of the next attend launches go to `buf` (8 x uint64 per CTA).
+lethe_status lethe_debug_set_timeline(lethe_ctx* ctx, unsigned long long* buf) {
+    if (!ctx) return LETHE_ERR_INVALID_ARG;
+    ctx->timeline = buf;
+    return LETHE_OK;
+}
+#endif
+
 lethe_status lethe_set_tuning(lethe_ctx* ctx, int variant, int splits) {
     if (!ctx) return LETHE_ERR_INVALID_ARG;
-    if (variant < 0 || variant > 3) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..3");
+    if (variant < 0 || variant > 7) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..7");
     if (!(splits == 0 || splits == 1 || splits == 2 || splits == 4 || splits == 8 || splits == 16))
         return fail(ctx, LETHE_ERR_INVALID_ARG, "splits must be 0, 1, 2, 4, 8 or 16");
     ctx->variant = variant;
@@ -223,6 +265,9 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
     a.layer_begin = layer_begin;
     a.n_items = (layer_end - layer_begin) * c->batch * c->n_kv_heads;
     a.gamma = gamma;
+#ifdef LETHE_TIMELINE
+    a.timeline = ctx->timeline;
+#endif
     for (int l = 0; l < c->n_layers; ++l) a.scale_log2[l] = scale[l] * 1.4426950408889634f;
 
     const bool paged = c->layout == LETHE_PAGED;

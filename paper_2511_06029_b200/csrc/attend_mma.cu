@@ -70,12 +70,24 @@ __global__ void __launch_bounds__(NW * 32) attend_mma_kernel(const __grid_consta
     EpilogueSmem& es = *reinterpret_cast<EpilogueSmem*>(cta_o + kMaxGroup * D);
     float* lg = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(&es) + sizeof(EpilogueSmem));
 
+    TL_MARK(a, 0);
     const ItemCoord ic = decode_item(a);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int gq = lane >> 2, tq = lane & 3;  // fragment coordinates: row group, column pair
     const int G = a.G, GP = a.GP;
     const bool append = a.k_new != nullptr;
     const int n_old = a.len[ic.item];
+    // Q^T fragments (B operand): b0 = Q[head gq][16 ks + 2 tq, +1], b1 = Q[head gq][16 ks + 8 + 2 tq, +1]
+    uint32_t bq[KS][2];
+    {
+        const uint32_t* qrow =
+            reinterpret_cast<const uint32_t*>((const T*)a.q + ((size_t)(ic.li * a.B + ic.b) * a.Hq + ic.hkv * G + gq) * D);
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            bq[ks][0] = (gq < G) ? qrow[8 * ks + tq] : 0u;
+            bq[ks][1] = (gq < G) ? qrow[8 * ks + 4 + tq] : 0u;
+        }
+    }
     T* out_rows = (T*)a.out + ((size_t)(ic.li * a.B + ic.b) * a.Hq + ic.hkv * G) * D;
     if (append && n_old >= a.cap_tokens) {  // full: leave the item untouched (every CTA of the cluster returns)
         if (ic.rank == 0) {
@@ -105,17 +117,6 @@ __global__ void __launch_bounds__(NW * 32) attend_mma_kernel(const __grid_consta
     }
     __syncthreads();  // the appended row is in global memory before any warp streams it
 
-    // Q^T fragments (B operand): b0 = Q[head gq][16 ks + 2 tq, +1], b1 = Q[head gq][16 ks + 8 + 2 tq, +1]
-    uint32_t bq[KS][2];
-    {
-        const uint32_t* qrow =
-            reinterpret_cast<const uint32_t*>((const T*)a.q + ((size_t)(ic.li * a.B + ic.b) * a.Hq + ic.hkv * G + gq) * D);
-#pragma unroll
-        for (int ks = 0; ks < KS; ++ks) {
-            bq[ks][0] = (gq < G) ? qrow[8 * ks + tq] : 0u;
-            bq[ks][1] = (gq < G) ? qrow[8 * ks + 4 + tq] : 0u;
-        }
-    }
     const float sl2 = a.scale_log2[ic.l];
 
     unsigned char* my_stage = stage_base + (size_t)warp * WARP_BYTES;
@@ -173,6 +174,7 @@ __global__ void __launch_bounds__(NW * 32) attend_mma_kernel(const __grid_consta
     const int k_row = (lane & 7) + ((lane >> 3) & 1) * 8, k_chunk = lane >> 4;
     const int v_row = (lane & 7) + ((lane >> 4) & 1) * 8, v_chunk = (lane >> 3) & 1;
 
+    TL_MARK(a, 1);
     for (int it = 0; it < my_count; ++it) {
         cp_async_wait<NSTAGE - 2>();
         __syncwarp();
@@ -236,6 +238,9 @@ __global__ void __launch_bounds__(NW * 32) attend_mma_kernel(const __grid_consta
         if (nxt < my_count) issue(my_first + nxt * NW, nxt % NSTAGE);
         cp_async_commit();
     }
+    TL_MARK(a, 2);
+    float rel_old[kRelPrefetch];
+    prefetch_rel<NW * 32>(a, ic, t0, min(t1, n), append_slot, rel_old);
     cp_async_wait<0>();
     __syncwarp();
     if (bad_page) record_error(a.status, LETHE_ERR_PAGE, ic.item);
@@ -259,7 +264,7 @@ __global__ void __launch_bounds__(NW * 32) attend_mma_kernel(const __grid_consta
         wo[(2 * tq + 1) * D + 16 * mt + gq + 8] = o[mt][3];
     }
     combine_and_finish<T, D, NW>(a, ic, es, reinterpret_cast<float*>(stage_base), WARP_BYTES / 4, cta_o, lg, t0, t1,
-                                 append_slot, n);
+                                 append_slot, n, rel_old);
 }
 
 template <int D, int NW, int NSTAGE>
@@ -272,12 +277,8 @@ template <int D, int NW, int NSTAGE, bool PAGED>
 static cudaError_t launch_mma_t(const AttendArgs& a, cudaStream_t stream) {
     auto kern = attend_mma_kernel<D, NW, NSTAGE, PAGED>;
     const size_t smem = mma_smem<D, NW, NSTAGE>(a.chunk_tokens, a.GP);
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = prepare_kernel((const void*)kern, smem);
     if (e != cudaSuccess) return e;
-    if (a.splits > 8) {
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-        if (e != cudaSuccess) return e;
-    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(a.n_items * a.splits), 1, 1);
     cfg.blockDim = dim3(NW * 32, 1, 1);
@@ -293,19 +294,27 @@ static cudaError_t launch_mma_t(const AttendArgs& a, cudaStream_t stream) {
     return cudaLaunchKernelEx(&cfg, kern, a);
 }
 
-// Shared memory one CTA of the tensor-core kernel needs (shape: 0 = 4 warps x 3 stages, 1 = 8 warps x 3 stages).
+// Kernel shapes (warps per CTA, pipeline stages per warp), selected by `shape`.
+#define LETHE_MMA_SHAPES(X, D) \
+    X(0, D, 4, 3) X(1, D, 8, 3) X(2, D, 4, 2) X(3, D, 8, 2) X(4, D, 4, 4) X(5, D, 2, 4)
+
 size_t mma_smem_bytes(int D, int shape, int chunk_tokens, int GP) {
-    if (D == 64) return shape == 0 ? mma_smem<64, 4, 4>(chunk_tokens, GP) : mma_smem<64, 8, 4>(chunk_tokens, GP);
-    return shape == 0 ? mma_smem<128, 4, 3>(chunk_tokens, GP) : mma_smem<128, 8, 3>(chunk_tokens, GP);
+#define X(id, DD, NW, NS) \
+    if (shape == id && D == DD) return mma_smem<DD, NW, NS>(chunk_tokens, GP);
+    LETHE_MMA_SHAPES(X, 128)
+    LETHE_MMA_SHAPES(X, 64)
+#undef X
+    return (size_t)-1;
 }
 
 cudaError_t launch_attend_mma(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream) {
-    if (D == 64) {
-        if (shape == 0) return paged ? launch_mma_t<64, 4, 4, true>(a, stream) : launch_mma_t<64, 4, 4, false>(a, stream);
-        return paged ? launch_mma_t<64, 8, 4, true>(a, stream) : launch_mma_t<64, 8, 4, false>(a, stream);
-    }
-    if (shape == 0) return paged ? launch_mma_t<128, 4, 3, true>(a, stream) : launch_mma_t<128, 4, 3, false>(a, stream);
-    return paged ? launch_mma_t<128, 8, 3, true>(a, stream) : launch_mma_t<128, 8, 3, false>(a, stream);
+#define X(id, DD, NW, NS)                                                                           \
+    if (shape == id && D == DD)                                                                     \
+        return paged ? launch_mma_t<DD, NW, NS, true>(a, stream) : launch_mma_t<DD, NW, NS, false>(a, stream);
+    LETHE_MMA_SHAPES(X, 128)
+    LETHE_MMA_SHAPES(X, 64)
+#undef X
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace lethe

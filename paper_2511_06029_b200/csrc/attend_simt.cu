@@ -64,13 +64,12 @@ __global__ void __launch_bounds__(NW * 32) attend_simt_kernel(const __grid_const
     const bool append = a.k_new != nullptr;
     const int n_old = a.len[ic.item];
     T* out_rows = (T*)a.out + ((size_t)(ic.li * a.B + ic.b) * a.Hq + ic.hkv * G) * D;
-    if (append && n_old >= a.cap_tokens) {  // full: leave the item untouched (uniform over the cluster)
+    if (append && n_old >= a.cap_tokens) {  // full: leave the item untouched (every CTA of the cluster returns)
         if (ic.rank == 0) {
             for (int i = tid; i < G * D; i += NW * 32) out_rows[i] = from_float<T>(0.f);
             if (a.lse && tid < G) a.lse[(size_t)(ic.li * a.B + ic.b) * a.Hq + ic.hkv * G + tid] = -INFINITY;
             if (tid == 0) record_error(a.status, LETHE_ERR_CAPACITY, ic.item);
         }
-        if (a.splits > 1) { cg::this_cluster().sync(); cg::this_cluster().sync(); }
         return;
     }
     const int n = n_old + (append ? 1 : 0);
@@ -176,7 +175,9 @@ __global__ void __launch_bounds__(NW * 32) attend_simt_kernel(const __grid_const
 #pragma unroll
         for (int e = 0; e < E; ++e) wo[(warp * kMaxGroup + h) * D + lane * E + e] = o[h][e];
     }
-    combine_and_finish<T, D, NW>(a, ic, es, wo, kMaxGroup * D, cta_o, lg, t0, t1, append_slot, n);
+    float rel_old[kRelPrefetch];
+    prefetch_rel<NW * 32>(a, ic, t0, min(t1, n), append_slot, rel_old);
+    combine_and_finish<T, D, NW>(a, ic, es, wo, kMaxGroup * D, cta_o, lg, t0, t1, append_slot, n, rel_old);
 }
 
 template <typename T, int D, int NW, bool PAGED>
@@ -184,12 +185,8 @@ static cudaError_t launch_simt_t(const AttendArgs& a, cudaStream_t stream) {
     auto kern = attend_simt_kernel<T, D, NW, PAGED>;
     const size_t smem = sizeof(EpilogueSmem) + (size_t)(NW + 1) * kMaxGroup * D * sizeof(float) +
                         (size_t)a.chunk_tokens * a.GP * sizeof(float);
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = prepare_kernel((const void*)kern, smem);
     if (e != cudaSuccess) return e;
-    if (a.splits > 8) {
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-        if (e != cudaSuccess) return e;
-    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(a.n_items * a.splits), 1, 1);
     cfg.blockDim = dim3(NW * 32, 1, 1);

@@ -38,8 +38,29 @@ struct AttendArgs {
     int splits;                // CTAs per item (cluster size)
     int chunk_tokens;          // logit-buffer capacity of one CTA, in tokens
     float gamma;
+#ifdef LETHE_TIMELINE
+    unsigned long long* timeline;  // debug builds only: 8 timestamps per CTA
+#endif
     float scale_log2[kMaxLayers];  // scale[l] * log2(e), by absolute layer
 };
+
+#ifdef LETHE_TIMELINE
+__device__ __forceinline__ void tl_mark(const AttendArgs& a, int slot) {
+    if (a.timeline && threadIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+        a.timeline[(size_t)blockIdx.x * 8 + slot] = t;
+        if (slot == 0) {
+            unsigned sm;
+            asm volatile("mov.u32 %0, %smid;" : "=r"(sm));
+            a.timeline[(size_t)blockIdx.x * 8 + 7] = sm;
+        }
+    }
+}
+#define TL_MARK(a, slot) tl_mark(a, slot)
+#else
+#define TL_MARK(a, slot)
+#endif
 
 // Cache state as the prune-round kernels see it.
 struct CacheView {
@@ -52,6 +73,10 @@ struct CacheView {
     long long n_pages;
     int L, B, Hkv, D, elt_bytes, capacity, cap_tokens, page_tokens, paged;
 };
+
+// Host: opt a kernel into the largest dynamic shared memory and non-portable cluster sizes, once per
+// (function, device); implemented in api.cu.
+cudaError_t prepare_kernel(const void* func, size_t smem_needed);
 
 __device__ __forceinline__ void record_error(int32_t* status, int code, int item) {
     if (atomicCAS(status, 0, code) == 0) status[1] = item;
@@ -138,6 +163,20 @@ struct EpilogueSmem {
     int flags[4];
 };
 
+// Old relevance values a thread will update: loaded early so that their latency hides behind the merge.
+constexpr int kRelPrefetch = 8;
+
+template <int NT>
+__device__ __forceinline__ void prefetch_rel(const AttendArgs& a, const ItemCoord& ic, int t0, int hi_tok,
+                                             int append_slot, float (&old)[kRelPrefetch]) {
+    const float* rel = a.rel + (size_t)ic.item * a.cap_tokens;
+#pragma unroll
+    for (int i = 0; i < kRelPrefetch; ++i) {
+        const int j = t0 + (int)threadIdx.x + i * NT;
+        old[i] = (j < hi_tok && j != append_slot) ? rel[j] : 0.f;
+    }
+}
+
 /*
  * Common tail of both attend kernels.  On entry every warp has written, for the tokens it streamed,
  *   es.wstat[w][h]   = (m, l): running max (log2 units) and sum of exp2(s - m) of head h
@@ -149,11 +188,12 @@ struct EpilogueSmem {
 template <typename T, int D, int NW>
 __device__ void combine_and_finish(const AttendArgs& a, const ItemCoord& ic, EpilogueSmem& es, float* wo, int wo_stride,
                                    float* cta_o /*[kMaxGroup][D]*/, const float* lg, int t0, int t1, int append_slot,
-                                   int n) {
+                                   int n, const float (&rel_old)[kRelPrefetch]) {
     const int tid = threadIdx.x;
     const int G = a.G;
     constexpr int NT = NW * 32;
     __syncthreads();
+    TL_MARK(a, 3);
     if (tid < kMaxGroup) {
         const int h = tid;
         float m = -INFINITY;
@@ -218,19 +258,38 @@ __device__ void combine_and_finish(const AttendArgs& a, const ItemCoord& ic, Epi
         }
     }
 
+    TL_MARK(a, 4);
     // Eq. 5: rel[j] = gamma * rel[j] + sum over the group's heads of p_hj, with the global (m, 1/l).
     float* rel = a.rel + (size_t)ic.item * a.cap_tokens;
     const int GP = a.GP;
     const int hi_tok = min(t1, n);
-    for (int j = t0 + tid; j < hi_tok; j += NT) {
+    float fm[kMaxGroup], fi[kMaxGroup];
+#pragma unroll
+    for (int h = 0; h < kMaxGroup; ++h) {
+        fm[h] = es.fin[h].x;
+        fi[h] = es.fin[h].y;
+    }
+    auto mass_of = [&](int j) {
         const float* row = lg + (size_t)(j - t0) * GP;
         float mass = 0.f;
-        for (int h = 0; h < G; ++h) mass += fast_exp2(row[h] - es.fin[h].x) * es.fin[h].y;
-        const float old = (j == append_slot) ? 0.f : rel[j];
-        rel[j] = fmaf(a.gamma, old, mass);
+#pragma unroll
+        for (int h = 0; h < kMaxGroup; ++h)
+            if (h < G) mass += fast_exp2(row[h] - fm[h]) * fi[h];
+        return mass;
+    };
+#pragma unroll
+    for (int i = 0; i < kRelPrefetch; ++i) {
+        const int j = t0 + tid + i * NT;
+        if (j < hi_tok) rel[j] = fmaf(a.gamma, rel_old[i], mass_of(j));
     }
+    for (int j = t0 + tid + kRelPrefetch * NT; j < hi_tok; j += NT) {
+        const float old = (j == append_slot) ? 0.f : rel[j];
+        rel[j] = fmaf(a.gamma, old, mass_of(j));
+    }
+    TL_MARK(a, 5);
     if (S > 1) cg::this_cluster().sync();  // peers may still be reading this CTA's shared memory
     if (append_slot >= 0 && ic.rank == 0 && tid == 0) a.len[ic.item] = n;
+    TL_MARK(a, 6);
 }
 
 }  // namespace lethe

@@ -337,7 +337,7 @@ cudaError_t launch_rasr_prune(const CacheView& c, const int32_t* budgets, int re
                               int max_k, int smem_tokens, int32_t* list_scratch, int32_t* status,
                               cudaStream_t stream) {
     const size_t smem = (size_t)smem_tokens * 4;
-    cudaError_t e = cudaFuncSetAttribute(rasr_prune_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = prepare_kernel((const void*)rasr_prune_kernel, smem);
     if (e != cudaSuccess) return e;
     rasr_prune_kernel<<<c.L * c.B * c.Hkv, kPruneThreads, smem, stream>>>(c, budgets, recent, sink, keep_idx, max_k,
                                                                          smem_tokens, list_scratch, status);
