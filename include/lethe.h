@@ -94,10 +94,16 @@ const char *lethe_last_error(const lethe_ctx *ctx);
  * {status, flat item index l*B*Hkv + b*Hkv + h of the first offender}. */
 lethe_status lethe_poll_status(lethe_ctx *ctx, void *stream, int32_t *info);
 
-/* Tuning knobs (HOST values).  variant: 0 = automatic, 1 = CUDA-core kernel, 2..7 = tensor-core (mma)
- * kernel (bf16 only) with (warps per CTA, pipeline stages per warp) = (4,3) (8,3) (4,2) (8,2) (4,4) (2,4).
- * splits: 0 = automatic, else CTAs per item (1, 2, 4, 8 or 16; they form one thread-block cluster).
- * Returns LETHE_ERR_INVALID_ARG for other values. */
+/* Tuning knobs (HOST values).
+ * variant: 0 = automatic; 1 = CUDA-core kernel; 2..7 = clustered tensor-core (mma) kernel with (warps per
+ * CTA, pipeline stages per warp) = (4,3) (8,3) (4,2) (8,2) (4,4) (2,4); 8..13 = persistent tensor-core
+ * kernel (one CTA per SM, dynamic item queue, cross-item prefetch) with (8,2) (6,3) (10,2) (8,3) (7,3) (5,4).
+ * Tensor-core variants need a bf16 cache (and 16-token pages when paged).
+ * splits: 0 = automatic, else CTAs per item (1, 2, 4, 8 or 16; they form one thread-block cluster); the
+ * persistent variants take 0 or 1.
+ * Returns LETHE_ERR_INVALID_ARG for other values.
+ * A context serialises its calls: issue them to one stream at a time (the status word and the persistent
+ * kernel's work queue are per context). */
 lethe_status lethe_set_tuning(lethe_ctx *ctx, int variant, int splits);
 
 /*

@@ -12,6 +12,8 @@ cudaError_t launch_attend_simt(const AttendArgs& a, int dtype, int D, bool paged
 size_t simt_smem_bytes(int D, int chunk_tokens, int GP);
 cudaError_t launch_attend_mma(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream);
 size_t mma_smem_bytes(int D, int shape, int chunk_tokens, int GP);
+cudaError_t launch_attend_stream(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream);
+size_t stream_smem_bytes(int D, int shape, int chunk_tokens, int GP);
 cudaError_t launch_sparsity(const CacheView& c, float* sparsity, cudaStream_t stream);
 cudaError_t launch_budgets(int L, int B, const float* sparsity, const long long* total, int k_min, int32_t* budgets,
                            int32_t* status, cudaStream_t stream);
@@ -56,7 +58,8 @@ struct lethe_ctx {
     int device;
     int sm_count;
     size_t max_smem;  // opt-in dynamic shared memory per CTA
-    int32_t* status;  // device: {code, item}
+    int32_t* status;      // device: {code, item} followed by the persistent kernel's work-queue words
+    unsigned int* sched;  // device: {next ticket, CTAs finished}; zero whenever no attend launch is running
     void* scratch;
     size_t scratch_bytes;
     void* staging;  // device staging of lethe_decode_attend_host
@@ -161,11 +164,12 @@ lethe_status lethe_create(lethe_ctx** out, int device, size_t scratch_bytes_hint
     ctx->sm_count = prop.multiProcessorCount;
     ctx->max_smem = prop.sharedMemPerBlockOptin;
     strcpy(ctx->err, "no error");
-    if (cudaMalloc((void**)&ctx->status, 2 * sizeof(int32_t)) != cudaSuccess ||
-        cudaMemset(ctx->status, 0, 2 * sizeof(int32_t)) != cudaSuccess) {
+    if (cudaMalloc((void**)&ctx->status, 4 * sizeof(int32_t)) != cudaSuccess ||
+        cudaMemset(ctx->status, 0, 4 * sizeof(int32_t)) != cudaSuccess) {
         delete ctx;
         return LETHE_ERR_CUDA;
     }
+    ctx->sched = reinterpret_cast<unsigned int*>(ctx->status + 2);
     if (scratch_bytes_hint) {
         if (ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, scratch_bytes_hint, "scratch") != LETHE_OK) {
             cudaFree(ctx->status);
@@ -223,7 +227,7 @@ lethe_status lethe_debug_set_timeline(lethe_ctx* ctx, unsigned long long* buf) {
 
 lethe_status lethe_set_tuning(lethe_ctx* ctx, int variant, int splits) {
     if (!ctx) return LETHE_ERR_INVALID_ARG;
-    if (variant < 0 || variant > 7) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..7");
+    if (variant < 0 || variant > 13) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..13");
     if (!(splits == 0 || splits == 1 || splits == 2 || splits == 4 || splits == 8 || splits == 16))
         return fail(ctx, LETHE_ERR_INVALID_ARG, "splits must be 0, 1, 2, 4, 8 or 16");
     ctx->variant = variant;
@@ -258,6 +262,7 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
     a.k = c->k; a.v = c->v; a.rel = c->rel; a.pos = c->pos; a.len = c->len; a.page_table = c->page_table;
     a.q = q; a.k_new = k_new; a.v_new = v_new; a.token_pos = token_pos; a.out = out; a.lse = lse;
     a.status = ctx->status;
+    a.sched = ctx->sched;
     a.n_pages = c->n_pages;
     a.B = c->batch; a.Hq = c->n_q_heads; a.Hkv = c->n_kv_heads; a.G = G; a.GP = (G + 1) & ~1;
     a.capacity = c->capacity; a.cap_tokens = cap_tokens_of(c);
@@ -272,29 +277,50 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
 
     const bool paged = c->layout == LETHE_PAGED;
     const bool mma_ok = c->dtype == LETHE_BF16 && (!paged || c->page_tokens == kGroupTokens);
-    int variant = ctx->variant;
-    if (variant == 0) variant = mma_ok ? 2 : 1;
-    if (variant >= 2 && !mma_ok) return fail(ctx, LETHE_ERR_UNSUPPORTED, "tensor-core variant needs bf16 and 16-token pages");
-
-    // CTAs per item: the smallest cluster whose logit buffer fits, grown until the grid covers the SMs twice.
     const int cap_groups = (a.cap_tokens + kGroupTokens - 1) / kGroupTokens;
-    auto smem_for = [&](int S) -> size_t {
-        const int chunk = ((cap_groups + S - 1) / S) * kGroupTokens;
-        return variant == 1 ? simt_smem_bytes(c->head_dim, chunk, a.GP) : mma_smem_bytes(c->head_dim, variant - 2, chunk, a.GP);
-    };
-    int S = ctx->splits;
-    if (S == 0) {
-        S = 1;
-        while (S < 16 && smem_for(S) > ctx->max_smem) S *= 2;
-        while (S < 8 && (long long)a.n_items * S < 2LL * ctx->sm_count && cap_groups / (2 * S) >= 4) S *= 2;
+    int variant = ctx->variant;
+    if (variant == 0) {
+        // enough items to give every SM several: the persistent kernel; few long items: the clustered one
+        auto stream_fits = [&](int shape) {
+            return stream_smem_bytes(c->head_dim, shape, cap_groups * kGroupTokens, a.GP) <= ctx->max_smem;
+        };
+        if (!mma_ok) variant = 1;
+        else if (a.n_items >= 2 * ctx->sm_count && ctx->splits <= 1 && stream_fits(4)) variant = 12;  // 7 warps x 3 stages
+        else if (a.n_items >= 2 * ctx->sm_count && ctx->splits <= 1 && stream_fits(1)) variant = 9;   // 6 warps x 3 stages
+        else if (a.n_items >= 2 * ctx->sm_count && ctx->splits <= 1 && stream_fits(0)) variant = 8;   // 8 warps x 2 stages
+        else variant = 4;
     }
-    if (smem_for(S) > ctx->max_smem)
-        return fail(ctx, LETHE_ERR_UNSUPPORTED, "capacity too large for the on-chip logit buffer at this split count");
-    a.splits = S;
-    a.chunk_tokens = ((cap_groups + S - 1) / S) * kGroupTokens;
+    if (variant >= 2 && !mma_ok) return fail(ctx, LETHE_ERR_UNSUPPORTED, "tensor-core variants need bf16 and 16-token pages");
 
-    cudaError_t e = variant == 1 ? launch_attend_simt(a, c->dtype, c->head_dim, paged, (cudaStream_t)stream)
-                                 : launch_attend_mma(a, c->head_dim, variant - 2, paged, (cudaStream_t)stream);
+    cudaError_t e;
+    if (variant >= 8) {  // persistent: one CTA per SM walks all items
+        if (ctx->splits > 1) return fail(ctx, LETHE_ERR_INVALID_ARG, "the persistent variant does not split items");
+        a.splits = 1;
+        a.chunk_tokens = cap_groups * kGroupTokens;
+        if (stream_smem_bytes(c->head_dim, variant - 8, a.chunk_tokens, a.GP) > ctx->max_smem)
+            return fail(ctx, LETHE_ERR_UNSUPPORTED, "capacity too large for the on-chip logit buffer of the persistent variant");
+        const int grid = a.n_items < ctx->sm_count ? a.n_items : ctx->sm_count;
+        e = launch_attend_stream(a, c->head_dim, variant - 8, paged, grid, (cudaStream_t)stream);
+    } else {
+        // CTAs per item: the smallest cluster whose logit buffer fits, grown until the grid covers the SMs twice.
+        auto smem_for = [&](int S) -> size_t {
+            const int chunk = ((cap_groups + S - 1) / S) * kGroupTokens;
+            return variant == 1 ? simt_smem_bytes(c->head_dim, chunk, a.GP)
+                                : mma_smem_bytes(c->head_dim, variant - 2, chunk, a.GP);
+        };
+        int S = ctx->splits;
+        if (S == 0) {
+            S = 1;
+            while (S < 16 && smem_for(S) > ctx->max_smem) S *= 2;
+            while (S < 8 && (long long)a.n_items * S < 2LL * ctx->sm_count && cap_groups / (2 * S) >= 4) S *= 2;
+        }
+        if (smem_for(S) > ctx->max_smem)
+            return fail(ctx, LETHE_ERR_UNSUPPORTED, "capacity too large for the on-chip logit buffer at this split count");
+        a.splits = S;
+        a.chunk_tokens = ((cap_groups + S - 1) / S) * kGroupTokens;
+        e = variant == 1 ? launch_attend_simt(a, c->dtype, c->head_dim, paged, (cudaStream_t)stream)
+                         : launch_attend_mma(a, c->head_dim, variant - 2, paged, (cudaStream_t)stream);
+    }
     if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attend launch");
     return LETHE_OK;
 }

@@ -30,7 +30,8 @@ struct AttendArgs {
     const int32_t* token_pos;
     void* out;
     float* lse;
-    int32_t* status;  // device status word: {code, item}
+    int32_t* status;      // device status word: {code, item}
+    unsigned int* sched;  // persistent kernel only: {next ticket, CTAs finished}, zero between launches
     long long n_pages;
     int B, Hq, Hkv, G, GP;  // GP = G rounded up to even: row pitch of the logit buffer
     int capacity, cap_tokens, page_tokens;

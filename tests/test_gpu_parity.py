@@ -68,6 +68,16 @@ CASES = [
     (torch.bfloat16, 128, 6, 2, 1000, 3, 16),
     (torch.bfloat16, 64, 8, 2, 300, 2, 2),
     (torch.bfloat16, 64, 10, 2, 500, 3, 4),
+    (torch.bfloat16, 128, 32, 8, 300, 4, 2),
+    (torch.bfloat16, 128, 28, 4, 300, 5, 4),
+    (torch.bfloat16, 64, 8, 2, 300, 6, 1),
+    (torch.bfloat16, 128, 8, 2, 300, 7, 2),
+    (torch.bfloat16, 128, 32, 8, 300, 8, 0),
+    (torch.bfloat16, 128, 28, 4, 700, 9, 1),
+    (torch.bfloat16, 64, 14, 2, 300, 10, 0),
+    (torch.bfloat16, 128, 4, 1, 300, 11, 0),
+    (torch.bfloat16, 64, 16, 2, 500, 12, 0),
+    (torch.bfloat16, 128, 6, 2, 300, 13, 0),
     (torch.bfloat16, 128, 8, 8, 260, 0, 0),
     (torch.float32, 128, 16, 2, 260, 0, 0),
 ]
@@ -92,6 +102,46 @@ def test_decode_attend_parity(ctx, dtype, D, Hq, Hkv, cap, variant, splits):
             vn = torch.randn((nl, B, Hkv, D), generator=g).to(dtype) if app else None
             tp = torch.tensor([1000 + step, 2000 + step], dtype=torch.int32) if app else None
             _step(ctx, oc, gc, q, kn, vn, tp, scale, 0.9, l0, l1)
+    finally:
+        ctx.set_tuning(0, 0)
+
+
+@pytest.mark.parametrize("variant", [8, 9, 10, 12, 13])
+def test_persistent_queue_many_items(ctx, variant):
+    """More items than SMs, so every CTA of the persistent kernel walks several items through its queue and
+    prefetches across item boundaries; lengths from 0 to several hundred, including tiny items that leave
+    some warps without work, and one full item."""
+    from paper_2511_06029_b200 import binding
+    L, B, Hq, Hkv, D, cap = 5, 8, 16, 8, 128, 400
+    lens = _lens(L, B, Hkv, cap - 6, seed=variant, special=(1, 2, 15, 16, 17, 31, 32, 33, 47, 48, 49, 127, 128, 129,
+                                                           255, 256, 257, 390))
+    oc = random_cache(L, B, Hq, Hkv, D, cap, lens, dtype=torch.bfloat16, seed=variant, rel_init="rand")
+    gc = to_device(oc)
+    ctx.set_tuning(variant, 0)
+    try:
+        g = torch.Generator().manual_seed(5)
+        scale = torch.tensor([0.09, 0.2, 0.05, 0.12, 0.07], dtype=torch.float32)
+        for step in range(4):
+            app = step != 1
+            q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+            kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16) if app else None
+            vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16) if app else None
+            tp = torch.arange(B, dtype=torch.int32) + 1000 * step if app else None
+            _step(ctx, oc, gc, q, kn, vn, tp, scale, 0.97, 0, L)
+        # an empty item and a full one in the same launch
+        oc.len[2, 3, 4] = 0; oc.len[4, 7, 7] = cap
+        sync_state(gc, oc)
+        q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+        _step(ctx, oc, gc, q, None, None, None, scale, 0.97, 0, L)            # attend only: empty item -> zeros, -inf
+        kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16).cuda()
+        out = torch.full((L, B, Hq, D), 7.0, dtype=torch.bfloat16, device="cuda")
+        before_k = gc.k[4, 7, 7].clone(); before_rel = gc.rel[4, 7, 7].clone()
+        ctx.decode_attend(gc, 0, L, q.cuda(), kn, kn, torch.zeros(B, dtype=torch.int32).cuda(), scale.tolist(), 0.97, out)
+        st, item = ctx.poll_status()
+        assert st == binding.ERR_CAPACITY and item == (4 * B + 7) * Hkv + 7
+        assert int(gc.len[4, 7, 7]) == cap and int(gc.len[2, 3, 4]) == 1
+        assert torch.equal(gc.k[4, 7, 7], before_k) and torch.equal(gc.rel[4, 7, 7], before_rel)
+        assert torch.all(out[4, 7, 14:16] == 0) and torch.isfinite(out.float()).all()
     finally:
         ctx.set_tuning(0, 0)
 
