@@ -27,7 +27,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from paper_2511_06029_b200 import synth  # noqa: E402
+from paper_2511_06029_b200 import dist_util, synth  # noqa: E402
 
 METRIC = "kv_token_heads_attended_per_s"
 UNIT = "token-heads/s"
@@ -359,18 +359,9 @@ def main():
         r.check()
     clocks = sampler.stop() if sampler else None
 
-    units = float(sum(th))
-    t_ms = total_ms
-    if dist is not None:
-        t = torch.tensor([total_ms, e_total_ms if not args.no_e2e else 0.0], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        u = torch.tensor([units, float(sum(e_th)) if not args.no_e2e else 0.0], device=dev, dtype=torch.float64)
-        dist.all_reduce(u, op=dist.ReduceOp.SUM)
-        t_ms, units = float(t[0]), float(u[0])
-        if not args.no_e2e:
-            e_total_ms, e_units = float(t[1]), float(u[1])
-    elif not args.no_e2e:
-        e_units = float(sum(e_th))
+    e_ms = e_total_ms if not args.no_e2e else 0.0
+    e_u = float(sum(e_th)) if not args.no_e2e else 0.0
+    (t_ms, e_total_ms), (units, e_units) = dist_util.reduce_job(dist, dev, [total_ms, e_ms], [float(sum(th)), e_u])
 
     if rank == 0:
         peak, which = measured_peak()
@@ -381,7 +372,7 @@ def main():
         h2d = (wq.n_layers * wq.batch * (wq.n_q_heads + 2 * wq.n_kv_heads) * wq.head_dim * 2 + wq.batch * 4)
         d2h = wq.n_layers * wq.batch * wq.n_q_heads * wq.head_dim * 2
         line = {
-            "metric": METRIC, "value": units / (t_ms * 1e-3), "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "metric": METRIC, "value": dist_util.job_value(units, t_ms), "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": t_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": workload_config(w, args, extra={
@@ -400,7 +391,7 @@ def main():
             "gpu_launches": launches, "clocks": clocks,
         }
         if not args.no_e2e:
-            line["e2e"] = {"value": e_units / (e_total_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            line["e2e"] = {"value": dist_util.job_value(e_units, e_total_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                            "d2h_bytes_per_step": d2h, "ms_per_step": e_total_ms / args.steps}
         if not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, r)
