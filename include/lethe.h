@@ -57,7 +57,8 @@ typedef enum {
     LETHE_ERR_CUDA = 4,        /* a CUDA runtime call failed; see lethe_last_error */
     LETHE_ERR_TIMEOUT = 5,     /* reserved: a bounded device-side wait ran out */
     LETHE_ERR_UNSUPPORTED = 6, /* valid request outside what the kernels cover */
-    LETHE_ERR_PAGE = 7         /* device-side: page id outside [0, n_pages) */
+    LETHE_ERR_PAGE = 7,        /* device-side: page id outside [0, n_pages) */
+    LETHE_ERR_TOO_LARGE = 8    /* lethe_rasr_prune_static: the cache exceeds LETHE_STATIC_PRUNE_MAX_ENTRIES */
 } lethe_status;
 
 enum { LETHE_F32 = 0, LETHE_BF16 = 1 };
@@ -186,6 +187,38 @@ lethe_status lethe_alloc_budgets(lethe_ctx *ctx, int n_layers, int batch, const 
  */
 lethe_status lethe_rasr_prune(lethe_ctx *ctx, const lethe_cache *cache, const int32_t *budgets, int32_t recent,
                               int32_t sink, int32_t *keep_idx, int32_t max_k, void *stream);
+
+/*
+ * lethe_rasr_prune without a context and without any allocation.  (The paper has no counterpart: this entry
+ * point exists for the way the library is deployed, not for the method.)
+ *
+ * Who needs it: callers that must not allocate device memory when a prune round is due — an inference server
+ * that handed all device memory to its own pool at start-up (a driver allocation could fail or fragment that
+ * pool), or a latency-critical decode loop in which a driver allocation, which may stall the whole device, is
+ * not acceptable.  Such callers cannot even create a lethe_ctx, whose creation allocates.
+ *
+ * Same semantics, arguments and results as lethe_rasr_prune, with these differences:
+ *   - it runs on the CURRENT CUDA device, which must be the one that holds the cache;
+ *   - its scratch (each item's list of survivors, LETHE_STATIC_PRUNE_MAX_ENTRIES int32 = 16 MiB, plus a
+ *     256-byte status block) is a fixed array inside the library image: every GPU that loads the library
+ *     carries it until the process exits.  A cache with n_layers * batch * n_kv_heads * cap_tokens above
+ *     LETHE_STATIC_PRUNE_MAX_ENTRIES is refused with LETHE_ERR_TOO_LARGE and nothing is enqueued;
+ *   - it calls no cudaMalloc / cudaFree and no allocating library routine; it enqueues one 8-byte memset, one
+ *     kernel and (with status_out) one 8-byte copy on `stream`;
+ *   - the first call on a device looks up the scratch's device address (cudaGetSymbolAddress).  Make that
+ *     first call before any stream capture begins;
+ *   - all calls share the one array, which still holds whatever the previous call left in it (the status
+ *     block is cleared at the start of each call; the lists are always written before they are read).  Two
+ *     calls whose kernels could overlap on the GPU — different streams without an ordering event, or several
+ *     host threads — race on it: order them;
+ *   - status_out: optional DEVICE pointer to int32[2], caller-owned; after the call's work on `stream` it
+ *     holds {0, 0} or {LETHE_ERR_BUDGET or LETHE_ERR_PAGE, flat item index} of the first device-side event.
+ * Host-detectable errors return LETHE_ERR_INVALID_ARG / LETHE_ERR_UNSUPPORTED / LETHE_ERR_TOO_LARGE /
+ * LETHE_ERR_CUDA and enqueue nothing.
+ */
+#define LETHE_STATIC_PRUNE_MAX_ENTRIES (4 * 1024 * 1024)
+lethe_status lethe_rasr_prune_static(const lethe_cache *cache, const int32_t *budgets, int32_t recent, int32_t sink,
+                                     int32_t *keep_idx, int32_t max_k, int32_t *status_out, void *stream);
 
 #ifdef __cplusplus
 }

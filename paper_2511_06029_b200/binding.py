@@ -15,14 +15,15 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("LETHE_LIB", os.path.join(_HERE, "liblethe.so"))   # LETHE_LIB: an alternative build
 
-OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_BUDGET, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED, ERR_PAGE = range(8)
+OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_BUDGET, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED, ERR_PAGE, ERR_TOO_LARGE = range(9)
+STATIC_PRUNE_MAX_ENTRIES = 4 * 1024 * 1024
 F32, BF16 = 0, 1
 CONTIG, PAGED = 0, 1
 VARIANT_AUTO, VARIANT_SIMT, VARIANT_MMA4, VARIANT_MMA8 = 0, 1, 2, 3
 
 EXPORTS = ["lethe_create", "lethe_destroy", "lethe_last_error", "lethe_poll_status", "lethe_set_tuning",
            "lethe_decode_attend", "lethe_decode_attend_host", "lethe_estimate_sparsity", "lethe_alloc_budgets",
-           "lethe_rasr_prune"]
+           "lethe_rasr_prune", "lethe_rasr_prune_static"]
 
 
 class LetheError(RuntimeError):
@@ -76,6 +77,8 @@ def load() -> ctypes.CDLL:
     lib.lethe_alloc_budgets.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp, vp, i32, vp, vp]
     lib.lethe_rasr_prune.restype = ctypes.c_int
     lib.lethe_rasr_prune.argtypes = [vp, cp, vp, i32, i32, vp, i32, vp]
+    lib.lethe_rasr_prune_static.restype = ctypes.c_int
+    lib.lethe_rasr_prune_static.argtypes = [cp, vp, i32, i32, vp, i32, vp, vp]
     _lib = lib
     return lib
 
@@ -121,6 +124,22 @@ class Cache:
     @property
     def cap_tokens(self) -> int:
         return self.capacity * self.page_tokens if self.page_table is not None else self.capacity
+
+
+def rasr_prune_static(cache: "Cache", budgets: torch.Tensor, recent: int, sink: int,
+                      keep_idx: Optional[torch.Tensor] = None, status_out: Optional[torch.Tensor] = None) -> int:
+    """lethe_rasr_prune_static: the prune step for callers that may not allocate device memory (no context, fixed
+    in-library scratch).  Runs on the current device and the current torch stream; returns the host-side status
+    (OK, or ERR_TOO_LARGE / ERR_INVALID_ARG / ... when nothing was enqueued).  status_out: device int32[2]."""
+    assert budgets.dtype == torch.int32 and budgets.is_cuda
+    max_k = 0
+    if keep_idx is not None:
+        assert keep_idx.dtype == torch.int32 and keep_idx.is_cuda
+        max_k = keep_idx.shape[-1]
+    if status_out is not None:
+        assert status_out.dtype == torch.int32 and status_out.is_cuda and status_out.numel() >= 2
+    return int(load().lethe_rasr_prune_static(ctypes.byref(cache.c), _dp(budgets), recent, sink, _dp(keep_idx), max_k,
+                                              _dp(status_out), _stream(cache.device)))
 
 
 class Context:

@@ -345,3 +345,78 @@ cudaError_t launch_rasr_prune(const CacheView& c, const int32_t* budgets, int re
 }
 
 }  // namespace lethe
+
+// ------------------------------------------------------------------ retention with no allocation at all
+// Scratch of lethe_rasr_prune_static: a status word (first 256 bytes) followed by the survivors' source-slot
+// lists of every item.  It lives in the library image, so each GPU that loads the library holds these
+// 16 MiB + 256 B until the process exits; every call reuses it and finds the previous call's contents.
+static __device__ __align__(256) int32_t g_static_prune_scratch[64 + LETHE_STATIC_PRUNE_MAX_ENTRIES];
+
+#include <mutex>
+
+namespace {
+// Device address of the scratch on the current device.  In host code the array's name is only a handle, not a
+// device address, so the address is asked for once per device (with that device current) and remembered.
+cudaError_t static_prune_scratch(int32_t** out) {
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static int32_t* addr[kMaxDevices] = {};
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_prune_scratch);
+        if (e != cudaSuccess) return e;
+        addr[dev] = static_cast<int32_t*>(p);
+    }
+    *out = addr[dev];
+    return cudaSuccess;
+}
+}  // namespace
+
+extern "C" lethe_status lethe_rasr_prune_static(const lethe_cache* c, const int32_t* budgets, int32_t recent,
+                                                int32_t sink, int32_t* keep_idx, int32_t max_k, int32_t* status_out,
+                                                void* stream) {
+    using namespace lethe;
+    if (!c || !budgets || !c->k || !c->v || !c->rel || !c->pos || !c->len) return LETHE_ERR_INVALID_ARG;
+    if (c->n_layers < 1 || c->batch < 1 || c->n_kv_heads < 1 || c->capacity < 1) return LETHE_ERR_INVALID_ARG;
+    if (c->head_dim != 64 && c->head_dim != 128) return LETHE_ERR_UNSUPPORTED;
+    if (c->dtype != LETHE_F32 && c->dtype != LETHE_BF16) return LETHE_ERR_INVALID_ARG;
+    if (c->layout != LETHE_CONTIG && c->layout != LETHE_PAGED) return LETHE_ERR_INVALID_ARG;
+    if (c->layout == LETHE_PAGED && (!c->page_table || c->page_tokens < 1 || c->n_pages < 1)) return LETHE_ERR_INVALID_ARG;
+    if (recent < 0 || sink < 0 || (keep_idx && max_k < 1)) return LETHE_ERR_INVALID_ARG;
+    if ((((uintptr_t)c->k) | ((uintptr_t)c->v)) & 15) return LETHE_ERR_INVALID_ARG;
+
+    CacheView v;
+    v.k = c->k; v.v = c->v; v.rel = c->rel; v.pos = c->pos; v.len = c->len; v.page_table = c->page_table;
+    v.n_pages = c->n_pages;
+    v.L = c->n_layers; v.B = c->batch; v.Hkv = c->n_kv_heads; v.D = c->head_dim;
+    v.elt_bytes = c->dtype == LETHE_BF16 ? 2 : 4;
+    v.capacity = c->capacity;
+    v.page_tokens = c->layout == LETHE_PAGED ? c->page_tokens : 1;
+    v.paged = c->layout == LETHE_PAGED;
+    const long long cap_tokens = (long long)c->capacity * v.page_tokens;
+    const long long items = (long long)v.L * v.B * v.Hkv;
+    if (cap_tokens > 0x7fffffffLL || items > 0x7fffffffLL) return LETHE_ERR_TOO_LARGE;
+    v.cap_tokens = (int)cap_tokens;
+    // one list entry per (item, slot): refuse what the fixed scratch cannot hold
+    if (items * cap_tokens > (long long)LETHE_STATIC_PRUNE_MAX_ENTRIES) return LETHE_ERR_TOO_LARGE;
+
+    int32_t* scratch = nullptr;
+    if (static_prune_scratch(&scratch) != cudaSuccess) return LETHE_ERR_CUDA;
+    int32_t* status = scratch;        // {code, item}: must start at zero for this call
+    int32_t* lists = scratch + 64;    // fully written before it is read: no clearing needed
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(status, 0, 2 * sizeof(int32_t), s) != cudaSuccess) return LETHE_ERR_CUDA;
+    // smem_tokens = 0: every item keeps its source list in the global scratch and re-reads its keys from rel
+    rasr_prune_kernel<<<(unsigned)items, kPruneThreads, 0, s>>>(v, budgets, recent, sink, keep_idx, keep_idx ? max_k : 0,
+                                                               0, lists, status);
+    if (cudaGetLastError() != cudaSuccess) return LETHE_ERR_CUDA;
+    if (status_out &&
+        cudaMemcpyAsync(status_out, status, 2 * sizeof(int32_t), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+        return LETHE_ERR_CUDA;
+    return LETHE_OK;
+}
