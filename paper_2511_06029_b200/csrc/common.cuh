@@ -58,9 +58,23 @@ __device__ __forceinline__ void tl_mark(const AttendArgs& a, int slot) {
         }
     }
 }
+__device__ __forceinline__ void tl_mark_at(const AttendArgs& a, int row, int slot) {
+    if (a.timeline && threadIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+        a.timeline[(size_t)row * 8 + slot] = t;
+        if (slot == 0) {
+            unsigned sm;
+            asm volatile("mov.u32 %0, %smid;" : "=r"(sm));
+            a.timeline[(size_t)row * 8 + 7] = sm;
+        }
+    }
+}
 #define TL_MARK(a, slot) tl_mark(a, slot)
+#define TL_MARK_AT(a, row, slot) tl_mark_at(a, row, slot)
 #else
 #define TL_MARK(a, slot)
+#define TL_MARK_AT(a, row, slot)
 #endif
 
 // Cache state as the prune-round kernels see it.
