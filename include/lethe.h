@@ -97,8 +97,9 @@ lethe_status lethe_poll_status(lethe_ctx *ctx, void *stream, int32_t *info);
 
 /* Tuning knobs (HOST values).
  * variant: 0 = automatic; 1 = CUDA-core kernel; 2..7 = clustered tensor-core (mma) kernel with (warps per
- * CTA, pipeline stages per warp) = (4,3) (8,3) (4,2) (8,2) (4,4) (2,4); 8..13 = persistent tensor-core
- * kernel (one CTA per SM, dynamic item queue, cross-item prefetch) with (8,2) (6,3) (10,2) (8,3) (7,3) (5,4).
+ * CTA, pipeline stages per warp) = (4,3) (8,3) (4,2) (8,2) (4,4) (2,4); 8..15 = persistent tensor-core
+ * kernel (one CTA per SM, dynamic item queue, cross-item prefetch) with (8,2) (6,3) (10,2) (8,3) (7,3) (5,4)
+ * (6,2) (5,3).
  * Tensor-core variants need a bf16 cache (and 16-token pages when paged).
  * splits: 0 = automatic, else CTAs per item (1, 2, 4, 8 or 16; they form one thread-block cluster); the
  * persistent variants take 0 or 1.

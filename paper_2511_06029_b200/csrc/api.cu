@@ -227,7 +227,7 @@ lethe_status lethe_debug_set_timeline(lethe_ctx* ctx, unsigned long long* buf) {
 
 lethe_status lethe_set_tuning(lethe_ctx* ctx, int variant, int splits) {
     if (!ctx) return LETHE_ERR_INVALID_ARG;
-    if (variant < 0 || variant > 13) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..13");
+    if (variant < 0 || variant > 15) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..15");
     if (!(splits == 0 || splits == 1 || splits == 2 || splits == 4 || splits == 8 || splits == 16))
         return fail(ctx, LETHE_ERR_INVALID_ARG, "splits must be 0, 1, 2, 4, 8 or 16");
     ctx->variant = variant;
@@ -285,9 +285,16 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
             return stream_smem_bytes(c->head_dim, shape, cap_groups * kGroupTokens, a.GP) <= ctx->max_smem;
         };
         if (!mma_ok) variant = 1;
-        else if (a.n_items >= 2 * ctx->sm_count && ctx->splits <= 1 && stream_fits(4)) variant = 12;  // 7 warps x 3 stages
-        else if (a.n_items >= 2 * ctx->sm_count && ctx->splits <= 1 && stream_fits(1)) variant = 9;   // 6 warps x 3 stages
-        else if (a.n_items >= 2 * ctx->sm_count && ctx->splits <= 1 && stream_fits(0)) variant = 8;   // 8 warps x 2 stages
+        else if (a.n_items >= 2 * ctx->sm_count && ctx->splits <= 1) {
+            // persistent kernel: deepest pipeline whose stages + logit buffer fit in shared memory
+            static const int pref[] = {4, 1, 0, 7, 6};  // (7,3) (6,3) (8,2) (5,3) (6,2)
+            variant = 4;
+            for (int shape : pref)
+                if (stream_fits(shape)) {
+                    variant = 8 + shape;
+                    break;
+                }
+        }
         else variant = 4;
     }
     if (variant >= 2 && !mma_ok) return fail(ctx, LETHE_ERR_UNSUPPORTED, "tensor-core variants need bf16 and 16-token pages");

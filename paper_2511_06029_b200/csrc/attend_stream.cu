@@ -297,11 +297,11 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
                 wo[(2 * tq + 1) * D + 16 * mt + gq + 8] = o[mt][3];
             }
         }
+        int t_new = a.n_items;
+        if (tid == 0 && !drew_fail)  // ticket of the item after next; its latency hides behind the barrier wait
+            t_new = (int)atomicAdd(&sched[0], 1u);
         __syncthreads();  // B1: every warp's partials are in shared memory
         TL_MARK_AT(a, cur.item - a.layer_begin * a.B * a.Hkv, 2);
-        int t_new = a.n_items;
-        if (tid == 0 && !drew_fail)  // ticket of the item after next; its latency hides behind the epilogue
-            t_new = (int)atomicAdd(&sched[0], 1u);
         if (tid < kMaxGroup) {
             const int h = tid;
             float m = -INFINITY;
@@ -414,7 +414,8 @@ static cudaError_t launch_stream_t(const AttendArgs& a, int grid, cudaStream_t s
 }
 
 // Shapes of the persistent kernel: (warps per CTA, stages per warp).
-#define LETHE_STREAM_SHAPES(X, D) X(0, D, 8, 2) X(1, D, 6, 3) X(2, D, 10, 2) X(3, D, 8, 3) X(4, D, 7, 3) X(5, D, 5, 4)
+#define LETHE_STREAM_SHAPES(X, D) X(0, D, 8, 2) X(1, D, 6, 3) X(2, D, 10, 2) X(3, D, 8, 3) X(4, D, 7, 3) X(5, D, 5, 4) X(6, D, 6, 2) \
+        X(7, D, 5, 3)
 
 size_t stream_smem_bytes(int D, int shape, int chunk_tokens, int GP) {
 #define X(id, DD, NW, NS) \

@@ -318,3 +318,49 @@ def test_model_shaped_workloads_call_by_call(ctx, name, batch, steps):
         if (step + 1) % w.prune_interval == 0:
             bud, _ = _prune_both(ctx, oc, gc, T, w.k_min, w.recent, w.sink, cap)
             assert int(bud.sum()) == int(T.sum())
+
+
+def test_long_reasoning_shape_call_by_call(ctx):
+    """Long-reasoning geometry (Llama shape, budget 2048 per layer): one sequence, all 32 layers, items above
+    2000 tokens, default tuning; decode steps and a prune round."""
+    oracle.set_threads(min(8, oracle.max_threads()))
+    try:
+        w = synth.shrink(synth.WORKLOADS["longreason"], batch=1, prune_interval=3)
+        n0, cap = 2100, 2128
+        oc = cache_from_state(w, synth.initial_kv(w, n0, cap), cap)
+        gc = to_device(oc)
+        scale = synth.layer_scales(w)
+        T = torch.full((1,), w.n_layers * 2048, dtype=torch.int64)
+        for step in range(4):
+            x = synth.step_inputs(w, step)
+            _step(ctx, oc, gc, x["q"], x["k_new"], x["v_new"], x["token_pos"], scale, w.gamma, 0, w.n_layers, want_lse=False)
+            if step == 2:
+                _prune_both(ctx, oc, gc, T, w.k_min, w.recent, w.sink, cap)
+    finally:
+        oracle.set_threads(1)
+
+
+def test_ragged_paged_long_items(ctx):
+    """Ragged-batch geometry (Qwen shape, 16-token pages, shuffled page tables) with the shortest and the longest
+    sequence of the workload (1024 and 32768 tokens): decode steps, then a prune to a quarter of the length,
+    then decode steps on the pruned cache.  Long items take the clustered kernel (16 CTAs per item)."""
+    oracle.set_threads(min(8, oracle.max_threads()))
+    try:
+        w = synth.shrink(synth.WORKLOADS["ragged"], n_layers=2, batch=3, prompt_len=32768)
+        lens = torch.tensor([1024, 32768, 9001])
+        cap = 33280                                    # 2080 pages per item
+        st_c = synth.initial_kv(w, 32768, cap)
+        st_c["len"][:] = lens[None, :, None].to(torch.int32)
+        st_p = synth.to_paged(st_c, 16, seed=5, spare_pages=11)
+        del st_c
+        oc = cache_from_state(w, st_p, cap)
+        gc = to_device(oc)
+        scale = synth.layer_scales(w)
+        T = (w.n_layers * (lens // 4)).to(torch.int64)
+        for step in range(4):
+            x = synth.step_inputs(w, step)
+            _step(ctx, oc, gc, x["q"], x["k_new"], x["v_new"], x["token_pos"], scale, w.gamma, 0, w.n_layers, want_lse=False)
+            if step == 1:
+                _prune_both(ctx, oc, gc, T, w.k_min, w.recent, w.sink, 9000)
+    finally:
+        oracle.set_threads(1)
