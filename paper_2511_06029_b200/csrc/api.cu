@@ -279,23 +279,29 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
     const bool mma_ok = c->dtype == LETHE_BF16 && (!paged || c->page_tokens == kGroupTokens);
     const int cap_groups = (a.cap_tokens + kGroupTokens - 1) / kGroupTokens;
     int variant = ctx->variant;
+    // persistent kernel: logit-buffer tokens that fit beside a shape's stages (the rest overflows to scratch)
+    auto stream_chunk = [&](int shape) -> int {
+        const size_t fixed = stream_smem_bytes(c->head_dim, shape, 0, a.GP);
+        if (fixed >= ctx->max_smem) return 0;
+        const size_t tokens = (ctx->max_smem - fixed) / ((size_t)a.GP * 4);
+        const int fit = (int)(tokens / kGroupTokens) * kGroupTokens;
+        return fit < cap_groups * kGroupTokens ? fit : cap_groups * kGroupTokens;
+    };
     if (variant == 0) {
         // enough items to give every SM several: the persistent kernel; few long items: the clustered one
-        auto stream_fits = [&](int shape) {
-            return stream_smem_bytes(c->head_dim, shape, cap_groups * kGroupTokens, a.GP) <= ctx->max_smem;
-        };
         if (!mma_ok) variant = 1;
         else if (a.n_items >= 2 * ctx->sm_count && ctx->splits <= 1) {
-            // persistent kernel: deepest pipeline whose stages + logit buffer fit in shared memory
+            // deepest pipeline that still keeps the whole logit buffer on chip; failing that, the one that
+            // keeps the most of it there
             static const int pref[] = {4, 1, 0, 7, 6};  // (7,3) (6,3) (8,2) (5,3) (6,2)
-            variant = 4;
+            variant = 0;
             for (int shape : pref)
-                if (stream_fits(shape)) {
+                if (stream_chunk(shape) == cap_groups * kGroupTokens) {
                     variant = 8 + shape;
                     break;
                 }
-        }
-        else variant = 4;
+            if (variant == 0) variant = stream_chunk(6) >= 512 ? 8 + 6 : 4;
+        } else variant = 4;
     }
     if (variant >= 2 && !mma_ok) return fail(ctx, LETHE_ERR_UNSUPPORTED, "tensor-core variants need bf16 and 16-token pages");
 
@@ -303,10 +309,17 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
     if (variant >= 8) {  // persistent: one CTA per SM walks all items
         if (ctx->splits > 1) return fail(ctx, LETHE_ERR_INVALID_ARG, "the persistent variant does not split items");
         a.splits = 1;
-        a.chunk_tokens = cap_groups * kGroupTokens;
-        if (stream_smem_bytes(c->head_dim, variant - 8, a.chunk_tokens, a.GP) > ctx->max_smem)
-            return fail(ctx, LETHE_ERR_UNSUPPORTED, "capacity too large for the on-chip logit buffer of the persistent variant");
+        a.chunk_tokens = stream_chunk(variant - 8);
+        if (a.chunk_tokens < kGroupTokens)
+            return fail(ctx, LETHE_ERR_UNSUPPORTED, "no shared memory left for the logit buffer of this persistent shape");
         const int grid = a.n_items < ctx->sm_count ? a.n_items : ctx->sm_count;
+        if (a.chunk_tokens < cap_groups * kGroupTokens) {  // overflow of the logit buffer: one slice per CTA
+            a.spill_tokens = cap_groups * kGroupTokens - a.chunk_tokens;
+            const size_t need = (size_t)grid * a.spill_tokens * a.GP * sizeof(float);
+            st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "logit overflow scratch");
+            if (st != LETHE_OK) return st;
+            a.spill = (float*)ctx->scratch;
+        }
         e = launch_attend_stream(a, c->head_dim, variant - 8, paged, grid, (cudaStream_t)stream);
     } else {
         // CTAs per item: the smallest cluster whose logit buffer fits, grown until the grid covers the SMs twice.

@@ -73,6 +73,12 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
     float* wo_all = reinterpret_cast<float*>(smem_raw + (size_t)NW * WARP_BYTES);
     EpilogueSmem& es = *reinterpret_cast<EpilogueSmem*>(wo_all + (size_t)NW * wo_stride);
     float* lg = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(&es) + sizeof(EpilogueSmem));
+    // Logits of tokens beyond the shared-memory buffer overflow to this CTA's slice of global scratch.
+    const int chunk = a.chunk_tokens;
+    float* spill = a.spill ? a.spill + (size_t)blockIdx.x * a.spill_tokens * GP : nullptr;
+    auto lg_row = [&](int tok) -> float* {
+        return tok < chunk ? lg + (size_t)tok * GP : spill + (size_t)(tok - chunk) * GP;
+    };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int gq = lane >> 2, tq = lane & 3;
@@ -229,8 +235,8 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
             const float s10 = (tokB < cur.n) ? (ca[2] + cb[2]) * sl2 : -INFINITY;
             const float s11 = (tokB < cur.n) ? (ca[3] + cb[3]) * sl2 : -INFINITY;
             if (2 * tq < GP) {
-                *reinterpret_cast<float2*>(lg + (size_t)tokA * GP + 2 * tq) = make_float2(s00, s01);
-                *reinterpret_cast<float2*>(lg + (size_t)tokB * GP + 2 * tq) = make_float2(s10, s11);
+                *reinterpret_cast<float2*>(lg_row(tokA) + 2 * tq) = make_float2(s00, s01);
+                *reinterpret_cast<float2*>(lg_row(tokB) + 2 * tq) = make_float2(s10, s11);
             }
             float mx0 = fmaxf(s00, s10), mx1 = fmaxf(s01, s11);
 #pragma unroll
@@ -338,7 +344,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
             }
             float* relp = a.rel + (size_t)cur.item * a.cap_tokens;
             auto mass_of = [&](int j) {
-                const float* row = lg + (size_t)j * GP;
+                const float* row = lg_row(j);
                 float mass = 0.f;
 #pragma unroll
                 for (int h = 0; h < kMaxGroup; h += 2) {

@@ -32,6 +32,8 @@ struct AttendArgs {
     float* lse;
     int32_t* status;      // device status word: {code, item}
     unsigned int* sched;  // persistent kernel only: {next ticket, CTAs finished}, zero between launches
+    float* spill;         // persistent kernel only: global overflow of the logit buffer, [grid][spill_tokens][GP]
+    int spill_tokens;     // tokens per CTA the overflow can hold (0 = the shared-memory buffer covers cap_tokens)
     long long n_pages;
     int B, Hq, Hkv, G, GP;  // GP = G rounded up to even: row pitch of the logit buffer
     int capacity, cap_tokens, page_tokens;

@@ -364,3 +364,26 @@ def test_ragged_paged_long_items(ctx):
                 _prune_both(ctx, oc, gc, T, w.k_min, w.recent, w.sink, 9000)
     finally:
         oracle.set_threads(1)
+
+
+@pytest.mark.parametrize("variant,Hq,Hkv,cap", [(9, 28, 4, 3000), (12, 16, 4, 4200), (14, 28, 4, 6000)])
+def test_persistent_logit_overflow(ctx, variant, Hq, Hkv, cap):
+    """Items longer than the on-chip logit buffer of the persistent kernel: the logits of the tail tokens
+    overflow to global scratch and the relevance update must still be exact."""
+    oracle.set_threads(min(8, oracle.max_threads()))
+    try:
+        L, B, D = 2, 4, 128
+        lens = _lens(L, B, Hkv, cap - 4, seed=cap, special=(cap - 5, cap - 300, 17, 1800, 2048, 1))
+        oc = random_cache(L, B, Hq, Hkv, D, cap, lens, dtype=torch.bfloat16, seed=variant, rel_init="rand")
+        gc = to_device(oc)
+        ctx.set_tuning(variant, 0)
+        g = torch.Generator().manual_seed(8)
+        scale = torch.tensor([0.09, 0.05], dtype=torch.float32)
+        for step in range(3):
+            q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+            kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            _step(ctx, oc, gc, q, kn, vn, torch.arange(B, dtype=torch.int32) + 10 * step, scale, 0.9, 0, L)
+    finally:
+        ctx.set_tuning(0, 0)
+        oracle.set_threads(1)
