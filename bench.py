@@ -215,6 +215,43 @@ def timed_loop(r: Runner, steps: int, host: bool):
     return total_ms, attend_ms, prune_ms, th
 
 
+def per_layer_mode(r: Runner, steps: int):
+    """The same decode step issued the way a real model must (layer l+1's query does not exist before layer l
+    is done): one lethe_decode_attend launch per layer, the 32 launches replayed from a CUDA graph.  Returns
+    (ms per step, token-heads per step)."""
+    w, dev = r.w, r.dev
+    q, kn, vn = r.pool[0]
+
+    def one_step():
+        for l in range(w.n_layers):
+            r.ctx.decode_attend(r.cache, l, l + 1, q[l:l + 1], kn[l:l + 1], vn[l:l + 1], r.token_pos, r.scale, w.gamma,
+                                r.out[l:l + 1], None, scale_c=r.scale_c)
+
+    side = torch.cuda.Stream(dev)
+    side.wait_stream(torch.cuda.current_stream(dev))
+    with torch.cuda.stream(side):
+        one_step()                                   # first use of this kernel outside capture
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            one_step()
+    torch.cuda.current_stream(dev).wait_stream(side)
+    torch.cuda.synchronize(dev)
+    th0 = int(r.cache.len.sum().item())
+    items = r.cache.len.numel()
+    a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+    for _ in range(3):
+        graph.replay()
+    a.record()
+    for _ in range(steps):
+        graph.replay()
+    b.record()
+    torch.cuda.synchronize(dev)
+    ms = a.elapsed_time(b) / steps
+    th = th0 + items * (3 + (steps + 1) / 2.0)       # mean length over the timed replays
+    return ms, th
+
+
 def cpu_baseline(w, r: Runner | None, seconds=12.0, layers=4, seqs=4):
     """The oracle, as it stands, on a bounded sample of the workload on the host cores."""
     import oracle
@@ -296,6 +333,7 @@ def main():
                     help="untimed prune intervals run before warm-up so that lengths reach their budgets")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-per-layer", action="store_true")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
 
@@ -358,6 +396,15 @@ def main():
         barrier()
         r.check()
     clocks = sampler.stop() if sampler else None
+    per_layer = None
+    if not args.no_per_layer and world == 1:
+        pl_steps = min(32, max(4, w.prune_interval - (r.step_no % w.prune_interval) - 8))
+        ms_pl, th_pl = per_layer_mode(r, pl_steps)
+        r.check()
+        per_layer = {"ms_per_step": ms_pl, "token_heads_per_step": th_pl, "value": th_pl / (ms_pl * 1e-3),
+                     "algorithmic_GBs": th_pl * BYTES_PER_TOKEN_HEAD / (ms_pl * 1e-3) / 1e9,
+                     "mode": f"{w.n_layers} launches per step (one per layer), replayed from a CUDA graph, "
+                             f"{pl_steps} steps; not part of `value`"}
 
     e_ms = e_total_ms if not args.no_e2e else 0.0
     e_u = float(sum(e_th)) if not args.no_e2e else 0.0
@@ -382,7 +429,8 @@ def main():
                 "prune_rounds_timed": len(prune_ms),
                 "prune_round_ms": (sum(prune_ms) / len(prune_ms)) if prune_ms else None,
                 "attend_ms_per_step": avg_attend_ms,
-                "attend_ms_median": statistics.median(attend_ms)}),
+                "attend_ms_median": statistics.median(attend_ms),
+                "per_layer_launch": per_layer}),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": f"of {which}", "frac_of_8TBs_nominal": achieved / 8000.0,
                          "kernel": "attend (dominant kernel; one launch per step)",

@@ -55,7 +55,7 @@ __device__ __forceinline__ int opaque(int x) {
     return x;
 }
 
-template <int D, int NW, int NS, bool PAGED>
+template <int D, int NW, int NS, bool PAGED, bool SPILL>
 __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_constant__ AttendArgs a) {
     using T = __nv_bfloat16;
     constexpr int NT = NW * 32;
@@ -74,10 +74,11 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
     EpilogueSmem& es = *reinterpret_cast<EpilogueSmem*>(wo_all + (size_t)NW * wo_stride);
     float* lg = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(&es) + sizeof(EpilogueSmem));
     // Logits of tokens beyond the shared-memory buffer overflow to this CTA's slice of global scratch.
-    const int chunk = a.chunk_tokens;
-    float* spill = a.spill ? a.spill + (size_t)blockIdx.x * a.spill_tokens * GP : nullptr;
+    // (SPILL is a compile-time switch so that launches whose buffer covers the capacity pay nothing for it.)
+    const int chunk = SPILL ? a.chunk_tokens : 0x7fffffff;
+    float* spill = SPILL ? a.spill + (size_t)blockIdx.x * a.spill_tokens * GP : nullptr;
     auto lg_row = [&](int tok) -> float* {
-        return tok < chunk ? lg + (size_t)tok * GP : spill + (size_t)(tok - chunk) * GP;
+        return (!SPILL || tok < chunk) ? lg + (size_t)tok * GP : spill + (size_t)(tok - chunk) * GP;
     };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -235,8 +236,13 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
             const float s10 = (tokB < cur.n) ? (ca[2] + cb[2]) * sl2 : -INFINITY;
             const float s11 = (tokB < cur.n) ? (ca[3] + cb[3]) * sl2 : -INFINITY;
             if (2 * tq < GP) {
-                *reinterpret_cast<float2*>(lg_row(tokA) + 2 * tq) = make_float2(s00, s01);
-                *reinterpret_cast<float2*>(lg_row(tokB) + 2 * tq) = make_float2(s10, s11);
+                if (!SPILL || tokB < chunk) {  // common case: both rows of this thread live in shared memory
+                    *reinterpret_cast<float2*>(lg + (size_t)tokA * GP + 2 * tq) = make_float2(s00, s01);
+                    *reinterpret_cast<float2*>(lg + (size_t)tokB * GP + 2 * tq) = make_float2(s10, s11);
+                } else {
+                    *reinterpret_cast<float2*>(lg_row(tokA) + 2 * tq) = make_float2(s00, s01);
+                    *reinterpret_cast<float2*>(lg_row(tokB) + 2 * tq) = make_float2(s10, s11);
+                }
             }
             float mx0 = fmaxf(s00, s10), mx1 = fmaxf(s01, s11);
 #pragma unroll
@@ -344,7 +350,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
             }
             float* relp = a.rel + (size_t)cur.item * a.cap_tokens;
             auto mass_of = [&](int j) {
-                const float* row = lg_row(j);
+                const float* row = (!SPILL || j < chunk) ? lg + (size_t)j * GP : spill + (size_t)(j - chunk) * GP;
                 float mass = 0.f;
 #pragma unroll
                 for (int h = 0; h < kMaxGroup; h += 2) {
@@ -409,14 +415,21 @@ static size_t stream_smem(int chunk_tokens, int GP) {
            (size_t)chunk_tokens * GP * 4;
 }
 
-template <int D, int NW, int NS, bool PAGED>
+template <int D, int NW, int NS, bool PAGED, bool SPILL>
 static cudaError_t launch_stream_t(const AttendArgs& a, int grid, cudaStream_t stream) {
-    auto kern = attend_stream_kernel<D, NW, NS, PAGED>;
+    auto kern = attend_stream_kernel<D, NW, NS, PAGED, SPILL>;
     const size_t smem = stream_smem<D, NW, NS>(a.chunk_tokens, a.GP);
     cudaError_t e = prepare_kernel((const void*)kern, smem);
     if (e != cudaSuccess) return e;
     kern<<<grid, NW * 32, smem, stream>>>(a);
     return cudaGetLastError();
+}
+
+template <int D, int NW, int NS>
+static cudaError_t dispatch_stream(const AttendArgs& a, bool paged, int grid, cudaStream_t stream) {
+    const bool spill = a.spill != nullptr;
+    if (paged) return spill ? launch_stream_t<D, NW, NS, true, true>(a, grid, stream) : launch_stream_t<D, NW, NS, true, false>(a, grid, stream);
+    return spill ? launch_stream_t<D, NW, NS, false, true>(a, grid, stream) : launch_stream_t<D, NW, NS, false, false>(a, grid, stream);
 }
 
 // Shapes of the persistent kernel: (warps per CTA, stages per warp).
@@ -435,7 +448,7 @@ size_t stream_smem_bytes(int D, int shape, int chunk_tokens, int GP) {
 cudaError_t launch_attend_stream(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream) {
 #define X(id, DD, NW, NS)                                                                                   \
     if (shape == id && D == DD)                                                                             \
-        return paged ? launch_stream_t<DD, NW, NS, true>(a, grid, stream) : launch_stream_t<DD, NW, NS, false>(a, grid, stream);
+        return dispatch_stream<DD, NW, NS>(a, paged, grid, stream);
     LETHE_STREAM_SHAPES(X, 128)
     LETHE_STREAM_SHAPES(X, 64)
 #undef X
