@@ -33,9 +33,10 @@ METRIC = "kv_token_heads_attended_per_s"
 UNIT = "token-heads/s"
 BYTES_PER_TOKEN_HEAD = 520          # K row 256 B + V row 256 B + relevance read 4 B + write 4 B (D=128, bf16)
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes per token-head of the attend kernel from the ncu capture summarised under profiles/ (None until
-# a capture exists for the kernel in use).
-NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = None
+# DRAM bytes (read + write) per token-head of the default attend kernel, from the ncu capture summarised in
+# profiles/attend_stream_w7s3_llama8b.md (1.031 GB per launch of 1 970 008 token-heads; traffic grows in
+# proportion to the token-heads of a launch, so it is scaled to the launch bench.py times).
+NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = 523.5
 
 
 def measured_peak():
