@@ -253,13 +253,14 @@ def per_layer_mode(r: Runner, steps: int):
     return ms, th
 
 
-def cpu_baseline(w, r: Runner | None, seconds=12.0, layers=4, seqs=4):
+def cpu_baseline(w, r: Runner | None, seconds=12.0, layers=8, seqs=4):
     """The oracle, as it stands, on a bounded sample of the workload on the host cores."""
     import oracle
     threads = oracle.max_threads()
     oracle.set_threads(threads)
     ws = synth.shrink(w, n_layers=layers, batch=seqs)
-    cap = w.mean_budget + 256
+    max_steps = 512
+    cap = w.mean_budget + max_steps + 8
     st = synth.initial_kv(ws, w.mean_budget, cap)
     oc = oracle.OracleCache(ws.n_layers, seqs, ws.n_q_heads, ws.n_kv_heads, ws.head_dim, cap, st["k"], st["v"],
                             st["rel"], st["pos"], st["len"])
@@ -277,7 +278,7 @@ def cpu_baseline(w, r: Runner | None, seconds=12.0, layers=4, seqs=4):
         steps += 1
         if steps == 1:
             first = dt
-        if time.perf_counter() - t0 > seconds or steps >= 2000:
+        if time.perf_counter() - t0 > seconds or steps >= max_steps:
             break
     attend_s = time.perf_counter() - t0
     # one prune round on the sample, amortised like the GPU loop
@@ -361,16 +362,30 @@ def main():
     if dist is not None:
         dist.barrier()
 
-    capacity = args.capacity or (2 * w.mean_budget)
-    r = Runner(w, dev, rank, capacity, args.variant, args.splits)
-    # state preparation (untimed): a few full prune intervals so that relevance, sparsity-driven budgets and
-    # lengths are those of a steady-state trajectory (dense layers need several rounds to grow to their budget)
-    for _ in range(max(1, args.prep_rounds)):
-        for _ in range(w.prune_interval):
-            r.decode()
-        r.prune()
-    r.check()
-    max_budget = int(r.budgets.max().item())
+    def prepare(capacity):
+        """Runner brought to steady state (untimed): a few full prune intervals so that relevance, sparsity-driven
+        budgets and lengths are those of a long trajectory (dense layers need several rounds to grow to their
+        budget).  Returns the runner and the largest layer budget."""
+        r = Runner(w, dev, rank, capacity, args.variant, args.splits)
+        for _ in range(max(1, args.prep_rounds)):
+            for _ in range(w.prune_interval):
+                r.decode()
+            r.prune()
+        r.check()
+        return r, int(r.budgets.max().item())
+
+    # Capacity = largest layer budget + prune interval (+ slack), as a serving system would size it.  The budgets
+    # follow from the measured sparsity, so a pilot run at a generous capacity finds them first.
+    if args.capacity:
+        capacity = args.capacity
+        r, max_budget = prepare(capacity)
+    else:
+        pilot, max_budget = prepare(3 * w.mean_budget)
+        pilot.ctx.close()
+        del pilot
+        torch.cuda.empty_cache()
+        capacity = -(-(max_budget + w.prune_interval + 32) // 64) * 64
+        r, max_budget = prepare(capacity)
     if max_budget + w.prune_interval > capacity:
         raise SystemExit(f"capacity {capacity} too small for budget {max_budget} + interval {w.prune_interval}")
     for _ in range(max(args.warmup, 3)):

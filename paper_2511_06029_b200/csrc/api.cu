@@ -1,6 +1,7 @@
 // C ABI of the Lethe hot path: argument checking, launch geometry, context-owned scratch and status word.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -14,6 +15,8 @@ cudaError_t launch_attend_mma(const AttendArgs& a, int D, int shape, bool paged,
 size_t mma_smem_bytes(int D, int shape, int chunk_tokens, int GP);
 cudaError_t launch_attend_stream(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream);
 size_t stream_smem_bytes(int D, int shape, int chunk_tokens, int GP);
+cudaError_t launch_attend_async(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream);
+size_t async_smem_bytes(int D, int shape, int chunk_tokens, int GP);
 cudaError_t launch_sparsity(const CacheView& c, float* sparsity, cudaStream_t stream);
 cudaError_t launch_budgets(int L, int B, const float* sparsity, const long long* total, int k_min, int32_t* budgets,
                            int32_t* status, cudaStream_t stream);
@@ -227,7 +230,7 @@ lethe_status lethe_debug_set_timeline(lethe_ctx* ctx, unsigned long long* buf) {
 
 lethe_status lethe_set_tuning(lethe_ctx* ctx, int variant, int splits) {
     if (!ctx) return LETHE_ERR_INVALID_ARG;
-    if (variant < 0 || variant > 15) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..15");
+    if (variant < 0 || variant > 23) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..23");
     if (!(splits == 0 || splits == 1 || splits == 2 || splits == 4 || splits == 8 || splits == 16))
         return fail(ctx, LETHE_ERR_INVALID_ARG, "splits must be 0, 1, 2, 4, 8 or 16");
     ctx->variant = variant;
@@ -291,22 +294,41 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         // enough items to give every SM several: the persistent kernel; few long items: the clustered one
         if (!mma_ok) variant = 1;
         else if (a.n_items >= 2 * ctx->sm_count && ctx->splits <= 1) {
-            // deepest pipeline that still keeps the whole logit buffer on chip; failing that, the one that
-            // keeps the most of it there
-            static const int pref[] = {4, 1, 0, 7, 6};  // (7,3) (6,3) (8,2) (5,3) (6,2)
+            // Persistent kernels, best measured first, taking the first whose logit buffer(s) cover the
+            // capacity on chip: asynchronous epilogue (6,3) (5,3) (4,4), then the synchronous (7,3) (6,3) (8,2);
+            // if none does, the asynchronous (5,3) with the tail of long items overflowing to scratch.
+            const int cap_pad = cap_groups * kGroupTokens;
+            auto async_fits = [&](int shape) { return async_smem_bytes(c->head_dim, shape, cap_pad, a.GP) <= ctx->max_smem; };
             variant = 0;
-            for (int shape : pref)
-                if (stream_chunk(shape) == cap_groups * kGroupTokens) {
-                    variant = 8 + shape;
-                    break;
-                }
-            if (variant == 0) variant = stream_chunk(6) >= 512 ? 8 + 6 : 4;
+            for (int shape : {2, 3, 5})
+                if (variant == 0 && async_fits(shape)) variant = 16 + shape;
+            for (int shape : {4, 1, 0})
+                if (variant == 0 && stream_chunk(shape) == cap_pad) variant = 8 + shape;
+            if (variant == 0) variant = 16 + 3;
         } else variant = 4;
     }
     if (variant >= 2 && !mma_ok) return fail(ctx, LETHE_ERR_UNSUPPORTED, "tensor-core variants need bf16 and 16-token pages");
 
     cudaError_t e;
-    if (variant >= 8) {  // persistent: one CTA per SM walks all items
+    if (variant >= 16) {  // persistent, asynchronous epilogue: both logit buffers (item parity) share what is left
+        if (ctx->splits > 1) return fail(ctx, LETHE_ERR_INVALID_ARG, "the persistent variants do not split items");
+        a.splits = 1;
+        const size_t fixed = async_smem_bytes(c->head_dim, variant - 16, 0, a.GP);
+        int fit = 0;
+        if (fixed < ctx->max_smem) fit = (int)((ctx->max_smem - fixed) / ((size_t)2 * a.GP * 4) / kGroupTokens) * kGroupTokens;
+        a.chunk_tokens = fit < cap_groups * kGroupTokens ? fit : cap_groups * kGroupTokens;
+        if (a.chunk_tokens < kGroupTokens)
+            return fail(ctx, LETHE_ERR_UNSUPPORTED, "no shared memory left for the logit buffers of this persistent shape");
+        const int grid = a.n_items < ctx->sm_count ? a.n_items : ctx->sm_count;
+        if (a.chunk_tokens < cap_groups * kGroupTokens || getenv("LETHE_DEBUG_FORCE_SPILL")) {
+            a.spill_tokens = cap_groups * kGroupTokens - a.chunk_tokens + 16;
+            const size_t need = (size_t)grid * 2 * a.spill_tokens * a.GP * sizeof(float);
+            st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "logit overflow scratch");
+            if (st != LETHE_OK) return st;
+            a.spill = (float*)ctx->scratch;
+        }
+        e = launch_attend_async(a, c->head_dim, variant - 16, paged, grid, (cudaStream_t)stream);
+    } else if (variant >= 8) {  // persistent: one CTA per SM walks all items
         if (ctx->splits > 1) return fail(ctx, LETHE_ERR_INVALID_ARG, "the persistent variant does not split items");
         a.splits = 1;
         a.chunk_tokens = stream_chunk(variant - 8);

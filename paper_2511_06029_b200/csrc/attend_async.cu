@@ -1,0 +1,551 @@
+// Persistent tensor-core decode-attend kernel with an asynchronous epilogue (bf16, D in {64, 128}, G <= 8).
+//
+// Same per-group arithmetic and the same work queue as attend_stream.cu, but the CTA is warp-specialised:
+//   * NWS streaming warps never stop at a CTA-wide barrier.  When a warp has consumed its groups of item i it
+//     parks its partial (max, sum, O) in the item's parity buffer, signals an mbarrier and goes straight on to
+//     item i+1, whose first groups its pipeline has already prefetched;
+//   * 2 epilogue warps wait for that mbarrier, merge the partials, write out / lse, apply Eq. 5 to rel with the
+//     exact normaliser, store len, draw the ticket of the item after next (and read its len), and hand the
+//     parity buffer back through a second mbarrier.
+// The logit buffer, the partial-output buffer and the item descriptor are double-buffered by item parity, so the
+// epilogue of item i runs entirely under the HBM stream of item i+1.  Every mbarrier wait is bounded: if it
+// runs out, the CTA records LETHE_ERR_TIMEOUT, drains its copies and returns.
+#include "common.cuh"
+#include "mma_utils.cuh"
+
+#include <type_traits>
+
+namespace lethe {
+
+constexpr int kEpilogueWarps = 2;
+constexpr int kWaitLimit = 200000;  // polls of a blocking try_wait before giving up
+
+struct AsyncHeader {
+    unsigned long long full[2];   // streaming warps -> epilogue: item's partials are complete
+    unsigned long long empty[2];  // epilogue -> streaming warps: parity buffers are free, next descriptor is published
+    int desc_ticket[4];           // ring by item sequence number: ticket (>= n_items: no more work)
+    int desc_n_old[4];            //                              len of that item before this call
+    int abort;
+    int pad[3];
+    float2 wstat[2][16][kMaxGroup];
+};
+
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+    asm volatile("{ .reg .b64 st; mbarrier.arrive.shared::cta.b64 st, [%0]; }" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait; false = gave up (or another warp already did).
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, volatile int* abort_flag) {
+    for (int it = 0; it < kWaitLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (it > 16) __nanosleep(100);
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+struct AsyncItem {
+    int valid;
+    int item, li, l, b, hkv;
+    int n_old, n, full;
+    int count, app_idx;  // streaming warps only
+};
+
+__device__ __forceinline__ void async_decode(const AttendArgs& a, int ticket, int n_old, AsyncItem& it) {
+    it.valid = ticket < a.n_items;
+    const int t = it.valid ? ticket : 0;
+    it.hkv = t % a.Hkv;
+    it.b = (t / a.Hkv) % a.B;
+    it.li = t / (a.Hkv * a.B);
+    it.l = a.layer_begin + it.li;
+    it.item = (it.l * a.B + it.b) * a.Hkv + it.hkv;
+    const bool append = a.k_new != nullptr;
+    it.n_old = n_old;
+    it.full = append && n_old >= a.cap_tokens;
+    it.n = it.full ? 0 : n_old + (append ? 1 : 0);
+    it.count = 0;
+    it.app_idx = -1;
+}
+
+// Sec. 4.1: the generated token's k / v row enters the cache (kept out of line: once per item).
+template <bool PAGED>
+__device__ __noinline__ void append_row(const AttendArgs& a, int item, int li, int b, int hkv, int n_old, int row_bytes,
+                                        int lane) {
+    const size_t src = ((size_t)(li * a.B + b) * a.Hkv + hkv) * row_bytes;
+    bool bad = false;
+    char* kd = const_cast<char*>(row_ptr<PAGED>(a, a.k, item, n_old, row_bytes, &bad));
+    char* vd = const_cast<char*>(row_ptr<PAGED>(a, a.v, item, n_old, row_bytes, &bad));
+    if (kd && vd && lane * 16 < row_bytes) {
+        *reinterpret_cast<uint4*>(kd + lane * 16) = *reinterpret_cast<const uint4*>((const char*)a.k_new + src + lane * 16);
+        *reinterpret_cast<uint4*>(vd + lane * 16) = *reinterpret_cast<const uint4*>((const char*)a.v_new + src + lane * 16);
+    }
+    if (lane == 0) a.pos[(size_t)item * a.cap_tokens + n_old] = a.token_pos[b];
+    __syncwarp();
+}
+
+template <int D, int NWS, int NS, bool PAGED, bool SPILL>
+__global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_kernel(const __grid_constant__ AttendArgs a) {
+    using T = __nv_bfloat16;
+    constexpr int ROW_BYTES = D * 2;
+    constexpr int CHUNKS = ROW_BYTES / 16;
+    constexpr int TILE_BYTES = kGroupTokens * ROW_BYTES;
+    constexpr int STAGE_BYTES = 2 * TILE_BYTES;
+    constexpr int WARP_BYTES = NS * STAGE_BYTES;
+    constexpr int KS = D / 16;
+    constexpr int ET = kEpilogueWarps * 32;
+    static_assert(NS >= 2 && NS <= 6 && NWS <= 16, "shape");
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    // layout: stages [NWS][NS][K tile | V tile] | AsyncHeader | wo [2][NWS][GP][D] fp32 | lg [2][chunk][GP] fp32
+    const int G = a.G, GP = a.GP;
+    const int wo_stride = GP * D;  // floats per warp
+    AsyncHeader& hd = *reinterpret_cast<AsyncHeader*>(smem_raw + (size_t)NWS * WARP_BYTES);
+    float* wo_all = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(&hd) + sizeof(AsyncHeader));
+    float* lg_all = wo_all + (size_t)2 * NWS * wo_stride;
+    const int chunk = a.chunk_tokens;
+    float* spill_all = SPILL ? a.spill + (size_t)blockIdx.x * 2 * a.spill_tokens * GP : nullptr;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool append = a.k_new != nullptr;
+    unsigned int* sched = a.sched;
+    volatile int* abort_flag = &hd.abort;
+
+    // ---- set-up: barriers, first two descriptors
+    bool drew_fail = false;  // meaningful in the ticket-drawing lane only
+    if (tid == 0) {
+        mbar_init(&hd.full[0], NWS);
+        mbar_init(&hd.full[1], NWS);
+        mbar_init(&hd.empty[0], kEpilogueWarps);
+        mbar_init(&hd.empty[1], kEpilogueWarps);
+        hd.abort = 0;
+    }
+    if (warp == NWS && lane == 0) {
+        int t0 = (int)atomicAdd(&sched[0], 1u);
+        int t1 = a.n_items;
+        if (t0 >= a.n_items) drew_fail = true;
+        else {
+            t1 = (int)atomicAdd(&sched[0], 1u);
+            if (t1 >= a.n_items) drew_fail = true;
+        }
+        AsyncItem tmp;
+        async_decode(a, t0, 0, tmp);
+        hd.desc_ticket[0] = t0;
+        hd.desc_n_old[0] = tmp.valid ? a.len[tmp.item] : 0;
+        async_decode(a, t1, 0, tmp);
+        hd.desc_ticket[1] = t1;
+        hd.desc_n_old[1] = tmp.valid ? a.len[tmp.item] : 0;
+    }
+    __syncthreads();
+
+    if (warp < NWS) {
+        // =================================================================== streaming warps
+        const int gq = lane >> 2, tq = lane & 3;
+        auto load_q = [&](const AsyncItem& it, uint32_t (&bq)[KS][2]) {
+            const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
+                (const T*)a.q + ((size_t)(it.li * a.B + it.b) * a.Hq + it.hkv * G + gq) * D);
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                bq[ks][0] = (it.valid && gq < G) ? qrow[8 * ks + tq] : 0u;
+                bq[ks][1] = (it.valid && gq < G) ? qrow[8 * ks + 4 + tq] : 0u;
+            }
+        };
+        auto set_counts = [&](AsyncItem& it) {
+            const int ng = (it.n + kGroupTokens - 1) / kGroupTokens;
+            it.count = ng > warp ? (ng - warp + NWS - 1) / NWS : 0;
+            it.app_idx = -1;
+            if (append && !it.full && it.valid) {
+                const int g = it.n_old / kGroupTokens;
+                if (g % NWS == warp) it.app_idx = g / NWS;
+            }
+        };
+        unsigned char* my_stage = smem_raw + (size_t)warp * WARP_BYTES;
+        const uint32_t my_stage_u32 = smem_u32(my_stage);
+        bool bad_page = false;
+
+        auto issue = [&](const AsyncItem& it, int idx, int slot) {
+            const int grp = warp + idx * NWS;
+            const int tok0 = grp * kGroupTokens;
+            if (idx == it.app_idx) append_row<PAGED>(a, it.item, it.li, it.b, it.hkv, it.n_old, ROW_BYTES, lane);
+            const char* kb;
+            const char* vb;
+            bool ok = true;
+            if (PAGED) {
+                const int page = a.page_table[(size_t)it.item * a.capacity + grp];
+                ok = page >= 0 && page < a.n_pages;
+                if (!ok) bad_page = true;
+                const size_t off = (size_t)(ok ? page : 0) * TILE_BYTES;
+                kb = (const char*)a.k + off;
+                vb = (const char*)a.v + off;
+            } else {
+                const size_t off = ((size_t)it.item * a.capacity + tok0) * ROW_BYTES;
+                kb = (const char*)a.k + off;
+                vb = (const char*)a.v + off;
+            }
+            const uint32_t ks_u32 = my_stage_u32 + slot * STAGE_BYTES;
+            const uint32_t vs_u32 = ks_u32 + TILE_BYTES;
+#pragma unroll
+            for (int i = 0; i < kGroupTokens * CHUNKS / 32; ++i) {
+                const int c_idx = i * 32 + lane;
+                const int r = c_idx / CHUNKS, c = c_idx % CHUNKS;
+                const bool valid = ok && (tok0 + r < it.n);
+                const int soff = valid ? r * ROW_BYTES + c * 16 : 0;
+                const uint32_t doff = r * ROW_BYTES + ((c ^ (r & 7)) << 4);
+                cp_async16(ks_u32 + doff, kb + soff, valid ? 16 : 0);
+                cp_async16(vs_u32 + doff, vb + soff, valid ? 16 : 0);
+            }
+        };
+
+        const int k_row = (lane & 7) + ((lane >> 3) & 1) * 8, k_chunk = lane >> 4;
+        const int v_row = (lane & 7) + ((lane >> 4) & 1) * 8, v_chunk = (lane >> 3) & 1;
+
+        AsyncItem cur, nxt;
+        async_decode(a, hd.desc_ticket[0], hd.desc_n_old[0], cur);
+        set_counts(cur);
+        uint32_t bq[KS][2], bqn[KS][2];
+        load_q(cur, bq);
+        nxt.valid = 0;
+        int seq = 0;          // sequence number of the current item within this CTA
+        int vp = 0;           // stage slot of the current item's local group 0
+        unsigned issued = 0;  // bit j: local group j (< NS-1) of the current item was prefetched by the previous tail
+        bool alive = true;
+
+        while (cur.valid && alive) {
+            const int p = seq & 1;
+            const float sl2 = a.scale_log2[cur.l];
+            const uint32_t lg_u32 = smem_u32(lg_all + (size_t)p * chunk * GP);
+            float* spill = SPILL ? spill_all + (size_t)p * a.spill_tokens * GP : nullptr;
+            bool nxt_ready = false;
+            // descriptor of the next item: wait until the epilogue of item seq-1 (same parity as seq+1) has
+            // handed its buffers back, which also publishes that descriptor
+            auto acquire_next = [&]() {
+                const int sn = seq + 1;
+                if (sn >= 2 && !mbar_wait(&hd.empty[sn & 1], (unsigned)(((sn >> 1) - 1) & 1), abort_flag)) {
+                    alive = false;
+                    nxt.valid = 0;
+                } else {
+                    async_decode(a, hd.desc_ticket[sn & 3], hd.desc_n_old[sn & 3], nxt);
+                    set_counts(nxt);
+                    load_q(nxt, bqn);
+                }
+                nxt_ready = true;
+            };
+
+            bool topped = false;
+#pragma unroll
+            for (int j = 0; j < NS - 1; ++j) {
+                if (!((issued >> j) & 1u) && j < cur.count) {
+                    issue(cur, j, (vp + j) % NS);
+                    topped = true;
+                }
+            }
+            if (topped) cp_async_commit();
+            unsigned issued_next = 0;
+
+            float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+            float o[KS][4];
+#pragma unroll
+            for (int mt = 0; mt < KS; ++mt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) o[mt][i] = 0.f;
+
+            constexpr bool OVF = SPILL;
+            for (int it = 0; it < cur.count; ++it) {
+                if (topped && it < NS - 1) cp_async_wait<0>();
+                else cp_async_wait<NS - 2>();
+                __syncwarp();
+                {
+                    const int idx = it + NS - 1;
+                    const int slot = (vp + idx) % NS;
+                    if (idx < cur.count) issue(cur, idx, slot);
+                    else {
+                        if (!nxt_ready) acquire_next();
+                        const int j = idx - cur.count;
+                        if (nxt.valid && j < nxt.count) {
+                            issue(nxt, j, slot);
+                            issued_next |= 1u << j;
+                        }
+                    }
+                    cp_async_commit();
+                }
+                const int grp = warp + it * NWS;
+                const uint32_t ks_u32 = my_stage_u32 + ((vp + it) % NS) * STAGE_BYTES;
+                const uint32_t vs_u32 = ks_u32 + TILE_BYTES;
+
+                float ca[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    uint32_t af[4];
+                    ldmatrix_x4(ks_u32 + k_row * ROW_BYTES + (((2 * ks + k_chunk) ^ (k_row & 7)) << 4), af);
+                    if (ks & 1) mma_bf16(cb, af, bq[ks][0], bq[ks][1]);
+                    else mma_bf16(ca, af, bq[ks][0], bq[ks][1]);
+                }
+                const int tokA = grp * kGroupTokens + gq, tokB = tokA + 8;
+                const float s00 = (tokA < cur.n) ? (ca[0] + cb[0]) * sl2 : -INFINITY;
+                const float s01 = (tokA < cur.n) ? (ca[1] + cb[1]) * sl2 : -INFINITY;
+                const float s10 = (tokB < cur.n) ? (ca[2] + cb[2]) * sl2 : -INFINITY;
+                const float s11 = (tokB < cur.n) ? (ca[3] + cb[3]) * sl2 : -INFINITY;
+                if (2 * tq < GP) {
+                    if (!OVF || tokA < chunk) st_shared_f2(lg_u32 + (tokA * GP + 2 * tq) * 4, s00, s01);
+                    else *reinterpret_cast<float2*>(spill + (size_t)(tokA - chunk) * GP + 2 * tq) = make_float2(s00, s01);
+                    if (!OVF || tokB < chunk) st_shared_f2(lg_u32 + (tokB * GP + 2 * tq) * 4, s10, s11);
+                    else *reinterpret_cast<float2*>(spill + (size_t)(tokB - chunk) * GP + 2 * tq) = make_float2(s10, s11);
+                }
+                float mx0 = fmaxf(s00, s10), mx1 = fmaxf(s01, s11);
+#pragma unroll
+                for (int off = 4; off < 32; off <<= 1) {
+                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+                }
+                const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+                if (__any_sync(0xffffffffu, (mn0 > m0) || (mn1 > m1))) {
+                    const float c0 = exp2_diff(m0, mn0), c1 = exp2_diff(m1, mn1);
+                    l0 *= c0;
+                    l1 *= c1;
+#pragma unroll
+                    for (int mt = 0; mt < KS; ++mt) {
+                        o[mt][0] *= c0; o[mt][2] *= c0;
+                        o[mt][1] *= c1; o[mt][3] *= c1;
+                    }
+                    m0 = mn0;
+                    m1 = mn1;
+                }
+                const float p00 = fast_exp2(s00 - m0), p01 = fast_exp2(s01 - m1);
+                const float p10 = fast_exp2(s10 - m0), p11 = fast_exp2(s11 - m1);
+                l0 += p00 + p10;
+                l1 += p01 + p11;
+                const uint32_t pb0 = movmatrix_trans(pack_bf16(p00, p01));
+                const uint32_t pb1 = movmatrix_trans(pack_bf16(p10, p11));
+#pragma unroll
+                for (int mt = 0; mt < KS; ++mt) {
+                    uint32_t af[4];
+                    ldmatrix_x4_trans(vs_u32 + v_row * ROW_BYTES + (((2 * mt + v_chunk) ^ (v_row & 7)) << 4), af);
+                    mma_bf16(o[mt], af, pb0, pb1);
+                }
+            }
+            vp = (vp + cur.count) % NS;
+
+            // ---- park this warp's partials in the parity buffer and signal the epilogue warps
+#pragma unroll
+            for (int off = 4; off < 32; off <<= 1) {
+                l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+                l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+            }
+            if (gq == 0) {
+                hd.wstat[p][warp][2 * tq] = make_float2(m0, l0);
+                hd.wstat[p][warp][2 * tq + 1] = make_float2(m1, l1);
+            }
+            if (2 * tq < GP) {
+                float* wo = wo_all + ((size_t)p * NWS + warp) * wo_stride;
+#pragma unroll
+                for (int mt = 0; mt < KS; ++mt) {
+                    wo[(2 * tq) * D + 16 * mt + gq] = o[mt][0];
+                    wo[(2 * tq + 1) * D + 16 * mt + gq] = o[mt][1];
+                    wo[(2 * tq) * D + 16 * mt + gq + 8] = o[mt][2];
+                    wo[(2 * tq + 1) * D + 16 * mt + gq + 8] = o[mt][3];
+                }
+            }
+            // (overflowed logits written to global memory are released to the epilogue warps by the mbarrier
+            // arrive below, which has release semantics at CTA scope, like the shared-memory writes)
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&hd.full[p]);
+
+            // ---- rotate
+            if (!nxt_ready) acquire_next();
+            cur = nxt;
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                bq[ks][0] = bqn[ks][0];
+                bq[ks][1] = bqn[ks][1];
+            }
+            issued = issued_next;
+            ++seq;
+        }
+        cp_async_wait<0>();
+        if (bad_page && lane == 0) record_error(a.status, LETHE_ERR_PAGE, 0);
+    } else {
+        // =================================================================== epilogue warps
+        const int ew = warp - NWS;
+        const int et = ew * 32 + lane;
+        bool alive = true;
+        for (int seq = 0; alive; ++seq) {
+            const int p = seq & 1;
+            // the descriptor of item seq was published by epilogue warp 0 while finishing item seq-2; waiting
+            // for that hand-back (both epilogue warps arrive on it) makes the write visible to this warp too
+            if (seq >= 2 && !mbar_wait(&hd.empty[p], (unsigned)(((seq >> 1) - 1) & 1), abort_flag)) {
+                alive = false;
+                break;
+            }
+            AsyncItem it;
+            async_decode(a, hd.desc_ticket[seq & 3], hd.desc_n_old[seq & 3], it);
+            if (!it.valid) break;
+            if (!mbar_wait(&hd.full[p], (unsigned)((seq >> 1) & 1), abort_flag)) {
+                alive = false;
+                break;
+            }
+            // ticket of the item after next: its round trips hide behind the merge below
+            int t_new = a.n_items;
+            if (ew == 0 && lane == 0 && !drew_fail) t_new = (int)atomicAdd(&sched[0], 1u);
+
+            const uint32_t lg_u32 = smem_u32(lg_all + (size_t)p * chunk * GP);
+            const float* spill = SPILL ? spill_all + (size_t)p * a.spill_tokens * GP : nullptr;
+            float* relp = a.rel + (size_t)it.item * a.cap_tokens;
+            const int app = (append && !it.full) ? it.n_old : -1;
+
+            // merged statistics of every head (each thread computes them all: off the critical path)
+            float fm[kMaxGroup], fi[kMaxGroup];
+#pragma unroll
+            for (int h = 0; h < kMaxGroup; ++h) {
+                fm[h] = -INFINITY;
+                fi[h] = 0.f;
+                if (h < G) {
+                    float m = -INFINITY;
+#pragma unroll
+                    for (int w = 0; w < NWS; ++w) m = fmaxf(m, hd.wstat[p][w][h].x);
+                    float l = 0.f;
+#pragma unroll
+                    for (int w = 0; w < NWS; ++w) l += hd.wstat[p][w][h].y * exp2_diff(hd.wstat[p][w][h].x, m);
+                    fm[h] = m;
+                    fi[h] = l > 0.f ? 1.f / l : 0.f;
+                    if (a.lse && et == h)
+                        a.lse[(size_t)(it.li * a.B + it.b) * a.Hq + it.hkv * G + h] =
+                            l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                }
+            }
+            const bool item_overflows = SPILL && it.n > chunk;
+            auto mass_of = [&](int j) {
+                const bool in_smem = !item_overflows || j < chunk;
+                float mass = 0.f;
+#pragma unroll
+                for (int h = 0; h < kMaxGroup; h += 2) {
+                    if (h < GP) {
+                        const float2 s2 = in_smem ? ld_shared_f2(lg_u32 + (j * GP + h) * 4)
+                                                  : *reinterpret_cast<const float2*>(spill + (size_t)(j - chunk) * GP + h);
+                        mass += fast_exp2(s2.x - fm[h]) * fi[h];
+                        if (h + 1 < G) mass += fast_exp2(s2.y - fm[h + 1]) * fi[h + 1];
+                    }
+                }
+                return mass;
+            };
+            // Eq. 5 on rel[0..n): old values are fetched a batch ahead of their use
+            constexpr int RB = 8;
+            float oldv[RB];
+            auto fetch = [&](int base) {
+#pragma unroll
+                for (int i = 0; i < RB; ++i) {
+                    const int j = base + et + i * ET;
+                    oldv[i] = (j < it.n && j != app) ? relp[j] : 0.f;
+                }
+            };
+            fetch(0);
+            {
+                T* out = (T*)a.out + ((size_t)(it.li * a.B + it.b) * a.Hq + it.hkv * G) * D;
+                for (int idx = et; idx < G * D; idx += ET) {
+                    const int h = idx / D;
+                    float mh = -INFINITY, ih = 0.f;
+#pragma unroll
+                    for (int hh = 0; hh < kMaxGroup; ++hh)
+                        if (hh == h) {
+                            mh = fm[hh];
+                            ih = fi[hh];
+                        }
+                    float acc = 0.f;
+#pragma unroll
+                    for (int w = 0; w < NWS; ++w)
+                        acc += wo_all[((size_t)p * NWS + w) * wo_stride + idx] * exp2_diff(hd.wstat[p][w][h].x, mh);
+                    out[idx] = __float2bfloat16_rn(acc * ih);
+                }
+            }
+            for (int base = 0; base < it.n; base += RB * ET) {
+                float cur_old[RB];
+#pragma unroll
+                for (int i = 0; i < RB; ++i) cur_old[i] = oldv[i];
+                if (base + RB * ET < it.n) fetch(base + RB * ET);
+#pragma unroll
+                for (int i = 0; i < RB; ++i) {
+                    const int j = base + et + i * ET;
+                    if (j < it.n) relp[j] = fmaf(a.gamma, cur_old[i], mass_of(j));
+                }
+            }
+            if (ew == 0 && lane == 0) {
+                if (it.full) record_error(a.status, LETHE_ERR_CAPACITY, it.item);
+                else if (append) a.len[it.item] = it.n;
+                if (t_new >= a.n_items) drew_fail = true;
+                AsyncItem nx;
+                async_decode(a, t_new, 0, nx);
+                hd.desc_n_old[(seq + 2) & 3] = nx.valid ? a.len[nx.item] : 0;
+                hd.desc_ticket[(seq + 2) & 3] = t_new;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&hd.empty[p]);
+        }
+        if (!alive && lane == 0) record_error(a.status, LETHE_ERR_TIMEOUT, (int)blockIdx.x);
+        // ---- the last CTA out re-arms the queue for the next launch
+        if (ew == 0 && lane == 0) {
+            __threadfence();
+            const unsigned int done = atomicAdd(&sched[1], 1u);
+            if (done == gridDim.x - 1) {
+                sched[0] = 0u;
+                sched[1] = 0u;
+                __threadfence();
+            }
+        }
+    }
+}
+
+template <int D, int NWS, int NS>
+static size_t async_smem(int chunk_tokens, int GP) {
+    return (size_t)NWS * NS * 2 * kGroupTokens * D * 2 + sizeof(AsyncHeader) + (size_t)2 * NWS * GP * D * 4 +
+           (size_t)2 * chunk_tokens * GP * 4;
+}
+
+template <int D, int NWS, int NS, bool PAGED, bool SPILL>
+static cudaError_t launch_async_t(const AttendArgs& a, int grid, cudaStream_t stream) {
+    auto kern = attend_async_kernel<D, NWS, NS, PAGED, SPILL>;
+    const size_t smem = async_smem<D, NWS, NS>(a.chunk_tokens, a.GP);
+    cudaError_t e = prepare_kernel((const void*)kern, smem);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, (NWS + kEpilogueWarps) * 32, smem, stream>>>(a);
+    return cudaGetLastError();
+}
+
+template <int D, int NWS, int NS>
+static cudaError_t dispatch_async(const AttendArgs& a, bool paged, int grid, cudaStream_t stream) {
+    const bool spill = a.spill != nullptr;
+    if (paged) return spill ? launch_async_t<D, NWS, NS, true, true>(a, grid, stream) : launch_async_t<D, NWS, NS, true, false>(a, grid, stream);
+    return spill ? launch_async_t<D, NWS, NS, false, true>(a, grid, stream) : launch_async_t<D, NWS, NS, false, false>(a, grid, stream);
+}
+
+// Shapes: (streaming warps per CTA, stages per warp); two more warps run the epilogue.
+#define LETHE_ASYNC_SHAPES(X, D) X(0, D, 8, 2) X(1, D, 7, 2) X(2, D, 6, 3) X(3, D, 5, 3) X(4, D, 6, 2) X(5, D, 4, 4) X(6, D, 3, 5) \
+        X(7, D, 5, 4)
+
+size_t async_smem_bytes(int D, int shape, int chunk_tokens, int GP) {
+#define X(id, DD, NW, NS) \
+    if (shape == id && D == DD) return async_smem<DD, NW, NS>(chunk_tokens, GP);
+    LETHE_ASYNC_SHAPES(X, 128)
+    LETHE_ASYNC_SHAPES(X, 64)
+#undef X
+    return (size_t)-1;
+}
+
+cudaError_t launch_attend_async(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream) {
+#define X(id, DD, NW, NS) \
+    if (shape == id && D == DD) return dispatch_async<DD, NW, NS>(a, paged, grid, stream);
+    LETHE_ASYNC_SHAPES(X, 128)
+    LETHE_ASYNC_SHAPES(X, 64)
+#undef X
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace lethe

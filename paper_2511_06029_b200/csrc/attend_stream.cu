@@ -77,9 +77,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
     // (SPILL is a compile-time switch so that launches whose buffer covers the capacity pay nothing for it.)
     const int chunk = SPILL ? a.chunk_tokens : 0x7fffffff;
     float* spill = SPILL ? a.spill + (size_t)blockIdx.x * a.spill_tokens * GP : nullptr;
-    auto lg_row = [&](int tok) -> float* {
-        return (!SPILL || tok < chunk) ? lg + (size_t)tok * GP : spill + (size_t)(tok - chunk) * GP;
-    };
+    const uint32_t lg_u32 = smem_u32(lg);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int gq = lane >> 2, tq = lane & 3;
@@ -236,13 +234,10 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
             const float s10 = (tokB < cur.n) ? (ca[2] + cb[2]) * sl2 : -INFINITY;
             const float s11 = (tokB < cur.n) ? (ca[3] + cb[3]) * sl2 : -INFINITY;
             if (2 * tq < GP) {
-                if (!SPILL || tokB < chunk) {  // common case: both rows of this thread live in shared memory
-                    *reinterpret_cast<float2*>(lg + (size_t)tokA * GP + 2 * tq) = make_float2(s00, s01);
-                    *reinterpret_cast<float2*>(lg + (size_t)tokB * GP + 2 * tq) = make_float2(s10, s11);
-                } else {
-                    *reinterpret_cast<float2*>(lg_row(tokA) + 2 * tq) = make_float2(s00, s01);
-                    *reinterpret_cast<float2*>(lg_row(tokB) + 2 * tq) = make_float2(s10, s11);
-                }
+                if (!SPILL || tokA < chunk) st_shared_f2(lg_u32 + (tokA * GP + 2 * tq) * 4, s00, s01);
+                else *reinterpret_cast<float2*>(spill + (size_t)(tokA - chunk) * GP + 2 * tq) = make_float2(s00, s01);
+                if (!SPILL || tokB < chunk) st_shared_f2(lg_u32 + (tokB * GP + 2 * tq) * 4, s10, s11);
+                else *reinterpret_cast<float2*>(spill + (size_t)(tokB - chunk) * GP + 2 * tq) = make_float2(s10, s11);
             }
             float mx0 = fmaxf(s00, s10), mx1 = fmaxf(s01, s11);
 #pragma unroll
@@ -350,12 +345,13 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
             }
             float* relp = a.rel + (size_t)cur.item * a.cap_tokens;
             auto mass_of = [&](int j) {
-                const float* row = (!SPILL || j < chunk) ? lg + (size_t)j * GP : spill + (size_t)(j - chunk) * GP;
+                const bool in_smem = !SPILL || j < chunk;
                 float mass = 0.f;
 #pragma unroll
                 for (int h = 0; h < kMaxGroup; h += 2) {
                     if (h < GP) {
-                        const float2 s2 = *reinterpret_cast<const float2*>(row + h);
+                        const float2 s2 = in_smem ? ld_shared_f2(lg_u32 + (j * GP + h) * 4)
+                                                  : *reinterpret_cast<const float2*>(spill + (size_t)(j - chunk) * GP + h);
                         mass += fast_exp2(s2.x - fm[h]) * fi[h];
                         if (h + 1 < G) mass += fast_exp2(s2.y - fm[h + 1]) * fi[h + 1];
                     }

@@ -78,6 +78,12 @@ CASES = [
     (torch.bfloat16, 128, 4, 1, 300, 11, 0),
     (torch.bfloat16, 64, 16, 2, 500, 12, 0),
     (torch.bfloat16, 128, 6, 2, 300, 13, 0),
+    (torch.bfloat16, 128, 32, 8, 300, 16, 0),
+    (torch.bfloat16, 128, 28, 4, 700, 17, 1),
+    (torch.bfloat16, 64, 14, 2, 300, 18, 0),
+    (torch.bfloat16, 128, 4, 1, 300, 19, 0),
+    (torch.bfloat16, 64, 16, 2, 500, 20, 0),
+    (torch.bfloat16, 128, 6, 2, 300, 21, 0),
     (torch.bfloat16, 128, 8, 8, 260, 0, 0),
     (torch.float32, 128, 16, 2, 260, 0, 0),
 ]
@@ -106,7 +112,7 @@ def test_decode_attend_parity(ctx, dtype, D, Hq, Hkv, cap, variant, splits):
         ctx.set_tuning(0, 0)
 
 
-@pytest.mark.parametrize("variant", [8, 9, 10, 12, 13])
+@pytest.mark.parametrize("variant", [8, 9, 10, 12, 13, 16, 17, 18, 19, 21])
 def test_persistent_queue_many_items(ctx, variant):
     """More items than SMs, so every CTA of the persistent kernel walks several items through its queue and
     prefetches across item boundaries; lengths from 0 to several hundred, including tiny items that leave
@@ -366,7 +372,8 @@ def test_ragged_paged_long_items(ctx):
         oracle.set_threads(1)
 
 
-@pytest.mark.parametrize("variant,Hq,Hkv,cap", [(9, 28, 4, 3000), (12, 16, 4, 4200), (14, 28, 4, 6000)])
+@pytest.mark.parametrize("variant,Hq,Hkv,cap", [(9, 28, 4, 3000), (12, 16, 4, 4200), (14, 28, 4, 6000), (16, 28, 4, 3000),
+                                                (18, 16, 4, 4200), (20, 28, 4, 6000)])
 def test_persistent_logit_overflow(ctx, variant, Hq, Hkv, cap):
     """Items longer than the on-chip logit buffer of the persistent kernel: the logits of the tail tokens
     overflow to global scratch and the relevance update must still be exact."""
