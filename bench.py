@@ -336,6 +336,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-per-layer", action="store_true")
+    ap.add_argument("--pl-variant", type=int, default=0, help="kernel variant of the per-layer launch mode")
+    ap.add_argument("--pl-splits", type=int, default=0)
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
 
@@ -415,7 +417,9 @@ def main():
     per_layer = None
     if not args.no_per_layer and world == 1:
         pl_steps = min(32, max(4, w.prune_interval - (r.step_no % w.prune_interval) - 8))
+        r.ctx.set_tuning(args.pl_variant, args.pl_splits)
         ms_pl, th_pl = per_layer_mode(r, pl_steps)
+        r.ctx.set_tuning(args.variant, args.splits)
         r.check()
         per_layer = {"ms_per_step": ms_pl, "token_heads_per_step": th_pl, "value": th_pl / (ms_pl * 1e-3),
                      "algorithmic_GBs": th_pl * BYTES_PER_TOKEN_HEAD / (ms_pl * 1e-3) / 1e9,

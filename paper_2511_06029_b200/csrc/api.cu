@@ -305,7 +305,7 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
             for (int shape : {4, 1, 0})
                 if (variant == 0 && stream_chunk(shape) == cap_pad) variant = 8 + shape;
             if (variant == 0) variant = 16 + 3;
-        } else variant = 4;
+        } else variant = 2;  // few items per launch (one layer at a time): clustered kernel, 4 warps x 3 stages
     }
     if (variant >= 2 && !mma_ok) return fail(ctx, LETHE_ERR_UNSUPPORTED, "tensor-core variants need bf16 and 16-token pages");
 
@@ -354,7 +354,9 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         if (S == 0) {
             S = 1;
             while (S < 16 && smem_for(S) > ctx->max_smem) S *= 2;
-            while (S < 8 && (long long)a.n_items * S < 2LL * ctx->sm_count && cap_groups / (2 * S) >= 4) S *= 2;
+            // enough CTAs to cover the SMs once; larger clusters cost more in scheduling and barriers than they
+            // gain (measured: 64 items run best as 4-CTA clusters)
+            while (S < 8 && (long long)a.n_items * S < ctx->sm_count && cap_groups / (2 * S) >= 4) S *= 2;
         }
         if (smem_for(S) > ctx->max_smem)
             return fail(ctx, LETHE_ERR_UNSUPPORTED, "capacity too large for the on-chip logit buffer at this split count");
