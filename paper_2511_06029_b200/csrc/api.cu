@@ -295,8 +295,10 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         if (!mma_ok) variant = 1;
         else if (a.n_items >= 2 * ctx->sm_count && ctx->splits <= 1) {
             // Persistent kernels, best measured first, taking the first whose logit buffer(s) cover the
-            // capacity on chip: asynchronous epilogue (6,3) (5,3) (4,4), then the synchronous (7,3) (6,3) (8,2);
-            // if none does, the asynchronous (5,3) with the tail of long items overflowing to scratch.
+            // capacity on chip: asynchronous epilogue (6,3) (5,3) (4,4), then the synchronous (7,3) (6,3) (8,2).
+            // If none does, the tail of long items overflows to scratch: asynchronous (5,3) when each of its two
+            // buffers still holds most of the capacity, else the synchronous (6,3), whose single buffer is
+            // twice as long.
             const int cap_pad = cap_groups * kGroupTokens;
             auto async_fits = [&](int shape) { return async_smem_bytes(c->head_dim, shape, cap_pad, a.GP) <= ctx->max_smem; };
             variant = 0;
@@ -304,7 +306,11 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
                 if (variant == 0 && async_fits(shape)) variant = 16 + shape;
             for (int shape : {4, 1, 0})
                 if (variant == 0 && stream_chunk(shape) == cap_pad) variant = 8 + shape;
-            if (variant == 0) variant = 16 + 3;
+            if (variant == 0) {
+                const size_t fixed = async_smem_bytes(c->head_dim, 3, 0, a.GP);
+                const size_t async_chunk = fixed < ctx->max_smem ? (ctx->max_smem - fixed) / ((size_t)2 * a.GP * 4) : 0;
+                variant = (async_chunk * 10 >= (size_t)cap_pad * 6) ? 16 + 3 : 8 + 1;
+            }
         } else variant = 2;  // few items per launch (one layer at a time): clustered kernel, 4 warps x 3 stages
     }
     if (variant >= 2 && !mma_ok) return fail(ctx, LETHE_ERR_UNSUPPORTED, "tensor-core variants need bf16 and 16-token pages");
