@@ -173,7 +173,15 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
         const uint32_t my_stage_u32 = smem_u32(my_stage);
         bool bad_page = false;
 
-        auto issue = [&](const AsyncItem& it, int idx, int slot) {
+        // PAGED: page ids of this warp's local groups are fetched 32 at a time, one lane each, a block ahead of
+        // their use, so that staging a group never waits on a page-table load.
+        int pg_lo = 0, pg_hi = 0, pg_nxt = 0;  // current item: blocks pg_blk and pg_blk + 1; next item: block 0
+        int pg_blk = 0;
+        auto load_pages = [&](const AsyncItem& it, int blk) -> int {
+            const int g = blk * 32 + lane;
+            return (PAGED && it.valid && g < it.count) ? a.page_table[(size_t)it.item * a.capacity + warp + g * NWS] : 0;
+        };
+        auto issue = [&](const AsyncItem& it, int idx, int slot, bool is_cur) {
             const int grp = warp + idx * NWS;
             const int tok0 = grp * kGroupTokens;
             if (idx == it.app_idx) append_row<PAGED>(a, it.item, it.li, it.b, it.hkv, it.n_old, ROW_BYTES, lane);
@@ -181,7 +189,16 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
             const char* vb;
             bool ok = true;
             if (PAGED) {
-                const int page = a.page_table[(size_t)it.item * a.capacity + grp];
+                int page;
+                if (!is_cur) page = __shfl_sync(0xffffffffu, pg_nxt, idx & 31);  // only the first NS-1 groups
+                else {
+                    if ((idx >> 5) > pg_blk) {  // first group of the next block: rotate and fetch one more ahead
+                        pg_lo = pg_hi;
+                        ++pg_blk;
+                        pg_hi = load_pages(it, pg_blk + 1);
+                    }
+                    page = __shfl_sync(0xffffffffu, pg_lo, idx & 31);
+                }
                 ok = page >= 0 && page < a.n_pages;
                 if (!ok) bad_page = true;
                 const size_t off = (size_t)(ok ? page : 0) * TILE_BYTES;
@@ -214,6 +231,8 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
         set_counts(cur);
         uint32_t bq[KS][2], bqn[KS][2];
         load_q(cur, bq);
+        pg_lo = load_pages(cur, 0);
+        pg_hi = load_pages(cur, 1);
         nxt.valid = 0;
         int seq = 0;          // sequence number of the current item within this CTA
         int vp = 0;           // stage slot of the current item's local group 0
@@ -237,6 +256,7 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
                     async_decode(a, hd.desc_ticket[sn & 3], hd.desc_n_old[sn & 3], nxt);
                     set_counts(nxt);
                     load_q(nxt, bqn);
+                    pg_nxt = load_pages(nxt, 0);
                 }
                 nxt_ready = true;
             };
@@ -245,7 +265,7 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
 #pragma unroll
             for (int j = 0; j < NS - 1; ++j) {
                 if (!((issued >> j) & 1u) && j < cur.count) {
-                    issue(cur, j, (vp + j) % NS);
+                    issue(cur, j, (vp + j) % NS, true);
                     topped = true;
                 }
             }
@@ -267,12 +287,12 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
                 {
                     const int idx = it + NS - 1;
                     const int slot = (vp + idx) % NS;
-                    if (idx < cur.count) issue(cur, idx, slot);
+                    if (idx < cur.count) issue(cur, idx, slot, true);
                     else {
                         if (!nxt_ready) acquire_next();
                         const int j = idx - cur.count;
                         if (nxt.valid && j < nxt.count) {
-                            issue(nxt, j, slot);
+                            issue(nxt, j, slot, false);
                             issued_next |= 1u << j;
                         }
                     }
@@ -368,6 +388,9 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
                 bq[ks][0] = bqn[ks][0];
                 bq[ks][1] = bqn[ks][1];
             }
+            pg_lo = pg_nxt;
+            pg_blk = 0;
+            pg_hi = load_pages(cur, 1);
             issued = issued_next;
             ++seq;
         }

@@ -122,7 +122,15 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
     bool bad_page = false;
 
     // issue the copies of this warp's local group `idx` of item `it` into stage slot `slot`
-    auto issue = [&](const StreamItem& it, int idx, int slot) {
+    // PAGED: page ids of this warp's local groups are fetched 32 at a time, one lane each, a block ahead of their
+    // use, so that staging a group never waits on a page-table load.
+    int pg_lo = 0, pg_hi = 0, pg_nxt = 0;  // current item: blocks pg_blk and pg_blk + 1; next item: block 0
+    int pg_blk = 0;
+    auto load_pages = [&](const StreamItem& it, int count, int blk) -> int {
+        const int g = blk * 32 + lane;
+        return (PAGED && it.valid && g < count) ? a.page_table[(size_t)it.item * a.capacity + warp + g * NW] : 0;
+    };
+    auto issue = [&](const StreamItem& it, int idx, int slot, bool is_cur) {
         const int grp = warp + idx * NW;
         const int tok0 = grp * kGroupTokens;
         if (idx == it.app_idx) {  // Sec. 4.1: the generated token's k / v row enters the cache first
@@ -141,7 +149,16 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
         const char* vb;
         bool ok = true;
         if (PAGED) {
-            const int page = a.page_table[(size_t)it.item * a.capacity + grp];
+            int page;
+            if (!is_cur) page = __shfl_sync(0xffffffffu, pg_nxt, idx & 31);  // only the first NS-1 groups
+            else {
+                if ((idx >> 5) > pg_blk) {  // first group of the next block: rotate and fetch one more ahead
+                    pg_lo = pg_hi;
+                    ++pg_blk;
+                    pg_hi = load_pages(it, it.count, pg_blk + 1);
+                }
+                page = __shfl_sync(0xffffffffu, pg_lo, idx & 31);
+            }
             ok = page >= 0 && page < a.n_pages;
             if (!ok) bad_page = true;
             const size_t off = (size_t)(ok ? page : 0) * TILE_BYTES;
@@ -169,6 +186,9 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
     const int k_row = (lane & 7) + ((lane >> 3) & 1) * 8, k_chunk = lane >> 4;
     const int v_row = (lane & 7) + ((lane >> 4) & 1) * 8, v_chunk = (lane >> 3) & 1;
 
+    pg_lo = load_pages(cur, cur.count, 0);
+    pg_hi = load_pages(cur, cur.count, 1);
+
     int vp = 0;              // stage slot of the current item's local group 0
     unsigned issued = 0;     // bit j: local group j (< NS-1) of the current item was prefetched by the previous tail
 
@@ -180,7 +200,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
 #pragma unroll
         for (int j = 0; j < NS - 1; ++j) {
             if (!((issued >> j) & 1u) && j < cur.count) {
-                issue(cur, j, (vp + j) % NS);
+                issue(cur, j, (vp + j) % NS, true);
                 topped = true;
             }
         }
@@ -202,15 +222,16 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
             {              // refill the slot freed by group it-1 with the group NS-1 ahead (possibly of the next item)
                 const int idx = it + NS - 1;
                 const int slot = (vp + idx) % NS;
-                if (idx < cur.count) issue(cur, idx, slot);
+                if (idx < cur.count) issue(cur, idx, slot, true);
                 else if (nxt.valid) {
                     if (!nxt_ready) {
                         fill_counts<NW>(a, nxt, opaque(nxt_n_raw), warp);
+                        pg_nxt = load_pages(nxt, nxt.count, 0);
                         nxt_ready = true;
                     }
                     const int j = idx - cur.count;
                     if (j < nxt.count) {
-                        issue(nxt, j, slot);
+                        issue(nxt, j, slot, false);
                         issued_next |= 1u << j;
                     }
                 }
@@ -378,8 +399,14 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
         TL_MARK_AT(a, cur.item - a.layer_begin * a.B * a.Hkv, 4);
 
         // ---- rotate: next becomes current
-        if (nxt.valid && !nxt_ready) fill_counts<NW>(a, nxt, nxt_n_raw, warp);
+        if (nxt.valid && !nxt_ready) {
+            fill_counts<NW>(a, nxt, nxt_n_raw, warp);
+            pg_nxt = load_pages(nxt, nxt.count, 0);
+        }
         cur = nxt;
+        pg_lo = pg_nxt;
+        pg_blk = 0;
+        pg_hi = load_pages(cur, cur.valid ? cur.count : 0, 1);
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
             bq[ks][0] = bqn[ks][0];

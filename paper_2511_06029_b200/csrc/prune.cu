@@ -239,17 +239,17 @@ __global__ void __launch_bounds__(kPruneThreads) rasr_prune_kernel(CacheView c, 
                 if ((key & mask_hi) == prefix) atomicAdd(&hist[(key >> shift) & 0xffu], 1);
             }
             __syncthreads();
-            if (tid == 0) {
-                int remaining = sel_remaining;
-                int d = 255;
-                for (; d > 0; --d) {
-                    if (hist[d] >= remaining) break;
-                    remaining -= hist[d];
+            {   // bin holding the remaining-th largest key: suffix sums over the 256 bins by one block scan
+                const int remaining = sel_remaining;
+                const int h = tid < 256 ? hist[255 - tid] : 0;  // thread t looks at bin 255 - t
+                int ex, tot;
+                block_scan(h, warp_buf, ex, tot);               // ex = keys in bins above this thread's bin
+                if (tid < 256 && ex < remaining && ex + h >= remaining) {
+                    sel_prefix = prefix | ((uint32_t)(255 - tid) << shift);
+                    sel_remaining = remaining - ex;
                 }
-                sel_prefix = prefix | ((uint32_t)d << shift);
-                sel_remaining = remaining;
+                __syncthreads();
             }
-            __syncthreads();
         }
         T = sel_prefix;
         need_eq = sel_remaining;  // how many slots equal to T are kept (the oldest ones)
@@ -290,41 +290,54 @@ __global__ void __launch_bounds__(kPruneThreads) rasr_prune_kernel(CacheView c, 
     // ---- move rows in ascending waves
     const int row_bytes = c.D * c.elt_bytes;
     const int lanes_per_row = row_bytes / 16;            // 16-byte pieces per row (8, 16 or 32)
-    const int rows_per_wave = kPruneThreads / lanes_per_row;
+    constexpr int RPT = 4;                               // rows each thread slot carries per wave
+    const int slots = kPruneThreads / lanes_per_row;     // row slots per pass
+    const int rows_per_wave = slots * RPT;
     const int piece = tid % lanes_per_row, rslot = tid / lanes_per_row;
     bool bad = false;
-    // skip the unmoved prefix: destinations whose source is themselves
+    // destinations whose source is themselves (the unmoved prefix, and any later fixed point) are skipped
     for (int w0 = 0; w0 < keep_n; w0 += rows_per_wave) {
-        const int dst = w0 + rslot;
-        int src = -1;
-        if (dst < keep_n) src = src_list[dst];
-        uint4 kv = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
-        float rv = 0.f;
-        int pv = 0;
-        const bool moves = src >= 0 && src != dst;
-        if (moves) {
-            const char* ks = prune_row_ptr(c, c.k, item, src, row_bytes, &bad);
-            const char* vs = prune_row_ptr(c, c.v, item, src, row_bytes, &bad);
-            if (ks && vs) {
-                kv = *reinterpret_cast<const uint4*>(ks + piece * 16);
-                vv = *reinterpret_cast<const uint4*>(vs + piece * 16);
-            }
-            if (piece == 0) {
-                rv = rel[src];
-                pv = pos[src];
+        uint4 kv[RPT], vv[RPT];
+        float rv[RPT];
+        int pv[RPT], srcs[RPT];
+#pragma unroll
+        for (int r = 0; r < RPT; ++r) {
+            const int dst = w0 + r * slots + rslot;
+            int src = -1;
+            if (dst < keep_n) src = src_list[dst];
+            srcs[r] = (src >= 0 && src != dst) ? src : -1;
+            kv[r] = make_uint4(0, 0, 0, 0);
+            vv[r] = make_uint4(0, 0, 0, 0);
+            rv[r] = 0.f;
+            pv[r] = 0;
+            if (srcs[r] >= 0) {
+                const char* ks = prune_row_ptr(c, c.k, item, srcs[r], row_bytes, &bad);
+                const char* vs = prune_row_ptr(c, c.v, item, srcs[r], row_bytes, &bad);
+                if (ks && vs) {
+                    kv[r] = *reinterpret_cast<const uint4*>(ks + piece * 16);
+                    vv[r] = *reinterpret_cast<const uint4*>(vs + piece * 16);
+                }
+                if (piece == 0) {
+                    rv[r] = rel[srcs[r]];
+                    pv[r] = pos[srcs[r]];
+                }
             }
         }
-        __syncthreads();
-        if (moves) {
-            char* kd = prune_row_ptr(c, c.k, item, dst, row_bytes, &bad);
-            char* vd = prune_row_ptr(c, c.v, item, dst, row_bytes, &bad);
-            if (kd && vd) {
-                *reinterpret_cast<uint4*>(kd + piece * 16) = kv;
-                *reinterpret_cast<uint4*>(vd + piece * 16) = vv;
-            }
-            if (piece == 0) {
-                rel[dst] = rv;
-                pos[dst] = pv;
+        __syncthreads();  // every source row of this wave has been read
+#pragma unroll
+        for (int r = 0; r < RPT; ++r) {
+            if (srcs[r] >= 0) {
+                const int dst = w0 + r * slots + rslot;
+                char* kd = prune_row_ptr(c, c.k, item, dst, row_bytes, &bad);
+                char* vd = prune_row_ptr(c, c.v, item, dst, row_bytes, &bad);
+                if (kd && vd) {
+                    *reinterpret_cast<uint4*>(kd + piece * 16) = kv[r];
+                    *reinterpret_cast<uint4*>(vd + piece * 16) = vv[r];
+                }
+                if (piece == 0) {
+                    rel[dst] = rv[r];
+                    pos[dst] = pv[r];
+                }
             }
         }
         // no barrier needed here: the next wave's sources lie above every destination written so far
