@@ -20,6 +20,7 @@ size_t async_smem_bytes(int D, int shape, int chunk_tokens, int GP);
 cudaError_t launch_sparsity(const CacheView& c, float* sparsity, cudaStream_t stream);
 cudaError_t launch_budgets(int L, int B, const float* sparsity, const long long* total, int k_min, int32_t* budgets,
                            int32_t* status, cudaStream_t stream);
+cudaError_t launch_order(const int32_t* len, int n_items, int cap_tokens, int32_t* order, cudaStream_t stream);
 cudaError_t launch_rasr_prune(const CacheView& c, const int32_t* budgets, int recent, int sink, int32_t* keep_idx,
                               int max_k, int smem_tokens, int32_t* list_scratch, int32_t* status,
                               cudaStream_t stream);
@@ -65,6 +66,11 @@ struct lethe_ctx {
     unsigned int* sched;  // device: {next ticket, CTAs finished}; zero whenever no attend launch is running
     void* scratch;
     size_t scratch_bytes;
+    // longest-first item order written by the last lethe_rasr_prune, and the cache it describes
+    int32_t* order;
+    size_t order_bytes;
+    const int32_t* order_len;  // cache.len the order was computed from
+    int order_items;
     void* staging;  // device staging of lethe_decode_attend_host
     size_t staging_bytes;
     int variant, splits;
@@ -191,6 +197,7 @@ void lethe_destroy(lethe_ctx* ctx) {
     if (ctx->status) cudaFree(ctx->status);
     if (ctx->scratch) cudaFree(ctx->scratch);
     if (ctx->staging) cudaFree(ctx->staging);
+    if (ctx->order) cudaFree(ctx->order);
     delete ctx;
 }
 
@@ -266,6 +273,11 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
     a.q = q; a.k_new = k_new; a.v_new = v_new; a.token_pos = token_pos; a.out = out; a.lse = lse;
     a.status = ctx->status;
     a.sched = ctx->sched;
+    // Work-queue order from the last prune round: usable while the call covers the same items (all layers of the
+    // same cache).  Appends lengthen every item alike, so the order stays longest-first between rounds.
+    if (ctx->order && ctx->order_len == c->len && layer_begin == 0 && layer_end == c->n_layers &&
+        ctx->order_items == c->n_layers * c->batch * c->n_kv_heads)
+        a.order = ctx->order;
     a.n_pages = c->n_pages;
     a.B = c->batch; a.Hq = c->n_q_heads; a.Hkv = c->n_kv_heads; a.G = G; a.GP = (G + 1) & ~1;
     a.capacity = c->capacity; a.cap_tokens = cap_tokens_of(c);
@@ -471,6 +483,19 @@ lethe_status lethe_rasr_prune(lethe_ctx* ctx, const lethe_cache* c, const int32_
     cudaError_t e = launch_rasr_prune(v, budgets, recent, sink, keep_idx, keep_idx ? max_k : 0, smem_tokens,
                                       list_scratch, ctx->status, (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "rasr_prune launch");
+    // longest-first order of the items for the persistent attend kernels' work queue
+    const long long items = (long long)v.L * v.B * v.Hkv;
+    ctx->order_len = nullptr;
+    if (items >= 2LL * ctx->sm_count && items <= (1 << 20)) {
+        void* buf = ctx->order;
+        st = ensure(ctx, &buf, &ctx->order_bytes, (size_t)items * sizeof(int32_t), "item order");
+        ctx->order = (int32_t*)buf;
+        if (st != LETHE_OK) return st;
+        e = launch_order(c->len, (int)items, v.cap_tokens, ctx->order, (cudaStream_t)stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "item order launch");
+        ctx->order_len = c->len;
+        ctx->order_items = (int)items;
+    }
     return LETHE_OK;
 }
 

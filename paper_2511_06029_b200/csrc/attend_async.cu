@@ -138,6 +138,10 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
             t1 = (int)atomicAdd(&sched[0], 1u);
             if (t1 >= a.n_items) drew_fail = true;
         }
+        if (a.order) {  // longest-first order of the items (valid tickets only)
+            if (t0 < a.n_items) t0 = a.order[t0];
+            if (t1 < a.n_items) t1 = a.order[t1];
+        }
         AsyncItem tmp;
         async_decode(a, t0, 0, tmp);
         hd.desc_ticket[0] = t0;
@@ -504,6 +508,7 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
                 if (it.full) record_error(a.status, LETHE_ERR_CAPACITY, it.item);
                 else if (append) a.len[it.item] = it.n;
                 if (t_new >= a.n_items) drew_fail = true;
+                if (a.order && t_new < a.n_items) t_new = a.order[t_new];
                 AsyncItem nx;
                 async_decode(a, t_new, 0, nx);
                 hd.desc_n_old[(seq + 2) & 3] = nx.valid ? a.len[nx.item] : 0;

@@ -32,6 +32,7 @@ struct AttendArgs {
     float* lse;
     int32_t* status;      // device status word: {code, item}
     unsigned int* sched;  // persistent kernel only: {next ticket, CTAs finished}, zero between launches
+    const int32_t* order; // persistent kernels: ticket -> item of the call, longest items first (NULL = identity)
     float* spill;         // persistent kernel only: global overflow of the logit buffer, [grid][spill_tokens][GP]
     int spill_tokens;     // tokens per CTA the overflow can hold (0 = the shared-memory buffer covers cap_tokens)
     long long n_pages;

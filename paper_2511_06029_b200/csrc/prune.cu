@@ -357,6 +357,40 @@ cudaError_t launch_rasr_prune(const CacheView& c, const int32_t* budgets, int re
     return cudaGetLastError();
 }
 
+// ------------------------------------------------------------ longest-first item order for the attend queue
+// One CTA: counting sort of the items by len (1024 buckets over [0, cap_tokens]), longest bucket first.  The
+// order only steers the persistent attend kernels' work queue (longest items first shortens the tail of a
+// launch); any permutation gives the same results, so ties inside a bucket may land in any order.
+__global__ void __launch_bounds__(1024) order_kernel(const int32_t* __restrict__ len, int n_items, int cap_tokens,
+                                                     int32_t* __restrict__ order) {
+    __shared__ int cnt[1024];
+    __shared__ int base[1024];
+    const int tid = threadIdx.x;
+    cnt[tid] = 0;
+    __syncthreads();
+    auto bucket = [&](int n) {
+        long long bkt = (long long)n * 1023 / (cap_tokens > 0 ? cap_tokens : 1);
+        bkt = bkt < 0 ? 0 : (bkt > 1023 ? 1023 : bkt);
+        return 1023 - (int)bkt;  // bucket 0 = longest
+    };
+    for (int i = tid; i < n_items; i += 1024) atomicAdd(&cnt[bucket(len[i])], 1);
+    __syncthreads();
+    if (tid == 0) {
+        int run = 0;
+        for (int bkt = 0; bkt < 1024; ++bkt) {
+            base[bkt] = run;
+            run += cnt[bkt];
+        }
+    }
+    __syncthreads();
+    for (int i = tid; i < n_items; i += 1024) order[atomicAdd(&base[bucket(len[i])], 1)] = i;
+}
+
+cudaError_t launch_order(const int32_t* len, int n_items, int cap_tokens, int32_t* order, cudaStream_t stream) {
+    order_kernel<<<1, 1024, 0, stream>>>(len, n_items, cap_tokens, order);
+    return cudaGetLastError();
+}
+
 }  // namespace lethe
 
 // ------------------------------------------------------------------ retention with no allocation at all

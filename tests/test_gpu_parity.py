@@ -394,3 +394,48 @@ def test_persistent_logit_overflow(ctx, variant, Hq, Hkv, cap):
     finally:
         ctx.set_tuning(0, 0)
         oracle.set_threads(1)
+
+
+def test_free_running_overlap_llama_shape(ctx):
+    """End to end on its own scores: the GPU runs a Llama-8B-shaped trajectory (2 sequences, all layers, three
+    prune rounds) without being re-synchronised to the oracle; the retained sets of both are compared at the
+    end.  Budgets and lengths must agree exactly whenever the fp32 sparsities round to the same weights; the
+    retained sets may differ only where two scores are within the bf16/fp32 rounding of each other."""
+    oracle.set_threads(min(8, oracle.max_threads()))
+    try:
+        w = synth.shrink(synth.WORKLOADS["llama8b"], batch=2, prune_interval=8)
+        n0, cap = 260, 300
+        oc = cache_from_state(w, synth.initial_kv(w, n0, cap), cap)
+        gc = to_device(oc)
+        dev = gc.device
+        scale = synth.layer_scales(w)
+        T = torch.full((2,), w.n_layers * 180, dtype=torch.int64)
+        S = torch.zeros((w.n_layers, 2), dtype=torch.float32, device=dev)
+        bud = torch.zeros((w.n_layers, 2), dtype=torch.int32, device=dev)
+        for step in range(24):
+            x = synth.step_inputs(w, step)
+            st, *_ = oracle.decode_attend(oc, 0, w.n_layers, x["q"], x["k_new"], x["v_new"], x["token_pos"], scale, w.gamma)
+            assert st == oracle.OK
+            out = torch.empty_like(x["q"], device=dev)
+            ctx.decode_attend(gc, 0, w.n_layers, x["q"].to(dev), x["k_new"].to(dev), x["v_new"].to(dev),
+                              x["token_pos"].to(dev), scale.tolist(), w.gamma, out)
+            if (step + 1) % w.prune_interval == 0:
+                oracle_prune_round(oc, T, w.k_min, w.recent, w.sink)
+                ctx.estimate_sparsity(gc, S); ctx.alloc_budgets(S, T.to(dev), w.k_min, bud)
+                ctx.rasr_prune(gc, bud, w.recent, w.sink)
+        assert ctx.poll_status()[0] == 0
+        glen, olen = gc.len.cpu(), oc.len
+        same_len = (glen == olen).float().mean().item()
+        jac = []
+        gpos, opos = gc.pos.cpu(), oc.pos
+        for l in range(w.n_layers):
+            for b in range(2):
+                for h in range(w.n_kv_heads):
+                    a = set(gpos[l, b, h, :int(glen[l, b, h])].tolist()); o = set(opos[l, b, h, :int(olen[l, b, h])].tolist())
+                    jac.append(len(a & o) / max(1, len(a | o)))
+        jac = torch.tensor(jac)
+        print(f"free-running llama8b-shaped: items with equal length {same_len:.3f}; retained-set Jaccard "
+              f"min {jac.min():.4f} mean {jac.mean():.4f}")
+        assert jac.mean() > 0.97 and jac.min() > 0.8
+    finally:
+        oracle.set_threads(1)
