@@ -178,7 +178,7 @@ __device__ __forceinline__ void block_scan(int v, int* warp_buf, int& ex, int& t
  *  4. rows move in waves of ascending destinations: load wave -> barrier -> store wave.  Because the
  *     destination of a survivor never exceeds its source and waves ascend, no unread source is overwritten.
  */
-__global__ void __launch_bounds__(kPruneThreads) rasr_prune_kernel(CacheView c, const int32_t* __restrict__ budgets,
+__global__ void __launch_bounds__(kPruneThreads, 2) rasr_prune_kernel(CacheView c, const int32_t* __restrict__ budgets,
                                                                    int recent, int sink, int32_t* keep_idx, int max_k,
                                                                    int smem_tokens, int32_t* list_scratch,
                                                                    int32_t* status) {
@@ -375,14 +375,20 @@ __global__ void __launch_bounds__(1024) order_kernel(const int32_t* __restrict__
     };
     for (int i = tid; i < n_items; i += 1024) atomicAdd(&cnt[bucket(len[i])], 1);
     __syncthreads();
-    if (tid == 0) {
-        int run = 0;
-        for (int bkt = 0; bkt < 1024; ++bkt) {
-            base[bkt] = run;
-            run += cnt[bkt];
+    {   // exclusive prefix over the 1024 buckets (Hillis-Steele in shared memory)
+        base[tid] = cnt[tid];
+        __syncthreads();
+        for (int off = 1; off < 1024; off <<= 1) {
+            const int add = tid >= off ? base[tid - off] : 0;
+            __syncthreads();
+            base[tid] += add;
+            __syncthreads();
         }
+        const int incl = base[tid];
+        __syncthreads();
+        base[tid] = incl - cnt[tid];
+        __syncthreads();
     }
-    __syncthreads();
     for (int i = tid; i < n_items; i += 1024) order[atomicAdd(&base[bucket(len[i])], 1)] = i;
 }
 
