@@ -65,6 +65,9 @@ def lib():
         _lib.oracle_rasr_prune.restype = ctypes.c_int
         _lib.oracle_rasr_prune.argtypes = [ctypes.POINTER(_CCache), ctypes.c_void_p, ctypes.c_int32,
                                            ctypes.c_int32, ctypes.c_void_p, ctypes.c_int32]
+        _lib.oracle_segment_prune.restype = ctypes.c_int
+        _lib.oracle_segment_prune.argtypes = [ctypes.POINTER(_CCache), ctypes.c_int32, ctypes.c_float, ctypes.c_int32,
+                                              ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32]
         _lib.oracle_set_threads.argtypes = [ctypes.c_int]
         _lib.oracle_get_threads.restype = ctypes.c_int
         _lib.oracle_max_threads.restype = ctypes.c_int
@@ -182,4 +185,17 @@ def rasr_prune(cache: OracleCache, budgets: torch.Tensor, recent: int, sink: int
     cc = cache._c()
     st = lib().oracle_rasr_prune(ctypes.byref(cc), _ptr(budgets.contiguous()), int(recent), int(sink),
                                  _ptr(keep), int(max_k))
+    return st, keep
+
+
+def segment_prune(cache: OracleCache, n_segments: int, tau: float, recent: int, sink: int, l_evict: torch.Tensor,
+                  max_k: int = 0):
+    """Algorithm 1 in place (l_evict [L][B][Hkv] int32 is updated); returns (status, keep_idx or None)."""
+    assert l_evict.dtype == torch.int32 and tuple(l_evict.shape) == (cache.n_layers, cache.batch, cache.n_kv_heads)
+    keep = None
+    if max_k > 0:
+        keep = torch.zeros((cache.n_layers, cache.batch, cache.n_kv_heads, max_k), dtype=torch.int32)
+    cc = cache._c()
+    st = lib().oracle_segment_prune(ctypes.byref(cc), int(n_segments), ctypes.c_float(tau), int(recent), int(sink),
+                                    _ptr(l_evict), _ptr(keep), int(max_k))
     return st, keep

@@ -25,6 +25,12 @@
  *   oracle_rasr_prune         Sec. 4.3 last paragraph + Algorithm 1 (top-k by
  *                             score, sinks and the recent window always kept),
  *                             multi-round carry-over of Sec. 4.4.
+ *   oracle_segment_prune      Algorithm 1 as a whole (segmented breakpoint search
+ *                             of Sec. 4.2 / Eq. 4, retention set, eviction-threshold
+ *                             update) with the size trigger of Sec. 4.1, applied per
+ *                             (sequence, KV head).  Eq. 4 is read as
+ *                             v_head >= tau * v_cut (as printed, v_head / v_cut <= tau
+ *                             with tau > 1 could only fire at the first cut or never).
  *
  * Arithmetic: every floating-point step is done in double; stored results are
  * rounded once to their storage type (fp32, or bf16 round-to-nearest-even).
@@ -451,4 +457,88 @@ int oracle_rasr_prune(oracle_cache *c, const int32_t *budgets, int32_t recent, i
         free(keep);
     }
     return result;
+}
+
+/* ---- Algorithm 1: segmented breakpoint, retention set, eviction threshold ---- */
+/*
+ * For every (layer, sequence, KV head) with n = len tokens and threshold Le = l_evict[item]:
+ *   n <= Le : not triggered (Sec. 4.1): nothing changes.
+ *   else    : sort the scores (descending, equal scores: lower slot first); cut points
+ *             c_d = floor(n d / D), d = 1..D-1; the breakpoint is the first c_d with
+ *             top[0] >= tau * top[c_d] (one fp32 multiply, fp32 compare);
+ *             found    : keep the first `sink` slots, the last `recent` slots and the
+ *                        breakpoint highest-scoring slots; compact as oracle_rasr_prune
+ *                        does; Le <- max(Le, breakpoint + recent);
+ *             not found: keep everything ("conservatively delay pruning");
+ *                        Le <- min(2 Le, 2^30).
+ * l_evict [L][B][Hkv] int32 is read and updated in place.  keep_idx as in oracle_rasr_prune.
+ */
+int oracle_segment_prune(oracle_cache *c, int32_t n_segments, float tau, int32_t recent, int32_t sink,
+                         int32_t *l_evict, int32_t *keep_idx, int32_t max_k) {
+    int st = check_cache(c);
+    if (st) return st;
+    if (!l_evict || n_segments < 2 || !(tau >= 1.0f) || recent < 0 || sink < 0) return ORACLE_ERR_INVALID_ARG;
+    if (keep_idx && max_k < 1) return ORACLE_ERR_INVALID_ARG;
+    const int64_t capT = cap_tokens(c);
+    const size_t row_bytes = (size_t)c->head_dim * elt_size(c->dtype);
+    const int n_items = c->n_layers * c->batch * c->n_kv_heads;
+    for (int w = 0; w < n_items; ++w) {
+        const int64_t item = w;
+        const int64_t n = c->len[item];
+        const int64_t Le = l_evict[item];
+        int32_t *kout = keep_idx ? keep_idx + item * max_k : NULL;
+        if (kout)
+            for (int i = 0; i < max_k; ++i) kout[i] = (i < n) ? i : -1;
+        if (n <= Le) continue; /* not triggered */
+
+        cand_t *top = (cand_t *)malloc(sizeof(cand_t) * (size_t)n);
+        for (int64_t j = 0; j < n; ++j) {
+            top[j].score = c->rel[item * capT + j];
+            top[j].idx = (int32_t)j;
+        }
+        qsort(top, (size_t)n, sizeof(cand_t), cand_cmp);
+        int64_t breakpoint = -1;
+        for (int d = 1; d < n_segments; ++d) {
+            const int64_t cut = (n * d) / n_segments;
+            if (cut >= n) break;
+            const float v_head = top[0].score, v_cut = top[cut].score;
+            const float rhs = tau * v_cut; /* one IEEE fp32 multiply (no contraction: built with -ffp-contract=off) */
+            if (v_head >= rhs) {
+                breakpoint = cut;
+                break;
+            }
+        }
+        if (breakpoint < 0) { /* no sharp drop: delay pruning */
+            int64_t twice = 2 * Le;
+            if (twice > (1 << 30)) twice = (1 << 30);
+            l_evict[item] = (int32_t)twice;
+            free(top);
+            continue;
+        }
+        char *keep = (char *)calloc((size_t)n, 1);
+        for (int64_t j = 0; j < sink && j < n; ++j) keep[j] = 1;
+        for (int64_t j = (n - recent > 0 ? n - recent : 0); j < n; ++j) keep[j] = 1;
+        for (int64_t i = 0; i < breakpoint; ++i) keep[top[i].idx] = 1;
+        int64_t m = 0;
+        for (int64_t s = 0; s < n; ++s) {
+            if (!keep[s]) continue;
+            if (kout && m < max_k) kout[m] = (int32_t)s;
+            if (s != m) {
+                const int64_t so = row_offset(c, item, s), d_o = row_offset(c, item, m);
+                memmove((char *)c->k + d_o * elt_size(c->dtype), (char *)c->k + so * elt_size(c->dtype), row_bytes);
+                memmove((char *)c->v + d_o * elt_size(c->dtype), (char *)c->v + so * elt_size(c->dtype), row_bytes);
+                c->rel[item * capT + m] = c->rel[item * capT + s];
+                c->pos[item * capT + m] = c->pos[item * capT + s];
+            }
+            ++m;
+        }
+        if (kout)
+            for (int64_t i = m; i < max_k; ++i) kout[i] = -1;
+        c->len[item] = (int32_t)m;
+        const int64_t grown = breakpoint + recent;
+        l_evict[item] = (int32_t)(grown > Le ? grown : Le);
+        free(keep);
+        free(top);
+    }
+    return ORACLE_OK;
 }

@@ -358,3 +358,72 @@ def test_multi_item_budgets_are_per_layer_and_sequence():
                 assert int(c.len[l, b, h]) == min(int(lens[l, b, h]), int(budgets[l, b]))
                 kk = [i for i in keep[l, b, h].tolist() if i >= 0]
                 assert len(kk) == int(c.len[l, b, h]) and kk == sorted(kk)
+
+
+# --------------------------------------------------------------------------- Algorithm 1 (segmented breakpoint)
+
+def _segment_one(rel, D, tau, recent, sink, l_evict, seed=0):
+    n = len(rel)
+    c = random_cache(1, 1, 1, 1, 4, n + 2, n, seed=seed)
+    c.rel[0, 0, 0, :n] = torch.tensor(rel, dtype=torch.float32)
+    before = c.clone()
+    le = torch.tensor([[[l_evict]]], dtype=torch.int32)
+    st, keep = oracle.segment_prune(c, D, tau, recent, sink, le, max_k=n + 2)
+    kept = [i for i in keep[0, 0, 0].tolist() if i >= 0]
+    return st, kept, int(le[0, 0, 0]), c, before
+
+
+def test_golden_segment_prune():
+    g = GOLD["segment"]
+    st, kept, le, c, before = _segment_one(g["rel"], g["segments"], g["tau"], g["recent"], g["sink"], g["l_evict"])
+    assert st == oracle.OK and kept == g["expect_keep"] and le == g["expect_l_evict"]
+    idx = torch.tensor(kept)
+    assert torch.equal(c.k[0, 0, 0, :len(kept)], before.k[0, 0, 0, idx]) and int(c.len[0, 0, 0]) == len(kept)
+    nb = g["no_break"]
+    st, kept, le, c, before = _segment_one(g["rel"], g["segments"], nb["tau"], g["recent"], g["sink"], g["l_evict"])
+    assert kept == nb["expect_keep"] and le == nb["expect_l_evict"] and torch.equal(c.k, before.k)
+    nt = g["not_triggered"]
+    st, kept, le, c, before = _segment_one(g["rel"], g["segments"], g["tau"], g["recent"], g["sink"], nt["l_evict"])
+    assert kept == list(range(8)) and le == nt["expect_l_evict"] and torch.equal(c.rel, before.rel)
+
+
+def test_segment_prune_against_library_sort_and_invariants():
+    """The sort step through torch.sort(stable=True); breakpoint, retention set and threshold update checked
+    against the definitions; tau = 1 always breaks at the first cut, a huge tau never breaks."""
+    g = torch.Generator().manual_seed(23)
+    for trial in range(80):
+        n = int(torch.randint(2, 400, (1,), generator=g)); D = int(torch.randint(2, 12, (1,), generator=g))
+        sink = int(torch.randint(0, 5, (1,), generator=g)); recent = int(torch.randint(0, 40, (1,), generator=g))
+        tau = [1.0, 1.5, 4.0, 50.0, 400.0, 1e30][trial % 6]
+        rel = torch.rand(n, generator=g) ** 6                       # heavy-tailed scores
+        rel[torch.randint(0, n, (n // 4,), generator=g)] = 0.125      # ties
+        le0 = int(torch.randint(0, n + 5, (1,), generator=g))
+        st, kept, le, c, before = _segment_one(rel.tolist(), D, tau, recent, sink, le0, seed=trial)
+        assert st == oracle.OK
+        if n <= le0:
+            assert kept == list(range(n)) and le == le0
+            continue
+        order = torch.sort(rel, descending=True, stable=True)
+        top_v, top_i = order.values, order.indices
+        bp = -1
+        for d in range(1, D):
+            cpt = n * d // D
+            if float(top_v[0]) >= float(torch.tensor(tau, dtype=torch.float32) * top_v[cpt]):
+                bp = cpt; break
+        if tau == 1.0:
+            assert bp == n // D
+        if tau == 1e30 and float(top_v[0]) > 0 and float(top_v[(n * 1) // D]) > 0:
+            assert bp == -1
+        if bp < 0:
+            assert kept == list(range(n)) and le == min(2 * le0, 1 << 30) and torch.equal(c.k, before.k)
+            continue
+        prot = set(range(min(sink, n))) | set(range(max(0, n - recent), n))
+        want = sorted(prot | set(top_i[:bp].tolist()))
+        assert kept == want and le == max(le0, bp + recent)
+        assert bp <= len(kept) <= bp + sink + recent
+        idx = torch.tensor(kept)
+        assert torch.equal(c.k[0, 0, 0, :len(kept)], before.k[0, 0, 0, idx]) and torch.equal(c.pos[0, 0, 0, :len(kept)], before.pos[0, 0, 0, idx])
+        dropped = sorted(set(range(n)) - set(kept))
+        salient = sorted(set(kept) - prot)
+        if dropped and salient:
+            assert rel[salient].min() >= rel[dropped].max()
