@@ -426,6 +426,24 @@ def main():
                      "mode": f"{w.n_layers} launches per step (one per layer), replayed from a CUDA graph, "
                              f"{pl_steps} steps; not part of `value`"}
 
+    # Algorithm 1 (threshold-triggered, budget-free retention) timed once on the live state, after everything
+    # that enters `value`: first with the paper's default sparse_ratio (tau = 400), then with a small tau that
+    # does find breakpoints and therefore also compacts.
+    segment = None
+    if not args.no_per_layer and world == 1:
+        le = torch.zeros_like(r.cache.len)
+        segment = {}
+        for tau in (400.0, 4.0):
+            le.zero_()
+            before = int(r.cache.len.sum().item())
+            a_ev = torch.cuda.Event(enable_timing=True); b_ev = torch.cuda.Event(enable_timing=True)
+            a_ev.record()
+            r.ctx.segment_prune(r.cache, 8, tau, w.recent, w.sink, le)
+            b_ev.record()
+            torch.cuda.synchronize(dev)
+            segment[f"tau_{int(tau)}"] = {"ms": a_ev.elapsed_time(b_ev), "token_heads_before": before,
+                                          "token_heads_after": int(r.cache.len.sum().item())}
+        r.check()
     e_ms = e_total_ms if not args.no_e2e else 0.0
     e_u = float(sum(e_th)) if not args.no_e2e else 0.0
     (t_ms, e_total_ms), (units, e_units) = dist_util.reduce_job(dist, dev, [total_ms, e_ms], [float(sum(th)), e_u])
@@ -450,7 +468,8 @@ def main():
                 "prune_round_ms": (sum(prune_ms) / len(prune_ms)) if prune_ms else None,
                 "attend_ms_per_step": avg_attend_ms,
                 "attend_ms_median": statistics.median(attend_ms),
-                "per_layer_launch": per_layer}),
+                "per_layer_launch": per_layer,
+                "segment_prune_8_segments": segment}),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": f"of {which}", "frac_of_8TBs_nominal": achieved / 8000.0,
                          "kernel": "attend (dominant kernel; one launch per step)",

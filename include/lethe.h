@@ -15,6 +15,8 @@
  *   lethe_alloc_budgets      per-layer token budgets from those sparsities (Sec. 4.2)
  *   lethe_rasr_prune         protected top-k retention + in-place stable compaction
  *                            (Sec. 4.3; sink / recent sets of Algorithm 1)
+ *   lethe_segment_prune      Algorithm 1 itself: segmented breakpoint search, retention
+ *                            set and eviction-threshold update (Sec. 4.2)
  *
  * General conventions
  *   - Unless marked HOST, every pointer is a DEVICE pointer to memory owned by the
@@ -189,6 +191,25 @@ lethe_status lethe_alloc_budgets(lethe_ctx *ctx, int n_layers, int batch, const 
  */
 lethe_status lethe_rasr_prune(lethe_ctx *ctx, const lethe_cache *cache, const int32_t *budgets, int32_t recent,
                               int32_t sink, int32_t *keep_idx, int32_t max_k, void *stream);
+
+/*
+ * Algorithm 1 (segmented attention-based token shrinking) with the size trigger of Sec. 4.1, for every item,
+ * in place — the paper's budget-free retention rule, an alternative to lethe_alloc_budgets + lethe_rasr_prune.
+ * With n = len[item] and Le = l_evict[item]:
+ *   n <= Le: not triggered, the item is not touched.
+ *   else   : order the scores rel[0..n) descending (equal scores: lower slot first); cut points
+ *            c_d = floor(n d / n_segments), d = 1 .. n_segments-1; the breakpoint is the first c_d with
+ *            top[0] >= tau * top[c_d] (one fp32 multiply; Eq. 4 as printed, v_head / v_cut <= tau with tau > 1,
+ *            could only hold at the first cut or never, so it is read the other way round);
+ *            found    : slots j < min(sink, n), slots j >= n - recent and the `breakpoint` highest-scoring slots
+ *                       survive and are compacted exactly as by lethe_rasr_prune; Le <- max(Le, breakpoint + recent);
+ *            not found: nothing is pruned ("conservatively delay pruning"); Le <- min(2 Le, 2^30).
+ *   n_segments >= 2; tau >= 1 (the paper's sparse_ratio, 400 by default); l_evict [L][B][Hkv] int32, read and
+ *   updated; keep_idx / max_k as in lethe_rasr_prune.
+ */
+lethe_status lethe_segment_prune(lethe_ctx *ctx, const lethe_cache *cache, int32_t n_segments, float tau,
+                                 int32_t recent, int32_t sink, int32_t *l_evict, int32_t *keep_idx, int32_t max_k,
+                                 void *stream);
 
 /*
  * lethe_rasr_prune without a context and without any allocation.  (The paper has no counterpart: this entry

@@ -23,7 +23,7 @@ VARIANT_AUTO, VARIANT_SIMT, VARIANT_MMA4, VARIANT_MMA8 = 0, 1, 2, 3
 
 EXPORTS = ["lethe_create", "lethe_destroy", "lethe_last_error", "lethe_poll_status", "lethe_set_tuning",
            "lethe_decode_attend", "lethe_decode_attend_host", "lethe_estimate_sparsity", "lethe_alloc_budgets",
-           "lethe_rasr_prune", "lethe_rasr_prune_static"]
+           "lethe_rasr_prune", "lethe_rasr_prune_static", "lethe_segment_prune"]
 
 
 class LetheError(RuntimeError):
@@ -77,6 +77,8 @@ def load() -> ctypes.CDLL:
     lib.lethe_alloc_budgets.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp, vp, i32, vp, vp]
     lib.lethe_rasr_prune.restype = ctypes.c_int
     lib.lethe_rasr_prune.argtypes = [vp, cp, vp, i32, i32, vp, i32, vp]
+    lib.lethe_segment_prune.restype = ctypes.c_int
+    lib.lethe_segment_prune.argtypes = [vp, cp, i32, ctypes.c_float, i32, i32, vp, vp, i32, vp]
     lib.lethe_rasr_prune_static.restype = ctypes.c_int
     lib.lethe_rasr_prune_static.argtypes = [cp, vp, i32, i32, vp, i32, vp, vp]
     _lib = lib
@@ -223,3 +225,13 @@ class Context:
             max_k = keep_idx.shape[-1]
         self._check(self.lib.lethe_rasr_prune(self.h, ctypes.byref(cache.c), _dp(budgets), recent, sink,
                                               _dp(keep_idx), max_k, _stream(self.device)))
+
+    def segment_prune(self, cache: Cache, n_segments: int, tau: float, recent: int, sink: int, l_evict: torch.Tensor,
+                      keep_idx: Optional[torch.Tensor] = None):
+        assert l_evict.dtype == torch.int32 and l_evict.is_cuda and l_evict.is_contiguous()
+        max_k = 0
+        if keep_idx is not None:
+            assert keep_idx.dtype == torch.int32 and keep_idx.is_cuda
+            max_k = keep_idx.shape[-1]
+        self._check(self.lib.lethe_segment_prune(self.h, ctypes.byref(cache.c), n_segments, tau, recent, sink,
+                                                 _dp(l_evict), _dp(keep_idx), max_k, _stream(self.device)))

@@ -20,6 +20,9 @@ size_t async_smem_bytes(int D, int shape, int chunk_tokens, int GP);
 cudaError_t launch_sparsity(const CacheView& c, float* sparsity, cudaStream_t stream);
 cudaError_t launch_budgets(int L, int B, const float* sparsity, const long long* total, int k_min, int32_t* budgets,
                            int32_t* status, cudaStream_t stream);
+cudaError_t launch_segment_prune(const CacheView& c, int n_segments, float tau, int recent, int sink, int32_t* l_evict,
+                                 int32_t* keep_idx, int max_k, int smem_tokens, int32_t* list_scratch, int32_t* status,
+                                 cudaStream_t stream);
 cudaError_t launch_order(const int32_t* len, int n_items, int cap_tokens, int32_t* order, cudaStream_t stream);
 cudaError_t launch_rasr_prune(const CacheView& c, const int32_t* budgets, int recent, int sink, int32_t* keep_idx,
                               int max_k, int smem_tokens, int32_t* list_scratch, int32_t* status,
@@ -459,6 +462,39 @@ lethe_status lethe_alloc_budgets(lethe_ctx* ctx, int n_layers, int batch, const 
     return LETHE_OK;
 }
 
+// Shared by the two retention entry points: where the survivor lists live, then the longest-first item order.
+static lethe_status prune_scratch(lethe_ctx* ctx, const CacheView& v, int* smem_tokens, int32_t** list_scratch) {
+    // keys / source list live in shared memory when an item fits; otherwise the list goes to global scratch
+    const size_t budget_smem = ctx->max_smem - 8 * 1024;
+    *smem_tokens = v.cap_tokens;
+    *list_scratch = nullptr;
+    if ((size_t)*smem_tokens * 4 > budget_smem) {
+        *smem_tokens = (int)(budget_smem / 4);
+        const size_t need = (size_t)v.L * v.B * v.Hkv * v.cap_tokens * sizeof(int32_t);
+        lethe_status st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "prune scratch");
+        if (st != LETHE_OK) return st;
+        *list_scratch = (int32_t*)ctx->scratch;
+    }
+    return LETHE_OK;
+}
+
+static lethe_status refresh_order(lethe_ctx* ctx, const lethe_cache* c, const CacheView& v, void* stream) {
+    // longest-first order of the items for the persistent attend kernels' work queue
+    const long long items = (long long)v.L * v.B * v.Hkv;
+    ctx->order_len = nullptr;
+    if (items >= 2LL * ctx->sm_count && items <= (1 << 20)) {
+        void* buf = ctx->order;
+        lethe_status st = ensure(ctx, &buf, &ctx->order_bytes, (size_t)items * sizeof(int32_t), "item order");
+        ctx->order = (int32_t*)buf;
+        if (st != LETHE_OK) return st;
+        cudaError_t e = launch_order(c->len, (int)items, v.cap_tokens, ctx->order, (cudaStream_t)stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "item order launch");
+        ctx->order_len = c->len;
+        ctx->order_items = (int)items;
+    }
+    return LETHE_OK;
+}
+
 lethe_status lethe_rasr_prune(lethe_ctx* ctx, const lethe_cache* c, const int32_t* budgets, int32_t recent,
                               int32_t sink, int32_t* keep_idx, int32_t max_k, void* stream) {
     lethe_status st = check_cache(ctx, c);
@@ -469,34 +505,36 @@ lethe_status lethe_rasr_prune(lethe_ctx* ctx, const lethe_cache* c, const int32_
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, LETHE_ERR_CUDA, "cannot select the context's device");
     const CacheView v = view_of(c);
-    // keys / source list live in shared memory when an item fits; otherwise the list goes to global scratch
-    const size_t budget_smem = ctx->max_smem - 8 * 1024;
-    int smem_tokens = v.cap_tokens;
-    int32_t* list_scratch = nullptr;
-    if ((size_t)smem_tokens * 4 > budget_smem) {
-        smem_tokens = (int)(budget_smem / 4);
-        const size_t need = (size_t)v.L * v.B * v.Hkv * v.cap_tokens * sizeof(int32_t);
-        st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "prune scratch");
-        if (st != LETHE_OK) return st;
-        list_scratch = (int32_t*)ctx->scratch;
-    }
+    int smem_tokens;
+    int32_t* list_scratch;
+    st = prune_scratch(ctx, v, &smem_tokens, &list_scratch);
+    if (st != LETHE_OK) return st;
     cudaError_t e = launch_rasr_prune(v, budgets, recent, sink, keep_idx, keep_idx ? max_k : 0, smem_tokens,
                                       list_scratch, ctx->status, (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "rasr_prune launch");
-    // longest-first order of the items for the persistent attend kernels' work queue
-    const long long items = (long long)v.L * v.B * v.Hkv;
-    ctx->order_len = nullptr;
-    if (items >= 2LL * ctx->sm_count && items <= (1 << 20)) {
-        void* buf = ctx->order;
-        st = ensure(ctx, &buf, &ctx->order_bytes, (size_t)items * sizeof(int32_t), "item order");
-        ctx->order = (int32_t*)buf;
-        if (st != LETHE_OK) return st;
-        e = launch_order(c->len, (int)items, v.cap_tokens, ctx->order, (cudaStream_t)stream);
-        if (e != cudaSuccess) return cuda_fail(ctx, e, "item order launch");
-        ctx->order_len = c->len;
-        ctx->order_items = (int)items;
-    }
-    return LETHE_OK;
+    return refresh_order(ctx, c, v, stream);
+}
+
+lethe_status lethe_segment_prune(lethe_ctx* ctx, const lethe_cache* c, int32_t n_segments, float tau, int32_t recent,
+                                 int32_t sink, int32_t* l_evict, int32_t* keep_idx, int32_t max_k, void* stream) {
+    lethe_status st = check_cache(ctx, c);
+    if (st != LETHE_OK) return st;
+    if (!l_evict) return fail(ctx, LETHE_ERR_INVALID_ARG, "l_evict is NULL");
+    if (n_segments < 2) return fail(ctx, LETHE_ERR_INVALID_ARG, "n_segments must be at least 2");
+    if (!(tau >= 1.0f)) return fail(ctx, LETHE_ERR_INVALID_ARG, "tau must be >= 1");
+    if (recent < 0 || sink < 0) return fail(ctx, LETHE_ERR_INVALID_ARG, "recent and sink must be >= 0");
+    if (keep_idx && max_k < 1) return fail(ctx, LETHE_ERR_INVALID_ARG, "max_k must be positive with keep_idx");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, LETHE_ERR_CUDA, "cannot select the context's device");
+    const CacheView v = view_of(c);
+    int smem_tokens;
+    int32_t* list_scratch;
+    st = prune_scratch(ctx, v, &smem_tokens, &list_scratch);
+    if (st != LETHE_OK) return st;
+    cudaError_t e = launch_segment_prune(v, n_segments, tau, recent, sink, l_evict, keep_idx, keep_idx ? max_k : 0,
+                                         smem_tokens, list_scratch, ctx->status, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "segment_prune launch");
+    return refresh_order(ctx, c, v, stream);
 }
 
 }  // extern "C"

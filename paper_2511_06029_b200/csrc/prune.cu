@@ -167,117 +167,82 @@ __device__ __forceinline__ void block_scan(int v, int* warp_buf, int& ex, int& t
     __syncthreads();
 }
 
-/*
- * One CTA per item.
- *  1. keys: score_key(rel[j]) into shared memory (or re-read from global when the item is too long).
- *  2. 4-pass, 8-bit radix select of the `take`-th largest candidate key -> threshold T, count above it.
- *  3. ascending sweep: keep = protected | key > T | (key == T and among the first need_eq such slots);
- *     block scans turn the keep flags into destination slots; the source slot of every destination is
- *     written to a list (shared memory, in place over the keys; global scratch for items longer than
- *     smem_tokens, whose keys are then re-read from rel).
- *  4. rows move in waves of ascending destinations: load wave -> barrier -> store wave.  Because the
- *     destination of a survivor never exceeds its source and waves ascend, no unread source is overwritten.
- */
-__global__ void __launch_bounds__(kPruneThreads, 2) rasr_prune_kernel(CacheView c, const int32_t* __restrict__ budgets,
-                                                                   int recent, int sink, int32_t* keep_idx, int max_k,
-                                                                   int smem_tokens, int32_t* list_scratch,
-                                                                   int32_t* status) {
-    extern __shared__ __align__(16) uint32_t dyn[];  // keys, later the source list  [smem_tokens]
-    __shared__ int hist[256];
-    __shared__ int warp_buf[kPruneThreads / 32];
-    __shared__ uint32_t sel_prefix;
-    __shared__ int sel_remaining;
+struct PruneShared {
+    int hist[256];
+    int warp_buf[kPruneThreads / 32];
+    uint32_t sel_prefix;
+    int sel_remaining;
+    float bcast;
+    int ibcast;
+};
 
-    const size_t item = blockIdx.x;
+// take-th largest key (take >= 1) among slots [lo, hi): 4 passes of an 8-bit radix select.  T receives that key
+// and need_eq how many of the slots equal to T belong to the top `take` (the oldest ones are meant).
+template <class KeyAt>
+__device__ __forceinline__ void radix_select(PruneShared& sh, KeyAt key_at, int lo, int hi, int take, uint32_t& T,
+                                             int& need_eq) {
     const int tid = threadIdx.x;
-    const int l = (int)(item / ((size_t)c.B * c.Hkv));
-    const int b = (int)((item / c.Hkv) % c.B);
-    const int n = c.len[item];
-    long long k = budgets[(size_t)l * c.B + b];
-    if (k < 0) k = 0;
-    int32_t* kout = keep_idx ? keep_idx + item * max_k : nullptr;
-    if (k >= n) {  // identity
-        if (kout)
-            for (int i = tid; i < max_k; i += kPruneThreads) kout[i] = (i < n) ? i : -1;
-        return;
+    if (tid == 0) {
+        sh.sel_prefix = 0u;
+        sh.sel_remaining = take;
     }
-    const int n_sink = min(sink, n), n_recent = min(recent, n);
-    const int cand_lo = n_sink;
-    const int cand_hi = max(n - n_recent, cand_lo);
-    const int n_prot = n - (cand_hi - cand_lo);
-    if (n_prot > k) {
-        k = n_prot;
-        if (tid == 0) record_error(status, LETHE_ERR_BUDGET, (int)item);
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        const uint32_t mask_hi = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+        if (tid < 256) sh.hist[tid] = 0;
+        __syncthreads();
+        const uint32_t prefix = sh.sel_prefix;
+        for (int j = lo + tid; j < hi; j += kPruneThreads) {
+            const uint32_t key = key_at(j);
+            if ((key & mask_hi) == prefix) atomicAdd(&sh.hist[(key >> shift) & 0xffu], 1);
+        }
+        __syncthreads();
+        // bin holding the remaining-th largest key: suffix sums over the 256 bins by one block scan
+        const int remaining = sh.sel_remaining;
+        const int h = tid < 256 ? sh.hist[255 - tid] : 0;  // thread t looks at bin 255 - t
+        int ex, tot;
+        block_scan(h, sh.warp_buf, ex, tot);               // ex = keys in bins above this thread's bin
+        if (tid < 256 && ex < remaining && ex + h >= remaining) {
+            sh.sel_prefix = prefix | ((uint32_t)(255 - tid) << shift);
+            sh.sel_remaining = remaining - ex;
+        }
+        __syncthreads();
     }
-    const int keep_n = (int)k;
-    const int take = keep_n - n_prot;
-    float* rel = c.rel + item * c.cap_tokens;
-    int32_t* pos = c.pos + item * c.cap_tokens;
-    const bool in_smem = n <= smem_tokens;
-
-    if (in_smem)
-        for (int j = tid; j < n; j += kPruneThreads) dyn[j] = score_key(rel[j]);
+    T = sh.sel_prefix;
+    need_eq = sh.sel_remaining;
     __syncthreads();
-    auto key_at = [&](int j) -> uint32_t { return in_smem ? dyn[j] : score_key(rel[j]); };
+}
 
-    // ---- radix select: T = take-th largest candidate key (take >= 1), n_gt = candidates above T
-    uint32_t T = 0xffffffffu;
-    int need_eq = 0;
-    if (take > 0) {
-        if (tid == 0) {
-            sel_prefix = 0u;
-            sel_remaining = take;
-        }
-        for (int pass = 0; pass < 4; ++pass) {
-            const int shift = 24 - 8 * pass;
-            const uint32_t mask_hi = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
-            if (tid < 256) hist[tid] = 0;
-            __syncthreads();
-            const uint32_t prefix = sel_prefix;
-            for (int j = cand_lo + tid; j < cand_hi; j += kPruneThreads) {
-                const uint32_t key = key_at(j);
-                if ((key & mask_hi) == prefix) atomicAdd(&hist[(key >> shift) & 0xffu], 1);
-            }
-            __syncthreads();
-            {   // bin holding the remaining-th largest key: suffix sums over the 256 bins by one block scan
-                const int remaining = sel_remaining;
-                const int h = tid < 256 ? hist[255 - tid] : 0;  // thread t looks at bin 255 - t
-                int ex, tot;
-                block_scan(h, warp_buf, ex, tot);               // ex = keys in bins above this thread's bin
-                if (tid < 256 && ex < remaining && ex + h >= remaining) {
-                    sel_prefix = prefix | ((uint32_t)(255 - tid) << shift);
-                    sel_remaining = remaining - ex;
-                }
-                __syncthreads();
-            }
-        }
-        T = sel_prefix;
-        need_eq = sel_remaining;  // how many slots equal to T are kept (the oldest ones)
-    }
-
-    // ---- ascending sweep: destinations by prefix sums; source list written over consumed keys
-    int32_t* src_list = in_smem ? reinterpret_cast<int32_t*>(dyn) : list_scratch + item * c.cap_tokens;
+// Ascending sweep over slots [0, n): a slot survives if it is protected (j < prot_lo or j >= prot_hi) or if it
+// lies in [sel_lo, sel_hi) and is selected (key > T, or key == T among the first need_eq such slots).  Block
+// scans turn the flags into destination slots; the source slot of every destination goes to src_list (which
+// may alias the key array: a destination never exceeds its source, and a chunk's keys are read before its
+// scans' barriers) and to kout.  Returns the number of survivors.
+template <class KeyAt>
+__device__ __forceinline__ int sweep_keep(PruneShared& sh, KeyAt key_at, int n, int prot_lo, int prot_hi, int sel_lo,
+                                          int sel_hi, bool any_selected, uint32_t T, int need_eq, int32_t* src_list,
+                                          int32_t* kout, int max_k) {
+    const int tid = threadIdx.x;
     int run_keep = 0, run_eq = 0;
     for (int base = 0; base < n; base += kPruneThreads) {
         const int j = base + tid;
         int is_keep = 0, is_eq = 0;
-        uint32_t key = 0;
         if (j < n) {
-            if (j < cand_lo || j >= cand_hi) is_keep = 1;
-            else if (take > 0) {
-                key = key_at(j);
+            if (j < prot_lo || j >= prot_hi) is_keep = 1;
+            if (any_selected && j >= sel_lo && j < sel_hi) {
+                const uint32_t key = key_at(j);
                 if (key > T) is_keep = 1;
                 else if (key == T) is_eq = 1;
             }
         }
         int ex_keep, ex_eq, tot_keep, tot_eq;
         // first the rank among slots equal to the threshold (slot order), then the keep scan that depends on it
-        block_scan(is_eq, warp_buf, ex_eq, tot_eq);
+        block_scan(is_eq, sh.warp_buf, ex_eq, tot_eq);
         if (is_eq && run_eq + ex_eq < need_eq) is_keep = 1;
-        block_scan(is_keep, warp_buf, ex_keep, tot_keep);
+        block_scan(is_keep, sh.warp_buf, ex_keep, tot_keep);
         if (is_keep) {
             const int dst = run_keep + ex_keep;
-            src_list[dst] = j;  // dst <= j, and every key of this chunk was read before the scans' barriers
+            src_list[dst] = j;
             if (kout && dst < max_k) kout[dst] = j;
         }
         run_keep += tot_keep;
@@ -285,16 +250,22 @@ __global__ void __launch_bounds__(kPruneThreads, 2) rasr_prune_kernel(CacheView 
     }
     __syncthreads();
     if (kout)
-        for (int i = keep_n + tid; i < max_k; i += kPruneThreads) kout[i] = -1;
+        for (int i = run_keep + tid; i < max_k; i += kPruneThreads) kout[i] = -1;
+    return run_keep;
+}
 
-    // ---- move rows in ascending waves
+// Rows of K, V, rel, pos move to their destinations in ascending waves: load wave -> barrier -> store wave.
+// Because a survivor's destination never exceeds its source and waves ascend, no unread source is overwritten.
+__device__ __forceinline__ void move_rows(const CacheView& c, size_t item, int keep_n, const int32_t* src_list, bool& bad) {
+    const int tid = threadIdx.x;
+    float* rel = c.rel + item * c.cap_tokens;
+    int32_t* pos = c.pos + item * c.cap_tokens;
     const int row_bytes = c.D * c.elt_bytes;
     const int lanes_per_row = row_bytes / 16;            // 16-byte pieces per row (8, 16 or 32)
     constexpr int RPT = 4;                               // rows each thread slot carries per wave
     const int slots = kPruneThreads / lanes_per_row;     // row slots per pass
     const int rows_per_wave = slots * RPT;
     const int piece = tid % lanes_per_row, rslot = tid / lanes_per_row;
-    bool bad = false;
     // destinations whose source is themselves (the unmoved prefix, and any later fixed point) are skipped
     for (int w0 = 0; w0 < keep_n; w0 += rows_per_wave) {
         uint4 kv[RPT], vv[RPT];
@@ -342,8 +313,152 @@ __global__ void __launch_bounds__(kPruneThreads, 2) rasr_prune_kernel(CacheView 
         }
         // no barrier needed here: the next wave's sources lie above every destination written so far
     }
+}
+
+/*
+ * RASR retention, one CTA per item.
+ *  1. keys: score_key(rel[j]) into shared memory (or re-read from global when the item is too long).
+ *  2. radix select of the `take`-th largest candidate key -> threshold T.
+ *  3. ascending sweep -> destination of every survivor (source list in shared memory, in place over the keys;
+ *     global scratch for items longer than smem_tokens).
+ *  4. rows move in ascending waves.
+ */
+__global__ void __launch_bounds__(kPruneThreads, 2) rasr_prune_kernel(CacheView c, const int32_t* __restrict__ budgets,
+                                                                   int recent, int sink, int32_t* keep_idx, int max_k,
+                                                                   int smem_tokens, int32_t* list_scratch,
+                                                                   int32_t* status) {
+    extern __shared__ __align__(16) uint32_t dyn[];  // keys, later the source list  [smem_tokens]
+    __shared__ PruneShared sh;
+
+    const size_t item = blockIdx.x;
+    const int tid = threadIdx.x;
+    const int l = (int)(item / ((size_t)c.B * c.Hkv));
+    const int b = (int)((item / c.Hkv) % c.B);
+    const int n = c.len[item];
+    long long k = budgets[(size_t)l * c.B + b];
+    if (k < 0) k = 0;
+    int32_t* kout = keep_idx ? keep_idx + item * max_k : nullptr;
+    if (k >= n) {  // identity
+        if (kout)
+            for (int i = tid; i < max_k; i += kPruneThreads) kout[i] = (i < n) ? i : -1;
+        return;
+    }
+    const int n_sink = min(sink, n), n_recent = min(recent, n);
+    const int cand_lo = n_sink;
+    const int cand_hi = max(n - n_recent, cand_lo);
+    const int n_prot = n - (cand_hi - cand_lo);
+    if (n_prot > k) {
+        k = n_prot;
+        if (tid == 0) record_error(status, LETHE_ERR_BUDGET, (int)item);
+    }
+    const int take = (int)k - n_prot;
+    const float* rel = c.rel + item * c.cap_tokens;
+    const bool in_smem = n <= smem_tokens;
+
+    if (in_smem)
+        for (int j = tid; j < n; j += kPruneThreads) dyn[j] = score_key(rel[j]);
+    __syncthreads();
+    auto key_at = [&](int j) -> uint32_t { return in_smem ? dyn[j] : score_key(rel[j]); };
+
+    uint32_t T = 0xffffffffu;
+    int need_eq = 0;
+    if (take > 0) radix_select(sh, key_at, cand_lo, cand_hi, take, T, need_eq);
+
+    int32_t* src_list = in_smem ? reinterpret_cast<int32_t*>(dyn) : list_scratch + item * c.cap_tokens;
+    const int keep_n = sweep_keep(sh, key_at, n, cand_lo, cand_hi, cand_lo, cand_hi, take > 0, T, need_eq, src_list, kout, max_k);
+    bool bad = false;
+    move_rows(c, item, keep_n, src_list, bad);
     if (bad && tid == 0) record_error(status, LETHE_ERR_PAGE, (int)item);
     if (tid == 0) c.len[item] = keep_n;
+}
+
+/*
+ * Algorithm 1 (segmented attention-based token shrinking), one CTA per item, with the size trigger of Sec. 4.1.
+ *  n <= l_evict: untouched.  Otherwise the value at every cut point floor(n d / D) of the descending order is
+ *  found with a radix select (no full sort), the first cut with v_head >= tau * v_cut is the breakpoint, the
+ *  breakpoint highest scores plus sinks plus the recent window survive (same sweep and row moves as the RASR
+ *  kernel), and l_evict grows to max(l_evict, breakpoint + recent); without a breakpoint nothing is pruned and
+ *  l_evict doubles.
+ */
+__global__ void __launch_bounds__(kPruneThreads, 2) segment_prune_kernel(CacheView c, int n_segments, float tau, int recent,
+                                                                      int sink, int32_t* __restrict__ l_evict,
+                                                                      int32_t* keep_idx, int max_k, int smem_tokens,
+                                                                      int32_t* list_scratch, int32_t* status) {
+    extern __shared__ __align__(16) uint32_t dyn[];
+    __shared__ PruneShared sh;
+
+    const size_t item = blockIdx.x;
+    const int tid = threadIdx.x;
+    const int n = c.len[item];
+    const int le = l_evict[item];
+    int32_t* kout = keep_idx ? keep_idx + item * max_k : nullptr;
+    auto identity = [&]() {
+        if (kout)
+            for (int i = tid; i < max_k; i += kPruneThreads) kout[i] = (i < n) ? i : -1;
+    };
+    if (n <= le) {  // not triggered
+        identity();
+        return;
+    }
+    const float* rel = c.rel + item * c.cap_tokens;
+    const bool in_smem = n <= smem_tokens;
+    if (in_smem)
+        for (int j = tid; j < n; j += kPruneThreads) dyn[j] = score_key(rel[j]);
+    __syncthreads();
+    auto key_at = [&](int j) -> uint32_t { return in_smem ? dyn[j] : score_key(rel[j]); };
+    auto key_value = [](uint32_t key) -> float {  // inverse of score_key
+        return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+    };
+
+    // v at a rank of the descending order = (rank + 1)-th largest key
+    uint32_t T;
+    int need_eq;
+    radix_select(sh, key_at, 0, n, 1, T, need_eq);
+    const float v_head = key_value(T);
+    int breakpoint = -1;
+    for (int d = 1; d < n_segments; ++d) {
+        const int cut = (int)(((long long)n * d) / n_segments);
+        if (cut >= n) break;
+        float v_cut = v_head;
+        if (cut > 0) {
+            radix_select(sh, key_at, 0, n, cut + 1, T, need_eq);
+            v_cut = key_value(T);
+        }
+        if (v_head >= __fmul_rn(tau, v_cut)) {
+            breakpoint = cut;
+            break;
+        }
+    }
+    if (breakpoint < 0) {  // no sharp drop: delay pruning, double the threshold
+        identity();
+        if (tid == 0) l_evict[item] = (int32_t)min(2LL * le, (long long)(1 << 30));
+        return;
+    }
+    T = 0xffffffffu;
+    need_eq = 0;
+    if (breakpoint > 0) radix_select(sh, key_at, 0, n, breakpoint, T, need_eq);
+    int32_t* src_list = in_smem ? reinterpret_cast<int32_t*>(dyn) : list_scratch + item * c.cap_tokens;
+    const int keep_n = sweep_keep(sh, key_at, n, min(sink, n), max(n - recent, 0), 0, n, breakpoint > 0, T, need_eq, src_list,
+                                  kout, max_k);
+    bool bad = false;
+    move_rows(c, item, keep_n, src_list, bad);
+    if (bad && tid == 0) record_error(status, LETHE_ERR_PAGE, (int)item);
+    if (tid == 0) {
+        c.len[item] = keep_n;
+        l_evict[item] = max(le, breakpoint + recent);
+    }
+}
+
+cudaError_t launch_segment_prune(const CacheView& c, int n_segments, float tau, int recent, int sink, int32_t* l_evict,
+                                 int32_t* keep_idx, int max_k, int smem_tokens, int32_t* list_scratch, int32_t* status,
+                                 cudaStream_t stream) {
+    const size_t smem = (size_t)smem_tokens * 4;
+    cudaError_t e = prepare_kernel((const void*)segment_prune_kernel, smem);
+    if (e != cudaSuccess) return e;
+    segment_prune_kernel<<<c.L * c.B * c.Hkv, kPruneThreads, smem, stream>>>(c, n_segments, tau, recent, sink, l_evict,
+                                                                            keep_idx, max_k, smem_tokens, list_scratch,
+                                                                            status);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_rasr_prune(const CacheView& c, const int32_t* budgets, int recent, int sink, int32_t* keep_idx,
