@@ -15,7 +15,10 @@ cudaError_t launch_attend_mma(const AttendArgs& a, int D, int shape, bool paged,
 size_t mma_smem_bytes(int D, int shape, int chunk_tokens, int GP);
 cudaError_t launch_attend_stream(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream);
 size_t stream_smem_bytes(int D, int shape, int chunk_tokens, int GP);
-cudaError_t launch_attend_async(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream);
+cudaError_t launch_attend_async(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream, bool tma,
+                                const void* maps);
+bool build_tma_maps(void* encode, void* k, void* v, unsigned long long rows, int D, void* out_maps);
+size_t tma_maps_bytes();
 size_t async_smem_bytes(int D, int shape, int chunk_tokens, int GP);
 cudaError_t launch_sparsity(const CacheView& c, float* sparsity, cudaStream_t stream);
 cudaError_t launch_budgets(int L, int B, const float* sparsity, const long long* total, int k_min, int32_t* budgets,
@@ -77,6 +80,13 @@ struct lethe_ctx {
     void* staging;  // device staging of lethe_decode_attend_host
     size_t staging_bytes;
     int variant, splits;
+    // TMA variant: tensor maps of the last cache seen (rebuilt when k, v, the row count or D change)
+    alignas(64) unsigned char tma_maps[512];
+    const void* tma_k;
+    const void* tma_v;
+    unsigned long long tma_rows;
+    int tma_d;
+    void* tma_encode;  // cuTensorMapEncodeTiled, resolved on first use
 #ifdef LETHE_TIMELINE
     unsigned long long* timeline;
 #endif
@@ -240,7 +250,7 @@ lethe_status lethe_debug_set_timeline(lethe_ctx* ctx, unsigned long long* buf) {
 
 lethe_status lethe_set_tuning(lethe_ctx* ctx, int variant, int splits) {
     if (!ctx) return LETHE_ERR_INVALID_ARG;
-    if (variant < 0 || variant > 23) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..23");
+    if (variant < 0 || variant > 31) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..31");
     if (!(splits == 0 || splits == 1 || splits == 2 || splits == 4 || splits == 8 || splits == 16))
         return fail(ctx, LETHE_ERR_INVALID_ARG, "splits must be 0, 1, 2, 4, 8 or 16");
     ctx->variant = variant;
@@ -333,8 +343,29 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
     cudaError_t e;
     if (variant >= 16) {  // persistent, asynchronous epilogue: both logit buffers (item parity) share what is left
         if (ctx->splits > 1) return fail(ctx, LETHE_ERR_INVALID_ARG, "the persistent variants do not split items");
+        const bool tma = variant >= 24;
+        const int shape = tma ? variant - 24 : variant - 16;
+        if (tma) {  // tensor maps over K and V as [rows][D]
+            const unsigned long long rows = paged ? (unsigned long long)c->n_pages * c->page_tokens
+                                                  : (unsigned long long)c->n_layers * c->batch * c->n_kv_heads * c->capacity;
+            if (rows > 0x7fffffffULL) return fail(ctx, LETHE_ERR_UNSUPPORTED, "cache too large for the TMA variant");
+            if (sizeof(ctx->tma_maps) < tma_maps_bytes()) return fail(ctx, LETHE_ERR_CUDA, "tensor map storage");
+            if (!ctx->tma_encode) {
+                cudaDriverEntryPointQueryResult qres;
+                if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ctx->tma_encode, cudaEnableDefault, &qres) != cudaSuccess ||
+                    qres != cudaDriverEntryPointSuccess || !ctx->tma_encode) {
+                    ctx->tma_encode = nullptr;
+                    return fail(ctx, LETHE_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+                }
+            }
+            if (ctx->tma_k != c->k || ctx->tma_v != c->v || ctx->tma_rows != rows || ctx->tma_d != c->head_dim) {
+                if (!build_tma_maps(ctx->tma_encode, c->k, c->v, rows, c->head_dim, ctx->tma_maps))
+                    return fail(ctx, LETHE_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+                ctx->tma_k = c->k; ctx->tma_v = c->v; ctx->tma_rows = rows; ctx->tma_d = c->head_dim;
+            }
+        }
         a.splits = 1;
-        const size_t fixed = async_smem_bytes(c->head_dim, variant - 16, 0, a.GP);
+        const size_t fixed = async_smem_bytes(c->head_dim, shape, 0, a.GP);
         int fit = 0;
         if (fixed < ctx->max_smem) fit = (int)((ctx->max_smem - fixed) / ((size_t)2 * a.GP * 4) / kGroupTokens) * kGroupTokens;
         a.chunk_tokens = fit < cap_groups * kGroupTokens ? fit : cap_groups * kGroupTokens;
@@ -348,7 +379,7 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
             if (st != LETHE_OK) return st;
             a.spill = (float*)ctx->scratch;
         }
-        e = launch_attend_async(a, c->head_dim, variant - 16, paged, grid, (cudaStream_t)stream);
+        e = launch_attend_async(a, c->head_dim, shape, paged, grid, (cudaStream_t)stream, tma, ctx->tma_maps);
     } else if (variant >= 8) {  // persistent: one CTA per SM walks all items
         if (ctx->splits > 1) return fail(ctx, LETHE_ERR_INVALID_ARG, "the persistent variant does not split items");
         a.splits = 1;

@@ -13,14 +13,22 @@
 #include "common.cuh"
 #include "mma_utils.cuh"
 
-#include <type_traits>
+#include <string.h>
+
+#include <cuda.h>  // CUtensorMap (type only: the encoder is resolved at run time by the host code)
 
 namespace lethe {
 
 constexpr int kEpilogueWarps = 2;
 constexpr int kWaitLimit = 200000;  // polls of a blocking try_wait before giving up
 
+// Tensor maps of K and V for the TMA variant (rows x D, box 16 rows x 64 elements, 128-byte swizzle).
+struct alignas(64) TmaMaps {
+    CUtensorMap k, v;
+};
+
 struct AsyncHeader {
+    unsigned long long tma_full[16][6];  // TMA variant: per warp, per stage slot: the tile has landed
     unsigned long long full[2];   // streaming warps -> epilogue: item's partials are complete
     unsigned long long empty[2];  // epilogue -> streaming warps: parity buffers are free, next descriptor is published
     int desc_ticket[4];           // ring by item sequence number: ticket (>= n_items: no more work)
@@ -45,6 +53,33 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned 
         : "memory");
     return ok != 0;
 }
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, unsigned bytes) {
+    asm volatile("{ .reg .b64 st; mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+// One box (64 elements x 16 rows) of a 2-D tensor map into shared memory; completion is counted on `bar`.
+// x is always 0 or 64 elements (a multiple of 16 bytes), y is a row index.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, unsigned long long* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// Bounded wait for a tile: polls without backing off for a long while (the data is usually microseconds away).
+__device__ __forceinline__ bool mbar_wait_tile(unsigned long long* bar, unsigned parity, volatile int* abort_flag) {
+    for (int it = 0; it < kWaitLimit * 8; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 1023) == 1023) {
+            if (*abort_flag) return false;
+            __nanosleep(200);
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+
 // Bounded wait; false = gave up (or another warp already did).
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, volatile int* abort_flag) {
     for (int it = 0; it < kWaitLimit; ++it) {
@@ -95,8 +130,9 @@ __device__ __noinline__ void append_row(const AttendArgs& a, int item, int li, i
     __syncwarp();
 }
 
-template <int D, int NWS, int NS, bool PAGED, bool SPILL>
-__global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_kernel(const __grid_constant__ AttendArgs a) {
+template <int D, int NWS, int NS, bool PAGED, bool SPILL, bool TMA>
+__global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
+    attend_async_kernel(const __grid_constant__ AttendArgs a, const __grid_constant__ TmaMaps maps) {
     using T = __nv_bfloat16;
     constexpr int ROW_BYTES = D * 2;
     constexpr int CHUNKS = ROW_BYTES / 16;
@@ -106,8 +142,10 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
     constexpr int KS = D / 16;
     constexpr int ET = kEpilogueWarps * 32;
     static_assert(NS >= 2 && NS <= 6 && NWS <= 16, "shape");
-    extern __shared__ __align__(128) unsigned char smem_raw[];
+    extern __shared__ __align__(1024) unsigned char smem_raw[];  // TMA tiles with a 128-byte swizzle need 1 KB alignment
     // layout: stages [NWS][NS][K tile | V tile] | AsyncHeader | wo [2][NWS][GP][D] fp32 | lg [2][chunk][GP] fp32
+    // Tile layout.  cp.async: rows of ROW_BYTES with the 16-byte chunk index XORed by (row & 7).  TMA: one 2 KB box
+    // per 64 elements of D (16 rows x 128 B, chunk index XORed by (row & 7) by the hardware swizzle).
     const int G = a.G, GP = a.GP;
     const int wo_stride = GP * D;  // floats per warp
     AsyncHeader& hd = *reinterpret_cast<AsyncHeader*>(smem_raw + (size_t)NWS * WARP_BYTES);
@@ -128,7 +166,24 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
         mbar_init(&hd.full[1], NWS);
         mbar_init(&hd.empty[0], kEpilogueWarps);
         mbar_init(&hd.empty[1], kEpilogueWarps);
+        if (TMA)
+            for (int w = 0; w < NWS; ++w)
+                for (int sl = 0; sl < NS; ++sl) mbar_init(&hd.tma_full[w][sl], 1);
         hd.abort = 0;
+    }
+    if (TMA && (smem_u32(smem_raw) & 1023u)) {  // would break the hardware swizzle: refuse rather than compute garbage
+        if (tid == 0) record_error(a.status, LETHE_ERR_UNSUPPORTED, (int)blockIdx.x);
+        // still take part in the queue protocol so that the launch ends cleanly
+        if (tid == 0) {
+            (void)atomicAdd(&sched[0], 1u);
+            __threadfence();
+            const unsigned int done = atomicAdd(&sched[1], 1u);
+            if (done == gridDim.x - 1) {
+                sched[0] = 0u;
+                sched[1] = 0u;
+            }
+        }
+        return;
     }
     if (warp == NWS && lane == 0) {
         int t0 = (int)atomicAdd(&sched[0], 1u);
@@ -176,6 +231,9 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
         unsigned char* my_stage = smem_raw + (size_t)warp * WARP_BYTES;
         const uint32_t my_stage_u32 = smem_u32(my_stage);
         bool bad_page = false;
+        unsigned slot_bad = 0;    // TMA: slots whose tile must be ignored (page id outside the pool)
+        unsigned slot_phase = 0;  // TMA: parity of the next completion of each slot's mbarrier
+        unsigned slot_busy = 0;   // TMA: slots with a load in flight or landed but not yet consumed
 
         // PAGED: page ids of this warp's local groups are fetched 32 at a time, one lane each, a block ahead of
         // their use, so that staging a group never waits on a page-table load.
@@ -188,7 +246,13 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
         auto issue = [&](const AsyncItem& it, int idx, int slot, bool is_cur) {
             const int grp = warp + idx * NWS;
             const int tok0 = grp * kGroupTokens;
-            if (idx == it.app_idx) append_row<PAGED>(a, it.item, it.li, it.b, it.hkv, it.n_old, ROW_BYTES, lane);
+            if (idx == it.app_idx) {
+                append_row<PAGED>(a, it.item, it.li, it.b, it.hkv, it.n_old, ROW_BYTES, lane);
+                if (TMA) {  // the row was written through the generic proxy; the TMA load reads through the async proxy
+                    fence_proxy_async();
+                    __syncwarp();
+                }
+            }
             const char* kb;
             const char* vb;
             bool ok = true;
@@ -215,6 +279,23 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
             }
             const uint32_t ks_u32 = my_stage_u32 + slot * STAGE_BYTES;
             const uint32_t vs_u32 = ks_u32 + TILE_BYTES;
+            if constexpr (TMA) {
+                // row index of the group's first token in the 2-D view of the cache (rows x D)
+                const long long row0 = (long long)((kb - (const char*)a.k) / ROW_BYTES);
+                if (!ok) slot_bad |= 1u << slot;
+                else slot_bad &= ~(1u << slot);
+                slot_busy |= 1u << slot;
+                if (lane == 0) {
+                    unsigned long long* bar = &hd.tma_full[warp][slot];
+                    mbar_arrive_expect_tx(bar, STAGE_BYTES);
+#pragma unroll
+                    for (int hx = 0; hx < D / 64; ++hx) {
+                        tma_load_2d(ks_u32 + hx * 2048, &maps.k, hx * 64, (int)row0, bar);
+                        tma_load_2d(vs_u32 + hx * 2048, &maps.v, hx * 64, (int)row0, bar);
+                    }
+                }
+                return;
+            }
 #pragma unroll
             for (int i = 0; i < kGroupTokens * CHUNKS / 32; ++i) {
                 const int c_idx = i * 32 + lane;
@@ -285,8 +366,30 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
 
             constexpr bool OVF = SPILL;
             for (int it = 0; it < cur.count; ++it) {
-                if (topped && it < NS - 1) cp_async_wait<0>();
-                else cp_async_wait<NS - 2>();
+                const int cslot = (vp + it) % NS;
+                if constexpr (TMA) {
+                    if (!mbar_wait_tile(&hd.tma_full[warp][cslot], (slot_phase >> cslot) & 1u, abort_flag)) {
+                        alive = false;
+                        break;
+                    }
+                    slot_phase ^= 1u << cslot;
+                    slot_busy &= ~(1u << cslot);
+                    // rows past the item's end (and tiles of a bad page) hold whatever memory held: V rows must be
+                    // zero so that a zero probability times them stays zero; K rows are masked by the logit test
+                    const int grp_w = warp + it * NWS;
+                    int valid_rows = cur.n - grp_w * kGroupTokens;
+                    if ((slot_bad >> cslot) & 1u) valid_rows = 0;
+                    if (valid_rows < kGroupTokens) {
+                        const uint32_t vt = my_stage_u32 + cslot * STAGE_BYTES + TILE_BYTES;
+                        for (int e = lane; e < (kGroupTokens - valid_rows) * CHUNKS; e += 32) {
+                            const int r = valid_rows + e / CHUNKS, cch = e % CHUNKS;
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vt + (cch >> 3) * 2048 + r * 128 + ((cch & 7) << 4)), "r"(0) : "memory");
+                        }
+                    }
+                } else {
+                    if (topped && it < NS - 1) cp_async_wait<0>();
+                    else cp_async_wait<NS - 2>();
+                }
                 __syncwarp();
                 {
                     const int idx = it + NS - 1;
@@ -310,7 +413,9 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
 #pragma unroll
                 for (int ks = 0; ks < KS; ++ks) {
                     uint32_t af[4];
-                    ldmatrix_x4(ks_u32 + k_row * ROW_BYTES + (((2 * ks + k_chunk) ^ (k_row & 7)) << 4), af);
+                    const int kc = 2 * ks + k_chunk;
+                    if constexpr (TMA) ldmatrix_x4(ks_u32 + (kc >> 3) * 2048 + k_row * 128 + (((kc & 7) ^ (k_row & 7)) << 4), af);
+                    else ldmatrix_x4(ks_u32 + k_row * ROW_BYTES + ((kc ^ (k_row & 7)) << 4), af);
                     if (ks & 1) mma_bf16(cb, af, bq[ks][0], bq[ks][1]);
                     else mma_bf16(ca, af, bq[ks][0], bq[ks][1]);
                 }
@@ -353,7 +458,9 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
 #pragma unroll
                 for (int mt = 0; mt < KS; ++mt) {
                     uint32_t af[4];
-                    ldmatrix_x4_trans(vs_u32 + v_row * ROW_BYTES + (((2 * mt + v_chunk) ^ (v_row & 7)) << 4), af);
+                    const int vc = 2 * mt + v_chunk;
+                    if constexpr (TMA) ldmatrix_x4_trans(vs_u32 + (vc >> 3) * 2048 + v_row * 128 + (((vc & 7) ^ (v_row & 7)) << 4), af);
+                    else ldmatrix_x4_trans(vs_u32 + v_row * ROW_BYTES + ((vc ^ (v_row & 7)) << 4), af);
                     mma_bf16(o[mt], af, pb0, pb1);
                 }
             }
@@ -399,6 +506,13 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1) attend_async_k
             ++seq;
         }
         cp_async_wait<0>();
+        if (TMA) {  // only after a timeout can loads still be in flight: wait for them (bounded) before leaving
+            for (int sl = 0; sl < NS; ++sl)
+                if ((slot_busy >> sl) & 1u) {
+                    for (int spin = 0; spin < kWaitLimit; ++spin)
+                        if (mbar_try_wait(&hd.tma_full[warp][sl], (slot_phase >> sl) & 1u)) break;
+                }
+        }
         if (bad_page && lane == 0) record_error(a.status, LETHE_ERR_PAGE, 0);
     } else {
         // =================================================================== epilogue warps
@@ -537,21 +651,24 @@ static size_t async_smem(int chunk_tokens, int GP) {
            (size_t)2 * chunk_tokens * GP * 4;
 }
 
-template <int D, int NWS, int NS, bool PAGED, bool SPILL>
-static cudaError_t launch_async_t(const AttendArgs& a, int grid, cudaStream_t stream) {
-    auto kern = attend_async_kernel<D, NWS, NS, PAGED, SPILL>;
+template <int D, int NWS, int NS, bool PAGED, bool SPILL, bool TMA>
+static cudaError_t launch_async_t(const AttendArgs& a, const TmaMaps& maps, int grid, cudaStream_t stream) {
+    auto kern = attend_async_kernel<D, NWS, NS, PAGED, SPILL, TMA>;
     const size_t smem = async_smem<D, NWS, NS>(a.chunk_tokens, a.GP);
     cudaError_t e = prepare_kernel((const void*)kern, smem);
     if (e != cudaSuccess) return e;
-    kern<<<grid, (NWS + kEpilogueWarps) * 32, smem, stream>>>(a);
+    kern<<<grid, (NWS + kEpilogueWarps) * 32, smem, stream>>>(a, maps);
     return cudaGetLastError();
 }
 
-template <int D, int NWS, int NS>
-static cudaError_t dispatch_async(const AttendArgs& a, bool paged, int grid, cudaStream_t stream) {
+template <int D, int NWS, int NS, bool TMA>
+static cudaError_t dispatch_async(const AttendArgs& a, const TmaMaps& maps, bool paged, int grid, cudaStream_t stream) {
     const bool spill = a.spill != nullptr;
-    if (paged) return spill ? launch_async_t<D, NWS, NS, true, true>(a, grid, stream) : launch_async_t<D, NWS, NS, true, false>(a, grid, stream);
-    return spill ? launch_async_t<D, NWS, NS, false, true>(a, grid, stream) : launch_async_t<D, NWS, NS, false, false>(a, grid, stream);
+    if (paged)
+        return spill ? launch_async_t<D, NWS, NS, true, true, TMA>(a, maps, grid, stream)
+                     : launch_async_t<D, NWS, NS, true, false, TMA>(a, maps, grid, stream);
+    return spill ? launch_async_t<D, NWS, NS, false, true, TMA>(a, maps, grid, stream)
+                 : launch_async_t<D, NWS, NS, false, false, TMA>(a, maps, grid, stream);
 }
 
 // Shapes: (streaming warps per CTA, stages per warp); two more warps run the epilogue.
@@ -567,13 +684,43 @@ size_t async_smem_bytes(int D, int shape, int chunk_tokens, int GP) {
     return (size_t)-1;
 }
 
-cudaError_t launch_attend_async(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream) {
-#define X(id, DD, NW, NS) \
-    if (shape == id && D == DD) return dispatch_async<DD, NW, NS>(a, paged, grid, stream);
+// tma: stage K / V tiles with cp.async.bulk.tensor through `maps` (a TmaMaps built by the caller) instead of
+// 16-byte cp.async; maps may be NULL when tma is false.
+cudaError_t launch_attend_async(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream, bool tma,
+                                const void* maps) {
+    TmaMaps none;
+    memset(&none, 0, sizeof(none));
+    const TmaMaps& m = (tma && maps) ? *reinterpret_cast<const TmaMaps*>(maps) : none;
+#define X(id, DD, NW, NS)                                                                            \
+    if (shape == id && D == DD)                                                                      \
+        return tma ? dispatch_async<DD, NW, NS, true>(a, m, paged, grid, stream) : dispatch_async<DD, NW, NS, false>(a, m, paged, grid, stream);
     LETHE_ASYNC_SHAPES(X, 128)
     LETHE_ASYNC_SHAPES(X, 64)
 #undef X
     return cudaErrorInvalidValue;
 }
+
+// Host: fill a TmaMaps for K and V seen as 2-D bf16 tensors [rows][D] with a (16 rows x 64 elements) box and the
+// 128-byte swizzle.  `encode` is cuTensorMapEncodeTiled, resolved by the caller.  Returns false on failure.
+bool build_tma_maps(void* encode, void* k, void* v, unsigned long long rows, int D, void* out_maps) {
+    typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    encode_fn fn = reinterpret_cast<encode_fn>(encode);
+    TmaMaps* m = reinterpret_cast<TmaMaps*>(out_maps);
+    const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)D * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kGroupTokens};
+    const cuuint32_t estr[2] = {1, 1};
+    for (int which = 0; which < 2; ++which) {
+        CUresult r = fn(which ? &m->v : &m->k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, which ? v : k, dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return false;
+    }
+    return true;
+}
+
+size_t tma_maps_bytes() { return sizeof(TmaMaps); }
 
 }  // namespace lethe

@@ -84,6 +84,10 @@ CASES = [
     (torch.bfloat16, 128, 4, 1, 300, 19, 0),
     (torch.bfloat16, 64, 16, 2, 500, 20, 0),
     (torch.bfloat16, 128, 6, 2, 300, 21, 0),
+    (torch.bfloat16, 128, 32, 8, 300, 24, 0),
+    (torch.bfloat16, 128, 28, 4, 700, 26, 0),
+    (torch.bfloat16, 64, 14, 2, 300, 27, 0),
+    (torch.bfloat16, 64, 16, 2, 500, 29, 0),
     (torch.bfloat16, 128, 8, 8, 260, 0, 0),
     (torch.float32, 128, 16, 2, 260, 0, 0),
 ]
@@ -112,7 +116,7 @@ def test_decode_attend_parity(ctx, dtype, D, Hq, Hkv, cap, variant, splits):
         ctx.set_tuning(0, 0)
 
 
-@pytest.mark.parametrize("variant", [8, 9, 10, 12, 13, 16, 17, 18, 19, 21])
+@pytest.mark.parametrize("variant", [8, 9, 10, 12, 13, 16, 17, 18, 19, 21, 24, 26, 27, 29])
 def test_persistent_queue_many_items(ctx, variant):
     """More items than SMs, so every CTA of the persistent kernel walks several items through its queue and
     prefetches across item boundaries; lengths from 0 to several hundred, including tiny items that leave
@@ -176,7 +180,7 @@ def test_empty_and_full_items(ctx):
     assert ctx.poll_status()[0] == 0                                     # the status word was cleared
 
 
-@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("variant", [1, 2, 9, 18, 26])
 def test_paged_decode_and_prune_parity(ctx, variant):
     """16-token pages behind a shuffled page table: decode steps and prune rounds, call by call."""
     w = synth.shrink(synth.WORKLOADS["ragged"], n_layers=2, batch=3, prompt_len=200)
@@ -188,7 +192,7 @@ def test_paged_decode_and_prune_parity(ctx, variant):
     gc = to_device(oc)
     scale = synth.layer_scales(w)
     T = torch.tensor([150 * 2, 90 * 2, 400 * 2], dtype=torch.int64)
-    ctx.set_tuning(variant, 2)
+    ctx.set_tuning(variant, 2 if variant < 8 else 0)
     try:
         for step in range(6):
             x = synth.step_inputs(w, step)
@@ -373,7 +377,7 @@ def test_ragged_paged_long_items(ctx):
 
 
 @pytest.mark.parametrize("variant,Hq,Hkv,cap", [(9, 28, 4, 3000), (12, 16, 4, 4200), (14, 28, 4, 6000), (16, 28, 4, 3000),
-                                                (18, 16, 4, 4200), (20, 28, 4, 6000)])
+                                                (18, 16, 4, 4200), (20, 28, 4, 6000), (26, 16, 4, 4200)])
 def test_persistent_logit_overflow(ctx, variant, Hq, Hkv, cap):
     """Items longer than the on-chip logit buffer of the persistent kernel: the logits of the tail tokens
     overflow to global scratch and the relevance update must still be exact."""
