@@ -1,7 +1,6 @@
 // C ABI of the Lethe hot path: argument checking, launch geometry, context-owned scratch and status word.
 #include <math.h>
 #include <stdio.h>
-#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -372,8 +371,8 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         if (a.chunk_tokens < kGroupTokens)
             return fail(ctx, LETHE_ERR_UNSUPPORTED, "no shared memory left for the logit buffers of this persistent shape");
         const int grid = a.n_items < ctx->sm_count ? a.n_items : ctx->sm_count;
-        if (a.chunk_tokens < cap_groups * kGroupTokens || getenv("LETHE_DEBUG_FORCE_SPILL")) {
-            a.spill_tokens = cap_groups * kGroupTokens - a.chunk_tokens + 16;
+        if (a.chunk_tokens < cap_groups * kGroupTokens) {
+            a.spill_tokens = cap_groups * kGroupTokens - a.chunk_tokens;
             const size_t need = (size_t)grid * 2 * a.spill_tokens * a.GP * sizeof(float);
             st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "logit overflow scratch");
             if (st != LETHE_OK) return st;
