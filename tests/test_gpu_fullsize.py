@@ -1,7 +1,7 @@
-"""Parity at the full size of the Llama-8B-shaped workload, in exactly the launch configuration bench.py times
-(its Runner: all 32 layers x 8 sequences x 8 KV heads in one lethe_decode_attend call, default tuning, capacity
-2048).  The oracle cannot run the whole state in seconds, so it recomputes sampled items one by one from
-snapshots of the GPU state taken just before the call."""
+"""Parity at the full size of the Llama-8B-shaped workload (the one bench.py times) and of the Qwen-7B-shaped one,
+in exactly the launch configuration bench.py uses (its Runner: all layers x sequences x KV heads in one
+lethe_decode_attend call, default tuning).  The oracle cannot run the whole state in seconds, so it recomputes
+sampled items one by one from snapshots of the GPU state taken just before the call."""
 import pytest
 import torch
 
@@ -18,13 +18,14 @@ def _item_cache(k, v, rel, pos, n, G, D, cap):
                               pos.reshape(1, 1, 1, cap).contiguous(), torch.tensor([[[n]]], dtype=torch.int32))
 
 
-def test_llama8b_full_size_sampled_items():
+@pytest.mark.parametrize("name,cap_factor", [("llama8b", 2), ("qwen7b", 3)])
+def test_full_size_sampled_items(name, cap_factor):
     import bench
     from paper_2511_06029_b200 import synth
     gpu_context().close()                          # builds the library if needed
-    w = synth.WORKLOADS["llama8b"]
+    w = synth.WORKLOADS[name]
     dev = torch.device("cuda", 0)
-    cap = 2 * w.mean_budget
+    cap = cap_factor * w.mean_budget
     r = bench.Runner(w, dev, 0, cap, 0, 0)
     for _ in range(w.prune_interval):               # one prep round, as bench.py does
         r.decode()
@@ -78,7 +79,7 @@ def test_llama8b_full_size_sampled_items():
     seqs = [1, B - 1]
     rel_seq = {b: c.rel[:, b].cpu().clone() for b in seqs}
     snaps = {}
-    items = [(l, b, h) for b in seqs for (l, h) in [(0, 0), (7, 3), (19, 5), (31, 7)]]
+    items = [(l, b, h) for b in seqs for (l, h) in [(0, 0), (7, 3 % H), (19, 5 % H), (L - 1, H - 1)]]
     for (l, b, h) in items:
         snaps[(l, b, h)] = tuple(t[l, b, h].cpu().clone() for t in (c.k, c.v, c.rel, c.pos))
     r.prune()
@@ -109,3 +110,5 @@ def test_llama8b_full_size_sampled_items():
     lens_after = c.len.cpu()
     assert torch.all(lens_after <= torch.minimum(lens, bud[:, :, None].expand(L, B, H)))
     r.ctx.close()
+    del r, c
+    torch.cuda.empty_cache()
