@@ -35,6 +35,10 @@ __global__ void __launch_bounds__(NW * 32) attend_mma_kernel(const __grid_consta
     float* lg = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(&es) + sizeof(EpilogueSmem));
 
     TL_MARK(a, 0);
+    // Programmatic dependent launch: when the launch carries the attribute this CTA may have been scheduled while
+    // the previous kernel of the stream was still draining; everything it reads may come from that kernel, so it
+    // waits here for it to complete (a no-op for ordinary launches).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const ItemCoord ic = decode_item(a);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int gq = lane >> 2, tq = lane & 3;  // fragment coordinates: row group, column pair
@@ -203,6 +207,8 @@ __global__ void __launch_bounds__(NW * 32) attend_mma_kernel(const __grid_consta
         cp_async_commit();
     }
     TL_MARK(a, 2);
+    // the streaming part is over: let the next kernel of the stream be scheduled onto the SMs as they free up
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     float rel_old[kRelPrefetch];
     prefetch_rel<NW * 32>(a, ic, t0, min(t1, n), append_slot, rel_old);
     cp_async_wait<0>();
@@ -248,13 +254,16 @@ static cudaError_t launch_mma_t(const AttendArgs& a, cudaStream_t stream) {
     cfg.blockDim = dim3(NW * 32, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)a.splits;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // launches of this kernel may overlap their scheduling with the tail of the previous kernel in the stream
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, kern, a);
 }
 
