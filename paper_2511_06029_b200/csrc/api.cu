@@ -76,6 +76,8 @@ struct lethe_ctx {
     size_t order_bytes;
     const int32_t* order_len;  // cache.len the order was computed from
     int order_items;
+    void* flat;  // scratch-merged split mode: arrival counters (zero between launches), partials, logits
+    size_t flat_bytes;
     void* staging;  // device staging of lethe_decode_attend_host
     size_t staging_bytes;
     int variant, splits;
@@ -210,6 +212,7 @@ void lethe_destroy(lethe_ctx* ctx) {
     if (ctx->scratch) cudaFree(ctx->scratch);
     if (ctx->staging) cudaFree(ctx->staging);
     if (ctx->order) cudaFree(ctx->order);
+    if (ctx->flat) cudaFree(ctx->flat);
     delete ctx;
 }
 
@@ -249,9 +252,11 @@ lethe_status lethe_debug_set_timeline(lethe_ctx* ctx, unsigned long long* buf) {
 
 lethe_status lethe_set_tuning(lethe_ctx* ctx, int variant, int splits) {
     if (!ctx) return LETHE_ERR_INVALID_ARG;
-    if (variant < 0 || variant > 31) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..31");
-    if (!(splits == 0 || splits == 1 || splits == 2 || splits == 4 || splits == 8 || splits == 16))
-        return fail(ctx, LETHE_ERR_INVALID_ARG, "splits must be 0, 1, 2, 4, 8 or 16");
+    if (variant < 0 || variant > 37) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..37");
+    const bool flat_variant = variant >= 32;
+    if (flat_variant ? (splits < 0 || splits > 16)
+                     : !(splits == 0 || splits == 1 || splits == 2 || splits == 4 || splits == 8 || splits == 16))
+        return fail(ctx, LETHE_ERR_INVALID_ARG, "splits must be 0, 1, 2, 4, 8 or 16 (0..16 for the scratch-merged variants)");
     ctx->variant = variant;
     ctx->splits = splits;
     return LETHE_OK;
@@ -340,7 +345,37 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
     if (variant >= 2 && !mma_ok) return fail(ctx, LETHE_ERR_UNSUPPORTED, "tensor-core variants need bf16 and 16-token pages");
 
     cudaError_t e;
-    if (variant >= 16) {  // persistent, asynchronous epilogue: both logit buffers (item parity) share what is left
+    if (variant >= 32) {  // clustered kernel's arithmetic, CTAs of an item merged through scratch instead of a cluster
+        const int shape = variant - 32;
+        int S = ctx->splits;
+        if (S == 0) {  // chunks of about 256 tokens, at most 16 per item
+            S = (a.cap_tokens + 255) / 256;
+            if (S > 16) S = 16;
+            if (S < 1) S = 1;
+        }
+        const int chunk = ((cap_groups + S - 1) / S) * kGroupTokens;
+        if (mma_smem_bytes(c->head_dim, shape, chunk, a.GP) > ctx->max_smem)
+            return fail(ctx, LETHE_ERR_UNSUPPORTED, "capacity too large for the on-chip logit buffer at this split count");
+        a.splits = S;
+        a.chunk_tokens = chunk;
+        a.flat_pitch = cap_groups * kGroupTokens;
+        auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+        const size_t cnt_bytes = up((size_t)a.n_items * sizeof(int));
+        const size_t part_bytes = up((size_t)a.n_items * S * (16 + (size_t)G * c->head_dim) * sizeof(float));
+        const size_t lg_bytes = up((size_t)a.n_items * a.flat_pitch * a.GP * sizeof(float));
+        const size_t need = cnt_bytes + part_bytes + lg_bytes;
+        if (need > ctx->flat_bytes) {
+            st = ensure(ctx, &ctx->flat, &ctx->flat_bytes, need, "scratch-merge buffers");
+            if (st != LETHE_OK) return st;
+            if (cudaMemsetAsync(ctx->flat, 0, ctx->flat_bytes, (cudaStream_t)stream) != cudaSuccess)
+                return fail(ctx, LETHE_ERR_CUDA, "clearing the scratch-merge buffers failed");
+        }
+        // counters sit at the front: they stay zero between launches whatever n_items later calls use
+        a.flat_cnt = (int*)ctx->flat;
+        a.flat_part = (float*)((char*)ctx->flat + cnt_bytes);
+        a.flat_lg = (float*)((char*)ctx->flat + cnt_bytes + part_bytes);
+        e = launch_attend_mma(a, c->head_dim, shape, paged, (cudaStream_t)stream);
+    } else if (variant >= 16) {  // persistent, asynchronous epilogue: both logit buffers (item parity) share what is left
         if (ctx->splits > 1) return fail(ctx, LETHE_ERR_INVALID_ARG, "the persistent variants do not split items");
         const bool tma = variant >= 24;
         const int shape = tma ? variant - 24 : variant - 16;

@@ -17,7 +17,7 @@
 
 namespace lethe {
 
-template <int D, int NW, int NSTAGE, bool PAGED>
+template <int D, int NW, int NSTAGE, bool PAGED, bool FLAT>
 __global__ void __launch_bounds__(NW * 32) attend_mma_kernel(const __grid_constant__ AttendArgs a) {
     using T = __nv_bfloat16;
     constexpr int ROW_BYTES = D * 2;
@@ -210,7 +210,7 @@ __global__ void __launch_bounds__(NW * 32) attend_mma_kernel(const __grid_consta
     // the streaming part is over: let the next kernel of the stream be scheduled onto the SMs as they free up
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     float rel_old[kRelPrefetch];
-    prefetch_rel<NW * 32>(a, ic, t0, min(t1, n), append_slot, rel_old);
+    if constexpr (!FLAT) prefetch_rel<NW * 32>(a, ic, t0, min(t1, n), append_slot, rel_old);
     cp_async_wait<0>();
     __syncwarp();
     if (bad_page) record_error(a.status, LETHE_ERR_PAGE, ic.item);
@@ -233,8 +233,11 @@ __global__ void __launch_bounds__(NW * 32) attend_mma_kernel(const __grid_consta
         wo[(2 * tq) * D + 16 * mt + gq + 8] = o[mt][2];
         wo[(2 * tq + 1) * D + 16 * mt + gq + 8] = o[mt][3];
     }
-    combine_and_finish<T, D, NW>(a, ic, es, reinterpret_cast<float*>(stage_base), WARP_BYTES / 4, cta_o, lg, t0, t1,
-                                 append_slot, n, rel_old);
+    if constexpr (FLAT)
+        flat_finish<T, D, NW>(a, ic, es, reinterpret_cast<float*>(stage_base), WARP_BYTES / 4, cta_o, lg, t0, t1, append_slot, n);
+    else
+        combine_and_finish<T, D, NW>(a, ic, es, reinterpret_cast<float*>(stage_base), WARP_BYTES / 4, cta_o, lg, t0, t1,
+                                     append_slot, n, rel_old);
 }
 
 template <int D, int NW, int NSTAGE>
@@ -243,9 +246,9 @@ static size_t mma_smem(int chunk_tokens, int GP) {
            (size_t)chunk_tokens * GP * 4;
 }
 
-template <int D, int NW, int NSTAGE, bool PAGED>
+template <int D, int NW, int NSTAGE, bool PAGED, bool FLAT>
 static cudaError_t launch_mma_t(const AttendArgs& a, cudaStream_t stream) {
-    auto kern = attend_mma_kernel<D, NW, NSTAGE, PAGED>;
+    auto kern = attend_mma_kernel<D, NW, NSTAGE, PAGED, FLAT>;
     const size_t smem = mma_smem<D, NW, NSTAGE>(a.chunk_tokens, a.GP);
     cudaError_t e = prepare_kernel((const void*)kern, smem);
     if (e != cudaSuccess) return e;
@@ -256,7 +259,7 @@ static cudaError_t launch_mma_t(const AttendArgs& a, cudaStream_t stream) {
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)a.splits;
+    attr[0].val.clusterDim.x = FLAT ? 1u : (unsigned)a.splits;  // scratch-merged mode needs no co-scheduling
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     // launches of this kernel may overlap their scheduling with the tail of the previous kernel in the stream
@@ -265,6 +268,13 @@ static cudaError_t launch_mma_t(const AttendArgs& a, cudaStream_t stream) {
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, kern, a);
+}
+
+template <int D, int NW, int NS>
+static cudaError_t dispatch_mma(const AttendArgs& a, bool paged, cudaStream_t stream) {
+    const bool flat = a.flat_cnt != nullptr;
+    if (paged) return flat ? launch_mma_t<D, NW, NS, true, true>(a, stream) : launch_mma_t<D, NW, NS, true, false>(a, stream);
+    return flat ? launch_mma_t<D, NW, NS, false, true>(a, stream) : launch_mma_t<D, NW, NS, false, false>(a, stream);
 }
 
 // Kernel shapes (warps per CTA, pipeline stages per warp), selected by `shape`.
@@ -283,7 +293,7 @@ size_t mma_smem_bytes(int D, int shape, int chunk_tokens, int GP) {
 cudaError_t launch_attend_mma(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream) {
 #define X(id, DD, NW, NS)                                                                           \
     if (shape == id && D == DD)                                                                     \
-        return paged ? launch_mma_t<DD, NW, NS, true>(a, stream) : launch_mma_t<DD, NW, NS, false>(a, stream);
+        return dispatch_mma<DD, NW, NS>(a, paged, stream);
     LETHE_MMA_SHAPES(X, 128)
     LETHE_MMA_SHAPES(X, 64)
 #undef X

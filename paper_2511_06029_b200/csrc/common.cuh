@@ -32,6 +32,12 @@ struct AttendArgs {
     float* lse;
     int32_t* status;      // device status word: {code, item}
     unsigned int* sched;  // persistent kernel only: {next ticket, CTAs finished}, zero between launches
+    // scratch-merged split ("flat") mode of the clustered kernel: the CTAs of an item do not form a cluster; each
+    // publishes its partial result and logits, the last one to arrive finishes the item
+    int* flat_cnt;        // [n_items] arrival counters, zero between launches
+    float* flat_part;     // [n_items][splits][16 + G * D]: 8 x (max, sum), then O
+    float* flat_lg;       // [n_items][flat_pitch][GP] scaled logits
+    int flat_pitch;       // tokens per item in flat_lg
     const int32_t* order; // persistent kernels: ticket -> item of the call, longest items first (NULL = identity)
     float* spill;         // persistent kernel only: global overflow of the logit buffer, [grid][spill_tokens][GP]
     int spill_tokens;     // tokens per CTA the overflow can hold (0 = the shared-memory buffer covers cap_tokens)
@@ -248,18 +254,20 @@ __device__ void combine_and_finish(const AttendArgs& a, const ItemCoord& ic, Epi
     } else {
         cg::cluster_group cluster = cg::this_cluster();
         cluster.sync();  // every CTA's cta_o / cta_stat is complete and visible cluster-wide
+        // all ranks' (max, sum) pairs into local shared memory with one remote round trip (wstat is free by now)
+        if (tid < S * kMaxGroup) {
+            const int r = tid / kMaxGroup, h = tid % kMaxGroup;
+            es.wstat[r][h] = cluster.map_shared_rank(&es.cta_stat[0], r)[h];
+        }
+        __syncthreads();
         if (tid < kMaxGroup) {
             const int h = tid;
             float m = -INFINITY;
-            for (int r = 0; r < S; ++r) m = fmaxf(m, cluster.map_shared_rank(&es.cta_stat[0], r)[h].x);
+            for (int r = 0; r < S; ++r) m = fmaxf(m, es.wstat[r][h].x);
             float l = 0.f;
-            for (int r = 0; r < S; ++r) {
-                const float2 st = cluster.map_shared_rank(&es.cta_stat[0], r)[h];
-                l += st.y * exp2_diff(st.x, m);
-            }
+            for (int r = 0; r < S; ++r) l += es.wstat[r][h].y * exp2_diff(es.wstat[r][h].x, m);
             const float inv = l > 0.f ? 1.f / l : 0.f;
-            for (int r = 0; r < S; ++r)
-                es.rscale[r][h] = exp2_diff(cluster.map_shared_rank(&es.cta_stat[0], r)[h].x, m) * inv;
+            for (int r = 0; r < S; ++r) es.rscale[r][h] = exp2_diff(es.wstat[r][h].x, m) * inv;
             es.fin[h] = make_float2(m, inv);
             if (lse && ic.rank == 0 && h < G) lse[h] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
         }
@@ -308,6 +316,124 @@ __device__ void combine_and_finish(const AttendArgs& a, const ItemCoord& ic, Epi
     if (S > 1) cg::this_cluster().sync();  // peers may still be reading this CTA's shared memory
     if (append_slot >= 0 && ic.rank == 0 && tid == 0) a.len[ic.item] = n;
     TL_MARK(a, 6);
+}
+
+/*
+ * Tail of the clustered kernel in scratch-merged mode.  Same inputs as combine_and_finish.  Every CTA merges its
+ * warps, publishes (max, sum, O) and its logits to global scratch and bumps the item's arrival counter; the CTA
+ * that arrives last merges all partials, writes out / lse, applies Eq. 5 to the whole item, resets the counter
+ * and stores len.  Nobody waits for anybody, so the CTAs need not be co-scheduled.
+ */
+template <typename T, int D, int NW>
+__device__ void flat_finish(const AttendArgs& a, const ItemCoord& ic, EpilogueSmem& es, float* wo, int wo_stride,
+                            float* cta_o /*[kMaxGroup][D]*/, const float* lg, int t0, int t1, int append_slot, int n) {
+    const int tid = threadIdx.x;
+    const int G = a.G, GP = a.GP, S = a.splits;
+    constexpr int NT = NW * 32;
+    __syncthreads();
+    if (tid < kMaxGroup) {
+        const int h = tid;
+        float m = -INFINITY;
+        for (int w = 0; w < NW; ++w) m = fmaxf(m, es.wstat[w][h].x);
+        float l = 0.f;
+        for (int w = 0; w < NW; ++w) {
+            const float sc = exp2_diff(es.wstat[w][h].x, m);
+            es.wscale[w][h] = sc;
+            l += es.wstat[w][h].y * sc;
+        }
+        es.cta_stat[h] = make_float2(m, l);
+    }
+    __syncthreads();
+    const int part_floats = 16 + G * D;
+    float* part = a.flat_part + ((size_t)ic.item_call * S + ic.rank) * part_floats;
+    if (tid < kMaxGroup) reinterpret_cast<float2*>(part)[tid] = es.cta_stat[tid];
+    for (int idx = tid; idx < G * D; idx += NT) {
+        const int h = idx / D;
+        float acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) acc += wo[w * wo_stride + idx] * es.wscale[w][h];
+        part[16 + idx] = acc;
+    }
+    float* glg = a.flat_lg + ((size_t)ic.item_call * a.flat_pitch + t0) * GP;
+    const int n_lg = (min(t1, n) - t0) * GP;
+    for (int i = tid; 2 * i < n_lg; i += NT)  // GP is even and t0 a multiple of 16: 8-byte pieces are aligned
+        reinterpret_cast<float2*>(glg)[i] = reinterpret_cast<const float2*>(lg)[i];
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) es.flags[0] = (atomicAdd(&a.flat_cnt[ic.item_call], 1) == S - 1) ? 1 : 0;
+    __syncthreads();
+    if (!es.flags[0]) return;
+    __threadfence();  // the other CTAs' partials and logits were published before their arrivals
+
+    const float* parts = a.flat_part + (size_t)ic.item_call * S * part_floats;
+    // all (max, sum) pairs into shared memory with one round trip, then eight threads merge them
+    if (tid < S * kMaxGroup) {
+        const int r = tid / kMaxGroup, h = tid % kMaxGroup;
+        es.wstat[r][h] = __ldcg(reinterpret_cast<const float2*>(parts + (size_t)r * part_floats) + h);
+    }
+    __syncthreads();
+    if (tid < kMaxGroup) {
+        const int h = tid;
+        float m = -INFINITY;
+        for (int r = 0; r < S; ++r) m = fmaxf(m, es.wstat[r][h].x);
+        float l = 0.f;
+        for (int r = 0; r < S; ++r) l += es.wstat[r][h].y * exp2_diff(es.wstat[r][h].x, m);
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        for (int r = 0; r < S; ++r) es.rscale[r][h] = exp2_diff(es.wstat[r][h].x, m) * inv;
+        es.fin[h] = make_float2(m, inv);
+        if (a.lse && h < G)
+            a.lse[(size_t)(ic.li * a.B + ic.b) * a.Hq + ic.hkv * G + h] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+    }
+    __syncthreads();
+    T* out = (T*)a.out + ((size_t)(ic.li * a.B + ic.b) * a.Hq + ic.hkv * G) * D;
+    for (int idx = tid; idx < G * D; idx += NT) {
+        const int h = idx / D;
+        float acc = 0.f;
+#pragma unroll 4
+        for (int r = 0; r < S; ++r) acc += __ldcg(parts + (size_t)r * part_floats + 16 + idx) * es.rscale[r][h];
+        out[idx] = from_float<T>(acc);
+    }
+    float fm[kMaxGroup], fi[kMaxGroup];
+#pragma unroll
+    for (int h = 0; h < kMaxGroup; ++h) {
+        fm[h] = es.fin[h].x;
+        fi[h] = es.fin[h].y;
+    }
+    // Eq. 5 over the whole item: logits (L2-resident, written by the item's CTAs) and old scores are fetched for
+    // a batch of tokens before any of them is used
+    float* rel = a.rel + (size_t)ic.item * a.cap_tokens;
+    const float2* item_lg = reinterpret_cast<const float2*>(a.flat_lg + (size_t)ic.item_call * a.flat_pitch * GP);
+    const int GP2 = GP / 2;
+    constexpr int RB = 4;
+    for (int base = 0; base < n; base += RB * NT) {
+        float2 lgv[RB][kMaxGroup / 2];
+        float oldv[RB];
+#pragma unroll
+        for (int i = 0; i < RB; ++i) {
+            const int j = base + tid + i * NT;
+#pragma unroll
+            for (int h2 = 0; h2 < kMaxGroup / 2; ++h2)
+                lgv[i][h2] = (j < n && h2 < GP2) ? __ldcg(item_lg + (size_t)j * GP2 + h2) : make_float2(0.f, 0.f);
+            oldv[i] = (j < n && j != append_slot) ? rel[j] : 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < RB; ++i) {
+            const int j = base + tid + i * NT;
+            if (j < n) {
+                float mass = 0.f;
+#pragma unroll
+                for (int h2 = 0; h2 < kMaxGroup / 2; ++h2) {
+                    if (2 * h2 < G) mass += fast_exp2(lgv[i][h2].x - fm[2 * h2]) * fi[2 * h2];
+                    if (2 * h2 + 1 < G) mass += fast_exp2(lgv[i][h2].y - fm[2 * h2 + 1]) * fi[2 * h2 + 1];
+                }
+                rel[j] = fmaf(a.gamma, oldv[i], mass);
+            }
+        }
+    }
+    if (tid == 0) {
+        a.flat_cnt[ic.item_call] = 0;
+        if (append_slot >= 0) a.len[ic.item] = n;
+    }
 }
 
 }  // namespace lethe

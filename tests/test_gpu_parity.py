@@ -88,6 +88,12 @@ CASES = [
     (torch.bfloat16, 128, 28, 4, 700, 26, 0),
     (torch.bfloat16, 64, 14, 2, 300, 27, 0),
     (torch.bfloat16, 64, 16, 2, 500, 29, 0),
+    (torch.bfloat16, 128, 32, 8, 300, 32, 0),
+    (torch.bfloat16, 128, 28, 4, 700, 33, 3),
+    (torch.bfloat16, 64, 14, 2, 300, 34, 5),
+    (torch.bfloat16, 128, 8, 1, 1000, 35, 16),
+    (torch.bfloat16, 64, 16, 2, 500, 36, 1),
+    (torch.bfloat16, 128, 6, 2, 300, 37, 7),
     (torch.bfloat16, 128, 8, 8, 260, 0, 0),
     (torch.float32, 128, 16, 2, 260, 0, 0),
 ]
@@ -180,7 +186,7 @@ def test_empty_and_full_items(ctx):
     assert ctx.poll_status()[0] == 0                                     # the status word was cleared
 
 
-@pytest.mark.parametrize("variant", [1, 2, 9, 18, 26])
+@pytest.mark.parametrize("variant", [1, 2, 9, 18, 26, 32])
 def test_paged_decode_and_prune_parity(ctx, variant):
     """16-token pages behind a shuffled page table: decode steps and prune rounds, call by call."""
     w = synth.shrink(synth.WORKLOADS["ragged"], n_layers=2, batch=3, prompt_len=200)
@@ -192,7 +198,7 @@ def test_paged_decode_and_prune_parity(ctx, variant):
     gc = to_device(oc)
     scale = synth.layer_scales(w)
     T = torch.tensor([150 * 2, 90 * 2, 400 * 2], dtype=torch.int64)
-    ctx.set_tuning(variant, 2 if variant < 8 else 0)
+    ctx.set_tuning(variant, 2 if variant < 8 else (3 if variant >= 32 else 0))
     try:
         for step in range(6):
             x = synth.step_inputs(w, step)
