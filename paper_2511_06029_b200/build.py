@@ -1,6 +1,7 @@
 """Build liblethe.so (the CUDA library behind the C ABI) in-tree with nvcc for sm_100a."""
 from __future__ import annotations
 
+import hashlib
 import os
 import subprocess
 import sys
@@ -20,12 +21,24 @@ def _nvcc() -> str:
     raise RuntimeError("nvcc not found")
 
 
+STAMP = LIB + ".srchash"   # hash of the sources the library was built from (file times do not survive a copy)
+
+
+def _source_hash() -> str:
+    h = hashlib.sha256()
+    deps = sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh")))
+    deps.append(os.path.join(HERE, "..", "include", "lethe.h"))
+    for d in deps:
+        h.update(os.path.basename(d).encode())
+        h.update(open(d, "rb").read())
+    h.update(" ".join(NVCC_FLAGS).encode())
+    return h.hexdigest()
+
+
 def _stale() -> bool:
-    if not os.path.exists(LIB):
+    if not os.path.exists(LIB) or not os.path.exists(STAMP):
         return True
-    t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(HERE, "..", "include", "lethe.h")]
-    return any(os.path.getmtime(d) > t for d in deps)
+    return open(STAMP).read().strip() != _source_hash()
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
@@ -47,6 +60,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if p.returncode:
             raise RuntimeError(f"nvcc failed on {src}")
     subprocess.run([_nvcc(), "-shared", "-o", LIB, *objs, "-lcudart"], check=True)
+    with open(STAMP, "w") as f:
+        f.write(_source_hash())
     return LIB
 
 

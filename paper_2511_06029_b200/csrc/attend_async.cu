@@ -672,8 +672,7 @@ static cudaError_t dispatch_async(const AttendArgs& a, const TmaMaps& maps, bool
 }
 
 // Shapes: (streaming warps per CTA, stages per warp); two more warps run the epilogue.
-#define LETHE_ASYNC_SHAPES(X, D) X(0, D, 8, 2) X(1, D, 7, 2) X(2, D, 6, 3) X(3, D, 5, 3) X(4, D, 6, 2) X(5, D, 4, 4) X(6, D, 3, 5) \
-        X(7, D, 5, 4)
+#define LETHE_ASYNC_SHAPES(X, D) X(0, D, 8, 2) X(1, D, 7, 2) X(2, D, 6, 3) X(3, D, 5, 3) X(4, D, 6, 2) X(5, D, 4, 4)
 
 size_t async_smem_bytes(int D, int shape, int chunk_tokens, int GP) {
 #define X(id, DD, NW, NS) \
