@@ -68,6 +68,9 @@ def lib():
         _lib.oracle_segment_prune.restype = ctypes.c_int
         _lib.oracle_segment_prune.argtypes = [ctypes.POINTER(_CCache), ctypes.c_int32, ctypes.c_float, ctypes.c_int32,
                                               ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32]
+        _lib.oracle_prefill_seed.restype = ctypes.c_int
+        _lib.oracle_prefill_seed.argtypes = [ctypes.POINTER(_CCache), ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p,
+                                             ctypes.c_float]
         _lib.oracle_set_threads.argtypes = [ctypes.c_int]
         _lib.oracle_get_threads.restype = ctypes.c_int
         _lib.oracle_max_threads.restype = ctypes.c_int
@@ -199,3 +202,11 @@ def segment_prune(cache: OracleCache, n_segments: int, tau: float, recent: int, 
     st = lib().oracle_segment_prune(ctypes.byref(cc), int(n_segments), ctypes.c_float(tau), int(recent), int(sink),
                                     _ptr(l_evict), _ptr(keep), int(max_k))
     return st, keep
+
+
+def prefill_seed(cache: OracleCache, q_prompt: torch.Tensor, scale: torch.Tensor, gamma: float) -> int:
+    """rel[0..P) of every item from the causal prefill attention of the P prompt queries (q_prompt [L][B][P][Hq][D])."""
+    assert q_prompt.dtype == cache.k.dtype and q_prompt.dim() == 5 and scale.dtype == torch.float32
+    cc = cache._c()
+    return lib().oracle_prefill_seed(ctypes.byref(cc), _ptr(q_prompt), int(q_prompt.shape[2]), _ptr(scale),
+                                     ctypes.c_float(gamma))

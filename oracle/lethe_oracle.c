@@ -25,6 +25,10 @@
  *   oracle_rasr_prune         Sec. 4.3 last paragraph + Algorithm 1 (top-k by
  *                             score, sinks and the recent window always kept),
  *                             multi-round carry-over of Sec. 4.4.
+ *   oracle_prefill_seed       Eq. 2 with Q > 1 (token importance from the prefill
+ *                             attention) folded through the recurrence of Eq. 5:
+ *                             the relevance the prompt tokens would have had if the
+ *                             prompt had been fed one token at a time.
  *   oracle_segment_prune      Algorithm 1 as a whole (segmented breakpoint search
  *                             of Sec. 4.2 / Eq. 4, retention set, eviction-threshold
  *                             update) with the size trigger of Sec. 4.1, applied per
@@ -539,6 +543,62 @@ int oracle_segment_prune(oracle_cache *c, int32_t n_segments, float tau, int32_t
         l_evict[item] = (int32_t)(grown > Le ? grown : Le);
         free(keep);
         free(top);
+    }
+    return ORACLE_OK;
+}
+
+/* ---- relevance of the prompt from the prefill attention (Eq. 2, Q > 1; Eq. 5) ---- */
+/*
+ * q_prompt [L][B][P][Hq][D] (cache dtype): the queries of the P prompt tokens; their keys are slots 0..P-1 of
+ * every item (len >= P required).  With causal attention rows
+ *   A_h(i, j) = softmax over j <= i of scale_l * q_{i,h} . K_j        (i, j < P)
+ * Eq. 5 run over the prompt positions as steps gives, for every slot j < P,
+ *   rel[j] = sum_{i = j}^{P-1} gamma^(P-1-i) * sum_{h in group} A_h(i, j).
+ * rel[0..P) is overwritten; nothing else changes.
+ */
+int oracle_prefill_seed(oracle_cache *c, const void *q_prompt, int32_t prompt_len, const float *scale, float gamma) {
+    int st = check_cache(c);
+    if (st) return st;
+    if (!q_prompt || !scale || prompt_len < 1 || !(gamma > 0.0f && gamma <= 1.0f)) return ORACLE_ERR_INVALID_ARG;
+    const int B = c->batch, Hq = c->n_q_heads, Hkv = c->n_kv_heads, D = c->head_dim, P = prompt_len;
+    const int G = Hq / Hkv;
+    const int64_t capT = cap_tokens(c);
+    const int n_items = c->n_layers * B * Hkv;
+    for (int w = 0; w < n_items; ++w)
+        if (c->len[w] < P) return ORACLE_ERR_CAPACITY;
+#ifdef _OPENMP
+#pragma omp parallel for num_threads(g_threads) schedule(dynamic, 1)
+#endif
+    for (int w = 0; w < n_items; ++w) {
+        const int l = w / (B * Hkv), b = (w / Hkv) % B, hkv = w % Hkv;
+        const int64_t item = w;
+        double *acc = (double *)calloc((size_t)P, sizeof(double));
+        double *p = (double *)malloc((size_t)P * sizeof(double));
+        for (int i = 0; i < P; ++i) {
+            const double wgt = pow((double)gamma, (double)(P - 1 - i));
+            for (int g = 0; g < G; ++g) {
+                const int h = hkv * G + g;
+                const int64_t qoff = ((((int64_t)l * B + b) * P + i) * Hq + h) * D;
+                double m = -INFINITY;
+                for (int j = 0; j <= i; ++j) {
+                    const int64_t koff = row_offset(c, item, j);
+                    double s = 0.0;
+                    for (int d = 0; d < D; ++d) s += load_elt(q_prompt, c->dtype, qoff + d) * load_elt(c->k, c->dtype, koff + d);
+                    s *= (double)scale[l];
+                    p[j] = s;
+                    if (s > m) m = s;
+                }
+                double Z = 0.0;
+                for (int j = 0; j <= i; ++j) {
+                    p[j] = exp(p[j] - m);
+                    Z += p[j];
+                }
+                for (int j = 0; j <= i; ++j) acc[j] += wgt * p[j] / Z;
+            }
+        }
+        for (int j = 0; j < P; ++j) c->rel[item * capT + j] = (float)acc[j];
+        free(acc);
+        free(p);
     }
     return ORACLE_OK;
 }

@@ -427,3 +427,56 @@ def test_segment_prune_against_library_sort_and_invariants():
         salient = sorted(set(kept) - prot)
         if dropped and salient:
             assert rel[salient].min() >= rel[dropped].max()
+
+
+# --------------------------------------------------------------------------- prefill seeding (Eq. 2 with Q > 1)
+
+def test_prefill_seed_equals_token_by_token_decode():
+    """Eq. 5 defines the relevance by a recurrence over steps; feeding the prompt one token at a time through the
+    (separately pinned) decode step must leave exactly the scores that the prefill formula gives at once."""
+    for dtype, Hq, Hkv, gamma in [(torch.float32, 4, 2, 0.9), (torch.bfloat16, 7, 1, 0.97), (torch.float32, 3, 3, 1.0)]:
+        L, B, D, P, cap = 2, 2, 8, 21, 24
+        g = torch.Generator().manual_seed(Hq)
+        kk = torch.randn((L, B, Hkv, cap, D), generator=g).to(dtype); vv = torch.randn((L, B, Hkv, cap, D), generator=g).to(dtype)
+        qp = torch.randn((L, B, P, Hq, D), generator=g).to(dtype)
+        scale = torch.tensor([0.4, 0.15], dtype=torch.float32)
+        mk = lambda n: oracle.OracleCache(L, B, Hq, Hkv, D, cap, kk.clone(), vv.clone(), torch.zeros((L, B, Hkv, cap)),
+                                          torch.zeros((L, B, Hkv, cap), dtype=torch.int32),
+                                          torch.full((L, B, Hkv), n, dtype=torch.int32))
+        step = mk(0)
+        for i in range(P):
+            st, *_ = oracle.decode_attend(step, 0, L, qp[:, :, i].contiguous(), kk[:, :, :, i].contiguous(),
+                                          vv[:, :, :, i].contiguous(), torch.full((B,), i, dtype=torch.int32), scale, gamma)
+            assert st == oracle.OK
+        once = mk(P)
+        once.rel[:] = 123.0                                   # must be overwritten, not accumulated
+        assert oracle.prefill_seed(once, qp, scale, gamma) == oracle.OK
+        assert torch.allclose(once.rel[..., :P], step.rel[..., :P], rtol=2e-5, atol=1e-7)
+        assert torch.all(once.rel[..., P:] == 123.0)
+
+
+def test_prefill_seed_against_library_softmax_and_closed_forms():
+    L, B, Hq, Hkv, D, P, cap = 1, 1, 4, 2, 16, 33, 40
+    c = random_cache(L, B, Hq, Hkv, D, cap, P, seed=6)
+    g = torch.Generator().manual_seed(4)
+    qp = torch.randn((L, B, P, Hq, D), generator=g)
+    scale = torch.tensor([0.3]); gamma = 0.8
+    assert oracle.prefill_seed(c, qp, scale, gamma) == oracle.OK
+    wgt = gamma ** torch.arange(P - 1, -1, -1, dtype=torch.float64)
+    mask = torch.tril(torch.ones(P, P, dtype=torch.bool))
+    for hk in range(Hkv):
+        want = torch.zeros(P, dtype=torch.float64)
+        for gq in range(2):
+            s = (qp[0, 0, :, hk * 2 + gq].double() @ c.k[0, 0, hk, :P].double().T) * 0.3
+            a = torch.softmax(s.masked_fill(~mask, float("-inf")), dim=1)
+            want += (wgt[:, None] * a).sum(0)
+        assert torch.allclose(c.rel[0, 0, hk, :P].double(), want, rtol=1e-6, atol=1e-9)
+        # total mass: every prompt row hands out G units, decayed: G (1 - gamma^P) / (1 - gamma)
+        assert abs(c.rel[0, 0, hk, :P].double().sum().item() - 2 * (1 - gamma ** P) / (1 - gamma)) < 1e-5
+    # q = 0: row i spreads 1/(i+1) over slots 0..i
+    c2 = random_cache(1, 1, 1, 1, 4, 8, 5, seed=1)
+    assert oracle.prefill_seed(c2, torch.zeros((1, 1, 5, 1, 4)), torch.tensor([1.0]), 1.0) == oracle.OK
+    want = torch.tensor([sum(1.0 / (i + 1) for i in range(j, 5)) for j in range(5)])
+    assert torch.allclose(c2.rel[0, 0, 0, :5], want, atol=1e-6)
+    short = random_cache(1, 1, 1, 1, 4, 8, 3, seed=1)
+    assert oracle.prefill_seed(short, torch.zeros((1, 1, 5, 1, 4)), torch.tensor([1.0]), 1.0) == oracle.ERR_CAPACITY
