@@ -15,6 +15,8 @@
  *   lethe_alloc_budgets      per-layer token budgets from those sparsities (Sec. 4.2)
  *   lethe_rasr_prune         protected top-k retention + in-place stable compaction
  *                            (Sec. 4.3; sink / recent sets of Algorithm 1)
+ *   lethe_prefill_seed       the same relevance for the prompt, from the prefill attention
+ *                            (Eq. 2 with Q > 1)
  *   lethe_segment_prune      Algorithm 1 itself: segmented breakpoint search, retention
  *                            set and eviction-threshold update (Sec. 4.2)
  *
@@ -213,6 +215,18 @@ lethe_status lethe_rasr_prune(lethe_ctx *ctx, const lethe_cache *cache, const in
 lethe_status lethe_segment_prune(lethe_ctx *ctx, const lethe_cache *cache, int32_t n_segments, float tau,
                                  int32_t recent, int32_t sink, int32_t *l_evict, int32_t *keep_idx, int32_t max_k,
                                  void *stream);
+
+/*
+ * Relevance of the prompt tokens from the prefill attention (Eq. 2 with Q > 1, folded through Eq. 5), so that
+ * decoding does not start from rel = 0.  q_prompt [L][B][P][Hq][D] (bf16) holds the queries of the P = prompt_len
+ * prompt tokens; their keys must already be slots 0..P-1 of every item (len >= P, else the item is skipped and
+ * LETHE_ERR_CAPACITY recorded).  With causal rows A_h(i, :) = softmax over j <= i of scale_l * q_{i,h} . K_j,
+ *   rel[j] = sum_{i=j}^{P-1} gamma^(P-1-i) * sum_{h in group} A_h(i, j)        for j < P
+ * which is what P single-token decode steps would have left.  rel[0..P) is overwritten; nothing else changes.
+ * scale: HOST float[L].  bf16 caches only; contiguous or paged.
+ */
+lethe_status lethe_prefill_seed(lethe_ctx *ctx, const lethe_cache *cache, const void *q_prompt, int32_t prompt_len,
+                                const float *scale, float gamma, void *stream);
 
 /*
  * lethe_rasr_prune without a context and without any allocation.  (The paper has no counterpart: this entry

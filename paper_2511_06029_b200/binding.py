@@ -23,7 +23,7 @@ VARIANT_AUTO, VARIANT_SIMT, VARIANT_MMA4, VARIANT_MMA8 = 0, 1, 2, 3
 
 EXPORTS = ["lethe_create", "lethe_destroy", "lethe_last_error", "lethe_poll_status", "lethe_set_tuning",
            "lethe_decode_attend", "lethe_decode_attend_host", "lethe_estimate_sparsity", "lethe_alloc_budgets",
-           "lethe_rasr_prune", "lethe_rasr_prune_static", "lethe_segment_prune"]
+           "lethe_rasr_prune", "lethe_rasr_prune_static", "lethe_segment_prune", "lethe_prefill_seed"]
 
 
 class LetheError(RuntimeError):
@@ -79,6 +79,8 @@ def load() -> ctypes.CDLL:
     lib.lethe_rasr_prune.argtypes = [vp, cp, vp, i32, i32, vp, i32, vp]
     lib.lethe_segment_prune.restype = ctypes.c_int
     lib.lethe_segment_prune.argtypes = [vp, cp, i32, ctypes.c_float, i32, i32, vp, vp, i32, vp]
+    lib.lethe_prefill_seed.restype = ctypes.c_int
+    lib.lethe_prefill_seed.argtypes = [vp, cp, vp, i32, ctypes.POINTER(ctypes.c_float), ctypes.c_float, vp]
     lib.lethe_rasr_prune_static.restype = ctypes.c_int
     lib.lethe_rasr_prune_static.argtypes = [cp, vp, i32, i32, vp, i32, vp, vp]
     _lib = lib
@@ -235,3 +237,9 @@ class Context:
             max_k = keep_idx.shape[-1]
         self._check(self.lib.lethe_segment_prune(self.h, ctypes.byref(cache.c), n_segments, tau, recent, sink,
                                                  _dp(l_evict), _dp(keep_idx), max_k, _stream(self.device)))
+
+    def prefill_seed(self, cache: Cache, q_prompt: torch.Tensor, scale, gamma: float):
+        """q_prompt [L][B][P][Hq][D] on the device, cache dtype; overwrites rel[0..P) of every item."""
+        assert q_prompt.is_cuda and q_prompt.is_contiguous() and q_prompt.dim() == 5
+        self._check(self.lib.lethe_prefill_seed(self.h, ctypes.byref(cache.c), _dp(q_prompt), q_prompt.shape[2],
+                                                self._scale(scale), gamma, _stream(self.device)))

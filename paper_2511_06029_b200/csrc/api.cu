@@ -31,6 +31,25 @@ cudaError_t launch_rasr_prune(const CacheView& c, const int32_t* budgets, int re
                               cudaStream_t stream);
 }  // namespace lethe
 
+namespace lethe {
+struct PrefillArgs {
+    const void* k;
+    const int32_t* page_table;
+    const int32_t* len;
+    float* rel;
+    const void* q;
+    float2* stats;
+    int32_t* status;
+    long long n_pages;
+    int B, Hq, Hkv, G, HP, P;
+    int capacity, cap_tokens, page_tokens, paged;
+    float gamma_log2;
+    float scale_log2[kMaxLayers];
+};
+size_t prefill_stats_bytes(int items, int P, int HP);
+cudaError_t launch_prefill(const PrefillArgs& a, int items, int D, cudaStream_t stream);
+}  // namespace lethe
+
 using namespace lethe;
 
 #include <map>
@@ -600,6 +619,44 @@ lethe_status lethe_segment_prune(lethe_ctx* ctx, const lethe_cache* c, int32_t n
                                          smem_tokens, list_scratch, ctx->status, (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "segment_prune launch");
     return refresh_order(ctx, c, v, stream);
+}
+
+lethe_status lethe_prefill_seed(lethe_ctx* ctx, const lethe_cache* c, const void* q_prompt, int32_t prompt_len,
+                                const float* scale, float gamma, void* stream) {
+    lethe_status st = check_cache(ctx, c);
+    if (st != LETHE_OK) return st;
+    if (!q_prompt || !scale) return fail(ctx, LETHE_ERR_INVALID_ARG, "q_prompt and scale are required");
+    if (prompt_len < 1 || prompt_len > cap_tokens_of(c)) return fail(ctx, LETHE_ERR_INVALID_ARG, "prompt_len out of range");
+    if (!(gamma > 0.f && gamma <= 1.f)) return fail(ctx, LETHE_ERR_INVALID_ARG, "gamma must be in (0, 1]");
+    if (c->dtype != LETHE_BF16) return fail(ctx, LETHE_ERR_UNSUPPORTED, "prefill seeding needs a bf16 cache");
+    if (c->n_layers > kMaxLayers) return fail(ctx, LETHE_ERR_UNSUPPORTED, "more than 128 layers");
+    const int G = c->n_q_heads / c->n_kv_heads;
+    if (G > kMaxGroup) return fail(ctx, LETHE_ERR_UNSUPPORTED, "more than 8 query heads per KV head");
+    if ((uintptr_t)q_prompt & 15) return fail(ctx, LETHE_ERR_INVALID_ARG, "q_prompt must be 16-byte aligned");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, LETHE_ERR_CUDA, "cannot select the context's device");
+    PrefillArgs a;
+    memset(&a, 0, sizeof(a));
+    a.k = c->k; a.page_table = c->page_table; a.len = c->len; a.rel = c->rel; a.q = q_prompt;
+    a.status = ctx->status;
+    a.n_pages = c->n_pages;
+    a.B = c->batch; a.Hq = c->n_q_heads; a.Hkv = c->n_kv_heads; a.G = G; a.P = prompt_len;
+    a.HP = G <= 1 ? 1 : (G <= 2 ? 2 : (G <= 4 ? 4 : 8));
+    a.capacity = c->capacity; a.cap_tokens = cap_tokens_of(c);
+    a.paged = c->layout == LETHE_PAGED;
+    a.page_tokens = a.paged ? c->page_tokens : 1;
+    a.gamma_log2 = log2f(gamma);
+    for (int l = 0; l < c->n_layers; ++l) {
+        if (!(scale[l] == scale[l]) || fabsf(scale[l]) > 1e30f) return fail(ctx, LETHE_ERR_INVALID_ARG, "scale must be finite");
+        a.scale_log2[l] = scale[l] * 1.4426950408889634f;
+    }
+    const int items = c->n_layers * c->batch * c->n_kv_heads;
+    st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, prefill_stats_bytes(items, prompt_len, a.HP), "prefill statistics");
+    if (st != LETHE_OK) return st;
+    a.stats = (float2*)ctx->scratch;
+    cudaError_t e = launch_prefill(a, items, c->head_dim, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "prefill_seed launch");
+    return LETHE_OK;
 }
 
 }  // extern "C"
