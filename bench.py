@@ -349,6 +349,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-per-layer", action="store_true")
+    ap.add_argument("--with-prefill", action="store_true",
+                    help="also time lethe_prefill_seed on a prompt of the workload's length (informational)")
     ap.add_argument("--pl-variant", type=int, default=0, help="kernel variant of the per-layer launch mode")
     ap.add_argument("--pl-splits", type=int, default=0)
     args = ap.parse_args()
@@ -457,6 +459,38 @@ def main():
             segment[f"tau_{int(tau)}"] = {"ms": a_ev.elapsed_time(b_ev), "token_heads_before": before,
                                           "token_heads_after": int(r.cache.len.sum().item())}
         r.check()
+    prefill = None
+    if args.with_prefill and world == 1:
+        from paper_2511_06029_b200 import binding
+        P = w.prompt_len
+        gq = torch.Generator(device=dev); gq.manual_seed(99)
+        kp = torch.randn((w.n_layers, w.batch, w.n_kv_heads, P, w.head_dim), generator=gq, device=dev).to(w.dtype)
+        pc = binding.Cache(w.n_q_heads, kp, torch.zeros_like(kp),
+                           torch.zeros((w.n_layers, w.batch, w.n_kv_heads, P), device=dev),
+                           torch.zeros((w.n_layers, w.batch, w.n_kv_heads, P), dtype=torch.int32, device=dev),
+                           torch.full((w.n_layers, w.batch, w.n_kv_heads), P, dtype=torch.int32, device=dev))
+        qp = torch.randn((w.n_layers, w.batch, P, w.n_q_heads, w.head_dim), generator=gq, device=dev).to(w.dtype)
+        for _ in range(2):
+            r.ctx.prefill_seed(pc, qp, r.scale, w.gamma)
+        a_ev = torch.cuda.Event(enable_timing=True); b_ev = torch.cuda.Event(enable_timing=True)
+        a_ev.record()
+        for _ in range(5):
+            r.ctx.prefill_seed(pc, qp, r.scale, w.gamma)
+        b_ev.record()
+        torch.cuda.synchronize(dev)
+        r.check()
+        ms_p = a_ev.elapsed_time(b_ev) / 5
+        flops = 2.0 * pc.len.numel() * w.group * (P * (P + 1) / 2) * w.head_dim * 2   # two passes over the causal half
+        peaks = {}
+        try:
+            peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        except Exception:
+            pass
+        tf = flops / (ms_p * 1e-3) / 1e12
+        prefill = {"prompt_len": P, "ms": ms_p, "useful_TFLOPs": tf, "bound": "tensor",
+                   "frac_of_measured_bf16_burst": (tf / peaks["bf16_tflops"]) if "bf16_tflops" in peaks else None,
+                   "note": "two mma.sync passes (statistics, column sums); launches: 2 per call"}
+        del pc, kp, qp
     e_ms = e_total_ms if not args.no_e2e else 0.0
     e_u = float(sum(e_th)) if not args.no_e2e else 0.0
     (t_ms, e_total_ms), (units, e_units) = dist_util.reduce_job(dist, dev, [total_ms, e_ms], [float(sum(th)), e_u])
@@ -482,7 +516,8 @@ def main():
                 "attend_ms_per_step": avg_attend_ms,
                 "attend_ms_median": statistics.median(attend_ms),
                 "per_layer_launch": per_layer,
-                "segment_prune_8_segments": segment}),
+                "segment_prune_8_segments": segment,
+                "prefill_seed": prefill}),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": f"of {which}", "frac_of_8TBs_nominal": achieved / 8000.0,
                          "kernel": "attend (dominant kernel; one launch per step)",
