@@ -343,14 +343,14 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         if (!mma_ok) variant = 1;
         else if (a.n_items >= 2 * ctx->sm_count && ctx->splits <= 1) {
             // Persistent kernels, best measured first, taking the first whose logit buffer(s) cover the
-            // capacity on chip: asynchronous epilogue (6,3) (5,3) (4,4), then the synchronous (7,3) (6,3) (8,2).
+            // capacity on chip: asynchronous epilogue (5,3) (6,3) (8,2) (4,4), then the synchronous (7,3) (6,3) (8,2).
             // If none does, the tail of long items overflows to scratch: asynchronous (5,3) when each of its two
             // buffers still holds most of the capacity, else the synchronous (6,3), whose single buffer is
             // twice as long.
             const int cap_pad = cap_groups * kGroupTokens;
             auto async_fits = [&](int shape) { return async_smem_bytes(c->head_dim, shape, cap_pad, a.GP) <= ctx->max_smem; };
             variant = 0;
-            for (int shape : {2, 3, 5})
+            for (int shape : {3, 2, 0, 5})
                 if (variant == 0 && async_fits(shape)) variant = 16 + shape;
             for (int shape : {4, 1, 0})
                 if (variant == 0 && stream_chunk(shape) == cap_pad) variant = 8 + shape;

@@ -367,6 +367,26 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
             constexpr bool OVF = SPILL;
             for (int it = 0; it < cur.count; ++it) {
                 const int cslot = (vp + it) % NS;
+                // Refill first, wait second: the slot of group it-1 is free as soon as every lane has left the
+                // previous iteration, so the copy of the group NS-1 ahead (possibly of the next item) is already
+                // in flight while this warp waits for group `it`.
+                __syncwarp();
+                const bool strict = !TMA && topped && it < NS - 1;  // after a top-up the group order is not the commit order
+                if (strict) cp_async_wait<0>();
+                {
+                    const int idx = it + NS - 1;
+                    const int slot = (vp + idx) % NS;
+                    if (idx < cur.count) issue(cur, idx, slot, true);
+                    else {
+                        if (!nxt_ready) acquire_next();
+                        const int j = idx - cur.count;
+                        if (nxt.valid && j < nxt.count) {
+                            issue(nxt, j, slot, false);
+                            issued_next |= 1u << j;
+                        }
+                    }
+                    cp_async_commit();
+                }
                 if constexpr (TMA) {
                     if (!mbar_wait_tile(&hd.tma_full[warp][cslot], (slot_phase >> cslot) & 1u, abort_flag)) {
                         alive = false;
@@ -387,24 +407,9 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
                         }
                     }
                 } else {
-                    if (topped && it < NS - 1) cp_async_wait<0>();
-                    else cp_async_wait<NS - 2>();
+                    if (!strict) cp_async_wait<NS - 1>();  // everything but the NS-1 newest groups, i.e. group `it`, has landed
                 }
                 __syncwarp();
-                {
-                    const int idx = it + NS - 1;
-                    const int slot = (vp + idx) % NS;
-                    if (idx < cur.count) issue(cur, idx, slot, true);
-                    else {
-                        if (!nxt_ready) acquire_next();
-                        const int j = idx - cur.count;
-                        if (nxt.valid && j < nxt.count) {
-                            issue(nxt, j, slot, false);
-                            issued_next |= 1u << j;
-                        }
-                    }
-                    cp_async_commit();
-                }
                 const int grp = warp + it * NWS;
                 const uint32_t ks_u32 = my_stage_u32 + ((vp + it) % NS) * STAGE_BYTES;
                 const uint32_t vs_u32 = ks_u32 + TILE_BYTES;

@@ -216,10 +216,13 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
             for (int i = 0; i < 4; ++i) o[mt][i] = 0.f;
 
         for (int it = 0; it < cur.count; ++it) {
-            if (topped && it < NS - 1) cp_async_wait<0>();
-            else cp_async_wait<NS - 2>();
-            __syncwarp();  // group `it` has landed for every lane; every lane is done with group it-1
-            {              // refill the slot freed by group it-1 with the group NS-1 ahead (possibly of the next item)
+            // Refill first, wait second: the slot of group it-1 is free once every lane has left the previous
+            // iteration, so the copy of the group NS-1 ahead (possibly of the next item) is already in flight
+            // while this warp waits for group `it`.
+            __syncwarp();
+            const bool strict = topped && it < NS - 1;  // after a top-up the group order is not the commit order
+            if (strict) cp_async_wait<0>();
+            {
                 const int idx = it + NS - 1;
                 const int slot = (vp + idx) % NS;
                 if (idx < cur.count) issue(cur, idx, slot, true);
@@ -237,6 +240,8 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
                 }
                 cp_async_commit();
             }
+            if (!strict) cp_async_wait<NS - 1>();  // everything but the NS-1 newest groups, i.e. group `it`, has landed
+            __syncwarp();
             const int grp = warp + it * NW;
             const uint32_t ks_u32 = my_stage_u32 + ((vp + it) % NS) * STAGE_BYTES;
             const uint32_t vs_u32 = ks_u32 + TILE_BYTES;
