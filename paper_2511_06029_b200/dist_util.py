@@ -27,3 +27,18 @@ def reduce_job(dist, device, times_ms: Sequence[float], units: Sequence[float]) 
 def job_value(units_total: float, max_time_ms: float) -> float:
     """Whole-job throughput: all units of all ranks over the slowest rank's time."""
     return units_total / (max_time_ms * 1e-3)
+
+
+def allreduce_layer_sparsity(dist, local_sparsity: torch.Tensor, local_kv_heads: int, total_kv_heads: int) -> torch.Tensor:
+    """Layer sparsity of a cache sharded by KV head (tensor-parallel attention).
+
+    `lethe_estimate_sparsity` returns, per (layer, sequence), the mean Hoyer sparsity over the KV heads a rank
+    holds.  The layer value of Sec. 4.2 is the mean over all heads, so ranks exchange one [L][B] fp32 tensor per
+    prune round: sum over ranks of (local mean x local head count), divided by the total head count.  Every rank
+    then calls `lethe_alloc_budgets` on the same values and, the allocator being integer arithmetic, gets the
+    same budgets.  This is the only exchange a head-sharded run of the path needs.
+    """
+    s = local_sparsity.to(torch.float32) * float(local_kv_heads)
+    if dist is not None:
+        dist.all_reduce(s, op=dist.ReduceOp.SUM)
+    return s / float(total_kv_heads)

@@ -43,3 +43,44 @@ def test_two_rank_sharding_and_reduction():
     assert dist_util.job_value(300.0, 15.0) == 20000.0
     t, u = dist_util.reduce_job(None, None, [1.0], [2.0])
     assert t == [1.0] and u == [2.0]
+
+
+def _tp_worker(rank, world, port, ret):
+    """Each rank holds half of the KV heads of the same cache; after the one all-reduce both must allocate the
+    budgets an unsharded run allocates, and prune their own heads exactly as the unsharded run prunes them."""
+    import oracle
+    os.environ["MASTER_ADDR"] = "127.0.0.1"; os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        L, B, Hq, Hkv, D, cap, n = 4, 2, 8, 4, 8, 96, 80
+        g = torch.Generator().manual_seed(5)
+        k = torch.randn((L, B, Hkv, cap, D), generator=g); v = torch.randn((L, B, Hkv, cap, D), generator=g)
+        rel = torch.rand((L, B, Hkv, cap), generator=g) ** 4
+        pos = torch.arange(cap, dtype=torch.int32).expand(L, B, Hkv, cap).contiguous()
+        full = oracle.OracleCache(L, B, Hq, Hkv, D, cap, k.clone(), v.clone(), rel.clone(), pos.clone(),
+                                  torch.full((L, B, Hkv), n, dtype=torch.int32))
+        hs = slice(rank * 2, rank * 2 + 2)
+        mine = oracle.OracleCache(L, B, Hq // 2, 2, D, cap, k[:, :, hs].contiguous(), v[:, :, hs].contiguous(),
+                                  rel[:, :, hs].contiguous(), pos[:, :, hs].contiguous(),
+                                  torch.full((L, B, 2), n, dtype=torch.int32))
+        T = torch.tensor([L * 40, L * 55], dtype=torch.int64)
+        _, S_full = oracle.estimate_sparsity(full)
+        _, bud_full = oracle.alloc_budgets(S_full, T, 12)
+        oracle.rasr_prune(full, bud_full, 8, 4)
+        _, S_loc = oracle.estimate_sparsity(mine)
+        S_all = dist_util.allreduce_layer_sparsity(dist, S_loc, 2, Hkv)
+        _, bud = oracle.alloc_budgets(S_all.contiguous(), T, 12)
+        oracle.rasr_prune(mine, bud, 8, 4)
+        ret[rank] = (torch.allclose(S_all, S_full, atol=1e-6), torch.equal(bud, bud_full),
+                     torch.equal(mine.len, full.len[:, :, hs]), torch.equal(mine.pos, full.pos[:, :, hs]),
+                     torch.equal(mine.k, full.k[:, :, hs]))
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_rank_head_sharded_prune_round():
+    mgr = mp.Manager(); ret = mgr.dict()
+    mp.spawn(_tp_worker, args=(2, _free_port(), ret), nprocs=2, join=True)
+    for rank in range(2):
+        assert all(ret[rank]), ret[rank]
