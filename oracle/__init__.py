@@ -68,6 +68,9 @@ def lib():
         _lib.oracle_segment_prune.restype = ctypes.c_int
         _lib.oracle_segment_prune.argtypes = [ctypes.POINTER(_CCache), ctypes.c_int32, ctypes.c_float, ctypes.c_int32,
                                               ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32]
+        _lib.oracle_collapsed_prune.restype = ctypes.c_int
+        _lib.oracle_collapsed_prune.argtypes = [ctypes.POINTER(_CCache), ctypes.c_void_p, ctypes.c_int32,
+                                                ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int32]
         _lib.oracle_prefill_seed.restype = ctypes.c_int
         _lib.oracle_prefill_seed.argtypes = [ctypes.POINTER(_CCache), ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p,
                                              ctypes.c_float]
@@ -201,6 +204,21 @@ def segment_prune(cache: OracleCache, n_segments: int, tau: float, recent: int, 
     cc = cache._c()
     st = lib().oracle_segment_prune(ctypes.byref(cc), int(n_segments), ctypes.c_float(tau), int(recent), int(sink),
                                     _ptr(l_evict), _ptr(keep), int(max_k))
+    return st, keep
+
+
+COLLAPSE_HEADS, COLLAPSE_HEADS_BATCH = 0, 1
+
+
+def collapsed_prune(cache: OracleCache, budgets: torch.Tensor, recent: int, sink: int, scope: int, max_k: int = 0):
+    """Eq. 2 as printed: one score and one retention set per (layer, sequence) [scope 0, budgets [L][B]] or per
+    layer [scope 1, budgets [L]]; returns (status, keep_idx [groups][max_k] or None)."""
+    groups = cache.n_layers * cache.batch if scope == COLLAPSE_HEADS else cache.n_layers
+    assert budgets.dtype == torch.int32 and budgets.numel() == groups
+    keep = torch.zeros((groups, max_k), dtype=torch.int32) if max_k > 0 else None
+    cc = cache._c()
+    st = lib().oracle_collapsed_prune(ctypes.byref(cc), _ptr(budgets.contiguous()), int(recent), int(sink), int(scope),
+                                      _ptr(keep), int(max_k))
     return st, keep
 
 

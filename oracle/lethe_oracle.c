@@ -35,6 +35,10 @@
  *                             (sequence, KV head).  Eq. 4 is read as
  *                             v_head >= tau * v_cut (as printed, v_head / v_cut <= tau
  *                             with tau > 1 could only fire at the first cut or never).
+ *   oracle_collapsed_prune    Eq. 2 as printed: ONE score per token per layer, the relevance
+ *                             summed over all heads (and, in the wider scope, over the
+ *                             batch), and one retention set shared by everything summed
+ *                             over; same protected top-k and compaction as oracle_rasr_prune.
  *
  * Arithmetic: every floating-point step is done in double; stored results are
  * rounded once to their storage type (fp32, or bf16 round-to-nearest-even).
@@ -545,6 +549,101 @@ int oracle_segment_prune(oracle_cache *c, int32_t n_segments, float tau, int32_t
         free(top);
     }
     return ORACLE_OK;
+}
+
+/* ---- Eq. 2 as printed: one collapsed score, one retention set per group ---- */
+/*
+ * scope 0: a group is the Hkv items of one (layer, sequence); budgets [L][B].
+ * scope 1: a group is the B * Hkv items of one layer (Eq. 2 also sums over b); budgets [L].
+ * Slot j must mean the same token in every item of a group, so all of them must have the same
+ * len (true when they were only ever appended to and pruned together); a group that breaks this
+ * is left untouched and the call reports ORACLE_ERR_INVALID_ARG.
+ *   score[j] = sum over the group's items, in ascending (b, h) order, of rel[item][j]
+ * The sum decides an integer result (who is kept), so it is taken in fp32 — the precision rel is
+ * stored in — one rounded add per item.  With k = the group's budget: k >= n keeps everything;
+ * otherwise sinks, the recent window and the highest scores among the rest (ties to the lower
+ * slot) are kept exactly as in oracle_rasr_prune, and the same slot list compacts every item of
+ * the group (each keeps its own K, V, rel and pos rows).
+ * keep_idx (optional) [groups][max_k]: the survivors' old slots, ascending, padded with -1.
+ */
+int oracle_collapsed_prune(oracle_cache *c, const int32_t *budgets, int32_t recent, int32_t sink, int32_t scope,
+                           int32_t *keep_idx, int32_t max_k) {
+    int st = check_cache(c);
+    if (st) return st;
+    if (!budgets || recent < 0 || sink < 0 || (scope != 0 && scope != 1)) return ORACLE_ERR_INVALID_ARG;
+    if (keep_idx && max_k < 1) return ORACLE_ERR_INVALID_ARG;
+    const int64_t capT = cap_tokens(c);
+    const size_t row_bytes = (size_t)c->head_dim * elt_size(c->dtype);
+    const int per_group = scope == 0 ? c->n_kv_heads : c->batch * c->n_kv_heads;
+    const int n_groups = scope == 0 ? c->n_layers * c->batch : c->n_layers;
+    int result = ORACLE_OK;
+    for (int g = 0; g < n_groups; ++g) {
+        const int64_t first = (int64_t)g * per_group; /* items of a group are consecutive in [L][B][Hkv] order */
+        const int64_t n = c->len[first];
+        int32_t *kout = keep_idx ? keep_idx + (int64_t)g * max_k : NULL;
+        if (kout)
+            for (int i = 0; i < max_k; ++i) kout[i] = -1;
+        int aligned = 1;
+        for (int t = 1; t < per_group; ++t)
+            if (c->len[first + t] != n) aligned = 0;
+        if (!aligned) {
+            if (result == ORACLE_OK) result = ORACLE_ERR_INVALID_ARG;
+            continue;
+        }
+        int64_t k = budgets[g];
+        if (k < 0) k = 0;
+        if (k >= n) {
+            if (kout)
+                for (int64_t i = 0; i < n && i < max_k; ++i) kout[i] = (int32_t)i;
+            continue;
+        }
+        const int64_t n_sink = sink < n ? sink : n;
+        const int64_t n_recent = recent < n ? recent : n;
+        int64_t cand_lo = n_sink, cand_hi = n - n_recent;
+        if (cand_hi < cand_lo) cand_hi = cand_lo;
+        const int64_t n_prot = n - (cand_hi - cand_lo);
+        if (n_prot > k) {
+            k = n_prot;
+            if (result == ORACLE_OK) result = ORACLE_ERR_BUDGET;
+        }
+        const int64_t take = k - n_prot;
+
+        char *keep = (char *)calloc((size_t)(n > 0 ? n : 1), 1);
+        for (int64_t j = 0; j < cand_lo; ++j) keep[j] = 1;
+        for (int64_t j = cand_hi; j < n; ++j) keep[j] = 1;
+        if (take > 0) {
+            const int64_t nc = cand_hi - cand_lo;
+            cand_t *cand = (cand_t *)malloc(sizeof(cand_t) * (size_t)nc);
+            for (int64_t j = 0; j < nc; ++j) {
+                float score = 0.0f;
+                for (int t = 0; t < per_group; ++t) score = score + c->rel[(first + t) * capT + cand_lo + j];
+                cand[j].score = score;
+                cand[j].idx = (int32_t)(cand_lo + j);
+            }
+            qsort(cand, (size_t)nc, sizeof(cand_t), cand_cmp);
+            for (int64_t i = 0; i < take; ++i) keep[cand[i].idx] = 1;
+            free(cand);
+        }
+        for (int t = 0; t < per_group; ++t) {
+            const int64_t item = first + t;
+            int64_t m = 0;
+            for (int64_t s = 0; s < n; ++s) {
+                if (!keep[s]) continue;
+                if (t == 0 && kout && m < max_k) kout[m] = (int32_t)s;
+                if (s != m) {
+                    const int64_t so = row_offset(c, item, s), d_o = row_offset(c, item, m);
+                    memmove((char *)c->k + d_o * elt_size(c->dtype), (char *)c->k + so * elt_size(c->dtype), row_bytes);
+                    memmove((char *)c->v + d_o * elt_size(c->dtype), (char *)c->v + so * elt_size(c->dtype), row_bytes);
+                    c->rel[item * capT + m] = c->rel[item * capT + s];
+                    c->pos[item * capT + m] = c->pos[item * capT + s];
+                }
+                ++m;
+            }
+            c->len[item] = (int32_t)m;
+        }
+        free(keep);
+    }
+    return result;
 }
 
 /* ---- relevance of the prompt from the prefill attention (Eq. 2, Q > 1; Eq. 5) ---- */

@@ -480,3 +480,140 @@ def test_prefill_seed_against_library_softmax_and_closed_forms():
     assert torch.allclose(c2.rel[0, 0, 0, :5], want, atol=1e-6)
     short = random_cache(1, 1, 1, 1, 4, 8, 3, seed=1)
     assert oracle.prefill_seed(short, torch.zeros((1, 1, 5, 1, 4)), torch.tensor([1.0]), 1.0) == oracle.ERR_CAPACITY
+
+
+# ----------------------------------------------------------------------------- collapsed score (Eq. 2 as printed)
+
+def _collapsed_cache(rel, D=4, seed=0, extra=2):
+    """rel [B][Hkv][n] -> one-layer cache with those scores."""
+    rel = torch.tensor(rel, dtype=torch.float32)
+    B, H, n = rel.shape
+    c = random_cache(1, B, H, H, D, n + extra, n, seed=seed)
+    c.rel[0, :, :, :n] = rel
+    return c
+
+
+def test_golden_collapsed():
+    g = GOLD["collapsed"]
+    c = _collapsed_cache(g["rel"])
+    st, keep = oracle.collapsed_prune(c, torch.tensor([g["heads"]["budget"]] * 2, dtype=torch.int32), g["recent"], g["sink"],
+                                      oracle.COLLAPSE_HEADS, max_k=8)
+    assert st == oracle.OK
+    assert [[i for i in row if i >= 0] for row in keep.tolist()] == g["heads"]["expect"]
+    for case in g["heads_batch"]:
+        c = _collapsed_cache(g["rel"])
+        st, keep = oracle.collapsed_prune(c, torch.tensor([case["budget"]], dtype=torch.int32), g["recent"], g["sink"],
+                                          oracle.COLLAPSE_HEADS_BATCH, max_k=8)
+        assert st == oracle.OK and [i for i in keep[0].tolist() if i >= 0] == case["expect"]
+        assert torch.all(c.len == case["budget"])
+
+
+def test_collapsed_with_one_item_per_group_is_the_per_head_rule():
+    """One KV head per sequence (and one sequence for the batch scope): the collapsed sum is the head's own score,
+    so the call must leave exactly the bytes oracle_rasr_prune leaves."""
+    for scope, B in ((oracle.COLLAPSE_HEADS, 3), (oracle.COLLAPSE_HEADS_BATCH, 1)):
+        a = random_cache(2, B, 2, 1, 8, 300, 260, seed=3, rel_init="rand")
+        a.rel[:, :, :, 50:90] = 0.5                                    # ties
+        b = a.clone()
+        bud = torch.tensor([[90] * B, [400] * B], dtype=torch.int32)
+        st_a, keep_a = oracle.rasr_prune(a, bud, 16, 4, max_k=300)
+        st_b, keep_b = oracle.collapsed_prune(b, bud.flatten() if scope == oracle.COLLAPSE_HEADS else bud[:, 0].contiguous(),
+                                              16, 4, scope, max_k=300)
+        assert st_a == st_b == oracle.OK and torch.equal(keep_a.reshape(keep_b.shape), keep_b)
+        for name in ("k", "v", "rel", "pos", "len"):
+            assert torch.equal(getattr(a, name), getattr(b, name)), name
+
+
+def test_collapsed_brute_force_tiny():
+    """Sum the heads with numpy fp32 in (b, h) order, enumerate every size-k superset of the protected set, and
+    check that the kept set is the best one (largest collapsed sum, then lexicographically smallest), that all
+    items of a group were compacted by that same list and that each kept its own rows."""
+    import numpy as np
+    g = torch.Generator().manual_seed(29)
+    for trial in range(80):
+        B = int(torch.randint(1, 3, (1,), generator=g)); H = int(torch.randint(1, 4, (1,), generator=g))
+        n = int(torch.randint(3, 11, (1,), generator=g))
+        sink = int(torch.randint(0, 3, (1,), generator=g)); recent = int(torch.randint(0, 3, (1,), generator=g))
+        prot = set(range(min(sink, n))) | set(range(n - min(recent, n), n))
+        if len(prot) >= n:
+            continue
+        k = int(torch.randint(len(prot), n, (1,), generator=g))
+        rel = torch.randint(0, 4, (B, H, n), generator=g).float() * 0.25
+        for scope in (oracle.COLLAPSE_HEADS, oracle.COLLAPSE_HEADS_BATCH):
+            c = _collapsed_cache(rel.tolist(), seed=trial)
+            before = c.clone()
+            groups = B if scope == oracle.COLLAPSE_HEADS else 1
+            st, keep = oracle.collapsed_prune(c, torch.full((groups,), k, dtype=torch.int32), recent, sink, scope, max_k=n)
+            assert st == oracle.OK
+            for gi in range(groups):
+                members = [(gi, h) for h in range(H)] if scope == oracle.COLLAPSE_HEADS else [(b, h) for b in range(B) for h in range(H)]
+                score = np.zeros(n, dtype=np.float32)
+                for (b, h) in members:
+                    score = (score + rel[b, h].numpy()).astype(np.float32)
+                rest = [j for j in range(n) if j not in prot]
+                best = min((-float(sum(score[j] for j in extra)), tuple(extra))
+                           for extra in itertools.combinations(rest, k - len(prot)))
+                kept = [i for i in keep[gi].tolist() if i >= 0]
+                assert tuple(sorted(set(kept) - prot)) == best[1] and prot <= set(kept) and len(kept) == k
+                idx = torch.tensor(kept, dtype=torch.long)
+                for (b, h) in members:
+                    assert int(c.len[0, b, h]) == k
+                    for name in ("k", "v", "rel", "pos"):
+                        assert torch.equal(getattr(c, name)[0, b, h, :k], getattr(before, name)[0, b, h, idx]), name
+
+
+def test_collapsed_identical_heads_keep_what_each_head_would_keep():
+    """When every head of a sequence holds the same scores the sum is a power-of-two multiple of them (4 heads):
+    order and ties are unchanged, so the shared set equals every head's own set."""
+    a = random_cache(1, 2, 4, 4, 8, 500, 450, seed=8, rel_init="rand")
+    a.rel[:] = a.rel[:, :, :1]
+    a.rel[:, :, :, 100:160] = 0.25
+    b = a.clone()
+    bud = torch.tensor([[120, 333]], dtype=torch.int32)
+    st_a, _ = oracle.rasr_prune(a, bud, 32, 4)
+    st_b, _ = oracle.collapsed_prune(b, bud.flatten(), 32, 4, oracle.COLLAPSE_HEADS)
+    assert st_a == st_b == oracle.OK
+    for name in ("k", "v", "rel", "pos", "len"):
+        assert torch.equal(getattr(a, name), getattr(b, name)), name
+
+
+def test_collapsed_sum_is_taken_in_fp32_in_head_order():
+    """Slot 1 holds (2^24, 1, 1), slot 2 holds (2^24, 2, 0).  Exactly both sum to 2^24 + 2 and the older slot 1
+    would win the tie; in fp32, adding head by head, slot 1 stays at 2^24 (each +1 rounds back to even) and slot 2
+    reaches 2^24 + 2, so slot 2 is the one kept.  The decision is documented as an fp32 one."""
+    big = float(2 ** 24)
+    rel = [[[0, big, big, 0, 0], [0, 1, 2, 0, 0], [0, 1, 0, 0, 0]]]
+    c = _collapsed_cache(rel)
+    st, keep = oracle.collapsed_prune(c, torch.tensor([3], dtype=torch.int32), 1, 1, oracle.COLLAPSE_HEADS, max_k=5)
+    assert st == oracle.OK and [i for i in keep[0].tolist() if i >= 0] == [0, 2, 4]
+
+
+def test_collapsed_special_cases():
+    base = random_cache(2, 2, 4, 2, 8, 64, 50, seed=4, rel_init="rand")
+    # budget >= length: identity
+    c = base.clone()
+    st, keep = oracle.collapsed_prune(c, torch.tensor([50, 60, 70, 80], dtype=torch.int32), 8, 2, oracle.COLLAPSE_HEADS, max_k=64)
+    assert st == oracle.OK and keep[0].tolist() == list(range(50)) + [-1] * 14
+    for name in ("k", "v", "rel", "pos", "len"):
+        assert torch.equal(getattr(c, name), getattr(base, name))
+    # heads of one sequence out of step: that group is refused and untouched, the others are pruned
+    c = base.clone(); c.len[0, 1, 1] = 49
+    ref = c.clone()
+    st, keep = oracle.collapsed_prune(c, torch.tensor([20] * 4, dtype=torch.int32), 8, 2, oracle.COLLAPSE_HEADS, max_k=64)
+    assert st == oracle.ERR_INVALID_ARG
+    assert c.len[0, 1].tolist() == [50, 49] and torch.equal(c.k[0, 1], ref.k[0, 1]) and torch.all(keep[1] == -1)
+    assert c.len[0, 0].tolist() == [20, 20] and c.len[1].flatten().tolist() == [20] * 4
+    # protected set above the budget: exactly the protected set, flagged
+    c = base.clone()
+    st, keep = oracle.collapsed_prune(c, torch.tensor([5, 5], dtype=torch.int32), 8, 2, oracle.COLLAPSE_HEADS_BATCH, max_k=64)
+    assert st == oracle.ERR_BUDGET and torch.all(c.len == 10)
+    assert [i for i in keep[0].tolist() if i >= 0] == [0, 1] + list(range(42, 50))
+    # batch scope on (B, Hkv) equals head scope on the same items seen as (1, B * Hkv)
+    a = base.clone()
+    b = oracle.OracleCache(2, 1, 8, 4, 8, 64, base.k.reshape(2, 1, 4, 64, 8).clone(), base.v.reshape(2, 1, 4, 64, 8).clone(),
+                           base.rel.reshape(2, 1, 4, 64).clone(), base.pos.reshape(2, 1, 4, 64).clone(),
+                           base.len.reshape(2, 1, 4).clone())
+    bud = torch.tensor([17, 33], dtype=torch.int32)
+    st_a, keep_a = oracle.collapsed_prune(a, bud, 8, 2, oracle.COLLAPSE_HEADS_BATCH, max_k=64)
+    st_b, keep_b = oracle.collapsed_prune(b, bud, 8, 2, oracle.COLLAPSE_HEADS, max_k=64)
+    assert st_a == st_b == oracle.OK and torch.equal(keep_a, keep_b) and torch.equal(a.k.flatten(), b.k.flatten())
