@@ -441,6 +441,24 @@ def main():
                      "mode": f"{w.n_layers} launches per step (one per layer), replayed from a CUDA graph, "
                              f"{pl_steps} steps; not part of `value`"}
 
+    # Retention by the collapsed score of Eq. 2 (one set per sequence), timed once on the live state with the
+    # budgets a RASR round would get now: the row traffic of such a round.  Only the heads' lengths are aligned here (the
+    # earlier rounds pruned head by head), so this is a timing of the call, not a meaningful retention.
+    collapsed = None
+    if not args.no_per_layer and world == 1:
+        from paper_2511_06029_b200 import binding as _b
+        r.ctx.estimate_sparsity(r.cache, r.S)
+        r.ctx.alloc_budgets(r.S, r.T, w.k_min, r.budgets)
+        before = int(r.cache.len.sum().item())
+        a_ev = torch.cuda.Event(enable_timing=True); b_ev = torch.cuda.Event(enable_timing=True)
+        a_ev.record()
+        r.ctx.collapsed_prune(r.cache, r.budgets, w.recent, w.sink, _b.COLLAPSE_HEADS)
+        b_ev.record()
+        torch.cuda.synchronize(dev)
+        r.check()
+        collapsed = {"scope": "heads (one set per layer and sequence)", "ms": a_ev.elapsed_time(b_ev),
+                     "token_heads_before": before, "token_heads_after": int(r.cache.len.sum().item())}
+
     # Algorithm 1 (threshold-triggered, budget-free retention) timed once on the live state, after everything
     # that enters `value`: first with the paper's default sparse_ratio (tau = 400), then with a small tau that
     # does find breakpoints and therefore also compacts.
@@ -517,6 +535,7 @@ def main():
                 "attend_ms_median": statistics.median(attend_ms),
                 "per_layer_launch": per_layer,
                 "segment_prune_8_segments": segment,
+                "collapsed_prune": collapsed,
                 "prefill_seed": prefill}),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": f"of {which}", "frac_of_8TBs_nominal": achieved / 8000.0,

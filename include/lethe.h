@@ -19,6 +19,7 @@
  *                            (Eq. 2 with Q > 1)
  *   lethe_segment_prune      Algorithm 1 itself: segmented breakpoint search, retention
  *                            set and eviction-threshold update (Sec. 4.2)
+ *   lethe_collapsed_prune    retention by the head- and batch-collapsed score of Eq. 2
  *
  * General conventions
  *   - Unless marked HOST, every pointer is a DEVICE pointer to memory owned by the
@@ -215,6 +216,29 @@ lethe_status lethe_rasr_prune(lethe_ctx *ctx, const lethe_cache *cache, const in
 lethe_status lethe_segment_prune(lethe_ctx *ctx, const lethe_cache *cache, int32_t n_segments, float tau,
                                  int32_t recent, int32_t sink, int32_t *l_evict, int32_t *keep_idx, int32_t max_k,
                                  void *stream);
+
+/*
+ * Retention with the collapsed score of Eq. 2 as the paper prints it: the attention a token received is summed
+ * over ALL heads of the layer (LETHE_COLLAPSE_HEADS) and also over the batch (LETHE_COLLAPSE_HEADS_BATCH), giving
+ * one score per token and ONE retention set shared by every item summed over, instead of one per KV head.
+ *   group   : the Hkv items of one (layer, sequence), or the B * Hkv items of one layer;
+ *   budgets : one int32 per group — [L][B], or [L];
+ *   score[j] = sum of rel[item][j] over the group's items in ascending (sequence, KV head) order, in fp32 with
+ *              one rounded add per item (the sum decides who is kept, so its precision and order are fixed);
+ *   then exactly as lethe_rasr_prune: k >= n keeps everything; otherwise the first `sink` and last `recent`
+ *   slots plus the highest scores among the rest (ties to the lower slot) survive, and every item of the group is
+ *   compacted in place by that one slot list (each keeps its own K, V, rel, pos rows); len becomes the count.
+ * Slot j must be the same token in every item of a group, so all of them must have the same len — true for a
+ * cache that was only ever appended to and pruned with this call.  A group that breaks this is left untouched
+ * and LETHE_ERR_INVALID_ARG is recorded (with its first item); a budget below the protected count keeps exactly
+ * the protected slots and records LETHE_ERR_BUDGET.
+ * keep_idx (optional) [groups][max_k] int32: old slots of the survivors, ascending, padded with -1 (all -1 for
+ * a refused group).
+ */
+typedef enum { LETHE_COLLAPSE_HEADS = 0, LETHE_COLLAPSE_HEADS_BATCH = 1 } lethe_collapse;
+
+lethe_status lethe_collapsed_prune(lethe_ctx *ctx, const lethe_cache *cache, const int32_t *budgets, int32_t recent,
+                                   int32_t sink, int32_t scope, int32_t *keep_idx, int32_t max_k, void *stream);
 
 /*
  * Relevance of the prompt tokens from the prefill attention (Eq. 2 with Q > 1, folded through Eq. 5), so that

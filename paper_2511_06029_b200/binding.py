@@ -23,7 +23,8 @@ VARIANT_AUTO, VARIANT_SIMT, VARIANT_MMA4, VARIANT_MMA8 = 0, 1, 2, 3
 
 EXPORTS = ["lethe_create", "lethe_destroy", "lethe_last_error", "lethe_poll_status", "lethe_set_tuning",
            "lethe_decode_attend", "lethe_decode_attend_host", "lethe_estimate_sparsity", "lethe_alloc_budgets",
-           "lethe_rasr_prune", "lethe_rasr_prune_static", "lethe_segment_prune", "lethe_prefill_seed"]
+           "lethe_rasr_prune", "lethe_rasr_prune_static", "lethe_segment_prune", "lethe_prefill_seed",
+           "lethe_collapsed_prune"]
 
 
 class LetheError(RuntimeError):
@@ -77,6 +78,8 @@ def load() -> ctypes.CDLL:
     lib.lethe_alloc_budgets.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp, vp, i32, vp, vp]
     lib.lethe_rasr_prune.restype = ctypes.c_int
     lib.lethe_rasr_prune.argtypes = [vp, cp, vp, i32, i32, vp, i32, vp]
+    lib.lethe_collapsed_prune.restype = ctypes.c_int
+    lib.lethe_collapsed_prune.argtypes = [vp, cp, vp, i32, i32, i32, vp, i32, vp]
     lib.lethe_segment_prune.restype = ctypes.c_int
     lib.lethe_segment_prune.argtypes = [vp, cp, i32, ctypes.c_float, i32, i32, vp, vp, i32, vp]
     lib.lethe_prefill_seed.restype = ctypes.c_int
@@ -144,6 +147,9 @@ def rasr_prune_static(cache: "Cache", budgets: torch.Tensor, recent: int, sink: 
         assert status_out.dtype == torch.int32 and status_out.is_cuda and status_out.numel() >= 2
     return int(load().lethe_rasr_prune_static(ctypes.byref(cache.c), _dp(budgets), recent, sink, _dp(keep_idx), max_k,
                                               _dp(status_out), _stream(cache.device)))
+
+
+COLLAPSE_HEADS, COLLAPSE_HEADS_BATCH = 0, 1
 
 
 class Context:
@@ -237,6 +243,17 @@ class Context:
             max_k = keep_idx.shape[-1]
         self._check(self.lib.lethe_segment_prune(self.h, ctypes.byref(cache.c), n_segments, tau, recent, sink,
                                                  _dp(l_evict), _dp(keep_idx), max_k, _stream(self.device)))
+
+    def collapsed_prune(self, cache: Cache, budgets: torch.Tensor, recent: int, sink: int, scope: int,
+                        keep_idx: Optional[torch.Tensor] = None):
+        """scope COLLAPSE_HEADS: budgets [L][B]; COLLAPSE_HEADS_BATCH: budgets [L]; keep_idx [groups][max_k]."""
+        assert budgets.dtype == torch.int32 and budgets.is_cuda and budgets.is_contiguous()
+        max_k = 0
+        if keep_idx is not None:
+            assert keep_idx.dtype == torch.int32 and keep_idx.is_cuda
+            max_k = keep_idx.shape[-1]
+        self._check(self.lib.lethe_collapsed_prune(self.h, ctypes.byref(cache.c), _dp(budgets), recent, sink, scope,
+                                                   _dp(keep_idx), max_k, _stream(self.device)))
 
     def prefill_seed(self, cache: Cache, q_prompt: torch.Tensor, scale, gamma: float):
         """q_prompt [L][B][P][Hq][D] on the device, cache dtype; overwrites rel[0..P) of every item."""

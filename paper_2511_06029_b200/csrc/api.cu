@@ -26,6 +26,9 @@ cudaError_t launch_segment_prune(const CacheView& c, int n_segments, float tau, 
                                  int32_t* keep_idx, int max_k, int smem_tokens, int32_t* list_scratch, int32_t* status,
                                  cudaStream_t stream);
 cudaError_t launch_order(const int32_t* len, int n_items, int cap_tokens, int32_t* order, cudaStream_t stream);
+cudaError_t launch_collapsed_prune(const CacheView& c, const int32_t* budgets, int recent, int sink, int per_group,
+                                   int32_t* keep_idx, int max_k, int smem_tokens, uint32_t* key_scratch,
+                                   int32_t* lists, int32_t* plan, int32_t* status, cudaStream_t stream);
 cudaError_t launch_rasr_prune(const CacheView& c, const int32_t* budgets, int recent, int sink, int32_t* keep_idx,
                               int max_k, int smem_tokens, int32_t* list_scratch, int32_t* status,
                               cudaStream_t stream);
@@ -618,6 +621,39 @@ lethe_status lethe_segment_prune(lethe_ctx* ctx, const lethe_cache* c, int32_t n
     cudaError_t e = launch_segment_prune(v, n_segments, tau, recent, sink, l_evict, keep_idx, keep_idx ? max_k : 0,
                                          smem_tokens, list_scratch, ctx->status, (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "segment_prune launch");
+    return refresh_order(ctx, c, v, stream);
+}
+
+lethe_status lethe_collapsed_prune(lethe_ctx* ctx, const lethe_cache* c, const int32_t* budgets, int32_t recent,
+                                   int32_t sink, int32_t scope, int32_t* keep_idx, int32_t max_k, void* stream) {
+    lethe_status st = check_cache(ctx, c);
+    if (st != LETHE_OK) return st;
+    if (!budgets) return fail(ctx, LETHE_ERR_INVALID_ARG, "budgets is NULL");
+    if (recent < 0 || sink < 0) return fail(ctx, LETHE_ERR_INVALID_ARG, "recent and sink must be >= 0");
+    if (scope != LETHE_COLLAPSE_HEADS && scope != LETHE_COLLAPSE_HEADS_BATCH)
+        return fail(ctx, LETHE_ERR_INVALID_ARG, "scope must be LETHE_COLLAPSE_HEADS or LETHE_COLLAPSE_HEADS_BATCH");
+    if (keep_idx && max_k < 1) return fail(ctx, LETHE_ERR_INVALID_ARG, "max_k must be positive with keep_idx");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, LETHE_ERR_CUDA, "cannot select the context's device");
+    const CacheView v = view_of(c);
+    const int per_group = scope == LETHE_COLLAPSE_HEADS ? v.Hkv : v.B * v.Hkv;
+    const size_t groups = (size_t)v.L * v.B * v.Hkv / per_group;
+    // scratch: plan [groups] (padded to 256 bytes) | lists [groups][cap_tokens] | keys [groups][cap_tokens] if a
+    // group's keys do not fit in shared memory
+    const size_t budget_smem = ctx->max_smem - 8 * 1024;
+    int smem_tokens = v.cap_tokens;
+    const bool spill_keys = (size_t)smem_tokens * 4 > budget_smem;
+    if (spill_keys) smem_tokens = (int)(budget_smem / 4);
+    const size_t plan_bytes = (groups * sizeof(int32_t) + 255) / 256 * 256;
+    const size_t list_bytes = groups * v.cap_tokens * sizeof(int32_t);
+    st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, plan_bytes + list_bytes * (spill_keys ? 2 : 1), "collapsed prune scratch");
+    if (st != LETHE_OK) return st;
+    int32_t* plan = (int32_t*)ctx->scratch;
+    int32_t* lists = (int32_t*)((char*)ctx->scratch + plan_bytes);
+    uint32_t* keys = spill_keys ? (uint32_t*)((char*)ctx->scratch + plan_bytes + list_bytes) : nullptr;
+    cudaError_t e = launch_collapsed_prune(v, budgets, recent, sink, per_group, keep_idx, keep_idx ? max_k : 0, smem_tokens,
+                                           keys, lists, plan, ctx->status, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "collapsed_prune launch");
     return refresh_order(ctx, c, v, stream);
 }
 

@@ -472,6 +472,109 @@ cudaError_t launch_rasr_prune(const CacheView& c, const int32_t* budgets, int re
     return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------ collapsed score (Eq. 2 as printed)
+/*
+ * One score per token per group (scope 0: the Hkv items of a (layer, sequence); scope 1: the B * Hkv items of a
+ * layer) and one retention set shared by the group.  Two launches:
+ *   collapsed_select_kernel  one CTA per group: checks that the group's items have one length, sums rel over the
+ *                            items in ascending item order (fp32, one rounded add each: the sum decides who is
+ *                            kept, so its precision and order are part of the result), radix-selects the
+ *                            threshold, sweeps the survivors' source slots into lists[group] and writes
+ *                            plan[group] = survivors, or -1 when nothing moves;
+ *   collapsed_move_kernel    one CTA per item: compacts the item by its group's list.
+ * Items of a group are consecutive in the [L][B][Hkv] order, so group g owns items [g * per_group, (g+1) * per_group).
+ */
+__global__ void __launch_bounds__(kPruneThreads, 2) collapsed_select_kernel(CacheView c, const int32_t* __restrict__ budgets,
+                                                                         int recent, int sink, int per_group,
+                                                                         int32_t* keep_idx, int max_k, int smem_tokens,
+                                                                         uint32_t* key_scratch, int32_t* lists,
+                                                                         int32_t* plan, int32_t* status) {
+    extern __shared__ __align__(16) uint32_t dyn[];  // keys [smem_tokens]
+    __shared__ PruneShared sh;
+
+    const size_t group = blockIdx.x;
+    const size_t first = group * per_group;
+    const int tid = threadIdx.x;
+    const int n = c.len[first];
+    int32_t* kout = keep_idx ? keep_idx + group * max_k : nullptr;
+
+    int differs = 0;
+    for (int t = 1 + tid; t < per_group; t += kPruneThreads) differs |= (c.len[first + t] != n);
+    if (__syncthreads_or(differs)) {  // slots do not mean the same token in every item: refuse the group
+        if (tid == 0) {
+            record_error(status, LETHE_ERR_INVALID_ARG, (int)first);
+            plan[group] = -1;
+        }
+        if (kout)
+            for (int i = tid; i < max_k; i += kPruneThreads) kout[i] = -1;
+        return;
+    }
+    long long k = budgets[group];
+    if (k < 0) k = 0;
+    if (k >= n) {  // identity
+        if (tid == 0) plan[group] = -1;
+        if (kout)
+            for (int i = tid; i < max_k; i += kPruneThreads) kout[i] = (i < n) ? i : -1;
+        return;
+    }
+    const int n_sink = min(sink, n), n_recent = min(recent, n);
+    const int cand_lo = n_sink;
+    const int cand_hi = max(n - n_recent, cand_lo);
+    const int n_prot = n - (cand_hi - cand_lo);
+    if (n_prot > k) {
+        k = n_prot;
+        if (tid == 0) record_error(status, LETHE_ERR_BUDGET, (int)first);
+    }
+    const int take = (int)k - n_prot;
+
+    const bool in_smem = n <= smem_tokens;
+    uint32_t* keys = in_smem ? dyn : key_scratch + group * c.cap_tokens;
+    const float* rel0 = c.rel + first * c.cap_tokens;
+    for (int j = tid; j < n; j += kPruneThreads) {
+        float s = 0.f;
+        for (int t = 0; t < per_group; ++t) s = __fadd_rn(s, rel0[(size_t)t * c.cap_tokens + j]);
+        keys[j] = score_key(s);
+    }
+    __syncthreads();
+    auto key_at = [&](int j) -> uint32_t { return keys[j]; };
+
+    uint32_t T = 0xffffffffu;
+    int need_eq = 0;
+    if (take > 0) radix_select(sh, key_at, cand_lo, cand_hi, take, T, need_eq);
+    const int keep_n = sweep_keep(sh, key_at, n, cand_lo, cand_hi, cand_lo, cand_hi, take > 0, T, need_eq,
+                                  lists + group * c.cap_tokens, kout, max_k);
+    if (tid == 0) plan[group] = keep_n;
+}
+
+__global__ void __launch_bounds__(kPruneThreads, 2) collapsed_move_kernel(CacheView c, int per_group,
+                                                                       const int32_t* __restrict__ lists,
+                                                                       const int32_t* __restrict__ plan,
+                                                                       int32_t* status) {
+    const size_t item = blockIdx.x;
+    const size_t group = item / per_group;
+    const int keep_n = plan[group];
+    if (keep_n < 0) return;
+    bool bad = false;
+    move_rows(c, item, keep_n, lists + group * c.cap_tokens, bad);
+    if (bad && threadIdx.x == 0) record_error(status, LETHE_ERR_PAGE, (int)item);
+    if (threadIdx.x == 0) c.len[item] = keep_n;
+}
+
+cudaError_t launch_collapsed_prune(const CacheView& c, const int32_t* budgets, int recent, int sink, int per_group,
+                                   int32_t* keep_idx, int max_k, int smem_tokens, uint32_t* key_scratch,
+                                   int32_t* lists, int32_t* plan, int32_t* status, cudaStream_t stream) {
+    const size_t smem = (size_t)smem_tokens * 4;
+    cudaError_t e = prepare_kernel((const void*)collapsed_select_kernel, smem);
+    if (e != cudaSuccess) return e;
+    const int items = c.L * c.B * c.Hkv;
+    collapsed_select_kernel<<<items / per_group, kPruneThreads, smem, stream>>>(
+        c, budgets, recent, sink, per_group, keep_idx, max_k, smem_tokens, key_scratch, lists, plan, status);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    collapsed_move_kernel<<<items, kPruneThreads, 0, stream>>>(c, per_group, lists, plan, status);
+    return cudaGetLastError();
+}
+
 // ------------------------------------------------------------ longest-first item order for the attend queue
 // One CTA: counting sort of the items by len (1024 buckets over [0, cap_tokens]), longest bucket first.  The
 // order only steers the persistent attend kernels' work queue (longest items first shortens the tail of a
