@@ -6,6 +6,7 @@
 #include <new>
 
 #include "common.cuh"
+#include "prefill.cuh"
 
 namespace lethe {
 cudaError_t launch_attend_simt(const AttendArgs& a, int dtype, int D, bool paged, cudaStream_t stream);
@@ -32,25 +33,6 @@ cudaError_t launch_collapsed_prune(const CacheView& c, const int32_t* budgets, i
 cudaError_t launch_rasr_prune(const CacheView& c, const int32_t* budgets, int recent, int sink, int32_t* keep_idx,
                               int max_k, int smem_tokens, int32_t* list_scratch, int32_t* status,
                               cudaStream_t stream);
-}  // namespace lethe
-
-namespace lethe {
-struct PrefillArgs {
-    const void* k;
-    const int32_t* page_table;
-    const int32_t* len;
-    float* rel;
-    const void* q;
-    float2* stats;
-    int32_t* status;
-    long long n_pages;
-    int B, Hq, Hkv, G, HP, P;
-    int capacity, cap_tokens, page_tokens, paged;
-    float gamma_log2;
-    float scale_log2[kMaxLayers];
-};
-size_t prefill_stats_bytes(int items, int P, int HP);
-cudaError_t launch_prefill(const PrefillArgs& a, int items, int D, cudaStream_t stream);
 }  // namespace lethe
 
 using namespace lethe;
@@ -103,6 +85,7 @@ struct lethe_ctx {
     void* staging;  // device staging of lethe_decode_attend_host
     size_t staging_bytes;
     int variant, splits;
+    int prefill_engine;  // 0 = tcgen05 kernels, 1 = mma.sync kernels
     // TMA variant: tensor maps of the last cache seen (rebuilt when k, v, the row count or D change)
     alignas(64) unsigned char tma_maps[512];
     const void* tma_k;
@@ -274,7 +257,11 @@ lethe_status lethe_debug_set_timeline(lethe_ctx* ctx, unsigned long long* buf) {
 
 lethe_status lethe_set_tuning(lethe_ctx* ctx, int variant, int splits) {
     if (!ctx) return LETHE_ERR_INVALID_ARG;
-    if (variant < 0 || variant > 37) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..37");
+    if (variant == 40 || variant == 41) {  // engine of lethe_prefill_seed; the attend tuning is left as it is
+        ctx->prefill_engine = variant == 41 ? 1 : 0;
+        return LETHE_OK;
+    }
+    if (variant < 0 || variant > 37) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..37, 40 or 41");
     const bool flat_variant = variant >= 32;
     if (flat_variant ? (splits < 0 || splits > 16)
                      : !(splits == 0 || splits == 1 || splits == 2 || splits == 4 || splits == 8 || splits == 16))
@@ -690,7 +677,8 @@ lethe_status lethe_prefill_seed(lethe_ctx* ctx, const lethe_cache* c, const void
     st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, prefill_stats_bytes(items, prompt_len, a.HP), "prefill statistics");
     if (st != LETHE_OK) return st;
     a.stats = (float2*)ctx->scratch;
-    cudaError_t e = launch_prefill(a, items, c->head_dim, (cudaStream_t)stream);
+    cudaError_t e = ctx->prefill_engine == 1 ? launch_prefill(a, items, c->head_dim, (cudaStream_t)stream)
+                                             : launch_prefill_tc(a, items, c->head_dim, (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "prefill_seed launch");
     return LETHE_OK;
 }

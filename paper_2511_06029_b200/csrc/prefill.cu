@@ -11,33 +11,12 @@
 // Columns are laid out query-major with the G heads of the group padded to HP = 1, 2, 4 or 8.
 #include "common.cuh"
 #include "mma_utils.cuh"
+#include "prefill.cuh"
 
 namespace lethe {
 
-struct PrefillArgs {
-    const void* k;
-    const int32_t* page_table;
-    const int32_t* len;
-    float* rel;
-    const void* q;   // [L][B][P][Hq][D]
-    float2* stats;   // [items][P][HP]: (max in log2 units, sum)
-    int32_t* status;
-    long long n_pages;
-    int B, Hq, Hkv, G, HP, P;
-    int capacity, cap_tokens, page_tokens, paged;
-    float gamma_log2;
-    float scale_log2[kMaxLayers];
-};
-
 constexpr int kPrefillWarps = 8;
 constexpr int kPrefillKeyTile = 64;  // keys per staged tile in the statistics kernel
-
-__device__ __forceinline__ const char* prefill_row(const PrefillArgs& a, int item, int slot, int row_bytes) {
-    if (!a.paged) return (const char*)a.k + ((size_t)item * a.capacity + slot) * row_bytes;
-    int page = a.page_table[(size_t)item * a.capacity + slot / a.page_tokens];
-    if (page < 0 || page >= a.n_pages) page = 0;  // never read outside the pool (the decode and prune calls report bad ids)
-    return (const char*)a.k + ((size_t)page * a.page_tokens + slot % a.page_tokens) * row_bytes;
-}
 
 // Stage `rows` key rows starting at slot j0 into a swizzled tile (16-byte chunk index XOR (row & 7)); rows at or
 // beyond `limit` are zero-filled.  All threads of the CTA take part.

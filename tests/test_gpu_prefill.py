@@ -17,12 +17,18 @@ def ctx():
     c.close()
 
 
+TCGEN05, MMA_SYNC = 40, 41                                           # lethe_set_tuning codes of the two engines
+
+
+@pytest.mark.parametrize("engine", [TCGEN05, MMA_SYNC])
 @pytest.mark.parametrize("Hq,Hkv,D,P", [(32, 8, 128, 300), (28, 4, 128, 129), (8, 8, 128, 64), (4, 2, 64, 257),
-                                        (6, 2, 128, 17), (5, 1, 64, 1), (16, 2, 128, 200)])
-def test_prefill_seed_parity(ctx, Hq, Hkv, D, P):
+                                        (6, 2, 128, 17), (5, 1, 64, 1), (16, 2, 128, 200), (8, 2, 128, 128),
+                                        (14, 2, 64, 385)])
+def test_prefill_seed_parity(ctx, engine, Hq, Hkv, D, P):
     oracle.set_threads(min(8, oracle.max_threads()))
+    ctx.set_tuning(engine, 0)
     try:
-        L, B, cap = 2, 2, 320
+        L, B, cap = 2, 2, max(320, P + 16)
         lens = torch.full((L, B, Hkv), P, dtype=torch.int32)
         lens[0, 0, 0] = min(cap, P + 7)                               # a longer item: slots beyond P stay as they are
         oc = random_cache(L, B, Hq, Hkv, D, cap, lens, dtype=torch.bfloat16, seed=P, rel_init="rand")
@@ -45,11 +51,14 @@ def test_prefill_seed_parity(ctx, Hq, Hkv, D, P):
         assert torch.allclose(got[..., :P].double().sum(-1), torch.full((L, B, Hkv), want, dtype=torch.float64), rtol=2e-3)
     finally:
         oracle.set_threads(1)
+        ctx.set_tuning(TCGEN05, 0)
 
 
-def test_prefill_seed_paged_then_decode(ctx):
+@pytest.mark.parametrize("engine", [TCGEN05, MMA_SYNC])
+def test_prefill_seed_paged_then_decode(ctx, engine):
     """Paged cache: seed the prompt's relevance, then continue with decode steps; both sides stay in step."""
     oracle.set_threads(min(8, oracle.max_threads()))
+    ctx.set_tuning(engine, 0)
     try:
         w = synth.shrink(synth.WORKLOADS["ragged"], n_layers=2, batch=2, prompt_len=150)
         cap = 192
@@ -75,6 +84,28 @@ def test_prefill_seed_paged_then_decode(ctx):
         assert ctx.poll_status()[0] == 0
     finally:
         oracle.set_threads(1)
+        ctx.set_tuning(TCGEN05, 0)
+
+
+def test_prefill_seed_engines_agree_on_a_long_prompt(ctx):
+    """Prompt of several tiles per operand (P = 1100, G = 7 padded to 8 columns per query): the two engines run the
+    same arithmetic in a different summation order."""
+    L, B, Hq, Hkv, D, P, cap = 1, 2, 14, 2, 128, 1100, 1120
+    oc = random_cache(L, B, Hq, Hkv, D, cap, P, dtype=torch.bfloat16, seed=5, rel_init="rand")
+    qp = torch.randn((L, B, P, Hq, D), generator=torch.Generator().manual_seed(6)).to(torch.bfloat16).cuda()
+    res = {}
+    for engine in (TCGEN05, MMA_SYNC):
+        gc = to_device(oc)
+        ctx.set_tuning(engine, 0)
+        ctx.prefill_seed(gc, qp, [0.11], 0.995)
+        assert ctx.poll_status()[0] == 0
+        res[engine] = gc.rel.cpu()
+    ctx.set_tuning(TCGEN05, 0)
+    assert torch.allclose(res[TCGEN05][..., :P], res[MMA_SYNC][..., :P], rtol=2e-4, atol=1e-7)
+    assert torch.equal(res[TCGEN05][..., P:], oc.rel[..., P:])
+    G = Hq // Hkv
+    want = G * (1 - 0.995 ** P) / (1 - 0.995)
+    assert torch.allclose(res[TCGEN05][..., :P].double().sum(-1), torch.full((L, B, Hkv), want, dtype=torch.float64), rtol=2e-3)
 
 
 def test_prefill_seed_rejects_bad_input(ctx):
