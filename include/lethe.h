@@ -110,8 +110,9 @@ lethe_status lethe_poll_status(lethe_ctx *ctx, void *stream, int32_t *info);
  * 32..37 = the clustered kernel's six shapes with the CTAs of an item merged through global scratch (the last
  * CTA to finish completes the item) instead of a thread-block cluster; splits may then be any value 0..16.
  * Tensor-core variants need a bf16 cache (and 16-token pages when paged).
- * variant 40 / 41 select the engine of lethe_prefill_seed and leave everything else as it is: 40 = tcgen05
- * kernels (accumulators in tensor memory; the default), 41 = mma.sync kernels; splits is ignored.
+ * variant 40..42 select the engine of lethe_prefill_seed and leave everything else as it is: 40 = tcgen05
+ * kernels (accumulators in tensor memory; operand tiles by TMA for contiguous caches, by cp.async for paged
+ * ones; the default), 41 = mma.sync kernels, 42 = tcgen05 kernels with cp.async tiles always; splits is ignored.
  * splits: 0 = automatic, else CTAs per item (1, 2, 4, 8 or 16; they form one thread-block cluster); the
  * persistent variants take 0 or 1.
  * Returns LETHE_ERR_INVALID_ARG for other values.

@@ -85,7 +85,7 @@ struct lethe_ctx {
     void* staging;  // device staging of lethe_decode_attend_host
     size_t staging_bytes;
     int variant, splits;
-    int prefill_engine;  // 0 = tcgen05 kernels, 1 = mma.sync kernels
+    int prefill_engine;  // 0 = tcgen05 kernels (TMA producers when the cache is contiguous), 1 = mma.sync kernels, 2 = tcgen05 with cp.async producers
     // TMA variant: tensor maps of the last cache seen (rebuilt when k, v, the row count or D change)
     alignas(64) unsigned char tma_maps[512];
     const void* tma_k;
@@ -255,13 +255,25 @@ lethe_status lethe_debug_set_timeline(lethe_ctx* ctx, unsigned long long* buf) {
 }
 #endif
 
+// cuTensorMapEncodeTiled through the runtime (no link-time dependency on the driver library); resolved once.
+static bool resolve_tma_encode(lethe_ctx* ctx) {
+    if (ctx->tma_encode) return true;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ctx->tma_encode, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !ctx->tma_encode) {
+        ctx->tma_encode = nullptr;
+        return false;
+    }
+    return true;
+}
+
 lethe_status lethe_set_tuning(lethe_ctx* ctx, int variant, int splits) {
     if (!ctx) return LETHE_ERR_INVALID_ARG;
-    if (variant == 40 || variant == 41) {  // engine of lethe_prefill_seed; the attend tuning is left as it is
-        ctx->prefill_engine = variant == 41 ? 1 : 0;
+    if (variant >= 40 && variant <= 42) {  // engine of lethe_prefill_seed; the attend tuning is left as it is
+        ctx->prefill_engine = variant - 40;
         return LETHE_OK;
     }
-    if (variant < 0 || variant > 37) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..37, 40 or 41");
+    if (variant < 0 || variant > 37) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..37 or 40..42");
     const bool flat_variant = variant >= 32;
     if (flat_variant ? (splits < 0 || splits > 16)
                      : !(splits == 0 || splits == 1 || splits == 2 || splits == 4 || splits == 8 || splits == 16))
@@ -393,14 +405,7 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
                                                   : (unsigned long long)c->n_layers * c->batch * c->n_kv_heads * c->capacity;
             if (rows > 0x7fffffffULL) return fail(ctx, LETHE_ERR_UNSUPPORTED, "cache too large for the TMA variant");
             if (sizeof(ctx->tma_maps) < tma_maps_bytes()) return fail(ctx, LETHE_ERR_CUDA, "tensor map storage");
-            if (!ctx->tma_encode) {
-                cudaDriverEntryPointQueryResult qres;
-                if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ctx->tma_encode, cudaEnableDefault, &qres) != cudaSuccess ||
-                    qres != cudaDriverEntryPointSuccess || !ctx->tma_encode) {
-                    ctx->tma_encode = nullptr;
-                    return fail(ctx, LETHE_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
-                }
-            }
+            if (!resolve_tma_encode(ctx)) return fail(ctx, LETHE_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
             if (ctx->tma_k != c->k || ctx->tma_v != c->v || ctx->tma_rows != rows || ctx->tma_d != c->head_dim) {
                 if (!build_tma_maps(ctx->tma_encode, c->k, c->v, rows, c->head_dim, ctx->tma_maps))
                     return fail(ctx, LETHE_ERR_CUDA, "cuTensorMapEncodeTiled failed");
@@ -674,11 +679,18 @@ lethe_status lethe_prefill_seed(lethe_ctx* ctx, const lethe_cache* c, const void
         a.scale_log2[l] = scale[l] * 1.4426950408889634f;
     }
     const int items = c->n_layers * c->batch * c->n_kv_heads;
-    st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, prefill_stats_bytes(items, prompt_len, a.HP), "prefill statistics");
+    const size_t stats_bytes = ctx->prefill_engine == 1 ? prefill_stats_bytes(items, prompt_len, a.HP)
+                                                        : prefill_tc_stats_bytes(items, prompt_len, a.HP);
+    st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, stats_bytes, "prefill statistics");
     if (st != LETHE_OK) return st;
     a.stats = (float2*)ctx->scratch;
-    cudaError_t e = ctx->prefill_engine == 1 ? launch_prefill(a, items, c->head_dim, (cudaStream_t)stream)
-                                             : launch_prefill_tc(a, items, c->head_dim, (cudaStream_t)stream);
+    cudaError_t e;
+    if (ctx->prefill_engine == 1) {
+        e = launch_prefill(a, items, c->head_dim, (cudaStream_t)stream);
+    } else {
+        const bool allow_tma = ctx->prefill_engine == 0 && resolve_tma_encode(ctx);
+        e = launch_prefill_tc(a, items, c->n_layers, c->head_dim, ctx->tma_encode, allow_tma, (cudaStream_t)stream);
+    }
     if (e != cudaSuccess) return cuda_fail(ctx, e, "prefill_seed launch");
     return LETHE_OK;
 }

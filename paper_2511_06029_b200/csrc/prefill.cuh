@@ -22,8 +22,9 @@ struct PrefillArgs {
 size_t prefill_stats_bytes(int items, int P, int HP);
 // mma.sync kernels (any bf16 cache)
 cudaError_t launch_prefill(const PrefillArgs& a, int items, int D, cudaStream_t stream);
-// tcgen05 kernels (accumulators in tensor memory)
-cudaError_t launch_prefill_tc(const PrefillArgs& a, int items, int D, cudaStream_t stream);
+// tcgen05 kernels (accumulators in tensor memory); their statistics scratch holds two partials per column
+size_t prefill_tc_stats_bytes(int items, int P, int HP);
+cudaError_t launch_prefill_tc(const PrefillArgs& a, int items, int L, int D, void* encode, bool allow_tma, cudaStream_t stream);
 
 __device__ __forceinline__ const char* prefill_row(const PrefillArgs& a, int item, int slot, int row_bytes) {
     if (!a.paged) return (const char*)a.k + ((size_t)item * a.capacity + slot) * row_bytes;

@@ -7,14 +7,26 @@
 //           thread that owns a row keeps that column's online (max, sum) over the keys j <= i in registers;
 //   COLSUM  the rows are 128 keys, the columns 128 (query, head) pairs; the thread that owns a key adds up
 //           exp2(logit - max) * weight / sum over the columns with i >= j.
-// In both, the reduction runs along the TMEM row a thread owns, so no value crosses threads.
+// In both, the reduction runs along the TMEM row a thread owns.  Two warps share a row (TMEM lanes are reachable
+// only from the warps whose index has the same low two bits): each takes 64 of the 128 columns.  STATS writes the
+// two partial (max, sum) pairs side by side and COLSUM merges them when it fetches a column's factor; COLSUM's two
+// partial sums of a key meet in rel[j], zeroed by STATS, through two atomic adds (two addends commute, so the
+// result does not depend on their order).
 //
-// Roles (288 threads): warps 0-3 read TMEM and do the arithmetic (warp w owns TMEM lanes 32 w .. 32 w + 31),
-// warp 4 allocates TMEM and one of its lanes issues the MMAs, warps 5-8 copy operand tiles with cp.async into the
-// 128-byte-swizzled K-major layout the MMA's shared-memory descriptors name.  Hand-offs are mbarriers: loaders ->
-// MMA (a_full, b_full), MMA -> loaders (a_empty, b_empty, by tcgen05.commit), MMA -> softmax (t_full, by
-// tcgen05.commit), softmax -> MMA (t_empty).  Every wait is bounded: when one runs out the CTA sets an abort
-// flag, every role leaves its loop, LETHE_ERR_TIMEOUT is recorded, TMEM is freed and the CTA returns.
+// (query, head) columns are numbered query-major over the G heads of the group: column c of a block that starts
+// at query q0 is (q0 + c / G, c % G); a block holds qpb = 128 / G queries and its last 128 - qpb G columns are
+// unused (zero operand rows, never counted).
+//
+// Roles: warps 0-7 read TMEM and do the arithmetic (warp w owns TMEM lanes 32 (w % 4) .. + 31 and columns
+// 64 (w / 4) .. + 63), warp 8 allocates TMEM and one of its lanes issues the MMAs, and the operand tiles arrive in
+// the 128-byte-swizzled K-major layout the MMA's shared-memory descriptors name either by TMA (one lane of warp 9
+// issues cp.async.bulk.tensor boxes; contiguous caches) or by 16-byte cp.async from warps 9-12 (paged caches).
+// Hand-offs are mbarriers: producer -> MMA (a_full, b_full), MMA -> producer (a_empty, b_empty, by
+// tcgen05.commit), MMA -> softmax (t_full, by tcgen05.commit), softmax -> MMA (t_empty).  Every wait is bounded:
+// when one runs out the CTA sets an abort flag, every role leaves its loop, LETHE_ERR_TIMEOUT is recorded, TMEM is
+// freed and the CTA returns.
+#include <cuda.h>
+
 #include "common.cuh"
 #include "mma_utils.cuh"
 #include "prefill.cuh"
@@ -22,17 +34,26 @@
 namespace lethe {
 namespace {
 
-constexpr int kTcSoftmaxWarps = 4;
-constexpr int kTcLoaderWarps = 4;
+constexpr int kTcSoftmaxWarps = 8;
+constexpr int kTcSoftmaxThreads = kTcSoftmaxWarps * 32;
 constexpr int kTcMmaWarp = kTcSoftmaxWarps;                                   // warp index of the MMA warp
-constexpr int kTcThreads = (kTcSoftmaxWarps + 1 + kTcLoaderWarps) * 32;       // 288
+constexpr int kTcLoaderWarps = 4;                                             // cp.async path only
 constexpr int kTcLoaderThreads = kTcLoaderWarps * 32;
 constexpr int kTcTile = 128;                                                  // rows of either operand: M = N = 128
 constexpr int kTcStages = 3;                                                  // stages of the streamed operand
 constexpr int kTcTmemCols = 2 * kTcTile;                                      // two accumulator buffers
 constexpr int kTcWaitLimit = 400000;
 
+template <bool TMA>
+__host__ __device__ constexpr int tc_threads() { return (kTcSoftmaxWarps + 1 + (TMA ? 1 : kTcLoaderWarps)) * 32; }
+
 enum { kModeStats = 0, kModeColsum = 1 };
+
+// Tensor maps of the TMA path: K as [items][capacity][D] with a 128-row box, the prompt's queries as
+// [L B][P][Hq][D] with a (qpb queries x G heads) box; 64-element (128-byte) inner boxes, 128-byte swizzle.
+struct alignas(64) TcMaps {
+    CUtensorMap k, q;
+};
 
 struct TcShared {
     unsigned long long a_full[2], a_empty[2];
@@ -40,7 +61,8 @@ struct TcShared {
     unsigned long long t_full[2], t_empty[2];
     uint32_t tmem_base;
     int abort;
-    float2 cf[kTcSoftmaxWarps][2][kTcTile];  // COLSUM: (max, weight / sum) of the columns of the tiles in flight, one copy per warp
+    // COLSUM: (-max, weight / sum) of the 64 columns a warp reads, of the tiles in flight; one copy per warp
+    alignas(16) float2 cf[kTcSoftmaxWarps][2][kTcTile / 2];
 };
 
 __device__ __forceinline__ void tc_mbar_init(unsigned long long* bar, int count) {
@@ -48,6 +70,10 @@ __device__ __forceinline__ void tc_mbar_init(unsigned long long* bar, int count)
 }
 __device__ __forceinline__ void tc_mbar_arrive(unsigned long long* bar) {
     asm volatile("{ .reg .b64 st; mbarrier.arrive.shared::cta.b64 st, [%0]; }" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_mbar_expect_tx(unsigned long long* bar, unsigned bytes) {
+    asm volatile("{ .reg .b64 st; mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
 }
 __device__ __forceinline__ bool tc_mbar_try_wait(unsigned long long* bar, unsigned parity) {
     unsigned ok;
@@ -71,6 +97,21 @@ __device__ __forceinline__ bool tc_wait(unsigned long long* bar, unsigned parity
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// One box of a tensor map into shared memory; completion is counted in bytes on `bar`.  x is 0 or 64 elements (a
+// multiple of 16 bytes); the other coordinates have no alignment rule.
+__device__ __forceinline__ void tc_tma_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, unsigned long long* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ void tc_tma_4d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w, unsigned long long* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(smem_u32(bar))
+        : "memory");
+}
 
 // Shared-memory matrix descriptor of a K-major bf16 operand tile stored as rows of 128 bytes (64 elements) with the
 // 128-byte swizzle (16-byte chunk index XOR (row & 7)); groups of eight rows are 1024 bytes apart.
@@ -126,7 +167,7 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
 }
 
 // Which tiles of the streamed operand meet A block `a`.
-//   STATS : A = query block a (qpb queries x HP heads = 128 rows); streamed = key tiles 0 .. (last query of a) / 128
+//   STATS : A = query block a (qpb queries x G heads); streamed = key tiles 0 .. (last query of a) / 128
 //   COLSUM: A = key tile a; streamed = query blocks from the one holding key 128 a to the last
 template <int MODE>
 __device__ __forceinline__ void tc_range(int a, int P, int qpb, int& begin, int& end) {
@@ -139,28 +180,28 @@ __device__ __forceinline__ void tc_range(int a, int P, int qpb, int& begin, int&
     }
 }
 
-template <int D>
 __device__ __forceinline__ uint32_t tc_chunk_addr(uint32_t tile, int r, int c) {
     // 16-byte chunk c of row r: halves of 64 elements are separate 128-row regions
     return tile + (c >> 3) * (kTcTile * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4);
 }
 
-// 128 (query, head) columns starting at query qf, as K-major rows; columns of missing queries / padded heads are zero.
+// cp.async path: the (query, head) columns of the block starting at query qf, as K-major rows; rows of missing
+// queries and the unused tail are zero.
 template <int D>
-__device__ __forceinline__ void tc_load_queries(const PrefillArgs& a, int l, int b, int hkv, int qf, uint32_t tile, int ltid) {
+__device__ __forceinline__ void tc_load_queries(const PrefillArgs& a, int l, int b, int hkv, int qf, int used, uint32_t tile, int ltid) {
     constexpr int CH = D * 2 / 16;
 #pragma unroll 4
     for (int idx = ltid; idx < kTcTile * CH; idx += kTcLoaderThreads) {
         const int r = idx / CH, c = idx % CH;
-        const int qi = qf + r / a.HP, h = r % a.HP;
-        const bool ok = qi < a.P && h < a.G;
+        const int qi = qf + r / a.G, h = r % a.G;
+        const bool ok = r < used && qi < a.P;
         const char* src = (const char*)a.q +
                           ((((size_t)l * a.B + b) * a.P + (ok ? qi : 0)) * a.Hq + hkv * a.G + (ok ? h : 0)) * (D * 2) + c * 16;
-        cp_async16(tc_chunk_addr<D>(tile, r, c), src, ok ? 16 : 0);
+        cp_async16(tc_chunk_addr(tile, r, c), src, ok ? 16 : 0);
     }
 }
 
-// 128 keys starting at slot j0; rows at or beyond the prompt are zero.
+// cp.async path: 128 keys starting at slot j0; rows at or beyond the prompt are zero.
 template <int D>
 __device__ __forceinline__ void tc_load_keys(const PrefillArgs& a, int item, int j0, uint32_t tile, int ltid) {
     constexpr int CH = D * 2 / 16;
@@ -170,13 +211,15 @@ __device__ __forceinline__ void tc_load_keys(const PrefillArgs& a, int item, int
         const int j = j0 + r;
         const bool ok = j < a.P;
         const char* src = prefill_row(a, item, ok ? j : 0, D * 2) + c * 16;
-        cp_async16(tc_chunk_addr<D>(tile, r, c), src, ok ? 16 : 0);
+        cp_async16(tc_chunk_addr(tile, r, c), src, ok ? 16 : 0);
     }
 }
 
-template <int D, int MODE>
-__global__ void __launch_bounds__(kTcThreads, 1) prefill_tc_kernel(const __grid_constant__ PrefillArgs a) {
+template <int D, int MODE, bool TMA>
+__global__ void __launch_bounds__(tc_threads<TMA>(), 1)
+    prefill_tc_kernel(const __grid_constant__ PrefillArgs a, const __grid_constant__ TcMaps maps) {
     constexpr int TILE_BYTES = kTcTile * D * 2;
+    constexpr int HALF_BYTES = kTcTile * 128;  // one 64-element half of a tile
     constexpr int KS = D / 16;
     extern __shared__ unsigned char dyn_raw[];
     __shared__ TcShared sh;
@@ -184,30 +227,48 @@ __global__ void __launch_bounds__(kTcThreads, 1) prefill_tc_kernel(const __grid_
     const int item = blockIdx.x;
     const int hkv = item % a.Hkv, b = (item / a.Hkv) % a.B, l = item / (a.Hkv * a.B);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int P = a.P, HP = a.HP, qpb = kTcTile / HP;
+    const int P = a.P, G = a.G, HP = a.HP, qpb = kTcTile / G, used = qpb * G;
     if (a.len[item] < P) {  // the prompt's keys are not all there: skip the item (uniform for the CTA)
         if (MODE == kModeStats && tid == 0) record_error(a.status, LETHE_ERR_CAPACITY, item);
         return;
     }
     // operand tiles: 1024-byte aligned (the swizzle pattern is anchored at 1024-byte boundaries)
     const uint32_t dyn = (smem_u32(dyn_raw) + 1023u) & ~1023u;
-    const uint32_t a_tile[2] = {dyn, dyn + TILE_BYTES};
+    const uint32_t a_tile0 = dyn;
     const uint32_t b_tile0 = dyn + 2 * TILE_BYTES;
     volatile int* abort_flag = &sh.abort;
 
     if (tid == 0) {
+        const int producers = TMA ? 1 : kTcLoaderThreads;
         for (int i = 0; i < 2; ++i) {
-            tc_mbar_init(&sh.a_full[i], kTcLoaderThreads);
+            tc_mbar_init(&sh.a_full[i], producers);
             tc_mbar_init(&sh.a_empty[i], 1);
             tc_mbar_init(&sh.t_full[i], 1);
-            tc_mbar_init(&sh.t_empty[i], kTcSoftmaxWarps * 32);
+            tc_mbar_init(&sh.t_empty[i], kTcSoftmaxThreads);
         }
         for (int i = 0; i < kTcStages; ++i) {
-            tc_mbar_init(&sh.b_full[i], kTcLoaderThreads);
+            tc_mbar_init(&sh.b_full[i], producers);
             tc_mbar_init(&sh.b_empty[i], 1);
         }
         sh.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (TMA && used < kTcTile) {
+        // rows the query boxes never write: zero them once (in every buffer that will hold queries)
+        const uint32_t first = MODE == kModeStats ? a_tile0 : b_tile0;
+        const int n_buf = MODE == kModeStats ? 2 : kTcStages;
+        const int tail_chunks = (kTcTile - used) * 8;  // 16-byte chunks per 64-element half
+        for (int idx = tid; idx < n_buf * (D / 64) * tail_chunks; idx += tc_threads<TMA>()) {
+            const int c = idx % tail_chunks, hb = idx / tail_chunks;  // hb = buffer * halves + half
+            const uint32_t addr = first + (hb / (D / 64)) * TILE_BYTES + (hb % (D / 64)) * HALF_BYTES + used * 128 + c * 16;
+            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0) : "memory");
+        }
+        tc_fence_proxy_async();
+    }
+    if (MODE == kModeStats && warp < kTcSoftmaxWarps) {
+        // COLSUM adds its two partial sums of every key into rel: start them at zero
+        float* rel = a.rel + (size_t)item * a.cap_tokens;
+        for (int j = tid; j < P; j += kTcSoftmaxThreads) rel[j] = 0.f;
     }
     if (warp == kTcMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)),
@@ -223,39 +284,76 @@ __global__ void __launch_bounds__(kTcThreads, 1) prefill_tc_kernel(const __grid_
     const int nA = MODE == kModeStats ? (P + qpb - 1) / qpb : (P + kTcTile - 1) / kTcTile;
 
     if (warp > kTcMmaWarp) {
-        // ------------------------------------------------------------------ loaders
-        const int ltid = tid - (kTcMmaWarp + 1) * 32;
-        int step = 0, prev_stage = -1, prev_a = -1;
-        bool prev_first = false, alive = true;
-        for (int ab = 0; ab < nA && alive; ++ab) {
-            int t0, t1;
-            tc_range<MODE>(ab, P, qpb, t0, t1);
-            for (int t = t0; t < t1; ++t, ++step) {
-                const int s = step % kTcStages;
-                const bool first = t == t0;
-                if (first) {
-                    if (ab >= 2 && !tc_wait(&sh.a_empty[ab & 1], (unsigned)(((ab >> 1) - 1) & 1), abort_flag)) { alive = false; break; }
-                    if (MODE == kModeStats) tc_load_queries<D>(a, l, b, hkv, ab * qpb, a_tile[ab & 1], ltid);
-                    else tc_load_keys<D>(a, item, ab * kTcTile, a_tile[ab & 1], ltid);
+        // ------------------------------------------------------------------ producers
+        if (TMA) {
+            if (warp == kTcMmaWarp + 1 && lane == 0) {
+                const unsigned q_bytes = (unsigned)used * D * 2, k_bytes = TILE_BYTES;
+                auto load_queries = [&](int q0, uint32_t tile, unsigned long long* bar) {
+#pragma unroll
+                    for (int hf = 0; hf < D / 64; ++hf) tc_tma_4d(tile + hf * HALF_BYTES, &maps.q, 64 * hf, hkv * G, q0, l * a.B + b, bar);
+                };
+                auto load_keys = [&](int j0, uint32_t tile, unsigned long long* bar) {
+#pragma unroll
+                    for (int hf = 0; hf < D / 64; ++hf) tc_tma_3d(tile + hf * HALF_BYTES, &maps.k, 64 * hf, j0, item, bar);
+                };
+                int step = 0;
+                bool alive = true;
+                for (int ab = 0; ab < nA && alive; ++ab) {
+                    int t0, t1;
+                    tc_range<MODE>(ab, P, qpb, t0, t1);
+                    for (int t = t0; t < t1; ++t, ++step) {
+                        const int s = step % kTcStages;
+                        if (t == t0) {
+                            if (ab >= 2 && !tc_wait(&sh.a_empty[ab & 1], (unsigned)(((ab >> 1) - 1) & 1), abort_flag)) { alive = false; break; }
+                            const uint32_t at = a_tile0 + (ab & 1) * TILE_BYTES;
+                            tc_mbar_expect_tx(&sh.a_full[ab & 1], MODE == kModeStats ? q_bytes : k_bytes);
+                            if (MODE == kModeStats) load_queries(ab * qpb, at, &sh.a_full[ab & 1]);
+                            else load_keys(ab * kTcTile, at, &sh.a_full[ab & 1]);
+                        }
+                        if (step >= kTcStages && !tc_wait(&sh.b_empty[s], (unsigned)(((step / kTcStages) - 1) & 1), abort_flag)) { alive = false; break; }
+                        const uint32_t bt = b_tile0 + s * TILE_BYTES;
+                        tc_mbar_expect_tx(&sh.b_full[s], MODE == kModeStats ? k_bytes : q_bytes);
+                        if (MODE == kModeStats) load_keys(t * kTcTile, bt, &sh.b_full[s]);
+                        else load_queries(t * qpb, bt, &sh.b_full[s]);
+                    }
                 }
-                if (step >= kTcStages && !tc_wait(&sh.b_empty[s], (unsigned)(((step / kTcStages) - 1) & 1), abort_flag)) { alive = false; break; }
-                if (MODE == kModeStats) tc_load_keys<D>(a, item, t * kTcTile, b_tile0 + s * TILE_BYTES, ltid);
-                else tc_load_queries<D>(a, l, b, hkv, t * qpb, b_tile0 + s * TILE_BYTES, ltid);
-                cp_async_commit();
-                if (prev_stage >= 0) {  // the previous step's copies have landed: publish them to the MMA's proxy
-                    cp_async_wait<1>();
-                    tc_fence_proxy_async();
-                    if (prev_first) tc_mbar_arrive(&sh.a_full[prev_a & 1]);
-                    tc_mbar_arrive(&sh.b_full[prev_stage]);
-                }
-                prev_stage = s; prev_a = ab; prev_first = first;
             }
-        }
-        cp_async_wait<0>();
-        if (alive && prev_stage >= 0) {
-            tc_fence_proxy_async();
-            if (prev_first) tc_mbar_arrive(&sh.a_full[prev_a & 1]);
-            tc_mbar_arrive(&sh.b_full[prev_stage]);
+            __syncwarp();
+        } else {
+            const int ltid = tid - (kTcMmaWarp + 1) * 32;
+            int step = 0, prev_stage = -1, prev_a = -1;
+            bool prev_first = false, alive = true;
+            for (int ab = 0; ab < nA && alive; ++ab) {
+                int t0, t1;
+                tc_range<MODE>(ab, P, qpb, t0, t1);
+                for (int t = t0; t < t1; ++t, ++step) {
+                    const int s = step % kTcStages;
+                    const bool first = t == t0;
+                    if (first) {
+                        if (ab >= 2 && !tc_wait(&sh.a_empty[ab & 1], (unsigned)(((ab >> 1) - 1) & 1), abort_flag)) { alive = false; break; }
+                        const uint32_t at = a_tile0 + (ab & 1) * TILE_BYTES;
+                        if (MODE == kModeStats) tc_load_queries<D>(a, l, b, hkv, ab * qpb, used, at, ltid);
+                        else tc_load_keys<D>(a, item, ab * kTcTile, at, ltid);
+                    }
+                    if (step >= kTcStages && !tc_wait(&sh.b_empty[s], (unsigned)(((step / kTcStages) - 1) & 1), abort_flag)) { alive = false; break; }
+                    if (MODE == kModeStats) tc_load_keys<D>(a, item, t * kTcTile, b_tile0 + s * TILE_BYTES, ltid);
+                    else tc_load_queries<D>(a, l, b, hkv, t * qpb, used, b_tile0 + s * TILE_BYTES, ltid);
+                    cp_async_commit();
+                    if (prev_stage >= 0) {  // the previous step's copies have landed: publish them to the MMA's proxy
+                        cp_async_wait<1>();
+                        tc_fence_proxy_async();
+                        if (prev_first) tc_mbar_arrive(&sh.a_full[prev_a & 1]);
+                        tc_mbar_arrive(&sh.b_full[prev_stage]);
+                    }
+                    prev_stage = s; prev_a = ab; prev_first = first;
+                }
+            }
+            cp_async_wait<0>();
+            if (alive && prev_stage >= 0) {
+                tc_fence_proxy_async();
+                if (prev_first) tc_mbar_arrive(&sh.a_full[prev_a & 1]);
+                tc_mbar_arrive(&sh.b_full[prev_stage]);
+            }
         }
     } else if (warp == kTcMmaWarp) {
         // ------------------------------------------------------------------ MMA issue (one lane)
@@ -272,11 +370,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) prefill_tc_kernel(const __grid_
                     if (!tc_wait(&sh.b_full[s], (unsigned)((step / kTcStages) & 1), abort_flag)) { alive = false; break; }
                     if (step >= 2 && !tc_wait(&sh.t_empty[buf], (unsigned)(((step >> 1) - 1) & 1), abort_flag)) { alive = false; break; }
                     tc_fence_after();
-                    const uint32_t at = a_tile[ab & 1], bt = b_tile0 + s * TILE_BYTES;
+                    const uint32_t at = a_tile0 + (ab & 1) * TILE_BYTES, bt = b_tile0 + s * TILE_BYTES;
 #pragma unroll
                     for (int ks = 0; ks < KS; ++ks) {
                         // 16 elements of K per MMA: 32 bytes along the swizzled row; the second 64 elements are the next region
-                        const uint32_t off = (ks >> 2) * (kTcTile * 128) + (ks & 3) * 32;
+                        const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
                         tc_mma(tmem + buf * kTcTile, tc_smem_desc(at + off), tc_smem_desc(bt + off), idesc, ks > 0 ? 1u : 0u);
                     }
                     tc_commit(&sh.b_empty[s]);
@@ -288,54 +386,76 @@ __global__ void __launch_bounds__(kTcThreads, 1) prefill_tc_kernel(const __grid_
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ softmax warps
-        const int r = tid;  // TMEM lane = tile row
+        const int quarter = warp & 3, half = warp >> 2;
+        const int r = quarter * 32 + lane;  // TMEM lane = tile row
         const float sl2 = a.scale_log2[l];
-        const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
+        const uint32_t t_lane = tmem + ((uint32_t)(quarter * 32) << 16) + half * 64;
+        const size_t half_stride = (size_t)gridDim.x * P * HP;  // STATS partials of the upper 64 key columns come second
         int step = 0;
         bool alive = true;
-        // COLSUM: every warp keeps its own copy of the tile's 128 column factors (lane x fetches columns x, x + 32,
-        // x + 64, x + 96 one step ahead), so the softmax warps never wait for one another
+        // COLSUM: every warp keeps its own copy of the factors of the 64 columns it reads (lane x fetches columns
+        // x and x + 32 of its half one step ahead), so the softmax warps never wait for one another
         auto column_factor = [&](int u, int col) -> float2 {
-            const int qc = u * qpb + col / HP, h = col % HP;
+            const int qc = u * qpb + col / G, h = col % G;
             float2 f = make_float2(0.f, 0.f);
-            if (qc < P && h < a.G) {
-                const float2 st = a.stats[((size_t)item * P + qc) * HP + h];
+            if (col < used && qc < P) {
+                const size_t at = ((size_t)item * P + qc) * HP + h;
+                const float2 s0 = a.stats[at], s1 = a.stats[half_stride + at];  // (max, sum) over keys 0-63 / 64-127 of every tile
+                const float mx = fmaxf(s0.x, s1.x);
+                const float sum = s0.y * exp2_diff(s0.x, mx) + s1.y * exp2_diff(s1.x, mx);
                 const float wgt = fast_exp2((float)(P - 1 - qc) * a.gamma_log2);
-                f = make_float2(st.x, st.y > 0.f ? wgt / st.y : 0.f);
+                f = make_float2(-mx, sum > 0.f ? wgt / sum : 0.f);
             }
             return f;
         };
         for (int ab = 0; ab < nA && alive; ++ab) {
             int t0, t1;
             tc_range<MODE>(ab, P, qpb, t0, t1);
-            // STATS state of this thread's column; COLSUM accumulators of this thread's key
-            const int qi = ab * qpb + r / HP;
-            const bool row_ok = MODE == kModeStats ? (qi < P && (r % HP) < a.G) : (ab * kTcTile + r < P);
+            // STATS: state of this thread's column over its half of every key tile; COLSUM: partial sum of its key
+            const int qi = ab * qpb + r / G;
+            const bool row_ok = MODE == kModeStats ? (r < used && qi < P) : (ab * kTcTile + r < P);
             float m = -INFINITY, lsum = 0.f;
             float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
-            float2 f_next[4];
+            float2 f_next[2];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) f_next[k] = MODE == kModeColsum ? column_factor(t0, lane + 32 * k) : make_float2(0.f, 0.f);
+            for (int k = 0; k < 2; ++k)
+                f_next[k] = MODE == kModeColsum ? column_factor(t0, half * 64 + lane + 32 * k) : make_float2(0.f, 0.f);
             for (int t = t0; t < t1; ++t, ++step) {
                 const int buf = step & 1;
                 if (MODE == kModeColsum) {
                     __syncwarp();
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
+                    for (int k = 0; k < 2; ++k) {
                         sh.cf[warp][buf][lane + 32 * k] = f_next[k];
-                        if (t + 1 < t1) f_next[k] = column_factor(t + 1, lane + 32 * k);
+                        if (t + 1 < t1) f_next[k] = column_factor(t + 1, half * 64 + lane + 32 * k);
                     }
                     __syncwarp();
                 }
                 if (!tc_wait(&sh.t_full[buf], (unsigned)((step >> 1) & 1), abort_flag)) { alive = false; break; }
                 tc_fence_after();
 #pragma unroll 1
-                for (int ch = 0; ch < kTcTile / 32; ++ch) {
+                for (int ch = 0; ch < 2; ++ch) {
                     uint32_t v[32];
                     tc_ld32(t_lane + buf * kTcTile + ch * 32, v);
+                    const int cbase = half * 64 + ch * 32;  // first tile column of this chunk
                     if (MODE == kModeStats) {
-                        const int nv = qi - (t * kTcTile + ch * 32) + 1;  // keys of this chunk that query qi sees
-                        if (row_ok && nv > 0) {
+                        const int nv = qi - (t * kTcTile + cbase) + 1;  // keys of this chunk that query qi sees
+                        if (row_ok && nv >= 32 && sl2 >= 0.f) {
+                            float rm = __uint_as_float(v[0]);
+#pragma unroll
+                            for (int c = 1; c < 32; ++c) rm = fmaxf(rm, __uint_as_float(v[c]));
+                            const float mx = fmaxf(m, rm * sl2), nmx = -mx;
+                            float l0 = lsum * exp2_diff(m, mx), l1 = 0.f, l2 = 0.f, l3 = 0.f;
+#pragma unroll
+                            for (int c = 0; c < 32; c += 4) {
+                                l0 += fast_exp2(fmaf(__uint_as_float(v[c]), sl2, nmx));
+                                l1 += fast_exp2(fmaf(__uint_as_float(v[c + 1]), sl2, nmx));
+                                l2 += fast_exp2(fmaf(__uint_as_float(v[c + 2]), sl2, nmx));
+                                l3 += fast_exp2(fmaf(__uint_as_float(v[c + 3]), sl2, nmx));
+                            }
+                            lsum = (l0 + l1) + (l2 + l3);
+                            m = mx;
+                        } else if (row_ok && nv > 0) {
                             float mx = m;
 #pragma unroll
                             for (int c = 0; c < 32; ++c) {
@@ -343,29 +463,35 @@ __global__ void __launch_bounds__(kTcThreads, 1) prefill_tc_kernel(const __grid_
                                 v[c] = __float_as_uint(x);
                                 if (c < nv) mx = fmaxf(mx, x);
                             }
-                            float l0 = lsum * exp2_diff(m, mx), l1 = 0.f, l2 = 0.f, l3 = 0.f;
+                            float l0 = lsum * exp2_diff(m, mx), l1 = 0.f;
 #pragma unroll
-                            for (int c = 0; c < 32; c += 4) {
+                            for (int c = 0; c < 32; c += 2) {
                                 if (c < nv) l0 += fast_exp2(__uint_as_float(v[c]) - mx);
                                 if (c + 1 < nv) l1 += fast_exp2(__uint_as_float(v[c + 1]) - mx);
-                                if (c + 2 < nv) l2 += fast_exp2(__uint_as_float(v[c + 2]) - mx);
-                                if (c + 3 < nv) l3 += fast_exp2(__uint_as_float(v[c + 3]) - mx);
                             }
-                            lsum = (l0 + l1) + (l2 + l3);
+                            lsum = l0 + l1;
                             m = mx;
                         }
                     } else {
-                        // column cc = (query t * qpb + cc / HP, head cc % HP) counts for key j when query >= j
-                        const int c_start = (ab * kTcTile + r - t * qpb) * HP - ch * 32;  // first counted column of this chunk
-                        if (row_ok && c_start < 32) {
-                            const float2* cf = sh.cf[warp][buf] + ch * 32;
+                        // tile column cc = (query t qpb + cc / G, head cc % G) counts for key j when its query >= j
+                        const int c_lo = (ab * kTcTile + r - t * qpb) * G - cbase;  // first counted column of this chunk
+                        const int c_hi = used - cbase;                             // columns beyond are unused
+                        const float4* cf4 = reinterpret_cast<const float4*>(sh.cf[warp][buf] + ch * 32);
+                        if (row_ok && c_lo <= 0 && c_hi >= 32) {
 #pragma unroll
                             for (int c = 0; c < 32; c += 4) {
-                                const float2 f0 = cf[c], f1 = cf[c + 1], f2 = cf[c + 2], f3 = cf[c + 3];
-                                if (c >= c_start) acc0 += fast_exp2(__uint_as_float(v[c]) * sl2 - f0.x) * f0.y;
-                                if (c + 1 >= c_start) acc1 += fast_exp2(__uint_as_float(v[c + 1]) * sl2 - f1.x) * f1.y;
-                                if (c + 2 >= c_start) acc2 += fast_exp2(__uint_as_float(v[c + 2]) * sl2 - f2.x) * f2.y;
-                                if (c + 3 >= c_start) acc3 += fast_exp2(__uint_as_float(v[c + 3]) * sl2 - f3.x) * f3.y;
+                                const float4 fa = cf4[c / 2], fb = cf4[c / 2 + 1];  // (-max, w) of columns c, c+1 | c+2, c+3
+                                acc0 = fmaf(fast_exp2(fmaf(__uint_as_float(v[c]), sl2, fa.x)), fa.y, acc0);
+                                acc1 = fmaf(fast_exp2(fmaf(__uint_as_float(v[c + 1]), sl2, fa.z)), fa.w, acc1);
+                                acc2 = fmaf(fast_exp2(fmaf(__uint_as_float(v[c + 2]), sl2, fb.x)), fb.y, acc2);
+                                acc3 = fmaf(fast_exp2(fmaf(__uint_as_float(v[c + 3]), sl2, fb.z)), fb.w, acc3);
+                            }
+                        } else if (row_ok && c_lo < 32 && c_hi > 0) {
+#pragma unroll
+                            for (int c = 0; c < 32; c += 2) {
+                                const float4 fa = cf4[c / 2];
+                                if (c >= c_lo && c < c_hi) acc0 = fmaf(fast_exp2(fmaf(__uint_as_float(v[c]), sl2, fa.x)), fa.y, acc0);
+                                if (c + 1 >= c_lo && c + 1 < c_hi) acc1 = fmaf(fast_exp2(fmaf(__uint_as_float(v[c + 1]), sl2, fa.z)), fa.w, acc1);
                             }
                         }
                     }
@@ -374,8 +500,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) prefill_tc_kernel(const __grid_
                 tc_mbar_arrive(&sh.t_empty[buf]);
             }
             if (alive && row_ok) {
-                if (MODE == kModeStats) a.stats[((size_t)item * P + qi) * HP + r % HP] = make_float2(m, lsum);
-                else a.rel[(size_t)item * a.cap_tokens + ab * kTcTile + r] = (acc0 + acc1) + (acc2 + acc3);
+                if (MODE == kModeStats) a.stats[half * half_stride + ((size_t)item * P + qi) * HP + r % G] = make_float2(m, lsum);
+                else atomicAdd(a.rel + (size_t)item * a.cap_tokens + ab * kTcTile + r, (acc0 + acc1) + (acc2 + acc3));
             }
         }
     }
@@ -388,22 +514,52 @@ __global__ void __launch_bounds__(kTcThreads, 1) prefill_tc_kernel(const __grid_
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTcTmemCols) : "memory");
 }
 
-template <int D>
-cudaError_t launch_tc(const PrefillArgs& a, int items, cudaStream_t stream) {
+template <int D, bool TMA>
+cudaError_t launch_tc(const PrefillArgs& a, const TcMaps& maps, int items, cudaStream_t stream) {
     const size_t smem = 1024 + (size_t)(2 + kTcStages) * kTcTile * D * 2;
-    cudaError_t e = prepare_kernel((const void*)prefill_tc_kernel<D, kModeStats>, smem);
+    cudaError_t e = prepare_kernel((const void*)prefill_tc_kernel<D, kModeStats, TMA>, smem);
     if (e != cudaSuccess) return e;
-    e = prepare_kernel((const void*)prefill_tc_kernel<D, kModeColsum>, smem);
+    e = prepare_kernel((const void*)prefill_tc_kernel<D, kModeColsum, TMA>, smem);
     if (e != cudaSuccess) return e;
-    prefill_tc_kernel<D, kModeStats><<<items, kTcThreads, smem, stream>>>(a);
-    prefill_tc_kernel<D, kModeColsum><<<items, kTcThreads, smem, stream>>>(a);
+    prefill_tc_kernel<D, kModeStats, TMA><<<items, tc_threads<TMA>(), smem, stream>>>(a, maps);
+    prefill_tc_kernel<D, kModeColsum, TMA><<<items, tc_threads<TMA>(), smem, stream>>>(a, maps);
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_prefill_tc(const PrefillArgs& a, int items, int D, cudaStream_t stream) {
-    return D == 128 ? launch_tc<128>(a, items, stream) : launch_tc<64>(a, items, stream);
+// Two (max, sum) partials per (query, head) column.
+size_t prefill_tc_stats_bytes(int items, int P, int HP) { return 2 * (size_t)items * P * HP * sizeof(float2); }
+
+// encode: cuTensorMapEncodeTiled resolved by the caller, or NULL; the TMA path is taken for contiguous caches when
+// it is there and `allow_tma` is set, the cp.async path otherwise.
+cudaError_t launch_prefill_tc(const PrefillArgs& a, int items, int L, int D, void* encode, bool allow_tma, cudaStream_t stream) {
+    TcMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    bool tma = false;
+    if (encode && allow_tma && !a.paged) {
+        typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                      const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+        encode_fn fn = reinterpret_cast<encode_fn>(encode);
+        const cuuint32_t qpb = (cuuint32_t)(kTcTile / a.G);
+        const cuuint64_t kd[3] = {(cuuint64_t)D, (cuuint64_t)a.capacity, (cuuint64_t)items};
+        const cuuint64_t ks[2] = {(cuuint64_t)D * 2, (cuuint64_t)a.capacity * D * 2};
+        const cuuint32_t kb[3] = {64, (cuuint32_t)kTcTile, 1};
+        const cuuint64_t qd[4] = {(cuuint64_t)D, (cuuint64_t)a.Hq, (cuuint64_t)a.P, (cuuint64_t)L * a.B};
+        const cuuint64_t qs[3] = {(cuuint64_t)D * 2, (cuuint64_t)a.Hq * D * 2, (cuuint64_t)a.P * a.Hq * D * 2};
+        const cuuint32_t qb[4] = {64, (cuuint32_t)a.G, qpb, 1};
+        const cuuint32_t es[4] = {1, 1, 1, 1};
+        const CUresult r1 = fn(&maps.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(a.k), kd, ks, kb, es,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        const CUresult r2 = fn(&maps.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(a.q), qd, qs, qb, es,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        tma = r1 == CUDA_SUCCESS && r2 == CUDA_SUCCESS;
+    }
+    if (tma) return D == 128 ? launch_tc<128, true>(a, maps, items, stream) : launch_tc<64, true>(a, maps, items, stream);
+    return D == 128 ? launch_tc<128, false>(a, maps, items, stream) : launch_tc<64, false>(a, maps, items, stream);
 }
 
 }  // namespace lethe

@@ -17,10 +17,10 @@ def ctx():
     c.close()
 
 
-TCGEN05, MMA_SYNC = 40, 41                                           # lethe_set_tuning codes of the two engines
+TCGEN05, MMA_SYNC, TCGEN05_CP_ASYNC = 40, 41, 42                     # lethe_set_tuning codes of the engines
 
 
-@pytest.mark.parametrize("engine", [TCGEN05, MMA_SYNC])
+@pytest.mark.parametrize("engine", [TCGEN05, MMA_SYNC, TCGEN05_CP_ASYNC])
 @pytest.mark.parametrize("Hq,Hkv,D,P", [(32, 8, 128, 300), (28, 4, 128, 129), (8, 8, 128, 64), (4, 2, 64, 257),
                                         (6, 2, 128, 17), (5, 1, 64, 1), (16, 2, 128, 200), (8, 2, 128, 128),
                                         (14, 2, 64, 385)])
@@ -94,7 +94,7 @@ def test_prefill_seed_engines_agree_on_a_long_prompt(ctx):
     oc = random_cache(L, B, Hq, Hkv, D, cap, P, dtype=torch.bfloat16, seed=5, rel_init="rand")
     qp = torch.randn((L, B, P, Hq, D), generator=torch.Generator().manual_seed(6)).to(torch.bfloat16).cuda()
     res = {}
-    for engine in (TCGEN05, MMA_SYNC):
+    for engine in (TCGEN05, MMA_SYNC, TCGEN05_CP_ASYNC):
         gc = to_device(oc)
         ctx.set_tuning(engine, 0)
         ctx.prefill_seed(gc, qp, [0.11], 0.995)
@@ -102,6 +102,7 @@ def test_prefill_seed_engines_agree_on_a_long_prompt(ctx):
         res[engine] = gc.rel.cpu()
     ctx.set_tuning(TCGEN05, 0)
     assert torch.allclose(res[TCGEN05][..., :P], res[MMA_SYNC][..., :P], rtol=2e-4, atol=1e-7)
+    assert torch.allclose(res[TCGEN05_CP_ASYNC][..., :P], res[MMA_SYNC][..., :P], rtol=2e-4, atol=1e-7)
     assert torch.equal(res[TCGEN05][..., P:], oc.rel[..., P:])
     G = Hq // Hkv
     want = G * (1 - 0.995 ** P) / (1 - 0.995)
