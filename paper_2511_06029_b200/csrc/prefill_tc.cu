@@ -151,7 +151,7 @@ __device__ __forceinline__ void tc_commit(unsigned long long* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-// 32 consecutive columns of this thread's TMEM lane.
+// 32 consecutive columns of this thread's TMEM lane (asynchronous: tc_ld_wait before the registers are used).
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -163,8 +163,8 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
           "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
         : "r"(taddr)
         : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Which tiles of the streamed operand meet A block `a`.
 //   STATS : A = query block a (qpb queries x G heads); streamed = key tiles 0 .. (last query of a) / 128
@@ -395,18 +395,25 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
         bool alive = true;
         // COLSUM: every warp keeps its own copy of the factors of the 64 columns it reads (lane x fetches columns
         // x and x + 32 of its half one step ahead), so the softmax warps never wait for one another
-        auto column_factor = [&](int u, int col) -> float2 {
+        // the two partial (max, sum) pairs of a column are fetched one step ahead and kept raw, so that nothing waits
+        // for the loads until the next step turns them into the factor
+        auto fetch_stats = [&](int u, int col, float2& s0, float2& s1) {
             const int qc = u * qpb + col / G, h = col % G;
-            float2 f = make_float2(0.f, 0.f);
+            s0 = make_float2(-INFINITY, 0.f);
+            s1 = s0;
             if (col < used && qc < P) {
                 const size_t at = ((size_t)item * P + qc) * HP + h;
-                const float2 s0 = a.stats[at], s1 = a.stats[half_stride + at];  // (max, sum) over keys 0-63 / 64-127 of every tile
-                const float mx = fmaxf(s0.x, s1.x);
-                const float sum = s0.y * exp2_diff(s0.x, mx) + s1.y * exp2_diff(s1.x, mx);
-                const float wgt = fast_exp2((float)(P - 1 - qc) * a.gamma_log2);
-                f = make_float2(-mx, sum > 0.f ? wgt / sum : 0.f);
+                s0 = a.stats[at];                // over keys 0-63 of every tile
+                s1 = a.stats[half_stride + at];  // over keys 64-127
             }
-            return f;
+        };
+        auto column_factor = [&](int u, int col, const float2& s0, const float2& s1) -> float2 {
+            const int qc = u * qpb + col / G;
+            const float mx = fmaxf(s0.x, s1.x);
+            const float sum = s0.y * exp2_diff(s0.x, mx) + s1.y * exp2_diff(s1.x, mx);
+            if (!(sum > 0.f)) return make_float2(0.f, 0.f);
+            const float wgt = fast_exp2((float)(P - 1 - qc) * a.gamma_log2);
+            return make_float2(-mx, wgt / sum);
         };
         for (int ab = 0; ab < nA && alive; ++ab) {
             int t0, t1;
@@ -416,34 +423,47 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
             const bool row_ok = MODE == kModeStats ? (r < used && qi < P) : (ab * kTcTile + r < P);
             float m = -INFINITY, lsum = 0.f;
             float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
-            float2 f_next[2];
+            float2 s_next[2][2];
 #pragma unroll
-            for (int k = 0; k < 2; ++k)
-                f_next[k] = MODE == kModeColsum ? column_factor(t0, half * 64 + lane + 32 * k) : make_float2(0.f, 0.f);
+            for (int k = 0; k < 2; ++k) {
+                s_next[k][0] = s_next[k][1] = make_float2(-INFINITY, 0.f);
+                if (MODE == kModeColsum) fetch_stats(t0, half * 64 + lane + 32 * k, s_next[k][0], s_next[k][1]);
+            }
             for (int t = t0; t < t1; ++t, ++step) {
                 const int buf = step & 1;
                 if (MODE == kModeColsum) {
                     __syncwarp();
 #pragma unroll
                     for (int k = 0; k < 2; ++k) {
-                        sh.cf[warp][buf][lane + 32 * k] = f_next[k];
-                        if (t + 1 < t1) f_next[k] = column_factor(t + 1, half * 64 + lane + 32 * k);
+                        sh.cf[warp][buf][lane + 32 * k] = column_factor(t, half * 64 + lane + 32 * k, s_next[k][0], s_next[k][1]);
+                        if (t + 1 < t1) fetch_stats(t + 1, half * 64 + lane + 32 * k, s_next[k][0], s_next[k][1]);
                     }
                     __syncwarp();
                 }
                 if (!tc_wait(&sh.t_full[buf], (unsigned)((step >> 1) & 1), abort_flag)) { alive = false; break; }
                 tc_fence_after();
-#pragma unroll 1
+                uint32_t va[32], vb[32];
+                tc_ld32(t_lane + buf * kTcTile, va);
+                tc_ld32(t_lane + buf * kTcTile + 32, vb);
+                tc_ld_wait();
+                tc_fence_before();
+                tc_mbar_arrive(&sh.t_empty[buf]);  // the tile is in registers: the MMA may overwrite this buffer
+#pragma unroll
                 for (int ch = 0; ch < 2; ++ch) {
-                    uint32_t v[32];
-                    tc_ld32(t_lane + buf * kTcTile + ch * 32, v);
+                    uint32_t (&v)[32] = ch == 0 ? va : vb;
                     const int cbase = half * 64 + ch * 32;  // first tile column of this chunk
                     if (MODE == kModeStats) {
                         const int nv = qi - (t * kTcTile + cbase) + 1;  // keys of this chunk that query qi sees
                         if (row_ok && nv >= 32 && sl2 >= 0.f) {
-                            float rm = __uint_as_float(v[0]);
+                            float r0 = __uint_as_float(v[0]), r1 = __uint_as_float(v[1]), r2 = __uint_as_float(v[2]), r3 = __uint_as_float(v[3]);
 #pragma unroll
-                            for (int c = 1; c < 32; ++c) rm = fmaxf(rm, __uint_as_float(v[c]));
+                            for (int c = 4; c < 32; c += 4) {
+                                r0 = fmaxf(r0, __uint_as_float(v[c]));
+                                r1 = fmaxf(r1, __uint_as_float(v[c + 1]));
+                                r2 = fmaxf(r2, __uint_as_float(v[c + 2]));
+                                r3 = fmaxf(r3, __uint_as_float(v[c + 3]));
+                            }
+                            const float rm = fmaxf(fmaxf(r0, r1), fmaxf(r2, r3));
                             const float mx = fmaxf(m, rm * sl2), nmx = -mx;
                             float l0 = lsum * exp2_diff(m, mx), l1 = 0.f, l2 = 0.f, l3 = 0.f;
 #pragma unroll
@@ -496,8 +516,6 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
                         }
                     }
                 }
-                tc_fence_before();
-                tc_mbar_arrive(&sh.t_empty[buf]);
             }
             if (alive && row_ok) {
                 if (MODE == kModeStats) a.stats[half * half_stride + ((size_t)item * P + qi) * HP + r % G] = make_float2(m, lsum);
