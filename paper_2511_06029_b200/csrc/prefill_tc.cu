@@ -49,6 +49,22 @@ __host__ __device__ constexpr int tc_threads() { return (kTcSoftmaxWarps + 1 + (
 
 enum { kModeStats = 0, kModeColsum = 1 };
 
+#ifdef LETHE_TC_TIMELINE
+// Debug build only: nanosecond stamps of CTA 0 of the COLSUM pass, [role][step][4].
+__device__ unsigned long long g_tc_timeline[3 * 64 * 4];
+__device__ __forceinline__ unsigned long long tc_now() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+#define TC_MARK(role, step, k)                                                                                  \
+    do {                                                                                                        \
+        if (MODE == kModeColsum && blockIdx.x == 0 && (step) < 64) g_tc_timeline[((role) * 64 + (step)) * 4 + (k)] = tc_now(); \
+    } while (0)
+#else
+#define TC_MARK(role, step, k) do { } while (0)
+#endif
+
 // Tensor maps of the TMA path: K as [items][capacity][D] with a 128-row box, the prompt's queries as
 // [L B][P][Hq][D] with a (qpb queries x G heads) box; 64-element (128-byte) inner boxes, 128-byte swizzle.
 struct alignas(64) TcMaps {
@@ -270,6 +286,21 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
         float* rel = a.rel + (size_t)item * a.cap_tokens;
         for (int j = tid; j < P; j += kTcSoftmaxThreads) rel[j] = 0.f;
     }
+    if (MODE == kModeColsum) {
+        // turn the item's two partial (max, sum) pairs of every (query, head) column into the column's factor
+        // (-max, decay weight / sum), in place over the first partial; the softmax warps then only copy factors
+        const size_t part = (size_t)gridDim.x * P * HP;
+        for (int idx = tid; idx < P * G; idx += tc_threads<TMA>()) {
+            const int qc = idx / G, h = idx - qc * G;
+            const size_t at = ((size_t)item * P + qc) * HP + h;
+            const float2 s0 = a.stats[at], s1 = a.stats[part + at];
+            const float mx = fmaxf(s0.x, s1.x);
+            const float sum = s0.y * exp2_diff(s0.x, mx) + s1.y * exp2_diff(s1.x, mx);
+            float2 f = make_float2(0.f, 0.f);
+            if (sum > 0.f) f = make_float2(-mx, fast_exp2((float)(P - 1 - qc) * a.gamma_log2) / sum);
+            a.stats[at] = f;
+        }
+    }
     if (warp == kTcMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)),
                      "r"(kTcTmemCols)
@@ -366,9 +397,12 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
                 tc_range<MODE>(ab, P, qpb, t0, t1);
                 for (int t = t0; t < t1; ++t, ++step) {
                     const int s = step % kTcStages, buf = step & 1;
+                    TC_MARK(1, step, 0);
                     if (t == t0 && !tc_wait(&sh.a_full[ab & 1], (unsigned)((ab >> 1) & 1), abort_flag)) { alive = false; break; }
                     if (!tc_wait(&sh.b_full[s], (unsigned)((step / kTcStages) & 1), abort_flag)) { alive = false; break; }
+                    TC_MARK(1, step, 1);
                     if (step >= 2 && !tc_wait(&sh.t_empty[buf], (unsigned)(((step >> 1) - 1) & 1), abort_flag)) { alive = false; break; }
+                    TC_MARK(1, step, 2);
                     tc_fence_after();
                     const uint32_t at = a_tile0 + (ab & 1) * TILE_BYTES, bt = b_tile0 + s * TILE_BYTES;
 #pragma unroll
@@ -380,6 +414,7 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
                     tc_commit(&sh.b_empty[s]);
                     if (t == t1 - 1) tc_commit(&sh.a_empty[ab & 1]);
                     tc_commit(&sh.t_full[buf]);
+                    TC_MARK(1, step, 3);
                 }
             }
         }
@@ -393,27 +428,19 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
         const size_t half_stride = (size_t)gridDim.x * P * HP;  // STATS partials of the upper 64 key columns come second
         int step = 0;
         bool alive = true;
-        // COLSUM: every warp keeps its own copy of the factors of the 64 columns it reads (lane x fetches columns
-        // x and x + 32 of its half one step ahead), so the softmax warps never wait for one another
-        // the two partial (max, sum) pairs of a column are fetched one step ahead and kept raw, so that nothing waits
-        // for the loads until the next step turns them into the factor
-        auto fetch_stats = [&](int u, int col, float2& s0, float2& s1) {
-            const int qc = u * qpb + col / G, h = col % G;
-            s0 = make_float2(-INFINITY, 0.f);
-            s1 = s0;
-            if (col < used && qc < P) {
-                const size_t at = ((size_t)item * P + qc) * HP + h;
-                s0 = a.stats[at];                // over keys 0-63 of every tile
-                s1 = a.stats[half_stride + at];  // over keys 64-127
-            }
-        };
-        auto column_factor = [&](int u, int col, const float2& s0, const float2& s1) -> float2 {
-            const int qc = u * qpb + col / G;
-            const float mx = fmaxf(s0.x, s1.x);
-            const float sum = s0.y * exp2_diff(s0.x, mx) + s1.y * exp2_diff(s1.x, mx);
-            if (!(sum > 0.f)) return make_float2(0.f, 0.f);
-            const float wgt = fast_exp2((float)(P - 1 - qc) * a.gamma_log2);
-            return make_float2(-mx, wgt / sum);
+        // COLSUM: every warp keeps its own copy of the factors of the 64 columns it reads (lane x owns columns x and
+        // x + 32 of its half, fetched one step ahead), so the softmax warps never wait for one another
+        int col_q[2], col_h[2];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const int col = half * 64 + lane + 32 * k;
+            col_q[k] = col < used ? col / G : -1;
+            col_h[k] = col % G;
+        }
+        auto fetch_factor = [&](int u, int k) -> float2 {
+            const int qc = u * qpb + col_q[k];
+            if (col_q[k] < 0 || qc >= P) return make_float2(0.f, 0.f);
+            return a.stats[((size_t)item * P + qc) * HP + col_h[k]];
         };
         for (int ab = 0; ab < nA && alive; ++ab) {
             int t0, t1;
@@ -423,24 +450,23 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
             const bool row_ok = MODE == kModeStats ? (r < used && qi < P) : (ab * kTcTile + r < P);
             float m = -INFINITY, lsum = 0.f;
             float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
-            float2 s_next[2][2];
+            float2 f_next[2];
 #pragma unroll
-            for (int k = 0; k < 2; ++k) {
-                s_next[k][0] = s_next[k][1] = make_float2(-INFINITY, 0.f);
-                if (MODE == kModeColsum) fetch_stats(t0, half * 64 + lane + 32 * k, s_next[k][0], s_next[k][1]);
-            }
+            for (int k = 0; k < 2; ++k) f_next[k] = MODE == kModeColsum ? fetch_factor(t0, k) : make_float2(0.f, 0.f);
             for (int t = t0; t < t1; ++t, ++step) {
                 const int buf = step & 1;
                 if (MODE == kModeColsum) {
                     __syncwarp();
 #pragma unroll
                     for (int k = 0; k < 2; ++k) {
-                        sh.cf[warp][buf][lane + 32 * k] = column_factor(t, half * 64 + lane + 32 * k, s_next[k][0], s_next[k][1]);
-                        if (t + 1 < t1) fetch_stats(t + 1, half * 64 + lane + 32 * k, s_next[k][0], s_next[k][1]);
+                        sh.cf[warp][buf][lane + 32 * k] = f_next[k];
+                        if (t + 1 < t1) f_next[k] = fetch_factor(t + 1, k);
                     }
                     __syncwarp();
                 }
+                if (tid == 0) TC_MARK(0, step, 0);
                 if (!tc_wait(&sh.t_full[buf], (unsigned)((step >> 1) & 1), abort_flag)) { alive = false; break; }
+                if (tid == 0) TC_MARK(0, step, 1);
                 tc_fence_after();
                 uint32_t va[32], vb[32];
                 tc_ld32(t_lane + buf * kTcTile, va);
@@ -448,6 +474,7 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
                 tc_ld_wait();
                 tc_fence_before();
                 tc_mbar_arrive(&sh.t_empty[buf]);  // the tile is in registers: the MMA may overwrite this buffer
+                if (tid == 0) TC_MARK(0, step, 2);
 #pragma unroll
                 for (int ch = 0; ch < 2; ++ch) {
                     uint32_t (&v)[32] = ch == 0 ? va : vb;
@@ -516,6 +543,7 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
                         }
                     }
                 }
+                if (tid == 0) TC_MARK(0, step, 3);
             }
             if (alive && row_ok) {
                 if (MODE == kModeStats) a.stats[half * half_stride + ((size_t)item * P + qi) * HP + r % G] = make_float2(m, lsum);
@@ -581,3 +609,9 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, int items, int L, int D, voi
 }
 
 }  // namespace lethe
+
+#ifdef LETHE_TC_TIMELINE
+extern "C" int lethe_debug_tc_timeline(unsigned long long* host_dst) {
+    return (int)cudaMemcpyFromSymbol(host_dst, lethe::g_tc_timeline, sizeof(unsigned long long) * 3 * 64 * 4);
+}
+#endif
