@@ -488,26 +488,36 @@ def main():
                            torch.zeros((w.n_layers, w.batch, w.n_kv_heads, P), dtype=torch.int32, device=dev),
                            torch.full((w.n_layers, w.batch, w.n_kv_heads), P, dtype=torch.int32, device=dev))
         qp = torch.randn((w.n_layers, w.batch, P, w.n_q_heads, w.head_dim), generator=gq, device=dev).to(w.dtype)
-        for _ in range(2):
-            r.ctx.prefill_seed(pc, qp, r.scale, w.gamma)
-        a_ev = torch.cuda.Event(enable_timing=True); b_ev = torch.cuda.Event(enable_timing=True)
-        a_ev.record()
-        for _ in range(5):
-            r.ctx.prefill_seed(pc, qp, r.scale, w.gamma)
-        b_ev.record()
-        torch.cuda.synchronize(dev)
-        r.check()
-        ms_p = a_ev.elapsed_time(b_ev) / 5
         flops = 2.0 * pc.len.numel() * w.group * (P * (P + 1) / 2) * w.head_dim * 2   # two passes over the causal half
+        exps = 2.0 * pc.len.numel() * w.group * (P * (P + 1) / 2)                      # one exponential per logit and pass
         peaks = {}
         try:
             peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
         except Exception:
             pass
-        tf = flops / (ms_p * 1e-3) / 1e12
-        prefill = {"prompt_len": P, "ms": ms_p, "useful_TFLOPs": tf, "bound": "tensor",
-                   "frac_of_measured_bf16_burst": (tf / peaks["bf16_tflops"]) if "bf16_tflops" in peaks else None,
-                   "note": "two mma.sync passes (statistics, column sums); launches: 2 per call"}
+        xu_peak = 148 * 16 * peaks.get("sm_max_mhz", 1965.0) * 1e6                      # ex2 per second: 16 per SM per clock
+        engines = {}
+        for name_e, code in (("tcgen05", 40), ("mma_sync", 41)):
+            r.ctx.set_tuning(code, 0)
+            for _ in range(2):
+                r.ctx.prefill_seed(pc, qp, r.scale, w.gamma)
+            a_ev = torch.cuda.Event(enable_timing=True); b_ev = torch.cuda.Event(enable_timing=True)
+            a_ev.record()
+            for _ in range(5):
+                r.ctx.prefill_seed(pc, qp, r.scale, w.gamma)
+            b_ev.record()
+            torch.cuda.synchronize(dev)
+            r.check()
+            ms_p = a_ev.elapsed_time(b_ev) / 5
+            tf = flops / (ms_p * 1e-3) / 1e12
+            engines[name_e] = {"ms": ms_p, "useful_TFLOPs": tf,
+                               "frac_of_measured_bf16_burst": (tf / peaks["bf16_tflops"]) if "bf16_tflops" in peaks else None,
+                               "frac_of_ex2_peak": exps / (ms_p * 1e-3) / xu_peak}
+        r.ctx.set_tuning(40, 0)
+        prefill = {"prompt_len": P, "engines": engines, "bound": "alu (ex2: one exponential per logit and pass)",
+                   "ex2_peak_per_s": xu_peak,
+                   "note": "two passes (statistics, column sums), 2 launches per call; tcgen05 = default engine "
+                           "(accumulators in tensor memory, TMA operand tiles), mma_sync = the legacy tensor path"}
         del pc, kp, qp
     e_ms = e_total_ms if not args.no_e2e else 0.0
     e_u = float(sum(e_th)) if not args.no_e2e else 0.0

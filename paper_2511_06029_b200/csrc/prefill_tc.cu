@@ -40,7 +40,9 @@ constexpr int kTcMmaWarp = kTcSoftmaxWarps;                                   //
 constexpr int kTcLoaderWarps = 4;                                             // cp.async path only
 constexpr int kTcLoaderThreads = kTcLoaderWarps * 32;
 constexpr int kTcTile = 128;                                                  // rows of either operand: M = N = 128
-constexpr int kTcStages = 3;                                                  // stages of the streamed operand
+constexpr int kTcStages = 2;                                                  // stages of the streamed operand
+constexpr int kTcABuffers = 1;                                                // buffers of the block operand
+constexpr int kTcCtasPerSm = 2;                                               // co-resident CTAs hide each other's waits
 constexpr int kTcTmemCols = 2 * kTcTile;                                      // two accumulator buffers
 constexpr int kTcWaitLimit = 400000;
 
@@ -72,7 +74,7 @@ struct alignas(64) TcMaps {
 };
 
 struct TcShared {
-    unsigned long long a_full[2], a_empty[2];
+    unsigned long long a_full[kTcABuffers], a_empty[kTcABuffers];
     unsigned long long b_full[kTcStages], b_empty[kTcStages];
     unsigned long long t_full[2], t_empty[2];
     uint32_t tmem_base;
@@ -232,7 +234,7 @@ __device__ __forceinline__ void tc_load_keys(const PrefillArgs& a, int item, int
 }
 
 template <int D, int MODE, bool TMA>
-__global__ void __launch_bounds__(tc_threads<TMA>(), 1)
+__global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
     prefill_tc_kernel(const __grid_constant__ PrefillArgs a, const __grid_constant__ TcMaps maps) {
     constexpr int TILE_BYTES = kTcTile * D * 2;
     constexpr int HALF_BYTES = kTcTile * 128;  // one 64-element half of a tile
@@ -251,14 +253,16 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
     // operand tiles: 1024-byte aligned (the swizzle pattern is anchored at 1024-byte boundaries)
     const uint32_t dyn = (smem_u32(dyn_raw) + 1023u) & ~1023u;
     const uint32_t a_tile0 = dyn;
-    const uint32_t b_tile0 = dyn + 2 * TILE_BYTES;
+    const uint32_t b_tile0 = dyn + kTcABuffers * TILE_BYTES;
     volatile int* abort_flag = &sh.abort;
 
     if (tid == 0) {
         const int producers = TMA ? 1 : kTcLoaderThreads;
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < kTcABuffers; ++i) {
             tc_mbar_init(&sh.a_full[i], producers);
             tc_mbar_init(&sh.a_empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
             tc_mbar_init(&sh.t_full[i], 1);
             tc_mbar_init(&sh.t_empty[i], kTcSoftmaxThreads);
         }
@@ -272,7 +276,7 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
     if (TMA && used < kTcTile) {
         // rows the query boxes never write: zero them once (in every buffer that will hold queries)
         const uint32_t first = MODE == kModeStats ? a_tile0 : b_tile0;
-        const int n_buf = MODE == kModeStats ? 2 : kTcStages;
+        const int n_buf = MODE == kModeStats ? kTcABuffers : kTcStages;
         const int tail_chunks = (kTcTile - used) * 8;  // 16-byte chunks per 64-element half
         for (int idx = tid; idx < n_buf * (D / 64) * tail_chunks; idx += tc_threads<TMA>()) {
             const int c = idx % tail_chunks, hb = idx / tail_chunks;  // hb = buffer * halves + half
@@ -335,11 +339,11 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
                     for (int t = t0; t < t1; ++t, ++step) {
                         const int s = step % kTcStages;
                         if (t == t0) {
-                            if (ab >= 2 && !tc_wait(&sh.a_empty[ab & 1], (unsigned)(((ab >> 1) - 1) & 1), abort_flag)) { alive = false; break; }
-                            const uint32_t at = a_tile0 + (ab & 1) * TILE_BYTES;
-                            tc_mbar_expect_tx(&sh.a_full[ab & 1], MODE == kModeStats ? q_bytes : k_bytes);
-                            if (MODE == kModeStats) load_queries(ab * qpb, at, &sh.a_full[ab & 1]);
-                            else load_keys(ab * kTcTile, at, &sh.a_full[ab & 1]);
+                            if (ab >= kTcABuffers && !tc_wait(&sh.a_empty[ab % kTcABuffers], (unsigned)(((ab / kTcABuffers) - 1) & 1), abort_flag)) { alive = false; break; }
+                            const uint32_t at = a_tile0 + (ab % kTcABuffers) * TILE_BYTES;
+                            tc_mbar_expect_tx(&sh.a_full[ab % kTcABuffers], MODE == kModeStats ? q_bytes : k_bytes);
+                            if (MODE == kModeStats) load_queries(ab * qpb, at, &sh.a_full[ab % kTcABuffers]);
+                            else load_keys(ab * kTcTile, at, &sh.a_full[ab % kTcABuffers]);
                         }
                         if (step >= kTcStages && !tc_wait(&sh.b_empty[s], (unsigned)(((step / kTcStages) - 1) & 1), abort_flag)) { alive = false; break; }
                         const uint32_t bt = b_tile0 + s * TILE_BYTES;
@@ -352,8 +356,8 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
             __syncwarp();
         } else {
             const int ltid = tid - (kTcMmaWarp + 1) * 32;
-            int step = 0, prev_stage = -1, prev_a = -1;
-            bool prev_first = false, alive = true;
+            int step = 0;
+            bool alive = true;
             for (int ab = 0; ab < nA && alive; ++ab) {
                 int t0, t1;
                 tc_range<MODE>(ab, P, qpb, t0, t1);
@@ -361,29 +365,22 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
                     const int s = step % kTcStages;
                     const bool first = t == t0;
                     if (first) {
-                        if (ab >= 2 && !tc_wait(&sh.a_empty[ab & 1], (unsigned)(((ab >> 1) - 1) & 1), abort_flag)) { alive = false; break; }
-                        const uint32_t at = a_tile0 + (ab & 1) * TILE_BYTES;
+                        if (ab >= kTcABuffers && !tc_wait(&sh.a_empty[ab % kTcABuffers], (unsigned)(((ab / kTcABuffers) - 1) & 1), abort_flag)) { alive = false; break; }
+                        const uint32_t at = a_tile0 + (ab % kTcABuffers) * TILE_BYTES;
                         if (MODE == kModeStats) tc_load_queries<D>(a, l, b, hkv, ab * qpb, used, at, ltid);
                         else tc_load_keys<D>(a, item, ab * kTcTile, at, ltid);
                     }
                     if (step >= kTcStages && !tc_wait(&sh.b_empty[s], (unsigned)(((step / kTcStages) - 1) & 1), abort_flag)) { alive = false; break; }
                     if (MODE == kModeStats) tc_load_keys<D>(a, item, t * kTcTile, b_tile0 + s * TILE_BYTES, ltid);
                     else tc_load_queries<D>(a, l, b, hkv, t * qpb, used, b_tile0 + s * TILE_BYTES, ltid);
+                    // the step's copies must have landed and be visible to the MMA's proxy before it is told; nothing
+                    // is held back (a later wait of this loop may depend on the MMA of this very step)
                     cp_async_commit();
-                    if (prev_stage >= 0) {  // the previous step's copies have landed: publish them to the MMA's proxy
-                        cp_async_wait<1>();
-                        tc_fence_proxy_async();
-                        if (prev_first) tc_mbar_arrive(&sh.a_full[prev_a & 1]);
-                        tc_mbar_arrive(&sh.b_full[prev_stage]);
-                    }
-                    prev_stage = s; prev_a = ab; prev_first = first;
+                    cp_async_wait<0>();
+                    tc_fence_proxy_async();
+                    if (first) tc_mbar_arrive(&sh.a_full[ab % kTcABuffers]);
+                    tc_mbar_arrive(&sh.b_full[s]);
                 }
-            }
-            cp_async_wait<0>();
-            if (alive && prev_stage >= 0) {
-                tc_fence_proxy_async();
-                if (prev_first) tc_mbar_arrive(&sh.a_full[prev_a & 1]);
-                tc_mbar_arrive(&sh.b_full[prev_stage]);
             }
         }
     } else if (warp == kTcMmaWarp) {
@@ -398,13 +395,13 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
                 for (int t = t0; t < t1; ++t, ++step) {
                     const int s = step % kTcStages, buf = step & 1;
                     TC_MARK(1, step, 0);
-                    if (t == t0 && !tc_wait(&sh.a_full[ab & 1], (unsigned)((ab >> 1) & 1), abort_flag)) { alive = false; break; }
+                    if (t == t0 && !tc_wait(&sh.a_full[ab % kTcABuffers], (unsigned)((ab / kTcABuffers) & 1), abort_flag)) { alive = false; break; }
                     if (!tc_wait(&sh.b_full[s], (unsigned)((step / kTcStages) & 1), abort_flag)) { alive = false; break; }
                     TC_MARK(1, step, 1);
                     if (step >= 2 && !tc_wait(&sh.t_empty[buf], (unsigned)(((step >> 1) - 1) & 1), abort_flag)) { alive = false; break; }
                     TC_MARK(1, step, 2);
                     tc_fence_after();
-                    const uint32_t at = a_tile0 + (ab & 1) * TILE_BYTES, bt = b_tile0 + s * TILE_BYTES;
+                    const uint32_t at = a_tile0 + (ab % kTcABuffers) * TILE_BYTES, bt = b_tile0 + s * TILE_BYTES;
 #pragma unroll
                     for (int ks = 0; ks < KS; ++ks) {
                         // 16 elements of K per MMA: 32 bytes along the swizzled row; the second 64 elements are the next region
@@ -412,7 +409,7 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
                         tc_mma(tmem + buf * kTcTile, tc_smem_desc(at + off), tc_smem_desc(bt + off), idesc, ks > 0 ? 1u : 0u);
                     }
                     tc_commit(&sh.b_empty[s]);
-                    if (t == t1 - 1) tc_commit(&sh.a_empty[ab & 1]);
+                    if (t == t1 - 1) tc_commit(&sh.a_empty[ab % kTcABuffers]);
                     tc_commit(&sh.t_full[buf]);
                     TC_MARK(1, step, 3);
                 }
@@ -468,16 +465,16 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
                 if (!tc_wait(&sh.t_full[buf], (unsigned)((step >> 1) & 1), abort_flag)) { alive = false; break; }
                 if (tid == 0) TC_MARK(0, step, 1);
                 tc_fence_after();
-                uint32_t va[32], vb[32];
-                tc_ld32(t_lane + buf * kTcTile, va);
-                tc_ld32(t_lane + buf * kTcTile + 32, vb);
-                tc_ld_wait();
-                tc_fence_before();
-                tc_mbar_arrive(&sh.t_empty[buf]);  // the tile is in registers: the MMA may overwrite this buffer
-                if (tid == 0) TC_MARK(0, step, 2);
 #pragma unroll
                 for (int ch = 0; ch < 2; ++ch) {
-                    uint32_t (&v)[32] = ch == 0 ? va : vb;
+                    uint32_t v[32];
+                    tc_ld32(t_lane + buf * kTcTile + ch * 32, v);
+                    tc_ld_wait();
+                    if (ch == 1) {  // the tile is in registers: the MMA may overwrite this buffer
+                        tc_fence_before();
+                        tc_mbar_arrive(&sh.t_empty[buf]);
+                        if (tid == 0) TC_MARK(0, step, 2);
+                    }
                     const int cbase = half * 64 + ch * 32;  // first tile column of this chunk
                     if (MODE == kModeStats) {
                         const int nv = qi - (t * kTcTile + cbase) + 1;  // keys of this chunk that query qi sees
@@ -562,7 +559,7 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), 1)
 
 template <int D, bool TMA>
 cudaError_t launch_tc(const PrefillArgs& a, const TcMaps& maps, int items, cudaStream_t stream) {
-    const size_t smem = 1024 + (size_t)(2 + kTcStages) * kTcTile * D * 2;
+    const size_t smem = 1024 + (size_t)(kTcABuffers + kTcStages) * kTcTile * D * 2;
     cudaError_t e = prepare_kernel((const void*)prefill_tc_kernel<D, kModeStats, TMA>, smem);
     if (e != cudaSuccess) return e;
     e = prepare_kernel((const void*)prefill_tc_kernel<D, kModeColsum, TMA>, smem);
