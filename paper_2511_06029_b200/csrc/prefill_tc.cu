@@ -79,8 +79,8 @@ struct TcShared {
     unsigned long long t_full[2], t_empty[2];
     uint32_t tmem_base;
     int abort;
-    // COLSUM: (-max, weight / sum) of the 64 columns a warp reads, of the tiles in flight; one copy per warp
-    alignas(16) float2 cf[kTcSoftmaxWarps][2][kTcTile / 2];
+    // COLSUM: bias (log2(weight / sum) - max) of the 64 columns a warp reads, of the tiles in flight; one copy per warp
+    alignas(16) float cf[kTcSoftmaxWarps][2][kTcTile / 2];
 };
 
 __device__ __forceinline__ void tc_mbar_init(unsigned long long* bar, int count) {
@@ -291,8 +291,8 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
         for (int j = tid; j < P; j += kTcSoftmaxThreads) rel[j] = 0.f;
     }
     if (MODE == kModeColsum) {
-        // turn the item's two partial (max, sum) pairs of every (query, head) column into the column's factor
-        // (-max, decay weight / sum), in place over the first partial; the softmax warps then only copy factors
+        // turn the item's two partial (max, sum) pairs of every (query, head) column into the column's bias
+        // log2(decay weight / sum) - max, in place over the first partial; the softmax warps then only copy biases
         const size_t part = (size_t)gridDim.x * P * HP;
         for (int idx = tid; idx < P * G; idx += tc_threads<TMA>()) {
             const int qc = idx / G, h = idx - qc * G;
@@ -300,9 +300,9 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
             const float2 s0 = a.stats[at], s1 = a.stats[part + at];
             const float mx = fmaxf(s0.x, s1.x);
             const float sum = s0.y * exp2_diff(s0.x, mx) + s1.y * exp2_diff(s1.x, mx);
-            float2 f = make_float2(0.f, 0.f);
-            if (sum > 0.f) f = make_float2(-mx, fast_exp2((float)(P - 1 - qc) * a.gamma_log2) / sum);
-            a.stats[at] = f;
+            // exp2(logit - max) * weight / sum = exp2(logit + bias) with one bias per column
+            const float bias = sum > 0.f ? (float)(P - 1 - qc) * a.gamma_log2 - mx - __log2f(sum) : -INFINITY;
+            a.stats[at] = make_float2(bias, 0.f);
         }
     }
     if (warp == kTcMmaWarp) {
@@ -434,10 +434,10 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
             col_q[k] = col < used ? col / G : -1;
             col_h[k] = col % G;
         }
-        auto fetch_factor = [&](int u, int k) -> float2 {
+        auto fetch_factor = [&](int u, int k) -> float {
             const int qc = u * qpb + col_q[k];
-            if (col_q[k] < 0 || qc >= P) return make_float2(0.f, 0.f);
-            return a.stats[((size_t)item * P + qc) * HP + col_h[k]];
+            if (col_q[k] < 0 || qc >= P) return -INFINITY;
+            return a.stats[((size_t)item * P + qc) * HP + col_h[k]].x;
         };
         for (int ab = 0; ab < nA && alive; ++ab) {
             int t0, t1;
@@ -447,9 +447,9 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
             const bool row_ok = MODE == kModeStats ? (r < used && qi < P) : (ab * kTcTile + r < P);
             float m = -INFINITY, lsum = 0.f;
             float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
-            float2 f_next[2];
+            float f_next[2];
 #pragma unroll
-            for (int k = 0; k < 2; ++k) f_next[k] = MODE == kModeColsum ? fetch_factor(t0, k) : make_float2(0.f, 0.f);
+            for (int k = 0; k < 2; ++k) f_next[k] = MODE == kModeColsum ? fetch_factor(t0, k) : 0.f;
             for (int t = t0; t < t1; ++t, ++step) {
                 const int buf = step & 1;
                 if (MODE == kModeColsum) {
@@ -524,18 +524,20 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
                         if (row_ok && c_lo <= 0 && c_hi >= 32) {
 #pragma unroll
                             for (int c = 0; c < 32; c += 4) {
-                                const float4 fa = cf4[c / 2], fb = cf4[c / 2 + 1];  // (-max, w) of columns c, c+1 | c+2, c+3
-                                acc0 = fmaf(fast_exp2(fmaf(__uint_as_float(v[c]), sl2, fa.x)), fa.y, acc0);
-                                acc1 = fmaf(fast_exp2(fmaf(__uint_as_float(v[c + 1]), sl2, fa.z)), fa.w, acc1);
-                                acc2 = fmaf(fast_exp2(fmaf(__uint_as_float(v[c + 2]), sl2, fb.x)), fb.y, acc2);
-                                acc3 = fmaf(fast_exp2(fmaf(__uint_as_float(v[c + 3]), sl2, fb.z)), fb.w, acc3);
+                                const float4 fb = cf4[c / 4];  // biases of columns c .. c + 3
+                                acc0 += fast_exp2(fmaf(__uint_as_float(v[c]), sl2, fb.x));
+                                acc1 += fast_exp2(fmaf(__uint_as_float(v[c + 1]), sl2, fb.y));
+                                acc2 += fast_exp2(fmaf(__uint_as_float(v[c + 2]), sl2, fb.z));
+                                acc3 += fast_exp2(fmaf(__uint_as_float(v[c + 3]), sl2, fb.w));
                             }
                         } else if (row_ok && c_lo < 32 && c_hi > 0) {
 #pragma unroll
-                            for (int c = 0; c < 32; c += 2) {
-                                const float4 fa = cf4[c / 2];
-                                if (c >= c_lo && c < c_hi) acc0 = fmaf(fast_exp2(fmaf(__uint_as_float(v[c]), sl2, fa.x)), fa.y, acc0);
-                                if (c + 1 >= c_lo && c + 1 < c_hi) acc1 = fmaf(fast_exp2(fmaf(__uint_as_float(v[c + 1]), sl2, fa.z)), fa.w, acc1);
+                            for (int c = 0; c < 32; c += 4) {
+                                const float4 fb = cf4[c / 4];
+                                if (c >= c_lo && c < c_hi) acc0 += fast_exp2(fmaf(__uint_as_float(v[c]), sl2, fb.x));
+                                if (c + 1 >= c_lo && c + 1 < c_hi) acc1 += fast_exp2(fmaf(__uint_as_float(v[c + 1]), sl2, fb.y));
+                                if (c + 2 >= c_lo && c + 2 < c_hi) acc2 += fast_exp2(fmaf(__uint_as_float(v[c + 2]), sl2, fb.z));
+                                if (c + 3 >= c_lo && c + 3 < c_hi) acc3 += fast_exp2(fmaf(__uint_as_float(v[c + 3]), sl2, fb.w));
                             }
                         }
                     }
