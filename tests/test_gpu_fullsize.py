@@ -1,4 +1,5 @@
-"""Parity at the full size of the Llama-8B-shaped workload (the one bench.py times) and of the Qwen-7B-shaped one,
+"""Parity at the full size of the Llama-8B-shaped workload (the one bench.py times), of the Qwen-7B-shaped one and of
+the long-reasoning stress shape,
 in exactly the launch configuration bench.py uses (its Runner: all layers x sequences x KV heads in one
 lethe_decode_attend call, default tuning).  The oracle cannot run the whole state in seconds, so it recomputes
 sampled items one by one from snapshots of the GPU state taken just before the call."""
@@ -18,7 +19,7 @@ def _item_cache(k, v, rel, pos, n, G, D, cap):
                               pos.reshape(1, 1, 1, cap).contiguous(), torch.tensor([[[n]]], dtype=torch.int32))
 
 
-@pytest.mark.parametrize("name,cap_factor", [("llama8b", 2), ("qwen7b", 3)])
+@pytest.mark.parametrize("name,cap_factor", [("llama8b", 2), ("qwen7b", 3), ("longreason", 3)])
 def test_full_size_sampled_items(name, cap_factor):
     import bench
     from paper_2511_06029_b200 import synth
