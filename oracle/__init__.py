@@ -22,7 +22,7 @@ _SRC = os.path.join(_HERE, "lethe_oracle.c")
 _LIB = os.path.join(_HERE, "liblethe_oracle.so")
 
 OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_BUDGET = 0, 1, 2, 3
-F32, BF16 = 0, 1
+F32, BF16, FP8 = 0, 1, 2
 
 
 def build(force: bool = False) -> str:
@@ -41,7 +41,7 @@ class _CCache(ctypes.Structure):
         ("paged", ctypes.c_int32), ("capacity", ctypes.c_int32), ("page_tokens", ctypes.c_int32),
         ("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("rel", ctypes.c_void_p),
         ("pos", ctypes.c_void_p), ("len", ctypes.c_void_p), ("page_table", ctypes.c_void_p),
-        ("n_pages", ctypes.c_int64),
+        ("n_pages", ctypes.c_int64), ("k_scale", ctypes.c_void_p), ("v_scale", ctypes.c_void_p),
     ]
 
 
@@ -74,6 +74,10 @@ def lib():
         _lib.oracle_prefill_seed.restype = ctypes.c_int
         _lib.oracle_prefill_seed.argtypes = [ctypes.POINTER(_CCache), ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p,
                                              ctypes.c_float]
+        _lib.oracle_e4m3_decode.restype = ctypes.c_double
+        _lib.oracle_e4m3_decode.argtypes = [ctypes.c_uint8]
+        _lib.oracle_e4m3_encode.restype = ctypes.c_uint8
+        _lib.oracle_e4m3_encode.argtypes = [ctypes.c_float]
         _lib.oracle_set_threads.argtypes = [ctypes.c_int]
         _lib.oracle_get_threads.restype = ctypes.c_int
         _lib.oracle_max_threads.restype = ctypes.c_int
@@ -104,6 +108,8 @@ def _dtype_code(dt: torch.dtype) -> int:
         return F32
     if dt == torch.bfloat16:
         return BF16
+    if dt == torch.float8_e4m3fn:
+        return FP8
     raise ValueError(f"unsupported dtype {dt}")
 
 
@@ -123,6 +129,13 @@ class OracleCache:
     len: torch.Tensor
     page_tokens: int = 0
     page_table: Optional[torch.Tensor] = None
+    k_scale: Optional[torch.Tensor] = None      # float8_e4m3fn caches: fp32 [L] (None = 1): stored byte x means scale * x
+    v_scale: Optional[torch.Tensor] = None
+
+    @property
+    def act_dtype(self) -> torch.dtype:
+        """Type of q, k_new, v_new and out: the cache's own, bf16 for a quantised cache."""
+        return torch.bfloat16 if self.k.dtype == torch.float8_e4m3fn else self.k.dtype
 
     @property
     def paged(self) -> bool:
@@ -137,13 +150,17 @@ class OracleCache:
                        _dtype_code(self.k.dtype), 1 if self.paged else 0, self.capacity, self.page_tokens,
                        self.k.data_ptr(), self.v.data_ptr(), self.rel.data_ptr(), self.pos.data_ptr(),
                        self.len.data_ptr(), self.page_table.data_ptr() if self.paged else None,
-                       self.k.shape[0] if self.paged else 0)
+                       self.k.shape[0] if self.paged else 0,
+                       None if self.k_scale is None else self.k_scale.data_ptr(),
+                       None if self.v_scale is None else self.v_scale.data_ptr())
 
     def clone(self) -> "OracleCache":
         return OracleCache(self.n_layers, self.batch, self.n_q_heads, self.n_kv_heads, self.head_dim,
                            self.capacity, self.k.clone(), self.v.clone(), self.rel.clone(), self.pos.clone(),
                            self.len.clone(), self.page_tokens,
-                           None if self.page_table is None else self.page_table.clone())
+                           None if self.page_table is None else self.page_table.clone(),
+                           None if self.k_scale is None else self.k_scale.clone(),
+                           None if self.v_scale is None else self.v_scale.clone())
 
 
 def decode_attend(cache: OracleCache, layer_begin: int, layer_end: int, q: torch.Tensor,
@@ -152,11 +169,13 @@ def decode_attend(cache: OracleCache, layer_begin: int, layer_end: int, q: torch
                   want_lse: bool = False, want_probs: bool = False):
     """One decode step for layers [layer_begin, layer_end); returns (status, out, lse, probs)."""
     nl = layer_end - layer_begin
-    out = torch.zeros((nl, cache.batch, cache.n_q_heads, cache.head_dim), dtype=cache.k.dtype)
+    out = torch.zeros((nl, cache.batch, cache.n_q_heads, cache.head_dim), dtype=cache.act_dtype)
     lse = torch.zeros((nl, cache.batch, cache.n_q_heads), dtype=torch.float32) if want_lse else None
     probs = (torch.zeros((nl, cache.batch, cache.n_q_heads, cache.cap_tokens), dtype=torch.float64)
              if want_probs else None)
-    assert q.dtype == cache.k.dtype and scale.dtype == torch.float32 and scale.numel() == cache.n_layers
+    assert q.dtype == cache.act_dtype and scale.dtype == torch.float32 and scale.numel() == cache.n_layers
+    for sc in (cache.k_scale, cache.v_scale):
+        assert sc is None or (sc.dtype == torch.float32 and sc.numel() == cache.n_layers and sc.is_contiguous())
     if token_pos is not None:
         assert token_pos.dtype == torch.int32
     cc = cache._c()

@@ -40,6 +40,10 @@
  *                             batch), and one retention set shared by everything summed
  *                             over; same protected top-k and compaction as oracle_rasr_prune.
  *
+ * K and V may also be stored quantised (e4m3 bytes with one scale per layer): the paper's
+ * related-work section notes that quantised caches compose with eviction; it defines no
+ * format, so the format is this build's choice (stated at oracle_decode_attend).
+ *
  * Arithmetic: every floating-point step is done in double; stored results are
  * rounded once to their storage type (fp32, or bf16 round-to-nearest-even).
  * Integer steps (budgets, selection, compaction) have exactly one right answer.
@@ -60,11 +64,12 @@
 #endif
 
 enum { ORACLE_OK = 0, ORACLE_ERR_INVALID_ARG = 1, ORACLE_ERR_CAPACITY = 2, ORACLE_ERR_BUDGET = 3 };
-enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
+enum { ORACLE_F32 = 0, ORACLE_BF16 = 1, ORACLE_FP8 = 2 };
 
 typedef struct {
     int32_t n_layers, batch, n_q_heads, n_kv_heads, head_dim;
-    int32_t dtype;       /* ORACLE_F32 or ORACLE_BF16 (bf16 held as uint16) */
+    int32_t dtype;       /* storage type of K and V: ORACLE_F32, ORACLE_BF16 (held as uint16) or ORACLE_FP8
+                            (e4m3fn bytes; q, k_new, v_new, out are then bf16) */
     int32_t paged;       /* 0 contiguous, 1 paged */
     int32_t capacity;    /* contiguous: token slots per item; paged: pages per item */
     int32_t page_tokens; /* tokens per page when paged, else ignored */
@@ -74,6 +79,8 @@ typedef struct {
     int32_t *len;
     int32_t *page_table;
     int64_t n_pages;
+    const float *k_scale; /* ORACLE_FP8 only, [n_layers] or NULL (= 1): a stored key byte x means k_scale[l] * x */
+    const float *v_scale; /* the same for values */
 } oracle_cache;
 
 static int g_threads = 1;
@@ -116,8 +123,40 @@ static uint16_t double_to_bf16(double x) {
     return (uint16_t)(u >> 16);
 }
 
+/* e4m3fn (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no infinities; S.1111.111 is NaN; largest
+ * finite value 448; subnormals are multiples of 2^-9). */
+static double e4m3_to_double(uint8_t b) {
+    const int e = (b >> 3) & 15, m = b & 7;
+    double x;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) x = ldexp((double)m, -9);
+    else x = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return (b & 0x80) ? -x : x;
+}
+
+/* float -> e4m3fn: round to nearest, ties to even; magnitudes beyond the largest finite value saturate to it
+ * (the conversion a quantised cache uses: no value becomes NaN by overflow). */
+static uint8_t float_to_e4m3(float f) {
+    if (f != f) return 0x7f;
+    const uint8_t sign = signbit(f) ? 0x80 : 0x00;
+    const float a = fabsf(f);
+    if (a > 448.0f) return sign | 0x7e;
+    if (a < 0.015625f) return sign | (uint8_t)rintf(a * 512.0f); /* subnormal step 2^-9; 8 is the smallest normal */
+    int ex;
+    const float fr = frexpf(a, &ex);                  /* a = fr * 2^ex, fr in [0.5, 1) */
+    int q = (int)rintf((2.0f * fr - 1.0f) * 8.0f);    /* mantissa in eighths, 0..8 (rintf: ties to even) */
+    int e = ex - 1 + 7;
+    if (q == 8) {
+        q = 0;
+        e += 1;
+    }
+    const int code = (e << 3) | q;
+    return sign | (uint8_t)(code > 0x7e ? 0x7e : code);
+}
+
 static double load_elt(const void *base, int dtype, int64_t idx) {
     if (dtype == ORACLE_BF16) return bf16_to_double(((const uint16_t *)base)[idx]);
+    if (dtype == ORACLE_FP8) return e4m3_to_double(((const uint8_t *)base)[idx]);
     return (double)((const float *)base)[idx];
 }
 
@@ -126,7 +165,14 @@ static void store_elt(void *base, int dtype, int64_t idx, double x) {
     else ((float *)base)[idx] = (float)x;
 }
 
-static size_t elt_size(int dtype) { return dtype == ORACLE_BF16 ? 2 : 4; }
+static size_t elt_size(int dtype) { return dtype == ORACLE_BF16 ? 2 : (dtype == ORACLE_FP8 ? 1 : 4); }
+
+/* type of q, k_new, v_new and out: the cache's own, except that a quantised cache takes bf16 activations */
+static int act_dtype(int dtype) { return dtype == ORACLE_FP8 ? ORACLE_BF16 : dtype; }
+
+/* test hooks for the two conversions */
+double oracle_e4m3_decode(uint8_t b) { return e4m3_to_double(b); }
+uint8_t oracle_e4m3_encode(float f) { return float_to_e4m3(f); }
 
 static int64_t cap_tokens(const oracle_cache *c) {
     return c->paged ? (int64_t)c->capacity * c->page_tokens : (int64_t)c->capacity;
@@ -148,7 +194,7 @@ static int check_cache(const oracle_cache *c) {
     if (!c || !c->k || !c->v || !c->rel || !c->pos || !c->len) return ORACLE_ERR_INVALID_ARG;
     if (c->n_layers < 1 || c->batch < 1 || c->n_kv_heads < 1 || c->head_dim < 1) return ORACLE_ERR_INVALID_ARG;
     if (c->n_q_heads < c->n_kv_heads || c->n_q_heads % c->n_kv_heads) return ORACLE_ERR_INVALID_ARG;
-    if (c->dtype != ORACLE_F32 && c->dtype != ORACLE_BF16) return ORACLE_ERR_INVALID_ARG;
+    if (c->dtype != ORACLE_F32 && c->dtype != ORACLE_BF16 && c->dtype != ORACLE_FP8) return ORACLE_ERR_INVALID_ARG;
     if (c->capacity < 1) return ORACLE_ERR_INVALID_ARG;
     if (c->paged && (!c->page_table || c->page_tokens < 1)) return ORACLE_ERR_INVALID_ARG;
     return ORACLE_OK;
@@ -157,8 +203,12 @@ static int check_cache(const oracle_cache *c) {
 /* ---- decode step: append, attend, relevance (Sec. 4.1, Eq. 3, Eq. 5) ------ */
 /*
  * For layers [layer_begin, layer_end), with li = layer - layer_begin:
- *   q, out        [layers][B][Hq][D]   (cache dtype)
- *   k_new, v_new  [layers][B][Hkv][D]  (cache dtype) or both NULL = attend only
+ *   q, out        [layers][B][Hq][D]   (cache dtype; bf16 when the cache is ORACLE_FP8)
+ *   k_new, v_new  [layers][B][Hkv][D]  (same type as q) or both NULL = attend only
+ * A quantised (ORACLE_FP8) cache holds K / k_scale[l] and V / v_scale[l] as e4m3fn bytes: an appended row is
+ * divided by the layer's scale in fp32 (one IEEE division) and rounded to nearest-even with saturation; when
+ * read, a byte x counts as scale * x exactly.  Quantisation composes with pruning (Sec. 2, related work on
+ * quantised caches): rows are moved as bytes, scores never see the storage type.
  *   token_pos     [B] original position written to pos[] for the appended token
  *   scale         [n_layers] softmax scale of each layer (indexed by absolute layer)
  *   lse           optional [layers][B][Hq]   log-sum-exp of the scaled logits
@@ -200,16 +250,27 @@ int oracle_decode_attend(oracle_cache *c, int layer_begin, int layer_end, const 
         const int hkv = w % Hkv;
         const int64_t item = item_index(c, l, b, hkv);
         int64_t n = c->len[item];
+        const int act = act_dtype(c->dtype);
+        const float ks = (c->dtype == ORACLE_FP8 && c->k_scale) ? c->k_scale[l] : 1.0f;
+        const float vs = (c->dtype == ORACLE_FP8 && c->v_scale) ? c->v_scale[l] : 1.0f;
 
         /* Sec. 4.1: the cache grows by the token just generated.  It enters with
          * zero relevance and takes part in this step's attention. */
         if (k_new) {
             const int64_t src = (((int64_t)li * B + b) * Hkv + hkv) * D;
             const int64_t dst = row_offset(c, item, n);
-            memcpy((char *)c->k + dst * elt_size(c->dtype), (const char *)k_new + src * elt_size(c->dtype),
-                   D * elt_size(c->dtype));
-            memcpy((char *)c->v + dst * elt_size(c->dtype), (const char *)v_new + src * elt_size(c->dtype),
-                   D * elt_size(c->dtype));
+            if (c->dtype == ORACLE_FP8) {
+                for (int d = 0; d < D; ++d) {
+                    const float kx = (float)load_elt(k_new, ORACLE_BF16, src + d), vx = (float)load_elt(v_new, ORACLE_BF16, src + d);
+                    ((uint8_t *)c->k)[dst + d] = float_to_e4m3(kx / ks);
+                    ((uint8_t *)c->v)[dst + d] = float_to_e4m3(vx / vs);
+                }
+            } else {
+                memcpy((char *)c->k + dst * elt_size(c->dtype), (const char *)k_new + src * elt_size(c->dtype),
+                       D * elt_size(c->dtype));
+                memcpy((char *)c->v + dst * elt_size(c->dtype), (const char *)v_new + src * elt_size(c->dtype),
+                       D * elt_size(c->dtype));
+            }
             c->rel[item * capT + n] = 0.0f;
             c->pos[item * capT + n] = token_pos[b];
             n += 1;
@@ -225,7 +286,7 @@ int oracle_decode_attend(oracle_cache *c, int layer_begin, int layer_end, const 
             const int h = hkv * G + g;
             const int64_t qoff = (((int64_t)li * B + b) * Hq + h) * D;
             if (n == 0) {
-                for (int d = 0; d < D; ++d) store_elt(out, c->dtype, qoff + d, 0.0);
+                for (int d = 0; d < D; ++d) store_elt(out, act, qoff + d, 0.0);
                 if (lse) lse[((int64_t)li * B + b) * Hq + h] = -INFINITY;
                 continue;
             }
@@ -233,7 +294,7 @@ int oracle_decode_attend(oracle_cache *c, int layer_begin, int layer_end, const 
             for (int64_t j = 0; j < n; ++j) {
                 const int64_t koff = row_offset(c, item, j);
                 double s = 0.0;
-                for (int d = 0; d < D; ++d) s += load_elt(q, c->dtype, qoff + d) * load_elt(c->k, c->dtype, koff + d);
+                for (int d = 0; d < D; ++d) s += load_elt(q, act, qoff + d) * ((double)ks * load_elt(c->k, c->dtype, koff + d));
                 s *= (double)scale[l];
                 p[j] = s;
                 if (s > m) m = s;
@@ -248,10 +309,10 @@ int oracle_decode_attend(oracle_cache *c, int layer_begin, int layer_end, const 
                 p[j] /= Z;
                 mass[j] += p[j];
                 const int64_t voff = row_offset(c, item, j);
-                for (int d = 0; d < D; ++d) o[d] += p[j] * load_elt(c->v, c->dtype, voff + d);
+                for (int d = 0; d < D; ++d) o[d] += p[j] * ((double)vs * load_elt(c->v, c->dtype, voff + d));
                 if (probs) probs[(((int64_t)li * B + b) * Hq + h) * capT + j] = p[j];
             }
-            for (int d = 0; d < D; ++d) store_elt(out, c->dtype, qoff + d, o[d]);
+            for (int d = 0; d < D; ++d) store_elt(out, act, qoff + d, o[d]);
             if (lse) lse[((int64_t)li * B + b) * Hq + h] = (float)(m + log(Z));
         }
 
@@ -659,6 +720,7 @@ int oracle_prefill_seed(oracle_cache *c, const void *q_prompt, int32_t prompt_le
     int st = check_cache(c);
     if (st) return st;
     if (!q_prompt || !scale || prompt_len < 1 || !(gamma > 0.0f && gamma <= 1.0f)) return ORACLE_ERR_INVALID_ARG;
+    if (c->dtype == ORACLE_FP8) return ORACLE_ERR_INVALID_ARG; /* prompt keys are seeded before quantisation */
     const int B = c->batch, Hq = c->n_q_heads, Hkv = c->n_kv_heads, D = c->head_dim, P = prompt_len;
     const int G = Hq / Hkv;
     const int64_t capT = cap_tokens(c);

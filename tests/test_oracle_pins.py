@@ -617,3 +617,113 @@ def test_collapsed_special_cases():
     st_a, keep_a = oracle.collapsed_prune(a, bud, 8, 2, oracle.COLLAPSE_HEADS_BATCH, max_k=64)
     st_b, keep_b = oracle.collapsed_prune(b, bud, 8, 2, oracle.COLLAPSE_HEADS, max_k=64)
     assert st_a == st_b == oracle.OK and torch.equal(keep_a, keep_b) and torch.equal(a.k.flatten(), b.k.flatten())
+
+
+# ----------------------------------------------------------------------------- quantised (e4m3) K / V storage
+
+def _fp8_cache(L, B, Hq, Hkv, D, cap, n, seed, k_scale, v_scale):
+    """Cache whose K / V bytes are random e4m3 codes (no NaN codes), with per-layer scales."""
+    g = torch.Generator().manual_seed(seed)
+    def codes():
+        c = torch.randint(0, 256, (L, B, Hkv, cap, D), generator=g, dtype=torch.int32)
+        c[(c & 0x7f) == 0x7f] = 0x30
+        return c.to(torch.uint8).view(torch.float8_e4m3fn)
+    rel = torch.rand((L, B, Hkv, cap), generator=g)
+    pos = torch.arange(cap, dtype=torch.int32).expand(L, B, Hkv, cap).contiguous()
+    return oracle.OracleCache(L, B, Hq, Hkv, D, cap, codes(), codes(), rel, pos, torch.full((L, B, Hkv), n, dtype=torch.int32),
+                              k_scale=torch.tensor(k_scale, dtype=torch.float32), v_scale=torch.tensor(v_scale, dtype=torch.float32))
+
+
+def test_e4m3_conversions_against_closed_forms_and_the_library():
+    lib = oracle.lib()
+    # decode: every code against the library's table, a few against the format's definition
+    codes = torch.arange(256, dtype=torch.uint8)
+    ref = codes.view(torch.float8_e4m3fn).double()
+    got = torch.tensor([lib.oracle_e4m3_decode(int(c)) for c in codes], dtype=torch.float64)
+    assert bool(((ref == got) | (ref.isnan() & got.isnan())).all())
+    for code, value in ((0x38, 1.0), (0x7e, 448.0), (0x08, 2.0 ** -6), (0x01, 2.0 ** -9), (0x07, 7 * 2.0 ** -9), (0xb8, -1.0), (0x00, 0.0)):
+        assert lib.oracle_e4m3_decode(code) == value
+    # encode: exact values round-trip; midpoints between neighbours go to the even code; overflow saturates
+    finite = [c for c in range(0x7f)]
+    for c in finite:
+        assert lib.oracle_e4m3_encode(lib.oracle_e4m3_decode(c)) == c
+        assert lib.oracle_e4m3_encode(-lib.oracle_e4m3_decode(c)) == (c | 0x80)
+    for c in range(0x7e):
+        mid = 0.5 * (lib.oracle_e4m3_decode(c) + lib.oracle_e4m3_decode(c + 1))      # exactly representable in fp32
+        assert lib.oracle_e4m3_encode(mid) == (c if c % 2 == 0 else c + 1), c
+        assert lib.oracle_e4m3_encode(float(torch.nextafter(torch.tensor(mid), torch.tensor(1e9)))) == c + 1
+        assert lib.oracle_e4m3_encode(float(torch.nextafter(torch.tensor(mid), torch.tensor(-1e9)))) == c
+    for big in (448.0001, 464.0, 480.0, 1e6, 3e38):
+        assert lib.oracle_e4m3_encode(big) == 0x7e and lib.oracle_e4m3_encode(-big) == 0xfe
+    # the library's cast on random in-range values
+    g = torch.Generator().manual_seed(0)
+    x = (torch.randn(20000, generator=g) * torch.exp(torch.randn(20000, generator=g) * 3)).clamp(-448, 448)
+    want = x.to(torch.float8_e4m3fn).view(torch.uint8)
+    got = torch.tensor([lib.oracle_e4m3_encode(float(v)) for v in x.tolist()], dtype=torch.uint8)
+    assert torch.equal(want, got)
+
+
+def test_quantised_cache_attends_like_the_cache_of_its_dequantised_values():
+    """Reading a byte x as scale * x is exact, so a quantised cache must give what the fp32 cache holding those
+    products gives: the same relevance bit for bit, the same output up to the bf16 rounding of out."""
+    L, B, Hq, Hkv, D, cap, n = 2, 2, 8, 2, 16, 40, 33
+    ks, vs = [0.25, 0.5], [2.0, 0.125]                                  # powers of two: scale * x is exact in fp32 too
+    q8 = _fp8_cache(L, B, Hq, Hkv, D, cap, n, 3, ks, vs)
+    kf = q8.k.float() * torch.tensor(ks).reshape(L, 1, 1, 1, 1)
+    vf = q8.v.float() * torch.tensor(vs).reshape(L, 1, 1, 1, 1)
+    f32 = oracle.OracleCache(L, B, Hq, Hkv, D, cap, kf, vf, q8.rel.clone(), q8.pos.clone(), q8.len.clone())
+    g = torch.Generator().manual_seed(4)
+    q = (torch.randn((L, B, Hq, D), generator=g) * 0.3).to(torch.bfloat16)
+    scale = torch.tensor([0.2, 0.35], dtype=torch.float32)
+    st8, out8, lse8, _ = oracle.decode_attend(q8, 0, L, q, None, None, None, scale, 0.9, want_lse=True)
+    st32, out32, lse32, _ = oracle.decode_attend(f32, 0, L, q.float(), None, None, None, scale, 0.9, want_lse=True)
+    assert st8 == st32 == oracle.OK and out8.dtype == torch.bfloat16
+    assert torch.equal(q8.rel, f32.rel) and torch.equal(lse8, lse32)
+    assert (out8.float() - out32).abs().max() <= 2.0 ** -8 * out32.abs().max()
+    # non-trivial scales (not powers of two) against the double-precision definition
+    q8b = _fp8_cache(1, 1, 4, 1, 8, 12, 9, 5, [0.3], [1.7])
+    qq = (torch.randn((1, 1, 4, 8), generator=g) * 0.5).to(torch.bfloat16)
+    st, out, _, probs = oracle.decode_attend(q8b, 0, 1, qq, None, None, None, torch.tensor([0.4]), 1.0, want_probs=True)
+    kd = q8b.k.double()[0, 0, 0, :9] * float(torch.tensor(0.3, dtype=torch.float32))
+    vd = q8b.v.double()[0, 0, 0, :9] * float(torch.tensor(1.7, dtype=torch.float32))
+    p = torch.softmax((qq.double()[0, 0] @ kd.T) * float(torch.tensor(0.4, dtype=torch.float32)), dim=-1)
+    assert torch.allclose(probs[0, 0, :, :9], p, rtol=1e-12, atol=1e-15)
+    assert torch.allclose(out[0, 0].double(), p @ vd, rtol=2.0 ** -8, atol=1e-6)
+
+
+def test_quantised_append_rounds_like_the_library_and_saturates():
+    L, B, Hq, Hkv, D, cap, n = 1, 2, 4, 2, 32, 16, 5
+    ks, vs = [0.37], [3.0]
+    c = _fp8_cache(L, B, Hq, Hkv, D, cap, n, 6, ks, vs)
+    before = c.clone()
+    g = torch.Generator().manual_seed(8)
+    q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+    kn = (torch.randn((L, B, Hkv, D), generator=g) * 20).to(torch.bfloat16)
+    vn = (torch.randn((L, B, Hkv, D), generator=g) * 100).to(torch.bfloat16)
+    kn[0, 0, 0, :4] = torch.tensor([1e4, -1e4, 0.0, 165.76], dtype=torch.bfloat16)   # beyond 448 * 0.37: saturates
+    st, *_ = oracle.decode_attend(c, 0, L, q, kn, vn, torch.tensor([7, 9], dtype=torch.int32), torch.tensor([0.1]), 0.9)
+    assert st == oracle.OK and torch.all(c.len == n + 1)
+    tk = kn.float() / torch.tensor(ks[0], dtype=torch.float32)
+    tv = vn.float() / torch.tensor(vs[0], dtype=torch.float32)
+    want_k = tk.clamp(-448, 448).to(torch.float8_e4m3fn).view(torch.uint8)      # the library rounds, the clamp saturates
+    want_v = tv.clamp(-448, 448).to(torch.float8_e4m3fn).view(torch.uint8)
+    assert torch.equal(c.k.view(torch.uint8)[0, :, :, n], want_k[0]) and torch.equal(c.v.view(torch.uint8)[0, :, :, n], want_v[0])
+    assert c.k.view(torch.uint8)[0, 0, 0, n, 0] == 0x7e and c.k.view(torch.uint8)[0, 0, 0, n, 1] == 0xfe
+    assert torch.equal(c.k.view(torch.uint8)[..., :n, :], before.k.view(torch.uint8)[..., :n, :])
+    assert torch.equal(c.pos[0, :, :, n], torch.tensor([[7, 7], [9, 9]], dtype=torch.int32))
+
+
+def test_quantised_cache_prunes_by_moving_bytes():
+    c = _fp8_cache(2, 2, 4, 2, 16, 64, 50, 9, [1.0, 1.0], [1.0, 1.0])
+    before = c.clone()
+    st, keep = oracle.rasr_prune(c, torch.tensor([[20, 60], [33, 12]], dtype=torch.int32), 8, 2, max_k=64)
+    assert st == oracle.OK
+    for l in range(2):
+        for b in range(2):
+            for h in range(2):
+                m = int(c.len[l, b, h])
+                idx = keep[l, b, h, :m].long()
+                assert torch.equal(c.k.view(torch.uint8)[l, b, h, :m], before.k.view(torch.uint8)[l, b, h, idx])
+                assert torch.equal(c.v.view(torch.uint8)[l, b, h, :m], before.v.view(torch.uint8)[l, b, h, idx])
+                assert torch.equal(c.rel[l, b, h, :m], before.rel[l, b, h, idx])
+    assert c.len[0, 0].tolist() == [20, 20] and c.len[0, 1].tolist() == [50, 50]
