@@ -66,14 +66,15 @@ typedef enum {
     LETHE_ERR_TOO_LARGE = 8    /* lethe_rasr_prune_static: the cache exceeds LETHE_STATIC_PRUNE_MAX_ENTRIES */
 } lethe_status;
 
-enum { LETHE_F32 = 0, LETHE_BF16 = 1 };
+enum { LETHE_F32 = 0, LETHE_BF16 = 1, LETHE_FP8_E4M3 = 2 };
 enum { LETHE_CONTIG = 0, LETHE_PAGED = 1 };
 
 /* Cache state of all layers (Sec. 4.1: per-layer K, V; Sec. 4.3: the score vector s_t). */
 typedef struct {
     int32_t n_layers, batch, n_q_heads, n_kv_heads;
     int32_t head_dim;    /* 64 or 128 */
-    int32_t dtype;       /* LETHE_F32 or LETHE_BF16: type of k, v, q, k_new, v_new, out */
+    int32_t dtype;       /* LETHE_F32 or LETHE_BF16: type of k, v, q, k_new, v_new, out.  LETHE_FP8_E4M3: k and v are
+                            e4m3 bytes (see k_scale), q, k_new, v_new, out are bf16 */
     int32_t layout;      /* LETHE_CONTIG or LETHE_PAGED */
     int32_t capacity;    /* CONTIG: token slots per item.  PAGED: page-table entries per item */
     int32_t page_tokens; /* PAGED: tokens per page (16); CONTIG: ignored */
@@ -83,8 +84,18 @@ typedef struct {
     int32_t *len;        /* [L][B][Hkv]              retained tokens per item                           */
     int32_t *page_table; /* PAGED: [L][B][Hkv][capacity] page ids (never written by the library)       */
     int64_t n_pages;     /* PAGED: pages in each pool                                                    */
+    const float *k_scale; /* LETHE_FP8_E4M3 only: HOST float[L] or NULL (= 1): a stored key byte x means k_scale[l] * x */
+    const float *v_scale; /* the same for values                                                                      */
 } lethe_cache;
-/* cap_tokens = capacity (CONTIG) or capacity * page_tokens (PAGED).  k, v and rel must be 16-byte aligned. */
+/* cap_tokens = capacity (CONTIG) or capacity * page_tokens (PAGED).  k, v and rel must be 16-byte aligned.
+ *
+ * Quantised caches (LETHE_FP8_E4M3).  The paper's related work notes that quantised caches compose with eviction
+ * and fixes no format; this library's is: e4m3 bytes (1-4-3, bias 7, no infinities, largest value 448) with one
+ * positive scale per layer for keys and one for values.  lethe_decode_attend appends k_new / k_scale[l] and
+ * v_new / v_scale[l] (fp32 division, round to nearest even, saturating at +-448) and reads a byte x as exactly
+ * scale * x; the prune calls move rows as bytes and never look at the storage type.  Supported: head_dim 64 or
+ * 128, up to 8 query heads per KV head, contiguous or 16-token pages; lethe_prefill_seed is not (prompt keys are
+ * scored before they are quantised). */
 
 /* Create a context on CUDA device `device`.  scratch_bytes_hint (0 = default) sizes the
  * device scratch the calls may use; it grows on demand (growth synchronises the device).

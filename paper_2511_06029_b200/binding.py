@@ -17,7 +17,7 @@ LIB_PATH = os.environ.get("LETHE_LIB", os.path.join(_HERE, "liblethe.so"))   # L
 
 OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_BUDGET, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED, ERR_PAGE, ERR_TOO_LARGE = range(9)
 STATIC_PRUNE_MAX_ENTRIES = 4 * 1024 * 1024
-F32, BF16 = 0, 1
+F32, BF16, FP8_E4M3 = 0, 1, 2
 CONTIG, PAGED = 0, 1
 VARIANT_AUTO, VARIANT_SIMT, VARIANT_MMA4, VARIANT_MMA8 = 0, 1, 2, 3
 
@@ -40,6 +40,7 @@ class lethe_cache(ctypes.Structure):
         ("layout", ctypes.c_int32), ("capacity", ctypes.c_int32), ("page_tokens", ctypes.c_int32),
         ("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("rel", ctypes.c_void_p), ("pos", ctypes.c_void_p),
         ("len", ctypes.c_void_p), ("page_table", ctypes.c_void_p), ("n_pages", ctypes.c_int64),
+        ("k_scale", ctypes.c_void_p), ("v_scale", ctypes.c_void_p),
     ]
 
 
@@ -102,13 +103,14 @@ class Cache:
     """Device tensors of the cache plus the C descriptor that points at them (the tensors stay owned here)."""
 
     def __init__(self, n_q_heads: int, k: torch.Tensor, v: torch.Tensor, rel: torch.Tensor, pos: torch.Tensor,
-                 len_: torch.Tensor, page_table: Optional[torch.Tensor] = None):
+                 len_: torch.Tensor, page_table: Optional[torch.Tensor] = None, k_scale=None, v_scale=None):
+        """k_scale, v_scale: per-layer scales of a float8_e4m3fn cache (sequences of L floats; None = 1)."""
         self.k, self.v, self.rel, self.pos, self.len, self.page_table = k, v, rel, pos, len_, page_table
         for t in (k, v, rel, pos, len_) + ((page_table,) if page_table is not None else ()):
             assert t.is_cuda and t.is_contiguous()
         assert rel.dtype == torch.float32 and pos.dtype == torch.int32 and len_.dtype == torch.int32
         L, B, Hkv = len_.shape
-        dt = {torch.float32: F32, torch.bfloat16: BF16}[k.dtype]
+        dt = {torch.float32: F32, torch.bfloat16: BF16, torch.float8_e4m3fn: FP8_E4M3}[k.dtype]
         if page_table is None:
             assert k.dim() == 5 and tuple(k.shape[:3]) == (L, B, Hkv)
             cap, D, layout, pt, npages = k.shape[3], k.shape[4], CONTIG, 0, 0
@@ -122,7 +124,25 @@ class Cache:
         self.capacity, self.page_tokens = cap, pt
         self.c = lethe_cache(L, B, n_q_heads, Hkv, D, dt, layout, cap, pt, k.data_ptr(), v.data_ptr(),
                              rel.data_ptr(), pos.data_ptr(), len_.data_ptr(),
-                             page_table.data_ptr() if page_table is not None else None, npages)
+                             page_table.data_ptr() if page_table is not None else None, npages, None, None)
+        # host arrays of the per-layer scales, kept alive here
+        self._k_scale = self._v_scale = None
+        if dt == FP8_E4M3:
+            for name, sc in (("k_scale", k_scale), ("v_scale", v_scale)):
+                if sc is None:
+                    continue
+                vals = [float(x) for x in (sc.tolist() if isinstance(sc, torch.Tensor) else sc)]
+                assert len(vals) == L
+                arr = (ctypes.c_float * L)(*vals)
+                setattr(self, "_" + name, arr)
+                setattr(self.c, name, ctypes.cast(arr, ctypes.c_void_p))
+        else:
+            assert k_scale is None and v_scale is None, "scales belong to quantised caches"
+
+    @property
+    def act_dtype(self) -> torch.dtype:
+        """Type of q, k_new, v_new and out."""
+        return torch.bfloat16 if self.k.dtype == torch.float8_e4m3fn else self.k.dtype
 
     @property
     def device(self):

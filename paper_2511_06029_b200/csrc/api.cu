@@ -10,6 +10,8 @@
 
 namespace lethe {
 cudaError_t launch_attend_simt(const AttendArgs& a, int dtype, int D, bool paged, cudaStream_t stream);
+size_t kv8_smem_bytes(int D, int shape, int chunk_tokens, int GP);
+cudaError_t launch_attend_kv8(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream);
 size_t simt_smem_bytes(int D, int chunk_tokens, int GP);
 cudaError_t launch_attend_mma(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream);
 size_t mma_smem_bytes(int D, int shape, int chunk_tokens, int GP);
@@ -144,7 +146,13 @@ lethe_status check_cache(lethe_ctx* ctx, const lethe_cache* c) {
         return fail(ctx, LETHE_ERR_INVALID_ARG, "cache dimensions must be positive");
     if (c->n_q_heads % c->n_kv_heads) return fail(ctx, LETHE_ERR_INVALID_ARG, "n_q_heads must be a multiple of n_kv_heads");
     if (c->head_dim != 64 && c->head_dim != 128) return fail(ctx, LETHE_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
-    if (c->dtype != LETHE_F32 && c->dtype != LETHE_BF16) return fail(ctx, LETHE_ERR_INVALID_ARG, "unknown dtype");
+    if (c->dtype != LETHE_F32 && c->dtype != LETHE_BF16 && c->dtype != LETHE_FP8_E4M3)
+        return fail(ctx, LETHE_ERR_INVALID_ARG, "unknown dtype");
+    if (c->dtype == LETHE_FP8_E4M3)
+        for (int l = 0; l < c->n_layers; ++l) {
+            const float ks = c->k_scale ? c->k_scale[l] : 1.f, vs = c->v_scale ? c->v_scale[l] : 1.f;
+            if (!(ks > 0.f && ks < 1e30f && vs > 0.f && vs < 1e30f)) return fail(ctx, LETHE_ERR_INVALID_ARG, "k_scale and v_scale must be positive and finite");
+        }
     if (c->layout != LETHE_CONTIG && c->layout != LETHE_PAGED) return fail(ctx, LETHE_ERR_INVALID_ARG, "unknown layout");
     if (c->capacity < 1) return fail(ctx, LETHE_ERR_INVALID_ARG, "capacity must be positive");
     if (c->layout == LETHE_PAGED) {
@@ -165,7 +173,7 @@ CacheView view_of(const lethe_cache* c) {
     v.k = c->k; v.v = c->v; v.rel = c->rel; v.pos = c->pos; v.len = c->len; v.page_table = c->page_table;
     v.n_pages = c->n_pages;
     v.L = c->n_layers; v.B = c->batch; v.Hkv = c->n_kv_heads; v.D = c->head_dim;
-    v.elt_bytes = c->dtype == LETHE_BF16 ? 2 : 4;
+    v.elt_bytes = c->dtype == LETHE_BF16 ? 2 : (c->dtype == LETHE_FP8_E4M3 ? 1 : 4);
     v.capacity = c->capacity; v.cap_tokens = cap_tokens_of(c);
     v.page_tokens = c->layout == LETHE_PAGED ? c->page_tokens : 1;
     v.paged = c->layout == LETHE_PAGED;
@@ -332,6 +340,35 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
     const bool mma_ok = c->dtype == LETHE_BF16 && (!paged || c->page_tokens == kGroupTokens);
     const int cap_groups = (a.cap_tokens + kGroupTokens - 1) / kGroupTokens;
     int variant = ctx->variant;
+
+    if (c->dtype == LETHE_FP8_E4M3) {
+        // quantised cache: its own clustered tensor-core kernel; variants 2..7 pick its shape, the rest mean "default"
+        if (paged && c->page_tokens != kGroupTokens) return fail(ctx, LETHE_ERR_UNSUPPORTED, "quantised caches need 16-token pages");
+        if (c->n_layers > kMaxLayers) return fail(ctx, LETHE_ERR_UNSUPPORTED, "more than 128 layers");
+        for (int l = 0; l < c->n_layers; ++l) {
+            a.k_scale[l] = c->k_scale ? c->k_scale[l] : 1.f;
+            a.v_scale[l] = c->v_scale ? c->v_scale[l] : 1.f;
+            a.scale_log2[l] = scale[l] * a.k_scale[l] * 1.4426950408889634f;
+        }
+        const int shape = (variant >= 2 && variant <= 7) ? variant - 2 : 1;
+        auto smem_for = [&](int S) -> size_t {
+            const int chunk = ((cap_groups + S - 1) / S) * kGroupTokens;
+            return kv8_smem_bytes(c->head_dim, shape, chunk, a.GP);
+        };
+        int S = ctx->splits;
+        if (S == 0) {
+            S = 1;
+            while (S < 16 && smem_for(S) > ctx->max_smem) S *= 2;
+            while (S < 8 && (long long)a.n_items * S < ctx->sm_count && cap_groups / (2 * S) >= 4) S *= 2;
+        }
+        if (smem_for(S) > ctx->max_smem)
+            return fail(ctx, LETHE_ERR_UNSUPPORTED, "capacity too large for the on-chip logit buffer at this split count");
+        a.splits = S;
+        a.chunk_tokens = ((cap_groups + S - 1) / S) * kGroupTokens;
+        const cudaError_t e8 = launch_attend_kv8(a, c->head_dim, shape, paged, (cudaStream_t)stream);
+        if (e8 != cudaSuccess) return cuda_fail(ctx, e8, "decode_attend launch (quantised cache)");
+        return LETHE_OK;
+    }
     // persistent kernel: logit-buffer tokens that fit beside a shape's stages (the rest overflows to scratch)
     auto stream_chunk = [&](int shape) -> int {
         const size_t fixed = stream_smem_bytes(c->head_dim, shape, 0, a.GP);
@@ -483,7 +520,7 @@ lethe_status lethe_decode_attend_host(lethe_ctx* ctx, const lethe_cache* c, int 
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, LETHE_ERR_CUDA, "cannot select the context's device");
     const size_t nl = (size_t)(layer_end - layer_begin);
-    const size_t eb = c->dtype == LETHE_BF16 ? 2 : 4;
+    const size_t eb = c->dtype == LETHE_F32 ? 4 : 2;  // activations: fp32 with an fp32 cache, bf16 otherwise
     auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
     const size_t q_bytes = nl * c->batch * c->n_q_heads * c->head_dim * eb;
     const size_t kv_bytes = nl * c->batch * c->n_kv_heads * c->head_dim * eb;

@@ -51,7 +51,9 @@ struct AttendArgs {
 #ifdef LETHE_TIMELINE
     unsigned long long* timeline;  // debug builds only: 8 timestamps per CTA
 #endif
-    float scale_log2[kMaxLayers];  // scale[l] * log2(e), by absolute layer
+    float scale_log2[kMaxLayers];  // scale[l] * log2(e) (times the key scale for a quantised cache), by absolute layer
+    float k_scale[kMaxLayers];     // quantised caches: a stored key byte x means k_scale[l] * x (else unused)
+    float v_scale[kMaxLayers];     // the same for values
 };
 
 #ifdef LETHE_TIMELINE

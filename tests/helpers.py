@@ -55,17 +55,21 @@ def to_device(oc):
     from paper_2511_06029_b200 import binding
     dev = torch.device("cuda", 0)
     pt = None if oc.page_table is None else oc.page_table.to(dev)
-    return binding.Cache(oc.n_q_heads, oc.k.to(dev), oc.v.to(dev), oc.rel.to(dev), oc.pos.to(dev), oc.len.to(dev), pt)
+    return binding.Cache(oc.n_q_heads, oc.k.to(dev), oc.v.to(dev), oc.rel.to(dev), oc.pos.to(dev), oc.len.to(dev), pt,
+                         k_scale=oc.k_scale, v_scale=oc.v_scale)
 
 
 def sync_state(gc, oc):
     """Overwrite the GPU cache state with the oracle's (call-by-call parity: identical inputs for the next call)."""
-    gc.k.copy_(oc.k); gc.v.copy_(oc.v); gc.rel.copy_(oc.rel); gc.pos.copy_(oc.pos); gc.len.copy_(oc.len)
+    gc.k.view(torch.uint8).copy_(oc.k.view(torch.uint8)); gc.v.view(torch.uint8).copy_(oc.v.view(torch.uint8))
+    gc.rel.copy_(oc.rel); gc.pos.copy_(oc.pos); gc.len.copy_(oc.len)
 
 
 def logical_rows(k, v, rel, pos, ln, page_table=None, page_tokens=0):
     """Per item (K rows, V rows, rel, pos) of the first len slots, as CPU tensors, for either layout."""
     k, v, rel, pos, ln = k.cpu(), v.cpu(), rel.cpu(), pos.cpu(), ln.cpu()
+    if k.dtype == torch.float8_e4m3fn:                 # compare quantised rows as the bytes they are
+        k, v = k.view(torch.uint8), v.view(torch.uint8)
     L, B, H = ln.shape
     out = []
     for l in range(L):

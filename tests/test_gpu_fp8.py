@@ -1,0 +1,161 @@
+"""GPU parity of the quantised-cache path (K / V as e4m3 bytes with per-layer scales, bf16 activations) against the
+oracle: appended rows are quantised to the same bytes, outputs within 2e-2, relevance within 1e-3 relative, and the
+prune round moves the bytes exactly as the oracle does."""
+import pytest
+import torch
+
+import oracle
+from helpers import assert_state_matches, gpu_context, oracle_prune_round, sync_state, to_device
+from paper_2511_06029_b200 import binding, synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = gpu_context()
+    yield c
+    c.close()
+
+
+def fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed, k_scale=None, v_scale=None, page_tokens=0):
+    """Quantised cache drawn as the quantisation of Gaussian K / V (a few keys enlarged, as the workloads' anchors)."""
+    g = torch.Generator().manual_seed(seed)
+    ks = torch.tensor(k_scale if k_scale is not None else [1.0] * L, dtype=torch.float32)
+    vs = torch.tensor(v_scale if v_scale is not None else [1.0] * L, dtype=torch.float32)
+    k = torch.randn((L, B, Hkv, cap, D), generator=g)
+    k[:, :, :, ::17] *= 3.0
+    v = torch.randn((L, B, Hkv, cap, D), generator=g)
+    k8 = (k / ks.reshape(L, 1, 1, 1, 1)).clamp(-448, 448).to(torch.float8_e4m3fn)
+    v8 = (v / vs.reshape(L, 1, 1, 1, 1)).clamp(-448, 448).to(torch.float8_e4m3fn)
+    rel = torch.rand((L, B, Hkv, cap), generator=g)
+    pos = torch.arange(cap, dtype=torch.int32).expand(L, B, Hkv, cap).contiguous()
+    ln = torch.full((L, B, Hkv), lens, dtype=torch.int32) if isinstance(lens, int) else lens.to(torch.int32).contiguous()
+    if page_tokens:
+        assert cap % page_tokens == 0
+        pages_per_item = cap // page_tokens
+        n_pages = L * B * Hkv * pages_per_item + 3
+        perm = torch.randperm(n_pages, generator=g)[:L * B * Hkv * pages_per_item].to(torch.int32)
+        table = perm.reshape(L, B, Hkv, pages_per_item).contiguous()
+        pool_k = torch.zeros((n_pages, page_tokens, D), dtype=torch.uint8)
+        pool_v = torch.zeros((n_pages, page_tokens, D), dtype=torch.uint8)
+        pool_k[table.long().flatten()] = k8.view(torch.uint8).reshape(-1, page_tokens, D)
+        pool_v[table.long().flatten()] = v8.view(torch.uint8).reshape(-1, page_tokens, D)
+        return oracle.OracleCache(L, B, Hq, Hkv, D, pages_per_item, pool_k.view(torch.float8_e4m3fn), pool_v.view(torch.float8_e4m3fn),
+                                  rel, pos, ln, page_tokens, table, k_scale=ks, v_scale=vs)
+    return oracle.OracleCache(L, B, Hq, Hkv, D, cap, k8, v8, rel, pos, ln, k_scale=ks, v_scale=vs)
+
+
+def _step(ctx, oc, gc, q, kn, vn, tp, scale, gamma, want_lse=False):
+    L = oc.n_layers
+    st, ref, lse_ref, _ = oracle.decode_attend(oc, 0, L, q, kn, vn, tp, scale, gamma, want_lse=want_lse)
+    dev = gc.device
+    out = torch.empty_like(q, device=dev)
+    lse = torch.empty((L, oc.batch, oc.n_q_heads), dtype=torch.float32, device=dev) if want_lse else None
+    ctx.decode_attend(gc, 0, L, q.to(dev), None if kn is None else kn.to(dev), None if vn is None else vn.to(dev),
+                      None if tp is None else tp.to(dev), scale.tolist(), gamma, out, lse)
+    assert st == oracle.OK and ctx.poll_status()[0] == 0
+    # 2e-2 absolute for outputs of the usual size; outputs made large by a saturated value row (up to 448 * scale)
+    # carry the bf16 rounding of their own magnitude (2^-8 relative)
+    d = (out.cpu().float() - ref.float()).abs()
+    assert bool((d <= 2e-2 + 2.0 ** -7 * ref.float().abs()).all()), f"attention output error {d.max().item()}"
+    if want_lse:
+        assert torch.allclose(lse.cpu(), lse_ref, rtol=1e-4, atol=1e-4)
+    assert_state_matches(gc, oc)           # appended bytes, pos, len bit-exact; rel within 1e-3
+
+
+@pytest.mark.parametrize("paged", [False, True])
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 128), (7, 1, 128), (4, 4, 64), (16, 2, 64), (6, 2, 128)])
+def test_quantised_decode_parity(ctx, Hq, Hkv, D, paged):
+    """Ragged lengths over several 16-token groups and tails, attend-only and appending steps, scales that are not
+    powers of two, a new token beyond the representable range (saturates)."""
+    L, B, cap = 2, 3, 208
+    g = torch.Generator().manual_seed(Hq * 10 + D)
+    lens = torch.randint(1, cap - 8, (L, B, Hkv), generator=g)
+    lens.view(-1)[:4] = torch.tensor([1, 15, 16, 17])[: min(4, lens.numel())]
+    oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=Hq + D, k_scale=[0.37, 1.5], v_scale=[2.25, 0.6],
+                   page_tokens=16 if paged else 0)
+    gc = to_device(oc)
+    scale = torch.tensor([0.11, 0.07], dtype=torch.float32) * (128 / D) ** 0.5
+    for step in range(5):
+        q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+        if step == 1:
+            _step(ctx, oc, gc, q, None, None, None, scale, 0.95, want_lse=True)
+            continue
+        kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+        vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+        if step == 2:
+            kn[0, 0, 0, :3] = torch.tensor([1e4, -1e4, 165.5], dtype=torch.bfloat16)
+            vn[1, 1, 0, :2] = torch.tensor([-3e3, 269.0], dtype=torch.bfloat16)
+        _step(ctx, oc, gc, q, kn, vn, torch.arange(B, dtype=torch.int32) + 300 + step, scale, 0.95)
+
+
+@pytest.mark.parametrize("variant,splits", [(2, 1), (3, 2), (4, 4), (5, 1), (6, 8), (7, 2), (0, 0)])
+def test_quantised_decode_shapes_and_clusters(ctx, variant, splits):
+    """Every kernel shape and cluster size on items long enough to give every CTA of a cluster several groups."""
+    L, B, Hq, Hkv, D, cap = 1, 2, 8, 2, 128, 1100
+    g = torch.Generator().manual_seed(variant * 7 + splits)
+    lens = torch.tensor([[[1037, 700], [513, 1090]]])
+    oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=variant, k_scale=[0.8], v_scale=[1.25])
+    gc = to_device(oc)
+    ctx.set_tuning(variant, splits)
+    try:
+        scale = torch.tensor([0.09], dtype=torch.float32)
+        for step in range(2):
+            q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+            kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            _step(ctx, oc, gc, q, kn, vn, torch.tensor([5, 6], dtype=torch.int32), scale, 0.99)
+    finally:
+        ctx.set_tuning(0, 0)
+
+
+def test_quantised_trajectory_with_prune_rounds(ctx):
+    """Llama-8B-shaped geometry (2 layers, 2 sequences): decode steps with appends, a prune round every 6 steps on
+    the oracle's scores; bytes, positions and lengths stay identical throughout."""
+    oracle.set_threads(min(8, oracle.max_threads()))
+    try:
+        w = synth.shrink(synth.WORKLOADS["llama8b"], n_layers=2, batch=2)
+        L, B, Hq, Hkv, D, cap, n0 = 2, 2, w.n_q_heads, w.n_kv_heads, w.head_dim, 320, 270
+        oc = fp8_cache(L, B, Hq, Hkv, D, cap, n0, seed=21, k_scale=[0.5, 0.7], v_scale=[0.9, 1.1])
+        oc.rel.zero_()
+        gc = to_device(oc)
+        dev = gc.device
+        scale = synth.layer_scales(w)
+        T = torch.full((B,), L * 200, dtype=torch.int64)
+        S = torch.zeros((L, B), dtype=torch.float32, device=dev)
+        bud = torch.zeros((L, B), dtype=torch.int32, device=dev)
+        keep = torch.zeros((L, B, Hkv, cap), dtype=torch.int32, device=dev)
+        for step in range(18):
+            x = synth.step_inputs(w, step)
+            _step(ctx, oc, gc, x["q"], x["k_new"], x["v_new"], x["token_pos"], scale, w.gamma)
+            if step % 6 == 5:
+                sync_state(gc, oc)                                   # selection on the oracle's fp32 scores
+                st, S_o, bud_o, keep_o = oracle_prune_round(oc, T, w.k_min, w.recent, w.sink, max_k=cap)
+                assert st == oracle.OK
+                ctx.estimate_sparsity(gc, S); ctx.alloc_budgets(S, T.to(dev), w.k_min, bud)
+                ctx.rasr_prune(gc, bud, w.recent, w.sink, keep)
+                assert ctx.poll_status()[0] == 0
+                assert torch.equal(bud.cpu(), bud_o) and torch.equal(keep.cpu(), keep_o)
+                assert_state_matches(gc, oc, exact_rel=True)
+        assert int(oc.len.sum()) <= B * Hkv * (L * 200 + L * 6)          # every sequence was cut back to its total budget
+    finally:
+        oracle.set_threads(1)
+
+
+def test_quantised_cache_limits(ctx):
+    oc = fp8_cache(1, 1, 4, 1, 64, 32, 32, seed=1)
+    gc = to_device(oc)
+    q = torch.zeros((1, 1, 4, 64), dtype=torch.bfloat16, device="cuda")
+    kn = torch.zeros((1, 1, 1, 64), dtype=torch.bfloat16, device="cuda")
+    out = torch.empty_like(q)
+    ctx.decode_attend(gc, 0, 1, q, kn, kn, torch.zeros(1, dtype=torch.int32, device="cuda"), [0.1], 0.9, out)
+    st, item = ctx.poll_status()
+    assert st == binding.ERR_CAPACITY and item == 0 and int(gc.len[0, 0, 0]) == 32        # full: untouched, reported
+    with pytest.raises(binding.LetheError) as e:                                          # prompt seeding: bf16 caches only
+        ctx.prefill_seed(gc, torch.zeros((1, 1, 8, 4, 64), dtype=torch.bfloat16, device="cuda"), [0.1], 0.9)
+    assert e.value.status == binding.ERR_UNSUPPORTED
+    bad = binding.Cache(4, gc.k, gc.v, gc.rel, gc.pos, gc.len, k_scale=[0.0], v_scale=[1.0])
+    with pytest.raises(binding.LetheError) as e:
+        ctx.decode_attend(bad, 0, 1, q, None, None, None, [0.1], 0.9, out)
+    assert e.value.status == binding.ERR_INVALID_ARG
