@@ -40,8 +40,9 @@ def test_binding_prototypes_and_no_gpu_behaviour():
 
 def test_struct_layout_matches_header():
     """The ctypes mirror of lethe_cache has the field order and size the header implies (9 int32, pad, 6 pointers,
-    one int64 on LP64)."""
+    one int64, 2 pointers on LP64)."""
     assert [f[0] for f in binding.lethe_cache._fields_] == [
         "n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "dtype", "layout", "capacity", "page_tokens",
-        "k", "v", "rel", "pos", "len", "page_table", "n_pages"]
-    assert ctypes.sizeof(binding.lethe_cache) == 40 + 6 * 8 + 8
+        "k", "v", "rel", "pos", "len", "page_table", "n_pages", "k_scale", "v_scale"]
+    assert ctypes.sizeof(binding.lethe_cache) == 40 + 6 * 8 + 8 + 2 * 8
+    assert (binding.F32, binding.BF16, binding.FP8_E4M3) == (0, 1, 2)
