@@ -118,13 +118,19 @@ def make_state(w, device, capacity, n0, seed):
 class Runner:
     """The decode / prune loop around the C ABI (host logic of the harness: when to prune)."""
 
-    def __init__(self, w, device, rank, capacity, variant, splits, pool=8):
+    def __init__(self, w, device, rank, capacity, variant, splits, pool=8, kv="bf16"):
         from paper_2511_06029_b200 import binding
         self.w, self.dev, self.binding = w, device, binding
         self.ctx = binding.Context(device.index)
         self.ctx.set_tuning(variant, splits)
         k, v, rel, pos, ln = make_state(w, device, capacity, w.mean_budget, 1234 + 77 * rank)
-        self.cache = binding.Cache(w.n_q_heads, k, v, rel, pos, ln)
+        if kv == "fp8":   # quantised cache: e4m3 bytes, one scale per layer (anchor keys reach about 3 x 4 sigma)
+            ks, vs = [0.125] * w.n_layers, [0.0625] * w.n_layers
+            k = (k.float() / ks[0]).clamp(-448, 448).to(torch.float8_e4m3fn)
+            v = (v.float() / vs[0]).clamp(-448, 448).to(torch.float8_e4m3fn)
+            self.cache = binding.Cache(w.n_q_heads, k, v, rel, pos, ln, k_scale=ks, v_scale=vs)
+        else:
+            self.cache = binding.Cache(w.n_q_heads, k, v, rel, pos, ln)
         self.scale = synth.layer_scales(w).tolist()
         self.scale_c = self.ctx._scale(self.scale)
         L, B = w.n_layers, w.batch
@@ -349,6 +355,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-per-layer", action="store_true")
+    ap.add_argument("--kv", choices=["bf16", "fp8"], default="bf16",
+                    help="storage of K and V: bf16 (the headline configuration) or e4m3 bytes with per-layer scales")
     ap.add_argument("--with-prefill", action="store_true",
                     help="also time lethe_prefill_seed on a prompt of the workload's length (informational)")
     ap.add_argument("--pl-variant", type=int, default=0, help="kernel variant of the per-layer launch mode")
@@ -379,11 +387,14 @@ def main():
     if dist is not None:
         dist.barrier()
 
+    # algorithmic bytes per token-head: K row + V row + relevance read and write (rows are D bytes when quantised)
+    bytes_per_th = BYTES_PER_TOKEN_HEAD if args.kv == "bf16" else 2 * w.head_dim + 8
+
     def prepare(capacity):
         """Runner brought to steady state (untimed): a few full prune intervals so that relevance, sparsity-driven
         budgets and lengths are those of a long trajectory (dense layers need several rounds to grow to their
         budget).  Returns the runner and the largest layer budget."""
-        r = Runner(w, dev, rank, capacity, args.variant, args.splits)
+        r = Runner(w, dev, rank, capacity, args.variant, args.splits, kv=args.kv)
         for _ in range(max(1, args.prep_rounds)):
             for _ in range(w.prune_interval):
                 r.decode()
@@ -437,7 +448,7 @@ def main():
         r.ctx.set_tuning(args.variant, args.splits)
         r.check()
         per_layer = {"ms_per_step": ms_pl, "token_heads_per_step": th_pl, "value": th_pl / (ms_pl * 1e-3),
-                     "algorithmic_GBs": th_pl * BYTES_PER_TOKEN_HEAD / (ms_pl * 1e-3) / 1e9,
+                     "algorithmic_GBs": th_pl * bytes_per_th / (ms_pl * 1e-3) / 1e9,
                      "mode": f"{w.n_layers} launches per step (one per layer), replayed from a CUDA graph, "
                              f"{pl_steps} steps; not part of `value`"}
 
@@ -527,14 +538,16 @@ def main():
         peak, which = measured_peak()
         th_per_launch = sum(th) / len(th)
         avg_attend_ms = sum(attend_ms) / len(attend_ms)
-        achieved = th_per_launch * BYTES_PER_TOKEN_HEAD / (avg_attend_ms * 1e-3) / 1e9
+        achieved = th_per_launch * bytes_per_th / (avg_attend_ms * 1e-3) / 1e9
         wq = w
         h2d = (wq.n_layers * wq.batch * (wq.n_q_heads + 2 * wq.n_kv_heads) * wq.head_dim * 2 + wq.batch * 4)
         d2h = wq.n_layers * wq.batch * wq.n_q_heads * wq.head_dim * 2
         line = {
             "metric": METRIC, "value": dist_util.job_value(units, t_ms), "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": t_ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if args.kv == "bf16" else "fp8 K/V (e4m3 bytes, per-layer scales), bf16 activations, f16 mma, fp32 accumulation",
+            "data": "synthetic",
             "config": workload_config(w, args, extra={
                 "capacity": capacity, "variant": args.variant, "splits": args.splits,
                 "launch_mode": "all layers in one lethe_decode_attend call per step",
@@ -551,7 +564,7 @@ def main():
                          "peak_source": f"of {which}", "frac_of_8TBs_nominal": achieved / 8000.0,
                          "kernel": "attend (dominant kernel; one launch per step)",
                          "traffic": (NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD * th_per_launch
-                                     if NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD else None)},
+                                     if (NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD and args.kv == "bf16") else None)},
             "gpu_launches": launches, "clocks": clocks,
         }
         if not args.no_e2e:

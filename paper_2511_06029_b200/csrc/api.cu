@@ -350,7 +350,7 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
             a.v_scale[l] = c->v_scale ? c->v_scale[l] : 1.f;
             a.scale_log2[l] = scale[l] * a.k_scale[l] * 1.4426950408889634f;
         }
-        const int shape = (variant >= 2 && variant <= 7) ? variant - 2 : 1;
+        const int shape = (variant >= 2 && variant <= 7) ? variant - 2 : 0;
         auto smem_for = [&](int S) -> size_t {
             const int chunk = ((cap_groups + S - 1) / S) * kGroupTokens;
             return kv8_smem_bytes(c->head_dim, shape, chunk, a.GP);

@@ -333,7 +333,7 @@ static cudaError_t launch_kv8_t(const AttendArgs& a, cudaStream_t stream) {
 
 // Kernel shapes (warps per CTA, pipeline stages per warp), selected by `shape`: tiles are half the size of the bf16
 // kernel's, so the pipelines are deeper.
-#define LETHE_KV8_SHAPES(X, D) X(0, D, 4, 4) X(1, D, 8, 4) X(2, D, 4, 6) X(3, D, 8, 6) X(4, D, 2, 8) X(5, D, 16, 2)
+#define LETHE_KV8_SHAPES(X, D) X(0, D, 4, 4) X(1, D, 8, 4) X(2, D, 4, 2) X(3, D, 4, 3) X(4, D, 2, 4) X(5, D, 8, 2)
 
 size_t kv8_smem_bytes(int D, int shape, int chunk_tokens, int GP) {
 #define X(id, DD, NW, NS) \
