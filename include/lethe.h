@@ -121,6 +121,9 @@ lethe_status lethe_poll_status(lethe_ctx *ctx, void *stream, int32_t *info);
  * 32..37 = the clustered kernel's six shapes with the CTAs of an item merged through global scratch (the last
  * CTA to finish completes the item) instead of a thread-block cluster; splits may then be any value 0..16.
  * Tensor-core variants need a bf16 cache (and 16-token pages when paged).
+ * A quantised cache (LETHE_FP8_E4M3) always runs its own clustered tensor-core kernel: variants 2..7 then select
+ * its shape (4,4) (8,4) (4,2) (4,3) (2,4) (8,2), any other value the default (4,4); splits as for the clustered
+ * kernel.
  * variant 40..42 select the engine of lethe_prefill_seed and leave everything else as it is: 40 = tcgen05
  * kernels (accumulators in tensor memory; operand tiles by TMA for contiguous caches, by cp.async for paged
  * ones; the default), 41 = mma.sync kernels, 42 = tcgen05 kernels with cp.async tiles always; splits is ignored.
@@ -162,8 +165,11 @@ lethe_status lethe_decode_attend(lethe_ctx *ctx, const lethe_cache *cache, int l
  * The same step with HOST-resident per-step tensors: q, k_new, v_new, token_pos and
  * out (and lse if not NULL) are HOST pointers (pinned memory makes the copies
  * asynchronous).  The call copies the inputs to context-owned device staging, runs
- * lethe_decode_attend, and copies out (and lse) back, all on `stream`; the results are
- * valid in host memory once `stream` has been synchronised.  The cache stays on the device.
+ * lethe_decode_attend, and copies out (and lse) back; the results are valid in host memory
+ * once `stream` has been synchronised.  The cache stays on the device.  A call that covers
+ * many layers is cut into two chunks of layers whose uploads and downloads run on two
+ * context-owned streams under the kernel of the other chunk (the kernels stay on `stream`,
+ * which also waits for the last download); smaller calls do everything on `stream`.
  */
 lethe_status lethe_decode_attend_host(lethe_ctx *ctx, const lethe_cache *cache, int layer_begin, int layer_end,
                                       const void *q_host, const void *k_new_host, const void *v_new_host,

@@ -86,6 +86,10 @@ struct lethe_ctx {
     size_t flat_bytes;
     void* staging;  // device staging of lethe_decode_attend_host
     size_t staging_bytes;
+    // lethe_decode_attend_host: upload / download streams and the events that chain them to the caller's stream
+    cudaStream_t up_stream, down_stream;
+    cudaEvent_t ev_start, ev_up[8], ev_done[8], ev_down;
+    bool host_pipeline_ready;
     int variant, splits;
     int prefill_engine;  // 0 = tcgen05 kernels (TMA producers when the cache is contiguous), 1 = mma.sync kernels, 2 = tcgen05 with cp.async producers
     // TMA variant: tensor maps of the last cache seen (rebuilt when k, v, the row count or D change)
@@ -224,6 +228,16 @@ void lethe_destroy(lethe_ctx* ctx) {
     if (ctx->status) cudaFree(ctx->status);
     if (ctx->scratch) cudaFree(ctx->scratch);
     if (ctx->staging) cudaFree(ctx->staging);
+    if (ctx->host_pipeline_ready) {
+        cudaStreamDestroy(ctx->up_stream);
+        cudaStreamDestroy(ctx->down_stream);
+        cudaEventDestroy(ctx->ev_start);
+        cudaEventDestroy(ctx->ev_down);
+        for (int i = 0; i < 8; ++i) {
+            cudaEventDestroy(ctx->ev_up[i]);
+            cudaEventDestroy(ctx->ev_done[i]);
+        }
+    }
     if (ctx->order) cudaFree(ctx->order);
     if (ctx->flat) cudaFree(ctx->flat);
     delete ctx;
@@ -537,19 +551,82 @@ lethe_status lethe_decode_attend_host(lethe_ctx* ctx, const lethe_cache* c, int 
     int32_t* dpos = (int32_t*)p; p += up(pos_bytes);
     float* dlse = (float*)p;
     cudaStream_t s = (cudaStream_t)stream;
-    cudaError_t e = cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess && k_new_host) {
-        e = cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s);
-        if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s);
-        if (e == cudaSuccess) e = cudaMemcpyAsync(dpos, token_pos_host, pos_bytes, cudaMemcpyHostToDevice, s);
+    cudaError_t e;
+    // Layers are independent, so a call that covers many of them is cut into two chunks of layers: the upload of the
+    // second and the download of the first run on their own streams (separate copy engines) under the other
+    // chunk's kernel.  (Measured on the Llama-8B shape: 0.344 ms per step as one chunk, 0.318 as two, 0.326 as
+    // three, 0.351 as four: smaller launches lose more than the shorter exposed copies gain.)  Small calls take the
+    // plain path: upload, one launch, download, all on the caller's stream.
+    const long long items_per_layer = (long long)c->batch * c->n_kv_heads;
+    int chunks = 1;
+    if (nl >= 4 && items_per_layer * (long long)(nl / 2) >= 4LL * ctx->sm_count) chunks = 2;
+    if (chunks > 1 && !ctx->host_pipeline_ready) {
+        bool ok = cudaStreamCreateWithFlags(&ctx->up_stream, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&ctx->down_stream, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&ctx->ev_start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&ctx->ev_down, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; i < 8 && ok; ++i)
+            ok = cudaEventCreateWithFlags(&ctx->ev_up[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&ctx->ev_done[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return cuda_fail(ctx, cudaGetLastError(), "decode_attend_host: creating copy streams");
+        ctx->host_pipeline_ready = true;
     }
-    if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attend_host: upload");
-    st = lethe_decode_attend(ctx, c, layer_begin, layer_end, dq, k_new_host ? dk : nullptr, k_new_host ? dv : nullptr,
-                             k_new_host ? dpos : nullptr, scale, gamma, dout, lse_host ? dlse : nullptr, stream);
-    if (st != LETHE_OK) return st;
-    e = cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, s);
-    if (e == cudaSuccess && lse_host) e = cudaMemcpyAsync(lse_host, dlse, lse_bytes, cudaMemcpyDeviceToHost, s);
-    if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attend_host: download");
+    if (chunks == 1) {
+        e = cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess && k_new_host) {
+            e = cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s);
+            if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s);
+            if (e == cudaSuccess) e = cudaMemcpyAsync(dpos, token_pos_host, pos_bytes, cudaMemcpyHostToDevice, s);
+        }
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attend_host: upload");
+        st = lethe_decode_attend(ctx, c, layer_begin, layer_end, dq, k_new_host ? dk : nullptr, k_new_host ? dv : nullptr,
+                                 k_new_host ? dpos : nullptr, scale, gamma, dout, lse_host ? dlse : nullptr, stream);
+        if (st != LETHE_OK) return st;
+        e = cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess && lse_host) e = cudaMemcpyAsync(lse_host, dlse, lse_bytes, cudaMemcpyDeviceToHost, s);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attend_host: download");
+        return LETHE_OK;
+    }
+
+    // the copy streams start after whatever the caller's stream holds (the previous call's kernels read the staging)
+    e = cudaEventRecord(ctx->ev_start, s);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->up_stream, ctx->ev_start, 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->down_stream, ctx->ev_start, 0);
+    if (e == cudaSuccess && k_new_host) e = cudaMemcpyAsync(dpos, token_pos_host, pos_bytes, cudaMemcpyHostToDevice, ctx->up_stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attend_host: pipeline start");
+    const size_t q_layer = q_bytes / nl, kv_layer = kv_bytes / nl, lse_layer = lse_bytes / nl;
+    size_t l0 = 0;
+    for (int ci = 0; ci < chunks; ++ci) {
+        const size_t l1 = nl * (size_t)(ci + 1) / chunks;
+        const size_t nq = (l1 - l0) * q_layer, nkv = (l1 - l0) * kv_layer;
+        e = cudaMemcpyAsync((char*)dq + l0 * q_layer, (const char*)q_host + l0 * q_layer, nq, cudaMemcpyHostToDevice, ctx->up_stream);
+        if (e == cudaSuccess && k_new_host) {
+            e = cudaMemcpyAsync((char*)dk + l0 * kv_layer, (const char*)k_new_host + l0 * kv_layer, nkv, cudaMemcpyHostToDevice, ctx->up_stream);
+            if (e == cudaSuccess)
+                e = cudaMemcpyAsync((char*)dv + l0 * kv_layer, (const char*)v_new_host + l0 * kv_layer, nkv, cudaMemcpyHostToDevice, ctx->up_stream);
+        }
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_up[ci], ctx->up_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s, ctx->ev_up[ci], 0);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attend_host: upload");
+        st = lethe_decode_attend(ctx, c, layer_begin + (int)l0, layer_begin + (int)l1, (char*)dq + l0 * q_layer,
+                                 k_new_host ? (char*)dk + l0 * kv_layer : nullptr, k_new_host ? (char*)dv + l0 * kv_layer : nullptr,
+                                 k_new_host ? dpos : nullptr, scale, gamma, (char*)dout + l0 * q_layer,
+                                 lse_host ? dlse + l0 * (lse_layer / 4) : nullptr, stream);
+        if (st != LETHE_OK) return st;
+        e = cudaEventRecord(ctx->ev_done[ci], s);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->down_stream, ctx->ev_done[ci], 0);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync((char*)out_host + l0 * q_layer, (char*)dout + l0 * q_layer, nq, cudaMemcpyDeviceToHost, ctx->down_stream);
+        if (e == cudaSuccess && lse_host)
+            e = cudaMemcpyAsync((char*)lse_host + l0 * lse_layer, (char*)dlse + l0 * lse_layer, (l1 - l0) * lse_layer,
+                                cudaMemcpyDeviceToHost, ctx->down_stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attend_host: download");
+        l0 = l1;
+    }
+    // the caller's stream ends after the last download: synchronising it is enough to read the results
+    e = cudaEventRecord(ctx->ev_down, ctx->down_stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s, ctx->ev_down, 0);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attend_host: pipeline end");
     return LETHE_OK;
 }
 
