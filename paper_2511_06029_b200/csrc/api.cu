@@ -11,6 +11,8 @@
 namespace lethe {
 cudaError_t launch_attend_simt(const AttendArgs& a, int dtype, int D, bool paged, cudaStream_t stream);
 size_t kv8_smem_bytes(int D, int shape, int chunk_tokens, int GP);
+size_t kv8_stream_smem_bytes(int D, int shape, int chunk_tokens, int GP);
+cudaError_t launch_attend_kv8_stream(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream);
 cudaError_t launch_attend_kv8(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream);
 size_t simt_smem_bytes(int D, int chunk_tokens, int GP);
 cudaError_t launch_attend_mma(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream);
@@ -364,7 +366,31 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
             a.v_scale[l] = c->v_scale ? c->v_scale[l] : 1.f;
             a.scale_log2[l] = scale[l] * a.k_scale[l] * 1.4426950408889634f;
         }
-        const int shape = (variant >= 2 && variant <= 7) ? variant - 2 : 0;
+        // many items: the persistent kernel (variants 8..13 pick its shape); few: the clustered one (variants 2..7)
+        const bool want_persistent = variant >= 8 && variant <= 13;
+        const bool want_clustered = variant >= 2 && variant <= 7;
+        if ((want_persistent || (!want_clustered && a.n_items >= 2 * ctx->sm_count)) && ctx->splits <= 1) {
+            const int pshape = want_persistent ? variant - 8 : 1;
+            const size_t fixed = kv8_stream_smem_bytes(c->head_dim, pshape, 0, a.GP);
+            int fit = 0;
+            if (fixed < ctx->max_smem) fit = (int)((ctx->max_smem - fixed) / ((size_t)a.GP * 4) / kGroupTokens) * kGroupTokens;
+            a.splits = 1;
+            a.chunk_tokens = fit < cap_groups * kGroupTokens ? fit : cap_groups * kGroupTokens;
+            if (a.chunk_tokens < kGroupTokens)
+                return fail(ctx, LETHE_ERR_UNSUPPORTED, "no shared memory left for the logit buffer of this persistent shape");
+            const int grid = a.n_items < ctx->sm_count ? a.n_items : ctx->sm_count;
+            if (a.chunk_tokens < cap_groups * kGroupTokens) {  // overflow of the logit buffer: one slice per CTA
+                a.spill_tokens = cap_groups * kGroupTokens - a.chunk_tokens;
+                const size_t need = (size_t)grid * a.spill_tokens * a.GP * sizeof(float);
+                st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "logit overflow scratch");
+                if (st != LETHE_OK) return st;
+                a.spill = (float*)ctx->scratch;
+            }
+            const cudaError_t ep = launch_attend_kv8_stream(a, c->head_dim, pshape, paged, grid, (cudaStream_t)stream);
+            if (ep != cudaSuccess) return cuda_fail(ctx, ep, "decode_attend launch (quantised cache, persistent)");
+            return LETHE_OK;
+        }
+        const int shape = want_clustered ? variant - 2 : 0;
         auto smem_for = [&](int S) -> size_t {
             const int chunk = ((cap_groups + S - 1) / S) * kGroupTokens;
             return kv8_smem_bytes(c->head_dim, shape, chunk, a.GP);

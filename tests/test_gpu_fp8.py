@@ -90,7 +90,8 @@ def test_quantised_decode_parity(ctx, Hq, Hkv, D, paged):
         _step(ctx, oc, gc, q, kn, vn, torch.arange(B, dtype=torch.int32) + 300 + step, scale, 0.95)
 
 
-@pytest.mark.parametrize("variant,splits", [(2, 1), (3, 2), (4, 4), (5, 1), (6, 8), (7, 2), (0, 0)])
+@pytest.mark.parametrize("variant,splits", [(2, 1), (3, 2), (4, 4), (5, 1), (6, 8), (7, 2), (0, 0), (8, 0), (9, 0), (10, 1),
+                                            (11, 0), (12, 0), (13, 0)])
 def test_quantised_decode_shapes_and_clusters(ctx, variant, splits):
     """Every kernel shape and cluster size on items long enough to give every CTA of a cluster several groups."""
     L, B, Hq, Hkv, D, cap = 1, 2, 8, 2, 128, 1100
@@ -159,3 +160,42 @@ def test_quantised_cache_limits(ctx):
     with pytest.raises(binding.LetheError) as e:
         ctx.decode_attend(bad, 0, 1, q, None, None, None, [0.1], 0.9, out)
     assert e.value.status == binding.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_quantised_persistent_kernel_many_items(ctx, paged):
+    """Enough items for the persistent kernel to be the automatic choice (more than two per SM): ragged lengths,
+    appends, attend-only step; then a capacity small enough that logits overflow to scratch (forced shape)."""
+    L, B, Hq, Hkv, D, cap = 4, 10, 16, 8, 128, 160
+    g = torch.Generator().manual_seed(31 + paged)
+    lens = torch.randint(1, cap - 6, (L, B, Hkv), generator=g)
+    oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=5, k_scale=[0.4, 0.6, 0.8, 1.0], v_scale=[1.0, 0.5, 2.0, 0.75],
+                   page_tokens=16 if paged else 0)
+    gc = to_device(oc)
+    scale = torch.tensor([0.1, 0.08, 0.12, 0.09], dtype=torch.float32)
+    for step in range(4):
+        q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+        if step == 2:
+            _step(ctx, oc, gc, q, None, None, None, scale, 0.97, want_lse=True)
+            continue
+        kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+        vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+        _step(ctx, oc, gc, q, kn, vn, torch.arange(B, dtype=torch.int32) + 500 + step, scale, 0.97)
+
+
+def test_quantised_persistent_kernel_logit_overflow(ctx):
+    """Items longer than the on-chip logit buffer of the widest shape: the tail's logits go through global scratch."""
+    L, B, Hq, Hkv, D, cap = 1, 2, 16, 2, 128, 12000
+    g = torch.Generator().manual_seed(3)
+    lens = torch.tensor([[[11950, 9000], [4000, 11990]]])
+    oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=9, k_scale=[0.5], v_scale=[1.5])
+    gc = to_device(oc)
+    ctx.set_tuning(12, 0)                                     # (16 warps, 2 stages): least room for logits
+    try:
+        for step in range(2):
+            q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+            kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            _step(ctx, oc, gc, q, kn, vn, torch.tensor([1, 2], dtype=torch.int32), torch.tensor([0.05]), 0.99)
+    finally:
+        ctx.set_tuning(0, 0)
