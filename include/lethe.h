@@ -123,7 +123,8 @@ lethe_status lethe_poll_status(lethe_ctx *ctx, void *stream, int32_t *info);
  * Tensor-core variants need a bf16 cache (and 16-token pages when paged).
  * A quantised cache (LETHE_FP8_E4M3) runs its own tensor-core kernels: variants 2..7 force the clustered one with
  * shape (4,4) (8,4) (4,2) (4,3) (2,4) (8,2) (splits as above), variants 8..13 the persistent one with shape (8,4)
- * (12,3) (10,4) (8,5) (16,2) (12,2); any other value chooses by the number of items.
+ * (12,3) (10,4) (8,5) (16,2) (12,2); any other value means the clustered kernel with shape (4,4), the faster of
+ * the two at every size measured.
  * variant 40..42 select the engine of lethe_prefill_seed and leave everything else as it is: 40 = tcgen05
  * kernels (accumulators in tensor memory; operand tiles by TMA for contiguous caches, by cp.async for paged
  * ones; the default), 41 = mma.sync kernels, 42 = tcgen05 kernels with cp.async tiles always; splits is ignored.

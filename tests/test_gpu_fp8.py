@@ -164,8 +164,8 @@ def test_quantised_cache_limits(ctx):
 
 @pytest.mark.parametrize("paged", [False, True])
 def test_quantised_persistent_kernel_many_items(ctx, paged):
-    """Enough items for the persistent kernel to be the automatic choice (more than two per SM): ragged lengths,
-    appends, attend-only step; then a capacity small enough that logits overflow to scratch (forced shape)."""
+    """The persistent kernel (forced: shape (12,3)) on more than two items per SM, then the automatic choice on the
+    same state: ragged lengths, appends, an attend-only step."""
     L, B, Hq, Hkv, D, cap = 4, 10, 16, 8, 128, 160
     g = torch.Generator().manual_seed(31 + paged)
     lens = torch.randint(1, cap - 6, (L, B, Hkv), generator=g)
@@ -173,14 +173,18 @@ def test_quantised_persistent_kernel_many_items(ctx, paged):
                    page_tokens=16 if paged else 0)
     gc = to_device(oc)
     scale = torch.tensor([0.1, 0.08, 0.12, 0.09], dtype=torch.float32)
-    for step in range(4):
-        q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
-        if step == 2:
-            _step(ctx, oc, gc, q, None, None, None, scale, 0.97, want_lse=True)
-            continue
-        kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
-        vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
-        _step(ctx, oc, gc, q, kn, vn, torch.arange(B, dtype=torch.int32) + 500 + step, scale, 0.97)
+    try:
+        for step in range(5):
+            ctx.set_tuning(9 if step < 3 else 0, 0)
+            q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+            if step == 2:
+                _step(ctx, oc, gc, q, None, None, None, scale, 0.97, want_lse=True)
+                continue
+            kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            _step(ctx, oc, gc, q, kn, vn, torch.arange(B, dtype=torch.int32) + 500 + step, scale, 0.97)
+    finally:
+        ctx.set_tuning(0, 0)
 
 
 def test_quantised_persistent_kernel_logit_overflow(ctx):
