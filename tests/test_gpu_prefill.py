@@ -23,7 +23,7 @@ TCGEN05, MMA_SYNC, TCGEN05_CP_ASYNC = 40, 41, 42                     # lethe_set
 @pytest.mark.parametrize("engine", [TCGEN05, MMA_SYNC, TCGEN05_CP_ASYNC])
 @pytest.mark.parametrize("Hq,Hkv,D,P", [(32, 8, 128, 300), (28, 4, 128, 129), (8, 8, 128, 64), (4, 2, 64, 257),
                                         (6, 2, 128, 17), (5, 1, 64, 1), (16, 2, 128, 200), (8, 2, 128, 128),
-                                        (14, 2, 64, 385)])
+                                        (14, 2, 64, 385), (10, 2, 128, 200), (12, 2, 64, 150)])
 def test_prefill_seed_parity(ctx, engine, Hq, Hkv, D, P):
     oracle.set_threads(min(8, oracle.max_threads()))
     ctx.set_tuning(engine, 0)
@@ -107,6 +107,27 @@ def test_prefill_seed_engines_agree_on_a_long_prompt(ctx):
     G = Hq // Hkv
     want = G * (1 - 0.995 ** P) / (1 - 0.995)
     assert torch.allclose(res[TCGEN05][..., :P].double().sum(-1), torch.full((L, B, Hkv), want, dtype=torch.float64), rtol=2e-3)
+
+
+@pytest.mark.parametrize("engine", [TCGEN05, MMA_SYNC, TCGEN05_CP_ASYNC])
+def test_prefill_seed_capacity_below_one_tile(ctx, engine):
+    """A cache whose capacity is smaller than the 128-row operand tile (the tile runs past the item's rows)."""
+    L, B, Hq, Hkv, D, P, cap = 2, 3, 8, 2, 128, 40, 48
+    oc = random_cache(L, B, Hq, Hkv, D, cap, 44, dtype=torch.bfloat16, seed=12, rel_init="rand")
+    gc = to_device(oc)
+    qp = torch.randn((L, B, P, Hq, D), generator=torch.Generator().manual_seed(13)).to(torch.bfloat16)
+    scale = torch.tensor([0.09, 0.12], dtype=torch.float32)
+    before = oc.clone()
+    assert oracle.prefill_seed(oc, qp, scale, 0.95) == oracle.OK
+    ctx.set_tuning(engine, 0)
+    try:
+        ctx.prefill_seed(gc, qp.cuda(), scale.tolist(), 0.95)
+        assert ctx.poll_status()[0] == 0
+    finally:
+        ctx.set_tuning(TCGEN05, 0)
+    got = gc.rel.cpu()
+    assert torch.allclose(got[..., :P], oc.rel[..., :P], rtol=1e-3, atol=1e-6)
+    assert torch.equal(got[..., P:], before.rel[..., P:])
 
 
 def test_prefill_seed_rejects_bad_input(ctx):
