@@ -294,6 +294,9 @@ def cpu_baseline(w, r: Runner | None, seconds=12.0, layers=8, seqs=4):
     oracle.rasr_prune(oc, bud, w.recent, w.sink)
     prune_s = time.perf_counter() - t1
     per_step = attend_s / steps + prune_s / w.prune_interval
+    overlap = None
+    if r is not None:
+        overlap = retained_set_overlap(w, ws, r.dev, oc, cap, steps, layers, seqs, scale)
     # the same oracle on one core, on a few more steps of the same sample (decode only; the prune share is ~1 %)
     oracle.set_threads(1)
     t1 = time.perf_counter()
@@ -311,7 +314,48 @@ def cpu_baseline(w, r: Runner | None, seconds=12.0, layers=8, seqs=4):
             "sample": f"{layers} layers x {seqs} sequences x {w.n_kv_heads} KV heads at ~{w.mean_budget} tokens, "
                       f"{steps} decode steps in {attend_s:.1f} s plus one prune round ({prune_s * 1e3:.0f} ms) "
                       f"amortised over {w.prune_interval} steps",
-            "ms_per_sample_step": per_step * 1e3, "token_heads_per_sample_step": th / steps}
+            "ms_per_sample_step": per_step * 1e3, "token_heads_per_sample_step": th / steps,
+            "retained_set_overlap": overlap}
+
+
+def retained_set_overlap(w, ws, dev, oc, cap, steps, layers, seqs, scale):
+    """End-to-end agreement of what is kept: the GPU path replays the sample the oracle was just timed on (same
+    initial cache, same per-step inputs, same number of steps, then one prune round), free-running on its own
+    scores, and the retained positions of every item are compared with the oracle's."""
+    from paper_2511_06029_b200 import binding
+    st = synth.initial_kv(ws, w.mean_budget, cap)
+    gc = binding.Cache(ws.n_q_heads, *(st[k].to(dev) for k in ("k", "v", "rel", "pos", "len")))
+    ctx = binding.Context(dev.index)
+    try:
+        sc = scale.tolist()
+        out = torch.empty((layers, seqs, ws.n_q_heads, ws.head_dim), dtype=ws.dtype, device=dev)
+        for i in range(steps):
+            x = synth.step_inputs(ws, i)
+            ctx.decode_attend(gc, 0, layers, x["q"].to(dev), x["k_new"].to(dev), x["v_new"].to(dev),
+                              x["token_pos"].to(dev), sc, w.gamma, out)
+        S = torch.zeros((layers, seqs), dtype=torch.float32, device=dev)
+        bud = torch.zeros((layers, seqs), dtype=torch.int32, device=dev)
+        T = torch.full((seqs,), layers * w.mean_budget, dtype=torch.int64, device=dev)
+        ctx.estimate_sparsity(gc, S)
+        ctx.alloc_budgets(S, T, w.k_min, bud)
+        ctx.rasr_prune(gc, bud, w.recent, w.sink)
+        status, _ = ctx.poll_status()
+        glen, gpos = gc.len.cpu(), gc.pos.cpu()
+    finally:
+        ctx.close()
+    jac, same = [], 0
+    for l in range(layers):
+        for b in range(seqs):
+            for h in range(ws.n_kv_heads):
+                a = set(gpos[l, b, h, :int(glen[l, b, h])].tolist())
+                o = set(oc.pos[l, b, h, :int(oc.len[l, b, h])].tolist())
+                jac.append(len(a & o) / max(1, len(a | o)))
+                same += a == o
+    return {"items": len(jac), "decode_steps": steps, "device_status": status,
+            "jaccard_mean": sum(jac) / len(jac), "jaccard_min": min(jac), "identical_sets": same / len(jac),
+            "equal_lengths": float((glen == oc.len).float().mean()),
+            "note": "GPU free-running on its own fp32 scores vs the oracle (fp64), retained positions per (layer, sequence, KV head) "
+                    "after the sample's decode steps and one prune round"}
 
 
 def run_reference(args, w):
@@ -572,6 +616,7 @@ def main():
                            "d2h_bytes_per_step": d2h, "ms_per_step": e_total_ms / args.steps}
         if not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, r)
+            line["retained_set_overlap"] = line["cpu_baseline"].pop("retained_set_overlap", None)
         print(json.dumps(line))
     if dist is not None:
         dist.barrier()
