@@ -126,8 +126,8 @@ lethe_status lethe_poll_status(lethe_ctx *ctx, void *stream, int32_t *info);
  * (12,3) (10,4) (8,5) (16,2) (12,2); any other value means the clustered kernel with shape (4,4), the faster of
  * the two at every size measured.
  * variant 40..42 select the engine of lethe_prefill_seed and leave everything else as it is: 40 = tcgen05
- * kernels (accumulators in tensor memory; operand tiles by TMA for contiguous caches, by cp.async for paged
- * ones; the default), 41 = mma.sync kernels, 42 = tcgen05 kernels with cp.async tiles always; splits is ignored.
+ * kernels (accumulators in tensor memory, operand tiles by TMA; the default), 41 = mma.sync kernels,
+ * 42 = tcgen05 kernels with cp.async tiles; splits is ignored.
  * splits: 0 = automatic, else CTAs per item (1, 2, 4, 8 or 16; they form one thread-block cluster); the
  * persistent variants take 0 or 1.
  * Returns LETHE_ERR_INVALID_ARG for other values.

@@ -20,7 +20,8 @@
 // Roles: warps 0-7 read TMEM and do the arithmetic (warp w owns TMEM lanes 32 (w % 4) .. + 31 and columns
 // 64 (w / 4) .. + 63), warp 8 allocates TMEM and one of its lanes issues the MMAs, and the operand tiles arrive in
 // the 128-byte-swizzled K-major layout the MMA's shared-memory descriptors name either by TMA (one lane of warp 9
-// issues cp.async.bulk.tensor boxes; contiguous caches) or by 16-byte cp.async from warps 9-12 (paged caches).
+// issues cp.async.bulk.tensor boxes: one per 128-row tile of a contiguous cache, one per page of a paged one) or
+// by 16-byte cp.async from warps 9-12 (selectable; also the fallback when no tensor map can be made).
 // Hand-offs are mbarriers: producer -> MMA (a_full, b_full), MMA -> producer (a_empty, b_empty, by
 // tcgen05.commit), MMA -> softmax (t_full, by tcgen05.commit), softmax -> MMA (t_empty).  Every wait is bounded:
 // when one runs out the CTA sets an abort flag, every role leaves its loop, LETHE_ERR_TIMEOUT is recorded, TMEM is
@@ -328,8 +329,27 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
                     for (int hf = 0; hf < D / 64; ++hf) tc_tma_4d(tile + hf * HALF_BYTES, &maps.q, 64 * hf, hkv * G, q0, l * a.B + b, bar);
                 };
                 auto load_keys = [&](int j0, uint32_t tile, unsigned long long* bar) {
+                    if (!a.paged) {
 #pragma unroll
-                    for (int hf = 0; hf < D / 64; ++hf) tc_tma_3d(tile + hf * HALF_BYTES, &maps.k, 64 * hf, j0, item, bar);
+                        for (int hf = 0; hf < D / 64; ++hf) tc_tma_3d(tile + hf * HALF_BYTES, &maps.k, 64 * hf, j0, item, bar);
+                        return;
+                    }
+                    // paged: one box per page (the map sees the pool as [pages][page_tokens][D]); slots beyond the
+                    // item's table and bad ids read page 0 — rows that no query sees
+                    const int pt = a.page_tokens, per_tile = kTcTile / pt;
+                    int pages[8];
+#pragma unroll
+                    for (int pg = 0; pg < 8; ++pg) {
+                        const int slot = j0 / pt + pg;
+                        int page = (pg < per_tile && slot < a.capacity) ? a.page_table[(size_t)item * a.capacity + slot] : 0;
+                        pages[pg] = (page < 0 || page >= a.n_pages) ? 0 : page;
+                    }
+#pragma unroll
+                    for (int pg = 0; pg < 8; ++pg)
+                        if (pg < per_tile)
+#pragma unroll
+                            for (int hf = 0; hf < D / 64; ++hf)
+                                tc_tma_3d(tile + hf * HALF_BYTES + pg * pt * 128, &maps.k, 64 * hf, 0, pages[pg], bar);
                 };
                 int step = 0;
                 bool alive = true;
@@ -576,21 +596,25 @@ cudaError_t launch_tc(const PrefillArgs& a, const TcMaps& maps, int items, cudaS
 // Two (max, sum) partials per (query, head) column.
 size_t prefill_tc_stats_bytes(int items, int P, int HP) { return 2 * (size_t)items * P * HP * sizeof(float2); }
 
-// encode: cuTensorMapEncodeTiled resolved by the caller, or NULL; the TMA path is taken for contiguous caches when
-// it is there and `allow_tma` is set, the cp.async path otherwise.
+// encode: cuTensorMapEncodeTiled resolved by the caller, or NULL; the TMA path is taken when it is there, `allow_tma`
+// is set and the maps can be made, the cp.async path otherwise.
 cudaError_t launch_prefill_tc(const PrefillArgs& a, int items, int L, int D, void* encode, bool allow_tma, cudaStream_t stream) {
     TcMaps maps;
     memset(&maps, 0, sizeof(maps));
     bool tma = false;
-    if (encode && allow_tma && !a.paged) {
+    // paged pools take one box per page: pages of 16 to 128 tokens that divide the 128-row tile
+    const bool pages_ok = !a.paged || (a.page_tokens >= 16 && a.page_tokens <= kTcTile && kTcTile % a.page_tokens == 0 &&
+                                       a.n_pages <= 0x7fffffffLL);
+    if (encode && allow_tma && pages_ok) {
         typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                       const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                       CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
         encode_fn fn = reinterpret_cast<encode_fn>(encode);
         const cuuint32_t qpb = (cuuint32_t)(kTcTile / a.G);
-        const cuuint64_t kd[3] = {(cuuint64_t)D, (cuuint64_t)a.capacity, (cuuint64_t)items};
-        const cuuint64_t ks[2] = {(cuuint64_t)D * 2, (cuuint64_t)a.capacity * D * 2};
-        const cuuint32_t kb[3] = {64, (cuuint32_t)kTcTile, 1};
+        const cuuint64_t rows = a.paged ? (cuuint64_t)a.page_tokens : (cuuint64_t)a.capacity;   // rows of one item / page
+        const cuuint64_t kd[3] = {(cuuint64_t)D, rows, a.paged ? (cuuint64_t)a.n_pages : (cuuint64_t)items};
+        const cuuint64_t ks[2] = {(cuuint64_t)D * 2, rows * D * 2};
+        const cuuint32_t kb[3] = {64, a.paged ? (cuuint32_t)a.page_tokens : (cuuint32_t)kTcTile, 1};
         const cuuint64_t qd[4] = {(cuuint64_t)D, (cuuint64_t)a.Hq, (cuuint64_t)a.P, (cuuint64_t)L * a.B};
         const cuuint64_t qs[3] = {(cuuint64_t)D * 2, (cuuint64_t)a.Hq * D * 2, (cuuint64_t)a.P * a.Hq * D * 2};
         const cuuint32_t qb[4] = {64, (cuuint32_t)a.G, qpb, 1};
