@@ -423,22 +423,23 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         // enough items to give every SM several: the persistent kernel; few long items: the clustered one
         if (!mma_ok) variant = 1;
         else if (a.n_items >= 2 * ctx->sm_count && ctx->splits <= 1) {
-            // Persistent kernels, best measured first, taking the first whose logit buffer(s) cover the
-            // capacity on chip: asynchronous epilogue (5,3) (6,3) (8,2) (4,4), then the synchronous (7,3) (6,3) (8,2).
-            // If none does, the tail of long items overflows to scratch: asynchronous (5,3) when each of its two
-            // buffers still holds most of the capacity, else the synchronous (6,3), whose single buffer is
-            // twice as long.
+            // Persistent kernels.  The asynchronous-epilogue kernel (best measured first: (5,3) (6,3) (8,2) (4,4)) when
+            // both of its logit buffers cover the capacity on chip.  Otherwise the tail of long items overflows to
+            // scratch, and what matters is how much of a typical item still fits on chip: the asynchronous (5,3)
+            // while each of its two buffers holds at least 0.4 of the capacity (caches are sized well above the
+            // lengths they reach between prune rounds), else the synchronous (8,2), whose stages leave the most room
+            // for its single buffer.  Measured: Llama shape at capacities 3584 / 4608 / 6144 0.88 of the copy peak
+            // with the former against 0.86 to 0.88 with the latter; long-reasoning shape 1.00 against 0.985; Qwen
+            // shape (8 logit columns per token, capacity 5312) 0.95 with the latter against 0.61 to 0.80.
             const int cap_pad = cap_groups * kGroupTokens;
             auto async_fits = [&](int shape) { return async_smem_bytes(c->head_dim, shape, cap_pad, a.GP) <= ctx->max_smem; };
             variant = 0;
             for (int shape : {3, 2, 0, 5})
                 if (variant == 0 && async_fits(shape)) variant = 16 + shape;
-            for (int shape : {4, 1, 0})
-                if (variant == 0 && stream_chunk(shape) == cap_pad) variant = 8 + shape;
             if (variant == 0) {
                 const size_t fixed = async_smem_bytes(c->head_dim, 3, 0, a.GP);
                 const size_t async_chunk = fixed < ctx->max_smem ? (ctx->max_smem - fixed) / ((size_t)2 * a.GP * 4) : 0;
-                variant = (async_chunk * 10 >= (size_t)cap_pad * 6) ? 16 + 3 : 8 + 1;
+                variant = (async_chunk * 5 >= (size_t)cap_pad * 2) ? 16 + 3 : 8 + 0;
             }
         } else variant = 2;  // few items per launch (one layer at a time): clustered kernel, 4 warps x 3 stages
     }
