@@ -60,7 +60,7 @@ class ClockSampler:
         self.p = None
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                       "-lms", "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+                                       "-lms", "50", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
 
@@ -141,7 +141,8 @@ class Runner:
             kn = torch.randn((L, B, w.n_kv_heads, w.head_dim), generator=g, device=device).to(w.dtype)
             vn = torch.randn((L, B, w.n_kv_heads, w.head_dim), generator=g, device=device).to(w.dtype)
             self.pool.append((q, kn, vn))
-        self.host_pool = [tuple(t.cpu().pin_memory() for t in p) for p in self.pool[:4]]
+        # pinned host copies of the same inputs: the end-to-end loop replays exactly the device loop's sequence
+        self.host_pool = [tuple(t.cpu().pin_memory() for t in p) for p in self.pool]
         self.out = torch.empty((L, B, w.n_q_heads, w.head_dim), dtype=w.dtype, device=device)
         self.out_host = torch.empty((L, B, w.n_q_heads, w.head_dim), dtype=w.dtype).pin_memory()
         self.token_pos = torch.zeros((B,), dtype=torch.int32, device=device)
@@ -387,7 +388,7 @@ def workload_config(w, args, extra=None):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--steps", type=int, default=1024)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b")
