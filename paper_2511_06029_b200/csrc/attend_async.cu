@@ -231,6 +231,7 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
         unsigned char* my_stage = smem_raw + (size_t)warp * WARP_BYTES;
         const uint32_t my_stage_u32 = smem_u32(my_stage);
         bool bad_page = false;
+        const uint64_t stream_policy = l2_evict_first_policy();  // K / V tiles are read once: evict-first in L2
         unsigned slot_bad = 0;    // TMA: slots whose tile must be ignored (page id outside the pool)
         unsigned slot_phase = 0;  // TMA: parity of the next completion of each slot's mbarrier
         unsigned slot_busy = 0;   // TMA: slots with a load in flight or landed but not yet consumed
@@ -303,8 +304,8 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
                 const bool valid = ok && (tok0 + r < it.n);
                 const int soff = valid ? r * ROW_BYTES + c * 16 : 0;
                 const uint32_t doff = r * ROW_BYTES + ((c ^ (r & 7)) << 4);
-                cp_async16(ks_u32 + doff, kb + soff, valid ? 16 : 0);
-                cp_async16(vs_u32 + doff, vb + soff, valid ? 16 : 0);
+                cp_async16_hint(ks_u32 + doff, kb + soff, valid ? 16 : 0, stream_policy);
+                cp_async16_hint(vs_u32 + doff, vb + soff, valid ? 16 : 0, stream_policy);
             }
         };
 

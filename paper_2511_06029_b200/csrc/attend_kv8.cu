@@ -115,6 +115,7 @@ __global__ void __launch_bounds__(NW * 32) attend_kv8_kernel(const __grid_consta
     const int t0 = g_begin * kGroupTokens, t1 = g_end * kGroupTokens;
 
     bool bad_page = false;
+    const uint64_t stream_policy = l2_evict_first_policy();  // K / V tiles are read once: evict-first in L2
     // Sec. 4.1: append the generated token's key / value, quantised; the CTA whose range holds slot n_old stores it.
     if (append && n_old >= t0 && n_old < t1 && warp == 0) {
         const size_t src = ((size_t)(ic.li * a.B + ic.b) * a.Hkv + ic.hkv) * D;  // elements
@@ -168,8 +169,8 @@ __global__ void __launch_bounds__(NW * 32) attend_kv8_kernel(const __grid_consta
             const bool valid = ok && (tok0 + r < n);
             const int soff = valid ? r * ROW_BYTES + c * 16 : 0;  // rows past n are zero-filled, never read
             const uint32_t doff = swz(r, c);
-            cp_async16(ks_u32 + doff, kb + soff, valid ? 16 : 0);
-            cp_async16(vs_u32 + doff, vb + soff, valid ? 16 : 0);
+            cp_async16_hint(ks_u32 + doff, kb + soff, valid ? 16 : 0, stream_policy);
+            cp_async16_hint(vs_u32 + doff, vb + soff, valid ? 16 : 0, stream_policy);
         }
     };
 

@@ -120,6 +120,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
     unsigned char* my_stage = smem_raw + (size_t)warp * WARP_BYTES;
     const uint32_t my_stage_u32 = smem_u32(my_stage);
     bool bad_page = false;
+    const uint64_t stream_policy = l2_evict_first_policy();
 
     // issue the copies of this warp's local group `idx` of item `it` into stage slot `slot`
     // PAGED: page ids of this warp's local groups are fetched 32 at a time, one lane each, a block ahead of their
@@ -178,8 +179,8 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
             const bool valid = ok && (tok0 + r < it.n);
             const int soff = valid ? r * ROW_BYTES + c * 16 : 0;  // rows past n are zero-filled, never read
             const uint32_t doff = r * ROW_BYTES + ((c ^ (r & 7)) << 4);
-            cp_async16(ks_u32 + doff, kb + soff, valid ? 16 : 0);
-            cp_async16(vs_u32 + doff, vb + soff, valid ? 16 : 0);
+            cp_async16_hint(ks_u32 + doff, kb + soff, valid ? 16 : 0, stream_policy);
+            cp_async16_hint(vs_u32 + doff, vb + soff, valid ? 16 : 0, stream_policy);
         }
     };
 
