@@ -121,6 +121,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
     const uint32_t my_stage_u32 = smem_u32(my_stage);
     bool bad_page = false;
     const uint64_t stream_policy = l2_evict_first_policy();
+    const uint64_t spill_policy = l2_evict_last_policy();
 
     // issue the copies of this warp's local group `idx` of item `it` into stage slot `slot`
     // PAGED: page ids of this warp's local groups are fetched 32 at a time, one lane each, a block ahead of their
@@ -262,9 +263,9 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
             const float s11 = (tokB < cur.n) ? (ca[3] + cb[3]) * sl2 : -INFINITY;
             if (2 * tq < GP) {
                 if (!SPILL || tokA < chunk) st_shared_f2(lg_u32 + (tokA * GP + 2 * tq) * 4, s00, s01);
-                else *reinterpret_cast<float2*>(spill + (size_t)(tokA - chunk) * GP + 2 * tq) = make_float2(s00, s01);
+                else st_global_f2_hint(spill + (size_t)(tokA - chunk) * GP + 2 * tq, s00, s01, spill_policy);
                 if (!SPILL || tokB < chunk) st_shared_f2(lg_u32 + (tokB * GP + 2 * tq) * 4, s10, s11);
-                else *reinterpret_cast<float2*>(spill + (size_t)(tokB - chunk) * GP + 2 * tq) = make_float2(s10, s11);
+                else st_global_f2_hint(spill + (size_t)(tokB - chunk) * GP + 2 * tq, s10, s11, spill_policy);
             }
             float mx0 = fmaxf(s00, s10), mx1 = fmaxf(s01, s11);
 #pragma unroll
@@ -378,7 +379,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
                 for (int h = 0; h < kMaxGroup; h += 2) {
                     if (h < GP) {
                         const float2 s2 = in_smem ? ld_shared_f2(lg_u32 + (j * GP + h) * 4)
-                                                  : *reinterpret_cast<const float2*>(spill + (size_t)(j - chunk) * GP + h);
+                                                  : ld_global_f2_hint(spill + (size_t)(j - chunk) * GP + h, spill_policy);
                         mass += fast_exp2(s2.x - fm[h]) * fi[h];
                         if (h + 1 < G) mass += fast_exp2(s2.y - fm[h + 1]) * fi[h + 1];
                     }

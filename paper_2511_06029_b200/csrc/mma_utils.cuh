@@ -22,6 +22,21 @@ __device__ __forceinline__ void cp_async16_hint(uint32_t dst, const void* src, i
     asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2, %3;" ::"r"(dst), "l"(src), "r"(src_bytes), "l"(policy)
                  : "memory");
 }
+// Logits that overflow the shared-memory buffer are written and read back within one item: evict-last keeps them
+// in L2 under the K / V stream.
+__device__ __forceinline__ uint64_t l2_evict_last_policy() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void st_global_f2_hint(float* ptr, float x, float y, uint64_t policy) {
+    asm volatile("st.global.L2::cache_hint.v2.f32 [%0], {%1, %2}, %3;" ::"l"(ptr), "f"(x), "f"(y), "l"(policy) : "memory");
+}
+__device__ __forceinline__ float2 ld_global_f2_hint(const float* ptr, uint64_t policy) {
+    float2 v;
+    asm volatile("ld.global.L2::cache_hint.v2.f32 {%0, %1}, [%2], %3;" : "=f"(v.x), "=f"(v.y) : "l"(ptr), "l"(policy) : "memory");
+    return v;
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
