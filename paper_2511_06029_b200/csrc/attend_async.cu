@@ -59,10 +59,11 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, u
 }
 // One box (64 elements x 16 rows) of a 2-D tensor map into shared memory; completion is counted on `bar`.
 // x is always 0 or 64 elements (a multiple of 16 bytes), y is a row index.
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, unsigned long long* bar) {
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, unsigned long long* bar,
+                                            uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy)
         : "memory");
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
@@ -291,8 +292,8 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
                     mbar_arrive_expect_tx(bar, STAGE_BYTES);
 #pragma unroll
                     for (int hx = 0; hx < D / 64; ++hx) {
-                        tma_load_2d(ks_u32 + hx * 2048, &maps.k, hx * 64, (int)row0, bar);
-                        tma_load_2d(vs_u32 + hx * 2048, &maps.v, hx * 64, (int)row0, bar);
+                        tma_load_2d(ks_u32 + hx * 2048, &maps.k, hx * 64, (int)row0, bar, stream_policy);
+                        tma_load_2d(vs_u32 + hx * 2048, &maps.v, hx * 64, (int)row0, bar, stream_policy);
                     }
                 }
                 return;
