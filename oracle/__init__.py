@@ -22,7 +22,7 @@ _SRC = os.path.join(_HERE, "lethe_oracle.c")
 _LIB = os.path.join(_HERE, "liblethe_oracle.so")
 
 OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_BUDGET = 0, 1, 2, 3
-F32, BF16, FP8 = 0, 1, 2
+F32, BF16, FP8, FP8_E5M2 = 0, 1, 2, 3
 
 
 def build(force: bool = False) -> str:
@@ -78,6 +78,10 @@ def lib():
         _lib.oracle_e4m3_decode.argtypes = [ctypes.c_uint8]
         _lib.oracle_e4m3_encode.restype = ctypes.c_uint8
         _lib.oracle_e4m3_encode.argtypes = [ctypes.c_float]
+        _lib.oracle_e5m2_decode.restype = ctypes.c_double
+        _lib.oracle_e5m2_decode.argtypes = [ctypes.c_uint8]
+        _lib.oracle_e5m2_encode.restype = ctypes.c_uint8
+        _lib.oracle_e5m2_encode.argtypes = [ctypes.c_float]
         _lib.oracle_set_threads.argtypes = [ctypes.c_int]
         _lib.oracle_get_threads.restype = ctypes.c_int
         _lib.oracle_max_threads.restype = ctypes.c_int
@@ -110,6 +114,8 @@ def _dtype_code(dt: torch.dtype) -> int:
         return BF16
     if dt == torch.float8_e4m3fn:
         return FP8
+    if dt == torch.float8_e5m2:
+        return FP8_E5M2
     raise ValueError(f"unsupported dtype {dt}")
 
 
@@ -129,13 +135,13 @@ class OracleCache:
     len: torch.Tensor
     page_tokens: int = 0
     page_table: Optional[torch.Tensor] = None
-    k_scale: Optional[torch.Tensor] = None      # float8_e4m3fn caches: fp32 [L] (None = 1): stored byte x means scale * x
+    k_scale: Optional[torch.Tensor] = None      # float8 caches: fp32 [L] (None = 1): stored byte x means scale * x
     v_scale: Optional[torch.Tensor] = None
 
     @property
     def act_dtype(self) -> torch.dtype:
         """Type of q, k_new, v_new and out: the cache's own, bf16 for a quantised cache."""
-        return torch.bfloat16 if self.k.dtype == torch.float8_e4m3fn else self.k.dtype
+        return torch.bfloat16 if self.k.dtype in (torch.float8_e4m3fn, torch.float8_e5m2) else self.k.dtype
 
     @property
     def paged(self) -> bool:

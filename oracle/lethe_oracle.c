@@ -64,12 +64,13 @@
 #endif
 
 enum { ORACLE_OK = 0, ORACLE_ERR_INVALID_ARG = 1, ORACLE_ERR_CAPACITY = 2, ORACLE_ERR_BUDGET = 3 };
-enum { ORACLE_F32 = 0, ORACLE_BF16 = 1, ORACLE_FP8 = 2 };
+enum { ORACLE_F32 = 0, ORACLE_BF16 = 1, ORACLE_FP8 = 2, ORACLE_FP8_E5M2 = 3 };
+#define ORACLE_IS_FP8(dt) ((dt) == ORACLE_FP8 || (dt) == ORACLE_FP8_E5M2)
 
 typedef struct {
     int32_t n_layers, batch, n_q_heads, n_kv_heads, head_dim;
-    int32_t dtype;       /* storage type of K and V: ORACLE_F32, ORACLE_BF16 (held as uint16) or ORACLE_FP8
-                            (e4m3fn bytes; q, k_new, v_new, out are then bf16) */
+    int32_t dtype;       /* storage type of K and V: ORACLE_F32, ORACLE_BF16 (held as uint16), ORACLE_FP8 (e4m3fn
+                            bytes) or ORACLE_FP8_E5M2 (e5m2 bytes); with bytes, q, k_new, v_new, out are bf16 */
     int32_t paged;       /* 0 contiguous, 1 paged */
     int32_t capacity;    /* contiguous: token slots per item; paged: pages per item */
     int32_t page_tokens; /* tokens per page when paged, else ignored */
@@ -154,9 +155,41 @@ static uint8_t float_to_e4m3(float f) {
     return sign | (uint8_t)(code > 0x7e ? 0x7e : code);
 }
 
+/* e5m2 (1 sign, 5 exponent bits with bias 15, 2 mantissa bits: the upper byte of an IEEE half).  Largest finite
+ * value 57344; subnormals are multiples of 2^-16.  Exponent 31 (infinity, NaN) never occurs in a cache: the
+ * encoder saturates. */
+static double e5m2_to_double(uint8_t b) {
+    const int e = (b >> 2) & 31, m = b & 3;
+    double x;
+    if (e == 31) return m ? NAN : INFINITY * ((b & 0x80) ? -1.0 : 1.0);
+    if (e == 0) x = ldexp((double)m, -16);
+    else x = ldexp(1.0 + (double)m / 4.0, e - 15);
+    return (b & 0x80) ? -x : x;
+}
+
+/* float -> e5m2: round to nearest, ties to even; magnitudes beyond the largest finite value saturate to it. */
+static uint8_t float_to_e5m2(float f) {
+    if (f != f) return 0x7f;
+    const uint8_t sign = signbit(f) ? 0x80 : 0x00;
+    const float a = fabsf(f);
+    if (a > 57344.0f) return sign | 0x7b;
+    if (a < 6.103515625e-05f) return sign | (uint8_t)rintf(a * 65536.0f); /* below 2^-14: step 2^-16; 4 is the smallest normal */
+    int ex;
+    const float fr = frexpf(a, &ex);
+    int q = (int)rintf((2.0f * fr - 1.0f) * 4.0f); /* mantissa in quarters, 0..4 */
+    int e = ex - 1 + 15;
+    if (q == 4) {
+        q = 0;
+        e += 1;
+    }
+    const int code = (e << 2) | q;
+    return sign | (uint8_t)(code > 0x7b ? 0x7b : code);
+}
+
 static double load_elt(const void *base, int dtype, int64_t idx) {
     if (dtype == ORACLE_BF16) return bf16_to_double(((const uint16_t *)base)[idx]);
     if (dtype == ORACLE_FP8) return e4m3_to_double(((const uint8_t *)base)[idx]);
+    if (dtype == ORACLE_FP8_E5M2) return e5m2_to_double(((const uint8_t *)base)[idx]);
     return (double)((const float *)base)[idx];
 }
 
@@ -165,14 +198,16 @@ static void store_elt(void *base, int dtype, int64_t idx, double x) {
     else ((float *)base)[idx] = (float)x;
 }
 
-static size_t elt_size(int dtype) { return dtype == ORACLE_BF16 ? 2 : (dtype == ORACLE_FP8 ? 1 : 4); }
+static size_t elt_size(int dtype) { return dtype == ORACLE_BF16 ? 2 : (ORACLE_IS_FP8(dtype) ? 1 : 4); }
 
 /* type of q, k_new, v_new and out: the cache's own, except that a quantised cache takes bf16 activations */
-static int act_dtype(int dtype) { return dtype == ORACLE_FP8 ? ORACLE_BF16 : dtype; }
+static int act_dtype(int dtype) { return ORACLE_IS_FP8(dtype) ? ORACLE_BF16 : dtype; }
 
 /* test hooks for the two conversions */
 double oracle_e4m3_decode(uint8_t b) { return e4m3_to_double(b); }
 uint8_t oracle_e4m3_encode(float f) { return float_to_e4m3(f); }
+double oracle_e5m2_decode(uint8_t b) { return e5m2_to_double(b); }
+uint8_t oracle_e5m2_encode(float f) { return float_to_e5m2(f); }
 
 static int64_t cap_tokens(const oracle_cache *c) {
     return c->paged ? (int64_t)c->capacity * c->page_tokens : (int64_t)c->capacity;
@@ -194,7 +229,7 @@ static int check_cache(const oracle_cache *c) {
     if (!c || !c->k || !c->v || !c->rel || !c->pos || !c->len) return ORACLE_ERR_INVALID_ARG;
     if (c->n_layers < 1 || c->batch < 1 || c->n_kv_heads < 1 || c->head_dim < 1) return ORACLE_ERR_INVALID_ARG;
     if (c->n_q_heads < c->n_kv_heads || c->n_q_heads % c->n_kv_heads) return ORACLE_ERR_INVALID_ARG;
-    if (c->dtype != ORACLE_F32 && c->dtype != ORACLE_BF16 && c->dtype != ORACLE_FP8) return ORACLE_ERR_INVALID_ARG;
+    if (c->dtype != ORACLE_F32 && c->dtype != ORACLE_BF16 && !ORACLE_IS_FP8(c->dtype)) return ORACLE_ERR_INVALID_ARG;
     if (c->capacity < 1) return ORACLE_ERR_INVALID_ARG;
     if (c->paged && (!c->page_table || c->page_tokens < 1)) return ORACLE_ERR_INVALID_ARG;
     return ORACLE_OK;
@@ -205,7 +240,7 @@ static int check_cache(const oracle_cache *c) {
  * For layers [layer_begin, layer_end), with li = layer - layer_begin:
  *   q, out        [layers][B][Hq][D]   (cache dtype; bf16 when the cache is ORACLE_FP8)
  *   k_new, v_new  [layers][B][Hkv][D]  (same type as q) or both NULL = attend only
- * A quantised (ORACLE_FP8) cache holds K / k_scale[l] and V / v_scale[l] as e4m3fn bytes: an appended row is
+ * A quantised (ORACLE_FP8, ORACLE_FP8_E5M2) cache holds K / k_scale[l] and V / v_scale[l] as e4m3fn or e5m2 bytes: an appended row is
  * divided by the layer's scale in fp32 (one IEEE division) and rounded to nearest-even with saturation; when
  * read, a byte x counts as scale * x exactly.  Quantisation composes with pruning (Sec. 2, related work on
  * quantised caches): rows are moved as bytes, scores never see the storage type.
@@ -251,19 +286,19 @@ int oracle_decode_attend(oracle_cache *c, int layer_begin, int layer_end, const 
         const int64_t item = item_index(c, l, b, hkv);
         int64_t n = c->len[item];
         const int act = act_dtype(c->dtype);
-        const float ks = (c->dtype == ORACLE_FP8 && c->k_scale) ? c->k_scale[l] : 1.0f;
-        const float vs = (c->dtype == ORACLE_FP8 && c->v_scale) ? c->v_scale[l] : 1.0f;
+        const float ks = (ORACLE_IS_FP8(c->dtype) && c->k_scale) ? c->k_scale[l] : 1.0f;
+        const float vs = (ORACLE_IS_FP8(c->dtype) && c->v_scale) ? c->v_scale[l] : 1.0f;
 
         /* Sec. 4.1: the cache grows by the token just generated.  It enters with
          * zero relevance and takes part in this step's attention. */
         if (k_new) {
             const int64_t src = (((int64_t)li * B + b) * Hkv + hkv) * D;
             const int64_t dst = row_offset(c, item, n);
-            if (c->dtype == ORACLE_FP8) {
+            if (ORACLE_IS_FP8(c->dtype)) {
                 for (int d = 0; d < D; ++d) {
                     const float kx = (float)load_elt(k_new, ORACLE_BF16, src + d), vx = (float)load_elt(v_new, ORACLE_BF16, src + d);
-                    ((uint8_t *)c->k)[dst + d] = float_to_e4m3(kx / ks);
-                    ((uint8_t *)c->v)[dst + d] = float_to_e4m3(vx / vs);
+                    ((uint8_t *)c->k)[dst + d] = c->dtype == ORACLE_FP8 ? float_to_e4m3(kx / ks) : float_to_e5m2(kx / ks);
+                    ((uint8_t *)c->v)[dst + d] = c->dtype == ORACLE_FP8 ? float_to_e4m3(vx / vs) : float_to_e5m2(vx / vs);
                 }
             } else {
                 memcpy((char *)c->k + dst * elt_size(c->dtype), (const char *)k_new + src * elt_size(c->dtype),
@@ -720,7 +755,7 @@ int oracle_prefill_seed(oracle_cache *c, const void *q_prompt, int32_t prompt_le
     int st = check_cache(c);
     if (st) return st;
     if (!q_prompt || !scale || prompt_len < 1 || !(gamma > 0.0f && gamma <= 1.0f)) return ORACLE_ERR_INVALID_ARG;
-    if (c->dtype == ORACLE_FP8) return ORACLE_ERR_INVALID_ARG; /* prompt keys are seeded before quantisation */
+    if (ORACLE_IS_FP8(c->dtype)) return ORACLE_ERR_INVALID_ARG; /* prompt keys are seeded before quantisation */
     const int B = c->batch, Hq = c->n_q_heads, Hkv = c->n_kv_heads, D = c->head_dim, P = prompt_len;
     const int G = Hq / Hkv;
     const int64_t capT = cap_tokens(c);

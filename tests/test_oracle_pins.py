@@ -727,3 +727,64 @@ def test_quantised_cache_prunes_by_moving_bytes():
                 assert torch.equal(c.v.view(torch.uint8)[l, b, h, :m], before.v.view(torch.uint8)[l, b, h, idx])
                 assert torch.equal(c.rel[l, b, h, :m], before.rel[l, b, h, idx])
     assert c.len[0, 0].tolist() == [20, 20] and c.len[0, 1].tolist() == [50, 50]
+
+
+def test_e5m2_conversions_against_closed_forms_and_the_library():
+    """The second byte format: e5m2, the upper byte of an IEEE half."""
+    lib = oracle.lib()
+    codes = torch.arange(256, dtype=torch.uint8)
+    ref = codes.view(torch.float8_e5m2).double()
+    got = torch.tensor([lib.oracle_e5m2_decode(int(c)) for c in codes], dtype=torch.float64)
+    assert bool(((ref == got) | (ref.isnan() & got.isnan())).all())
+    for code, value in ((0x3c, 1.0), (0x7b, 57344.0), (0x04, 2.0 ** -14), (0x01, 2.0 ** -16), (0xbc, -1.0), (0x3d, 1.25)):
+        assert lib.oracle_e5m2_decode(code) == value
+        # a byte is the upper half of the half-precision number of the same value
+        assert torch.tensor([code << 8], dtype=torch.int32).to(torch.int16).view(torch.float16).item() == value
+    for c in range(0x7c):                                    # finite codes round-trip; ties go to the even code
+        assert lib.oracle_e5m2_encode(lib.oracle_e5m2_decode(c)) == c
+        if c < 0x7b:
+            mid = 0.5 * (lib.oracle_e5m2_decode(c) + lib.oracle_e5m2_decode(c + 1))
+            assert lib.oracle_e5m2_encode(mid) == (c if c % 2 == 0 else c + 1), c
+            assert lib.oracle_e5m2_encode(float(torch.nextafter(torch.tensor(mid), torch.tensor(1e9)))) == c + 1
+            assert lib.oracle_e5m2_encode(float(torch.nextafter(torch.tensor(mid), torch.tensor(-1e9)))) == c
+    for big in (57345.0, 61440.0, 65536.0, 1e9, 3e38):     # never infinity: saturation
+        assert lib.oracle_e5m2_encode(big) == 0x7b and lib.oracle_e5m2_encode(-big) == 0xfb
+    g = torch.Generator().manual_seed(1)
+    x = (torch.randn(20000, generator=g) * torch.exp(torch.randn(20000, generator=g) * 5)).clamp(-57344, 57344)
+    want = x.to(torch.float8_e5m2).view(torch.uint8)
+    got = torch.tensor([lib.oracle_e5m2_encode(float(v)) for v in x.tolist()], dtype=torch.uint8)
+    assert torch.equal(want, got)
+
+
+def test_e5m2_cache_attends_like_the_cache_of_its_dequantised_values():
+    L, B, Hq, Hkv, D, cap, n = 1, 2, 4, 2, 16, 24, 19
+    g = torch.Generator().manual_seed(14)
+    def codes():
+        c = torch.randint(0, 256, (L, B, Hkv, cap, D), generator=g, dtype=torch.int32)
+        c[(c & 0x7c) == 0x7c] = 0x38                             # no infinities / NaNs
+        c[(c & 0x7f) > 0x48] = 0x40                               # keep magnitudes moderate
+        return c.to(torch.uint8).view(torch.float8_e5m2)
+    k8, v8 = codes(), codes()
+    rel = torch.rand((L, B, Hkv, cap), generator=g)
+    pos = torch.arange(cap, dtype=torch.int32).expand(L, B, Hkv, cap).contiguous()
+    ln = torch.full((L, B, Hkv), n, dtype=torch.int32)
+    q8 = oracle.OracleCache(L, B, Hq, Hkv, D, cap, k8, v8, rel.clone(), pos.clone(), ln.clone(),
+                            k_scale=torch.tensor([0.5]), v_scale=torch.tensor([0.25]))
+    f32 = oracle.OracleCache(L, B, Hq, Hkv, D, cap, k8.float() * 0.5, v8.float() * 0.25, rel.clone(), pos.clone(), ln.clone())
+    q = (torch.randn((L, B, Hq, D), generator=g) * 0.3).to(torch.bfloat16)
+    kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+    kn[0, 0, 0, 0] = 1e9                                          # saturates at 57344 * 0.5, never infinity
+    scale = torch.tensor([0.2], dtype=torch.float32)
+    tp = torch.tensor([3, 4], dtype=torch.int32)
+    st8, out8, _, _ = oracle.decode_attend(q8, 0, L, q, kn, kn, tp, scale, 0.9)
+    # the fp32 twin appends the dequantised bytes the quantised cache stored
+    kq = q8.k.float()[:, :, :, n] * 0.5
+    vq = q8.v.float()[:, :, :, n] * 0.25
+    st32, out32, _, _ = oracle.decode_attend(f32, 0, L, q.float(), kq.reshape(L, B, Hkv, D).contiguous(),
+                                             vq.reshape(L, B, Hkv, D).contiguous(), tp, scale, 0.9)
+    assert st8 == st32 == oracle.OK
+    assert q8.k.view(torch.uint8)[0, 0, 0, n, 0] == 0x7b
+    want = (kn.float() / 0.5).clamp(-57344, 57344).to(torch.float8_e5m2).view(torch.uint8)
+    assert torch.equal(q8.k.view(torch.uint8)[0, :, :, n], want[0])
+    assert torch.equal(q8.rel, f32.rel)
+    assert (out8.float() - out32).abs().max() <= 2.0 ** -8 * out32.abs().max()
