@@ -124,10 +124,11 @@ class Runner:
         self.ctx = binding.Context(device.index)
         self.ctx.set_tuning(variant, splits)
         k, v, rel, pos, ln = make_state(w, device, capacity, w.mean_budget, 1234 + 77 * rank)
-        if kv == "fp8":   # quantised cache: e4m3 bytes, one scale per layer (anchor keys reach about 3 x 4 sigma)
+        if kv != "bf16":   # quantised cache: bytes, one scale per layer (anchor keys reach about 3 x 4 sigma)
+            f8, fmax = (torch.float8_e4m3fn, 448.0) if kv == "fp8" else (torch.float8_e5m2, 57344.0)
             ks, vs = [0.125] * w.n_layers, [0.0625] * w.n_layers
-            k = (k.float() / ks[0]).clamp(-448, 448).to(torch.float8_e4m3fn)
-            v = (v.float() / vs[0]).clamp(-448, 448).to(torch.float8_e4m3fn)
+            k = (k.float() / ks[0]).clamp(-fmax, fmax).to(f8)
+            v = (v.float() / vs[0]).clamp(-fmax, fmax).to(f8)
             self.cache = binding.Cache(w.n_q_heads, k, v, rel, pos, ln, k_scale=ks, v_scale=vs)
         else:
             self.cache = binding.Cache(w.n_q_heads, k, v, rel, pos, ln)
@@ -400,8 +401,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-per-layer", action="store_true")
-    ap.add_argument("--kv", choices=["bf16", "fp8"], default="bf16",
-                    help="storage of K and V: bf16 (the headline configuration) or e4m3 bytes with per-layer scales")
+    ap.add_argument("--kv", choices=["bf16", "fp8", "fp8e5m2"], default="bf16",
+                    help="storage of K and V: bf16 (the headline configuration), or e4m3 / e5m2 bytes with per-layer scales")
     ap.add_argument("--with-prefill", action="store_true",
                     help="also time lethe_prefill_seed on a prompt of the workload's length (informational)")
     ap.add_argument("--pl-variant", type=int, default=0, help="kernel variant of the per-layer launch mode")
@@ -591,7 +592,8 @@ def main():
             "metric": METRIC, "value": dist_util.job_value(units, t_ms), "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": t_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16" if args.kv == "bf16" else "fp8 K/V (e4m3 bytes, per-layer scales), bf16 activations, f16 mma, fp32 accumulation",
+            "dtype": "bf16" if args.kv == "bf16" else
+                     f"fp8 K/V ({'e4m3' if args.kv == 'fp8' else 'e5m2'} bytes, per-layer scales), bf16 activations, f16 mma, fp32 accumulation",
             "data": "synthetic",
             "config": workload_config(w, args, extra={
                 "capacity": capacity, "variant": args.variant, "splits": args.splits,

@@ -66,15 +66,15 @@ typedef enum {
     LETHE_ERR_TOO_LARGE = 8    /* lethe_rasr_prune_static: the cache exceeds LETHE_STATIC_PRUNE_MAX_ENTRIES */
 } lethe_status;
 
-enum { LETHE_F32 = 0, LETHE_BF16 = 1, LETHE_FP8_E4M3 = 2 };
+enum { LETHE_F32 = 0, LETHE_BF16 = 1, LETHE_FP8_E4M3 = 2, LETHE_FP8_E5M2 = 3 };
 enum { LETHE_CONTIG = 0, LETHE_PAGED = 1 };
 
 /* Cache state of all layers (Sec. 4.1: per-layer K, V; Sec. 4.3: the score vector s_t). */
 typedef struct {
     int32_t n_layers, batch, n_q_heads, n_kv_heads;
     int32_t head_dim;    /* 64 or 128 */
-    int32_t dtype;       /* LETHE_F32 or LETHE_BF16: type of k, v, q, k_new, v_new, out.  LETHE_FP8_E4M3: k and v are
-                            e4m3 bytes (see k_scale), q, k_new, v_new, out are bf16 */
+    int32_t dtype;       /* LETHE_F32 or LETHE_BF16: type of k, v, q, k_new, v_new, out.  LETHE_FP8_E4M3 / LETHE_FP8_E5M2:
+                            k and v are bytes of that format (see k_scale), q, k_new, v_new, out are bf16 */
     int32_t layout;      /* LETHE_CONTIG or LETHE_PAGED */
     int32_t capacity;    /* CONTIG: token slots per item.  PAGED: page-table entries per item */
     int32_t page_tokens; /* PAGED: tokens per page (16); CONTIG: ignored */
@@ -84,15 +84,17 @@ typedef struct {
     int32_t *len;        /* [L][B][Hkv]              retained tokens per item                           */
     int32_t *page_table; /* PAGED: [L][B][Hkv][capacity] page ids (never written by the library)       */
     int64_t n_pages;     /* PAGED: pages in each pool                                                    */
-    const float *k_scale; /* LETHE_FP8_E4M3 only: HOST float[L] or NULL (= 1): a stored key byte x means k_scale[l] * x */
+    const float *k_scale; /* byte formats only: HOST float[L] or NULL (= 1): a stored key byte x means k_scale[l] * x */
     const float *v_scale; /* the same for values                                                                      */
 } lethe_cache;
 /* cap_tokens = capacity (CONTIG) or capacity * page_tokens (PAGED).  k, v and rel must be 16-byte aligned.
  *
- * Quantised caches (LETHE_FP8_E4M3).  The paper's related work notes that quantised caches compose with eviction
- * and fixes no format; this library's is: e4m3 bytes (1-4-3, bias 7, no infinities, largest value 448) with one
- * positive scale per layer for keys and one for values.  lethe_decode_attend appends k_new / k_scale[l] and
- * v_new / v_scale[l] (fp32 division, round to nearest even, saturating at +-448) and reads a byte x as exactly
+ * Quantised caches.  The paper's related work notes that quantised caches compose with eviction and fixes no
+ * format; this library offers two byte formats, each with one positive scale per layer for keys and one for values:
+ * LETHE_FP8_E4M3 (1-4-3, bias 7, no infinities, largest value 448) and LETHE_FP8_E5M2 (1-5-2, bias 15, the upper
+ * byte of an IEEE half, largest finite value 57344; coarser, but free to expand).  lethe_decode_attend appends
+ * k_new / k_scale[l] and v_new / v_scale[l] (fp32 division, round to nearest even, saturating at the largest finite
+ * value: no infinity or NaN is ever produced from finite input) and reads a byte x as exactly
  * scale * x; the prune calls move rows as bytes and never look at the storage type.  Supported: head_dim 64 or
  * 128, up to 8 query heads per KV head, contiguous or 16-token pages; lethe_prefill_seed is not (prompt keys are
  * scored before they are quantised). */
@@ -121,9 +123,9 @@ lethe_status lethe_poll_status(lethe_ctx *ctx, void *stream, int32_t *info);
  * 32..37 = the clustered kernel's six shapes with the CTAs of an item merged through global scratch (the last
  * CTA to finish completes the item) instead of a thread-block cluster; splits may then be any value 0..16.
  * Tensor-core variants need a bf16 cache (and 16-token pages when paged).
- * A quantised cache (LETHE_FP8_E4M3) runs its own tensor-core kernels: variants 2..7 force the clustered one with
+ * A quantised cache runs its own tensor-core kernels: variants 2..7 force the clustered one with
  * shape (4,4) (8,4) (4,2) (4,3) (2,4) (8,2) (splits as above), variants 8..13 the persistent one with shape (8,4)
- * (12,3) (10,4) (8,5) (16,2) (12,2); any other value means the clustered kernel with shape (4,4), the faster of
+ * (12,3) (10,4) (8,5) (16,2) (12,2) (e4m3 only); any other value means the clustered kernel with shape (4,4), the faster of
  * the two at every size measured.
  * variant 40..42 select the engine of lethe_prefill_seed and leave everything else as it is: 40 = tcgen05
  * kernels (accumulators in tensor memory, operand tiles by TMA; the default), 41 = mma.sync kernels,

@@ -17,7 +17,7 @@ LIB_PATH = os.environ.get("LETHE_LIB", os.path.join(_HERE, "liblethe.so"))   # L
 
 OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_BUDGET, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED, ERR_PAGE, ERR_TOO_LARGE = range(9)
 STATIC_PRUNE_MAX_ENTRIES = 4 * 1024 * 1024
-F32, BF16, FP8_E4M3 = 0, 1, 2
+F32, BF16, FP8_E4M3, FP8_E5M2 = 0, 1, 2, 3
 CONTIG, PAGED = 0, 1
 VARIANT_AUTO, VARIANT_SIMT, VARIANT_MMA4, VARIANT_MMA8 = 0, 1, 2, 3
 
@@ -104,13 +104,13 @@ class Cache:
 
     def __init__(self, n_q_heads: int, k: torch.Tensor, v: torch.Tensor, rel: torch.Tensor, pos: torch.Tensor,
                  len_: torch.Tensor, page_table: Optional[torch.Tensor] = None, k_scale=None, v_scale=None):
-        """k_scale, v_scale: per-layer scales of a float8_e4m3fn cache (sequences of L floats; None = 1)."""
+        """k_scale, v_scale: per-layer scales of a float8_e4m3fn / float8_e5m2 cache (sequences of L floats; None = 1)."""
         self.k, self.v, self.rel, self.pos, self.len, self.page_table = k, v, rel, pos, len_, page_table
         for t in (k, v, rel, pos, len_) + ((page_table,) if page_table is not None else ()):
             assert t.is_cuda and t.is_contiguous()
         assert rel.dtype == torch.float32 and pos.dtype == torch.int32 and len_.dtype == torch.int32
         L, B, Hkv = len_.shape
-        dt = {torch.float32: F32, torch.bfloat16: BF16, torch.float8_e4m3fn: FP8_E4M3}[k.dtype]
+        dt = {torch.float32: F32, torch.bfloat16: BF16, torch.float8_e4m3fn: FP8_E4M3, torch.float8_e5m2: FP8_E5M2}[k.dtype]
         if page_table is None:
             assert k.dim() == 5 and tuple(k.shape[:3]) == (L, B, Hkv)
             cap, D, layout, pt, npages = k.shape[3], k.shape[4], CONTIG, 0, 0
@@ -127,7 +127,7 @@ class Cache:
                              page_table.data_ptr() if page_table is not None else None, npages, None, None)
         # host arrays of the per-layer scales, kept alive here
         self._k_scale = self._v_scale = None
-        if dt == FP8_E4M3:
+        if dt in (FP8_E4M3, FP8_E5M2):
             for name, sc in (("k_scale", k_scale), ("v_scale", v_scale)):
                 if sc is None:
                     continue
@@ -142,7 +142,7 @@ class Cache:
     @property
     def act_dtype(self) -> torch.dtype:
         """Type of q, k_new, v_new and out."""
-        return torch.bfloat16 if self.k.dtype == torch.float8_e4m3fn else self.k.dtype
+        return torch.bfloat16 if self.k.dtype in (torch.float8_e4m3fn, torch.float8_e5m2) else self.k.dtype
 
     @property
     def device(self):

@@ -12,8 +12,10 @@ namespace lethe {
 cudaError_t launch_attend_simt(const AttendArgs& a, int dtype, int D, bool paged, cudaStream_t stream);
 size_t kv8_smem_bytes(int D, int shape, int chunk_tokens, int GP);
 size_t kv8_stream_smem_bytes(int D, int shape, int chunk_tokens, int GP);
+size_t kv8_async_smem_bytes(int D, int shape, int chunk_tokens, int GP);
+cudaError_t launch_attend_kv8_async(const AttendArgs& a, int D, int shape, bool paged, bool e5m2, int grid, cudaStream_t stream);
 cudaError_t launch_attend_kv8_stream(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream);
-cudaError_t launch_attend_kv8(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream);
+cudaError_t launch_attend_kv8(const AttendArgs& a, int D, int shape, bool paged, bool e5m2, cudaStream_t stream);
 size_t simt_smem_bytes(int D, int chunk_tokens, int GP);
 cudaError_t launch_attend_mma(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream);
 size_t mma_smem_bytes(int D, int shape, int chunk_tokens, int GP);
@@ -152,9 +154,10 @@ lethe_status check_cache(lethe_ctx* ctx, const lethe_cache* c) {
         return fail(ctx, LETHE_ERR_INVALID_ARG, "cache dimensions must be positive");
     if (c->n_q_heads % c->n_kv_heads) return fail(ctx, LETHE_ERR_INVALID_ARG, "n_q_heads must be a multiple of n_kv_heads");
     if (c->head_dim != 64 && c->head_dim != 128) return fail(ctx, LETHE_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
-    if (c->dtype != LETHE_F32 && c->dtype != LETHE_BF16 && c->dtype != LETHE_FP8_E4M3)
+    const bool bytes = c->dtype == LETHE_FP8_E4M3 || c->dtype == LETHE_FP8_E5M2;
+    if (c->dtype != LETHE_F32 && c->dtype != LETHE_BF16 && !bytes)
         return fail(ctx, LETHE_ERR_INVALID_ARG, "unknown dtype");
-    if (c->dtype == LETHE_FP8_E4M3)
+    if (bytes)
         for (int l = 0; l < c->n_layers; ++l) {
             const float ks = c->k_scale ? c->k_scale[l] : 1.f, vs = c->v_scale ? c->v_scale[l] : 1.f;
             if (!(ks > 0.f && ks < 1e30f && vs > 0.f && vs < 1e30f)) return fail(ctx, LETHE_ERR_INVALID_ARG, "k_scale and v_scale must be positive and finite");
@@ -179,7 +182,7 @@ CacheView view_of(const lethe_cache* c) {
     v.k = c->k; v.v = c->v; v.rel = c->rel; v.pos = c->pos; v.len = c->len; v.page_table = c->page_table;
     v.n_pages = c->n_pages;
     v.L = c->n_layers; v.B = c->batch; v.Hkv = c->n_kv_heads; v.D = c->head_dim;
-    v.elt_bytes = c->dtype == LETHE_BF16 ? 2 : (c->dtype == LETHE_FP8_E4M3 ? 1 : 4);
+    v.elt_bytes = c->dtype == LETHE_BF16 ? 2 : (c->dtype == LETHE_F32 ? 4 : 1);
     v.capacity = c->capacity; v.cap_tokens = cap_tokens_of(c);
     v.page_tokens = c->layout == LETHE_PAGED ? c->page_tokens : 1;
     v.paged = c->layout == LETHE_PAGED;
@@ -357,7 +360,7 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
     const int cap_groups = (a.cap_tokens + kGroupTokens - 1) / kGroupTokens;
     int variant = ctx->variant;
 
-    if (c->dtype == LETHE_FP8_E4M3) {
+    if (c->dtype == LETHE_FP8_E4M3 || c->dtype == LETHE_FP8_E5M2) {
         // quantised cache: its own clustered tensor-core kernel; variants 2..7 pick its shape, the rest mean "default"
         if (paged && c->page_tokens != kGroupTokens) return fail(ctx, LETHE_ERR_UNSUPPORTED, "quantised caches need 16-token pages");
         if (c->n_layers > kMaxLayers) return fail(ctx, LETHE_ERR_UNSUPPORTED, "more than 128 layers");
@@ -369,9 +372,31 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         // The clustered kernel (variants 2..7 pick its shape) is the default at every size: with two CTAs per SM
         // covering each other's epilogues it beats the persistent one (variants 8..13) on this conversion-bound
         // path (Llama-8B shape: 0.137 ms against 0.154 to 0.166 ms).
+        // variants 16..21: the persistent kernel with an asynchronous epilogue (both formats)
+        if (variant >= 16 && variant <= 21 && ctx->splits <= 1) {
+            const int ashape = variant - 16;
+            const size_t fixed = kv8_async_smem_bytes(c->head_dim, ashape, 0, a.GP);
+            int fit = 0;
+            if (fixed < ctx->max_smem) fit = (int)((ctx->max_smem - fixed) / ((size_t)2 * a.GP * 4) / kGroupTokens) * kGroupTokens;
+            a.splits = 1;
+            a.chunk_tokens = fit < cap_groups * kGroupTokens ? fit : cap_groups * kGroupTokens;
+            if (a.chunk_tokens < kGroupTokens)
+                return fail(ctx, LETHE_ERR_UNSUPPORTED, "no shared memory left for the logit buffers of this persistent shape");
+            const int grid = a.n_items < ctx->sm_count ? a.n_items : ctx->sm_count;
+            if (a.chunk_tokens < cap_groups * kGroupTokens) {
+                a.spill_tokens = cap_groups * kGroupTokens - a.chunk_tokens;
+                const size_t need = (size_t)grid * 2 * a.spill_tokens * a.GP * sizeof(float);
+                st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "logit overflow scratch");
+                if (st != LETHE_OK) return st;
+                a.spill = (float*)ctx->scratch;
+            }
+            const cudaError_t ea = launch_attend_kv8_async(a, c->head_dim, ashape, paged, c->dtype == LETHE_FP8_E5M2, grid, (cudaStream_t)stream);
+            if (ea != cudaSuccess) return cuda_fail(ctx, ea, "decode_attend launch (quantised cache, asynchronous epilogue)");
+            return LETHE_OK;
+        }
         const bool want_persistent = variant >= 8 && variant <= 13;
         const bool want_clustered = variant >= 2 && variant <= 7;
-        if (want_persistent && ctx->splits <= 1) {
+        if (want_persistent && ctx->splits <= 1 && c->dtype == LETHE_FP8_E4M3) {
             const int pshape = variant - 8;
             const size_t fixed = kv8_stream_smem_bytes(c->head_dim, pshape, 0, a.GP);
             int fit = 0;
@@ -407,7 +432,7 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
             return fail(ctx, LETHE_ERR_UNSUPPORTED, "capacity too large for the on-chip logit buffer at this split count");
         a.splits = S;
         a.chunk_tokens = ((cap_groups + S - 1) / S) * kGroupTokens;
-        const cudaError_t e8 = launch_attend_kv8(a, c->head_dim, shape, paged, (cudaStream_t)stream);
+        const cudaError_t e8 = launch_attend_kv8(a, c->head_dim, shape, paged, c->dtype == LETHE_FP8_E5M2, (cudaStream_t)stream);
         if (e8 != cudaSuccess) return cuda_fail(ctx, e8, "decode_attend launch (quantised cache)");
         return LETHE_OK;
     }

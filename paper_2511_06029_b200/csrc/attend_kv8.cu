@@ -1,5 +1,5 @@
-// Decode-attend kernel for quantised caches: K and V stored as e4m3 bytes with one scale per layer (a stored byte
-// x means scale * x), q / k_new / v_new / out in bf16.  D in {64, 128}, G <= 8, contiguous or 16-token pages.
+// Decode-attend kernel for quantised caches: K and V stored as e4m3 or e5m2 bytes with one scale per layer (a
+// stored byte x means scale * x), q / k_new / v_new / out in bf16.  D in {64, 128}, G <= 8, contiguous or 16-token pages.
 //
 // Same structure as the clustered bf16 kernel (tokens on the M axis of mma.m16n8k16, the group's heads on N, one
 // private cp.async pipeline per warp, logits parked in shared memory, CTAs of an item merged through distributed
@@ -12,7 +12,8 @@
 //                   consecutive tokens; a byte permute separates even and odd d, giving the A fragments of two
 //                   MMAs whose rows are the even and the odd dimensions of a 32-wide block.  Only the bookkeeping
 //                   of which accumulator row is which dimension changes.
-// e4m3 -> f16 is exact, the MMAs run in f16 with fp32 accumulation; P is rounded to f16.  The layer's key scale is
+// Byte -> f16 is exact (a conversion instruction per pair for e4m3, for e5m2 the byte permute alone: an e5m2 byte is
+// the upper byte of the half of the same value); the MMAs run in f16 with fp32 accumulation; P is rounded to f16.  The layer's key scale is
 // folded into the softmax scale on the host, the value scale multiplies the warp's partial output once.
 // Appending quantises: x / scale in fp32 (IEEE division), round to nearest even, saturate at +-448.
 #include <cuda_fp16.h>
@@ -36,14 +37,25 @@ __device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t x) {
     asm("{ .reg .b16 lo; cvt.u16.u32 lo, %1; cvt.rn.f16x2.e4m3x2 %0, lo; }" : "=r"(y) : "r"(x));
     return y;
 }
+// Bytes `sel_lo` and `sel_hi` (0..3) of x -> f16x2.  An e5m2 byte is the upper byte of the half of the same value,
+// so one byte permute does it; e4m3 goes through the conversion instruction.
+template <bool E5M2, int SEL_LO, int SEL_HI>
+__device__ __forceinline__ uint32_t bytes_to_f16x2(uint32_t x) {
+    if constexpr (E5M2) return __byte_perm(x, 0u, 0x0404 | (SEL_LO << 4) | (SEL_HI << 12));  // [0, lo, 0, hi]
+    else if constexpr (SEL_LO == 0 && SEL_HI == 1) return e4m3x2_to_f16x2(x);                 // the low 16 bits as they are
+    else if constexpr (SEL_LO == 2 && SEL_HI == 3) return e4m3x2_to_f16x2(x >> 16);
+    else return e4m3x2_to_f16x2(__byte_perm(x, 0u, 0x4400 | SEL_LO | (SEL_HI << 4)));        // [lo, hi, 0, 0]
+}
 __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
     __half2 v = __floats2half2_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
 // two fp32 -> two e4m3 bytes (round to nearest even, saturating), `lo` in the low byte
-__device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi) {
+template <bool E5M2>
+__device__ __forceinline__ uint32_t f32x2_to_fp8x2(float lo, float hi) {
     uint32_t y;
-    asm("{ .reg .b16 r; cvt.rn.satfinite.e4m3x2.f32 r, %2, %1; cvt.u32.u16 %0, r; }" : "=r"(y) : "f"(lo), "f"(hi));
+    if (E5M2) asm("{ .reg .b16 r; cvt.rn.satfinite.e5m2x2.f32 r, %2, %1; cvt.u32.u16 %0, r; }" : "=r"(y) : "f"(lo), "f"(hi));
+    else asm("{ .reg .b16 r; cvt.rn.satfinite.e4m3x2.f32 r, %2, %1; cvt.u32.u16 %0, r; }" : "=r"(y) : "f"(lo), "f"(hi));
     return y;
 }
 // bf16 pair (as stored) -> f16x2
@@ -54,7 +66,7 @@ __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t x) {
 
 }  // namespace
 
-template <int D, int NW, int NSTAGE, bool PAGED>
+template <int D, int NW, int NSTAGE, bool PAGED, bool E5M2>
 __global__ void __launch_bounds__(NW * 32) attend_kv8_kernel(const __grid_constant__ AttendArgs a) {
     using T = __nv_bfloat16;                               // type of q, k_new, v_new, out
     constexpr int ROW_BYTES = D;                           // one byte per element
@@ -128,7 +140,7 @@ __global__ void __launch_bounds__(NW * 32) attend_kv8_kernel(const __grid_consta
             auto quant4 = [](uint2 w, float s) -> uint32_t {
                 const float x0 = __uint_as_float(w.x << 16), x1 = __uint_as_float(w.x & 0xffff0000u);
                 const float x2 = __uint_as_float(w.y << 16), x3 = __uint_as_float(w.y & 0xffff0000u);
-                return f32x2_to_e4m3x2(__fdiv_rn(x0, s), __fdiv_rn(x1, s)) | (f32x2_to_e4m3x2(__fdiv_rn(x2, s), __fdiv_rn(x3, s)) << 16);
+                return f32x2_to_fp8x2<E5M2>(__fdiv_rn(x0, s), __fdiv_rn(x1, s)) | (f32x2_to_fp8x2<E5M2>(__fdiv_rn(x2, s), __fdiv_rn(x3, s)) << 16);
             };
             *reinterpret_cast<uint32_t*>(kd + lane * 4) = quant4(kw, ks_l);
             *reinterpret_cast<uint32_t*>(vd + lane * 4) = quant4(vw, vs_l);
@@ -210,8 +222,10 @@ __global__ void __launch_bounds__(NW * 32) attend_kv8_kernel(const __grid_consta
         for (int pr = 0; pr < KS / 2; ++pr) {  // 32 bytes of every key row: two k-steps
             uint32_t r[4];                     // rows gq | gq + 8 of bytes [32 pr, +16) | rows gq | gq + 8 of [32 pr + 16, +16)
             ldmatrix_x4(ks_u32 + swz(k_row, 2 * pr + k_chunk), r);
-            const uint32_t a0[4] = {e4m3x2_to_f16x2(r[0]), e4m3x2_to_f16x2(r[1]), e4m3x2_to_f16x2(r[0] >> 16), e4m3x2_to_f16x2(r[1] >> 16)};
-            const uint32_t a1[4] = {e4m3x2_to_f16x2(r[2]), e4m3x2_to_f16x2(r[3]), e4m3x2_to_f16x2(r[2] >> 16), e4m3x2_to_f16x2(r[3] >> 16)};
+            const uint32_t a0[4] = {bytes_to_f16x2<E5M2, 0, 1>(r[0]), bytes_to_f16x2<E5M2, 0, 1>(r[1]),
+                                    bytes_to_f16x2<E5M2, 2, 3>(r[0]), bytes_to_f16x2<E5M2, 2, 3>(r[1])};
+            const uint32_t a1[4] = {bytes_to_f16x2<E5M2, 0, 1>(r[2]), bytes_to_f16x2<E5M2, 0, 1>(r[3]),
+                                    bytes_to_f16x2<E5M2, 2, 3>(r[2]), bytes_to_f16x2<E5M2, 2, 3>(r[3])};
             mma_f16(ca, a0, bq[2 * pr][0], bq[2 * pr][1]);
             mma_f16(cb, a1, bq[2 * pr + 1][0], bq[2 * pr + 1][1]);
         }
@@ -262,8 +276,8 @@ __global__ void __launch_bounds__(NW * 32) attend_kv8_kernel(const __grid_consta
             uint32_t ae[4], ao[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                ae[i] = e4m3x2_to_f16x2(__byte_perm(r[i], 0u, 0x4420));  // even d: bytes 0 and 2 (tokens t, t+1)
-                ao[i] = e4m3x2_to_f16x2(__byte_perm(r[i], 0u, 0x4431));  // odd d:  bytes 1 and 3
+                ae[i] = bytes_to_f16x2<E5M2, 0, 2>(r[i]);  // even d: bytes 0 and 2 (tokens t, t+1)
+                ao[i] = bytes_to_f16x2<E5M2, 1, 3>(r[i]);  // odd d:  bytes 1 and 3
             }
             mma_f16(o[mt][0], ae, pb0, pb1);
             mma_f16(o[mt][1], ao, pb0, pb1);
@@ -311,9 +325,9 @@ static size_t kv8_smem(int chunk_tokens, int GP) {
            (size_t)chunk_tokens * GP * 4;
 }
 
-template <int D, int NW, int NSTAGE, bool PAGED>
+template <int D, int NW, int NSTAGE, bool PAGED, bool E5M2>
 static cudaError_t launch_kv8_t(const AttendArgs& a, cudaStream_t stream) {
-    auto kern = attend_kv8_kernel<D, NW, NSTAGE, PAGED>;
+    auto kern = attend_kv8_kernel<D, NW, NSTAGE, PAGED, E5M2>;
     const size_t smem = kv8_smem<D, NW, NSTAGE>(a.chunk_tokens, a.GP);
     cudaError_t e = prepare_kernel((const void*)kern, smem);
     if (e != cudaSuccess) return e;
@@ -345,10 +359,12 @@ size_t kv8_smem_bytes(int D, int shape, int chunk_tokens, int GP) {
     return (size_t)-1;
 }
 
-cudaError_t launch_attend_kv8(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream) {
-#define X(id, DD, NW, NS)                                                              \
-    if (shape == id && D == DD)                                                        \
-        return paged ? launch_kv8_t<DD, NW, NS, true>(a, stream) : launch_kv8_t<DD, NW, NS, false>(a, stream);
+cudaError_t launch_attend_kv8(const AttendArgs& a, int D, int shape, bool paged, bool e5m2, cudaStream_t stream) {
+#define X(id, DD, NW, NS)                                                                                           \
+    if (shape == id && D == DD) {                                                                                   \
+        if (e5m2) return paged ? launch_kv8_t<DD, NW, NS, true, true>(a, stream) : launch_kv8_t<DD, NW, NS, false, true>(a, stream); \
+        return paged ? launch_kv8_t<DD, NW, NS, true, false>(a, stream) : launch_kv8_t<DD, NW, NS, false, false>(a, stream);         \
+    }
     LETHE_KV8_SHAPES(X, 128)
     LETHE_KV8_SHAPES(X, 64)
 #undef X

@@ -1,0 +1,775 @@
+// Persistent decode-attend kernel with an asynchronous epilogue for quantised caches (K / V as e4m3 or e5m2 bytes with
+// one scale per layer, bf16 activations; D in {64, 128}, G <= 8).  The schedule, the work queue, the epilogue warps
+// and the double-buffered logits are those of the bf16 kernel of the same design (attend_async.cu); the streaming
+// warps build their MMA fragments from bytes as the clustered quantised kernel does (attend_kv8.cu): f16 MMAs, the
+// key bytes' permuted contraction order matched by the Q^T fragments, even / odd output dimensions separated by a
+// byte permute on the V side, the key scale folded into the softmax scale, the value scale applied to each warp's
+// partial output, and an append that quantises (fp32 division, round to nearest even, saturate).  Tiles are staged
+// with 16-byte cp.async only.
+#include <cuda_fp16.h>
+
+#include "common.cuh"
+#include "mma_utils.cuh"
+
+#include <string.h>
+
+#include <cuda.h>  // CUtensorMap (type only: the encoder is resolved at run time by the host code)
+
+namespace lethe {
+namespace {
+
+__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t x) {
+    uint32_t y;
+    asm("{ .reg .b16 lo; cvt.u16.u32 lo, %1; cvt.rn.f16x2.e4m3x2 %0, lo; }" : "=r"(y) : "r"(x));
+    return y;
+}
+// Bytes SEL_LO and SEL_HI (0..3) of x -> f16x2: a byte permute for e5m2 (the upper byte of the half of the same value), the
+// conversion instruction for e4m3.
+template <bool E5M2, int SEL_LO, int SEL_HI>
+__device__ __forceinline__ uint32_t bytes_to_f16x2(uint32_t x) {
+    if constexpr (E5M2) return __byte_perm(x, 0u, 0x0404 | (SEL_LO << 4) | (SEL_HI << 12));
+    else if constexpr (SEL_LO == 0 && SEL_HI == 1) return e4m3x2_to_f16x2(x);
+    else if constexpr (SEL_LO == 2 && SEL_HI == 3) return e4m3x2_to_f16x2(x >> 16);
+    else return e4m3x2_to_f16x2(__byte_perm(x, 0u, 0x4400 | SEL_LO | (SEL_HI << 4)));
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+template <bool E5M2>
+__device__ __forceinline__ uint32_t f32x2_to_fp8x2(float lo, float hi) {
+    uint32_t y;
+    if (E5M2) asm("{ .reg .b16 r; cvt.rn.satfinite.e5m2x2.f32 r, %2, %1; cvt.u32.u16 %0, r; }" : "=r"(y) : "f"(lo), "f"(hi));
+    else asm("{ .reg .b16 r; cvt.rn.satfinite.e4m3x2.f32 r, %2, %1; cvt.u32.u16 %0, r; }" : "=r"(y) : "f"(lo), "f"(hi));
+    return y;
+}
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t x) {
+    return pack_f16(__uint_as_float(x << 16), __uint_as_float(x & 0xffff0000u));
+}
+
+constexpr int kEpilogueWarps = 2;
+constexpr int kWaitLimit = 200000;  // polls of a blocking try_wait before giving up
+
+// Tensor maps of K and V for the TMA variant (rows x D, box 16 rows x 64 elements, 128-byte swizzle).
+struct alignas(64) TmaMaps {
+    CUtensorMap k, v;
+};
+
+struct AsyncHeader {
+    unsigned long long tma_full[16][6];  // TMA variant: per warp, per stage slot: the tile has landed
+    unsigned long long full[2];   // streaming warps -> epilogue: item's partials are complete
+    unsigned long long empty[2];  // epilogue -> streaming warps: parity buffers are free, next descriptor is published
+    int desc_ticket[4];           // ring by item sequence number: ticket (>= n_items: no more work)
+    int desc_n_old[4];            //                              len of that item before this call
+    int abort;
+    int pad[3];
+    float2 wstat[2][16][kMaxGroup];
+};
+
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+    asm volatile("{ .reg .b64 st; mbarrier.arrive.shared::cta.b64 st, [%0]; }" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, unsigned bytes) {
+    asm volatile("{ .reg .b64 st; mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+// One box (64 elements x 16 rows) of a 2-D tensor map into shared memory; completion is counted on `bar`.
+// x is always 0 or 64 elements (a multiple of 16 bytes), y is a row index.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, unsigned long long* bar,
+                                            uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// Bounded wait for a tile: polls without backing off for a long while (the data is usually microseconds away).
+__device__ __forceinline__ bool mbar_wait_tile(unsigned long long* bar, unsigned parity, volatile int* abort_flag) {
+    for (int it = 0; it < kWaitLimit * 8; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 1023) == 1023) {
+            if (*abort_flag) return false;
+            __nanosleep(200);
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+// Bounded wait; false = gave up (or another warp already did).
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, volatile int* abort_flag) {
+    for (int it = 0; it < kWaitLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (it > 16) __nanosleep(100);
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+struct AsyncItem {
+    int valid;
+    int item, li, l, b, hkv;
+    int n_old, n, full;
+    int count, app_idx;  // streaming warps only
+};
+
+__device__ __forceinline__ void async_decode(const AttendArgs& a, int ticket, int n_old, AsyncItem& it) {
+    it.valid = ticket < a.n_items;
+    const int t = it.valid ? ticket : 0;
+    it.hkv = t % a.Hkv;
+    it.b = (t / a.Hkv) % a.B;
+    it.li = t / (a.Hkv * a.B);
+    it.l = a.layer_begin + it.li;
+    it.item = (it.l * a.B + it.b) * a.Hkv + it.hkv;
+    const bool append = a.k_new != nullptr;
+    it.n_old = n_old;
+    it.full = append && n_old >= a.cap_tokens;
+    it.n = it.full ? 0 : n_old + (append ? 1 : 0);
+    it.count = 0;
+    it.app_idx = -1;
+}
+
+// Sec. 4.1: the generated token's k / v row enters the cache, quantised (kept out of line: once per item).
+template <bool PAGED, bool E5M2>
+__device__ __noinline__ void append_row_q(const AttendArgs& a, int item, int li, int l, int b, int hkv, int n_old, int D, int lane) {
+    using T = __nv_bfloat16;
+    const size_t src = ((size_t)(li * a.B + b) * a.Hkv + hkv) * D;  // elements
+    bool bad = false;
+    char* kd = const_cast<char*>(row_ptr<PAGED>(a, a.k, item, n_old, D, &bad));
+    char* vd = const_cast<char*>(row_ptr<PAGED>(a, a.v, item, n_old, D, &bad));
+    if (kd && vd && lane * 4 < D) {  // four elements per lane
+        const float ks_l = a.k_scale[l], vs_l = a.v_scale[l];
+        const uint2 kw = *reinterpret_cast<const uint2*>((const T*)a.k_new + src + lane * 4);
+        const uint2 vw = *reinterpret_cast<const uint2*>((const T*)a.v_new + src + lane * 4);
+        auto quant4 = [](uint2 w, float sc) -> uint32_t {
+            const float x0 = __uint_as_float(w.x << 16), x1 = __uint_as_float(w.x & 0xffff0000u);
+            const float x2 = __uint_as_float(w.y << 16), x3 = __uint_as_float(w.y & 0xffff0000u);
+            return f32x2_to_fp8x2<E5M2>(__fdiv_rn(x0, sc), __fdiv_rn(x1, sc)) | (f32x2_to_fp8x2<E5M2>(__fdiv_rn(x2, sc), __fdiv_rn(x3, sc)) << 16);
+        };
+        *reinterpret_cast<uint32_t*>(kd + lane * 4) = quant4(kw, ks_l);
+        *reinterpret_cast<uint32_t*>(vd + lane * 4) = quant4(vw, vs_l);
+    }
+    if (lane == 0) a.pos[(size_t)item * a.cap_tokens + n_old] = a.token_pos[b];
+    __syncwarp();
+}
+
+template <int D, int NWS, int NS, bool PAGED, bool SPILL, bool E5M2>
+__global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
+    attend_kv8_async_kernel(const __grid_constant__ AttendArgs a, const __grid_constant__ TmaMaps maps) {
+    using T = __nv_bfloat16;
+    constexpr bool TMA = false;                     // byte tiles are staged with cp.async only
+    constexpr int ROW_BYTES = D;                    // one byte per element
+    constexpr int CHUNKS = ROW_BYTES / 16;
+    constexpr int ROWS_PER_LINE = 128 / ROW_BYTES;  // rows sharing a 128-byte line of shared memory
+    constexpr int MT = D / 32;                      // 32-wide blocks of the output dimension
+    // bank-conflict-free placement of 16-byte chunk c of row r
+    auto swz = [](int r, int c) -> uint32_t {
+        return (uint32_t)(r * ROW_BYTES + ((c ^ ((r / ROWS_PER_LINE) & (CHUNKS - 1))) << 4));
+    };
+    constexpr int TILE_BYTES = kGroupTokens * ROW_BYTES;
+    constexpr int STAGE_BYTES = 2 * TILE_BYTES;
+    constexpr int WARP_BYTES = NS * STAGE_BYTES;
+    constexpr int KS = D / 16;
+    constexpr int ET = kEpilogueWarps * 32;
+    static_assert(NS >= 2 && NS <= 6 && NWS <= 16, "shape");
+    extern __shared__ __align__(1024) unsigned char smem_raw[];  // TMA tiles with a 128-byte swizzle need 1 KB alignment
+    // layout: stages [NWS][NS][K tile | V tile] | AsyncHeader | wo [2][NWS][GP][D] fp32 | lg [2][chunk][GP] fp32
+    // Tile layout.  cp.async: rows of ROW_BYTES with the 16-byte chunk index XORed by (row & 7).  TMA: one 2 KB box
+    // per 64 elements of D (16 rows x 128 B, chunk index XORed by (row & 7) by the hardware swizzle).
+    const int G = a.G, GP = a.GP;
+    const int wo_stride = GP * D;  // floats per warp
+    AsyncHeader& hd = *reinterpret_cast<AsyncHeader*>(smem_raw + (size_t)NWS * WARP_BYTES);
+    float* wo_all = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(&hd) + sizeof(AsyncHeader));
+    float* lg_all = wo_all + (size_t)2 * NWS * wo_stride;
+    const int chunk = a.chunk_tokens;
+    float* spill_all = SPILL ? a.spill + (size_t)blockIdx.x * 2 * a.spill_tokens * GP : nullptr;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool append = a.k_new != nullptr;
+    unsigned int* sched = a.sched;
+    volatile int* abort_flag = &hd.abort;
+
+    // ---- set-up: barriers, first two descriptors
+    bool drew_fail = false;  // meaningful in the ticket-drawing lane only
+    if (tid == 0) {
+        mbar_init(&hd.full[0], NWS);
+        mbar_init(&hd.full[1], NWS);
+        mbar_init(&hd.empty[0], kEpilogueWarps);
+        mbar_init(&hd.empty[1], kEpilogueWarps);
+        if (TMA)
+            for (int w = 0; w < NWS; ++w)
+                for (int sl = 0; sl < NS; ++sl) mbar_init(&hd.tma_full[w][sl], 1);
+        hd.abort = 0;
+    }
+    if (TMA && (smem_u32(smem_raw) & 1023u)) {  // would break the hardware swizzle: refuse rather than compute garbage
+        if (tid == 0) record_error(a.status, LETHE_ERR_UNSUPPORTED, (int)blockIdx.x);
+        // still take part in the queue protocol so that the launch ends cleanly
+        if (tid == 0) {
+            (void)atomicAdd(&sched[0], 1u);
+            __threadfence();
+            const unsigned int done = atomicAdd(&sched[1], 1u);
+            if (done == gridDim.x - 1) {
+                sched[0] = 0u;
+                sched[1] = 0u;
+            }
+        }
+        return;
+    }
+    if (warp == NWS && lane == 0) {
+        int t0 = (int)atomicAdd(&sched[0], 1u);
+        int t1 = a.n_items;
+        if (t0 >= a.n_items) drew_fail = true;
+        else {
+            t1 = (int)atomicAdd(&sched[0], 1u);
+            if (t1 >= a.n_items) drew_fail = true;
+        }
+        if (a.order) {  // longest-first order of the items (valid tickets only)
+            if (t0 < a.n_items) t0 = a.order[t0];
+            if (t1 < a.n_items) t1 = a.order[t1];
+        }
+        AsyncItem tmp;
+        async_decode(a, t0, 0, tmp);
+        hd.desc_ticket[0] = t0;
+        hd.desc_n_old[0] = tmp.valid ? a.len[tmp.item] : 0;
+        async_decode(a, t1, 0, tmp);
+        hd.desc_ticket[1] = t1;
+        hd.desc_n_old[1] = tmp.valid ? a.len[tmp.item] : 0;
+    }
+    __syncthreads();
+
+    if (warp < NWS) {
+        // =================================================================== streaming warps
+        const int gq = lane >> 2, tq = lane & 3;
+        auto load_q = [&](const AsyncItem& it, uint32_t (&bq)[KS][2]) {
+            // f16, in the permuted order of the key bytes: b0 = Q[head gq][16 ks + 4 tq + {0, 1}], b1 = ... + {2, 3}
+            const uint2* qrow = reinterpret_cast<const uint2*>(
+                (const T*)a.q + ((size_t)(it.li * a.B + it.b) * a.Hq + it.hkv * G + gq) * D);
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                uint2 w = make_uint2(0u, 0u);
+                if (it.valid && gq < G) w = qrow[4 * ks + tq];
+                bq[ks][0] = bf16x2_to_f16x2(w.x);
+                bq[ks][1] = bf16x2_to_f16x2(w.y);
+            }
+        };
+        auto set_counts = [&](AsyncItem& it) {
+            const int ng = (it.n + kGroupTokens - 1) / kGroupTokens;
+            it.count = ng > warp ? (ng - warp + NWS - 1) / NWS : 0;
+            it.app_idx = -1;
+            if (append && !it.full && it.valid) {
+                const int g = it.n_old / kGroupTokens;
+                if (g % NWS == warp) it.app_idx = g / NWS;
+            }
+        };
+        unsigned char* my_stage = smem_raw + (size_t)warp * WARP_BYTES;
+        const uint32_t my_stage_u32 = smem_u32(my_stage);
+        bool bad_page = false;
+        const uint64_t stream_policy = l2_evict_first_policy();  // K / V tiles are read once: evict-first in L2
+        unsigned slot_bad = 0;    // TMA: slots whose tile must be ignored (page id outside the pool)
+        unsigned slot_phase = 0;  // TMA: parity of the next completion of each slot's mbarrier
+        unsigned slot_busy = 0;   // TMA: slots with a load in flight or landed but not yet consumed
+
+        // PAGED: page ids of this warp's local groups are fetched 32 at a time, one lane each, a block ahead of
+        // their use, so that staging a group never waits on a page-table load.
+        int pg_lo = 0, pg_hi = 0, pg_nxt = 0;  // current item: blocks pg_blk and pg_blk + 1; next item: block 0
+        int pg_blk = 0;
+        auto load_pages = [&](const AsyncItem& it, int blk) -> int {
+            const int g = blk * 32 + lane;
+            return (PAGED && it.valid && g < it.count) ? a.page_table[(size_t)it.item * a.capacity + warp + g * NWS] : 0;
+        };
+        auto issue = [&](const AsyncItem& it, int idx, int slot, bool is_cur) {
+            const int grp = warp + idx * NWS;
+            const int tok0 = grp * kGroupTokens;
+            if (idx == it.app_idx) {
+                append_row_q<PAGED, E5M2>(a, it.item, it.li, it.l, it.b, it.hkv, it.n_old, D, lane);
+                if (TMA) {  // the row was written through the generic proxy; the TMA load reads through the async proxy
+                    fence_proxy_async();
+                    __syncwarp();
+                }
+            }
+            const char* kb;
+            const char* vb;
+            bool ok = true;
+            if (PAGED) {
+                int page;
+                if (!is_cur) page = __shfl_sync(0xffffffffu, pg_nxt, idx & 31);  // only the first NS-1 groups
+                else {
+                    if ((idx >> 5) > pg_blk) {  // first group of the next block: rotate and fetch one more ahead
+                        pg_lo = pg_hi;
+                        ++pg_blk;
+                        pg_hi = load_pages(it, pg_blk + 1);
+                    }
+                    page = __shfl_sync(0xffffffffu, pg_lo, idx & 31);
+                }
+                ok = page >= 0 && page < a.n_pages;
+                if (!ok) bad_page = true;
+                const size_t off = (size_t)(ok ? page : 0) * TILE_BYTES;
+                kb = (const char*)a.k + off;
+                vb = (const char*)a.v + off;
+            } else {
+                const size_t off = ((size_t)it.item * a.capacity + tok0) * ROW_BYTES;
+                kb = (const char*)a.k + off;
+                vb = (const char*)a.v + off;
+            }
+            const uint32_t ks_u32 = my_stage_u32 + slot * STAGE_BYTES;
+            const uint32_t vs_u32 = ks_u32 + TILE_BYTES;
+            if constexpr (TMA) {
+                // row index of the group's first token in the 2-D view of the cache (rows x D)
+                const long long row0 = (long long)((kb - (const char*)a.k) / ROW_BYTES);
+                if (!ok) slot_bad |= 1u << slot;
+                else slot_bad &= ~(1u << slot);
+                slot_busy |= 1u << slot;
+                if (lane == 0) {
+                    unsigned long long* bar = &hd.tma_full[warp][slot];
+                    mbar_arrive_expect_tx(bar, STAGE_BYTES);
+#pragma unroll
+                    for (int hx = 0; hx < D / 64; ++hx) {
+                        tma_load_2d(ks_u32 + hx * 2048, &maps.k, hx * 64, (int)row0, bar, stream_policy);
+                        tma_load_2d(vs_u32 + hx * 2048, &maps.v, hx * 64, (int)row0, bar, stream_policy);
+                    }
+                }
+                return;
+            }
+#pragma unroll
+            for (int i = 0; i < kGroupTokens * CHUNKS / 32; ++i) {
+                const int c_idx = i * 32 + lane;
+                const int r = c_idx / CHUNKS, c = c_idx % CHUNKS;
+                const bool valid = ok && (tok0 + r < it.n);
+                const int soff = valid ? r * ROW_BYTES + c * 16 : 0;
+                const uint32_t doff = swz(r, c);
+                cp_async16_hint(ks_u32 + doff, kb + soff, valid ? 16 : 0, stream_policy);
+                cp_async16_hint(vs_u32 + doff, vb + soff, valid ? 16 : 0, stream_policy);
+            }
+        };
+
+        const int k_row = (lane & 7) + ((lane >> 3) & 1) * 8, k_chunk = lane >> 4;
+        const int v_row = (lane & 7) + ((lane >> 4) & 1) * 8, v_chunk = (lane >> 3) & 1;
+
+        AsyncItem cur, nxt;
+        async_decode(a, hd.desc_ticket[0], hd.desc_n_old[0], cur);
+        set_counts(cur);
+        uint32_t bq[KS][2], bqn[KS][2];
+        load_q(cur, bq);
+        pg_lo = load_pages(cur, 0);
+        pg_hi = load_pages(cur, 1);
+        nxt.valid = 0;
+        int seq = 0;          // sequence number of the current item within this CTA
+        int vp = 0;           // stage slot of the current item's local group 0
+        unsigned issued = 0;  // bit j: local group j (< NS-1) of the current item was prefetched by the previous tail
+        bool alive = true;
+
+        while (cur.valid && alive) {
+            const int p = seq & 1;
+            const float sl2 = a.scale_log2[cur.l];
+            const uint32_t lg_u32 = smem_u32(lg_all + (size_t)p * chunk * GP);
+            float* spill = SPILL ? spill_all + (size_t)p * a.spill_tokens * GP : nullptr;
+            bool nxt_ready = false;
+            // descriptor of the next item: wait until the epilogue of item seq-1 (same parity as seq+1) has
+            // handed its buffers back, which also publishes that descriptor
+            auto acquire_next = [&]() {
+                const int sn = seq + 1;
+                if (sn >= 2 && !mbar_wait(&hd.empty[sn & 1], (unsigned)(((sn >> 1) - 1) & 1), abort_flag)) {
+                    alive = false;
+                    nxt.valid = 0;
+                } else {
+                    async_decode(a, hd.desc_ticket[sn & 3], hd.desc_n_old[sn & 3], nxt);
+                    set_counts(nxt);
+                    load_q(nxt, bqn);
+                    pg_nxt = load_pages(nxt, 0);
+                }
+                nxt_ready = true;
+            };
+
+            bool topped = false;
+#pragma unroll
+            for (int j = 0; j < NS - 1; ++j) {
+                if (!((issued >> j) & 1u) && j < cur.count) {
+                    issue(cur, j, (vp + j) % NS, true);
+                    topped = true;
+                }
+            }
+            if (topped) cp_async_commit();
+            unsigned issued_next = 0;
+
+            float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+            float o[KS][4];
+#pragma unroll
+            for (int mt = 0; mt < KS; ++mt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) o[mt][i] = 0.f;
+
+            constexpr bool OVF = SPILL;
+            for (int it = 0; it < cur.count; ++it) {
+                const int cslot = (vp + it) % NS;
+                // Refill first, wait second: the slot of group it-1 is free as soon as every lane has left the
+                // previous iteration, so the copy of the group NS-1 ahead (possibly of the next item) is already
+                // in flight while this warp waits for group `it`.
+                __syncwarp();
+                const bool strict = !TMA && topped && it < NS - 1;  // after a top-up the group order is not the commit order
+                if (strict) cp_async_wait<0>();
+                {
+                    const int idx = it + NS - 1;
+                    const int slot = (vp + idx) % NS;
+                    if (idx < cur.count) issue(cur, idx, slot, true);
+                    else {
+                        if (!nxt_ready) acquire_next();
+                        const int j = idx - cur.count;
+                        if (nxt.valid && j < nxt.count) {
+                            issue(nxt, j, slot, false);
+                            issued_next |= 1u << j;
+                        }
+                    }
+                    cp_async_commit();
+                }
+                if constexpr (TMA) {
+                    if (!mbar_wait_tile(&hd.tma_full[warp][cslot], (slot_phase >> cslot) & 1u, abort_flag)) {
+                        alive = false;
+                        break;
+                    }
+                    slot_phase ^= 1u << cslot;
+                    slot_busy &= ~(1u << cslot);
+                    // rows past the item's end (and tiles of a bad page) hold whatever memory held: V rows must be
+                    // zero so that a zero probability times them stays zero; K rows are masked by the logit test
+                    const int grp_w = warp + it * NWS;
+                    int valid_rows = cur.n - grp_w * kGroupTokens;
+                    if ((slot_bad >> cslot) & 1u) valid_rows = 0;
+                    if (valid_rows < kGroupTokens) {
+                        const uint32_t vt = my_stage_u32 + cslot * STAGE_BYTES + TILE_BYTES;
+                        for (int e = lane; e < (kGroupTokens - valid_rows) * CHUNKS; e += 32) {
+                            const int r = valid_rows + e / CHUNKS, cch = e % CHUNKS;
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vt + (cch >> 3) * 2048 + r * 128 + ((cch & 7) << 4)), "r"(0) : "memory");
+                        }
+                    }
+                } else {
+                    if (!strict) cp_async_wait<NS - 1>();  // everything but the NS-1 newest groups, i.e. group `it`, has landed
+                }
+                __syncwarp();
+                const int grp = warp + it * NWS;
+                const uint32_t ks_u32 = my_stage_u32 + ((vp + it) % NS) * STAGE_BYTES;
+                const uint32_t vs_u32 = ks_u32 + TILE_BYTES;
+
+                float ca[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int pr = 0; pr < KS / 2; ++pr) {  // 32 bytes of every key row: two k-steps
+                    uint32_t r[4];  // rows gq | gq + 8 of bytes [32 pr, +16) | rows gq | gq + 8 of bytes [32 pr + 16, +16)
+                    ldmatrix_x4(ks_u32 + swz(k_row, 2 * pr + k_chunk), r);
+                    const uint32_t a0[4] = {bytes_to_f16x2<E5M2, 0, 1>(r[0]), bytes_to_f16x2<E5M2, 0, 1>(r[1]),
+                                            bytes_to_f16x2<E5M2, 2, 3>(r[0]), bytes_to_f16x2<E5M2, 2, 3>(r[1])};
+                    const uint32_t a1[4] = {bytes_to_f16x2<E5M2, 0, 1>(r[2]), bytes_to_f16x2<E5M2, 0, 1>(r[3]),
+                                            bytes_to_f16x2<E5M2, 2, 3>(r[2]), bytes_to_f16x2<E5M2, 2, 3>(r[3])};
+                    mma_f16(ca, a0, bq[2 * pr][0], bq[2 * pr][1]);
+                    mma_f16(cb, a1, bq[2 * pr + 1][0], bq[2 * pr + 1][1]);
+                }
+                const int tokA = grp * kGroupTokens + gq, tokB = tokA + 8;
+                const float s00 = (tokA < cur.n) ? (ca[0] + cb[0]) * sl2 : -INFINITY;
+                const float s01 = (tokA < cur.n) ? (ca[1] + cb[1]) * sl2 : -INFINITY;
+                const float s10 = (tokB < cur.n) ? (ca[2] + cb[2]) * sl2 : -INFINITY;
+                const float s11 = (tokB < cur.n) ? (ca[3] + cb[3]) * sl2 : -INFINITY;
+                if (2 * tq < GP) {
+                    if (!OVF || tokA < chunk) st_shared_f2(lg_u32 + (tokA * GP + 2 * tq) * 4, s00, s01);
+                    else *reinterpret_cast<float2*>(spill + (size_t)(tokA - chunk) * GP + 2 * tq) = make_float2(s00, s01);
+                    if (!OVF || tokB < chunk) st_shared_f2(lg_u32 + (tokB * GP + 2 * tq) * 4, s10, s11);
+                    else *reinterpret_cast<float2*>(spill + (size_t)(tokB - chunk) * GP + 2 * tq) = make_float2(s10, s11);
+                }
+                float mx0 = fmaxf(s00, s10), mx1 = fmaxf(s01, s11);
+#pragma unroll
+                for (int off = 4; off < 32; off <<= 1) {
+                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+                }
+                const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+                if (__any_sync(0xffffffffu, (mn0 > m0) || (mn1 > m1))) {
+                    const float c0 = exp2_diff(m0, mn0), c1 = exp2_diff(m1, mn1);
+                    l0 *= c0;
+                    l1 *= c1;
+#pragma unroll
+                    for (int mt = 0; mt < KS; ++mt) {
+                        o[mt][0] *= c0; o[mt][2] *= c0;
+                        o[mt][1] *= c1; o[mt][3] *= c1;
+                    }
+                    m0 = mn0;
+                    m1 = mn1;
+                }
+                const float p00 = fast_exp2(s00 - m0), p01 = fast_exp2(s01 - m1);
+                const float p10 = fast_exp2(s10 - m0), p11 = fast_exp2(s11 - m1);
+                l0 += p00 + p10;
+                l1 += p01 + p11;
+                const uint32_t pb0 = movmatrix_trans(pack_f16(p00, p01));
+                const uint32_t pb1 = movmatrix_trans(pack_f16(p10, p11));
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    // per register: {tok: d, d+1}, {tok+1: d, d+1}; tokens 2tq, 2tq+1 (r[0], r[1]) and +8 (r[2], r[3]);
+                    // d = 32 mt + 2 gq (r[0], r[2]) and d + 16 (r[1], r[3])
+                    uint32_t r[4];
+                    ldmatrix_x4_trans(vs_u32 + swz(v_row, 2 * mt + v_chunk), r);
+                    uint32_t ae[4], ao[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        ae[i] = bytes_to_f16x2<E5M2, 0, 2>(r[i]);  // even d: bytes 0 and 2
+                        ao[i] = bytes_to_f16x2<E5M2, 1, 3>(r[i]);  // odd d:  bytes 1 and 3
+                    }
+                    mma_f16(o[2 * mt], ae, pb0, pb1);
+                    mma_f16(o[2 * mt + 1], ao, pb0, pb1);
+                }
+            }
+            vp = (vp + cur.count) % NS;
+
+            // ---- park this warp's partials in the parity buffer and signal the epilogue warps
+#pragma unroll
+            for (int off = 4; off < 32; off <<= 1) {
+                l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+                l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+            }
+            if (gq == 0) {
+                hd.wstat[p][warp][2 * tq] = make_float2(m0, l0);
+                hd.wstat[p][warp][2 * tq + 1] = make_float2(m1, l1);
+            }
+            if (2 * tq < GP) {
+                // accumulator o[2 mt + par]: rows gq / gq + 8 are d = 32 mt + 2 gq + par and d + 16; a value byte x
+                // means v_scale * x
+                const float vs_l = a.v_scale[cur.l];
+                float* wo = wo_all + ((size_t)p * NWS + warp) * wo_stride;
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                    for (int par = 0; par < 2; ++par) {
+                        const int d = 32 * mt + 2 * gq + par;
+                        wo[(2 * tq) * D + d] = o[2 * mt + par][0] * vs_l;
+                        wo[(2 * tq + 1) * D + d] = o[2 * mt + par][1] * vs_l;
+                        wo[(2 * tq) * D + d + 16] = o[2 * mt + par][2] * vs_l;
+                        wo[(2 * tq + 1) * D + d + 16] = o[2 * mt + par][3] * vs_l;
+                    }
+            }
+            // (overflowed logits written to global memory are released to the epilogue warps by the mbarrier
+            // arrive below, which has release semantics at CTA scope, like the shared-memory writes)
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&hd.full[p]);
+
+            // ---- rotate
+            if (!nxt_ready) acquire_next();
+            cur = nxt;
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                bq[ks][0] = bqn[ks][0];
+                bq[ks][1] = bqn[ks][1];
+            }
+            pg_lo = pg_nxt;
+            pg_blk = 0;
+            pg_hi = load_pages(cur, 1);
+            issued = issued_next;
+            ++seq;
+        }
+        cp_async_wait<0>();
+        if (TMA) {  // only after a timeout can loads still be in flight: wait for them (bounded) before leaving
+            for (int sl = 0; sl < NS; ++sl)
+                if ((slot_busy >> sl) & 1u) {
+                    for (int spin = 0; spin < kWaitLimit; ++spin)
+                        if (mbar_try_wait(&hd.tma_full[warp][sl], (slot_phase >> sl) & 1u)) break;
+                }
+        }
+        if (bad_page && lane == 0) record_error(a.status, LETHE_ERR_PAGE, 0);
+    } else {
+        // =================================================================== epilogue warps
+        const int ew = warp - NWS;
+        const int et = ew * 32 + lane;
+        bool alive = true;
+        for (int seq = 0; alive; ++seq) {
+            const int p = seq & 1;
+            // the descriptor of item seq was published by epilogue warp 0 while finishing item seq-2; waiting
+            // for that hand-back (both epilogue warps arrive on it) makes the write visible to this warp too
+            if (seq >= 2 && !mbar_wait(&hd.empty[p], (unsigned)(((seq >> 1) - 1) & 1), abort_flag)) {
+                alive = false;
+                break;
+            }
+            AsyncItem it;
+            async_decode(a, hd.desc_ticket[seq & 3], hd.desc_n_old[seq & 3], it);
+            if (!it.valid) break;
+            if (!mbar_wait(&hd.full[p], (unsigned)((seq >> 1) & 1), abort_flag)) {
+                alive = false;
+                break;
+            }
+            // ticket of the item after next: its round trips hide behind the merge below
+            int t_new = a.n_items;
+            if (ew == 0 && lane == 0 && !drew_fail) t_new = (int)atomicAdd(&sched[0], 1u);
+
+            const uint32_t lg_u32 = smem_u32(lg_all + (size_t)p * chunk * GP);
+            const float* spill = SPILL ? spill_all + (size_t)p * a.spill_tokens * GP : nullptr;
+            float* relp = a.rel + (size_t)it.item * a.cap_tokens;
+            const int app = (append && !it.full) ? it.n_old : -1;
+
+            // merged statistics of every head (each thread computes them all: off the critical path)
+            float fm[kMaxGroup], fi[kMaxGroup];
+#pragma unroll
+            for (int h = 0; h < kMaxGroup; ++h) {
+                fm[h] = -INFINITY;
+                fi[h] = 0.f;
+                if (h < G) {
+                    float m = -INFINITY;
+#pragma unroll
+                    for (int w = 0; w < NWS; ++w) m = fmaxf(m, hd.wstat[p][w][h].x);
+                    float l = 0.f;
+#pragma unroll
+                    for (int w = 0; w < NWS; ++w) l += hd.wstat[p][w][h].y * exp2_diff(hd.wstat[p][w][h].x, m);
+                    fm[h] = m;
+                    fi[h] = l > 0.f ? 1.f / l : 0.f;
+                    if (a.lse && et == h)
+                        a.lse[(size_t)(it.li * a.B + it.b) * a.Hq + it.hkv * G + h] =
+                            l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                }
+            }
+            const bool item_overflows = SPILL && it.n > chunk;
+            auto mass_of = [&](int j) {
+                const bool in_smem = !item_overflows || j < chunk;
+                float mass = 0.f;
+#pragma unroll
+                for (int h = 0; h < kMaxGroup; h += 2) {
+                    if (h < GP) {
+                        const float2 s2 = in_smem ? ld_shared_f2(lg_u32 + (j * GP + h) * 4)
+                                                  : *reinterpret_cast<const float2*>(spill + (size_t)(j - chunk) * GP + h);
+                        mass += fast_exp2(s2.x - fm[h]) * fi[h];
+                        if (h + 1 < G) mass += fast_exp2(s2.y - fm[h + 1]) * fi[h + 1];
+                    }
+                }
+                return mass;
+            };
+            // Eq. 5 on rel[0..n): old values are fetched a batch ahead of their use
+            constexpr int RB = 8;
+            float oldv[RB];
+            auto fetch = [&](int base) {
+#pragma unroll
+                for (int i = 0; i < RB; ++i) {
+                    const int j = base + et + i * ET;
+                    oldv[i] = (j < it.n && j != app) ? relp[j] : 0.f;
+                }
+            };
+            fetch(0);
+            {
+                T* out = (T*)a.out + ((size_t)(it.li * a.B + it.b) * a.Hq + it.hkv * G) * D;
+                for (int idx = et; idx < G * D; idx += ET) {
+                    const int h = idx / D;
+                    float mh = -INFINITY, ih = 0.f;
+#pragma unroll
+                    for (int hh = 0; hh < kMaxGroup; ++hh)
+                        if (hh == h) {
+                            mh = fm[hh];
+                            ih = fi[hh];
+                        }
+                    float acc = 0.f;
+#pragma unroll
+                    for (int w = 0; w < NWS; ++w)
+                        acc += wo_all[((size_t)p * NWS + w) * wo_stride + idx] * exp2_diff(hd.wstat[p][w][h].x, mh);
+                    out[idx] = __float2bfloat16_rn(acc * ih);
+                }
+            }
+            for (int base = 0; base < it.n; base += RB * ET) {
+                float cur_old[RB];
+#pragma unroll
+                for (int i = 0; i < RB; ++i) cur_old[i] = oldv[i];
+                if (base + RB * ET < it.n) fetch(base + RB * ET);
+#pragma unroll
+                for (int i = 0; i < RB; ++i) {
+                    const int j = base + et + i * ET;
+                    if (j < it.n) relp[j] = fmaf(a.gamma, cur_old[i], mass_of(j));
+                }
+            }
+            if (ew == 0 && lane == 0) {
+                if (it.full) record_error(a.status, LETHE_ERR_CAPACITY, it.item);
+                else if (append) a.len[it.item] = it.n;
+                if (t_new >= a.n_items) drew_fail = true;
+                if (a.order && t_new < a.n_items) t_new = a.order[t_new];
+                AsyncItem nx;
+                async_decode(a, t_new, 0, nx);
+                hd.desc_n_old[(seq + 2) & 3] = nx.valid ? a.len[nx.item] : 0;
+                hd.desc_ticket[(seq + 2) & 3] = t_new;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&hd.empty[p]);
+        }
+        if (!alive && lane == 0) record_error(a.status, LETHE_ERR_TIMEOUT, (int)blockIdx.x);
+        // ---- the last CTA out re-arms the queue for the next launch
+        if (ew == 0 && lane == 0) {
+            __threadfence();
+            const unsigned int done = atomicAdd(&sched[1], 1u);
+            if (done == gridDim.x - 1) {
+                sched[0] = 0u;
+                sched[1] = 0u;
+                __threadfence();
+            }
+        }
+    }
+}
+
+template <int D, int NWS, int NS>
+static size_t kv8a_smem(int chunk_tokens, int GP) {
+    return (size_t)NWS * NS * 2 * kGroupTokens * D + sizeof(AsyncHeader) + (size_t)2 * NWS * GP * D * 4 +
+           (size_t)2 * chunk_tokens * GP * 4;
+}
+
+template <int D, int NWS, int NS, bool PAGED, bool SPILL, bool E5M2>
+static cudaError_t launch_kv8a_t(const AttendArgs& a, const TmaMaps& maps, int grid, cudaStream_t stream) {
+    auto kern = attend_kv8_async_kernel<D, NWS, NS, PAGED, SPILL, E5M2>;
+    const size_t smem = kv8a_smem<D, NWS, NS>(a.chunk_tokens, a.GP);
+    cudaError_t e = prepare_kernel((const void*)kern, smem);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, (NWS + kEpilogueWarps) * 32, smem, stream>>>(a, maps);
+    return cudaGetLastError();
+}
+
+template <int D, int NWS, int NS, bool E5M2>
+static cudaError_t dispatch_kv8a(const AttendArgs& a, const TmaMaps& maps, bool paged, int grid, cudaStream_t stream) {
+    const bool spill = a.spill != nullptr;
+    if (paged)
+        return spill ? launch_kv8a_t<D, NWS, NS, true, true, E5M2>(a, maps, grid, stream)
+                     : launch_kv8a_t<D, NWS, NS, true, false, E5M2>(a, maps, grid, stream);
+    return spill ? launch_kv8a_t<D, NWS, NS, false, true, E5M2>(a, maps, grid, stream)
+                 : launch_kv8a_t<D, NWS, NS, false, false, E5M2>(a, maps, grid, stream);
+}
+
+// Shapes: (streaming warps per CTA, stages per warp); two more warps run the epilogue.  Tiles are half the size of the
+// bf16 kernel's, so the pipelines are deeper.
+#define LETHE_KV8A_SHAPES(X, D) X(0, D, 8, 4) X(1, D, 6, 5) X(2, D, 6, 6) X(3, D, 5, 6) X(4, D, 10, 3) X(5, D, 4, 6)
+
+}  // namespace
+
+size_t kv8_async_smem_bytes(int D, int shape, int chunk_tokens, int GP) {
+#define X(id, DD, NW, NS) \
+    if (shape == id && D == DD) return kv8a_smem<DD, NW, NS>(chunk_tokens, GP);
+    LETHE_KV8A_SHAPES(X, 128)
+    LETHE_KV8A_SHAPES(X, 64)
+#undef X
+    return (size_t)-1;
+}
+
+cudaError_t launch_attend_kv8_async(const AttendArgs& a, int D, int shape, bool paged, bool e5m2, int grid, cudaStream_t stream) {
+    TmaMaps none;
+    memset(&none, 0, sizeof(none));
+#define X(id, DD, NW, NS)                                                                                                \
+    if (shape == id && D == DD)                                                                                          \
+        return e5m2 ? dispatch_kv8a<DD, NW, NS, true>(a, none, paged, grid, stream) : dispatch_kv8a<DD, NW, NS, false>(a, none, paged, grid, stream);
+    LETHE_KV8A_SHAPES(X, 128)
+    LETHE_KV8A_SHAPES(X, 64)
+#undef X
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace lethe

@@ -655,7 +655,8 @@ extern "C" lethe_status lethe_rasr_prune_static(const lethe_cache* c, const int3
     if (!c || !budgets || !c->k || !c->v || !c->rel || !c->pos || !c->len) return LETHE_ERR_INVALID_ARG;
     if (c->n_layers < 1 || c->batch < 1 || c->n_kv_heads < 1 || c->capacity < 1) return LETHE_ERR_INVALID_ARG;
     if (c->head_dim != 64 && c->head_dim != 128) return LETHE_ERR_UNSUPPORTED;
-    if (c->dtype != LETHE_F32 && c->dtype != LETHE_BF16 && c->dtype != LETHE_FP8_E4M3) return LETHE_ERR_INVALID_ARG;
+    if (c->dtype != LETHE_F32 && c->dtype != LETHE_BF16 && c->dtype != LETHE_FP8_E4M3 && c->dtype != LETHE_FP8_E5M2)
+        return LETHE_ERR_INVALID_ARG;
     if (c->layout != LETHE_CONTIG && c->layout != LETHE_PAGED) return LETHE_ERR_INVALID_ARG;
     if (c->layout == LETHE_PAGED && (!c->page_table || c->page_tokens < 1 || c->n_pages < 1)) return LETHE_ERR_INVALID_ARG;
     if (recent < 0 || sink < 0 || (keep_idx && max_k < 1)) return LETHE_ERR_INVALID_ARG;
@@ -665,7 +666,7 @@ extern "C" lethe_status lethe_rasr_prune_static(const lethe_cache* c, const int3
     v.k = c->k; v.v = c->v; v.rel = c->rel; v.pos = c->pos; v.len = c->len; v.page_table = c->page_table;
     v.n_pages = c->n_pages;
     v.L = c->n_layers; v.B = c->batch; v.Hkv = c->n_kv_heads; v.D = c->head_dim;
-    v.elt_bytes = c->dtype == LETHE_BF16 ? 2 : (c->dtype == LETHE_FP8_E4M3 ? 1 : 4);
+    v.elt_bytes = c->dtype == LETHE_BF16 ? 2 : (c->dtype == LETHE_F32 ? 4 : 1);
     v.capacity = c->capacity;
     v.page_tokens = c->layout == LETHE_PAGED ? c->page_tokens : 1;
     v.paged = c->layout == LETHE_PAGED;

@@ -68,7 +68,7 @@ def sync_state(gc, oc):
 def logical_rows(k, v, rel, pos, ln, page_table=None, page_tokens=0):
     """Per item (K rows, V rows, rel, pos) of the first len slots, as CPU tensors, for either layout."""
     k, v, rel, pos, ln = k.cpu(), v.cpu(), rel.cpu(), pos.cpu(), ln.cpu()
-    if k.dtype == torch.float8_e4m3fn:                 # compare quantised rows as the bytes they are
+    if k.dtype in (torch.float8_e4m3fn, torch.float8_e5m2):   # compare quantised rows as the bytes they are
         k, v = k.view(torch.uint8), v.view(torch.uint8)
     L, B, H = ln.shape
     out = []

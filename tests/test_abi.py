@@ -45,4 +45,4 @@ def test_struct_layout_matches_header():
         "n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "dtype", "layout", "capacity", "page_tokens",
         "k", "v", "rel", "pos", "len", "page_table", "n_pages", "k_scale", "v_scale"]
     assert ctypes.sizeof(binding.lethe_cache) == 40 + 6 * 8 + 8 + 2 * 8
-    assert (binding.F32, binding.BF16, binding.FP8_E4M3) == (0, 1, 2)
+    assert (binding.F32, binding.BF16, binding.FP8_E4M3, binding.FP8_E5M2) == (0, 1, 2, 3)

@@ -18,16 +18,20 @@ def ctx():
     c.close()
 
 
-def fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed, k_scale=None, v_scale=None, page_tokens=0):
+FMT = {"e4m3": (torch.float8_e4m3fn, 448.0), "e5m2": (torch.float8_e5m2, 57344.0)}
+
+
+def fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed, k_scale=None, v_scale=None, page_tokens=0, fmt="e4m3"):
     """Quantised cache drawn as the quantisation of Gaussian K / V (a few keys enlarged, as the workloads' anchors)."""
+    f8, fmax = FMT[fmt]
     g = torch.Generator().manual_seed(seed)
     ks = torch.tensor(k_scale if k_scale is not None else [1.0] * L, dtype=torch.float32)
     vs = torch.tensor(v_scale if v_scale is not None else [1.0] * L, dtype=torch.float32)
     k = torch.randn((L, B, Hkv, cap, D), generator=g)
     k[:, :, :, ::17] *= 3.0
     v = torch.randn((L, B, Hkv, cap, D), generator=g)
-    k8 = (k / ks.reshape(L, 1, 1, 1, 1)).clamp(-448, 448).to(torch.float8_e4m3fn)
-    v8 = (v / vs.reshape(L, 1, 1, 1, 1)).clamp(-448, 448).to(torch.float8_e4m3fn)
+    k8 = (k / ks.reshape(L, 1, 1, 1, 1)).clamp(-fmax, fmax).to(f8)
+    v8 = (v / vs.reshape(L, 1, 1, 1, 1)).clamp(-fmax, fmax).to(f8)
     rel = torch.rand((L, B, Hkv, cap), generator=g)
     pos = torch.arange(cap, dtype=torch.int32).expand(L, B, Hkv, cap).contiguous()
     ln = torch.full((L, B, Hkv), lens, dtype=torch.int32) if isinstance(lens, int) else lens.to(torch.int32).contiguous()
@@ -41,7 +45,7 @@ def fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed, k_scale=None, v_scale=None, pag
         pool_v = torch.zeros((n_pages, page_tokens, D), dtype=torch.uint8)
         pool_k[table.long().flatten()] = k8.view(torch.uint8).reshape(-1, page_tokens, D)
         pool_v[table.long().flatten()] = v8.view(torch.uint8).reshape(-1, page_tokens, D)
-        return oracle.OracleCache(L, B, Hq, Hkv, D, pages_per_item, pool_k.view(torch.float8_e4m3fn), pool_v.view(torch.float8_e4m3fn),
+        return oracle.OracleCache(L, B, Hq, Hkv, D, pages_per_item, pool_k.view(f8), pool_v.view(f8),
                                   rel, pos, ln, page_tokens, table, k_scale=ks, v_scale=vs)
     return oracle.OracleCache(L, B, Hq, Hkv, D, cap, k8, v8, rel, pos, ln, k_scale=ks, v_scale=vs)
 
@@ -64,9 +68,10 @@ def _step(ctx, oc, gc, q, kn, vn, tp, scale, gamma, want_lse=False):
     assert_state_matches(gc, oc)           # appended bytes, pos, len bit-exact; rel within 1e-3
 
 
+@pytest.mark.parametrize("fmt", ["e4m3", "e5m2"])
 @pytest.mark.parametrize("paged", [False, True])
 @pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 128), (7, 1, 128), (4, 4, 64), (16, 2, 64), (6, 2, 128)])
-def test_quantised_decode_parity(ctx, Hq, Hkv, D, paged):
+def test_quantised_decode_parity(ctx, Hq, Hkv, D, paged, fmt):
     """Ragged lengths over several 16-token groups and tails, attend-only and appending steps, scales that are not
     powers of two, a new token beyond the representable range (saturates)."""
     L, B, cap = 2, 3, 208
@@ -74,7 +79,7 @@ def test_quantised_decode_parity(ctx, Hq, Hkv, D, paged):
     lens = torch.randint(1, cap - 8, (L, B, Hkv), generator=g)
     lens.view(-1)[:4] = torch.tensor([1, 15, 16, 17])[: min(4, lens.numel())]
     oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=Hq + D, k_scale=[0.37, 1.5], v_scale=[2.25, 0.6],
-                   page_tokens=16 if paged else 0)
+                   page_tokens=16 if paged else 0, fmt=fmt)
     gc = to_device(oc)
     scale = torch.tensor([0.11, 0.07], dtype=torch.float32) * (128 / D) ** 0.5
     for step in range(5):
@@ -85,19 +90,25 @@ def test_quantised_decode_parity(ctx, Hq, Hkv, D, paged):
         kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
         vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
         if step == 2:
-            kn[0, 0, 0, :3] = torch.tensor([1e4, -1e4, 165.5], dtype=torch.bfloat16)
-            vn[1, 1, 0, :2] = torch.tensor([-3e3, 269.0], dtype=torch.bfloat16)
+            big = 1e4 if fmt == "e4m3" else 1e6                      # beyond the format's range: saturates
+            kn[0, 0, 0, :3] = torch.tensor([big, -big, 165.5], dtype=torch.bfloat16)
+            vn[1, 1, 0, :2] = torch.tensor([-0.3 * big, 269.0], dtype=torch.bfloat16)
         _step(ctx, oc, gc, q, kn, vn, torch.arange(B, dtype=torch.int32) + 300 + step, scale, 0.95)
 
 
-@pytest.mark.parametrize("variant,splits", [(2, 1), (3, 2), (4, 4), (5, 1), (6, 8), (7, 2), (0, 0), (8, 0), (9, 0), (10, 1),
-                                            (11, 0), (12, 0), (13, 0)])
-def test_quantised_decode_shapes_and_clusters(ctx, variant, splits):
+@pytest.mark.parametrize("variant,splits,fmt", [(2, 1, "e4m3"), (3, 2, "e4m3"), (4, 4, "e4m3"), (5, 1, "e4m3"), (6, 8, "e4m3"),
+                                                (7, 2, "e4m3"), (0, 0, "e4m3"), (8, 0, "e4m3"), (9, 0, "e4m3"), (10, 1, "e4m3"),
+                                                (11, 0, "e4m3"), (12, 0, "e4m3"), (13, 0, "e4m3"),
+                                                (2, 1, "e5m2"), (3, 2, "e5m2"), (4, 4, "e5m2"), (5, 1, "e5m2"), (6, 8, "e5m2"),
+                                                (7, 2, "e5m2"), (0, 0, "e5m2"), (9, 0, "e5m2"),
+                                                (16, 0, "e4m3"), (17, 0, "e4m3"), (18, 0, "e4m3"), (19, 0, "e4m3"), (20, 0, "e4m3"),
+                                                (21, 0, "e4m3"), (16, 0, "e5m2"), (19, 0, "e5m2")])
+def test_quantised_decode_shapes_and_clusters(ctx, variant, splits, fmt):
     """Every kernel shape and cluster size on items long enough to give every CTA of a cluster several groups."""
     L, B, Hq, Hkv, D, cap = 1, 2, 8, 2, 128, 1100
     g = torch.Generator().manual_seed(variant * 7 + splits)
     lens = torch.tensor([[[1037, 700], [513, 1090]]])
-    oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=variant, k_scale=[0.8], v_scale=[1.25])
+    oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=variant, k_scale=[0.8], v_scale=[1.25], fmt=fmt)
     gc = to_device(oc)
     ctx.set_tuning(variant, splits)
     try:
@@ -111,14 +122,15 @@ def test_quantised_decode_shapes_and_clusters(ctx, variant, splits):
         ctx.set_tuning(0, 0)
 
 
-def test_quantised_trajectory_with_prune_rounds(ctx):
+@pytest.mark.parametrize("fmt", ["e4m3", "e5m2"])
+def test_quantised_trajectory_with_prune_rounds(ctx, fmt):
     """Llama-8B-shaped geometry (2 layers, 2 sequences): decode steps with appends, a prune round every 6 steps on
     the oracle's scores; bytes, positions and lengths stay identical throughout."""
     oracle.set_threads(min(8, oracle.max_threads()))
     try:
         w = synth.shrink(synth.WORKLOADS["llama8b"], n_layers=2, batch=2)
         L, B, Hq, Hkv, D, cap, n0 = 2, 2, w.n_q_heads, w.n_kv_heads, w.head_dim, 320, 270
-        oc = fp8_cache(L, B, Hq, Hkv, D, cap, n0, seed=21, k_scale=[0.5, 0.7], v_scale=[0.9, 1.1])
+        oc = fp8_cache(L, B, Hq, Hkv, D, cap, n0, seed=21, k_scale=[0.5, 0.7], v_scale=[0.9, 1.1], fmt=fmt)
         oc.rel.zero_()
         gc = to_device(oc)
         dev = gc.device
@@ -175,7 +187,7 @@ def test_quantised_persistent_kernel_many_items(ctx, paged):
     scale = torch.tensor([0.1, 0.08, 0.12, 0.09], dtype=torch.float32)
     try:
         for step in range(5):
-            ctx.set_tuning(9 if step < 3 else 0, 0)
+            ctx.set_tuning((9, 16, 19, 0, 0)[step], 0)
             q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
             if step == 2:
                 _step(ctx, oc, gc, q, None, None, None, scale, 0.97, want_lse=True)
@@ -187,14 +199,15 @@ def test_quantised_persistent_kernel_many_items(ctx, paged):
         ctx.set_tuning(0, 0)
 
 
-def test_quantised_persistent_kernel_logit_overflow(ctx):
+@pytest.mark.parametrize("variant", [12, 20])                  # synchronous (16,2) / asynchronous (10,3): least room for logits
+def test_quantised_persistent_kernel_logit_overflow(ctx, variant):
     """Items longer than the on-chip logit buffer of the widest shape: the tail's logits go through global scratch."""
     L, B, Hq, Hkv, D, cap = 1, 2, 16, 2, 128, 12000
     g = torch.Generator().manual_seed(3)
     lens = torch.tensor([[[11950, 9000], [4000, 11990]]])
     oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=9, k_scale=[0.5], v_scale=[1.5])
     gc = to_device(oc)
-    ctx.set_tuning(12, 0)                                     # (16 warps, 2 stages): least room for logits
+    ctx.set_tuning(variant, 0)
     try:
         for step in range(2):
             q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
