@@ -12,8 +12,6 @@ namespace lethe {
 cudaError_t launch_attend_simt(const AttendArgs& a, int dtype, int D, bool paged, cudaStream_t stream);
 size_t kv8_smem_bytes(int D, int shape, int chunk_tokens, int GP);
 size_t kv8_stream_smem_bytes(int D, int shape, int chunk_tokens, int GP);
-size_t kv8_async_smem_bytes(int D, int shape, int chunk_tokens, int GP);
-cudaError_t launch_attend_kv8_async(const AttendArgs& a, int D, int shape, bool paged, bool e5m2, int grid, cudaStream_t stream);
 cudaError_t launch_attend_kv8_stream(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream);
 cudaError_t launch_attend_kv8(const AttendArgs& a, int D, int shape, bool paged, bool e5m2, cudaStream_t stream);
 size_t simt_smem_bytes(int D, int chunk_tokens, int GP);
@@ -371,29 +369,8 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         }
         // The clustered kernel (variants 2..7 pick its shape) is the default at every size: with two CTAs per SM
         // covering each other's epilogues it beats the persistent one (variants 8..13) on this conversion-bound
-        // path (Llama-8B shape: 0.137 ms against 0.154 to 0.166 ms).
-        // variants 16..21: the persistent kernel with an asynchronous epilogue (both formats)
-        if (variant >= 16 && variant <= 21 && ctx->splits <= 1) {
-            const int ashape = variant - 16;
-            const size_t fixed = kv8_async_smem_bytes(c->head_dim, ashape, 0, a.GP);
-            int fit = 0;
-            if (fixed < ctx->max_smem) fit = (int)((ctx->max_smem - fixed) / ((size_t)2 * a.GP * 4) / kGroupTokens) * kGroupTokens;
-            a.splits = 1;
-            a.chunk_tokens = fit < cap_groups * kGroupTokens ? fit : cap_groups * kGroupTokens;
-            if (a.chunk_tokens < kGroupTokens)
-                return fail(ctx, LETHE_ERR_UNSUPPORTED, "no shared memory left for the logit buffers of this persistent shape");
-            const int grid = a.n_items < ctx->sm_count ? a.n_items : ctx->sm_count;
-            if (a.chunk_tokens < cap_groups * kGroupTokens) {
-                a.spill_tokens = cap_groups * kGroupTokens - a.chunk_tokens;
-                const size_t need = (size_t)grid * 2 * a.spill_tokens * a.GP * sizeof(float);
-                st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "logit overflow scratch");
-                if (st != LETHE_OK) return st;
-                a.spill = (float*)ctx->scratch;
-            }
-            const cudaError_t ea = launch_attend_kv8_async(a, c->head_dim, ashape, paged, c->dtype == LETHE_FP8_E5M2, grid, (cudaStream_t)stream);
-            if (ea != cudaSuccess) return cuda_fail(ctx, ea, "decode_attend launch (quantised cache, asynchronous epilogue)");
-            return LETHE_OK;
-        }
+        // path (Llama-8B shape: 0.124 ms against 0.153 to 0.161 ms; a version of the asynchronous-epilogue kernel for
+        // byte caches was measured too, 0.165 to 0.178 ms over six shapes, and is not kept).
         const bool want_persistent = variant >= 8 && variant <= 13;
         const bool want_clustered = variant >= 2 && variant <= 7;
         if (want_persistent && ctx->splits <= 1 && c->dtype == LETHE_FP8_E4M3) {

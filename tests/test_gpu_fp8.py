@@ -100,9 +100,7 @@ def test_quantised_decode_parity(ctx, Hq, Hkv, D, paged, fmt):
                                                 (7, 2, "e4m3"), (0, 0, "e4m3"), (8, 0, "e4m3"), (9, 0, "e4m3"), (10, 1, "e4m3"),
                                                 (11, 0, "e4m3"), (12, 0, "e4m3"), (13, 0, "e4m3"),
                                                 (2, 1, "e5m2"), (3, 2, "e5m2"), (4, 4, "e5m2"), (5, 1, "e5m2"), (6, 8, "e5m2"),
-                                                (7, 2, "e5m2"), (0, 0, "e5m2"), (9, 0, "e5m2"),
-                                                (16, 0, "e4m3"), (17, 0, "e4m3"), (18, 0, "e4m3"), (19, 0, "e4m3"), (20, 0, "e4m3"),
-                                                (21, 0, "e4m3"), (16, 0, "e5m2"), (19, 0, "e5m2")])
+                                                (7, 2, "e5m2"), (0, 0, "e5m2"), (9, 0, "e5m2")])
 def test_quantised_decode_shapes_and_clusters(ctx, variant, splits, fmt):
     """Every kernel shape and cluster size on items long enough to give every CTA of a cluster several groups."""
     L, B, Hq, Hkv, D, cap = 1, 2, 8, 2, 128, 1100
@@ -187,7 +185,7 @@ def test_quantised_persistent_kernel_many_items(ctx, paged):
     scale = torch.tensor([0.1, 0.08, 0.12, 0.09], dtype=torch.float32)
     try:
         for step in range(5):
-            ctx.set_tuning((9, 16, 19, 0, 0)[step], 0)
+            ctx.set_tuning(9 if step < 3 else 0, 0)
             q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
             if step == 2:
                 _step(ctx, oc, gc, q, None, None, None, scale, 0.97, want_lse=True)
@@ -199,15 +197,14 @@ def test_quantised_persistent_kernel_many_items(ctx, paged):
         ctx.set_tuning(0, 0)
 
 
-@pytest.mark.parametrize("variant", [12, 20])                  # synchronous (16,2) / asynchronous (10,3): least room for logits
-def test_quantised_persistent_kernel_logit_overflow(ctx, variant):
+def test_quantised_persistent_kernel_logit_overflow(ctx):
     """Items longer than the on-chip logit buffer of the widest shape: the tail's logits go through global scratch."""
     L, B, Hq, Hkv, D, cap = 1, 2, 16, 2, 128, 12000
     g = torch.Generator().manual_seed(3)
     lens = torch.tensor([[[11950, 9000], [4000, 11990]]])
     oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=9, k_scale=[0.5], v_scale=[1.5])
     gc = to_device(oc)
-    ctx.set_tuning(variant, 0)
+    ctx.set_tuning(12, 0)                                     # (16 warps, 2 stages): least room for logits
     try:
         for step in range(2):
             q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
