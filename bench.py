@@ -617,7 +617,7 @@ def main():
         if not args.no_e2e:
             line["e2e"] = {"value": dist_util.job_value(e_units, e_total_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                            "d2h_bytes_per_step": d2h, "ms_per_step": e_total_ms / args.steps}
-        if not args.no_cpu_baseline:
+        if not args.no_cpu_baseline and world == 1:   # the oracle is timed beside the single-GPU run only
             line["cpu_baseline"] = cpu_baseline(w, r)
             line["retained_set_overlap"] = line["cpu_baseline"].pop("retained_set_overlap", None)
         print(json.dumps(line))
