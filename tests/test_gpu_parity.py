@@ -382,6 +382,35 @@ def test_ragged_paged_long_items(ctx):
         oracle.set_threads(1)
 
 
+def test_ragged_paged_many_items_default_kernel(ctx):
+    """Ragged-batch geometry with enough items for the default choice to be the persistent kernel (320 items, G = 7,
+    16-token pages with shuffled tables, lengths from 400 to 6000 tokens): most items are longer than the on-chip
+    logit buffer, so the tail's logits go through scratch.  Decode steps, a prune to a third of each sequence's
+    length, decode steps on the pruned cache."""
+    oracle.set_threads(min(16, oracle.max_threads()))
+    try:
+        w = synth.shrink(synth.WORKLOADS["ragged"], n_layers=4, batch=20, prompt_len=6000)
+        cap = 6016
+        g = torch.Generator().manual_seed(77)
+        lens = torch.randint(400, 6001, (20,), generator=g)
+        lens[:4] = torch.tensor([400, 6000, 2047, 2049])
+        st_c = synth.initial_kv(w, 6000, cap)
+        st_c["len"][:] = lens[None, :, None].to(torch.int32)
+        st_p = synth.to_paged(st_c, 16, seed=6, spare_pages=9)
+        del st_c
+        oc = cache_from_state(w, st_p, cap)
+        gc = to_device(oc)
+        scale = synth.layer_scales(w)
+        T = (w.n_layers * (lens // 3)).to(torch.int64)
+        for step in range(3):
+            x = synth.step_inputs(w, step)
+            _step(ctx, oc, gc, x["q"], x["k_new"], x["v_new"], x["token_pos"], scale, w.gamma, 0, w.n_layers, want_lse=False)
+            if step == 0:
+                _prune_both(ctx, oc, gc, T, w.k_min, w.recent, w.sink, 2048)
+    finally:
+        oracle.set_threads(1)
+
+
 @pytest.mark.parametrize("variant,Hq,Hkv,cap", [(9, 28, 4, 3000), (12, 16, 4, 4200), (14, 28, 4, 6000), (16, 28, 4, 3000),
                                                 (18, 16, 4, 4200), (20, 28, 4, 6000), (26, 16, 4, 4200)])
 def test_persistent_logit_overflow(ctx, variant, Hq, Hkv, cap):
