@@ -25,8 +25,8 @@
  *   - Unless marked HOST, every pointer is a DEVICE pointer to memory owned by the
  *     caller; the library owns only the scratch inside lethe_ctx.
  *   - All arrays are dense row-major in the index order written beside them.
- *   - Every call that takes a `stream` enqueues its work there (a cudaStream_t passed as void*, NULL =
- *     the legacy default stream) and return without synchronising.
+ *   - Every call that takes a `stream` enqueues its work there (a cudaStream_t passed as
+ *     void*, NULL = the legacy default stream) and returns without synchronising.
  *   - Errors detectable on the host return a status and enqueue nothing.  Conditions
  *     only the device can see (a full cache on append, a budget below the protected
  *     count, a page id outside the pool) never trap: the kernel skips or clamps the
