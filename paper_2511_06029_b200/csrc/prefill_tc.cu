@@ -6,12 +6,13 @@
 //   STATS   the rows of a tile are 128 (query, head) columns of the attention matrix, its columns 128 keys; the
 //           thread that owns a row keeps that column's online (max, sum) over the keys j <= i in registers;
 //   COLSUM  the rows are 128 keys, the columns 128 (query, head) pairs; the thread that owns a key adds up
-//           exp2(logit - max) * weight / sum over the columns with i >= j.
+//           exp2(logit + bias) over the columns with i >= j, the bias of a column being log2(weight / sum) - max.
 // In both, the reduction runs along the TMEM row a thread owns.  Two warps share a row (TMEM lanes are reachable
 // only from the warps whose index has the same low two bits): each takes 64 of the 128 columns.  STATS writes the
-// two partial (max, sum) pairs side by side and COLSUM merges them when it fetches a column's factor; COLSUM's two
-// partial sums of a key meet in rel[j], zeroed by STATS, through two atomic adds (two addends commute, so the
-// result does not depend on their order).
+// two partial (max, sum) pairs side by side; the prologue of COLSUM merges them into the item's column biases
+// (in place); COLSUM's two partial sums of a key meet in rel[j], zeroed by STATS, through two atomic adds (two
+// addends commute, so the result does not depend on their order).  Two CTAs share an SM (one block buffer, two
+// streamed stages and 256 TMEM columns each) and cover each other's hand-off latencies.
 //
 // (query, head) columns are numbered query-major over the G heads of the group: column c of a block that starts
 // at query q0 is (q0 + c / G, c % G); a block holds qpb = 128 / G queries and its last 128 - qpb G columns are
