@@ -1,0 +1,44 @@
+"""The benchmark's output contract: one JSON line with the agreed keys, for the reference arm (CPU, runs anywhere)
+and for the GPU arm (short run)."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+BASE_KEYS = {"metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+             "vs_baseline", "dtype", "data", "config"}
+
+
+def _run(args, timeout):
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *args], capture_output=True, text=True,
+                       timeout=timeout, cwd=ROOT)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [l for l in p.stdout.strip().splitlines() if l.startswith("{")]
+    assert len(lines) == 1, p.stdout[-2000:]
+    return json.loads(lines[0])
+
+
+def test_reference_arm_prints_the_contract_line():
+    d = _run(["--impl", "reference", "--steps", "1", "--warmup", "1"], timeout=300)
+    assert BASE_KEYS <= set(d) and d["impl"] == "reference" and d["higher_is_better"] is True
+    assert d["metric"] == "kv_token_heads_attended_per_s" and d["unit"] == "token-heads/s" and d["value"] > 0
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1 and "sample" in d["cpu_baseline"]
+    assert d["e2e"] == {"value": d["value"], "unit": d["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+    assert d["vs_baseline"] is None and "workload" in d["config"]
+
+
+@pytest.mark.gpu
+def test_gpu_arm_prints_the_contract_line():
+    d = _run(["--steps", "160", "--warmup", "3", "--prep-rounds", "1", "--no-cpu-baseline", "--no-per-layer"], timeout=900)
+    assert BASE_KEYS <= set(d) and d["n_gpus"] == 1 and d["steps"] == 160 and d["scaling"] == "weak"
+    r = d["roofline"]
+    assert r["bound"] == "hbm" and r["unit"] == "GB/s" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
+    assert 0.3 < r["frac"] < 1.2 and r["traffic"] > 0
+    assert d["gpu_launches"] >= 160 and d["value"] > 1e9
+    e = d["e2e"]
+    assert e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0 and 0 < e["value"] < d["value"]
+    assert {"sm_mhz", "sm_max_mhz", "reasons"} <= set(d["clocks"])
+    assert d["config"]["prune_rounds_timed"] >= 1 and "workload" in d["config"]
