@@ -571,16 +571,22 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
                 }
             }
             const bool item_overflows = SPILL && it.n > chunk;
-            auto mass_of = [&](int j) {
+            // One token's G logits (from shared memory, or from the overflow area), then its attention mass.
+            auto load_row = [&](int j, float2 (&s)[kMaxGroup / 2]) {
                 const bool in_smem = !item_overflows || j < chunk;
+#pragma unroll
+                for (int h = 0; h < kMaxGroup; h += 2)
+                    if (h < GP)
+                        s[h / 2] = in_smem ? ld_shared_f2(lg_u32 + (j * GP + h) * 4)
+                                           : *reinterpret_cast<const float2*>(spill + (size_t)(j - chunk) * GP + h);
+            };
+            auto mass_from = [&](const float2 (&s)[kMaxGroup / 2]) {
                 float mass = 0.f;
 #pragma unroll
                 for (int h = 0; h < kMaxGroup; h += 2) {
                     if (h < GP) {
-                        const float2 s2 = in_smem ? ld_shared_f2(lg_u32 + (j * GP + h) * 4)
-                                                  : *reinterpret_cast<const float2*>(spill + (size_t)(j - chunk) * GP + h);
-                        mass += fast_exp2(s2.x - fm[h]) * fi[h];
-                        if (h + 1 < G) mass += fast_exp2(s2.y - fm[h + 1]) * fi[h + 1];
+                        mass += fast_exp2(s[h / 2].x - fm[h]) * fi[h];
+                        if (h + 1 < G) mass += fast_exp2(s[h / 2].y - fm[h + 1]) * fi[h + 1];
                     }
                 }
                 return mass;
@@ -619,10 +625,21 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
 #pragma unroll
                 for (int i = 0; i < RB; ++i) cur_old[i] = oldv[i];
                 if (base + RB * ET < it.n) fetch(base + RB * ET);
+                // kRelBatch rows are loaded before the first of them is used: the stores to rel would otherwise
+                // order the overflow area's loads one token at a time.
 #pragma unroll
-                for (int i = 0; i < RB; ++i) {
-                    const int j = base + et + i * ET;
-                    if (j < it.n) relp[j] = fmaf(a.gamma, cur_old[i], mass_of(j));
+                for (int i0 = 0; i0 < RB; i0 += kRelBatch) {
+                    float2 s[kRelBatch][kMaxGroup / 2];
+#pragma unroll
+                    for (int u = 0; u < kRelBatch; ++u) {
+                        const int j = base + et + (i0 + u) * ET;
+                        load_row(j < it.n ? j : it.n - 1, s[u]);
+                    }
+#pragma unroll
+                    for (int u = 0; u < kRelBatch; ++u) {
+                        const int j = base + et + (i0 + u) * ET;
+                        if (j < it.n) relp[j] = fmaf(a.gamma, cur_old[i0 + u], mass_from(s[u]));
+                    }
                 }
             }
             if (ew == 0 && lane == 0) {

@@ -372,16 +372,22 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
                 fi[h] = es.fin[h].y;
             }
             float* relp = a.rel + (size_t)cur.item * a.cap_tokens;
-            auto mass_of = [&](int j) {
+            // One token's G logits (from shared memory, or from the overflow area), then its attention mass.
+            auto load_row = [&](int j, float2 (&s)[kMaxGroup / 2]) {
                 const bool in_smem = !SPILL || j < chunk;
+#pragma unroll
+                for (int h = 0; h < kMaxGroup; h += 2)
+                    if (h < GP)
+                        s[h / 2] = in_smem ? ld_shared_f2(lg_u32 + (j * GP + h) * 4)
+                                           : ld_global_f2_hint(spill + (size_t)(j - chunk) * GP + h, spill_policy);
+            };
+            auto mass_from = [&](const float2 (&s)[kMaxGroup / 2]) {
                 float mass = 0.f;
 #pragma unroll
                 for (int h = 0; h < kMaxGroup; h += 2) {
                     if (h < GP) {
-                        const float2 s2 = in_smem ? ld_shared_f2(lg_u32 + (j * GP + h) * 4)
-                                                  : ld_global_f2_hint(spill + (size_t)(j - chunk) * GP + h, spill_policy);
-                        mass += fast_exp2(s2.x - fm[h]) * fi[h];
-                        if (h + 1 < G) mass += fast_exp2(s2.y - fm[h + 1]) * fi[h + 1];
+                        mass += fast_exp2(s[h / 2].x - fm[h]) * fi[h];
+                        if (h + 1 < G) mass += fast_exp2(s[h / 2].y - fm[h + 1]) * fi[h + 1];
                     }
                 }
                 return mass;
@@ -389,11 +395,29 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
 #pragma unroll
             for (int i = 0; i < kRelPrefetch; ++i) {
                 const int j = tid + i * NT;
-                if (j < cur.n) relp[j] = fmaf(a.gamma, rel_old[i], mass_of(j));
+                if (j < cur.n) {
+                    float2 s[kMaxGroup / 2];
+                    load_row(j, s);
+                    relp[j] = fmaf(a.gamma, rel_old[i], mass_from(s));
+                }
             }
-            for (int j = tid + kRelPrefetch * NT; j < cur.n; j += NT) {
-                const float old = (append && j == cur.n_old) ? 0.f : relp[j];
-                relp[j] = fmaf(a.gamma, old, mass_of(j));
+            // The tail of a long item: kRelBatch tokens per thread at a time, every load of the batch issued
+            // before the first use, so that the global-memory latency is paid once per batch.
+            for (int j0 = tid + kRelPrefetch * NT; j0 < cur.n; j0 += kRelBatch * NT) {
+                float old[kRelBatch];
+                float2 s[kRelBatch][kMaxGroup / 2];
+#pragma unroll
+                for (int u = 0; u < kRelBatch; ++u) {
+                    const int j = j0 + u * NT;
+                    const bool ok = j < cur.n;
+                    old[u] = (ok && !(append && j == cur.n_old)) ? relp[j] : 0.f;
+                    load_row(ok ? j : j0, s[u]);
+                }
+#pragma unroll
+                for (int u = 0; u < kRelBatch; ++u) {
+                    const int j = j0 + u * NT;
+                    if (j < cur.n) relp[j] = fmaf(a.gamma, old[u], mass_from(s[u]));
+                }
             }
         }
         if (tid == 0) {

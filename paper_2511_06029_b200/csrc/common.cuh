@@ -191,6 +191,7 @@ struct EpilogueSmem {
 
 // Old relevance values a thread will update: loaded early so that their latency hides behind the merge.
 constexpr int kRelPrefetch = 8;
+constexpr int kRelBatch = 4;  // tokens per thread per batch in the tail of a long item's relevance update
 
 template <int NT>
 __device__ __forceinline__ void prefetch_rel(const AttendArgs& a, const ItemCoord& ic, int t0, int hi_tok,
