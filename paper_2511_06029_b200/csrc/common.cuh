@@ -298,22 +298,51 @@ __device__ void combine_and_finish(const AttendArgs& a, const ItemCoord& ic, Epi
         fm[h] = es.fin[h].x;
         fi[h] = es.fin[h].y;
     }
-    auto mass_of = [&](int j) {
+    // Rows are loaded a batch ahead of the stores to rel: the compiler cannot tell that rel and the logit buffer
+    // never alias, and would otherwise keep every token's loads behind the previous token's store.
+    auto load_row = [&](int j, float (&s)[kMaxGroup]) {
         const float* row = lg + (size_t)(j - t0) * GP;
+#pragma unroll
+        for (int h = 0; h < kMaxGroup; ++h)
+            if (h < G) s[h] = row[h];
+    };
+    auto mass_from = [&](const float (&s)[kMaxGroup]) {
         float mass = 0.f;
 #pragma unroll
         for (int h = 0; h < kMaxGroup; ++h)
-            if (h < G) mass += fast_exp2(row[h] - fm[h]) * fi[h];
+            if (h < G) mass += fast_exp2(s[h] - fm[h]) * fi[h];
         return mass;
     };
 #pragma unroll
-    for (int i = 0; i < kRelPrefetch; ++i) {
-        const int j = t0 + tid + i * NT;
-        if (j < hi_tok) rel[j] = fmaf(a.gamma, rel_old[i], mass_of(j));
+    for (int i0 = 0; i0 < kRelPrefetch; i0 += kRelBatch) {
+        float s[kRelBatch][kMaxGroup];
+#pragma unroll
+        for (int u = 0; u < kRelBatch; ++u) {
+            const int j = t0 + tid + (i0 + u) * NT;
+            if (j < hi_tok) load_row(j, s[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < kRelBatch; ++u) {
+            const int j = t0 + tid + (i0 + u) * NT;
+            if (j < hi_tok) rel[j] = fmaf(a.gamma, rel_old[i0 + u], mass_from(s[u]));
+        }
     }
-    for (int j = t0 + tid + kRelPrefetch * NT; j < hi_tok; j += NT) {
-        const float old = (j == append_slot) ? 0.f : rel[j];
-        rel[j] = fmaf(a.gamma, old, mass_of(j));
+    for (int j0 = t0 + tid + kRelPrefetch * NT; j0 < hi_tok; j0 += kRelBatch * NT) {
+        float old[kRelBatch];
+        float s[kRelBatch][kMaxGroup];
+#pragma unroll
+        for (int u = 0; u < kRelBatch; ++u) {
+            const int j = j0 + u * NT;
+            if (j < hi_tok) {
+                old[u] = (j == append_slot) ? 0.f : rel[j];
+                load_row(j, s[u]);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kRelBatch; ++u) {
+            const int j = j0 + u * NT;
+            if (j < hi_tok) rel[j] = fmaf(a.gamma, old[u], mass_from(s[u]));
+        }
     }
     TL_MARK(a, 5);
     if (S > 1) cg::this_cluster().sync();  // peers may still be reading this CTA's shared memory
