@@ -8,7 +8,8 @@ One "step" = one decode step of the whole model shape (all layers, one lethe_dec
 step index hits the prune interval, one prune round (estimate_sparsity -> alloc_budgets -> rasr_prune).  The
 printed JSON line follows the driver's contract; `value` is KV token-heads attended per second with the cache
 and the step inputs resident in HBM, `e2e` is the same through lethe_decode_attend_host (per-step q / k_new /
-v_new from pinned host memory, out read back to the host, a stream synchronise every step).
+v_new in pinned host memory, out delivered to pinned host memory, a stream synchronise every step; with pinned
+buffers the persistent kernel moves those bytes over the bus itself instead of through copies, see `transfer`).
 """
 from __future__ import annotations
 
@@ -616,7 +617,10 @@ def main():
         }
         if not args.no_e2e:
             line["e2e"] = {"value": dist_util.job_value(e_units, e_total_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                           "d2h_bytes_per_step": d2h, "ms_per_step": e_total_ms / args.steps}
+                           "d2h_bytes_per_step": d2h, "ms_per_step": e_total_ms / args.steps,
+                           "transfer": "pinned host buffers; the library lets the attend kernel read the inputs from "
+                                       "them and write out into them where that is faster, else copies (both inside "
+                                       "the timed region)"}
         if not args.no_cpu_baseline and world == 1:   # the oracle is timed beside the single-GPU run only
             line["cpu_baseline"] = cpu_baseline(w, r)
             line["retained_set_overlap"] = line["cpu_baseline"].pop("retained_set_overlap", None)

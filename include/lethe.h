@@ -166,13 +166,19 @@ lethe_status lethe_decode_attend(lethe_ctx *ctx, const lethe_cache *cache, int l
 
 /*
  * The same step with HOST-resident per-step tensors: q, k_new, v_new, token_pos and
- * out (and lse if not NULL) are HOST pointers (pinned memory makes the copies
- * asynchronous).  The call copies the inputs to context-owned device staging, runs
- * lethe_decode_attend, and copies out (and lse) back; the results are valid in host memory
- * once `stream` has been synchronised.  The cache stays on the device.  A call that covers
- * many layers is cut into two chunks of layers whose uploads and downloads run on two
- * context-owned streams under the kernel of the other chunk (the kernels stay on `stream`,
- * which also waits for the last download); smaller calls do everything on `stream`.
+ * out (and lse if not NULL) are HOST pointers.  The results are valid in host memory once
+ * `stream` has been synchronised; the input buffers must stay unchanged until then.  The
+ * cache stays on the device.  Two paths, chosen per call from the kind of memory:
+ *  - page-locked buffers (cudaHostAlloc / cudaHostRegister): the kernel writes out (and
+ *    lse) straight into the caller's buffers, and when the launch takes the persistent
+ *    asynchronous-epilogue kernel it also reads q, k_new, v_new, token_pos from them, so
+ *    that no copy precedes or follows the launch; otherwise the inputs are uploaded to
+ *    context-owned device staging first;
+ *  - pageable buffers: inputs are uploaded to the staging, lethe_decode_attend runs, and
+ *    out (and lse) are copied back.  A call that covers many layers is cut into two
+ *    chunks of layers whose uploads and downloads run on two context-owned streams under
+ *    the kernel of the other chunk (the kernels stay on `stream`, which also waits for the
+ *    last download); smaller calls do everything on `stream`.
  */
 lethe_status lethe_decode_attend_host(lethe_ctx *ctx, const lethe_cache *cache, int layer_begin, int layer_end,
                                       const void *q_host, const void *k_new_host, const void *v_new_host,

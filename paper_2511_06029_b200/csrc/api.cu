@@ -93,6 +93,8 @@ struct lethe_ctx {
     cudaEvent_t ev_start, ev_up[8], ev_done[8], ev_down;
     bool host_pipeline_ready;
     int variant, splits;
+    int picked_variant;  // kernel family the last lethe_decode_attend resolved to (-1: none of the bf16 ones)
+    bool resolve_only;   // lethe_decode_attend stops after resolving the kernel (used by the host entry point)
     int prefill_engine;  // 0 = tcgen05 kernels (TMA producers when the cache is contiguous), 1 = mma.sync kernels, 2 = tcgen05 with cp.async producers
     // TMA variant: tensor maps of the last cache seen (rebuilt when k, v, the row count or D change)
     alignas(64) unsigned char tma_maps[512];
@@ -357,10 +359,12 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
     const bool mma_ok = c->dtype == LETHE_BF16 && (!paged || c->page_tokens == kGroupTokens);
     const int cap_groups = (a.cap_tokens + kGroupTokens - 1) / kGroupTokens;
     int variant = ctx->variant;
+    ctx->picked_variant = -1;
 
     if (c->dtype == LETHE_FP8_E4M3 || c->dtype == LETHE_FP8_E5M2) {
         // quantised cache: its own clustered tensor-core kernel; variants 2..7 pick its shape, the rest mean "default"
         if (paged && c->page_tokens != kGroupTokens) return fail(ctx, LETHE_ERR_UNSUPPORTED, "quantised caches need 16-token pages");
+        if (ctx->resolve_only) return LETHE_OK;
         if (c->n_layers > kMaxLayers) return fail(ctx, LETHE_ERR_UNSUPPORTED, "more than 128 layers");
         for (int l = 0; l < c->n_layers; ++l) {
             a.k_scale[l] = c->k_scale ? c->k_scale[l] : 1.f;
@@ -446,6 +450,8 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         } else variant = 2;  // few items per launch (one layer at a time): clustered kernel, 4 warps x 3 stages
     }
     if (variant >= 2 && !mma_ok) return fail(ctx, LETHE_ERR_UNSUPPORTED, "tensor-core variants need bf16 and 16-token pages");
+    ctx->picked_variant = variant;
+    if (ctx->resolve_only) return LETHE_OK;
 
     cudaError_t e;
     if (variant >= 32) {  // clustered kernel's arithmetic, CTAs of an item merged through scratch instead of a cluster
@@ -576,21 +582,64 @@ lethe_status lethe_decode_attend_host(lethe_ctx* ctx, const lethe_cache* c, int 
     if (st != LETHE_OK) return st;
     char* p = (char*)ctx->staging;
     void* dq = p; p += up(q_bytes);
-    void* dout = p; p += up(q_bytes);
+    void* dout = p; p += up(q_bytes);  // re-pointed below when the kernel can write the caller's buffer
     void* dk = p; p += up(kv_bytes);
     void* dv = p; p += up(kv_bytes);
     int32_t* dpos = (int32_t*)p; p += up(pos_bytes);
     float* dlse = (float*)p;
     cudaStream_t s = (cudaStream_t)stream;
     cudaError_t e;
-    // Layers are independent, so a call that covers many of them is cut into two chunks of layers: the upload of the
-    // second and the download of the first run on their own streams (separate copy engines) under the other
-    // chunk's kernel.  (Measured on the Llama-8B shape: 0.344 ms per step as one chunk, 0.318 as two, 0.326 as
-    // three, 0.351 as four: smaller launches lose more than the shorter exposed copies gain.)  Small calls take the
-    // plain path: upload, one launch, download, all on the caller's stream.
+    // Results that live in page-locked host memory are written there by the kernel itself (the device-side alias of
+    // the buffer): the stores cross the bus while the kernel runs and no download follows.  Pageable buffers are
+    // staged in device memory and copied.
+    auto device_alias = [](void* host, size_t bytes) -> void* {
+        cudaPointerAttributes lo, hi;
+        if (cudaPointerGetAttributes(&lo, host) != cudaSuccess ||
+            cudaPointerGetAttributes(&hi, (char*)host + bytes - 1) != cudaSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        if (lo.type != cudaMemoryTypeHost || hi.type != cudaMemoryTypeHost || !lo.devicePointer || !hi.devicePointer) return nullptr;
+        if ((char*)hi.devicePointer - (char*)lo.devicePointer != (ptrdiff_t)(bytes - 1)) return nullptr;
+        return lo.devicePointer;
+    };
+    void* out_alias = device_alias(out_host, q_bytes);
+    float* lse_alias = (lse_host && out_alias) ? (float*)device_alias(lse_host, lse_bytes) : nullptr;
+    if (lse_host && !lse_alias) out_alias = nullptr;  // one path for both results
+    if (out_alias) {
+        dout = out_alias;
+        if (lse_host) dlse = lse_alias;
+    }
+    // Inputs in page-locked memory: the asynchronous-epilogue kernel reads them over the bus itself, under the
+    // streaming of the previous item (an item's query rows are fetched an item ahead), and no upload precedes the
+    // launch.  Measured per step, outputs written by the kernel in both cases: Llama-8B shape 0.23 ms against 0.29 ms
+    // with the upload, long-reasoning shape 2.92 against 3.29; the synchronous persistent kernel loses (Qwen shape
+    // 0.86 against 0.76), so launches of every other kernel keep the staged upload.
+    if (out_alias) {
+        void* qa = device_alias((void*)q_host, q_bytes);
+        void* ka = k_new_host ? device_alias((void*)k_new_host, kv_bytes) : nullptr;
+        void* va = v_new_host ? device_alias((void*)v_new_host, kv_bytes) : nullptr;
+        void* pa = k_new_host ? device_alias((void*)token_pos_host, pos_bytes) : nullptr;
+        if (qa && (!k_new_host || (ka && va && pa))) {
+            ctx->resolve_only = true;
+            st = lethe_decode_attend(ctx, c, layer_begin, layer_end, qa, ka, va, (const int32_t*)pa, scale, gamma, dout,
+                                     lse_host ? dlse : nullptr, stream);
+            ctx->resolve_only = false;
+            if (st != LETHE_OK) return st;
+            if (ctx->picked_variant >= 16 && ctx->picked_variant < 32)
+                return lethe_decode_attend(ctx, c, layer_begin, layer_end, qa, ka, va, (const int32_t*)pa, scale, gamma,
+                                           dout, lse_host ? dlse : nullptr, stream);
+        }
+    }
+    // Staged path.  Layers are independent, so a call that covers many of them is cut into two chunks of layers: the
+    // upload of the second and the download of the first run on their own streams (separate copy engines) under the
+    // other chunk's kernel.  (Measured on the Llama-8B shape with staged results: 0.344 ms per step as one chunk,
+    // 0.318 as two, 0.326 as three, 0.351 as four: smaller launches lose more than the shorter exposed copies gain.)
+    // When the kernel writes the results itself there is no download to hide and one chunk is best (0.288 against
+    // 0.305 as two).  Small calls take the plain path: upload, one launch, download, all on the caller's stream.
     const long long items_per_layer = (long long)c->batch * c->n_kv_heads;
     int chunks = 1;
-    if (nl >= 4 && items_per_layer * (long long)(nl / 2) >= 4LL * ctx->sm_count) chunks = 2;
+    if (!out_alias && nl >= 4 && items_per_layer * (long long)(nl / 2) >= 4LL * ctx->sm_count) chunks = 2;
     if (chunks > 1 && !ctx->host_pipeline_ready) {
         bool ok = cudaStreamCreateWithFlags(&ctx->up_stream, cudaStreamNonBlocking) == cudaSuccess &&
                   cudaStreamCreateWithFlags(&ctx->down_stream, cudaStreamNonBlocking) == cudaSuccess &&
@@ -613,6 +662,7 @@ lethe_status lethe_decode_attend_host(lethe_ctx* ctx, const lethe_cache* c, int 
         st = lethe_decode_attend(ctx, c, layer_begin, layer_end, dq, k_new_host ? dk : nullptr, k_new_host ? dv : nullptr,
                                  k_new_host ? dpos : nullptr, scale, gamma, dout, lse_host ? dlse : nullptr, stream);
         if (st != LETHE_OK) return st;
+        if (out_alias) return LETHE_OK;
         e = cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, s);
         if (e == cudaSuccess && lse_host) e = cudaMemcpyAsync(lse_host, dlse, lse_bytes, cudaMemcpyDeviceToHost, s);
         if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attend_host: download");
@@ -644,6 +694,10 @@ lethe_status lethe_decode_attend_host(lethe_ctx* ctx, const lethe_cache* c, int 
                                  k_new_host ? dpos : nullptr, scale, gamma, (char*)dout + l0 * q_layer,
                                  lse_host ? dlse + l0 * (lse_layer / 4) : nullptr, stream);
         if (st != LETHE_OK) return st;
+        if (out_alias) {
+            l0 = l1;
+            continue;
+        }
         e = cudaEventRecord(ctx->ev_done[ci], s);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->down_stream, ctx->ev_done[ci], 0);
         if (e == cudaSuccess)
@@ -654,6 +708,7 @@ lethe_status lethe_decode_attend_host(lethe_ctx* ctx, const lethe_cache* c, int 
         if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attend_host: download");
         l0 = l1;
     }
+    if (out_alias) return LETHE_OK;
     // the caller's stream ends after the last download: synchronising it is enough to read the results
     e = cudaEventRecord(ctx->ev_down, ctx->down_stream);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(s, ctx->ev_down, 0);

@@ -480,12 +480,16 @@ def test_free_running_overlap_llama_shape(ctx):
         oracle.set_threads(1)
 
 
+@pytest.mark.parametrize("pinned", [True, False])
 @pytest.mark.parametrize("L,B,Hkv", [(2, 2, 2), (5, 16, 20)])
-def test_host_entry_point_matches_the_device_one(ctx, L, B, Hkv):
-    """lethe_decode_attend_host (pinned host tensors in, host tensors out) against lethe_decode_attend on a copy of
-    the same cache: the small call takes the single-stream path, the large one the chunked path whose copies
-    overlap the kernels.  Appended rows, positions and lengths must be identical, outputs and relevance equal up
-    to the kernels' tolerance (the chunks may run a different kernel variant than the whole call)."""
+def test_host_entry_point_matches_the_device_one(ctx, L, B, Hkv, pinned):
+    """lethe_decode_attend_host (host tensors in, host tensors out) against lethe_decode_attend on a copy of the
+    same cache.  Page-locked buffers: the kernel writes the results into them itself, and the large call (persistent
+    kernel) also reads its inputs from them; pageable buffers: staged copies, the small call on one stream, the
+    large one as two chunks whose copies overlap the kernels.  Appended rows, positions and lengths must be
+    identical, outputs and relevance equal up to the kernels' tolerance (the chunks may run a different kernel
+    variant than the whole call)."""
+    pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
     G, D, cap, n0 = 4, 64, 96, 70
     Hq = Hkv * G
     oc = random_cache(L, B, Hq, Hkv, D, cap, n0, dtype=torch.bfloat16, seed=L + B, rel_init="rand")
@@ -501,9 +505,9 @@ def test_host_entry_point_matches_the_device_one(ctx, L, B, Hkv):
         out_a = torch.empty_like(q, device=dev)
         lse_a = torch.empty((L, B, Hq), dtype=torch.float32, device=dev)
         ctx.decode_attend(ga, 0, L, q.to(dev), kn.to(dev), vn.to(dev), tp.to(dev), scale, 0.9, out_a, lse_a)
-        qh, kh, vh, th = q.pin_memory(), kn.pin_memory(), vn.pin_memory(), tp.pin_memory()
-        out_b = torch.empty_like(q).pin_memory()
-        lse_b = torch.empty((L, B, Hq), dtype=torch.float32).pin_memory()
+        qh, kh, vh, th = pin(q), pin(kn), pin(vn), pin(tp)
+        out_b = pin(torch.empty_like(q))
+        lse_b = pin(torch.empty((L, B, Hq), dtype=torch.float32))
         ctx.decode_attend_host(gb, 0, L, qh, kh, vh, th, scale, 0.9, out_b, lse_b)
         assert ctx.poll_status()[0] == 0                       # synchronises the stream: host results are valid
         assert (out_b.float() - out_a.cpu().float()).abs().max() <= 1e-2
@@ -513,8 +517,8 @@ def test_host_entry_point_matches_the_device_one(ctx, L, B, Hkv):
         assert torch.equal(gb.v.cpu().view(torch.int16), ga.v.cpu().view(torch.int16))
         assert torch.allclose(gb.rel.cpu(), ga.rel.cpu(), rtol=1e-3, atol=1e-6)
     # attend-only through the host path
-    q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16).pin_memory()
-    out_b = torch.empty_like(q).pin_memory()
+    q = pin(torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16))
+    out_b = pin(torch.empty_like(q))
     out_a = torch.empty_like(q, device=dev)
     ctx.decode_attend(ga, 0, L, q.to(dev), None, None, None, scale, 0.9, out_a)
     ctx.decode_attend_host(gb, 0, L, q, None, None, None, scale, 0.9, out_b, None)
