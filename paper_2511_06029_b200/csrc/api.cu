@@ -434,9 +434,9 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
             // scratch, and what matters is how much of a typical item still fits on chip: the asynchronous (5,3)
             // while each of its two buffers holds at least 0.4 of the capacity (caches are sized well above the
             // lengths they reach between prune rounds), else the synchronous (8,2), whose stages leave the most room
-            // for its single buffer.  Measured: Llama shape at capacities 3584 / 4608 / 6144 0.88 of the copy peak
-            // with the former against 0.86 to 0.88 with the latter; long-reasoning shape 1.00 against 0.985; Qwen
-            // shape (8 logit columns per token, capacity 5312) 0.95 with the latter against 0.61 to 0.80.
+            // for its single buffer.  Measured: Llama shape at capacities 3584 / 4608 / 6144 0.93 of the copy peak
+            // with the former against 0.90 to 0.95 with the latter; long-reasoning shape 1.04 against 1.02; Qwen
+            // shape (8 logit columns per token, capacity 5312) 0.99 with the latter against 0.84 to 0.93.
             const int cap_pad = cap_groups * kGroupTokens;
             auto async_fits = [&](int shape) { return async_smem_bytes(c->head_dim, shape, cap_pad, a.GP) <= ctx->max_smem; };
             variant = 0;
@@ -610,11 +610,13 @@ lethe_status lethe_decode_attend_host(lethe_ctx* ctx, const lethe_cache* c, int 
         dout = out_alias;
         if (lse_host) dlse = lse_alias;
     }
-    // Inputs in page-locked memory: the asynchronous-epilogue kernel reads them over the bus itself, under the
-    // streaming of the previous item (an item's query rows are fetched an item ahead), and no upload precedes the
-    // launch.  Measured per step, outputs written by the kernel in both cases: Llama-8B shape 0.23 ms against 0.29 ms
-    // with the upload, long-reasoning shape 2.92 against 3.29; the synchronous persistent kernel loses (Qwen shape
-    // 0.86 against 0.76), so launches of every other kernel keep the staged upload.
+    // Inputs in page-locked memory: the persistent kernels read them over the bus themselves, an item ahead of their
+    // use and under the streaming of the previous item, and no upload precedes the launch.  The asynchronous-epilogue
+    // kernel reads every input byte once (an epilogue warp stages an item's query rows and appended row in shared
+    // memory); the synchronous one fetches them per warp into registers.  Measured per step, results written by the
+    // kernel in both cases: Llama-8B shape 0.22 to 0.23 ms against 0.29 ms with the upload, long-reasoning shape 2.81
+    // against 3.20, Qwen shape 0.67 against 0.80.  Launches of the other kernels (one CTA or cluster per item, the
+    // query rows needed at once) keep the staged upload.
     if (out_alias) {
         void* qa = device_alias((void*)q_host, q_bytes);
         void* ka = k_new_host ? device_alias((void*)k_new_host, kv_bytes) : nullptr;
@@ -626,7 +628,7 @@ lethe_status lethe_decode_attend_host(lethe_ctx* ctx, const lethe_cache* c, int 
                                      lse_host ? dlse : nullptr, stream);
             ctx->resolve_only = false;
             if (st != LETHE_OK) return st;
-            if (ctx->picked_variant >= 16 && ctx->picked_variant < 32)
+            if (ctx->picked_variant >= 8 && ctx->picked_variant < 32)
                 return lethe_decode_attend(ctx, c, layer_begin, layer_end, qa, ka, va, (const int32_t*)pa, scale, gamma,
                                            dout, lse_host ? dlse : nullptr, stream);
         }

@@ -34,8 +34,14 @@ struct AsyncHeader {
     int desc_ticket[4];           // ring by item sequence number: ticket (>= n_items: no more work)
     int desc_n_old[4];            //                              len of that item before this call
     int abort;
-    int pad[3];
+    int new_pos[2];               // by item parity: position of the appended token
+    int pad;
     float2 wstat[2][16][kMaxGroup];
+    // The call's inputs of an item, staged once per item by an epilogue warp (by item parity): the G query rows and
+    // the appended k / v row.  Every byte of q, k_new, v_new is therefore read once per launch, which is what lets
+    // these buffers sit in page-locked host memory.
+    uint4 q_stage[2][kMaxGroup * 128 * 2 / 16];
+    uint4 new_stage[2][2][16];
 };
 
 __device__ __forceinline__ void mbar_init(unsigned long long* bar, int count) {
@@ -96,7 +102,16 @@ struct AsyncItem {
     int valid;
     int item, li, l, b, hkv;
     int n_old, n, full;
-    int count, app_idx;  // streaming warps only
+    int count, app_idx, par;  // streaming warps only (par: parity of the item's sequence number in this CTA)
+};
+
+// Registers that carry one item's inputs from global (or mapped host) memory to the staging area: loaded early,
+// stored once the staging slot is free.
+template <int D>
+struct StagedInputs {
+    uint4 q[D / 32];  // 16-byte chunks lane, lane + 32, ... of the item's G query rows
+    uint4 row;        // lanes 0..15: chunk of the appended k row; lanes 16..31: of the v row
+    int pos;
 };
 
 __device__ __forceinline__ void async_decode(const AttendArgs& a, int ticket, int n_old, AsyncItem& it) {
@@ -115,19 +130,46 @@ __device__ __forceinline__ void async_decode(const AttendArgs& a, int ticket, in
     it.app_idx = -1;
 }
 
-// Sec. 4.1: the generated token's k / v row enters the cache (kept out of line: once per item).
+template <int D>
+__device__ __forceinline__ void load_inputs(const AttendArgs& a, const AsyncItem& it, int lane, StagedInputs<D>& r) {
+    using T = __nv_bfloat16;
+    constexpr int ROW_CHUNKS = D * 2 / 16;
+    const int q_chunks = a.G * D * 2 / 16;
+    const uint4* qsrc = reinterpret_cast<const uint4*>((const T*)a.q + ((size_t)(it.li * a.B + it.b) * a.Hq + it.hkv * a.G) * D);
+#pragma unroll
+    for (int i = 0; i < D / 32; ++i) {
+        const int c = i * 32 + lane;
+        r.q[i] = (it.valid && c < q_chunks) ? qsrc[c] : make_uint4(0u, 0u, 0u, 0u);
+    }
+    r.row = make_uint4(0u, 0u, 0u, 0u);
+    r.pos = 0;
+    if (a.k_new && it.valid) {
+        const size_t src = ((size_t)(it.li * a.B + it.b) * a.Hkv + it.hkv) * ROW_CHUNKS;
+        const int c = lane & 15;
+        if (c < ROW_CHUNKS) r.row = reinterpret_cast<const uint4*>(lane < 16 ? a.k_new : a.v_new)[src + c];
+        if (lane == 0) r.pos = a.token_pos[it.b];
+    }
+}
+template <int D>
+__device__ __forceinline__ void store_inputs(AsyncHeader& hd, int par, int lane, const StagedInputs<D>& r) {
+#pragma unroll
+    for (int i = 0; i < D / 32; ++i) hd.q_stage[par][i * 32 + lane] = r.q[i];
+    hd.new_stage[par][lane >> 4][lane & 15] = r.row;
+    if (lane == 0) hd.new_pos[par] = r.pos;
+}
+
+// Sec. 4.1: the generated token's k / v row enters the cache, from the staging area (kept out of line: once per item).
 template <bool PAGED>
-__device__ __noinline__ void append_row(const AttendArgs& a, int item, int li, int b, int hkv, int n_old, int row_bytes,
-                                        int lane) {
-    const size_t src = ((size_t)(li * a.B + b) * a.Hkv + hkv) * row_bytes;
+__device__ __noinline__ void append_row(const AttendArgs& a, int item, int n_old, int row_bytes, const uint4* staged_k,
+                                        const uint4* staged_v, int token_pos, int lane) {
     bool bad = false;
     char* kd = const_cast<char*>(row_ptr<PAGED>(a, a.k, item, n_old, row_bytes, &bad));
     char* vd = const_cast<char*>(row_ptr<PAGED>(a, a.v, item, n_old, row_bytes, &bad));
     if (kd && vd && lane * 16 < row_bytes) {
-        *reinterpret_cast<uint4*>(kd + lane * 16) = *reinterpret_cast<const uint4*>((const char*)a.k_new + src + lane * 16);
-        *reinterpret_cast<uint4*>(vd + lane * 16) = *reinterpret_cast<const uint4*>((const char*)a.v_new + src + lane * 16);
+        *reinterpret_cast<uint4*>(kd + lane * 16) = staged_k[lane];
+        *reinterpret_cast<uint4*>(vd + lane * 16) = staged_v[lane];
     }
-    if (lane == 0) a.pos[(size_t)item * a.cap_tokens + n_old] = a.token_pos[b];
+    if (lane == 0) a.pos[(size_t)item * a.cap_tokens + n_old] = token_pos;
     __syncwarp();
 }
 
@@ -186,25 +228,36 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
         }
         return;
     }
-    if (warp == NWS && lane == 0) {
-        int t0 = (int)atomicAdd(&sched[0], 1u);
-        int t1 = a.n_items;
-        if (t0 >= a.n_items) drew_fail = true;
-        else {
-            t1 = (int)atomicAdd(&sched[0], 1u);
-            if (t1 >= a.n_items) drew_fail = true;
+    if (warp == NWS) {  // the first two tickets, and what their items need from the call's inputs
+        int t0 = a.n_items, t1 = a.n_items;
+        if (lane == 0) {
+            t0 = (int)atomicAdd(&sched[0], 1u);
+            if (t0 >= a.n_items) drew_fail = true;
+            else {
+                t1 = (int)atomicAdd(&sched[0], 1u);
+                if (t1 >= a.n_items) drew_fail = true;
+            }
+            if (a.order) {  // longest-first order of the items (valid tickets only)
+                if (t0 < a.n_items) t0 = a.order[t0];
+                if (t1 < a.n_items) t1 = a.order[t1];
+            }
         }
-        if (a.order) {  // longest-first order of the items (valid tickets only)
-            if (t0 < a.n_items) t0 = a.order[t0];
-            if (t1 < a.n_items) t1 = a.order[t1];
+        t0 = __shfl_sync(0xffffffffu, t0, 0);
+        t1 = __shfl_sync(0xffffffffu, t1, 0);
+        AsyncItem i0, i1;
+        async_decode(a, t0, 0, i0);
+        async_decode(a, t1, 0, i1);
+        StagedInputs<D> r0, r1;
+        load_inputs<D>(a, i0, lane, r0);
+        load_inputs<D>(a, i1, lane, r1);
+        if (lane == 0) {
+            hd.desc_ticket[0] = t0;
+            hd.desc_n_old[0] = i0.valid ? a.len[i0.item] : 0;
+            hd.desc_ticket[1] = t1;
+            hd.desc_n_old[1] = i1.valid ? a.len[i1.item] : 0;
         }
-        AsyncItem tmp;
-        async_decode(a, t0, 0, tmp);
-        hd.desc_ticket[0] = t0;
-        hd.desc_n_old[0] = tmp.valid ? a.len[tmp.item] : 0;
-        async_decode(a, t1, 0, tmp);
-        hd.desc_ticket[1] = t1;
-        hd.desc_n_old[1] = tmp.valid ? a.len[tmp.item] : 0;
+        store_inputs<D>(hd, 0, lane, r0);
+        store_inputs<D>(hd, 1, lane, r1);
     }
     __syncthreads();
 
@@ -212,8 +265,7 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
         // =================================================================== streaming warps
         const int gq = lane >> 2, tq = lane & 3;
         auto load_q = [&](const AsyncItem& it, uint32_t (&bq)[KS][2]) {
-            const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
-                (const T*)a.q + ((size_t)(it.li * a.B + it.b) * a.Hq + it.hkv * G + gq) * D);
+            const uint32_t* qrow = reinterpret_cast<const uint32_t*>(hd.q_stage[it.par]) + gq * (D / 2);
 #pragma unroll
             for (int ks = 0; ks < KS; ++ks) {
                 bq[ks][0] = (it.valid && gq < G) ? qrow[8 * ks + tq] : 0u;
@@ -249,7 +301,8 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
             const int grp = warp + idx * NWS;
             const int tok0 = grp * kGroupTokens;
             if (idx == it.app_idx) {
-                append_row<PAGED>(a, it.item, it.li, it.b, it.hkv, it.n_old, ROW_BYTES, lane);
+                append_row<PAGED>(a, it.item, it.n_old, ROW_BYTES, hd.new_stage[it.par][0], hd.new_stage[it.par][1],
+                                  hd.new_pos[it.par], lane);
                 if (TMA) {  // the row was written through the generic proxy; the TMA load reads through the async proxy
                     fence_proxy_async();
                     __syncwarp();
@@ -315,6 +368,7 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
 
         AsyncItem cur, nxt;
         async_decode(a, hd.desc_ticket[0], hd.desc_n_old[0], cur);
+        cur.par = 0;
         set_counts(cur);
         uint32_t bq[KS][2], bqn[KS][2];
         load_q(cur, bq);
@@ -341,6 +395,7 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
                     nxt.valid = 0;
                 } else {
                     async_decode(a, hd.desc_ticket[sn & 3], hd.desc_n_old[sn & 3], nxt);
+                    nxt.par = sn & 1;
                     set_counts(nxt);
                     load_q(nxt, bqn);
                     pg_nxt = load_pages(nxt, 0);
@@ -570,6 +625,21 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
                             l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
                 }
             }
+            // Epilogue warp 0 fetches what the item after next needs from the call's inputs; the loads complete
+            // behind the output and relevance work below.
+            AsyncItem nx;
+            StagedInputs<D> staged;
+            int nx_n_old = 0;
+            if (ew == 0) {
+                if (lane == 0) {
+                    if (t_new >= a.n_items) drew_fail = true;
+                    else if (a.order) t_new = a.order[t_new];
+                }
+                t_new = __shfl_sync(0xffffffffu, t_new, 0);
+                async_decode(a, t_new, 0, nx);
+                load_inputs<D>(a, nx, lane, staged);
+                if (lane == 0 && nx.valid) nx_n_old = a.len[nx.item];
+            }
             const bool item_overflows = SPILL && it.n > chunk;
             // One token's G logits (from shared memory, or from the overflow area), then its attention mass.
             auto load_row = [&](int j, float2 (&s)[kMaxGroup / 2]) {
@@ -642,15 +712,14 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
                     }
                 }
             }
-            if (ew == 0 && lane == 0) {
-                if (it.full) record_error(a.status, LETHE_ERR_CAPACITY, it.item);
-                else if (append) a.len[it.item] = it.n;
-                if (t_new >= a.n_items) drew_fail = true;
-                if (a.order && t_new < a.n_items) t_new = a.order[t_new];
-                AsyncItem nx;
-                async_decode(a, t_new, 0, nx);
-                hd.desc_n_old[(seq + 2) & 3] = nx.valid ? a.len[nx.item] : 0;
-                hd.desc_ticket[(seq + 2) & 3] = t_new;
+            if (ew == 0) {
+                store_inputs<D>(hd, p, lane, staged);  // item seq + 2 has the parity of this one, whose slot is free
+                if (lane == 0) {
+                    if (it.full) record_error(a.status, LETHE_ERR_CAPACITY, it.item);
+                    else if (append) a.len[it.item] = it.n;
+                    hd.desc_n_old[(seq + 2) & 3] = nx_n_old;
+                    hd.desc_ticket[(seq + 2) & 3] = t_new;
+                }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&hd.empty[p]);

@@ -113,9 +113,24 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
             bq[ks][1] = (it.valid && gq < G) ? qrow[8 * ks + 4 + tq] : 0u;
         }
     };
+    // The appended row of an item (lanes 0..15: 16-byte chunks of the k row, lanes 16..31: of the v row) and its
+    // position are fetched together with the query rows, an item ahead: the append itself then never waits on them.
+    auto load_new = [&](const StreamItem& it, uint4& row, int& pos) {
+        row = make_uint4(0u, 0u, 0u, 0u);
+        pos = 0;
+        if (append && it.valid) {
+            const size_t src = ((size_t)(it.li * a.B + it.b) * a.Hkv + it.hkv) * CHUNKS;
+            if ((lane & 15) < CHUNKS) row = reinterpret_cast<const uint4*>(lane < 16 ? a.k_new : a.v_new)[src + (lane & 15)];
+            pos = a.token_pos[it.b];
+        }
+    };
     uint32_t bq[KS][2], bqn[KS][2];
+    uint4 new_row, new_row_n;
+    int new_pos, new_pos_n;
     load_q(cur, bq);
     load_q(nxt, bqn);
+    load_new(cur, new_row, new_pos);
+    load_new(nxt, new_row_n, new_pos_n);
 
     unsigned char* my_stage = smem_raw + (size_t)warp * WARP_BYTES;
     const uint32_t my_stage_u32 = smem_u32(my_stage);
@@ -136,15 +151,12 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
         const int grp = warp + idx * NW;
         const int tok0 = grp * kGroupTokens;
         if (idx == it.app_idx) {  // Sec. 4.1: the generated token's k / v row enters the cache first
-            const size_t src = ((size_t)(it.li * a.B + it.b) * a.Hkv + it.hkv) * ROW_BYTES;
             bool bad = false;
             char* kd = const_cast<char*>(row_ptr<PAGED>(a, a.k, it.item, it.n_old, ROW_BYTES, &bad));
             char* vd = const_cast<char*>(row_ptr<PAGED>(a, a.v, it.item, it.n_old, ROW_BYTES, &bad));
-            if (kd && vd && lane * 16 < ROW_BYTES) {
-                *reinterpret_cast<uint4*>(kd + lane * 16) = *reinterpret_cast<const uint4*>((const char*)a.k_new + src + lane * 16);
-                *reinterpret_cast<uint4*>(vd + lane * 16) = *reinterpret_cast<const uint4*>((const char*)a.v_new + src + lane * 16);
-            }
-            if (lane == 0) a.pos[(size_t)it.item * a.cap_tokens + it.n_old] = a.token_pos[it.b];
+            if (kd && vd && (lane & 15) < CHUNKS)
+                *reinterpret_cast<uint4*>((lane < 16 ? kd : vd) + (lane & 15) * 16) = is_cur ? new_row : new_row_n;
+            if (lane == 0) a.pos[(size_t)it.item * a.cap_tokens + it.n_old] = is_cur ? new_pos : new_pos_n;
             __syncwarp();
         }
         const char* kb;
@@ -443,10 +455,13 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
             bq[ks][0] = bqn[ks][0];
             bq[ks][1] = bqn[ks][1];
         }
+        new_row = new_row_n;
+        new_pos = new_pos_n;
         issued = issued_next;
         decode_ticket(a, es.flags[2], nxt);
         nxt_n_raw = nxt.valid ? a.len[nxt.item] : 0;
         load_q(nxt, bqn);
+        load_new(nxt, new_row_n, new_pos_n);
     }
     cp_async_wait<0>();
     if (bad_page) record_error(a.status, LETHE_ERR_PAGE, 0);
