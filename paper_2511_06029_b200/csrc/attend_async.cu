@@ -5,8 +5,11 @@
 //     parks its partial (max, sum, O) in the item's parity buffer, signals an mbarrier and goes straight on to
 //     item i+1, whose first groups its pipeline has already prefetched;
 //   * 2 epilogue warps wait for that mbarrier, merge the partials, write out / lse, apply Eq. 5 to rel with the
-//     exact normaliser, store len, draw the ticket of the item after next (and read its len), and hand the
-//     parity buffer back through a second mbarrier.
+//     exact normaliser, store len, draw the ticket of the item after next (and read its len), copy that item's
+//     query rows and appended k / v row from the call's inputs into a staging area in shared memory, and hand
+//     the parity buffer back through a second mbarrier.  The streaming warps take their query fragments and the
+//     appended row from the staging area, so each input byte is read once per launch (the inputs may therefore
+//     sit in page-locked host memory and be read over the bus, an item ahead of their use).
 // The logit buffer, the partial-output buffer and the item descriptor are double-buffered by item parity, so the
 // epilogue of item i runs entirely under the HBM stream of item i+1.  Every mbarrier wait is bounded: if it
 // runs out, the CTA records LETHE_ERR_TIMEOUT, drains its copies and returns.
