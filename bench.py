@@ -189,18 +189,20 @@ def timed_loop(r: Runner, steps: int, host: bool):
     """Run `steps` steps; returns (total_ms, attend_ms list, prune_ms list, token_heads list)."""
     dev = r.dev
     stream = torch.cuda.current_stream(dev)
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * steps)]
+    ev = [] if host else [torch.cuda.Event(enable_timing=True) for _ in range(2 * steps)]   # per-launch times: device loop only
     prune_ev = []
     len_snap = [(0, r.cache.len.clone())]
     t_begin = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize(dev)
     t_begin.record(stream)
     for s in range(steps):
-        ev[2 * s].record(stream)
-        r.decode(host=host)
-        ev[2 * s + 1].record(stream)
         if host:
+            r.decode(host=True)
             stream.synchronize()               # the caller reads out before producing the next token
+        else:
+            ev[2 * s].record(stream)
+            r.decode(host=False)
+            ev[2 * s + 1].record(stream)
         if r.prune_due():
             a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
             a.record(stream)
@@ -213,7 +215,7 @@ def timed_loop(r: Runner, steps: int, host: bool):
     t_end.record(stream)
     torch.cuda.synchronize(dev)
     total_ms = t_begin.elapsed_time(t_end)
-    attend_ms = [ev[2 * s].elapsed_time(ev[2 * s + 1]) for s in range(steps)]
+    attend_ms = [] if host else [ev[2 * s].elapsed_time(ev[2 * s + 1]) for s in range(steps)]
     prune_ms = [a.elapsed_time(b) for a, b in prune_ev]
     # token-heads attended at step s = sum of len after that step's append
     items = r.cache.len.numel()
@@ -618,9 +620,9 @@ def main():
         if not args.no_e2e:
             line["e2e"] = {"value": dist_util.job_value(e_units, e_total_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                            "d2h_bytes_per_step": d2h, "ms_per_step": e_total_ms / args.steps,
-                           "transfer": "pinned host buffers; the library lets the attend kernel read the inputs from "
-                                       "them and write out into them where that is faster, else copies (both inside "
-                                       "the timed region)"}
+                           "transfer": "pinned host buffers; the attend kernel reads the step's inputs from them and "
+                                       "writes out into them over the bus, inside the timed launch (pageable buffers "
+                                       "would take staged copies)"}
         if not args.no_cpu_baseline and world == 1:   # the oracle is timed beside the single-GPU run only
             line["cpu_baseline"] = cpu_baseline(w, r)
             line["retained_set_overlap"] = line["cpu_baseline"].pop("retained_set_overlap", None)

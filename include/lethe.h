@@ -170,10 +170,10 @@ lethe_status lethe_decode_attend(lethe_ctx *ctx, const lethe_cache *cache, int l
  * `stream` has been synchronised; the input buffers must stay unchanged until then.  The
  * cache stays on the device.  Two paths, chosen per call from the kind of memory:
  *  - page-locked buffers (cudaHostAlloc / cudaHostRegister): the kernel writes out (and
- *    lse) straight into the caller's buffers, and when the launch takes one of the
- *    persistent kernels (many items per launch) it also reads q, k_new, v_new, token_pos
- *    from them, so that no copy precedes or follows the launch; otherwise the inputs are
- *    uploaded to context-owned device staging first;
+ *    lse) straight into the caller's buffers and, when the inputs are page-locked too,
+ *    reads q, k_new, v_new, token_pos from them, so that no copy precedes or follows the
+ *    launch (page-locked results with pageable inputs: the inputs are uploaded to
+ *    context-owned device staging first);
  *  - pageable buffers: inputs are uploaded to the staging, lethe_decode_attend runs, and
  *    out (and lse) are copied back.  A call that covers many layers is cut into two
  *    chunks of layers whose uploads and downloads run on two context-owned streams under

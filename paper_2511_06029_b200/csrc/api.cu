@@ -93,8 +93,6 @@ struct lethe_ctx {
     cudaEvent_t ev_start, ev_up[8], ev_done[8], ev_down;
     bool host_pipeline_ready;
     int variant, splits;
-    int picked_variant;  // kernel family the last lethe_decode_attend resolved to (-1: none of the bf16 ones)
-    bool resolve_only;   // lethe_decode_attend stops after resolving the kernel (used by the host entry point)
     int prefill_engine;  // 0 = tcgen05 kernels (TMA producers when the cache is contiguous), 1 = mma.sync kernels, 2 = tcgen05 with cp.async producers
     // TMA variant: tensor maps of the last cache seen (rebuilt when k, v, the row count or D change)
     alignas(64) unsigned char tma_maps[512];
@@ -359,12 +357,10 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
     const bool mma_ok = c->dtype == LETHE_BF16 && (!paged || c->page_tokens == kGroupTokens);
     const int cap_groups = (a.cap_tokens + kGroupTokens - 1) / kGroupTokens;
     int variant = ctx->variant;
-    ctx->picked_variant = -1;
 
     if (c->dtype == LETHE_FP8_E4M3 || c->dtype == LETHE_FP8_E5M2) {
         // quantised cache: its own clustered tensor-core kernel; variants 2..7 pick its shape, the rest mean "default"
         if (paged && c->page_tokens != kGroupTokens) return fail(ctx, LETHE_ERR_UNSUPPORTED, "quantised caches need 16-token pages");
-        if (ctx->resolve_only) return LETHE_OK;
         if (c->n_layers > kMaxLayers) return fail(ctx, LETHE_ERR_UNSUPPORTED, "more than 128 layers");
         for (int l = 0; l < c->n_layers; ++l) {
             a.k_scale[l] = c->k_scale ? c->k_scale[l] : 1.f;
@@ -450,8 +446,6 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         } else variant = 2;  // few items per launch (one layer at a time): clustered kernel, 4 warps x 3 stages
     }
     if (variant >= 2 && !mma_ok) return fail(ctx, LETHE_ERR_UNSUPPORTED, "tensor-core variants need bf16 and 16-token pages");
-    ctx->picked_variant = variant;
-    if (ctx->resolve_only) return LETHE_OK;
 
     cudaError_t e;
     if (variant >= 32) {  // clustered kernel's arithmetic, CTAs of an item merged through scratch instead of a cluster
@@ -610,28 +604,22 @@ lethe_status lethe_decode_attend_host(lethe_ctx* ctx, const lethe_cache* c, int 
         dout = out_alias;
         if (lse_host) dlse = lse_alias;
     }
-    // Inputs in page-locked memory: the persistent kernels read them over the bus themselves, an item ahead of their
-    // use and under the streaming of the previous item, and no upload precedes the launch.  The asynchronous-epilogue
-    // kernel reads every input byte once (an epilogue warp stages an item's query rows and appended row in shared
-    // memory); the synchronous one fetches them per warp into registers.  Measured per step, results written by the
-    // kernel in both cases: Llama-8B shape 0.22 to 0.23 ms against 0.29 ms with the upload, long-reasoning shape 2.81
-    // against 3.20, Qwen shape 0.67 against 0.80.  Launches of the other kernels (one CTA or cluster per item, the
-    // query rows needed at once) keep the staged upload.
+    // Inputs in page-locked memory as well: the kernels read them over the bus themselves and no upload precedes the
+    // launch.  The persistent kernels fetch them an item ahead of their use, under the streaming of the previous
+    // item; the asynchronous-epilogue kernel reads every input byte once (an epilogue warp stages an item's query
+    // rows and appended row in shared memory), the synchronous one fetches them per warp into registers.  Measured
+    // per step, results written by the kernel in both cases: Llama-8B shape 0.22 ms against 0.29 ms with the upload,
+    // long-reasoning shape 2.81 against 3.20, Qwen shape 0.67 against 0.80.  The kernels with one CTA or cluster per
+    // item need the query rows at once, so each CTA starts with a round trip over the bus, and still come out ahead
+    // of the upload (quantised Llama-8B shape 0.20 against 0.23, clustered bf16 kernel 0.35 against 0.37).
     if (out_alias) {
         void* qa = device_alias((void*)q_host, q_bytes);
         void* ka = k_new_host ? device_alias((void*)k_new_host, kv_bytes) : nullptr;
         void* va = v_new_host ? device_alias((void*)v_new_host, kv_bytes) : nullptr;
         void* pa = k_new_host ? device_alias((void*)token_pos_host, pos_bytes) : nullptr;
-        if (qa && (!k_new_host || (ka && va && pa))) {
-            ctx->resolve_only = true;
-            st = lethe_decode_attend(ctx, c, layer_begin, layer_end, qa, ka, va, (const int32_t*)pa, scale, gamma, dout,
-                                     lse_host ? dlse : nullptr, stream);
-            ctx->resolve_only = false;
-            if (st != LETHE_OK) return st;
-            if (ctx->picked_variant >= 8 && ctx->picked_variant < 32)
-                return lethe_decode_attend(ctx, c, layer_begin, layer_end, qa, ka, va, (const int32_t*)pa, scale, gamma,
-                                           dout, lse_host ? dlse : nullptr, stream);
-        }
+        if (qa && (!k_new_host || (ka && va && pa)))
+            return lethe_decode_attend(ctx, c, layer_begin, layer_end, qa, ka, va, (const int32_t*)pa, scale, gamma, dout,
+                                       lse_host ? dlse : nullptr, stream);
     }
     // Staged path.  Layers are independent, so a call that covers many of them is cut into two chunks of layers: the
     // upload of the second and the download of the first run on their own streams (separate copy engines) under the

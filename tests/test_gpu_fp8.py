@@ -213,3 +213,30 @@ def test_quantised_persistent_kernel_logit_overflow(ctx):
             _step(ctx, oc, gc, q, kn, vn, torch.tensor([1, 2], dtype=torch.int32), torch.tensor([0.05]), 0.99)
     finally:
         ctx.set_tuning(0, 0)
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_quantised_host_entry_point(ctx, pinned):
+    """lethe_decode_attend_host on a quantised cache against the oracle: page-locked buffers (the kernel reads its
+    inputs from them and writes the results into them) and pageable ones (staged copies)."""
+    L, B, Hq, Hkv, D, cap = 2, 3, 8, 2, 128, 112
+    g = torch.Generator().manual_seed(5)
+    lens = torch.randint(1, cap - 8, (L, B, Hkv), generator=g)
+    oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=9, k_scale=[0.37, 1.5], v_scale=[2.25, 0.6], fmt="e4m3")
+    gc = to_device(oc)
+    pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
+    scale = torch.tensor([0.11, 0.07], dtype=torch.float32)
+    for step in range(3):
+        q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+        kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+        vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+        tp = torch.arange(B, dtype=torch.int32) + 50 + step
+        st, ref, lse_ref, _ = oracle.decode_attend(oc, 0, L, q, kn, vn, tp, scale, 0.95, want_lse=True)
+        out = pin(torch.empty_like(q))
+        lse = pin(torch.empty((L, B, Hq), dtype=torch.float32))
+        ctx.decode_attend_host(gc, 0, L, pin(q), pin(kn), pin(vn), pin(tp), scale.tolist(), 0.95, out, lse)
+        assert st == oracle.OK and ctx.poll_status()[0] == 0      # the poll synchronises the stream
+        d = (out.float() - ref.float()).abs()
+        assert bool((d <= 2e-2 + 2.0 ** -7 * ref.float().abs()).all()), f"attention output error {d.max().item()}"
+        assert torch.allclose(lse, lse_ref, rtol=1e-4, atol=1e-4)
+        assert_state_matches(gc, oc)
