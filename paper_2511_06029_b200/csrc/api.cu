@@ -370,7 +370,8 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         // The clustered kernel (variants 2..7 pick its shape) is the default at every size: with two CTAs per SM
         // covering each other's epilogues it beats the persistent one (variants 8..13) on this conversion-bound
         // path (Llama-8B shape: 0.124 ms against 0.153 to 0.161 ms; a version of the asynchronous-epilogue kernel for
-        // byte caches was measured too, 0.165 to 0.178 ms over six shapes, and is not kept).
+        // byte caches was measured too: 0.156 to 0.178 ms with two epilogue warps, 0.131 ms at best with four and the
+        // batched relevance update (8 streaming warps x 2 stages), worse again with six; not kept).
         const bool want_persistent = variant >= 8 && variant <= 13;
         const bool want_clustered = variant >= 2 && variant <= 7;
         if (want_persistent && ctx->splits <= 1 && c->dtype == LETHE_FP8_E4M3) {
