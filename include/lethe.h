@@ -117,7 +117,7 @@ lethe_status lethe_poll_status(lethe_ctx *ctx, void *stream, int32_t *info);
  * variant: 0 = automatic; 1 = CUDA-core kernel; 2..7 = clustered tensor-core (mma) kernel with (warps per
  * CTA, pipeline stages per warp) = (4,3) (8,3) (4,2) (8,2) (4,4) (2,4); 8..15 = persistent tensor-core
  * kernel (one CTA per SM, dynamic item queue, cross-item prefetch) with (8,2) (6,3) (10,2) (8,3) (7,3) (5,4)
- * (6,2) (5,3); 16..21 = the persistent kernel with an asynchronous epilogue (two extra warps merge and write
+ * (6,2) (5,3); 16..21 = the persistent kernel with an asynchronous epilogue (extra warps, four with (8,2) and two otherwise, merge and write
  * item i while the streaming warps already read item i+1) with (8,2) (7,2) (6,3) (5,3) (6,2) (4,4); 24..29 = the same six shapes with
  * the K / V tiles staged by TMA (cp.async.bulk.tensor, 128-byte swizzle) instead of 16-byte cp.async;
  * 32..37 = the clustered kernel's six shapes with the CTAs of an item merged through global scratch (the last

@@ -426,24 +426,28 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         // enough items to give every SM several: the persistent kernel; few long items: the clustered one
         if (!mma_ok) variant = 1;
         else if (a.n_items >= 2 * ctx->sm_count && ctx->splits <= 1) {
-            // Persistent kernels.  The asynchronous-epilogue kernel (best measured first: (5,3) (6,3) (8,2) (4,4)) when
-            // both of its logit buffers cover the capacity on chip.  Otherwise the tail of long items overflows to
-            // scratch, and what matters is how much of a typical item still fits on chip: the asynchronous (5,3)
-            // while each of its two buffers holds at least 0.4 of the capacity (caches are sized well above the
-            // lengths they reach between prune rounds), else the synchronous (8,2), whose stages leave the most room
-            // for its single buffer.  Measured: Llama shape at capacities 3584 / 4608 / 6144 0.93 of the copy peak
-            // with the former against 0.90 to 0.95 with the latter; long-reasoning shape 1.04 against 1.02; Qwen
-            // shape (8 logit columns per token, capacity 5312) 0.99 with the latter against 0.84 to 0.93.
+            // Persistent kernels.  The asynchronous-epilogue kernel (best measured first: (8,2) with four epilogue
+            // warps, then (5,3) (6,3) (4,4) with two) when both of its logit buffers cover the capacity on chip.
+            // Otherwise the tail of long items overflows to scratch, and what matters is how much of a typical item
+            // still fits on chip: the asynchronous (8,2), else (5,3), while each of its two buffers holds at least
+            // 0.4 of the capacity (caches are sized well above the lengths they reach between prune rounds), else
+            // the synchronous (8,2), whose single buffer gets the most room.  Measured, of the copy peak: Llama
+            // shape at capacities 1600 / 2048 / 2560 / 3584 / 4608 / 6144 asynchronous (8,2) 1.02 / 1.00 / 0.95 /
+            // 1.00 / 0.99 / 0.99, asynchronous (5,3) 1.00 / 1.00 / 0.93 / 0.96 / 0.95 / 0.95, synchronous 0.97 /
+            // 0.96 / 0.93 / 0.97 / 0.96 / 0.92; long-reasoning shape 1.06 / 1.05 / 1.02; Qwen shape (8 logit columns
+            // per token, capacity 5312) 0.99 with the synchronous kernel against 0.84 to 0.93.
             const int cap_pad = cap_groups * kGroupTokens;
             auto async_fits = [&](int shape) { return async_smem_bytes(c->head_dim, shape, cap_pad, a.GP) <= ctx->max_smem; };
+            auto async_chunk = [&](int shape) -> size_t {
+                const size_t fixed = async_smem_bytes(c->head_dim, shape, 0, a.GP);
+                return fixed < ctx->max_smem ? (ctx->max_smem - fixed) / ((size_t)2 * a.GP * 4) : 0;
+            };
             variant = 0;
-            for (int shape : {3, 2, 0, 5})
+            for (int shape : {0, 3, 2, 5})
                 if (variant == 0 && async_fits(shape)) variant = 16 + shape;
-            if (variant == 0) {
-                const size_t fixed = async_smem_bytes(c->head_dim, 3, 0, a.GP);
-                const size_t async_chunk = fixed < ctx->max_smem ? (ctx->max_smem - fixed) / ((size_t)2 * a.GP * 4) : 0;
-                variant = (async_chunk * 5 >= (size_t)cap_pad * 2) ? 16 + 3 : 8 + 0;
-            }
+            for (int shape : {0, 3})
+                if (variant == 0 && async_chunk(shape) * 5 >= (size_t)cap_pad * 2) variant = 16 + shape;
+            if (variant == 0) variant = 8 + 0;
         } else variant = 2;  // few items per launch (one layer at a time): clustered kernel, 4 warps x 3 stages
     }
     if (variant >= 2 && !mma_ok) return fail(ctx, LETHE_ERR_UNSUPPORTED, "tensor-core variants need bf16 and 16-token pages");

@@ -4,7 +4,7 @@
 //   * NWS streaming warps never stop at a CTA-wide barrier.  When a warp has consumed its groups of item i it
 //     parks its partial (max, sum, O) in the item's parity buffer, signals an mbarrier and goes straight on to
 //     item i+1, whose first groups its pipeline has already prefetched;
-//   * 2 epilogue warps wait for that mbarrier, merge the partials, write out / lse, apply Eq. 5 to rel with the
+//   * 2 or 4 epilogue warps (epilogue_warps()) wait for that mbarrier, merge the partials, write out / lse, apply Eq. 5 to rel with the
 //     exact normaliser, store len, draw the ticket of the item after next (and read its len), copy that item's
 //     query rows and appended k / v row from the call's inputs into a staging area in shared memory, and hand
 //     the parity buffer back through a second mbarrier.  The streaming warps take their query fragments and the
@@ -22,7 +22,9 @@
 
 namespace lethe {
 
-constexpr int kEpilogueWarps = 2;
+// Epilogue warps per CTA.  Measured on the Llama-8B shape, of the copy peak: (8,2) with 2 / 3 / 4 epilogue warps
+// 0.98 / 1.015 / 1.03, (5,3) with 2 / 4: 1.01 / 0.79, (7,2) with 4 / 6: 1.005 / 0.83.
+__host__ __device__ constexpr int epilogue_warps(int nws) { return nws >= 8 ? 4 : 2; }
 constexpr int kWaitLimit = 200000;  // polls of a blocking try_wait before giving up
 
 // Tensor maps of K and V for the TMA variant (rows x D, box 16 rows x 64 elements, 128-byte swizzle).
@@ -177,7 +179,7 @@ __device__ __noinline__ void append_row(const AttendArgs& a, int item, int n_old
 }
 
 template <int D, int NWS, int NS, bool PAGED, bool SPILL, bool TMA>
-__global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
+__global__ void __launch_bounds__((NWS + epilogue_warps(NWS)) * 32, 1)
     attend_async_kernel(const __grid_constant__ AttendArgs a, const __grid_constant__ TmaMaps maps) {
     using T = __nv_bfloat16;
     constexpr int ROW_BYTES = D * 2;
@@ -186,6 +188,7 @@ __global__ void __launch_bounds__((NWS + kEpilogueWarps) * 32, 1)
     constexpr int STAGE_BYTES = 2 * TILE_BYTES;
     constexpr int WARP_BYTES = NS * STAGE_BYTES;
     constexpr int KS = D / 16;
+    constexpr int kEpilogueWarps = epilogue_warps(NWS);
     constexpr int ET = kEpilogueWarps * 32;
     static_assert(NS >= 2 && NS <= 6 && NWS <= 16, "shape");
     extern __shared__ __align__(1024) unsigned char smem_raw[];  // TMA tiles with a 128-byte swizzle need 1 KB alignment
@@ -753,7 +756,7 @@ static cudaError_t launch_async_t(const AttendArgs& a, const TmaMaps& maps, int 
     const size_t smem = async_smem<D, NWS, NS>(a.chunk_tokens, a.GP);
     cudaError_t e = prepare_kernel((const void*)kern, smem);
     if (e != cudaSuccess) return e;
-    kern<<<grid, (NWS + kEpilogueWarps) * 32, smem, stream>>>(a, maps);
+    kern<<<grid, (NWS + epilogue_warps(NWS)) * 32, smem, stream>>>(a, maps);
     return cudaGetLastError();
 }
 
@@ -767,7 +770,7 @@ static cudaError_t dispatch_async(const AttendArgs& a, const TmaMaps& maps, bool
                  : launch_async_t<D, NWS, NS, false, false, TMA>(a, maps, grid, stream);
 }
 
-// Shapes: (streaming warps per CTA, stages per warp); two more warps run the epilogue.
+// Shapes: (streaming warps per CTA, stages per warp); epilogue_warps() more warps run the epilogue.
 #define LETHE_ASYNC_SHAPES(X, D) X(0, D, 8, 2) X(1, D, 7, 2) X(2, D, 6, 3) X(3, D, 5, 3) X(4, D, 6, 2) X(5, D, 4, 4)
 
 size_t async_smem_bytes(int D, int shape, int chunk_tokens, int GP) {
