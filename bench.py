@@ -35,7 +35,7 @@ UNIT = "token-heads/s"
 BYTES_PER_TOKEN_HEAD = 520          # K row 256 B + V row 256 B + relevance read 4 B + write 4 B (D=128, bf16)
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) per token-head of the default attend kernel, from the ncu capture summarised in
-# profiles/attend_async_w5s3_llama8b.md (1.026 GB per launch of 1 970 008 token-heads; traffic grows in
+# profiles/attend_async_w8s2_llama8b.md (1.026 GB per launch of 1 969 552 token-heads; traffic grows in
 # proportion to the token-heads of a launch, so it is scaled to the launch bench.py times).
 NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = 521.0
 
