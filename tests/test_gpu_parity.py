@@ -506,7 +506,11 @@ def test_host_entry_point_matches_the_device_one(ctx, L, B, Hkv, pinned):
         lse_a = torch.empty((L, B, Hq), dtype=torch.float32, device=dev)
         ctx.decode_attend(ga, 0, L, q.to(dev), kn.to(dev), vn.to(dev), tp.to(dev), scale, 0.9, out_a, lse_a)
         qh, kh, vh, th = pin(q), pin(kn), pin(vn), pin(tp)
-        out_b = pin(torch.empty_like(q))
+        if pinned and step == 1:   # results into the middle of a larger page-locked allocation
+            big = torch.empty((3 * q.numel(),), dtype=torch.bfloat16).pin_memory()
+            out_b = big[q.numel():2 * q.numel()].view(q.shape)
+        else:
+            out_b = pin(torch.empty_like(q))
         lse_b = pin(torch.empty((L, B, Hq), dtype=torch.float32))
         ctx.decode_attend_host(gb, 0, L, qh, kh, vh, th, scale, 0.9, out_b, lse_b)
         assert ctx.poll_status()[0] == 0                       # synchronises the stream: host results are valid
