@@ -368,7 +368,8 @@ __global__ void __launch_bounds__(kPruneThreads, 2) rasr_prune_kernel(CacheView 
     const int keep_n = sweep_keep(sh, key_at, n, cand_lo, cand_hi, cand_lo, cand_hi, take > 0, T, need_eq, src_list, kout, max_k);
     bool bad = false;
     move_rows(c, item, keep_n, src_list, bad);
-    if (bad && tid == 0) record_error(status, LETHE_ERR_PAGE, (int)item);
+    // any thread may have met the bad page id (each carries its own row slots): reduce over the CTA
+    if (__syncthreads_or(bad) && tid == 0) record_error(status, LETHE_ERR_PAGE, (int)item);
     if (tid == 0) c.len[item] = keep_n;
 }
 
@@ -442,7 +443,7 @@ __global__ void __launch_bounds__(kPruneThreads, 2) segment_prune_kernel(CacheVi
                                   kout, max_k);
     bool bad = false;
     move_rows(c, item, keep_n, src_list, bad);
-    if (bad && tid == 0) record_error(status, LETHE_ERR_PAGE, (int)item);
+    if (__syncthreads_or(bad) && tid == 0) record_error(status, LETHE_ERR_PAGE, (int)item);
     if (tid == 0) {
         c.len[item] = keep_n;
         l_evict[item] = max(le, breakpoint + recent);
@@ -556,7 +557,7 @@ __global__ void __launch_bounds__(kPruneThreads, 2) collapsed_move_kernel(CacheV
     if (keep_n < 0) return;
     bool bad = false;
     move_rows(c, item, keep_n, lists + group * c.cap_tokens, bad);
-    if (bad && threadIdx.x == 0) record_error(status, LETHE_ERR_PAGE, (int)item);
+    if (__syncthreads_or(bad) && threadIdx.x == 0) record_error(status, LETHE_ERR_PAGE, (int)item);
     if (threadIdx.x == 0) c.len[item] = keep_n;
 }
 

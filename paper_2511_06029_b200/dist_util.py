@@ -3,9 +3,51 @@ the data path.  The only exchanges are the barrier around the timed region and t
 (elapsed time, units processed) into the whole-job figure: max of the times, sum of the units."""
 from __future__ import annotations
 
+import os
+import socket
+import subprocess
 from typing import Sequence, Tuple
 
 import torch
+
+
+def spawn_ranks(cmd: Sequence[str], n: int, timeout_s: float = 3600.0) -> int:
+    """Start `cmd` n times as the ranks of one job on this node (what a launcher would do): RANK / LOCAL_RANK =
+    0..n-1, WORLD_SIZE = n, rendezvous on 127.0.0.1 at a free port.  The ranks inherit stdout / stderr, so rank
+    0's result line reaches the caller's stdout.  Returns 0 if every rank exited 0; otherwise the remaining ranks
+    are stopped (by their own pids) and the first non-zero exit code is returned."""
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), LOCAL_WORLD_SIZE=str(n),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen(list(cmd), env=env))
+    import time
+    deadline = time.monotonic() + timeout_s
+    rc = 0
+    pending = set(range(n))
+    while pending and rc == 0:
+        for r in sorted(pending):
+            code = procs[r].poll()
+            if code is not None:
+                pending.discard(r)
+                if code != 0:
+                    rc = code
+        if time.monotonic() > deadline:
+            rc = 124
+        if pending and rc == 0:
+            time.sleep(0.05)
+    for r in pending:                                    # a rank failed or the job ran out of time: stop the others
+        procs[r].terminate()
+    for r in pending:
+        try:
+            procs[r].wait(timeout=10)
+        except subprocess.TimeoutExpired:
+            procs[r].kill()
+    return rc
 
 
 def rank_batch_ids(rank: int, per_rank_batch: int) -> torch.Tensor:

@@ -193,10 +193,12 @@ def step_inputs(w: Workload, step: int, device="cpu", batch_ids: Optional[torch.
     return {"q": q.to(w.dtype), "k_new": kn.to(w.dtype), "v_new": vn.to(w.dtype), "token_pos": token_pos}
 
 
-def ragged_lengths(w: Workload, lo: int = 1024, hi: int = 32768) -> torch.Tensor:
-    """Per-sequence KV length, uniform integer in [lo, hi] (ragged-batch workload)."""
+def ragged_lengths(w: Workload, lo: int = 1024, hi: int = 32768, n: Optional[int] = None) -> torch.Tensor:
+    """Per-sequence KV length, uniform integer in [lo, hi] (ragged-batch workload), for the global sequences
+    0..n-1 (default: the workload's batch).  A longer draw starts with the shorter one, so ranks that hold
+    different slices of one job agree on every sequence's length."""
     g = _gen(w.seed * 48271 + 9, "cpu")
-    return torch.randint(lo, hi + 1, (w.batch,), generator=g, dtype=torch.int64)
+    return torch.randint(lo, hi + 1, (n or w.batch,), generator=g, dtype=torch.int64)
 
 
 def to_paged(state: dict, page_tokens: int, seed: int, spare_pages: int = 0):

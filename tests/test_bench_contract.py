@@ -28,17 +28,30 @@ def test_reference_arm_prints_the_contract_line():
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1 and "sample" in d["cpu_baseline"]
     assert d["e2e"] == {"value": d["value"], "unit": d["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     assert d["vs_baseline"] is None and "workload" in d["config"]
+    sys.path.insert(0, ROOT)
+    import bench
+    assert set(d["config"]) == set(bench.CONFIG_KEYS)    # the same keys as the GPU arm prints (None where not applicable)
 
 
 @pytest.mark.gpu
 def test_gpu_arm_prints_the_contract_line():
-    d = _run(["--steps", "160", "--warmup", "3", "--prep-rounds", "1", "--no-cpu-baseline", "--no-per-layer"], timeout=900)
-    assert BASE_KEYS <= set(d) and d["n_gpus"] == 1 and d["steps"] == 160 and d["scaling"] == "weak"
+    d = _run(["--steps", "8", "--warmup", "3", "--prep-rounds", "1", "--no-cpu-baseline", "--no-per-layer"], timeout=900)
+    assert BASE_KEYS <= set(d) and d["n_gpus"] == 1 and d["steps"] == 8 and d["scaling"] == "weak"
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
     assert 0.3 < r["frac"] < 1.2 and r["traffic"] > 0
-    assert d["gpu_launches"] >= 160 and d["value"] > 1e9
+    assert d["gpu_launches"] >= 8 and d["value"] > 1e9
     e = d["e2e"]
     assert e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0 and 0 < e["value"] < d["value"]
     assert {"sm_mhz", "sm_max_mhz", "reasons"} <= set(d["clocks"])
-    assert d["config"]["prune_rounds_timed"] >= 1 and "workload" in d["config"]
+    # the prune round is timed on every run, however few steps the timed loop has
+    c = d["config"]
+    assert c["prune_rounds_timed"] >= 3 and c["prune_round_ms"] > 0 and "workload" in c
+    pr = c["prune_round"]
+    assert abs(pr["prune_round_us"] - (pr["estimate_sparsity_us"] + pr["alloc_budgets_us"] + pr["rasr_prune_us"])) < 1e-6
+    assert abs(pr["prune_amortised_us_per_step"] * pr["prune_interval"] - pr["prune_round_us"]) < 1e-6
+    assert pr["rows_moved"] > 0 and pr["token_heads_after"] < pr["token_heads_before"]
+    wp = r["with_amortised_prune"]
+    assert wp["ms_per_step"] > c["attend_ms_per_step"] and 0.3 < wp["frac"] <= r["frac"]
+    import bench
+    assert set(c) == set(bench.CONFIG_KEYS)

@@ -1,7 +1,10 @@
 """World-size-2 checks of the benchmark's multi-rank plumbing on CPU (gloo): sequence sharding is disjoint and
 complete, the job figure is sum(units) / max(time), and ranks see different synthetic sequences."""
+import json
 import os
 import socket
+import subprocess
+import sys
 
 import torch
 import torch.distributed as dist
@@ -84,3 +87,38 @@ def test_two_rank_head_sharded_prune_round():
     mp.spawn(_tp_worker, args=(2, _free_port(), ret), nprocs=2, join=True)
     for rank in range(2):
         assert all(ret[rank]), ret[rank]
+
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_bench_starts_its_own_ranks():
+    """`bench.py --gpus 2` without a launcher around it starts two ranks itself: here the launcher path alone
+    (gloo, CPU tensors, the job reduction only).  The line reports the ranks that actually joined, the slowest
+    rank's time and the sum of the units; the ranks hold disjoint global sequences."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_PORT")}
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--launcher-selftest"],
+                       capture_output=True, text=True, timeout=300, cwd=ROOT, env=env)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [l for l in p.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, p.stdout                     # rank 0 alone prints
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["max_ms"] == 15.0 and d["units"] == 300.0 and d["value"] == 20000.0
+    assert d["id_sum"] == sum(range(8))                  # sequences 0..3 on rank 0, 4..7 on rank 1
+
+
+def test_bench_refuses_more_gpus_than_visible():
+    """A plain `python bench.py --gpus N` on a machine with fewer than N devices must fail, not print n_gpus = N."""
+    import torch
+    n = (torch.cuda.device_count() if torch.cuda.is_available() else 0) + 1
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_PORT")}
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", str(max(n, 2)), "--steps", "1"],
+                       capture_output=True, text=True, timeout=300, cwd=ROOT, env=env)
+    assert p.returncode != 0 and "visible" in (p.stderr + p.stdout)
+    assert not [l for l in p.stdout.splitlines() if l.startswith("{")]
+
+
+def test_spawn_ranks_reports_a_failing_rank():
+    code = "import os, sys, time; r = int(os.environ['RANK']); time.sleep(0.2 * r); sys.exit(3 if r == 1 else 0)"
+    assert dist_util.spawn_ranks([sys.executable, "-c", code], 3) == 3
+    assert dist_util.spawn_ranks([sys.executable, "-c", "import os; assert os.environ['WORLD_SIZE'] == '2'"], 2) == 0
