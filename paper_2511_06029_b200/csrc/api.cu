@@ -101,9 +101,6 @@ struct lethe_ctx {
     unsigned long long tma_rows;
     int tma_d;
     void* tma_encode;  // cuTensorMapEncodeTiled, resolved on first use
-#ifdef LETHE_TIMELINE
-    unsigned long long* timeline;
-#endif
     char err[256];
 };
 
@@ -271,14 +268,6 @@ lethe_status lethe_poll_status(lethe_ctx* ctx, void* stream, int32_t* info) {
     return (lethe_status)h[0];
 }
 
-#ifdef LETHE_TIMELINE
-// Debug builds only: per-CTA timestamps of the next attend launches go to `buf` (8 x uint64 per CTA).
-lethe_status lethe_debug_set_timeline(lethe_ctx* ctx, unsigned long long* buf) {
-    if (!ctx) return LETHE_ERR_INVALID_ARG;
-    ctx->timeline = buf;
-    return LETHE_OK;
-}
-#endif
 
 // cuTensorMapEncodeTiled through the runtime (no link-time dependency on the driver library); resolved once.
 static bool resolve_tma_encode(lethe_ctx* ctx) {
@@ -348,9 +337,6 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
     a.layer_begin = layer_begin;
     a.n_items = (layer_end - layer_begin) * c->batch * c->n_kv_heads;
     a.gamma = gamma;
-#ifdef LETHE_TIMELINE
-    a.timeline = ctx->timeline;
-#endif
     for (int l = 0; l < c->n_layers; ++l) a.scale_log2[l] = scale[l] * 1.4426950408889634f;
 
     const bool paged = c->layout == LETHE_PAGED;

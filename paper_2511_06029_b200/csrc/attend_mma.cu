@@ -34,7 +34,6 @@ __global__ void __launch_bounds__(NW * 32) attend_mma_kernel(const __grid_consta
     EpilogueSmem& es = *reinterpret_cast<EpilogueSmem*>(cta_o + kMaxGroup * D);
     float* lg = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(&es) + sizeof(EpilogueSmem));
 
-    TL_MARK(a, 0);
     // Programmatic dependent launch: when the launch carries the attribute this CTA may have been scheduled while
     // the previous kernel of the stream was still draining; everything it reads may come from that kernel, so it
     // waits here for it to complete (a no-op for ordinary launches).
@@ -143,7 +142,6 @@ __global__ void __launch_bounds__(NW * 32) attend_mma_kernel(const __grid_consta
     const int k_row = (lane & 7) + ((lane >> 3) & 1) * 8, k_chunk = lane >> 4;
     const int v_row = (lane & 7) + ((lane >> 4) & 1) * 8, v_chunk = (lane >> 3) & 1;
 
-    TL_MARK(a, 1);
     for (int it = 0; it < my_count; ++it) {
         cp_async_wait<NSTAGE - 2>();
         __syncwarp();
@@ -207,7 +205,6 @@ __global__ void __launch_bounds__(NW * 32) attend_mma_kernel(const __grid_consta
         if (nxt < my_count) issue(my_first + nxt * NW, nxt % NSTAGE);
         cp_async_commit();
     }
-    TL_MARK(a, 2);
     // the streaming part is over: let the next kernel of the stream be scheduled onto the SMs as they free up
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     float rel_old[kRelPrefetch];

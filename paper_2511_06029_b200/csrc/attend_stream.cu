@@ -208,7 +208,6 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
 
     while (cur.valid) {
         const float sl2 = a.scale_log2[cur.l];
-        TL_MARK_AT(a, cur.item - a.layer_begin * a.B * a.Hkv, 0);
         // ---- top-up: whatever of the first NS-1 groups the previous tail did not prefetch
         bool topped = false;
 #pragma unroll
@@ -312,7 +311,6 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
             }
         }
         vp = (vp + cur.count) % NS;
-        TL_MARK_AT(a, cur.item - a.layer_begin * a.B * a.Hkv, 1);
 
         // ---- epilogue of the item: merge warps, write out / lse, Eq. 5 on rel[0..n)
         float rel_old[kRelPrefetch];
@@ -348,7 +346,6 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
         if (tid == 0 && !drew_fail)  // ticket of the item after next; its latency hides behind the barrier wait
             t_new = (int)atomicAdd(&sched[0], 1u);
         __syncthreads();  // B1: every warp's partials are in shared memory
-        TL_MARK_AT(a, cur.item - a.layer_begin * a.B * a.Hkv, 2);
         if (tid < kMaxGroup) {
             const int h = tid;
             float m = -INFINITY;
@@ -367,7 +364,6 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
                     l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
         }
         __syncthreads();  // B2
-        TL_MARK_AT(a, cur.item - a.layer_begin * a.B * a.Hkv, 3);
         {
             T* out = (T*)a.out + ((size_t)(cur.li * a.B + cur.b) * a.Hq + cur.hkv * G) * D;
             for (int idx = tid; idx < G * D; idx += NT) {
@@ -439,7 +435,6 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
             es.flags[2] = t_new;
         }
         __syncthreads();  // B3: lg / wo / wstat may be reused; the next ticket is visible
-        TL_MARK_AT(a, cur.item - a.layer_begin * a.B * a.Hkv, 4);
 
         // ---- rotate: next becomes current
         if (nxt.valid && !nxt_ready) {

@@ -48,45 +48,11 @@ struct AttendArgs {
     int splits;                // CTAs per item (cluster size)
     int chunk_tokens;          // logit-buffer capacity of one CTA, in tokens
     float gamma;
-#ifdef LETHE_TIMELINE
-    unsigned long long* timeline;  // debug builds only: 8 timestamps per CTA
-#endif
     float scale_log2[kMaxLayers];  // scale[l] * log2(e) (times the key scale for a quantised cache), by absolute layer
     float k_scale[kMaxLayers];     // quantised caches: a stored key byte x means k_scale[l] * x (else unused)
     float v_scale[kMaxLayers];     // the same for values
 };
 
-#ifdef LETHE_TIMELINE
-__device__ __forceinline__ void tl_mark(const AttendArgs& a, int slot) {
-    if (a.timeline && threadIdx.x == 0) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-        a.timeline[(size_t)blockIdx.x * 8 + slot] = t;
-        if (slot == 0) {
-            unsigned sm;
-            asm volatile("mov.u32 %0, %smid;" : "=r"(sm));
-            a.timeline[(size_t)blockIdx.x * 8 + 7] = sm;
-        }
-    }
-}
-__device__ __forceinline__ void tl_mark_at(const AttendArgs& a, int row, int slot) {
-    if (a.timeline && threadIdx.x == 0) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-        a.timeline[(size_t)row * 8 + slot] = t;
-        if (slot == 0) {
-            unsigned sm;
-            asm volatile("mov.u32 %0, %smid;" : "=r"(sm));
-            a.timeline[(size_t)row * 8 + 7] = sm;
-        }
-    }
-}
-#define TL_MARK(a, slot) tl_mark(a, slot)
-#define TL_MARK_AT(a, row, slot) tl_mark_at(a, row, slot)
-#else
-#define TL_MARK(a, slot)
-#define TL_MARK_AT(a, row, slot)
-#endif
 
 // Cache state as the prune-round kernels see it.
 struct CacheView {
@@ -220,7 +186,6 @@ __device__ void combine_and_finish(const AttendArgs& a, const ItemCoord& ic, Epi
     const int G = a.G;
     constexpr int NT = NW * 32;
     __syncthreads();
-    TL_MARK(a, 3);
     if (tid < kMaxGroup) {
         const int h = tid;
         float m = -INFINITY;
@@ -287,7 +252,6 @@ __device__ void combine_and_finish(const AttendArgs& a, const ItemCoord& ic, Epi
         }
     }
 
-    TL_MARK(a, 4);
     // Eq. 5: rel[j] = gamma * rel[j] + sum over the group's heads of p_hj, with the global (m, 1/l).
     float* rel = a.rel + (size_t)ic.item * a.cap_tokens;
     const int GP = a.GP;
@@ -344,10 +308,8 @@ __device__ void combine_and_finish(const AttendArgs& a, const ItemCoord& ic, Epi
             if (j < hi_tok) rel[j] = fmaf(a.gamma, old[u], mass_from(s[u]));
         }
     }
-    TL_MARK(a, 5);
     if (S > 1) cg::this_cluster().sync();  // peers may still be reading this CTA's shared memory
     if (append_slot >= 0 && ic.rank == 0 && tid == 0) a.len[ic.item] = n;
-    TL_MARK(a, 6);
 }
 
 /*

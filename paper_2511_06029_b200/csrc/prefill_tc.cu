@@ -53,21 +53,6 @@ __host__ __device__ constexpr int tc_threads() { return (kTcSoftmaxWarps + 1 + (
 
 enum { kModeStats = 0, kModeColsum = 1 };
 
-#ifdef LETHE_TC_TIMELINE
-// Debug build only: nanosecond stamps of CTA 0 of the COLSUM pass, [role][step][4].
-__device__ unsigned long long g_tc_timeline[3 * 64 * 4];
-__device__ __forceinline__ unsigned long long tc_now() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-#define TC_MARK(role, step, k)                                                                                  \
-    do {                                                                                                        \
-        if (MODE == kModeColsum && blockIdx.x == 0 && (step) < 64) g_tc_timeline[((role) * 64 + (step)) * 4 + (k)] = tc_now(); \
-    } while (0)
-#else
-#define TC_MARK(role, step, k) do { } while (0)
-#endif
 
 // Tensor maps of the TMA path: K as [items][capacity][D] with a 128-row box, the prompt's queries as
 // [L B][P][Hq][D] with a (qpb queries x G heads) box; 64-element (128-byte) inner boxes, 128-byte swizzle.
@@ -415,12 +400,9 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
                 tc_range<MODE>(ab, P, qpb, t0, t1);
                 for (int t = t0; t < t1; ++t, ++step) {
                     const int s = step % kTcStages, buf = step & 1;
-                    TC_MARK(1, step, 0);
                     if (t == t0 && !tc_wait(&sh.a_full[ab % kTcABuffers], (unsigned)((ab / kTcABuffers) & 1), abort_flag)) { alive = false; break; }
                     if (!tc_wait(&sh.b_full[s], (unsigned)((step / kTcStages) & 1), abort_flag)) { alive = false; break; }
-                    TC_MARK(1, step, 1);
                     if (step >= 2 && !tc_wait(&sh.t_empty[buf], (unsigned)(((step >> 1) - 1) & 1), abort_flag)) { alive = false; break; }
-                    TC_MARK(1, step, 2);
                     tc_fence_after();
                     const uint32_t at = a_tile0 + (ab % kTcABuffers) * TILE_BYTES, bt = b_tile0 + s * TILE_BYTES;
 #pragma unroll
@@ -432,7 +414,6 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
                     tc_commit(&sh.b_empty[s]);
                     if (t == t1 - 1) tc_commit(&sh.a_empty[ab % kTcABuffers]);
                     tc_commit(&sh.t_full[buf]);
-                    TC_MARK(1, step, 3);
                 }
             }
         }
@@ -482,9 +463,7 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
                     }
                     __syncwarp();
                 }
-                if (tid == 0) TC_MARK(0, step, 0);
                 if (!tc_wait(&sh.t_full[buf], (unsigned)((step >> 1) & 1), abort_flag)) { alive = false; break; }
-                if (tid == 0) TC_MARK(0, step, 1);
                 tc_fence_after();
 #pragma unroll
                 for (int ch = 0; ch < 2; ++ch) {
@@ -494,7 +473,6 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
                     if (ch == 1) {  // the tile is in registers: the MMA may overwrite this buffer
                         tc_fence_before();
                         tc_mbar_arrive(&sh.t_empty[buf]);
-                        if (tid == 0) TC_MARK(0, step, 2);
                     }
                     const int cbase = half * 64 + ch * 32;  // first tile column of this chunk
                     if (MODE == kModeStats) {
@@ -563,7 +541,6 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
                         }
                     }
                 }
-                if (tid == 0) TC_MARK(0, step, 3);
             }
             if (alive && row_ok) {
                 if (MODE == kModeStats) a.stats[half * half_stride + ((size_t)item * P + qi) * HP + r % G] = make_float2(m, lsum);
@@ -634,8 +611,3 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, int items, int L, int D, voi
 
 }  // namespace lethe
 
-#ifdef LETHE_TC_TIMELINE
-extern "C" int lethe_debug_tc_timeline(unsigned long long* host_dst) {
-    return (int)cudaMemcpyFromSymbol(host_dst, lethe::g_tc_timeline, sizeof(unsigned long long) * 3 * 64 * 4);
-}
-#endif
