@@ -60,7 +60,7 @@ typedef enum {
     LETHE_ERR_CAPACITY = 2,    /* device-side: append on an item with len == capacity */
     LETHE_ERR_BUDGET = 3,      /* budget below the protected (sink + recent) count, or total < L * k_min */
     LETHE_ERR_CUDA = 4,        /* a CUDA runtime call failed; see lethe_last_error */
-    LETHE_ERR_TIMEOUT = 5,     /* reserved: a bounded device-side wait ran out */
+    LETHE_ERR_TIMEOUT = 5,     /* device-side: a bounded wait inside a kernel ran out (see lethe_set_wait_limit) */
     LETHE_ERR_UNSUPPORTED = 6, /* valid request outside what the kernels cover */
     LETHE_ERR_PAGE = 7,        /* device-side: page id outside [0, n_pages) */
     LETHE_ERR_TOO_LARGE = 8    /* lethe_rasr_prune_static: the cache exceeds LETHE_STATIC_PRUNE_MAX_ENTRIES */
@@ -100,7 +100,11 @@ typedef struct {
  * scored before they are quantised). */
 
 /* Create a context on CUDA device `device`.  scratch_bytes_hint (0 = default) sizes the
- * device scratch the calls may use; it grows on demand (growth synchronises the device).
+ * device scratch the calls may use; it grows on demand.  Growth synchronises the device, frees the
+ * old buffer and allocates a larger one: a CUDA graph captured from earlier calls may still name the
+ * old buffer and must be captured again, and a call that would have to grow scratch while its stream
+ * is being captured is refused with LETHE_ERR_UNSUPPORTED (size the scratch with scratch_bytes_hint,
+ * or make the same call once before capturing).
  * Returns LETHE_ERR_CUDA if no usable sm_100 device / runtime is present. */
 lethe_status lethe_create(lethe_ctx **ctx, int device, size_t scratch_bytes_hint);
 void lethe_destroy(lethe_ctx *ctx);
@@ -136,6 +140,20 @@ lethe_status lethe_poll_status(lethe_ctx *ctx, void *stream, int32_t *info);
  * A context serialises its calls: issue them to one stream at a time (the status word and the persistent
  * kernel's work queue are per context). */
 lethe_status lethe_set_tuning(lethe_ctx *ctx, int variant, int splits);
+
+/*
+ * Failure detection inside the kernels (the paper has no counterpart).  The warp-specialised kernels — the
+ * persistent decode kernel with the asynchronous epilogue and the tensor-memory kernels of lethe_prefill_seed —
+ * hand work between their warps through mbarriers.  Every such wait is bounded: after `polls` looks at the
+ * barrier the waiting thread gives up, the CTA's other roles leave their loops, copies and MMAs still in flight
+ * are waited for (with the built-in limit), tensor memory is freed, the work queue is left ready for the next
+ * launch, and LETHE_ERR_TIMEOUT is recorded with the CTA (decode) or item (prefill) that gave up.  The launch
+ * always returns; the cache contents it was working on are then unspecified.  polls = 0 restores the defaults
+ * (hundreds of thousands of polls: seconds, far beyond any legitimate wait); a small value makes the waits run
+ * out on purpose, which is how the give-up path is tested without hanging anything (the first poll never
+ * blocks, so polls = 1 gives up unless the barrier has already completed).
+ */
+lethe_status lethe_set_wait_limit(lethe_ctx *ctx, int32_t polls);
 
 /*
  * One decode step for layers [layer_begin, layer_end)  (Sec. 4.1; Eq. 3; Eq. 5).
@@ -298,8 +316,12 @@ lethe_status lethe_prefill_seed(lethe_ctx *ctx, const lethe_cache *cache, const 
  *     LETHE_STATIC_PRUNE_MAX_ENTRIES is refused with LETHE_ERR_TOO_LARGE and nothing is enqueued;
  *   - it calls no cudaMalloc / cudaFree and no allocating library routine; it enqueues one 8-byte memset, one
  *     kernel and (with status_out) one 8-byte copy on `stream`;
- *   - the first call on a device looks up the scratch's device address (cudaGetSymbolAddress).  Make that
- *     first call before any stream capture begins;
+ *   - the first call on a device looks up the scratch's device address (cudaGetSymbolAddress).  With CUDA's lazy
+ *     module loading that first use is also when the runtime places this library's device image, the 16 MiB
+ *     array included, on the device: a one-time load that takes device memory from the driver and can fail
+ *     (LETHE_ERR_CUDA) if none is left.  So make the first call at start-up — on a small dummy cache if need be —
+ *     before the caller's own pool claims the rest of the device, and before any stream capture begins; from the
+ *     second call on, a call leaves the device's free memory exactly as it found it;
  *   - all calls share the one array, which still holds whatever the previous call left in it (the status
  *     block is cleared at the start of each call; the lists are always written before they are read).  Two
  *     calls whose kernels could overlap on the GPU — different streams without an ordering event, or several

@@ -21,7 +21,7 @@ F32, BF16, FP8_E4M3, FP8_E5M2 = 0, 1, 2, 3
 CONTIG, PAGED = 0, 1
 VARIANT_AUTO, VARIANT_SIMT, VARIANT_MMA4, VARIANT_MMA8 = 0, 1, 2, 3
 
-EXPORTS = ["lethe_create", "lethe_destroy", "lethe_last_error", "lethe_poll_status", "lethe_set_tuning",
+EXPORTS = ["lethe_create", "lethe_destroy", "lethe_last_error", "lethe_poll_status", "lethe_set_tuning", "lethe_set_wait_limit",
            "lethe_decode_attend", "lethe_decode_attend_host", "lethe_estimate_sparsity", "lethe_alloc_budgets",
            "lethe_rasr_prune", "lethe_rasr_prune_static", "lethe_segment_prune", "lethe_prefill_seed",
            "lethe_collapsed_prune"]
@@ -67,6 +67,8 @@ def load() -> ctypes.CDLL:
     lib.lethe_poll_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
     lib.lethe_set_tuning.restype = ctypes.c_int
     lib.lethe_set_tuning.argtypes = [vp, ctypes.c_int, ctypes.c_int]
+    lib.lethe_set_wait_limit.restype = ctypes.c_int
+    lib.lethe_set_wait_limit.argtypes = [vp, i32]
     attend_args = [vp, cp, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, ctypes.POINTER(ctypes.c_float),
                    ctypes.c_float, vp, vp, vp]
     lib.lethe_decode_attend.restype = ctypes.c_int
@@ -204,6 +206,9 @@ class Context:
 
     def set_tuning(self, variant: int = 0, splits: int = 0):
         self._check(self.lib.lethe_set_tuning(self.h, variant, splits))
+
+    def set_wait_limit(self, polls: int = 0):
+        self._check(self.lib.lethe_set_wait_limit(self.h, polls))
 
     def poll_status(self):
         """Synchronise the current stream and return (status, item) of the first device-side error since last poll."""

@@ -93,6 +93,7 @@ struct lethe_ctx {
     cudaEvent_t ev_start, ev_up[8], ev_done[8], ev_down;
     bool host_pipeline_ready;
     int variant, splits;
+    int wait_limit;  // poll limit of the kernels' bounded waits (0 = their defaults); lethe_set_wait_limit
     int prefill_engine;  // 0 = tcgen05 kernels (TMA producers when the cache is contiguous), 1 = mma.sync kernels, 2 = tcgen05 with cp.async producers
     // TMA variant: tensor maps of the last cache seen (rebuilt when k, v, the row count or D change)
     alignas(64) unsigned char tma_maps[512];
@@ -127,8 +128,15 @@ struct DeviceGuard {
     }
 };
 
-lethe_status ensure(lethe_ctx* ctx, void** buf, size_t* have, size_t need, const char* what) {
+// Grow a context-owned buffer.  Growth synchronises the device and frees the old buffer, so it must not happen
+// while `stream` is being captured (the capture would be invalidated, and a graph captured earlier may still name
+// the old buffer): that case is refused.
+lethe_status ensure(lethe_ctx* ctx, void** buf, size_t* have, size_t need, const char* what, void* stream = nullptr) {
     if (need <= *have) return LETHE_OK;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing((cudaStream_t)stream, &cap) != cudaSuccess) cudaGetLastError();
+    else if (cap != cudaStreamCaptureStatusNone)
+        return fail(ctx, LETHE_ERR_UNSUPPORTED, "%s would have to grow while the stream is being captured", what);
     cudaError_t e = cudaDeviceSynchronize();  // the old buffer may still be in use
     if (e != cudaSuccess) return cuda_fail(ctx, e, what);
     if (*buf) cudaFree(*buf);
@@ -297,9 +305,11 @@ lethe_status lethe_set_tuning(lethe_ctx* ctx, int variant, int splits) {
     return LETHE_OK;
 }
 
-lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer_begin, int layer_end, const void* q,
-                                 const void* k_new, const void* v_new, const int32_t* token_pos, const float* scale,
-                                 float gamma, void* out, float* lse, void* stream) {
+// Everything about a decode call that the host can check, for the device and the host entry points alike (the
+// host entry point checks before it sizes staging or enqueues a copy).  Alignment is a matter of device pointers.
+static lethe_status check_attend_args(lethe_ctx* ctx, const lethe_cache* c, int layer_begin, int layer_end, const void* q,
+                                      const void* k_new, const void* v_new, const int32_t* token_pos, const float* scale,
+                                      float gamma, const void* out, bool device_pointers) {
     lethe_status st = check_cache(ctx, c);
     if (st != LETHE_OK) return st;
     if (!q || !out || !scale) return fail(ctx, LETHE_ERR_INVALID_ARG, "q, out and scale are required");
@@ -309,12 +319,30 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
     if (k_new && !token_pos) return fail(ctx, LETHE_ERR_INVALID_ARG, "token_pos is required when appending");
     if (!(gamma > 0.f && gamma <= 1.f)) return fail(ctx, LETHE_ERR_INVALID_ARG, "gamma must be in (0, 1]");
     if (c->n_layers > kMaxLayers) return fail(ctx, LETHE_ERR_UNSUPPORTED, "more than 128 layers");
-    const int G = c->n_q_heads / c->n_kv_heads;
-    if (G > kMaxGroup) return fail(ctx, LETHE_ERR_UNSUPPORTED, "more than 8 query heads per KV head");
-    if (((uintptr_t)q | (uintptr_t)out | (uintptr_t)k_new | (uintptr_t)v_new) & 15)
+    if (c->n_q_heads / c->n_kv_heads > kMaxGroup) return fail(ctx, LETHE_ERR_UNSUPPORTED, "more than 8 query heads per KV head");
+    if (device_pointers && (((uintptr_t)q | (uintptr_t)out | (uintptr_t)k_new | (uintptr_t)v_new) & 15))
         return fail(ctx, LETHE_ERR_INVALID_ARG, "q, k_new, v_new, out must be 16-byte aligned");
     for (int l = layer_begin; l < layer_end; ++l)
         if (!(scale[l] == scale[l]) || fabsf(scale[l]) > 1e30f) return fail(ctx, LETHE_ERR_INVALID_ARG, "scale must be finite");
+    const bool bytes = c->dtype == LETHE_FP8_E4M3 || c->dtype == LETHE_FP8_E5M2;
+    if (bytes && c->layout == LETHE_PAGED && c->page_tokens != kGroupTokens)
+        return fail(ctx, LETHE_ERR_UNSUPPORTED, "quantised caches need 16-token pages");
+    return LETHE_OK;
+}
+
+lethe_status lethe_set_wait_limit(lethe_ctx* ctx, int32_t polls) {
+    if (!ctx) return LETHE_ERR_INVALID_ARG;
+    if (polls < 0) return fail(ctx, LETHE_ERR_INVALID_ARG, "the poll limit must be >= 0 (0 = default)");
+    ctx->wait_limit = polls;
+    return LETHE_OK;
+}
+
+lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer_begin, int layer_end, const void* q,
+                                 const void* k_new, const void* v_new, const int32_t* token_pos, const float* scale,
+                                 float gamma, void* out, float* lse, void* stream) {
+    lethe_status st = check_attend_args(ctx, c, layer_begin, layer_end, q, k_new, v_new, token_pos, scale, gamma, out, true);
+    if (st != LETHE_OK) return st;
+    const int G = c->n_q_heads / c->n_kv_heads;
 
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, LETHE_ERR_CUDA, "cannot select the context's device");
@@ -337,6 +365,7 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
     a.layer_begin = layer_begin;
     a.n_items = (layer_end - layer_begin) * c->batch * c->n_kv_heads;
     a.gamma = gamma;
+    a.wait_limit = ctx->wait_limit;
     for (int l = 0; l < c->n_layers; ++l) a.scale_log2[l] = scale[l] * 1.4426950408889634f;
 
     const bool paged = c->layout == LETHE_PAGED;
@@ -373,7 +402,7 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
             if (a.chunk_tokens < cap_groups * kGroupTokens) {  // overflow of the logit buffer: one slice per CTA
                 a.spill_tokens = cap_groups * kGroupTokens - a.chunk_tokens;
                 const size_t need = (size_t)grid * a.spill_tokens * a.GP * sizeof(float);
-                st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "logit overflow scratch");
+                st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "logit overflow scratch", stream);
                 if (st != LETHE_OK) return st;
                 a.spill = (float*)ctx->scratch;
             }
@@ -459,7 +488,7 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         const size_t lg_bytes = up((size_t)a.n_items * a.flat_pitch * a.GP * sizeof(float));
         const size_t need = cnt_bytes + part_bytes + lg_bytes;
         if (need > ctx->flat_bytes) {
-            st = ensure(ctx, &ctx->flat, &ctx->flat_bytes, need, "scratch-merge buffers");
+            st = ensure(ctx, &ctx->flat, &ctx->flat_bytes, need, "scratch-merge buffers", stream);
             if (st != LETHE_OK) return st;
             if (cudaMemsetAsync(ctx->flat, 0, ctx->flat_bytes, (cudaStream_t)stream) != cudaSuccess)
                 return fail(ctx, LETHE_ERR_CUDA, "clearing the scratch-merge buffers failed");
@@ -496,7 +525,7 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         if (a.chunk_tokens < cap_groups * kGroupTokens) {
             a.spill_tokens = cap_groups * kGroupTokens - a.chunk_tokens;
             const size_t need = (size_t)grid * 2 * a.spill_tokens * a.GP * sizeof(float);
-            st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "logit overflow scratch");
+            st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "logit overflow scratch", stream);
             if (st != LETHE_OK) return st;
             a.spill = (float*)ctx->scratch;
         }
@@ -511,7 +540,7 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         if (a.chunk_tokens < cap_groups * kGroupTokens) {  // overflow of the logit buffer: one slice per CTA
             a.spill_tokens = cap_groups * kGroupTokens - a.chunk_tokens;
             const size_t need = (size_t)grid * a.spill_tokens * a.GP * sizeof(float);
-            st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "logit overflow scratch");
+            st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "logit overflow scratch", stream);
             if (st != LETHE_OK) return st;
             a.spill = (float*)ctx->scratch;
         }
@@ -546,13 +575,10 @@ lethe_status lethe_decode_attend_host(lethe_ctx* ctx, const lethe_cache* c, int 
                                       const void* q_host, const void* k_new_host, const void* v_new_host,
                                       const int32_t* token_pos_host, const float* scale, float gamma, void* out_host,
                                       float* lse_host, void* stream) {
-    lethe_status st = check_cache(ctx, c);
+    // every host-detectable error is found here, before staging is sized or a copy is enqueued
+    lethe_status st = check_attend_args(ctx, c, layer_begin, layer_end, q_host, k_new_host, v_new_host, token_pos_host,
+                                        scale, gamma, out_host, false);
     if (st != LETHE_OK) return st;
-    if (!q_host || !out_host) return fail(ctx, LETHE_ERR_INVALID_ARG, "q and out are required");
-    if (layer_begin < 0 || layer_end > c->n_layers || layer_begin >= layer_end)
-        return fail(ctx, LETHE_ERR_INVALID_ARG, "bad layer range");
-    if ((k_new_host == nullptr) != (v_new_host == nullptr)) return fail(ctx, LETHE_ERR_INVALID_ARG, "k_new and v_new go together");
-    if (k_new_host && !token_pos_host) return fail(ctx, LETHE_ERR_INVALID_ARG, "token_pos is required when appending");
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, LETHE_ERR_CUDA, "cannot select the context's device");
     const size_t nl = (size_t)(layer_end - layer_begin);
@@ -562,22 +588,13 @@ lethe_status lethe_decode_attend_host(lethe_ctx* ctx, const lethe_cache* c, int 
     const size_t kv_bytes = nl * c->batch * c->n_kv_heads * c->head_dim * eb;
     const size_t pos_bytes = (size_t)c->batch * 4;
     const size_t lse_bytes = nl * c->batch * c->n_q_heads * 4;
-    const size_t total = 2 * up(q_bytes) + 2 * up(kv_bytes) + up(pos_bytes) + up(lse_bytes);
-    st = ensure(ctx, &ctx->staging, &ctx->staging_bytes, total, "staging");
-    if (st != LETHE_OK) return st;
-    char* p = (char*)ctx->staging;
-    void* dq = p; p += up(q_bytes);
-    void* dout = p; p += up(q_bytes);  // re-pointed below when the kernel can write the caller's buffer
-    void* dk = p; p += up(kv_bytes);
-    void* dv = p; p += up(kv_bytes);
-    int32_t* dpos = (int32_t*)p; p += up(pos_bytes);
-    float* dlse = (float*)p;
     cudaStream_t s = (cudaStream_t)stream;
     cudaError_t e;
     // Results that live in page-locked host memory are written there by the kernel itself (the device-side alias of
     // the buffer): the stores cross the bus while the kernel runs and no download follows.  Pageable buffers are
-    // staged in device memory and copied.
-    auto device_alias = [](void* host, size_t bytes) -> void* {
+    // staged in device memory and copied; so is a page-locked buffer whose alias is not 16-byte aligned (a pointer
+    // into the middle of a larger allocation), which the kernels' vector accesses could not use.
+    auto device_alias = [](void* host, size_t bytes, bool need16) -> void* {
         cudaPointerAttributes lo, hi;
         if (cudaPointerGetAttributes(&lo, host) != cudaSuccess ||
             cudaPointerGetAttributes(&hi, (char*)host + bytes - 1) != cudaSuccess) {
@@ -586,15 +603,12 @@ lethe_status lethe_decode_attend_host(lethe_ctx* ctx, const lethe_cache* c, int 
         }
         if (lo.type != cudaMemoryTypeHost || hi.type != cudaMemoryTypeHost || !lo.devicePointer || !hi.devicePointer) return nullptr;
         if ((char*)hi.devicePointer - (char*)lo.devicePointer != (ptrdiff_t)(bytes - 1)) return nullptr;
+        if (need16 && ((uintptr_t)lo.devicePointer & 15)) return nullptr;
         return lo.devicePointer;
     };
-    void* out_alias = device_alias(out_host, q_bytes);
-    float* lse_alias = (lse_host && out_alias) ? (float*)device_alias(lse_host, lse_bytes) : nullptr;
+    void* out_alias = device_alias(out_host, q_bytes, true);
+    float* lse_alias = (lse_host && out_alias) ? (float*)device_alias(lse_host, lse_bytes, false) : nullptr;
     if (lse_host && !lse_alias) out_alias = nullptr;  // one path for both results
-    if (out_alias) {
-        dout = out_alias;
-        if (lse_host) dlse = lse_alias;
-    }
     // Inputs in page-locked memory as well: the kernels read them over the bus themselves and no upload precedes the
     // launch.  The persistent kernels fetch them an item ahead of their use, under the streaming of the previous
     // item; the asynchronous-epilogue kernel reads every input byte once (an epilogue warp stages an item's query
@@ -604,13 +618,32 @@ lethe_status lethe_decode_attend_host(lethe_ctx* ctx, const lethe_cache* c, int 
     // item need the query rows at once, so each CTA starts with a round trip over the bus, and still come out ahead
     // of the upload (quantised Llama-8B shape 0.20 against 0.23, clustered bf16 kernel 0.35 against 0.37).
     if (out_alias) {
-        void* qa = device_alias((void*)q_host, q_bytes);
-        void* ka = k_new_host ? device_alias((void*)k_new_host, kv_bytes) : nullptr;
-        void* va = v_new_host ? device_alias((void*)v_new_host, kv_bytes) : nullptr;
-        void* pa = k_new_host ? device_alias((void*)token_pos_host, pos_bytes) : nullptr;
-        if (qa && (!k_new_host || (ka && va && pa)))
-            return lethe_decode_attend(ctx, c, layer_begin, layer_end, qa, ka, va, (const int32_t*)pa, scale, gamma, dout,
-                                       lse_host ? dlse : nullptr, stream);
+        void* qa = device_alias((void*)q_host, q_bytes, true);
+        void* ka = k_new_host ? device_alias((void*)k_new_host, kv_bytes, true) : nullptr;
+        void* va = v_new_host ? device_alias((void*)v_new_host, kv_bytes, true) : nullptr;
+        void* pa = k_new_host ? device_alias((void*)token_pos_host, pos_bytes, false) : nullptr;
+        if (qa && (!k_new_host || (ka && va && pa)))   // nothing is staged: the staging area is not touched
+            return lethe_decode_attend(ctx, c, layer_begin, layer_end, qa, ka, va, (const int32_t*)pa, scale, gamma, out_alias,
+                                       lse_host ? lse_alias : nullptr, stream);
+    }
+    // staging: the inputs always, the results only when the kernel cannot write the caller's buffers
+    const size_t in_bytes = up(q_bytes) + (k_new_host ? 2 * up(kv_bytes) + up(pos_bytes) : 0);
+    const size_t res_bytes = out_alias ? 0 : up(q_bytes) + (lse_host ? up(lse_bytes) : 0);
+    st = ensure(ctx, &ctx->staging, &ctx->staging_bytes, in_bytes + res_bytes, "staging", stream);
+    if (st != LETHE_OK) return st;
+    char* p = (char*)ctx->staging;
+    void* dq = p; p += up(q_bytes);
+    void* dk = nullptr; void* dv = nullptr; int32_t* dpos = nullptr;
+    if (k_new_host) {
+        dk = p; p += up(kv_bytes);
+        dv = p; p += up(kv_bytes);
+        dpos = (int32_t*)p; p += up(pos_bytes);
+    }
+    void* dout = out_alias;
+    float* dlse = lse_alias;
+    if (!out_alias) {
+        dout = p; p += up(q_bytes);
+        dlse = lse_host ? (float*)p : nullptr;
     }
     // Staged path.  Layers are independent, so a call that covers many of them is cut into two chunks of layers: the
     // upload of the second and the download of the first run on their own streams (separate copy engines) under the
@@ -723,7 +756,7 @@ lethe_status lethe_alloc_budgets(lethe_ctx* ctx, int n_layers, int batch, const 
 }
 
 // Shared by the two retention entry points: where the survivor lists live, then the longest-first item order.
-static lethe_status prune_scratch(lethe_ctx* ctx, const CacheView& v, int* smem_tokens, int32_t** list_scratch) {
+static lethe_status prune_scratch(lethe_ctx* ctx, const CacheView& v, int* smem_tokens, int32_t** list_scratch, void* stream) {
     // keys / source list live in shared memory when an item fits; otherwise the list goes to global scratch
     const size_t budget_smem = ctx->max_smem - 8 * 1024;
     *smem_tokens = v.cap_tokens;
@@ -731,7 +764,7 @@ static lethe_status prune_scratch(lethe_ctx* ctx, const CacheView& v, int* smem_
     if ((size_t)*smem_tokens * 4 > budget_smem) {
         *smem_tokens = (int)(budget_smem / 4);
         const size_t need = (size_t)v.L * v.B * v.Hkv * v.cap_tokens * sizeof(int32_t);
-        lethe_status st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "prune scratch");
+        lethe_status st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "prune scratch", stream);
         if (st != LETHE_OK) return st;
         *list_scratch = (int32_t*)ctx->scratch;
     }
@@ -744,7 +777,7 @@ static lethe_status refresh_order(lethe_ctx* ctx, const lethe_cache* c, const Ca
     ctx->order_len = nullptr;
     if (items >= 2LL * ctx->sm_count && items <= (1 << 20)) {
         void* buf = ctx->order;
-        lethe_status st = ensure(ctx, &buf, &ctx->order_bytes, (size_t)items * sizeof(int32_t), "item order");
+        lethe_status st = ensure(ctx, &buf, &ctx->order_bytes, (size_t)items * sizeof(int32_t), "item order", stream);
         ctx->order = (int32_t*)buf;
         if (st != LETHE_OK) return st;
         cudaError_t e = launch_order(c->len, (int)items, v.cap_tokens, ctx->order, (cudaStream_t)stream);
@@ -767,7 +800,7 @@ lethe_status lethe_rasr_prune(lethe_ctx* ctx, const lethe_cache* c, const int32_
     const CacheView v = view_of(c);
     int smem_tokens;
     int32_t* list_scratch;
-    st = prune_scratch(ctx, v, &smem_tokens, &list_scratch);
+    st = prune_scratch(ctx, v, &smem_tokens, &list_scratch, stream);
     if (st != LETHE_OK) return st;
     cudaError_t e = launch_rasr_prune(v, budgets, recent, sink, keep_idx, keep_idx ? max_k : 0, smem_tokens,
                                       list_scratch, ctx->status, (cudaStream_t)stream);
@@ -789,7 +822,7 @@ lethe_status lethe_segment_prune(lethe_ctx* ctx, const lethe_cache* c, int32_t n
     const CacheView v = view_of(c);
     int smem_tokens;
     int32_t* list_scratch;
-    st = prune_scratch(ctx, v, &smem_tokens, &list_scratch);
+    st = prune_scratch(ctx, v, &smem_tokens, &list_scratch, stream);
     if (st != LETHE_OK) return st;
     cudaError_t e = launch_segment_prune(v, n_segments, tau, recent, sink, l_evict, keep_idx, keep_idx ? max_k : 0,
                                          smem_tokens, list_scratch, ctx->status, (cudaStream_t)stream);
@@ -819,7 +852,7 @@ lethe_status lethe_collapsed_prune(lethe_ctx* ctx, const lethe_cache* c, const i
     if (spill_keys) smem_tokens = (int)(budget_smem / 4);
     const size_t plan_bytes = (groups * sizeof(int32_t) + 255) / 256 * 256;
     const size_t list_bytes = groups * v.cap_tokens * sizeof(int32_t);
-    st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, plan_bytes + list_bytes * (spill_keys ? 2 : 1), "collapsed prune scratch");
+    st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, plan_bytes + list_bytes * (spill_keys ? 2 : 1), "collapsed prune scratch", stream);
     if (st != LETHE_OK) return st;
     int32_t* plan = (int32_t*)ctx->scratch;
     int32_t* lists = (int32_t*)((char*)ctx->scratch + plan_bytes);
@@ -855,6 +888,7 @@ lethe_status lethe_prefill_seed(lethe_ctx* ctx, const lethe_cache* c, const void
     a.paged = c->layout == LETHE_PAGED;
     a.page_tokens = a.paged ? c->page_tokens : 1;
     a.gamma_log2 = log2f(gamma);
+    a.wait_limit = ctx->wait_limit;
     for (int l = 0; l < c->n_layers; ++l) {
         if (!(scale[l] == scale[l]) || fabsf(scale[l]) > 1e30f) return fail(ctx, LETHE_ERR_INVALID_ARG, "scale must be finite");
         a.scale_log2[l] = scale[l] * 1.4426950408889634f;
@@ -862,7 +896,7 @@ lethe_status lethe_prefill_seed(lethe_ctx* ctx, const lethe_cache* c, const void
     const int items = c->n_layers * c->batch * c->n_kv_heads;
     const size_t stats_bytes = ctx->prefill_engine == 1 ? prefill_stats_bytes(items, prompt_len, a.HP)
                                                         : prefill_tc_stats_bytes(items, prompt_len, a.HP);
-    st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, stats_bytes, "prefill statistics");
+    st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, stats_bytes, "prefill statistics", stream);
     if (st != LETHE_OK) return st;
     a.stats = (float2*)ctx->scratch;
     cudaError_t e;

@@ -25,7 +25,7 @@ namespace lethe {
 // Epilogue warps per CTA.  Measured on the Llama-8B shape, of the copy peak: (8,2) with 2 / 3 / 4 epilogue warps
 // 0.98 / 1.015 / 1.03, (5,3) with 2 / 4: 1.01 / 0.79, (7,2) with 4 / 6: 1.005 / 0.83.
 __host__ __device__ constexpr int epilogue_warps(int nws) { return nws >= 8 ? 4 : 2; }
-constexpr int kWaitLimit = 200000;  // polls of a blocking try_wait before giving up
+constexpr int kWaitLimit = 200000;  // default poll limit of a bounded wait (AttendArgs::wait_limit overrides it when > 0)
 
 // Tensor maps of K and V for the TMA variant (rows x D, box 16 rows x 64 elements, 128-byte swizzle).
 struct alignas(64) TmaMaps {
@@ -64,6 +64,16 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned 
         : "memory");
     return ok != 0;
 }
+// The same test without any waiting inside the instruction.
+__device__ __forceinline__ bool mbar_test_wait(unsigned long long* bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, unsigned bytes) {
     asm volatile("{ .reg .b64 st; mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(smem_u32(bar)), "r"(bytes)
                  : "memory");
@@ -80,8 +90,9 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 // Bounded wait for a tile: polls without backing off for a long while (the data is usually microseconds away).
-__device__ __forceinline__ bool mbar_wait_tile(unsigned long long* bar, unsigned parity, volatile int* abort_flag) {
-    for (int it = 0; it < kWaitLimit * 8; ++it) {
+__device__ __forceinline__ bool mbar_wait_tile(unsigned long long* bar, unsigned parity, volatile int* abort_flag, int limit) {
+    if (mbar_test_wait(bar, parity)) return true;  // poll 0 does not block, so a limit of one poll is exactly one look
+    for (long long it = 1; it < (long long)limit * 8; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 1023) == 1023) {
             if (*abort_flag) return false;
@@ -93,8 +104,9 @@ __device__ __forceinline__ bool mbar_wait_tile(unsigned long long* bar, unsigned
 }
 
 // Bounded wait; false = gave up (or another warp already did).
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, volatile int* abort_flag) {
-    for (int it = 0; it < kWaitLimit; ++it) {
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, volatile int* abort_flag, int limit) {
+    if (mbar_test_wait(bar, parity)) return true;
+    for (int it = 1; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
         if (it > 16) __nanosleep(100);
@@ -207,6 +219,7 @@ __global__ void __launch_bounds__((NWS + epilogue_warps(NWS)) * 32, 1)
     const bool append = a.k_new != nullptr;
     unsigned int* sched = a.sched;
     volatile int* abort_flag = &hd.abort;
+    const int wait_limit = a.wait_limit > 0 ? a.wait_limit : kWaitLimit;
 
     // ---- set-up: barriers, first two descriptors
     bool drew_fail = false;  // meaningful in the ticket-drawing lane only
@@ -396,7 +409,7 @@ __global__ void __launch_bounds__((NWS + epilogue_warps(NWS)) * 32, 1)
             // handed its buffers back, which also publishes that descriptor
             auto acquire_next = [&]() {
                 const int sn = seq + 1;
-                if (sn >= 2 && !mbar_wait(&hd.empty[sn & 1], (unsigned)(((sn >> 1) - 1) & 1), abort_flag)) {
+                if (sn >= 2 && !mbar_wait(&hd.empty[sn & 1], (unsigned)(((sn >> 1) - 1) & 1), abort_flag, wait_limit)) {
                     alive = false;
                     nxt.valid = 0;
                 } else {
@@ -451,7 +464,7 @@ __global__ void __launch_bounds__((NWS + epilogue_warps(NWS)) * 32, 1)
                     cp_async_commit();
                 }
                 if constexpr (TMA) {
-                    if (!mbar_wait_tile(&hd.tma_full[warp][cslot], (slot_phase >> cslot) & 1u, abort_flag)) {
+                    if (!mbar_wait_tile(&hd.tma_full[warp][cslot], (slot_phase >> cslot) & 1u, abort_flag, wait_limit)) {
                         alive = false;
                         break;
                     }
@@ -591,14 +604,14 @@ __global__ void __launch_bounds__((NWS + epilogue_warps(NWS)) * 32, 1)
             const int p = seq & 1;
             // the descriptor of item seq was published by epilogue warp 0 while finishing item seq-2; waiting
             // for that hand-back (both epilogue warps arrive on it) makes the write visible to this warp too
-            if (seq >= 2 && !mbar_wait(&hd.empty[p], (unsigned)(((seq >> 1) - 1) & 1), abort_flag)) {
+            if (seq >= 2 && !mbar_wait(&hd.empty[p], (unsigned)(((seq >> 1) - 1) & 1), abort_flag, wait_limit)) {
                 alive = false;
                 break;
             }
             AsyncItem it;
             async_decode(a, hd.desc_ticket[seq & 3], hd.desc_n_old[seq & 3], it);
             if (!it.valid) break;
-            if (!mbar_wait(&hd.full[p], (unsigned)((seq >> 1) & 1), abort_flag)) {
+            if (!mbar_wait(&hd.full[p], (unsigned)((seq >> 1) & 1), abort_flag, wait_limit)) {
                 alive = false;
                 break;
             }

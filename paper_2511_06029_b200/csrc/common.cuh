@@ -48,6 +48,7 @@ struct AttendArgs {
     int splits;                // CTAs per item (cluster size)
     int chunk_tokens;          // logit-buffer capacity of one CTA, in tokens
     float gamma;
+    int wait_limit;            // poll limit of the bounded mbarrier waits (0 = the kernel's default)
     float scale_log2[kMaxLayers];  // scale[l] * log2(e) (times the key scale for a quantised cache), by absolute layer
     float k_scale[kMaxLayers];     // quantised caches: a stored key byte x means k_scale[l] * x (else unused)
     float v_scale[kMaxLayers];     // the same for values

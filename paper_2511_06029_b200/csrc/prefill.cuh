@@ -16,6 +16,7 @@ struct PrefillArgs {
     int B, Hq, Hkv, G, HP, P;
     int capacity, cap_tokens, page_tokens, paged;
     float gamma_log2;
+    int wait_limit;  // poll limit of the bounded mbarrier waits of the tensor-memory kernels (0 = their default)
     float scale_log2[kMaxLayers];
 };
 

@@ -64,6 +64,8 @@ struct TcShared {
     unsigned long long a_full[kTcABuffers], a_empty[kTcABuffers];
     unsigned long long b_full[kTcStages], b_empty[kTcStages];
     unsigned long long t_full[2], t_empty[2];
+    unsigned long long mma_drained;  // used only after a timeout: every MMA issued so far has finished
+    int armed_a, armed_steps, mma_steps;  // TMA boxes and MMA steps issued when the roles left their loops
     uint32_t tmem_base;
     int abort;
     // COLSUM: bias (log2(weight / sum) - max) of the 64 columns a warp reads, of the tiles in flight; one copy per warp
@@ -88,9 +90,19 @@ __device__ __forceinline__ bool tc_mbar_try_wait(unsigned long long* bar, unsign
                  : "memory");
     return ok != 0;
 }
-// Bounded wait; false = gave up (or another thread already did).
-__device__ __forceinline__ bool tc_wait(unsigned long long* bar, unsigned parity, volatile int* abort_flag) {
-    for (int it = 0; it < kTcWaitLimit; ++it) {
+__device__ __forceinline__ bool tc_mbar_test_wait(unsigned long long* bar, unsigned parity) {  // never waits inside
+    unsigned ok;
+    asm volatile("{ .reg .pred p; mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(ok)
+                 : "r"(smem_u32(bar)), "r"(parity)
+                 : "memory");
+    return ok != 0;
+}
+// Bounded wait; false = gave up (or another thread already did).  Poll 0 does not block, so a limit of one poll
+// is exactly one look at the barrier.
+__device__ __forceinline__ bool tc_wait(unsigned long long* bar, unsigned parity, volatile int* abort_flag, int limit) {
+    if (tc_mbar_test_wait(bar, parity)) return true;
+    for (int it = 1; it < limit; ++it) {
         if (tc_mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
         if (it > 64) __nanosleep(64);
@@ -242,6 +254,16 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
     const uint32_t a_tile0 = dyn;
     const uint32_t b_tile0 = dyn + kTcABuffers * TILE_BYTES;
     volatile int* abort_flag = &sh.abort;
+    const int wait_limit = a.wait_limit > 0 ? a.wait_limit : kTcWaitLimit;
+    // After a wait has run out, copies and MMAs this CTA started may still be in flight; the thread that started them
+    // waits for them (with the fixed limit, whatever wait_limit says) before the CTA gives its shared and tensor
+    // memory back.
+    auto drain = [&](unsigned long long* bar, unsigned parity) {
+        for (int it = 0; it < kTcWaitLimit; ++it) {
+            if (tc_mbar_try_wait(bar, parity)) return;
+            if (it > 64) __nanosleep(64);
+        }
+    };
 
     if (tid == 0) {
         const int producers = TMA ? 1 : kTcLoaderThreads;
@@ -257,6 +279,10 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
             tc_mbar_init(&sh.b_full[i], producers);
             tc_mbar_init(&sh.b_empty[i], 1);
         }
+        tc_mbar_init(&sh.mma_drained, 1);
+        sh.armed_a = -1;
+        sh.armed_steps = 0;
+        sh.mma_steps = 0;
         sh.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -339,25 +365,29 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
                 };
                 int step = 0;
                 bool alive = true;
+                int a_armed = -1;  // last block operand whose box was issued
                 for (int ab = 0; ab < nA && alive; ++ab) {
                     int t0, t1;
                     tc_range<MODE>(ab, P, qpb, t0, t1);
                     for (int t = t0; t < t1; ++t, ++step) {
                         const int s = step % kTcStages;
                         if (t == t0) {
-                            if (ab >= kTcABuffers && !tc_wait(&sh.a_empty[ab % kTcABuffers], (unsigned)(((ab / kTcABuffers) - 1) & 1), abort_flag)) { alive = false; break; }
+                            if (ab >= kTcABuffers && !tc_wait(&sh.a_empty[ab % kTcABuffers], (unsigned)(((ab / kTcABuffers) - 1) & 1), abort_flag, wait_limit)) { alive = false; break; }
                             const uint32_t at = a_tile0 + (ab % kTcABuffers) * TILE_BYTES;
+                            a_armed = ab;
                             tc_mbar_expect_tx(&sh.a_full[ab % kTcABuffers], MODE == kModeStats ? q_bytes : k_bytes);
                             if (MODE == kModeStats) load_queries(ab * qpb, at, &sh.a_full[ab % kTcABuffers]);
                             else load_keys(ab * kTcTile, at, &sh.a_full[ab % kTcABuffers]);
                         }
-                        if (step >= kTcStages && !tc_wait(&sh.b_empty[s], (unsigned)(((step / kTcStages) - 1) & 1), abort_flag)) { alive = false; break; }
+                        if (step >= kTcStages && !tc_wait(&sh.b_empty[s], (unsigned)(((step / kTcStages) - 1) & 1), abort_flag, wait_limit)) { alive = false; break; }
                         const uint32_t bt = b_tile0 + s * TILE_BYTES;
                         tc_mbar_expect_tx(&sh.b_full[s], MODE == kModeStats ? k_bytes : q_bytes);
                         if (MODE == kModeStats) load_keys(t * kTcTile, bt, &sh.b_full[s]);
                         else load_queries(t * qpb, bt, &sh.b_full[s]);
                     }
                 }
+                sh.armed_a = a_armed;  // what was issued, for the drain after a timeout
+                sh.armed_steps = step;
             }
             __syncwarp();
         } else {
@@ -371,12 +401,12 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
                     const int s = step % kTcStages;
                     const bool first = t == t0;
                     if (first) {
-                        if (ab >= kTcABuffers && !tc_wait(&sh.a_empty[ab % kTcABuffers], (unsigned)(((ab / kTcABuffers) - 1) & 1), abort_flag)) { alive = false; break; }
+                        if (ab >= kTcABuffers && !tc_wait(&sh.a_empty[ab % kTcABuffers], (unsigned)(((ab / kTcABuffers) - 1) & 1), abort_flag, wait_limit)) { alive = false; break; }
                         const uint32_t at = a_tile0 + (ab % kTcABuffers) * TILE_BYTES;
                         if (MODE == kModeStats) tc_load_queries<D>(a, l, b, hkv, ab * qpb, used, at, ltid);
                         else tc_load_keys<D>(a, item, ab * kTcTile, at, ltid);
                     }
-                    if (step >= kTcStages && !tc_wait(&sh.b_empty[s], (unsigned)(((step / kTcStages) - 1) & 1), abort_flag)) { alive = false; break; }
+                    if (step >= kTcStages && !tc_wait(&sh.b_empty[s], (unsigned)(((step / kTcStages) - 1) & 1), abort_flag, wait_limit)) { alive = false; break; }
                     if (MODE == kModeStats) tc_load_keys<D>(a, item, t * kTcTile, b_tile0 + s * TILE_BYTES, ltid);
                     else tc_load_queries<D>(a, l, b, hkv, t * qpb, used, b_tile0 + s * TILE_BYTES, ltid);
                     // the step's copies must have landed and be visible to the MMA's proxy before it is told; nothing
@@ -400,9 +430,9 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
                 tc_range<MODE>(ab, P, qpb, t0, t1);
                 for (int t = t0; t < t1; ++t, ++step) {
                     const int s = step % kTcStages, buf = step & 1;
-                    if (t == t0 && !tc_wait(&sh.a_full[ab % kTcABuffers], (unsigned)((ab / kTcABuffers) & 1), abort_flag)) { alive = false; break; }
-                    if (!tc_wait(&sh.b_full[s], (unsigned)((step / kTcStages) & 1), abort_flag)) { alive = false; break; }
-                    if (step >= 2 && !tc_wait(&sh.t_empty[buf], (unsigned)(((step >> 1) - 1) & 1), abort_flag)) { alive = false; break; }
+                    if (t == t0 && !tc_wait(&sh.a_full[ab % kTcABuffers], (unsigned)((ab / kTcABuffers) & 1), abort_flag, wait_limit)) { alive = false; break; }
+                    if (!tc_wait(&sh.b_full[s], (unsigned)((step / kTcStages) & 1), abort_flag, wait_limit)) { alive = false; break; }
+                    if (step >= 2 && !tc_wait(&sh.t_empty[buf], (unsigned)(((step >> 1) - 1) & 1), abort_flag, wait_limit)) { alive = false; break; }
                     tc_fence_after();
                     const uint32_t at = a_tile0 + (ab % kTcABuffers) * TILE_BYTES, bt = b_tile0 + s * TILE_BYTES;
 #pragma unroll
@@ -416,6 +446,7 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
                     tc_commit(&sh.t_full[buf]);
                 }
             }
+            sh.mma_steps = step;
         }
         __syncwarp();
     } else {
@@ -463,7 +494,7 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
                     }
                     __syncwarp();
                 }
-                if (!tc_wait(&sh.t_full[buf], (unsigned)((step >> 1) & 1), abort_flag)) { alive = false; break; }
+                if (!tc_wait(&sh.t_full[buf], (unsigned)((step >> 1) & 1), abort_flag, wait_limit)) { alive = false; break; }
                 tc_fence_after();
 #pragma unroll
                 for (int ch = 0; ch < 2; ++ch) {
@@ -552,7 +583,22 @@ __global__ void __launch_bounds__(tc_threads<TMA>(), kTcCtasPerSm)
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    if (sh.abort && tid == 0) record_error(a.status, LETHE_ERR_TIMEOUT, item);
+    if (sh.abort) {  // uniform for the CTA
+        if (tid == 0) record_error(a.status, LETHE_ERR_TIMEOUT, item);
+        if (warp == kTcMmaWarp && lane == 0 && sh.mma_steps > 0) {
+            tc_commit(&sh.mma_drained);  // arrives once every MMA issued so far has finished
+            drain(&sh.mma_drained, 0u);
+        }
+        if (TMA && warp == kTcMmaWarp + 1 && lane == 0) {  // boxes issued but perhaps not landed yet
+            const int aa = sh.armed_a, steps = sh.armed_steps;
+            if (aa >= 0) drain(&sh.a_full[aa % kTcABuffers], (unsigned)((aa / kTcABuffers) & 1));
+            for (int st = max(0, steps - kTcStages); st < steps; ++st)
+                drain(&sh.b_full[st % kTcStages], (unsigned)((st / kTcStages) & 1));
+        }
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    }
     if (warp == kTcMmaWarp)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTcTmemCols) : "memory");
 }

@@ -482,49 +482,100 @@ def test_free_running_overlap_llama_shape(ctx):
 
 @pytest.mark.parametrize("pinned", [True, False])
 @pytest.mark.parametrize("L,B,Hkv", [(2, 2, 2), (5, 16, 20)])
-def test_host_entry_point_matches_the_device_one(ctx, L, B, Hkv, pinned):
-    """lethe_decode_attend_host (host tensors in, host tensors out) against lethe_decode_attend on a copy of the
-    same cache.  Page-locked buffers: the kernel writes the results into them itself, and the large call (persistent
-    kernel) also reads its inputs from them; pageable buffers: staged copies, the small call on one stream, the
-    large one as two chunks whose copies overlap the kernels.  Appended rows, positions and lengths must be
-    identical, outputs and relevance equal up to the kernels' tolerance (the chunks may run a different kernel
-    variant than the whole call)."""
+def test_host_entry_point_against_the_oracle(ctx, L, B, Hkv, pinned):
+    """lethe_decode_attend_host (host tensors in, host tensors out) against the oracle at the same tolerances as the
+    device entry point.  Page-locked buffers: the kernel writes the results into them itself, and the large call
+    (persistent kernel) also reads its inputs from them; pageable buffers: staged copies, the small call on one
+    stream, the large one as two chunks whose copies overlap the kernels.  One step delivers its results into the
+    middle of a larger page-locked allocation, one into a page-locked buffer that is not 16-byte aligned (which
+    must take the staged path instead of being refused)."""
     pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
     G, D, cap, n0 = 4, 64, 96, 70
     Hq = Hkv * G
     oc = random_cache(L, B, Hq, Hkv, D, cap, n0, dtype=torch.bfloat16, seed=L + B, rel_init="rand")
-    ga, gb = to_device(oc), to_device(oc)
-    dev = ga.device
+    gb = to_device(oc)
     g = torch.Generator().manual_seed(11)
-    scale = [0.12] * L
-    for step in range(3):
+    scale = torch.full((L,), 0.12)
+    for step in range(4):
         q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
         kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
         vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
         tp = torch.arange(B, dtype=torch.int32) + 100 + step
-        out_a = torch.empty_like(q, device=dev)
-        lse_a = torch.empty((L, B, Hq), dtype=torch.float32, device=dev)
-        ctx.decode_attend(ga, 0, L, q.to(dev), kn.to(dev), vn.to(dev), tp.to(dev), scale, 0.9, out_a, lse_a)
+        s, o_out, o_lse, _ = oracle.decode_attend(oc, 0, L, q, kn, vn, tp, scale, 0.9, want_lse=True)
+        assert s == oracle.OK
         qh, kh, vh, th = pin(q), pin(kn), pin(vn), pin(tp)
         if pinned and step == 1:   # results into the middle of a larger page-locked allocation
             big = torch.empty((3 * q.numel(),), dtype=torch.bfloat16).pin_memory()
             out_b = big[q.numel():2 * q.numel()].view(q.shape)
+        elif pinned and step == 2:  # page-locked but only 2-byte aligned: staged, not refused
+            big = torch.empty((q.numel() + 8,), dtype=torch.bfloat16).pin_memory()
+            out_b = big[1:1 + q.numel()].view(q.shape)
+            assert out_b.data_ptr() % 16 != 0
         else:
             out_b = pin(torch.empty_like(q))
         lse_b = pin(torch.empty((L, B, Hq), dtype=torch.float32))
-        ctx.decode_attend_host(gb, 0, L, qh, kh, vh, th, scale, 0.9, out_b, lse_b)
+        ctx.decode_attend_host(gb, 0, L, qh, kh, vh, th, scale.tolist(), 0.9, out_b, lse_b)
         assert ctx.poll_status()[0] == 0                       # synchronises the stream: host results are valid
-        assert (out_b.float() - out_a.cpu().float()).abs().max() <= 1e-2
-        assert torch.allclose(lse_b, lse_a.cpu(), rtol=1e-4, atol=1e-4)
-        assert torch.equal(gb.len.cpu(), ga.len.cpu()) and torch.equal(gb.pos.cpu(), ga.pos.cpu())
-        assert torch.equal(gb.k.cpu().view(torch.int16), ga.k.cpu().view(torch.int16))
-        assert torch.equal(gb.v.cpu().view(torch.int16), ga.v.cpu().view(torch.int16))
-        assert torch.allclose(gb.rel.cpu(), ga.rel.cpu(), rtol=1e-3, atol=1e-6)
+        assert (out_b.double() - o_out.double()).abs().max() <= OUT_TOL[torch.bfloat16]
+        assert torch.allclose(lse_b, o_lse, rtol=1e-4, atol=1e-4)
+        assert_state_matches(gb, oc)                           # appended rows, pos, len bit-exact; rel within 1e-3 rel
     # attend-only through the host path
-    q = pin(torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16))
+    q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+    s, o_out, _, _ = oracle.decode_attend(oc, 0, L, q, None, None, None, scale, 0.9)
     out_b = pin(torch.empty_like(q))
-    out_a = torch.empty_like(q, device=dev)
-    ctx.decode_attend(ga, 0, L, q.to(dev), None, None, None, scale, 0.9, out_a)
-    ctx.decode_attend_host(gb, 0, L, q, None, None, None, scale, 0.9, out_b, None)
+    ctx.decode_attend_host(gb, 0, L, pin(q), None, None, None, scale.tolist(), 0.9, out_b, None)
     assert ctx.poll_status()[0] == 0
-    assert (out_b.float() - out_a.cpu().float()).abs().max() <= 1e-2 and torch.equal(gb.len.cpu(), ga.len.cpu())
+    assert (out_b.double() - o_out.double()).abs().max() <= OUT_TOL[torch.bfloat16]
+    assert_state_matches(gb, oc)
+
+
+def test_host_entry_point_checks_before_it_enqueues(ctx):
+    """Host-detectable errors of lethe_decode_attend_host are found before anything is staged or copied: the
+    cache, the results and the status word stay as they were."""
+    from paper_2511_06029_b200 import binding
+    oc = random_cache(4, 2, 8, 2, 128, 32, 8, dtype=torch.bfloat16, seed=0)
+    gc = to_device(oc)
+    q = torch.zeros((4, 2, 8, 128), dtype=torch.bfloat16)
+    kn = torch.zeros((4, 2, 2, 128), dtype=torch.bfloat16)
+    tp = torch.zeros(2, dtype=torch.int32)
+    out = torch.full_like(q, 3.0)
+    for kwargs in [dict(gamma=0.0), dict(gamma=1.5), dict(scale=[0.1, float("nan"), 0.1, 0.1]), dict(l1=5)]:
+        with pytest.raises(binding.LetheError) as e:
+            ctx.decode_attend_host(gc, 0, kwargs.get("l1", 4), q, kn, kn, tp, kwargs.get("scale", [0.1] * 4),
+                                   kwargs.get("gamma", 0.9), out)
+        assert e.value.status == binding.ERR_INVALID_ARG
+    with pytest.raises(binding.LetheError):
+        ctx.decode_attend_host(gc, 0, 4, q, kn, None, tp, [0.1] * 4, 0.9, out)      # k_new without v_new
+    torch.cuda.synchronize()
+    assert torch.all(out == 3.0) and torch.equal(gc.len.cpu(), oc.len) and torch.equal(gc.k.cpu().view(torch.int16), oc.k.view(torch.int16))
+    assert ctx.poll_status()[0] == 0
+
+
+@pytest.mark.parametrize("ratio", [0.05, 0.1, 0.25, 0.5])
+def test_ragged_sweep_ratios_shortest_and_longest(ctx, ratio):
+    """The ragged workload's budget ratios: the shortest and the longest sequence (1024 and 32768 tokens, 16-token
+    pages, shuffled tables) attend at full length, are pruned to `ratio` of their length (never below the protected
+    count: at 0.05 the short sequence's budget is the floor), and attend again on the pruned cache — every call
+    against the oracle."""
+    oracle.set_threads(min(8, oracle.max_threads()))
+    try:
+        w = synth.shrink(synth.WORKLOADS["ragged"], n_layers=2, batch=2, prompt_len=32768)
+        lens = torch.tensor([1024, 32768])
+        cap = 33280
+        st_c = synth.initial_kv(w, 32768, cap)
+        st_c["len"][:] = lens[None, :, None].to(torch.int32)
+        st_p = synth.to_paged(st_c, 16, seed=int(ratio * 100), spare_pages=11)
+        del st_c
+        oc = cache_from_state(w, st_p, cap)
+        gc = to_device(oc)
+        scale = synth.layer_scales(w)
+        T = (w.n_layers * torch.clamp((lens.double() * ratio).long(), min=w.k_min)).to(torch.int64)
+        for step in range(4):
+            x = synth.step_inputs(w, step)
+            _step(ctx, oc, gc, x["q"], x["k_new"], x["v_new"], x["token_pos"], scale, w.gamma, 0, w.n_layers, want_lse=False)
+            if step == 1:
+                bud, _ = _prune_both(ctx, oc, gc, T, w.k_min, w.recent, w.sink, int(32770 * ratio) + 8)
+                assert int(bud.sum()) == int(T.sum())
+                assert int(oc.len[:, 1].max()) <= int(32770 * ratio) + w.n_layers * 32770   # pruned
+    finally:
+        oracle.set_threads(1)
