@@ -782,6 +782,10 @@ def main():
     barrier()
     r.check()
     if not args.no_e2e:
+        for _ in range(max(args.warmup, 3)):             # the host path's own warm-up (its first call sets up staging)
+            r.decode(host=True)
+            if r.prune_due():
+                r.prune()
         barrier()
         e_total_ms, _, _, e_th = timed_loop(r, args.steps, host=True)
         barrier()
