@@ -800,14 +800,17 @@ def main():
         room = w.prune_interval - (r.step_no % w.prune_interval)
         pl_steps = min(32, max(4, room - 8))
         r.ctx.set_tuning(args.pl_variant, args.pl_splits)
+        r.ctx.set_tuning(51, 0)                          # layer pipelining: cached K / V tiles are fetched under the previous launch's tail
         ms_pl, th_pl = per_layer_mode(r, pl_steps)
+        r.ctx.set_tuning(50, 0)
         r.ctx.set_tuning(args.variant, args.splits)
         r.check()
         gbs = th_pl * bytes_per_th / (ms_pl * 1e-3) / 1e9
         per_layer = {"ms_per_step": ms_pl, "token_heads_per_step": th_pl, "value": th_pl / (ms_pl * 1e-3),
                      "algorithmic_GBs": gbs, "frac": gbs / peak, "frac_of_8TBs_nominal": gbs / NOMINAL_HBM_GBS,
                      "mode": f"{w.n_layers} launches per step (one per layer), replayed from a CUDA graph, "
-                             f"{pl_steps} steps; not part of `value`"}
+                             f"{pl_steps} steps; layer pipelining on (a launch fetches cached K / V tiles before the "
+                             f"previous launch has completed, and reads its query only after it has); not part of `value`"}
 
     sweep = None
     if args.sweep and w.page_tokens and world == 1:

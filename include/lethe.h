@@ -131,6 +131,15 @@ lethe_status lethe_poll_status(lethe_ctx *ctx, void *stream, int32_t *info);
  * shape (4,4) (8,4) (4,2) (4,3) (2,4) (8,2) (splits as above), variants 8..13 the persistent one with shape (8,4)
  * (12,3) (10,4) (8,5) (16,2) (12,2) (e4m3 only); any other value means the clustered kernel with shape (4,4), the faster of
  * the two at every size measured.
+ * 44..49 = the clustered kernel's six shapes for launches of one layer at a time (few items per launch): the CTAs of
+ * an item merge by one-sided pushes through distributed shared memory (no cluster barriers), and — when variant 51
+ * is also set — a launch fetches cached K / V tiles while the previous launch is still finishing.
+ * variant 50 / 51 switch that layer pipelining off / on and leave everything else as it is.  It applies to a decode
+ * call that follows, through the same context and on the same stream, a decode call on the same cache over other
+ * layers (what a model's layer loop issues); such a call reads len, the page table and K / V rows of its own layers
+ * before the kernel enqueued just before it on the stream has completed, so between the two calls nothing else
+ * may be enqueued on that stream that writes those (any other call of this library in between switches the early
+ * fetch off for the next decode call by itself).
  * variant 40..42 select the engine of lethe_prefill_seed and leave everything else as it is: 40 = tcgen05
  * kernels (accumulators in tensor memory, operand tiles by TMA; the default), 41 = mma.sync kernels,
  * 42 = tcgen05 kernels with cp.async tiles; splits is ignored.

@@ -17,6 +17,8 @@ cudaError_t launch_attend_kv8(const AttendArgs& a, int D, int shape, bool paged,
 size_t simt_smem_bytes(int D, int chunk_tokens, int GP);
 cudaError_t launch_attend_mma(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream);
 size_t mma_smem_bytes(int D, int shape, int chunk_tokens, int GP);
+cudaError_t launch_attend_layer(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream);
+size_t layer_smem_bytes(int D, int shape, int chunk_tokens, int GP);
 cudaError_t launch_attend_stream(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream);
 size_t stream_smem_bytes(int D, int shape, int chunk_tokens, int GP);
 cudaError_t launch_attend_async(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream, bool tma,
@@ -94,6 +96,11 @@ struct lethe_ctx {
     bool host_pipeline_ready;
     int variant, splits;
     int wait_limit;  // poll limit of the kernels' bounded waits (0 = their defaults); lethe_set_wait_limit
+    // layer pipelining (tuning 51): the last call enqueued through this context, if it was a decode call
+    int pipeline_layers;
+    const int32_t* last_len;  // cache.len of that call (NULL: the last call was something else)
+    int last_l0, last_l1;
+    void* last_stream;
     int prefill_engine;  // 0 = tcgen05 kernels (TMA producers when the cache is contiguous), 1 = mma.sync kernels, 2 = tcgen05 with cp.async producers
     // TMA variant: tensor maps of the last cache seen (rebuilt when k, v, the row count or D change)
     alignas(64) unsigned char tma_maps[512];
@@ -295,8 +302,14 @@ lethe_status lethe_set_tuning(lethe_ctx* ctx, int variant, int splits) {
         ctx->prefill_engine = variant - 40;
         return LETHE_OK;
     }
-    if (variant < 0 || variant > 37) return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..37 or 40..42");
-    const bool flat_variant = variant >= 32;
+    if (variant == 50 || variant == 51) {  // layer pipelining of the one-layer-per-launch kernel; nothing else changes
+        ctx->pipeline_layers = variant - 50;
+        return LETHE_OK;
+    }
+    const bool layer_variant = variant >= 44 && variant <= 49;
+    if ((variant < 0 || variant > 37) && !layer_variant)
+        return fail(ctx, LETHE_ERR_INVALID_ARG, "variant must be 0..37, 40..42 or 44..51");
+    const bool flat_variant = variant >= 32 && variant <= 37;
     if (flat_variant ? (splits < 0 || splits > 16)
                      : !(splits == 0 || splits == 1 || splits == 2 || splits == 4 || splits == 8 || splits == 16))
         return fail(ctx, LETHE_ERR_INVALID_ARG, "splits must be 0, 1, 2, 4, 8 or 16 (0..16 for the scratch-merged variants)");
@@ -366,6 +379,15 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
     a.n_items = (layer_end - layer_begin) * c->batch * c->n_kv_heads;
     a.gamma = gamma;
     a.wait_limit = ctx->wait_limit;
+    // Layer pipelining: the kernel may fetch cached K / V tiles before the previous kernel of the stream is done only
+    // if that kernel cannot have written this call's items: it was this context's previous call, a decode call on
+    // the same cache and stream, over layers disjoint from this call's.
+    a.early_prefetch = ctx->pipeline_layers && ctx->last_len == c->len && ctx->last_stream == stream &&
+                       (layer_end <= ctx->last_l0 || layer_begin >= ctx->last_l1);
+    ctx->last_len = c->len;
+    ctx->last_l0 = layer_begin;
+    ctx->last_l1 = layer_end;
+    ctx->last_stream = stream;
     for (int l = 0; l < c->n_layers; ++l) a.scale_log2[l] = scale[l] * 1.4426950408889634f;
 
     const bool paged = c->layout == LETHE_PAGED;
@@ -463,12 +485,12 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
             for (int shape : {0, 3})
                 if (variant == 0 && async_chunk(shape) * 5 >= (size_t)cap_pad * 2) variant = 16 + shape;
             if (variant == 0) variant = 8 + 0;
-        } else variant = 2;  // few items per launch (one layer at a time): clustered kernel, 4 warps x 3 stages
+        } else variant = 44;  // few items per launch (one layer at a time): clustered kernel with the one-sided merge, 4 warps x 3 stages
     }
     if (variant >= 2 && !mma_ok) return fail(ctx, LETHE_ERR_UNSUPPORTED, "tensor-core variants need bf16 and 16-token pages");
 
     cudaError_t e;
-    if (variant >= 32) {  // clustered kernel's arithmetic, CTAs of an item merged through scratch instead of a cluster
+    if (variant >= 32 && variant <= 37) {  // clustered kernel's arithmetic, CTAs of an item merged through scratch instead of a cluster
         const int shape = variant - 32;
         int S = ctx->splits;
         if (S == 0) {  // chunks of about 256 tokens, at most 16 per item
@@ -498,7 +520,7 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         a.flat_part = (float*)((char*)ctx->flat + cnt_bytes);
         a.flat_lg = (float*)((char*)ctx->flat + cnt_bytes + part_bytes);
         e = launch_attend_mma(a, c->head_dim, shape, paged, (cudaStream_t)stream);
-    } else if (variant >= 16) {  // persistent, asynchronous epilogue: both logit buffers (item parity) share what is left
+    } else if (variant >= 16 && variant < 32) {  // persistent, asynchronous epilogue: both logit buffers (item parity) share what is left
         if (ctx->splits > 1) return fail(ctx, LETHE_ERR_INVALID_ARG, "the persistent variants do not split items");
         const bool tma = variant >= 24;
         const int shape = tma ? variant - 24 : variant - 16;
@@ -530,7 +552,7 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
             a.spill = (float*)ctx->scratch;
         }
         e = launch_attend_async(a, c->head_dim, shape, paged, grid, (cudaStream_t)stream, tma, ctx->tma_maps);
-    } else if (variant >= 8) {  // persistent: one CTA per SM walks all items
+    } else if (variant >= 8 && variant < 16) {  // persistent: one CTA per SM walks all items
         if (ctx->splits > 1) return fail(ctx, LETHE_ERR_INVALID_ARG, "the persistent variant does not split items");
         a.splits = 1;
         a.chunk_tokens = stream_chunk(variant - 8);
@@ -547,10 +569,12 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         e = launch_attend_stream(a, c->head_dim, variant - 8, paged, grid, (cudaStream_t)stream);
     } else {
         // CTAs per item: the smallest cluster whose logit buffer fits, grown until the grid covers the SMs twice.
+        const bool layer_kernel = variant >= 44;
         auto smem_for = [&](int S) -> size_t {
             const int chunk = ((cap_groups + S - 1) / S) * kGroupTokens;
             return variant == 1 ? simt_smem_bytes(c->head_dim, chunk, a.GP)
-                                : mma_smem_bytes(c->head_dim, variant - 2, chunk, a.GP);
+                                : (layer_kernel ? layer_smem_bytes(c->head_dim, variant - 44, chunk, a.GP)
+                                                : mma_smem_bytes(c->head_dim, variant - 2, chunk, a.GP));
         };
         int S = ctx->splits;
         if (S == 0) {
@@ -565,7 +589,8 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         a.splits = S;
         a.chunk_tokens = ((cap_groups + S - 1) / S) * kGroupTokens;
         e = variant == 1 ? launch_attend_simt(a, c->dtype, c->head_dim, paged, (cudaStream_t)stream)
-                         : launch_attend_mma(a, c->head_dim, variant - 2, paged, (cudaStream_t)stream);
+                         : (layer_kernel ? launch_attend_layer(a, c->head_dim, variant - 44, paged, (cudaStream_t)stream)
+                                         : launch_attend_mma(a, c->head_dim, variant - 2, paged, (cudaStream_t)stream));
     }
     if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attend launch");
     return LETHE_OK;
@@ -733,6 +758,7 @@ lethe_status lethe_decode_attend_host(lethe_ctx* ctx, const lethe_cache* c, int 
 lethe_status lethe_estimate_sparsity(lethe_ctx* ctx, const lethe_cache* c, float* sparsity, void* stream) {
     lethe_status st = check_cache(ctx, c);
     if (st != LETHE_OK) return st;
+    ctx->last_len = nullptr;  // the next decode call does not follow a decode call
     if (!sparsity) return fail(ctx, LETHE_ERR_INVALID_ARG, "sparsity is NULL");
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, LETHE_ERR_CUDA, "cannot select the context's device");
@@ -792,6 +818,7 @@ lethe_status lethe_rasr_prune(lethe_ctx* ctx, const lethe_cache* c, const int32_
                               int32_t sink, int32_t* keep_idx, int32_t max_k, void* stream) {
     lethe_status st = check_cache(ctx, c);
     if (st != LETHE_OK) return st;
+    ctx->last_len = nullptr;  // the next decode call does not follow a decode call
     if (!budgets) return fail(ctx, LETHE_ERR_INVALID_ARG, "budgets is NULL");
     if (recent < 0 || sink < 0) return fail(ctx, LETHE_ERR_INVALID_ARG, "recent and sink must be >= 0");
     if (keep_idx && max_k < 1) return fail(ctx, LETHE_ERR_INVALID_ARG, "max_k must be positive with keep_idx");
@@ -812,6 +839,7 @@ lethe_status lethe_segment_prune(lethe_ctx* ctx, const lethe_cache* c, int32_t n
                                  int32_t sink, int32_t* l_evict, int32_t* keep_idx, int32_t max_k, void* stream) {
     lethe_status st = check_cache(ctx, c);
     if (st != LETHE_OK) return st;
+    ctx->last_len = nullptr;  // the next decode call does not follow a decode call
     if (!l_evict) return fail(ctx, LETHE_ERR_INVALID_ARG, "l_evict is NULL");
     if (n_segments < 2) return fail(ctx, LETHE_ERR_INVALID_ARG, "n_segments must be at least 2");
     if (!(tau >= 1.0f)) return fail(ctx, LETHE_ERR_INVALID_ARG, "tau must be >= 1");
@@ -834,6 +862,7 @@ lethe_status lethe_collapsed_prune(lethe_ctx* ctx, const lethe_cache* c, const i
                                    int32_t sink, int32_t scope, int32_t* keep_idx, int32_t max_k, void* stream) {
     lethe_status st = check_cache(ctx, c);
     if (st != LETHE_OK) return st;
+    ctx->last_len = nullptr;  // the next decode call does not follow a decode call
     if (!budgets) return fail(ctx, LETHE_ERR_INVALID_ARG, "budgets is NULL");
     if (recent < 0 || sink < 0) return fail(ctx, LETHE_ERR_INVALID_ARG, "recent and sink must be >= 0");
     if (scope != LETHE_COLLAPSE_HEADS && scope != LETHE_COLLAPSE_HEADS_BATCH)
@@ -867,6 +896,7 @@ lethe_status lethe_prefill_seed(lethe_ctx* ctx, const lethe_cache* c, const void
                                 const float* scale, float gamma, void* stream) {
     lethe_status st = check_cache(ctx, c);
     if (st != LETHE_OK) return st;
+    ctx->last_len = nullptr;  // the next decode call does not follow a decode call
     if (!q_prompt || !scale) return fail(ctx, LETHE_ERR_INVALID_ARG, "q_prompt and scale are required");
     if (prompt_len < 1 || prompt_len > cap_tokens_of(c)) return fail(ctx, LETHE_ERR_INVALID_ARG, "prompt_len out of range");
     if (!(gamma > 0.f && gamma <= 1.f)) return fail(ctx, LETHE_ERR_INVALID_ARG, "gamma must be in (0, 1]");

@@ -49,6 +49,8 @@ struct AttendArgs {
     int chunk_tokens;          // logit-buffer capacity of one CTA, in tokens
     float gamma;
     int wait_limit;            // poll limit of the bounded mbarrier waits (0 = the kernel's default)
+    int early_prefetch;        // layer-pipelined clustered kernel: cached K / V tiles may be fetched before the previous
+                               // kernel of the stream has completed (it does not write this call's items)
     float scale_log2[kMaxLayers];  // scale[l] * log2(e) (times the key scale for a quantised cache), by absolute layer
     float k_scale[kMaxLayers];     // quantised caches: a stored key byte x means k_scale[l] * x (else unused)
     float v_scale[kMaxLayers];     // the same for values
@@ -171,6 +173,73 @@ __device__ __forceinline__ void prefetch_rel(const AttendArgs& a, const ItemCoor
     }
 }
 
+// Eq. 5 for the tokens [t0, hi_tok) of an item whose scaled logits (log2 units) are parked in `lg`:
+// rel[j] = gamma * rel[j] + sum over the group's heads of exp2(s_hj - m_h) / l_h, with fin[h] = (m_h, 1 / l_h) the
+// exact global statistics.  rel_old holds the values prefetch_rel loaded for the thread's first kRelPrefetch tokens;
+// with first_batch = kRelPrefetch those tokens are skipped and [t0, hi_tok) is a range that starts after them.
+template <int NT>
+__device__ __forceinline__ void relevance_update(const AttendArgs& a, const ItemCoord& ic, const float2* fin, const float* lg,
+                                                 int t0, int hi_tok, int append_slot, const float (&rel_old)[kRelPrefetch],
+                                                 int first_batch = 0) {
+    const int tid = threadIdx.x;
+    const int G = a.G;
+    float* rel = a.rel + (size_t)ic.item * a.cap_tokens;
+    const int GP = a.GP;
+    float fm[kMaxGroup], fi[kMaxGroup];
+#pragma unroll
+    for (int h = 0; h < kMaxGroup; ++h) {
+        fm[h] = fin[h].x;
+        fi[h] = fin[h].y;
+    }
+    // Rows are loaded a batch ahead of the stores to rel: the compiler cannot tell that rel and the logit buffer
+    // never alias, and would otherwise keep every token's loads behind the previous token's store.
+    auto load_row = [&](int j, float (&s)[kMaxGroup]) {
+        const float* row = lg + (size_t)(j - t0) * GP;
+#pragma unroll
+        for (int h = 0; h < kMaxGroup; ++h)
+            if (h < G) s[h] = row[h];
+    };
+    auto mass_from = [&](const float (&s)[kMaxGroup]) {
+        float mass = 0.f;
+#pragma unroll
+        for (int h = 0; h < kMaxGroup; ++h)
+            if (h < G) mass += fast_exp2(s[h] - fm[h]) * fi[h];
+        return mass;
+    };
+#pragma unroll
+    for (int i0 = 0; i0 < kRelPrefetch; i0 += kRelBatch) {
+        if (i0 < first_batch) continue;  // the caller has already updated the tokens rel_old was fetched for
+        float s[kRelBatch][kMaxGroup];
+#pragma unroll
+        for (int u = 0; u < kRelBatch; ++u) {
+            const int j = t0 + tid + (i0 + u) * NT;
+            if (j < hi_tok) load_row(j, s[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < kRelBatch; ++u) {
+            const int j = t0 + tid + (i0 + u) * NT;
+            if (j < hi_tok) rel[j] = fmaf(a.gamma, rel_old[i0 + u], mass_from(s[u]));
+        }
+    }
+    for (int j0 = t0 + tid + (first_batch ? 0 : kRelPrefetch * NT); j0 < hi_tok; j0 += kRelBatch * NT) {
+        float old[kRelBatch];
+        float s[kRelBatch][kMaxGroup];
+#pragma unroll
+        for (int u = 0; u < kRelBatch; ++u) {
+            const int j = j0 + u * NT;
+            if (j < hi_tok) {
+                old[u] = (j == append_slot) ? 0.f : rel[j];
+                load_row(j, s[u]);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kRelBatch; ++u) {
+            const int j = j0 + u * NT;
+            if (j < hi_tok) rel[j] = fmaf(a.gamma, old[u], mass_from(s[u]));
+        }
+    }
+}
+
 /*
  * Common tail of both attend kernels.  On entry every warp has written, for the tokens it streamed,
  *   es.wstat[w][h]   = (m, l): running max (log2 units) and sum of exp2(s - m) of head h
@@ -253,62 +322,7 @@ __device__ void combine_and_finish(const AttendArgs& a, const ItemCoord& ic, Epi
         }
     }
 
-    // Eq. 5: rel[j] = gamma * rel[j] + sum over the group's heads of p_hj, with the global (m, 1/l).
-    float* rel = a.rel + (size_t)ic.item * a.cap_tokens;
-    const int GP = a.GP;
-    const int hi_tok = min(t1, n);
-    float fm[kMaxGroup], fi[kMaxGroup];
-#pragma unroll
-    for (int h = 0; h < kMaxGroup; ++h) {
-        fm[h] = es.fin[h].x;
-        fi[h] = es.fin[h].y;
-    }
-    // Rows are loaded a batch ahead of the stores to rel: the compiler cannot tell that rel and the logit buffer
-    // never alias, and would otherwise keep every token's loads behind the previous token's store.
-    auto load_row = [&](int j, float (&s)[kMaxGroup]) {
-        const float* row = lg + (size_t)(j - t0) * GP;
-#pragma unroll
-        for (int h = 0; h < kMaxGroup; ++h)
-            if (h < G) s[h] = row[h];
-    };
-    auto mass_from = [&](const float (&s)[kMaxGroup]) {
-        float mass = 0.f;
-#pragma unroll
-        for (int h = 0; h < kMaxGroup; ++h)
-            if (h < G) mass += fast_exp2(s[h] - fm[h]) * fi[h];
-        return mass;
-    };
-#pragma unroll
-    for (int i0 = 0; i0 < kRelPrefetch; i0 += kRelBatch) {
-        float s[kRelBatch][kMaxGroup];
-#pragma unroll
-        for (int u = 0; u < kRelBatch; ++u) {
-            const int j = t0 + tid + (i0 + u) * NT;
-            if (j < hi_tok) load_row(j, s[u]);
-        }
-#pragma unroll
-        for (int u = 0; u < kRelBatch; ++u) {
-            const int j = t0 + tid + (i0 + u) * NT;
-            if (j < hi_tok) rel[j] = fmaf(a.gamma, rel_old[i0 + u], mass_from(s[u]));
-        }
-    }
-    for (int j0 = t0 + tid + kRelPrefetch * NT; j0 < hi_tok; j0 += kRelBatch * NT) {
-        float old[kRelBatch];
-        float s[kRelBatch][kMaxGroup];
-#pragma unroll
-        for (int u = 0; u < kRelBatch; ++u) {
-            const int j = j0 + u * NT;
-            if (j < hi_tok) {
-                old[u] = (j == append_slot) ? 0.f : rel[j];
-                load_row(j, s[u]);
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < kRelBatch; ++u) {
-            const int j = j0 + u * NT;
-            if (j < hi_tok) rel[j] = fmaf(a.gamma, old[u], mass_from(s[u]));
-        }
-    }
+    relevance_update<NT>(a, ic, es.fin, lg, t0, min(t1, n), append_slot, rel_old);
     if (S > 1) cg::this_cluster().sync();  // peers may still be reading this CTA's shared memory
     if (append_slot >= 0 && ic.rank == 0 && tid == 0) a.len[ic.item] = n;
 }

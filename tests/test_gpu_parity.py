@@ -94,6 +94,16 @@ CASES = [
     (torch.bfloat16, 128, 8, 1, 1000, 35, 16),
     (torch.bfloat16, 64, 16, 2, 500, 36, 1),
     (torch.bfloat16, 128, 6, 2, 300, 37, 7),
+    (torch.bfloat16, 128, 32, 8, 300, 44, 1),
+    (torch.bfloat16, 128, 32, 8, 300, 44, 2),
+    (torch.bfloat16, 128, 28, 4, 300, 44, 4),
+    (torch.bfloat16, 128, 28, 4, 700, 45, 1),
+    (torch.bfloat16, 128, 8, 1, 700, 45, 8),
+    (torch.bfloat16, 128, 6, 2, 1000, 45, 16),
+    (torch.bfloat16, 64, 8, 2, 300, 46, 2),
+    (torch.bfloat16, 64, 10, 2, 500, 47, 4),
+    (torch.bfloat16, 128, 32, 8, 300, 48, 0),
+    (torch.bfloat16, 64, 16, 2, 300, 49, 2),
     (torch.bfloat16, 128, 8, 8, 260, 0, 0),
     (torch.float32, 128, 16, 2, 260, 0, 0),
 ]
@@ -186,7 +196,7 @@ def test_empty_and_full_items(ctx):
     assert ctx.poll_status()[0] == 0                                     # the status word was cleared
 
 
-@pytest.mark.parametrize("variant", [1, 2, 9, 18, 26, 32])
+@pytest.mark.parametrize("variant", [1, 2, 9, 18, 26, 32, 44])
 def test_paged_decode_and_prune_parity(ctx, variant):
     """16-token pages behind a shuffled page table: decode steps and prune rounds, call by call."""
     w = synth.shrink(synth.WORKLOADS["ragged"], n_layers=2, batch=3, prompt_len=200)
@@ -198,7 +208,7 @@ def test_paged_decode_and_prune_parity(ctx, variant):
     gc = to_device(oc)
     scale = synth.layer_scales(w)
     T = torch.tensor([150 * 2, 90 * 2, 400 * 2], dtype=torch.int64)
-    ctx.set_tuning(variant, 2 if variant < 8 else (3 if variant >= 32 else 0))
+    ctx.set_tuning(variant, 2 if (variant < 8 or variant >= 44) else (3 if variant >= 32 else 0))
     try:
         for step in range(6):
             x = synth.step_inputs(w, step)
@@ -579,3 +589,48 @@ def test_ragged_sweep_ratios_shortest_and_longest(ctx, ratio):
                 assert torch.all(oc.len[:, 1].sum(0) == int(T[1]))      # every head of the long sequence holds its budgets
     finally:
         oracle.set_threads(1)
+
+
+@pytest.mark.parametrize("variant,splits", [(0, 0), (44, 4), (45, 2), (47, 1)])
+def test_layer_by_layer_launches_with_pipelining(ctx, variant, splits):
+    """The way a model issues the step: one launch per layer, with the layer pipelining on (a launch fetches cached
+    K / V tiles before the previous layer's launch has completed).  Several steps and a prune round in between; a
+    second context-free check: the same layer twice in a row must not take the early fetch (its own previous
+    launch appended to the same items), which the results would show as a stale length."""
+    w = synth.shrink(synth.WORKLOADS["llama8b"], n_layers=6, batch=3, prune_interval=4)
+    n0, cap = 333, 352
+    oc = cache_from_state(w, synth.initial_kv(w, n0, cap), cap)
+    oc.len[2, 1, 3] = 15; oc.len[4, 0, 0] = 1; oc.len[5, 2, 7] = 348
+    gc = to_device(oc)
+    dev = gc.device
+    scale = synth.layer_scales(w)
+    T = torch.full((3,), w.n_layers * 200, dtype=torch.int64)
+    ctx.set_tuning(variant, splits)
+    ctx.set_tuning(51, 0)
+    try:
+        for step in range(8):
+            x = synth.step_inputs(w, step)
+            s, o_out, _, _ = oracle.decode_attend(oc, 0, w.n_layers, x["q"], x["k_new"], x["v_new"], x["token_pos"], scale, w.gamma)
+            assert s == oracle.OK
+            out = torch.full_like(x["q"], float("nan"), device=dev)
+            q, kn, vn, tp = (x[k].to(dev) for k in ("q", "k_new", "v_new", "token_pos"))
+            for l in range(w.n_layers):                              # back to back, nothing in between
+                ctx.decode_attend(gc, l, l + 1, q[l:l + 1], kn[l:l + 1], vn[l:l + 1], tp, scale.tolist(), w.gamma, out[l:l + 1])
+            assert ctx.poll_status()[0] == 0
+            assert (out.cpu().double() - o_out.double()).abs().max() <= OUT_TOL[torch.bfloat16]
+            assert_state_matches(gc, oc)
+            if (step + 1) % w.prune_interval == 0:
+                _prune_both(ctx, oc, gc, T, w.k_min, w.recent, w.sink, cap)
+        # the same layer twice in a row: the second launch depends on the first one's append
+        for rep in range(2):
+            x = synth.step_inputs(w, 100 + rep)
+            s, o_out, _, _ = oracle.decode_attend(oc, 3, 4, x["q"][3:4], x["k_new"][3:4], x["v_new"][3:4], x["token_pos"], scale, w.gamma)
+            out = torch.zeros_like(x["q"][3:4], device=dev)
+            ctx.decode_attend(gc, 3, 4, x["q"][3:4].to(dev), x["k_new"][3:4].to(dev), x["v_new"][3:4].to(dev),
+                              x["token_pos"].to(dev), scale.tolist(), w.gamma, out)
+        assert ctx.poll_status()[0] == 0
+        assert (out.cpu().double() - o_out.double()).abs().max() <= OUT_TOL[torch.bfloat16]
+        assert_state_matches(gc, oc)
+    finally:
+        ctx.set_tuning(50, 0)
+        ctx.set_tuning(0, 0)
