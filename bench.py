@@ -208,6 +208,15 @@ class Runner:
         self.T = total_budget.to(torch.int64).to(device)
         self.step_no = 0
         self.launches = 0
+        self.epoch = 0                                   # anchor draw in force (drifting workloads)
+
+    def drift_if_due(self):
+        """Untimed harness work of a drifting workload: when the step counter has crossed a drift period, the anchor
+        set is re-drawn and the K rows whose flag changed are rescaled (rows are found through pos)."""
+        e = synth.drift_epoch(self.w, self.step_no)
+        if e != self.epoch and self.cache.page_table is None and self.cache.k.dtype == self.w.dtype:
+            synth.apply_drift(self.w, self.cache.k, self.cache.pos, self.batch_ids, self.epoch, e)
+        self.epoch = e
 
     def decode(self, host=False, append=True):
         w = self.w
@@ -303,6 +312,7 @@ def time_prune_rounds(r: Runner, rounds: int, bytes_per_th: int, attend_ms: floa
     row_bytes = bytes_per_th                              # a moved survivor: K row + V row + relevance 4 B + position 4 B
 
     def fill_interval():
+        r.drift_if_due()
         while True:
             r.decode()
             if r.prune_due():
@@ -729,6 +739,7 @@ def main():
             for _ in range(w.prune_interval):
                 r.decode()
             r.prune()
+            r.drift_if_due()
         r.check()
         return r, int(r.budgets.max().item())
 

@@ -42,7 +42,7 @@ class Workload:
     anchor_gain: float
     anchor_density: float = 0.01
     temp_range: Optional[tuple] = None   # per-layer attention temperature ~ U[a, b]
-    drift_period: int = 0                # re-draw anchors every this many positions (0 = never)
+    drift_period: int = 0                # re-draw the anchor set every this many decode steps (0 = never)
     page_tokens: int = 0                 # > 0: paged KV layout
 
     @property
@@ -111,11 +111,27 @@ def layer_anchor_density(w: Workload) -> torch.Tensor:
     return torch.full((w.n_layers,), w.anchor_density, dtype=torch.float64)
 
 
-def anchor_flags(w: Workload, positions: torch.Tensor, batch_ids: torch.Tensor) -> torch.Tensor:
-    """bool [L][len(batch_ids)][len(positions)]: is the token at an original position an anchor?
+def drift_epoch(w: Workload, step: int) -> int:
+    """Epoch of the anchor draw that is in force at decode step `step` (0 while the workload does not drift)."""
+    return step // w.drift_period if w.drift_period > 0 else 0
 
-    Counter-based (a hash of seed, layer or 0, sequence, position, drift epoch), so any position can be
-    queried on any device at any time with the same answer.
+
+def _anchor_hit(w: Workload, lay: torch.Tensor, bid: torch.Tensor, pos: torch.Tensor, epoch: int) -> torch.Tensor:
+    """Elementwise anchor test on broadcastable int64 tensors (layer, global sequence id, original position)."""
+    if w.anchor_rule == "per_seq":
+        lay = torch.zeros_like(lay)           # shared across layers
+    key = (w.seed + 1) * 1000003 + lay * 7368787 + bid * 15485863 + pos * 2654435761 + int(epoch) * 40503
+    u = (_mix64(key) & 0xFFFFFF).to(torch.float64) / float(1 << 24)
+    dens = layer_anchor_density(w).to(pos.device)
+    return u < dens[lay]
+
+
+def anchor_flags(w: Workload, positions: torch.Tensor, batch_ids: torch.Tensor, epoch: int = 0) -> torch.Tensor:
+    """bool [L][len(batch_ids)][len(positions)]: is the token at an original position an anchor during `epoch`?
+
+    Counter-based (a hash of seed, layer or 0, sequence, position, epoch), so any position can be queried on any
+    device at any time with the same answer.  A drifting workload re-draws the whole set every `drift_period`
+    decode steps: the draws of different epochs are independent, old tokens included.
     """
     dev = positions.device
     pos = positions.to(torch.int64)
@@ -126,15 +142,29 @@ def anchor_flags(w: Workload, positions: torch.Tensor, batch_ids: torch.Tensor) 
         chosen = torch.randperm(w.prompt_len, generator=g)[:16].to(dev)
         hit = (pos[:, None] == chosen[None, :]).any(dim=1)
         return hit[None, None, :].expand(L, bid.numel(), pos.numel()).clone()
-    epoch = (pos // w.drift_period) if w.drift_period > 0 else torch.zeros_like(pos)
     lay = torch.arange(L, device=dev, dtype=torch.int64)
-    if w.anchor_rule == "per_seq":
-        lay = torch.zeros_like(lay)           # shared across layers
-    key = (w.seed + 1) * 1000003 + lay[:, None, None] * 7368787 + bid[None, :, None] * 15485863 \
-        + pos[None, None, :] * 2654435761 + epoch[None, None, :] * 97
-    u = (_mix64(key) & 0xFFFFFF).to(torch.float64) / float(1 << 24)
-    dens = layer_anchor_density(w).to(dev)
-    return u < dens[:, None, None]
+    return _anchor_hit(w, lay[:, None, None], bid[None, :, None], pos[None, None, :], epoch)
+
+
+def apply_drift(w: Workload, k: torch.Tensor, pos: torch.Tensor, batch_ids: torch.Tensor, old_epoch: int,
+                new_epoch: int) -> None:
+    """Re-draw the anchors of a contiguous cache in place: K rows [L][B][Hkv][cap][D] of tokens that stop being
+    anchors are divided by the anchor gain, rows of tokens that become anchors are multiplied by it (fp32
+    arithmetic, one rounding to the cache dtype); `pos` [L][B][Hkv][cap] says which token sits in each slot.
+    Harness work between decode steps (an epoch boundary), not part of the method."""
+    if old_epoch == new_epoch or w.anchor_rule == "fixed16":
+        return
+    L, B = k.shape[0], k.shape[1]
+    lay = torch.arange(L, device=k.device, dtype=torch.int64)[:, None, None]
+    for b in range(B):
+        bid = batch_ids[b].to(torch.int64).to(k.device)
+        p = pos[:, b].to(torch.int64)                                       # [L][Hkv][cap]
+        f_old = _anchor_hit(w, lay, bid, p, old_epoch)
+        f_new = _anchor_hit(w, lay, bid, p, new_epoch)
+        factor = torch.ones(p.shape, dtype=torch.float32, device=k.device)
+        factor[f_new & ~f_old] = float(w.anchor_gain)
+        factor[f_old & ~f_new] = 1.0 / float(w.anchor_gain)
+        k[:, b] = (k[:, b].to(torch.float32) * factor[..., None]).to(k.dtype)
 
 
 def _randn(shape, g: torch.Generator, dtype: torch.dtype, device) -> torch.Tensor:
@@ -187,7 +217,7 @@ def step_inputs(w: Workload, step: int, device="cpu", batch_ids: Optional[torch.
     vn = _randn((L, B, H, D), g, w.dtype, device)
     p = w.prompt_len + step
     if w.anchor_rule != "fixed16":
-        fl = anchor_flags(w, torch.tensor([p], device=device), batch_ids)       # [L][B][1]
+        fl = anchor_flags(w, torch.tensor([p], device=device), batch_ids, drift_epoch(w, step))       # [L][B][1]
         kn = kn * torch.where(fl, w.anchor_gain, 1.0).to(torch.float32)[:, :, :, None]
     token_pos = torch.full((B,), p, dtype=torch.int32, device=device)
     return {"q": q.to(w.dtype), "k_new": kn.to(w.dtype), "v_new": vn.to(w.dtype), "token_pos": token_pos}

@@ -121,3 +121,42 @@ def test_paged_equals_contiguous():
         for ra_, rb_ in zip(logical(cc), logical(cp)):
             for u, v_ in zip(ra_, rb_):
                 assert torch.equal(u, v_)
+
+
+def test_long_reasoning_anchor_drift_is_a_real_redraw():
+    """The long-reasoning workload re-draws its anchor positions every 2048 decode steps: the sets of two epochs
+    are independent draws of the same density over ALL positions (old tokens included), the token generated at a
+    step is an anchor by the draw in force at that step, and re-drawing a cache rescales exactly the K rows whose
+    flag changed (by the anchor gain or its inverse), wherever pruning has moved them."""
+    from paper_2511_06029_b200 import synth
+    w = synth.shrink(synth.WORKLOADS["longreason"], n_layers=2, batch=3)
+    assert synth.drift_epoch(w, 0) == 0 and synth.drift_epoch(w, 2047) == 0 and synth.drift_epoch(w, 2048) == 1
+    pos = torch.arange(20000)
+    f0 = synth.anchor_flags(w, pos, torch.arange(3), 0)
+    f1 = synth.anchor_flags(w, pos, torch.arange(3), 1)
+    for f in (f0, f1):
+        assert 0.007 < f.float().mean() < 0.013                      # Bernoulli(1 %)
+    assert (f0 & f1).float().mean() < 0.0005                         # independent: overlap ~ 1e-4
+    assert torch.equal(f0[0], f0[1])                                 # shared across layers (per-sequence rule)
+    # a cache whose slots hold a shuffled subset of positions (as after pruning)
+    st = synth.initial_kv(w, 600, 608)
+    g = torch.Generator().manual_seed(3)
+    keep = torch.sort(torch.randperm(600, generator=g)[:200]).values
+    for key in ("k", "v"):
+        st[key][..., :200, :] = st[key][..., keep, :]
+    st["pos"][..., :200] = keep.to(torch.int32)
+    st["len"][:] = 200
+    k0 = st["k"].clone()
+    synth.apply_drift(w, st["k"], st["pos"], torch.arange(3), 0, 1)
+    ratio = (st["k"].float().norm(dim=-1) / k0.float().norm(dim=-1))[..., :200]
+    fl0 = synth.anchor_flags(w, keep, torch.arange(3), 0)[:, :, None, :].expand_as(ratio)
+    fl1 = synth.anchor_flags(w, keep, torch.arange(3), 1)[:, :, None, :].expand_as(ratio)
+    assert torch.allclose(ratio[fl1 & ~fl0], torch.tensor(3.0), rtol=2e-2)
+    assert torch.allclose(ratio[fl0 & ~fl1], torch.tensor(1 / 3.0), rtol=2e-2)
+    assert torch.equal(st["k"][..., :200, :][~(fl0 ^ fl1)], k0[..., :200, :][~(fl0 ^ fl1)])
+    # the generated token of step 2048 + 5 follows epoch 1
+    x = synth.step_inputs(w, 2053)
+    p = w.prompt_len + 2053
+    want = synth.anchor_flags(w, torch.tensor([p]), torch.arange(3), 1)[..., 0]            # [L][B]
+    big = x["k_new"].float().norm(dim=-1).mean(dim=-1) > 1.8 * (w.head_dim ** 0.5)          # anchor rows are x3
+    assert torch.equal(big, want)
