@@ -129,8 +129,11 @@ lethe_status lethe_poll_status(lethe_ctx *ctx, void *stream, int32_t *info);
  * Tensor-core variants need a bf16 cache (and 16-token pages when paged).
  * A quantised cache runs its own tensor-core kernels: variants 2..7 force the clustered one with
  * shape (4,4) (8,4) (4,2) (4,3) (2,4) (8,2) (splits as above), variants 8..13 the persistent one with shape (8,4)
- * (12,3) (10,4) (8,5) (16,2) (12,2) (e4m3 only); any other value means the clustered kernel with shape (4,4), the faster of
- * the two at every size measured.
+ * (12,3) (10,4) (8,5) (16,2) (12,2) (e4m3 only); variant 14 the tensor-memory kernel (tcgen05 kind::f8f6f4 MMAs on the
+ * cache's bytes with the query and the probabilities split into three e4m3 terms, K / V tiles by TMA, one CTA per SM;
+ * head_dim 128, splits 0 or 1, and a capacity whose logits fit on chip: 2 * (heads per KV head) * capacity * 4 bytes
+ * beside a 64 KB tile ring, else LETHE_ERR_UNSUPPORTED); any other value means the clustered kernel with shape
+ * (4,4), the fastest of the three at every size measured.
  * 44..49 = the clustered kernel's six shapes for launches of one layer at a time (few items per launch): the CTAs of
  * an item merge by one-sided pushes through distributed shared memory (no cluster barriers), and — when variant 51
  * is also set — a launch fetches cached K / V tiles while the previous launch is still finishing.

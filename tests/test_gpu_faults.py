@@ -90,6 +90,33 @@ def test_prefill_wait_runs_out_and_the_context_recovers(ctx, engine):
         ctx.set_tuning(40, 0)
 
 
+def test_quantised_tensor_memory_kernel_wait_runs_out(ctx):
+    """The tcgen05 kernel for byte caches: with a poll limit of one its first hand-off gives up; the CTAs wait for
+    the copies they started, free their tensor memory and return LETHE_ERR_TIMEOUT, and the same context then runs
+    the same launch correctly."""
+    from paper_2511_06029_b200 import binding
+    from test_gpu_fp8 import fp8_cache, _step
+    L, B, Hq, Hkv, D, cap = 2, 3, 16, 4, 128, 1600
+    oc = fp8_cache(L, B, Hq, Hkv, D, cap, 1500, seed=4, k_scale=[0.5, 0.7], v_scale=[0.9, 1.1])
+    broken, good = to_device(oc), to_device(oc)
+    g = torch.Generator().manual_seed(2)
+    q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+    kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+    scale = torch.tensor([0.09, 0.1])
+    ctx.set_tuning(14, 0)
+    try:
+        ctx.set_wait_limit(1)
+        out = torch.zeros_like(q, device="cuda")
+        ctx.decode_attend(broken, 0, L, q.cuda(), kn.cuda(), kn.cuda(), torch.zeros(B, dtype=torch.int32).cuda(), scale.tolist(), 0.95, out)
+        st, where = ctx.poll_status()
+        assert st == binding.ERR_TIMEOUT and 0 <= where < 148
+        ctx.set_wait_limit(0)
+        _step(ctx, oc, good, q, kn, kn, torch.zeros(B, dtype=torch.int32), scale, 0.95)
+    finally:
+        ctx.set_wait_limit(0)
+        ctx.set_tuning(0, 0)
+
+
 def _paged_state(lens_special=()):
     w = synth.shrink(synth.WORKLOADS["ragged"], n_layers=2, batch=2, prompt_len=400)
     cap = 416

@@ -240,3 +240,88 @@ def test_quantised_host_entry_point(ctx, pinned):
         assert bool((d <= 2e-2 + 2.0 ** -7 * ref.float().abs()).all()), f"attention output error {d.max().item()}"
         assert torch.allclose(lse, lse_ref, rtol=1e-4, atol=1e-4)
         assert_state_matches(gc, oc)
+
+
+TENSOR_MEMORY = 14                                                   # lethe_set_tuning code of the tcgen05 kernel
+
+
+@pytest.mark.parametrize("fmt", ["e4m3", "e5m2"])
+@pytest.mark.parametrize("paged", [False, True])
+@pytest.mark.parametrize("Hq,Hkv", [(8, 2), (7, 1), (16, 2), (5, 5), (24, 4)])
+def test_quantised_tensor_memory_kernel(ctx, Hq, Hkv, paged, fmt):
+    """The tcgen05 kernel (cache bytes straight into the MMAs, queries and probabilities as three e4m3 terms) on
+    G = 4, 7, 8, 1, 6: lengths around the 128-token tile (1, 127, 128, 129, 255, 256, 257), several tiles per item,
+    appending and attend-only steps, a new token beyond the representable range, an empty and a full item."""
+    L, B, D, cap = 2, 3, 128, 416
+    g = torch.Generator().manual_seed(Hq * 10 + paged)
+    lens = torch.randint(1, cap - 8, (L, B, Hkv), generator=g)
+    special = torch.tensor([1, 127, 128, 129, 255, 256, 257, 400])
+    lens.view(-1)[:min(8, lens.numel())] = special[:min(8, lens.numel())]
+    oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=Hq + 3, k_scale=[0.37, 1.5], v_scale=[2.25, 0.6],
+                   page_tokens=16 if paged else 0, fmt=fmt)
+    gc = to_device(oc)
+    scale = torch.tensor([0.11, 0.07], dtype=torch.float32)
+    ctx.set_tuning(TENSOR_MEMORY, 0)
+    try:
+        for step in range(5):
+            q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+            if step == 1:
+                _step(ctx, oc, gc, q, None, None, None, scale, 0.95, want_lse=True)
+                continue
+            kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            if step == 2:
+                big = 1e4 if fmt == "e4m3" else 1e6
+                kn[0, 0, 0, :3] = torch.tensor([big, -big, 165.5], dtype=torch.bfloat16)
+                vn[1, 1, 0, :2] = torch.tensor([-0.3 * big, 269.0], dtype=torch.bfloat16)
+            _step(ctx, oc, gc, q, kn, vn, torch.arange(B, dtype=torch.int32) + 300 + step, scale, 0.95, want_lse=(step == 3))
+        # an empty item (attend only) and a full one (append refused) in the same launches
+        oc.len[0, 1, 0] = 0; oc.len[1, 2, Hkv - 1] = cap
+        sync_state(gc, oc)
+        q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+        _step(ctx, oc, gc, q, None, None, None, scale, 0.95, want_lse=True)
+        kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16).cuda()
+        out = torch.full((L, B, Hq, D), 7.0, dtype=torch.bfloat16, device="cuda")
+        before = gc.k.clone()
+        ctx.decode_attend(gc, 0, L, q.cuda(), kn, kn, torch.zeros(B, dtype=torch.int32).cuda(), scale.tolist(), 0.95, out)
+        st, item = ctx.poll_status()
+        assert st == binding.ERR_CAPACITY and item == (1 * B + 2) * Hkv + Hkv - 1
+        assert int(gc.len[1, 2, Hkv - 1]) == cap and int(gc.len[0, 1, 0]) == 1
+        G = Hq // Hkv
+        assert torch.all(out[1, 2, (Hkv - 1) * G:] == 0) and torch.isfinite(out.float()).all()
+        if not paged:
+            assert torch.equal(gc.k[1, 2, Hkv - 1].view(torch.uint8), before[1, 2, Hkv - 1].view(torch.uint8))
+    finally:
+        ctx.set_tuning(0, 0)
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_quantised_tensor_memory_kernel_many_and_long_items(ctx, paged):
+    """More items than SMs (every CTA walks several through its queue and the ring runs across item boundaries),
+    with a few items of twenty tiles among short ones; uninitialised-looking bytes (NaN patterns) beyond the items'
+    ends must not leak into the results."""
+    L, B, Hq, Hkv, D, cap = 3, 9, 16, 8, 128, 2624
+    g = torch.Generator().manual_seed(17 + paged)
+    lens = torch.randint(1, 300, (L, B, Hkv), generator=g)
+    n_long = len(lens.view(-1)[::37])
+    lens.view(-1)[::37] = torch.randint(2000, cap - 8, (n_long,), generator=g)
+    oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=5, k_scale=[0.4, 0.6, 0.8], v_scale=[1.0, 0.5, 2.0],
+                   page_tokens=16 if paged else 0)
+    if not paged:                                                    # poison the rows beyond every item's end
+        idx = torch.arange(cap)[None, None, None, :] > lens[..., None] + 2
+        oc.k.view(torch.uint8)[idx] = 0x7F
+        oc.v.view(torch.uint8)[idx] = 0xFF
+    gc = to_device(oc)
+    scale = torch.tensor([0.1, 0.08, 0.12], dtype=torch.float32)
+    ctx.set_tuning(TENSOR_MEMORY, 0)
+    try:
+        for step in range(3):
+            q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+            if step == 1:
+                _step(ctx, oc, gc, q, None, None, None, scale, 0.97, want_lse=True)
+                continue
+            kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            _step(ctx, oc, gc, q, kn, vn, torch.arange(B, dtype=torch.int32) + 500 + step, scale, 0.97)
+    finally:
+        ctx.set_tuning(0, 0)
