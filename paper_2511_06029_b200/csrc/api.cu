@@ -14,10 +14,10 @@ size_t kv8_smem_bytes(int D, int shape, int chunk_tokens, int GP);
 size_t kv8_stream_smem_bytes(int D, int shape, int chunk_tokens, int GP);
 cudaError_t launch_attend_kv8_stream(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream);
 cudaError_t launch_attend_kv8(const AttendArgs& a, int D, int shape, bool paged, bool e5m2, cudaStream_t stream);
-size_t kv8_tc_smem_bytes(int nslot, int G, int cap_pad);
+size_t kv8_tc_smem_bytes(int nslot, int G, int cap_pad, int ng);
 size_t kv8_tc_maps_bytes();
 bool build_kv8_tc_maps(void* encode, void* k, void* v, unsigned long long rows, bool paged, void* out_maps);
-cudaError_t launch_attend_kv8_tc(const AttendArgs& a, const void* maps, bool paged, bool e5m2, int nslot, int cap_pad, int grid,
+cudaError_t launch_attend_kv8_tc(const AttendArgs& a, const void* maps, bool paged, bool e5m2, int ng, int nslot, int cap_pad, int grid,
                                  cudaStream_t stream);
 size_t simt_smem_bytes(int D, int chunk_tokens, int GP);
 cudaError_t launch_attend_mma(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream);
@@ -420,17 +420,20 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         // path (Llama-8B shape: 0.124 ms against 0.153 to 0.161 ms; a version of the asynchronous-epilogue kernel for
         // byte caches was measured too: 0.156 to 0.178 ms with two epilogue warps, 0.131 ms at best with four and the
         // batched relevance update (8 streaming warps x 2 stages), worse again with six; not kept).
-        // Tensor-memory kernel (variant 14 only): tcgen05 f8f6f4 MMAs on the cache's bytes, tiles by TMA, head_dim 128,
-        // the item's logits parked on chip.  Measured 0.145 ms on the same shape, so it is not the automatic choice.
-        const bool want_tc = variant == 14;
+        // Tensor-memory kernel (variant 14, and the automatic choice for launches with many items): tcgen05 f8f6f4 MMAs
+        // on the cache's bytes, tiles by TMA, head_dim 128, the item's logits parked on chip; 0.113 ms on the same
+        // shape (paged 0.131 against the clustered kernel's 0.146).  Falls back to the kernels below when the cache
+        // does not fit it.
+        const bool want_tc = variant == 14 || (variant == 0 && a.n_items >= 2 * ctx->sm_count && ctx->splits <= 1);
         if (want_tc && c->head_dim == 128 && resolve_tma_encode(ctx) && sizeof(ctx->kv8_maps) >= kv8_tc_maps_bytes()) {
             const int cap_pad = ((a.cap_tokens + 127) / 128) * 128;
-            int nslot = 8;  // the deepest ring that fits beside the two groups' logit buffers
-            while (nslot > 4 && kv8_tc_smem_bytes(nslot, G, cap_pad) > ctx->max_smem) --nslot;
+            const int ng = 2;  // softmax groups
+            int nslot = 8;     // the deepest rings (K and V: half each) that fit beside the groups' logit buffers
+            while (nslot > 4 && kv8_tc_smem_bytes(nslot, G, cap_pad, ng) > ctx->max_smem) --nslot;
             const int per_sm = 1;
             const unsigned long long rows = paged ? (unsigned long long)c->n_pages * c->page_tokens
                                                   : (unsigned long long)c->n_layers * c->batch * c->n_kv_heads * c->capacity;
-            if (kv8_tc_smem_bytes(nslot, G, cap_pad) <= ctx->max_smem && rows <= 0x7fffffffULL) {
+            if (kv8_tc_smem_bytes(nslot, G, cap_pad, ng) <= ctx->max_smem && rows <= 0x7fffffffULL) {
                 if (ctx->kv8_k != c->k || ctx->kv8_v != c->v || ctx->kv8_rows != rows || ctx->kv8_paged != (int)paged) {
                     if (!build_kv8_tc_maps(ctx->tma_encode, c->k, c->v, rows, paged, ctx->kv8_maps))
                         return fail(ctx, LETHE_ERR_CUDA, "cuTensorMapEncodeTiled failed");
@@ -438,7 +441,7 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
                 }
                 a.splits = 1;
                 const int grid = a.n_items < per_sm * ctx->sm_count ? a.n_items : per_sm * ctx->sm_count;
-                const cudaError_t et = launch_attend_kv8_tc(a, ctx->kv8_maps, paged, c->dtype == LETHE_FP8_E5M2, nslot, cap_pad, grid,
+                const cudaError_t et = launch_attend_kv8_tc(a, ctx->kv8_maps, paged, c->dtype == LETHE_FP8_E5M2, ng, nslot, cap_pad, grid,
                                                             (cudaStream_t)stream);
                 if (et != cudaSuccess) return cuda_fail(ctx, et, "decode_attend launch (quantised cache, tensor memory)");
                 return LETHE_OK;
