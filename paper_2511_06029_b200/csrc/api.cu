@@ -621,9 +621,13 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         if (S == 0) {
             S = 1;
             while (S < 16 && smem_for(S) > ctx->max_smem) S *= 2;
-            // enough CTAs to cover the SMs once; larger clusters cost more in scheduling and barriers than they
-            // gain (measured: 64 items run best as 4-CTA clusters)
-            while (S < 8 && (long long)a.n_items * S < ctx->sm_count && cap_groups / (2 * S) >= 4) S *= 2;
+            // enough CTAs to cover the SMs once, and 4-CTA clusters while the items are fewer than the SMs; larger
+            // clusters cost more in scheduling and merging than they gain (measured on ~1100-token items, per 32-layer
+            // step: 64 items per launch 0.317 ms with 4 CTAs per item against 0.394 with 2; 128 items 0.317 against
+            // 0.398; 256 items 0.310 with 1 against 0.318 with 4)
+            while (S < 8 && ((long long)a.n_items * S < ctx->sm_count || (a.n_items <= ctx->sm_count && S < 4)) &&
+                   cap_groups / (2 * S) >= 4)
+                S *= 2;
         }
         if (smem_for(S) > ctx->max_smem)
             return fail(ctx, LETHE_ERR_UNSUPPORTED, "capacity too large for the on-chip logit buffer at this split count");
