@@ -51,6 +51,7 @@ NCU_TRAFFIC = {
     "qwen7b": (520.1, "profiles/attend_stream_w8s2_qwen7b.md"),
     "longreason": (519.4, "profiles/attend_async_spill_w8s2_longreason.md"),
     "ragged": (520.4, "profiles/attend_stream_paged_w8s2_ragged.md"),
+    "llama8b:fp8": (288.7, "profiles/attend_kv8_tc_llama8b.md"),
 }
 RAGGED_RESIDENT_LAYERS = 7           # of 28: the full ragged state is 124 GB of K/V; one layer group is resident at a time
 SWEEP_RATIOS = (0.05, 0.1, 0.25, 0.5)
@@ -880,13 +881,13 @@ def main():
         B_r = w.batch
         h2d = (w.n_layers * B_r * (w.n_q_heads + 2 * w.n_kv_heads) * w.head_dim * 2 + B_r * 4)
         d2h = w.n_layers * B_r * w.n_q_heads * w.head_dim * 2
-        traffic = NCU_TRAFFIC.get(args.workload) if (args.kv == "bf16" and args.variant == 0) else None
+        traffic = NCU_TRAFFIC.get(args.workload if args.kv == "bf16" else f"{args.workload}:{args.kv}") if args.variant == 0 else None
         line = {
             "metric": METRIC, "value": dist_util.job_value(units, t_ms), "unit": UNIT, "n_gpus": n_ranks, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": t_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if args.kv == "bf16" else
-                     f"fp8 K/V ({'e4m3' if args.kv == 'fp8' else 'e5m2'} bytes, per-layer scales), bf16 activations, f16 mma, fp32 accumulation",
+                     f"fp8 K/V ({'e4m3' if args.kv == 'fp8' else 'e5m2'} bytes, per-layer scales), bf16 activations, 8-bit tensor-core products (queries and probabilities as three e4m3 terms), fp32 accumulation",
             "data": "synthetic",
             "config": workload_config(w, args, n_ranks, extra={
                 "resident_layers": w.n_layers if w.page_tokens else None,
