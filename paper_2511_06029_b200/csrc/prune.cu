@@ -256,62 +256,94 @@ __device__ __forceinline__ int sweep_keep(PruneShared& sh, KeyAt key_at, int n, 
 
 // Rows of K, V, rel, pos move to their destinations in ascending waves: load wave -> barrier -> store wave.
 // Because a survivor's destination never exceeds its source and waves ascend, no unread source is overwritten.
+// The loads of wave w + 1 are issued before the stores of wave w (its sources lie above every destination of wave
+// w, so the order between them is free): reads and writes then overlap instead of alternating, which matters
+// most where only one CTA fits an SM (long items).
+template <int RPT_>
+struct MoveWave {
+    static constexpr int RPT = RPT_;  // rows each thread slot carries per wave
+    uint4 kv[RPT], vv[RPT];
+    float rv[RPT];
+    int pv[RPT], srcs[RPT];
+};
+template <int RPT>
+__device__ __forceinline__ void move_wave_load(const CacheView& c, size_t item, int keep_n, const int32_t* src_list, int w0, int slots,
+                                               int rslot, int piece, int row_bytes, const float* rel, const int32_t* pos,
+                                               MoveWave<RPT>& w, bool& bad) {
+#pragma unroll
+    for (int r = 0; r < RPT; ++r) {
+        const int dst = w0 + r * slots + rslot;
+        int src = -1;
+        if (dst < keep_n) src = src_list[dst];
+        // destinations whose source is themselves (the unmoved prefix, and any later fixed point) are skipped
+        w.srcs[r] = (src >= 0 && src != dst) ? src : -1;
+        w.kv[r] = make_uint4(0, 0, 0, 0);
+        w.vv[r] = make_uint4(0, 0, 0, 0);
+        w.rv[r] = 0.f;
+        w.pv[r] = 0;
+        if (w.srcs[r] >= 0) {
+            const char* ks = prune_row_ptr(c, c.k, item, w.srcs[r], row_bytes, &bad);
+            const char* vs = prune_row_ptr(c, c.v, item, w.srcs[r], row_bytes, &bad);
+            if (ks && vs) {
+                w.kv[r] = *reinterpret_cast<const uint4*>(ks + piece * 16);
+                w.vv[r] = *reinterpret_cast<const uint4*>(vs + piece * 16);
+            }
+            if (piece == 0) {
+                w.rv[r] = rel[w.srcs[r]];
+                w.pv[r] = pos[w.srcs[r]];
+            }
+        }
+    }
+}
+template <int RPT>
+__device__ __forceinline__ void move_wave_store(const CacheView& c, size_t item, int w0, int slots, int rslot, int piece, int row_bytes,
+                                                float* rel, int32_t* pos, const MoveWave<RPT>& w, bool& bad) {
+#pragma unroll
+    for (int r = 0; r < RPT; ++r) {
+        if (w.srcs[r] >= 0) {
+            const int dst = w0 + r * slots + rslot;
+            char* kd = prune_row_ptr(c, c.k, item, dst, row_bytes, &bad);
+            char* vd = prune_row_ptr(c, c.v, item, dst, row_bytes, &bad);
+            if (kd && vd) {
+                *reinterpret_cast<uint4*>(kd + piece * 16) = w.kv[r];
+                *reinterpret_cast<uint4*>(vd + piece * 16) = w.vv[r];
+            }
+            if (piece == 0) {
+                rel[dst] = w.rv[r];
+                pos[dst] = w.pv[r];
+            }
+        }
+    }
+}
+template <int RPT, bool PIPELINED>
 __device__ __forceinline__ void move_rows(const CacheView& c, size_t item, int keep_n, const int32_t* src_list, bool& bad) {
     const int tid = threadIdx.x;
     float* rel = c.rel + item * c.cap_tokens;
     int32_t* pos = c.pos + item * c.cap_tokens;
     const int row_bytes = c.D * c.elt_bytes;
     const int lanes_per_row = row_bytes / 16;            // 16-byte pieces per row (8, 16 or 32)
-    constexpr int RPT = 4;                               // rows each thread slot carries per wave
     const int slots = kPruneThreads / lanes_per_row;     // row slots per pass
     const int rows_per_wave = slots * RPT;
     const int piece = tid % lanes_per_row, rslot = tid / lanes_per_row;
-    // destinations whose source is themselves (the unmoved prefix, and any later fixed point) are skipped
+    if (keep_n <= 0) return;
+    if (!PIPELINED) {  // two CTAs share the SM and cover each other's barriers: one wave in registers at a time
+        for (int w0 = 0; w0 < keep_n; w0 += rows_per_wave) {
+            MoveWave<RPT> cur;
+            move_wave_load(c, item, keep_n, src_list, w0, slots, rslot, piece, row_bytes, rel, pos, cur, bad);
+            __syncthreads();  // every source row of this wave has been read
+            move_wave_store(c, item, w0, slots, rslot, piece, row_bytes, rel, pos, cur, bad);
+            // no barrier needed here: the next wave's sources lie above every destination written so far
+        }
+        return;
+    }
+    MoveWave<RPT> cur, nxt;
+    move_wave_load(c, item, keep_n, src_list, 0, slots, rslot, piece, row_bytes, rel, pos, cur, bad);
     for (int w0 = 0; w0 < keep_n; w0 += rows_per_wave) {
-        uint4 kv[RPT], vv[RPT];
-        float rv[RPT];
-        int pv[RPT], srcs[RPT];
-#pragma unroll
-        for (int r = 0; r < RPT; ++r) {
-            const int dst = w0 + r * slots + rslot;
-            int src = -1;
-            if (dst < keep_n) src = src_list[dst];
-            srcs[r] = (src >= 0 && src != dst) ? src : -1;
-            kv[r] = make_uint4(0, 0, 0, 0);
-            vv[r] = make_uint4(0, 0, 0, 0);
-            rv[r] = 0.f;
-            pv[r] = 0;
-            if (srcs[r] >= 0) {
-                const char* ks = prune_row_ptr(c, c.k, item, srcs[r], row_bytes, &bad);
-                const char* vs = prune_row_ptr(c, c.v, item, srcs[r], row_bytes, &bad);
-                if (ks && vs) {
-                    kv[r] = *reinterpret_cast<const uint4*>(ks + piece * 16);
-                    vv[r] = *reinterpret_cast<const uint4*>(vs + piece * 16);
-                }
-                if (piece == 0) {
-                    rv[r] = rel[srcs[r]];
-                    pv[r] = pos[srcs[r]];
-                }
-            }
-        }
-        __syncthreads();  // every source row of this wave has been read
-#pragma unroll
-        for (int r = 0; r < RPT; ++r) {
-            if (srcs[r] >= 0) {
-                const int dst = w0 + r * slots + rslot;
-                char* kd = prune_row_ptr(c, c.k, item, dst, row_bytes, &bad);
-                char* vd = prune_row_ptr(c, c.v, item, dst, row_bytes, &bad);
-                if (kd && vd) {
-                    *reinterpret_cast<uint4*>(kd + piece * 16) = kv[r];
-                    *reinterpret_cast<uint4*>(vd + piece * 16) = vv[r];
-                }
-                if (piece == 0) {
-                    rel[dst] = rv[r];
-                    pos[dst] = pv[r];
-                }
-            }
-        }
-        // no barrier needed here: the next wave's sources lie above every destination written so far
+        __syncthreads();  // every source row of wave w0 has been read by every thread
+        const bool more = w0 + rows_per_wave < keep_n;
+        if (more) move_wave_load(c, item, keep_n, src_list, w0 + rows_per_wave, slots, rslot, piece, row_bytes, rel, pos, nxt, bad);
+        move_wave_store(c, item, w0, slots, rslot, piece, row_bytes, rel, pos, cur, bad);
+        if (more) cur = nxt;
     }
 }
 
@@ -323,7 +355,10 @@ __device__ __forceinline__ void move_rows(const CacheView& c, size_t item, int k
  *     global scratch for items longer than smem_tokens).
  *  4. rows move in ascending waves.
  */
-__global__ void __launch_bounds__(kPruneThreads, 2) rasr_prune_kernel(CacheView c, const int32_t* __restrict__ budgets,
+// DEEP: the item's keys take more shared memory than half an SM has, so one CTA has the SM (and its registers) to
+// itself and keeps two waves of rows in registers (the next wave's loads overlap this wave's stores).
+template <bool DEEP>
+__global__ void __launch_bounds__(kPruneThreads, DEEP ? 1 : 2) rasr_prune_kernel(CacheView c, const int32_t* __restrict__ budgets,
                                                                    int recent, int sink, int32_t* keep_idx, int max_k,
                                                                    int smem_tokens, int32_t* list_scratch,
                                                                    int32_t* status) {
@@ -367,7 +402,7 @@ __global__ void __launch_bounds__(kPruneThreads, 2) rasr_prune_kernel(CacheView 
     int32_t* src_list = in_smem ? reinterpret_cast<int32_t*>(dyn) : list_scratch + item * c.cap_tokens;
     const int keep_n = sweep_keep(sh, key_at, n, cand_lo, cand_hi, cand_lo, cand_hi, take > 0, T, need_eq, src_list, kout, max_k);
     bool bad = false;
-    move_rows(c, item, keep_n, src_list, bad);
+    move_rows<4, DEEP>(c, item, keep_n, src_list, bad);
     // any thread may have met the bad page id (each carries its own row slots): reduce over the CTA
     if (__syncthreads_or(bad) && tid == 0) record_error(status, LETHE_ERR_PAGE, (int)item);
     if (tid == 0) c.len[item] = keep_n;
@@ -442,7 +477,7 @@ __global__ void __launch_bounds__(kPruneThreads, 2) segment_prune_kernel(CacheVi
     const int keep_n = sweep_keep(sh, key_at, n, min(sink, n), max(n - recent, 0), 0, n, breakpoint > 0, T, need_eq, src_list,
                                   kout, max_k);
     bool bad = false;
-    move_rows(c, item, keep_n, src_list, bad);
+    move_rows<4, false>(c, item, keep_n, src_list, bad);
     if (__syncthreads_or(bad) && tid == 0) record_error(status, LETHE_ERR_PAGE, (int)item);
     if (tid == 0) {
         c.len[item] = keep_n;
@@ -466,10 +501,15 @@ cudaError_t launch_rasr_prune(const CacheView& c, const int32_t* budgets, int re
                               int max_k, int smem_tokens, int32_t* list_scratch, int32_t* status,
                               cudaStream_t stream) {
     const size_t smem = (size_t)smem_tokens * 4;
-    cudaError_t e = prepare_kernel((const void*)rasr_prune_kernel, smem);
+    const bool deep = smem > 100 * 1024;  // two CTAs of that size do not fit an SM
+    cudaError_t e = prepare_kernel(deep ? (const void*)rasr_prune_kernel<true> : (const void*)rasr_prune_kernel<false>, smem);
     if (e != cudaSuccess) return e;
-    rasr_prune_kernel<<<c.L * c.B * c.Hkv, kPruneThreads, smem, stream>>>(c, budgets, recent, sink, keep_idx, max_k,
-                                                                         smem_tokens, list_scratch, status);
+    if (deep)
+        rasr_prune_kernel<true><<<c.L * c.B * c.Hkv, kPruneThreads, smem, stream>>>(c, budgets, recent, sink, keep_idx, max_k,
+                                                                                   smem_tokens, list_scratch, status);
+    else
+        rasr_prune_kernel<false><<<c.L * c.B * c.Hkv, kPruneThreads, smem, stream>>>(c, budgets, recent, sink, keep_idx, max_k,
+                                                                                    smem_tokens, list_scratch, status);
     return cudaGetLastError();
 }
 
@@ -556,7 +596,7 @@ __global__ void __launch_bounds__(kPruneThreads, 2) collapsed_move_kernel(CacheV
     const int keep_n = plan[group];
     if (keep_n < 0) return;
     bool bad = false;
-    move_rows(c, item, keep_n, lists + group * c.cap_tokens, bad);
+    move_rows<4, false>(c, item, keep_n, lists + group * c.cap_tokens, bad);
     if (__syncthreads_or(bad) && threadIdx.x == 0) record_error(status, LETHE_ERR_PAGE, (int)item);
     if (threadIdx.x == 0) c.len[item] = keep_n;
 }
@@ -685,7 +725,7 @@ extern "C" lethe_status lethe_rasr_prune_static(const lethe_cache* c, const int3
     cudaStream_t s = (cudaStream_t)stream;
     if (cudaMemsetAsync(status, 0, 2 * sizeof(int32_t), s) != cudaSuccess) return LETHE_ERR_CUDA;
     // smem_tokens = 0: every item keeps its source list in the global scratch and re-reads its keys from rel
-    rasr_prune_kernel<<<(unsigned)items, kPruneThreads, 0, s>>>(v, budgets, recent, sink, keep_idx, keep_idx ? max_k : 0,
+    rasr_prune_kernel<false><<<(unsigned)items, kPruneThreads, 0, s>>>(v, budgets, recent, sink, keep_idx, keep_idx ? max_k : 0,
                                                                0, lists, status);
     if (cudaGetLastError() != cudaSuccess) return LETHE_ERR_CUDA;
     if (status_out &&
