@@ -325,3 +325,32 @@ def test_quantised_tensor_memory_kernel_many_and_long_items(ctx, paged):
             _step(ctx, oc, gc, q, kn, vn, torch.arange(B, dtype=torch.int32) + 500 + step, scale, 0.97)
     finally:
         ctx.set_tuning(0, 0)
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_quantised_automatic_choice_many_items(ctx, paged):
+    """No tuning set: a launch with more than two items per SM takes the library's automatic choice for quantised
+    caches.  Every item spans three or four tiles, so each CTA streams multi-tile items back to back; two prune
+    rounds in between change the lengths (and the work-queue order) under the kernel."""
+    L, B, Hq, Hkv, D, cap = 5, 8, 32, 8, 128, 512
+    assert L * B * Hkv >= 2 * torch.cuda.get_device_properties(0).multi_processor_count
+    g = torch.Generator().manual_seed(41 + paged)
+    lens = torch.randint(290, 440, (L, B, Hkv), generator=g)
+    oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=11, k_scale=[0.4, 0.6, 0.8, 0.5, 1.0], v_scale=[1.0, 0.5, 2.0, 0.7, 0.9],
+                   page_tokens=16 if paged else 0)
+    oc.rel.zero_()
+    gc = to_device(oc)
+    scale = torch.tensor([0.1, 0.08, 0.12, 0.09, 0.1], dtype=torch.float32)
+    ctx.set_tuning(0, 0)
+    for step in range(6):
+        q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+        kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+        vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+        _step(ctx, oc, gc, q, kn, vn, torch.arange(B, dtype=torch.int32) + 700 + step, scale, 0.97, want_lse=(step == 4))
+        if step in (1, 3):                                           # prune on the oracle's scores, as the parity bar prescribes
+            gc.rel.copy_(oc.rel)
+            budgets = torch.full((L, B), 200 + 40 * step, dtype=torch.int32)
+            st_o, _ = oracle.rasr_prune(oc, budgets, 16, 4)
+            ctx.rasr_prune(gc, budgets.cuda(), 16, 4)
+            assert st_o == oracle.OK and ctx.poll_status()[0] == 0
+            assert_state_matches(gc, oc, exact_rel=True)
