@@ -28,7 +28,8 @@
 //   warp 12    the same for the V tiles, into a ring of their own;
 //   warp 9     one lane issues the logit MMAs (K tiles); the warp owns the tensor-memory allocation;
 //   warp 10    one lane issues the output MMAs (V tiles);
-//   warps 0-.. NG (two or three) groups of four; group g owns items g, g + NG, ... of the CTA's sequence, start to finish (thread =
+//   warps 0-7  NG = 2 softmax groups of four (with three, the role warps follow at 12: measured, no gain, not instantiated);
+//              group g owns items g, g + NG, ... of the CTA's sequence, start to finish (thread =
 //              token in phase 1, thread = (head, four tokens) in phase 2, thread = dimension for the output rows).
 // The K stream runs about an item ahead of the V stream, so the groups are in different phases: while one
 // computes probabilities and finishes its item, the other parks the next item's logits, and the streams from HBM
