@@ -629,6 +629,14 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
                    cap_groups / (2 * S) >= 4)
                 S *= 2;
         }
+        if (ctx->variant == 0 && variant == 44) {
+            // automatic choice of the layer kernel's shape: two CTAs per SM matter more than a third pipeline stage
+            // (wide groups with long chunks, e.g. G = 7 at capacity 5312: 36 us per 128-item launch with two stages
+            // against 47 us with three, where only one CTA fits)
+            const int chunk = ((cap_groups + S - 1) / S) * kGroupTokens;
+            auto two_fit = [&](int shape) { return 2 * (layer_smem_bytes(c->head_dim, shape, chunk, a.GP) + 1024) <= 228 * 1024; };
+            if (!two_fit(0) && two_fit(2)) variant = 46;
+        }
         if (smem_for(S) > ctx->max_smem)
             return fail(ctx, LETHE_ERR_UNSUPPORTED, "capacity too large for the on-chip logit buffer at this split count");
         a.splits = S;
