@@ -354,3 +354,27 @@ def test_quantised_automatic_choice_many_items(ctx, paged):
             ctx.rasr_prune(gc, budgets.cuda(), 16, 4)
             assert st_o == oracle.OK and ctx.poll_status()[0] == 0
             assert_state_matches(gc, oc, exact_rel=True)
+
+
+def test_quantised_automatic_choice_large_capacity(ctx):
+    """No tuning set, many items, eight query heads per KV head and a capacity whose logits do not fit the
+    tensor-memory kernel's on-chip buffers: the automatic choice has to fall back to a kernel that holds (or
+    overflows) them, with the same results.  A few items are nearly as long as the capacity."""
+    L, B, Hq, Hkv, D, cap = 5, 8, 64, 8, 128, 2560
+    assert L * B * Hkv >= 2 * torch.cuda.get_device_properties(0).multi_processor_count
+    g = torch.Generator().manual_seed(77)
+    lens = torch.randint(1, 200, (L, B, Hkv), generator=g)
+    n_long = len(lens.view(-1)[::53])
+    lens.view(-1)[::53] = torch.randint(2300, cap - 8, (n_long,), generator=g)
+    oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=13, k_scale=[0.4, 0.6, 0.8, 0.5, 1.0], v_scale=[1.0, 0.5, 2.0, 0.7, 0.9])
+    gc = to_device(oc)
+    scale = torch.tensor([0.1, 0.08, 0.12, 0.09, 0.1], dtype=torch.float32)
+    ctx.set_tuning(0, 0)
+    for step in range(3):
+        q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+        if step == 1:
+            _step(ctx, oc, gc, q, None, None, None, scale, 0.97, want_lse=True)
+            continue
+        kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+        vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+        _step(ctx, oc, gc, q, kn, vn, torch.arange(B, dtype=torch.int32) + 900 + step, scale, 0.97)
