@@ -228,7 +228,9 @@ __device__ __forceinline__ uint32_t sw128_at(uint32_t base, int row, int col) {
     return base + row * 128 + ((((col >> 4) ^ (row & 7)) << 4) | (col & 15));
 }
 
-template <int NP, bool PAGED, bool E5M2, int NG>
+// GT: the number of query heads per KV head when it is known at compile time (the loops over heads then carry no
+// run-time bounds), 0 = read it from the arguments.
+template <int NP, bool PAGED, bool E5M2, int NG, int GT>
 __global__ void __launch_bounds__((4 * NG + kRoleWarps) * 32, 1)
     attend_kv8_tc_kernel(const __grid_constant__ AttendArgs a, const __grid_constant__ Kv8Maps maps, int nslot, int cap_pad) {
     using T = __nv_bfloat16;
@@ -248,7 +250,7 @@ __global__ void __launch_bounds__((4 * NG + kRoleWarps) * 32, 1)
     Kv8Header& hd = *reinterpret_cast<Kv8Header*>(reinterpret_cast<unsigned char*>(park_all) + (size_t)NG * a.G * cap_pad * 4);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int G = a.G;
+    const int G = GT ? GT : a.G;
     const bool append = a.k_new != nullptr;
     volatile int* abort_flag = &hd.abort;
     const int wait_limit = a.wait_limit > 0 ? a.wait_limit : kTc8WaitLimit;
@@ -794,9 +796,9 @@ bool build_kv8_tc_maps(void* encode, void* k, void* v, unsigned long long rows, 
     return r1 == CUDA_SUCCESS && r2 == CUDA_SUCCESS && r3 == CUDA_SUCCESS && r4 == CUDA_SUCCESS;
 }
 
-template <int NP, bool PAGED, bool E5M2, int NG>
+template <int NP, bool PAGED, bool E5M2, int NG, int GT>
 static cudaError_t launch_kv8_tc_t(const AttendArgs& a, const Kv8Maps& maps, int nslot, int cap_pad, int grid, cudaStream_t stream) {
-    auto kern = attend_kv8_tc_kernel<NP, PAGED, E5M2, NG>;
+    auto kern = attend_kv8_tc_kernel<NP, PAGED, E5M2, NG, GT>;
     const size_t smem = kv8_tc_smem_bytes(nslot, a.G, cap_pad, NG);
     cudaError_t e = prepare_kernel((const void*)kern, smem);
     if (e != cudaSuccess) return e;
@@ -819,14 +821,14 @@ cudaError_t launch_attend_kv8_tc(const AttendArgs& a, const void* maps_raw, bool
     Kv8Maps maps;
     memcpy(&maps, maps_raw, sizeof(maps));
     const bool wide = 3 * a.G > 16;
-#define LETHE_KV8TC2(NP, NG)                                                                                          \
-    (paged ? (e5m2 ? launch_kv8_tc_t<NP, true, true, NG>(a, maps, nslot, cap_pad, grid, stream)                        \
-                   : launch_kv8_tc_t<NP, true, false, NG>(a, maps, nslot, cap_pad, grid, stream))                      \
-           : (e5m2 ? launch_kv8_tc_t<NP, false, true, NG>(a, maps, nslot, cap_pad, grid, stream)                       \
-                   : launch_kv8_tc_t<NP, false, false, NG>(a, maps, nslot, cap_pad, grid, stream)))
-#define LETHE_KV8TC(NP) LETHE_KV8TC2(NP, 2)  // (three groups: built and measured, 0.1137 ms against 0.1130 ms with two on the Llama-8B shape; not instantiated)
-    return wide ? LETHE_KV8TC(32) : LETHE_KV8TC(16);
-#undef LETHE_KV8TC
+#define LETHE_KV8TC2(NP, NG, GT)                                                                                      \
+    (paged ? (e5m2 ? launch_kv8_tc_t<NP, true, true, NG, GT>(a, maps, nslot, cap_pad, grid, stream)                    \
+                   : launch_kv8_tc_t<NP, true, false, NG, GT>(a, maps, nslot, cap_pad, grid, stream))                  \
+           : (e5m2 ? launch_kv8_tc_t<NP, false, true, NG, GT>(a, maps, nslot, cap_pad, grid, stream)                   \
+                   : launch_kv8_tc_t<NP, false, false, NG, GT>(a, maps, nslot, cap_pad, grid, stream)))
+    // (three groups: built and measured, 0.1137 ms against 0.1130 ms with two on the Llama-8B shape; not instantiated)
+    if (a.G == 4) return LETHE_KV8TC2(16, 2, 4);
+    return wide ? LETHE_KV8TC2(32, 2, 0) : LETHE_KV8TC2(16, 2, 0);
 #undef LETHE_KV8TC2
 }
 
