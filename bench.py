@@ -51,7 +51,7 @@ NCU_TRAFFIC = {
     "qwen7b": (520.1, "profiles/attend_stream_w8s2_qwen7b.md"),
     "longreason": (519.4, "profiles/attend_async_spill_w8s2_longreason.md"),
     "ragged": (520.4, "profiles/attend_stream_paged_w8s2_ragged.md"),
-    "llama8b:fp8": (269.5, "profiles/attend_kv8_tc_llama8b.md"),
+    "llama8b:fp8": (267.5, "profiles/attend_kv8_tc_llama8b.md"),
 }
 RAGGED_RESIDENT_LAYERS = 7           # of 28: the full ragged state is 124 GB of K/V; one layer group is resident at a time
 SWEEP_RATIOS = (0.05, 0.1, 0.25, 0.5)

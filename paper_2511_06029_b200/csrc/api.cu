@@ -421,8 +421,8 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         // byte caches was measured too: 0.156 to 0.178 ms with two epilogue warps, 0.131 ms at best with four and the
         // batched relevance update (8 streaming warps x 2 stages), worse again with six; not kept).
         // Tensor-memory kernel (variant 14, and the automatic choice for launches with many items): tcgen05 f8f6f4 MMAs
-        // on the cache's bytes, tiles by TMA, head_dim 128, the item's logits parked on chip; 0.111 ms on the same
-        // shape (paged 0.131 against the clustered kernel's 0.146).  Falls back to the kernels below when the cache
+        // on the cache's bytes, tiles by TMA, head_dim 128, the item's logits parked on chip; 0.097 ms on the same
+        // shape (paged 0.121 against the clustered kernel's 0.146).  Falls back to the kernels below when the cache
         // does not fit it.
         const bool want_tc = variant == 14 || (variant == 0 && a.n_items >= 2 * ctx->sm_count && ctx->splits <= 1);
         if (want_tc && c->head_dim == 128 && resolve_tma_encode(ctx) && sizeof(ctx->kv8_maps) >= kv8_tc_maps_bytes()) {
