@@ -132,7 +132,8 @@ lethe_status lethe_poll_status(lethe_ctx *ctx, void *stream, int32_t *info);
  * (12,3) (10,4) (8,5) (16,2) (12,2) (e4m3 only); variant 14 the tensor-memory kernel (tcgen05 kind::f8f6f4 MMAs on the
  * cache's bytes with the query and the probabilities split into three e4m3 terms, K / V tiles by TMA, one CTA per SM;
  * head_dim 128, splits 0 or 1, and a capacity whose logits fit on chip: 2 * (heads per KV head) * capacity * 4 bytes
- * beside a 64 KB tile ring, else LETHE_ERR_UNSUPPORTED).  Automatic (variant 0): for launches of at least two items per
+ * beside a 64 KB tile ring; with more than five heads per KV head at least 0.4 of that, the rest overflows to
+ * scratch; else LETHE_ERR_UNSUPPORTED).  Automatic (variant 0): for launches of at least two items per
  * SM the tensor-memory kernel where the cache fits it, else (e4m3, head_dim 128) the persistent kernel with shape (8,4);
  * otherwise, and for any other value, the clustered kernel with shape (4,4).
  * 44..49 = the clustered kernel's six shapes for launches of one layer at a time (few items per launch): the CTAs of

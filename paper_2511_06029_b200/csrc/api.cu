@@ -426,22 +426,38 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
         // does not fit it.
         const bool want_tc = variant == 14 || (variant == 0 && a.n_items >= 2 * ctx->sm_count && ctx->splits <= 1);
         if (want_tc && c->head_dim == 128 && resolve_tma_encode(ctx) && sizeof(ctx->kv8_maps) >= kv8_tc_maps_bytes()) {
-            const int cap_pad = ((a.cap_tokens + 127) / 128) * 128;
+            const int cap_full = ((a.cap_tokens + 127) / 128) * 128;
             const int ng = 2;  // softmax groups
-            int nslot = 8;     // the deepest rings (K and V: half each) that fit beside the groups' logit buffers
-            while (nslot > 4 && kv8_tc_smem_bytes(nslot, G, cap_pad, ng) > ctx->max_smem) --nslot;
+            // The deepest rings (K and V: half each) that fit beside the groups' logit buffers.  A wide group (more than
+            // five heads) at a capacity that does not fit even beside four slots keeps the first `park` tokens of an
+            // item on chip and lets the rest overflow into a per-CTA slice of scratch (caches are sized well above the
+            // lengths items reach between rounds), provided at least 0.4 of the capacity stays on chip.
+            int nslot = 8, park = cap_full;
+            while (nslot > 4 && kv8_tc_smem_bytes(nslot, G, park, ng) > ctx->max_smem) --nslot;
+            if (kv8_tc_smem_bytes(nslot, G, park, ng) > ctx->max_smem && 3 * G > 16) {
+                const size_t fixed = kv8_tc_smem_bytes(nslot, G, 0, ng);
+                park = fixed < ctx->max_smem ? (int)((ctx->max_smem - fixed) / ((size_t)ng * G * 4) / 128) * 128 : 0;
+                if (park * 5 < cap_full * 2) park = 0;
+            }
             const int per_sm = 1;
+            const int grid = a.n_items < per_sm * ctx->sm_count ? a.n_items : per_sm * ctx->sm_count;
             const unsigned long long rows = paged ? (unsigned long long)c->n_pages * c->page_tokens
                                                   : (unsigned long long)c->n_layers * c->batch * c->n_kv_heads * c->capacity;
-            if (kv8_tc_smem_bytes(nslot, G, cap_pad, ng) <= ctx->max_smem && rows <= 0x7fffffffULL) {
+            if (park >= 128 && kv8_tc_smem_bytes(nslot, G, park, ng) <= ctx->max_smem && rows <= 0x7fffffffULL) {
+                if (park < cap_full) {
+                    a.spill_tokens = cap_full - park;
+                    const size_t need = (size_t)grid * ng * G * a.spill_tokens * sizeof(float);
+                    st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, need, "logit overflow scratch", stream);
+                    if (st != LETHE_OK) return st;
+                    a.spill = (float*)ctx->scratch;
+                }
                 if (ctx->kv8_k != c->k || ctx->kv8_v != c->v || ctx->kv8_rows != rows || ctx->kv8_paged != (int)paged) {
                     if (!build_kv8_tc_maps(ctx->tma_encode, c->k, c->v, rows, paged, ctx->kv8_maps))
                         return fail(ctx, LETHE_ERR_CUDA, "cuTensorMapEncodeTiled failed");
                     ctx->kv8_k = c->k; ctx->kv8_v = c->v; ctx->kv8_rows = rows; ctx->kv8_paged = (int)paged;
                 }
                 a.splits = 1;
-                const int grid = a.n_items < per_sm * ctx->sm_count ? a.n_items : per_sm * ctx->sm_count;
-                const cudaError_t et = launch_attend_kv8_tc(a, ctx->kv8_maps, paged, c->dtype == LETHE_FP8_E5M2, ng, nslot, cap_pad, grid,
+                const cudaError_t et = launch_attend_kv8_tc(a, ctx->kv8_maps, paged, c->dtype == LETHE_FP8_E5M2, ng, nslot, park, grid,
                                                             (cudaStream_t)stream);
                 if (et != cudaSuccess) return cuda_fail(ctx, et, "decode_attend launch (quantised cache, tensor memory)");
                 return LETHE_OK;

@@ -14,7 +14,9 @@
 // are recombined from the fp32 accumulators, once per token for the logits and once per item for the output.
 //
 // An item is processed in two streaming phases, K tiles then V tiles, so every cache byte still crosses HBM once:
-//   phase 1  logits of all tiles -> parked in shared memory (head-major), running maximum per thread;
+//   phase 1  logits of all tiles -> parked in shared memory (head-major; in the instances for wide groups and large
+//            capacities the tail of an item longer than that buffer goes to a per-CTA slice of global scratch, which
+//            stays in L2), running maximum per thread;
 //   phase 2  with the exact maximum known: p = exp2(s - m) from the parked logits, row sums, the three terms of p
 //            written as bytes in the MMA's operand layout, output accumulated in tensor memory — no online
 //            rescaling and no correction step;
@@ -234,7 +236,9 @@ __device__ __forceinline__ uint32_t sw128_at(uint32_t base, int row, int col) {
 
 // GT: the number of query heads per KV head when it is known at compile time (the loops over heads then carry no
 // run-time bounds), 0 = read it from the arguments.
-template <int NP, bool PAGED, bool E5M2, int NG, int GT>
+// SPILL: items may be longer than the on-chip logit buffer (cap_pad tokens per head); the logits of the tokens beyond
+// it are parked in this CTA's slice of global scratch.  A separate instance, so that caches that fit pay nothing.
+template <int NP, bool PAGED, bool E5M2, int NG, int GT, bool SPILL>
 __global__ void __launch_bounds__((4 * NG + kRoleWarps) * 32, 1)
     attend_kv8_tc_kernel(const __grid_constant__ AttendArgs a, const __grid_constant__ Kv8Maps maps, int nslot, int cap_pad) {
     using T = __nv_bfloat16;
@@ -560,6 +564,8 @@ __global__ void __launch_bounds__((4 * NG + kRoleWarps) * 32, 1)
         const int tg = w4 * 32 + lane;                             // thread within its group = TMEM lane
         const uint32_t t_lane = tmem + ((uint32_t)(w4 * 32) << 16);
         float* park = park_all + (size_t)g * G * cap_pad;
+        // [CTA][group][head][a.spill_tokens]; a tile lies wholly on one side (cap_pad is a multiple of the tile)
+        float* spill = SPILL ? a.spill + ((size_t)blockIdx.x * NG + g) * G * a.spill_tokens : nullptr;
         unsigned cs = 0, cw = 0;  // logit tiles read / probability tiles written by this group so far: buffer c & 3, phase c >> 2
         for (int seq = g, k = 0;; seq += NG, ++k) {
             if (!bar_wait(&hd.q_full[g], (unsigned)(k & 1), abort_flag, wait_limit)) break;
@@ -591,7 +597,8 @@ __global__ void __launch_bounds__((4 * NG + kRoleWarps) * 32, 1)
                     if (h < G) {
                         float s = fmaf(__uint_as_float(c[2 * G + h]), 0.00390625f, fmaf(__uint_as_float(c[G + h]), 0.0625f, __uint_as_float(c[h])));
                         s = tok < n ? s * sl2 : -INFINITY;
-                        park[(size_t)h * cap_pad + tok] = s;
+                        if (!SPILL || tok < cap_pad) park[(size_t)h * cap_pad + tok] = s;
+                        else spill[(size_t)h * a.spill_tokens + (tok - cap_pad)] = s;
                         mx[h] = fmaxf(mx[h], s);
                     }
                 }
@@ -633,7 +640,9 @@ __global__ void __launch_bounds__((4 * NG + kRoleWarps) * 32, 1)
                 for (int i = 0; i < 2; ++i) {
                     const int h = w4 + 4 * i;
                     if (h < G) {
-                        const float4 s4 = *reinterpret_cast<const float4*>(park + (size_t)h * cap_pad + t * kTile + 4 * lane);
+                        const float4 s4 = (!SPILL || t * kTile < cap_pad)
+                                              ? *reinterpret_cast<const float4*>(park + (size_t)h * cap_pad + t * kTile + 4 * lane)
+                                              : *reinterpret_cast<const float4*>(spill + (size_t)h * a.spill_tokens + (t * kTile - cap_pad) + 4 * lane);
                         const float off = 8.f - fm[h];  // probabilities are carried times 256: e4m3 keeps them normal down to 2^-14
                         const float p0 = s4.x == -INFINITY ? 0.f : fast_exp2(s4.x + off);
                         const float p1 = s4.y == -INFINITY ? 0.f : fast_exp2(s4.y + off);
@@ -706,7 +715,10 @@ __global__ void __launch_bounds__((4 * NG + kRoleWarps) * 32, 1)
                     float mass = 0.f;
 #pragma unroll
                     for (int h = 0; h < kMaxGroup; ++h)
-                        if (h < G) mass += fast_exp2(park[(size_t)h * cap_pad + j] - fm[h]) * inv[h];
+                        if (h < G) {
+                            const float sj = (!SPILL || j < cap_pad) ? park[(size_t)h * cap_pad + j] : spill[(size_t)h * a.spill_tokens + (j - cap_pad)];
+                            mass += fast_exp2(sj - fm[h]) * inv[h];
+                        }
                     return mass;
                 };
 #pragma unroll
@@ -772,9 +784,9 @@ __global__ void __launch_bounds__((4 * NG + kRoleWarps) * 32, 1)
 namespace lethe {
 namespace {
 
-template <int NP, bool PAGED, bool E5M2, int NG, int GT>
+template <int NP, bool PAGED, bool E5M2, int NG, int GT, bool SPILL>
 static cudaError_t launch_kv8_tc_t(const AttendArgs& a, const Kv8Maps& maps, int nslot, int cap_pad, int grid, cudaStream_t stream) {
-    auto kern = attend_kv8_tc_kernel<NP, PAGED, E5M2, NG, GT>;
+    auto kern = attend_kv8_tc_kernel<NP, PAGED, E5M2, NG, GT, SPILL>;
     const size_t smem = kv8_tc_smem_bytes(nslot, a.G, cap_pad, NG);
     cudaError_t e = prepare_kernel((const void*)kern, smem);
     if (e != cudaSuccess) return e;
@@ -793,15 +805,24 @@ static cudaError_t launch_kv8_tc_t(const AttendArgs& a, const Kv8Maps& maps, int
 
 // The four instances (contiguous / paged x e4m3 / e5m2) of one (operand width, group size) pair; one translation unit
 // per pair, so that they compile side by side.
-template <int NP, int GT>
+template <int NP, int GT, bool WITH_SPILL>
 cudaError_t launch_kv8_tc_pair(const AttendArgs& a, const void* maps_raw, bool paged, bool e5m2, int nslot, int cap_pad, int grid,
                                cudaStream_t stream) {
     Kv8Maps maps;
     memcpy(&maps, maps_raw, sizeof(maps));
-    return paged ? (e5m2 ? launch_kv8_tc_t<NP, true, true, 2, GT>(a, maps, nslot, cap_pad, grid, stream)
-                         : launch_kv8_tc_t<NP, true, false, 2, GT>(a, maps, nslot, cap_pad, grid, stream))
-                 : (e5m2 ? launch_kv8_tc_t<NP, false, true, 2, GT>(a, maps, nslot, cap_pad, grid, stream)
-                         : launch_kv8_tc_t<NP, false, false, 2, GT>(a, maps, nslot, cap_pad, grid, stream));
+    if (a.spill) {  // the instances with logit overflow exist for the wide groups only
+        if constexpr (WITH_SPILL)
+            return paged ? (e5m2 ? launch_kv8_tc_t<NP, true, true, 2, GT, true>(a, maps, nslot, cap_pad, grid, stream)
+                                 : launch_kv8_tc_t<NP, true, false, 2, GT, true>(a, maps, nslot, cap_pad, grid, stream))
+                         : (e5m2 ? launch_kv8_tc_t<NP, false, true, 2, GT, true>(a, maps, nslot, cap_pad, grid, stream)
+                                 : launch_kv8_tc_t<NP, false, false, 2, GT, true>(a, maps, nslot, cap_pad, grid, stream));
+        else
+            return cudaErrorInvalidValue;
+    }
+    return paged ? (e5m2 ? launch_kv8_tc_t<NP, true, true, 2, GT, false>(a, maps, nslot, cap_pad, grid, stream)
+                         : launch_kv8_tc_t<NP, true, false, 2, GT, false>(a, maps, nslot, cap_pad, grid, stream))
+                 : (e5m2 ? launch_kv8_tc_t<NP, false, true, 2, GT, false>(a, maps, nslot, cap_pad, grid, stream)
+                         : launch_kv8_tc_t<NP, false, false, 2, GT, false>(a, maps, nslot, cap_pad, grid, stream));
 }
 
 }  // namespace

@@ -5,7 +5,7 @@ namespace lethe {
 
 cudaError_t launch_kv8_tc_n16(const AttendArgs& a, const void* maps, bool paged, bool e5m2, int nslot, int cap_pad, int grid,
                             cudaStream_t stream) {
-    return launch_kv8_tc_pair<16, 0>(a, maps, paged, e5m2, nslot, cap_pad, grid, stream);
+    return launch_kv8_tc_pair<16, 0, false>(a, maps, paged, e5m2, nslot, cap_pad, grid, stream);
 }
 
 }  // namespace lethe

@@ -356,17 +356,19 @@ def test_quantised_automatic_choice_many_items(ctx, paged):
             assert_state_matches(gc, oc, exact_rel=True)
 
 
-def test_quantised_automatic_choice_large_capacity(ctx):
-    """No tuning set, many items, eight query heads per KV head and a capacity whose logits do not fit the
-    tensor-memory kernel's on-chip buffers: the automatic choice has to fall back to a kernel that holds (or
-    overflows) them, with the same results.  A few items are nearly as long as the capacity."""
-    L, B, Hq, Hkv, D, cap = 5, 8, 64, 8, 128, 2560
+@pytest.mark.parametrize("Hq,paged", [(64, False), (56, True), (48, False)])
+def test_quantised_automatic_choice_large_capacity(ctx, Hq, paged):
+    """No tuning set, many items, eight / seven / six query heads per KV head and a capacity whose logits do not fit
+    on chip beside the tile rings: the automatic choice has to take a kernel that overflows them (the tail of the
+    long items goes through scratch), with the same results.  A few items are nearly as long as the capacity."""
+    L, B, Hkv, D, cap = 5, 8, 8, 128, 2560
     assert L * B * Hkv >= 2 * torch.cuda.get_device_properties(0).multi_processor_count
     g = torch.Generator().manual_seed(77)
     lens = torch.randint(1, 200, (L, B, Hkv), generator=g)
     n_long = len(lens.view(-1)[::53])
     lens.view(-1)[::53] = torch.randint(2300, cap - 8, (n_long,), generator=g)
-    oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=13, k_scale=[0.4, 0.6, 0.8, 0.5, 1.0], v_scale=[1.0, 0.5, 2.0, 0.7, 0.9])
+    oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=13, k_scale=[0.4, 0.6, 0.8, 0.5, 1.0], v_scale=[1.0, 0.5, 2.0, 0.7, 0.9],
+                   page_tokens=16 if paged else 0)
     gc = to_device(oc)
     scale = torch.tensor([0.1, 0.08, 0.12, 0.09, 0.1], dtype=torch.float32)
     ctx.set_tuning(0, 0)
