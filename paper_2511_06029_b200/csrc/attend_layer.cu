@@ -60,7 +60,9 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(unsigned long long* bar, u
     return ok != 0;
 }
 
-template <int D, int NW, int NSTAGE, bool PAGED>
+// GT: query heads per KV head when known at compile time (0 = from the arguments): the merge, output and relevance
+// loops over heads then carry no run-time bounds.
+template <int D, int NW, int NSTAGE, bool PAGED, int GT>
 __global__ void __launch_bounds__(NW * 32) attend_layer_kernel(const __grid_constant__ AttendArgs a) {
     using T = __nv_bfloat16;
     constexpr int NT = NW * 32;
@@ -82,7 +84,7 @@ __global__ void __launch_bounds__(NW * 32) attend_layer_kernel(const __grid_cons
     const ItemCoord ic = decode_item(a);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int gq = lane >> 2, tq = lane & 3;
-    const int G = a.G, GP = a.GP, S = a.splits;
+    const int G = GT ? GT : a.G, GP = GT ? ((GT + 1) & ~1) : a.GP, S = a.splits;
     const bool append = a.k_new != nullptr;
 
     if (tid == 0) {
@@ -430,7 +432,7 @@ __global__ void __launch_bounds__(NW * 32) attend_layer_kernel(const __grid_cons
         float none[kRelPrefetch];
 #pragma unroll
         for (int i = 0; i < kRelPrefetch; ++i) none[i] = 0.f;
-        relevance_update<NT>(a, ic, fin, lg + (size_t)PF * NT * GP, t0 + PF * NT, hi_tok, append_slot, none, kRelPrefetch);
+        relevance_update<NT, GT>(a, ic, fin, lg + (size_t)PF * NT * GP, t0 + PF * NT, hi_tok, append_slot, none, kRelPrefetch);
     }
     if (append_slot >= 0 && ic.rank == 0 && tid == 0) a.len[ic.item] = n;
 }
@@ -440,9 +442,9 @@ static size_t layer_smem(int chunk_tokens, int GP) {
     return (size_t)NW * NSTAGE * 2 * kGroupTokens * D * 2 + sizeof(LayerSmem) + (size_t)chunk_tokens * GP * 4;
 }
 
-template <int D, int NW, int NSTAGE, bool PAGED>
+template <int D, int NW, int NSTAGE, bool PAGED, int GT>
 static cudaError_t launch_layer_t(const AttendArgs& a, cudaStream_t stream) {
-    auto kern = attend_layer_kernel<D, NW, NSTAGE, PAGED>;
+    auto kern = attend_layer_kernel<D, NW, NSTAGE, PAGED, GT>;
     const size_t smem = layer_smem<D, NW, NSTAGE>(a.chunk_tokens, a.GP);
     cudaError_t e = prepare_kernel((const void*)kern, smem);
     if (e != cudaSuccess) return e;
@@ -477,9 +479,14 @@ size_t layer_smem_bytes(int D, int shape, int chunk_tokens, int GP) {
 }
 
 cudaError_t launch_attend_layer(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream) {
+    // the automatic choices for the two common geometries with their group size compiled in
+    if (D == 128 && shape == 0 && a.G == 4)
+        return paged ? launch_layer_t<128, 4, 3, true, 4>(a, stream) : launch_layer_t<128, 4, 3, false, 4>(a, stream);
+    if (D == 128 && shape == 2 && a.G == 7)
+        return paged ? launch_layer_t<128, 4, 2, true, 7>(a, stream) : launch_layer_t<128, 4, 2, false, 7>(a, stream);
 #define X(id, DD, NW, NS)                                                                    \
     if (shape == id && D == DD)                                                              \
-        return paged ? launch_layer_t<DD, NW, NS, true>(a, stream) : launch_layer_t<DD, NW, NS, false>(a, stream);
+        return paged ? launch_layer_t<DD, NW, NS, true, 0>(a, stream) : launch_layer_t<DD, NW, NS, false, 0>(a, stream);
     LETHE_LAYER_SHAPES(X, 128)
     LETHE_LAYER_SHAPES(X, 64)
 #undef X

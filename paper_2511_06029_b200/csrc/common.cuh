@@ -177,14 +177,14 @@ __device__ __forceinline__ void prefetch_rel(const AttendArgs& a, const ItemCoor
 // rel[j] = gamma * rel[j] + sum over the group's heads of exp2(s_hj - m_h) / l_h, with fin[h] = (m_h, 1 / l_h) the
 // exact global statistics.  rel_old holds the values prefetch_rel loaded for the thread's first kRelPrefetch tokens;
 // with first_batch = kRelPrefetch those tokens are skipped and [t0, hi_tok) is a range that starts after them.
-template <int NT>
+template <int NT, int GT = 0>  // GT: the group size when it is a compile-time constant of the caller, else 0
 __device__ __forceinline__ void relevance_update(const AttendArgs& a, const ItemCoord& ic, const float2* fin, const float* lg,
                                                  int t0, int hi_tok, int append_slot, const float (&rel_old)[kRelPrefetch],
                                                  int first_batch = 0) {
     const int tid = threadIdx.x;
-    const int G = a.G;
+    const int G = GT ? GT : a.G;
     float* rel = a.rel + (size_t)ic.item * a.cap_tokens;
-    const int GP = a.GP;
+    const int GP = GT ? ((GT + 1) & ~1) : a.GP;
     float fm[kMaxGroup], fi[kMaxGroup];
 #pragma unroll
     for (int h = 0; h < kMaxGroup; ++h) {
