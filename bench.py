@@ -737,15 +737,17 @@ def main():
     def prepare(capacity):
         """Runner brought to steady state (untimed): a few full prune intervals so that relevance, sparsity-driven
         budgets and lengths are those of a long trajectory (dense layers need several rounds to grow to their
-        budget).  Returns the runner and the largest layer budget."""
+        budget).  Returns the runner and the largest layer budget any of those rounds handed out."""
         r = Runner(w, dev, rank, capacity, args.variant, args.splits, kv=args.kv)
+        largest = 0
         for _ in range(max(1, args.prep_rounds)):
             for _ in range(w.prune_interval):
                 r.decode()
             r.prune()
+            largest = max(largest, int(r.budgets.max().item()))   # budgets move from round to round with the relevance
             r.drift_if_due()
         r.check()
-        return r, int(r.budgets.max().item())
+        return r, largest
 
     lens_seq = None
     if w.page_tokens:

@@ -55,7 +55,8 @@ __device__ __forceinline__ int opaque(int x) {
     return x;
 }
 
-template <int D, int NW, int NS, bool PAGED, bool SPILL>
+// GT: query heads per KV head when known at compile time (0 = from the arguments).
+template <int D, int NW, int NS, bool PAGED, bool SPILL, int GT = 0>
 __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_constant__ AttendArgs a) {
     using T = __nv_bfloat16;
     constexpr int NT = NW * 32;
@@ -68,7 +69,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_stream_kernel(const __grid_
     static_assert(NS >= 2 && NS <= 5, "pipeline depth");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     // layout: stages [NW][NS][K tile | V tile] | wo [NW][GP][D] fp32 | EpilogueSmem | lg [chunk_tokens][GP]
-    const int G = a.G, GP = a.GP;
+    const int G = GT ? GT : a.G, GP = GT ? ((GT + 1) & ~1) : a.GP;
     const int wo_stride = GP * D;
     float* wo_all = reinterpret_cast<float*>(smem_raw + (size_t)NW * WARP_BYTES);
     EpilogueSmem& es = *reinterpret_cast<EpilogueSmem*>(wo_all + (size_t)NW * wo_stride);
@@ -479,9 +480,9 @@ static size_t stream_smem(int chunk_tokens, int GP) {
            (size_t)chunk_tokens * GP * 4;
 }
 
-template <int D, int NW, int NS, bool PAGED, bool SPILL>
+template <int D, int NW, int NS, bool PAGED, bool SPILL, int GT = 0>
 static cudaError_t launch_stream_t(const AttendArgs& a, int grid, cudaStream_t stream) {
-    auto kern = attend_stream_kernel<D, NW, NS, PAGED, SPILL>;
+    auto kern = attend_stream_kernel<D, NW, NS, PAGED, SPILL, GT>;
     const size_t smem = stream_smem<D, NW, NS>(a.chunk_tokens, a.GP);
     cudaError_t e = prepare_kernel((const void*)kern, smem);
     if (e != cudaSuccess) return e;
@@ -489,11 +490,11 @@ static cudaError_t launch_stream_t(const AttendArgs& a, int grid, cudaStream_t s
     return cudaGetLastError();
 }
 
-template <int D, int NW, int NS>
+template <int D, int NW, int NS, int GT = 0>
 static cudaError_t dispatch_stream(const AttendArgs& a, bool paged, int grid, cudaStream_t stream) {
     const bool spill = a.spill != nullptr;
-    if (paged) return spill ? launch_stream_t<D, NW, NS, true, true>(a, grid, stream) : launch_stream_t<D, NW, NS, true, false>(a, grid, stream);
-    return spill ? launch_stream_t<D, NW, NS, false, true>(a, grid, stream) : launch_stream_t<D, NW, NS, false, false>(a, grid, stream);
+    if (paged) return spill ? launch_stream_t<D, NW, NS, true, true, GT>(a, grid, stream) : launch_stream_t<D, NW, NS, true, false, GT>(a, grid, stream);
+    return spill ? launch_stream_t<D, NW, NS, false, true, GT>(a, grid, stream) : launch_stream_t<D, NW, NS, false, false, GT>(a, grid, stream);
 }
 
 // Shapes of the persistent kernel: (warps per CTA, stages per warp).
@@ -510,6 +511,8 @@ size_t stream_smem_bytes(int D, int shape, int chunk_tokens, int GP) {
 }
 
 cudaError_t launch_attend_stream(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream) {
+    // the automatic choice for wide groups (seven query heads per KV head: the Qwen geometry), group size compiled in
+    if (D == 128 && shape == 0 && a.G == 7) return dispatch_stream<128, 8, 2, 7>(a, paged, grid, stream);
 #define X(id, DD, NW, NS)                                                                                   \
     if (shape == id && D == DD)                                                                             \
         return dispatch_stream<DD, NW, NS>(a, paged, grid, stream);
