@@ -47,10 +47,10 @@ NOMINAL_HBM_GBS = 8000.0
 # captures summarised under profiles/ (traffic grows in proportion to the token-heads of a launch, so the
 # per-token-head figure of the capture is scaled to the launch bench.py times).  None = no capture on record.
 NCU_TRAFFIC = {
-    "llama8b": (519.9, "profiles/attend_async_w8s2_llama8b_bench.md"),
-    "qwen7b": (520.1, "profiles/attend_stream_w8s2_qwen7b.md"),
-    "longreason": (519.4, "profiles/attend_async_spill_w8s2_longreason.md"),
-    "ragged": (520.4, "profiles/attend_stream_paged_w8s2_ragged.md"),
+    "llama8b": (519.8, "profiles/attend_async_w8s2_llama8b_bench.md"),
+    "qwen7b": (521.5, "profiles/attend_stream_w8s2_qwen7b.md"),
+    "longreason": (519.1, "profiles/attend_async_spill_w8s2_longreason.md"),
+    "ragged": (520.5, "profiles/attend_stream_paged_w8s2_ragged.md"),
     "llama8b:fp8": (267.5, "profiles/attend_kv8_tc_llama8b.md"),
 }
 RAGGED_RESIDENT_LAYERS = 7           # of 28: the full ragged state is 124 GB of K/V; one layer group is resident at a time
