@@ -63,6 +63,28 @@ __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t x) {
     const float lo = __uint_as_float(x << 16), hi = __uint_as_float(x & 0xffff0000u);
     return pack_f16(lo, hi);
 }
+// two bf16 values times a power of two -> two f16 values (exact while the products are within f16's range)
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2_scaled(uint32_t x, float mul) {
+    return pack_f16(__uint_as_float(x << 16) * mul, __uint_as_float(x & 0xffff0000u) * mul);
+}
+// The divisor (a power of two, returned in `div`) that brings the largest magnitude of a query row into [128, 256), and
+// its inverse (the return value).  The row is spread over the four lanes that share gq = lane >> 2; w holds this lane's
+// bf16 pairs.
+template <int KS>
+__device__ __forceinline__ float query_row_scale(const uint2 (&w)[KS], float& div) {
+    float big = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+        big = fmaxf(big, fmaxf(fabsf(__uint_as_float(w[ks].x << 16)), fabsf(__uint_as_float(w[ks].x & 0xffff0000u))));
+        big = fmaxf(big, fmaxf(fabsf(__uint_as_float(w[ks].y << 16)), fabsf(__uint_as_float(w[ks].y & 0xffff0000u))));
+    }
+    big = fmaxf(big, __shfl_xor_sync(0xffffffffu, big, 1));
+    big = fmaxf(big, __shfl_xor_sync(0xffffffffu, big, 2));
+    int ex = (int)((__float_as_uint(big) >> 23) & 0xffu) - 7;  // biased exponent of the divisor
+    ex = big > 0.f && big < INFINITY ? min(max(ex, 2), 252) : 127;
+    div = __uint_as_float((uint32_t)ex << 23);
+    return __uint_as_float((uint32_t)(254 - ex) << 23);
+}
 
 }  // namespace
 
@@ -99,16 +121,21 @@ __global__ void __launch_bounds__(NW * 32) attend_kv8_kernel(const __grid_consta
     const int n_old = a.len[ic.item];
     // Q^T fragments (B operand) in f16, in the permuted order of the key bytes: step ks covers d = 16 ks .. + 15,
     // b0 = Q[head gq][16 ks + 4 tq + {0, 1}], b1 = Q[head gq][16 ks + 4 tq + {2, 3}]
+    // f16 holds 6e-8 .. 65504, so the row of head gq is first divided by the power of two that brings its largest
+    // magnitude into [128, 256) (exact); qdiv is that divisor, and the head's logits are multiplied back below.
     uint32_t bq[KS][2];
+    float qdiv = 1.f;
     {
         const uint2* qrow =
             reinterpret_cast<const uint2*>((const T*)a.q + ((size_t)(ic.li * a.B + ic.b) * a.Hq + ic.hkv * G + gq) * D);
+        uint2 w[KS];
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) w[ks] = gq < G ? qrow[4 * ks + tq] : make_uint2(0u, 0u);
+        const float inv = query_row_scale(w, qdiv);
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
-            uint2 w = make_uint2(0u, 0u);
-            if (gq < G) w = qrow[4 * ks + tq];
-            bq[ks][0] = bf16x2_to_f16x2(w.x);
-            bq[ks][1] = bf16x2_to_f16x2(w.y);
+            bq[ks][0] = bf16x2_to_f16x2_scaled(w[ks].x, inv);
+            bq[ks][1] = bf16x2_to_f16x2_scaled(w[ks].y, inv);
         }
     }
     T* out_rows = (T*)a.out + ((size_t)(ic.li * a.B + ic.b) * a.Hq + ic.hkv * G) * D;
@@ -150,6 +177,8 @@ __global__ void __launch_bounds__(NW * 32) attend_kv8_kernel(const __grid_consta
     __syncthreads();  // the appended row is in global memory before any warp streams it
 
     const float sl2 = a.scale_log2[ic.l];  // softmax scale x key scale x log2(e)
+    // this thread's two logit columns are heads 2 tq and 2 tq + 1: their divisors sit in the lanes with gq = head
+    const float sl2_0 = sl2 * __shfl_sync(0xffffffffu, qdiv, (2 * tq) * 4), sl2_1 = sl2 * __shfl_sync(0xffffffffu, qdiv, (2 * tq + 1) * 4);
 
     unsigned char* my_stage = stage_base + (size_t)warp * WARP_BYTES;
     const uint32_t my_stage_u32 = smem_u32(my_stage);
@@ -230,10 +259,10 @@ __global__ void __launch_bounds__(NW * 32) attend_kv8_kernel(const __grid_consta
             mma_f16(cb, a1, bq[2 * pr + 1][0], bq[2 * pr + 1][1]);
         }
         const int tokA = grp * kGroupTokens + gq, tokB = tokA + 8;
-        float s00 = (tokA < n) ? (ca[0] + cb[0]) * sl2 : -INFINITY;  // token A, head 2tq
-        float s01 = (tokA < n) ? (ca[1] + cb[1]) * sl2 : -INFINITY;  // token A, head 2tq+1
-        float s10 = (tokB < n) ? (ca[2] + cb[2]) * sl2 : -INFINITY;
-        float s11 = (tokB < n) ? (ca[3] + cb[3]) * sl2 : -INFINITY;
+        float s00 = (tokA < n) ? (ca[0] + cb[0]) * sl2_0 : -INFINITY;  // token A, head 2tq
+        float s01 = (tokA < n) ? (ca[1] + cb[1]) * sl2_1 : -INFINITY;  // token A, head 2tq+1
+        float s10 = (tokB < n) ? (ca[2] + cb[2]) * sl2_0 : -INFINITY;
+        float s11 = (tokB < n) ? (ca[3] + cb[3]) * sl2_1 : -INFINITY;
         if (2 * tq < GP) {
             float2* row = reinterpret_cast<float2*>(lg + (size_t)(tokA - t0) * GP + 2 * tq);
             row[0] = make_float2(s00, s01);

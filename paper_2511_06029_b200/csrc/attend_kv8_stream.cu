@@ -36,8 +36,27 @@ __device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi) {
     asm("{ .reg .b16 r; cvt.rn.satfinite.e4m3x2.f32 r, %2, %1; cvt.u32.u16 %0, r; }" : "=r"(y) : "f"(lo), "f"(hi));
     return y;
 }
-__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t x) {
-    return pack_f16(__uint_as_float(x << 16), __uint_as_float(x & 0xffff0000u));
+// two bf16 values times a power of two -> two f16 values (exact while the products are within f16's range)
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2_scaled(uint32_t x, float mul) {
+    return pack_f16(__uint_as_float(x << 16) * mul, __uint_as_float(x & 0xffff0000u) * mul);
+}
+// The divisor (a power of two, returned in `div`) that brings the largest magnitude of a query row into [128, 256), and
+// its inverse (the return value): f16 holds 6e-8 .. 65504, bf16 queries can be anything.  The row is spread over the
+// four lanes that share gq = lane >> 2; w holds this lane's bf16 pairs.
+template <int KS>
+__device__ __forceinline__ float query_row_scale(const uint2 (&w)[KS], float& div) {
+    float big = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+        big = fmaxf(big, fmaxf(fabsf(__uint_as_float(w[ks].x << 16)), fabsf(__uint_as_float(w[ks].x & 0xffff0000u))));
+        big = fmaxf(big, fmaxf(fabsf(__uint_as_float(w[ks].y << 16)), fabsf(__uint_as_float(w[ks].y & 0xffff0000u))));
+    }
+    big = fmaxf(big, __shfl_xor_sync(0xffffffffu, big, 1));
+    big = fmaxf(big, __shfl_xor_sync(0xffffffffu, big, 2));
+    int ex = (int)((__float_as_uint(big) >> 23) & 0xffu) - 7;  // biased exponent of the divisor
+    ex = big > 0.f && big < INFINITY ? min(max(ex, 2), 252) : 127;
+    div = __uint_as_float((uint32_t)ex << 23);
+    return __uint_as_float((uint32_t)(254 - ex) << 23);
 }
 
 struct StreamItem {
@@ -137,21 +156,25 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_kv8_stream_kernel(const __g
     fill_counts<NW>(a, cur, cur.valid ? a.len[cur.item] : 0, warp);
     int nxt_n_raw = nxt.valid ? a.len[nxt.item] : 0;  // consumed lazily (see opaque) so the load stays in flight
 
-    auto load_q = [&](const StreamItem& it, uint32_t (&bq)[KS][2]) {
-        // f16, in the permuted order of the key bytes: b0 = Q[head gq][16 ks + 4 tq + {0, 1}], b1 = ... + {2, 3}
+    auto load_q = [&](const StreamItem& it, uint32_t (&bq)[KS][2], float& qdiv) {
+        // f16, in the permuted order of the key bytes: b0 = Q[head gq][16 ks + 4 tq + {0, 1}], b1 = ... + {2, 3}; the row is
+        // divided by the power of two qdiv first (see query_row_scale), the head's logits are multiplied back
         const uint2* qrow = reinterpret_cast<const uint2*>(
             (const T*)a.q + ((size_t)(it.li * a.B + it.b) * a.Hq + it.hkv * G + gq) * D);
+        uint2 w[KS];
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) w[ks] = (it.valid && gq < G) ? qrow[4 * ks + tq] : make_uint2(0u, 0u);
+        const float inv = query_row_scale(w, qdiv);
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
-            uint2 w = make_uint2(0u, 0u);
-            if (it.valid && gq < G) w = qrow[4 * ks + tq];
-            bq[ks][0] = bf16x2_to_f16x2(w.x);
-            bq[ks][1] = bf16x2_to_f16x2(w.y);
+            bq[ks][0] = bf16x2_to_f16x2_scaled(w[ks].x, inv);
+            bq[ks][1] = bf16x2_to_f16x2_scaled(w[ks].y, inv);
         }
     };
     uint32_t bq[KS][2], bqn[KS][2];
-    load_q(cur, bq);
-    load_q(nxt, bqn);
+    float qdiv = 1.f, qdivn = 1.f;
+    load_q(cur, bq, qdiv);
+    load_q(nxt, bqn, qdivn);
 
     unsigned char* my_stage = smem_raw + (size_t)warp * WARP_BYTES;
     const uint32_t my_stage_u32 = smem_u32(my_stage);
@@ -240,6 +263,8 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_kv8_stream_kernel(const __g
 
     while (cur.valid) {
         const float sl2 = a.scale_log2[cur.l];
+        // this thread's two logit columns are heads 2 tq and 2 tq + 1: their divisors sit in the lanes with gq = head
+        const float sl2_0 = sl2 * __shfl_sync(0xffffffffu, qdiv, (2 * tq) * 4), sl2_1 = sl2 * __shfl_sync(0xffffffffu, qdiv, (2 * tq + 1) * 4);
         // ---- top-up: whatever of the first NS-1 groups the previous tail did not prefetch
         bool topped = false;
 #pragma unroll
@@ -302,10 +327,10 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_kv8_stream_kernel(const __g
                 mma_f16(cb, a1, bq[2 * pr + 1][0], bq[2 * pr + 1][1]);
             }
             const int tokA = grp * kGroupTokens + gq, tokB = tokA + 8;
-            const float s00 = (tokA < cur.n) ? (ca[0] + cb[0]) * sl2 : -INFINITY;
-            const float s01 = (tokA < cur.n) ? (ca[1] + cb[1]) * sl2 : -INFINITY;
-            const float s10 = (tokB < cur.n) ? (ca[2] + cb[2]) * sl2 : -INFINITY;
-            const float s11 = (tokB < cur.n) ? (ca[3] + cb[3]) * sl2 : -INFINITY;
+            const float s00 = (tokA < cur.n) ? (ca[0] + cb[0]) * sl2_0 : -INFINITY;
+            const float s01 = (tokA < cur.n) ? (ca[1] + cb[1]) * sl2_1 : -INFINITY;
+            const float s10 = (tokB < cur.n) ? (ca[2] + cb[2]) * sl2_0 : -INFINITY;
+            const float s11 = (tokB < cur.n) ? (ca[3] + cb[3]) * sl2_1 : -INFINITY;
             if (2 * tq < GP) {
                 if (!SPILL || tokA < chunk) st_shared_f2(lg_u32 + (tokA * GP + 2 * tq) * 4, s00, s01);
                 else *reinterpret_cast<float2*>(spill + (size_t)(tokA - chunk) * GP + 2 * tq) = make_float2(s00, s01);
@@ -475,10 +500,11 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_kv8_stream_kernel(const __g
             bq[ks][0] = bqn[ks][0];
             bq[ks][1] = bqn[ks][1];
         }
+        qdiv = qdivn;
         issued = issued_next;
         decode_ticket(a, es.flags[2], nxt);
         nxt_n_raw = nxt.valid ? a.len[nxt.item] : 0;
-        load_q(nxt, bqn);
+        load_q(nxt, bqn, qdivn);
     }
     cp_async_wait<0>();
     if (bad_page) record_error(a.status, LETHE_ERR_PAGE, 0);

@@ -9,7 +9,8 @@
 //   output   O^T[128 dims x N] += V tile^T (the same memory image, read MN-major) . Ps^T
 //
 // The other operand has to be an 8-bit float as well.  A bf16 query value is split exactly into three e4m3 terms,
-// q = t1 + t2 / 16 + t3 / 256, and the probabilities likewise, p * 256 = u1 + u2 / 16 + u3 / 256 (12 bits, one more
+// q = t1 + t2 / 16 + t3 / 256 (after its row has been divided by a power of two that puts the row's largest magnitude
+// into e4m3's range; the head's logits are multiplied back), and the probabilities likewise, p * 256 = u1 + u2 / 16 + u3 / 256 (12 bits, one more
 // than the f16 the mma.sync kernels round them to); the terms sit on the N axis (N = 3 G padded to 16 or 32) and
 // are recombined from the fp32 accumulators, once per token for the logits and once per item for the output.
 //
@@ -75,6 +76,7 @@ struct alignas(64) Kv8Maps {
 
 struct Kv8Desc {
     int valid, item, li, l, b, hkv, n_old, n, full, T;
+    float qmul[kMaxGroup];  // per head: the power of two its query row was divided by before the split (see the set-up warp)
 };
 
 struct Kv8Header {
@@ -371,13 +373,27 @@ __global__ void __launch_bounds__((4 * NG + kRoleWarps) * 32, 1)
                     proxy_fence_all();  // the new rows are read back by TMA (the async proxy) below
                 }
                 // the item's query rows as the B operand of the logit MMAs: row (term * G + h), 128 bytes of d
+                // e4m3 covers 2^-9 .. 448, so each row is first divided by a power of two that brings its largest
+                // magnitude into [128, 256) (exact; the three terms then hold every bf16 value of the row down to 2^-25
+                // of that maximum); the logits of the head are multiplied back when they are read out of tensor memory
                 const uint32_t qb = qs_u32 + par * NP * 128;
 #pragma unroll
                 for (int h = 0; h < kMaxGroup; ++h) {
+                    d.qmul[h] = 1.f;
                     if (h < G) {
+                        float x0 = __uint_as_float(qw[h].x << 16), x1 = __uint_as_float(qw[h].x & 0xffff0000u);
+                        float x2 = __uint_as_float(qw[h].y << 16), x3 = __uint_as_float(qw[h].y & 0xffff0000u);
+                        float big = fmaxf(fmaxf(fabsf(x0), fabsf(x1)), fmaxf(fabsf(x2), fabsf(x3)));
+#pragma unroll
+                        for (int off = 16; off > 0; off >>= 1) big = fmaxf(big, __shfl_xor_sync(0xffffffffu, big, off));
+                        // exponent field of the maximum -> 2^(e - 7), clamped so that both it and its inverse are normal
+                        int ex = (int)((__float_as_uint(big) >> 23) & 0xffu) - 7;   // biased exponent of the divisor
+                        ex = big > 0.f && big < INFINITY ? min(max(ex, 2), 252) : 127;
+                        const float div = __uint_as_float((uint32_t)ex << 23), inv = __uint_as_float((uint32_t)(254 - ex) << 23);
+                        d.qmul[h] = div;
+                        x0 *= inv; x1 *= inv; x2 *= inv; x3 *= inv;
                         uint32_t terms[3];
-                        split3(__uint_as_float(qw[h].x << 16), __uint_as_float(qw[h].x & 0xffff0000u), __uint_as_float(qw[h].y << 16),
-                               __uint_as_float(qw[h].y & 0xffff0000u), terms);
+                        split3(x0, x1, x2, x3, terms);
 #pragma unroll
                         for (int t3 = 0; t3 < 3; ++t3)
                             asm volatile("st.shared.b32 [%0], %1;" ::"r"(sw128_at(qb, t3 * G + h, lane * 4)), "r"(terms[t3]) : "memory");
@@ -573,7 +589,9 @@ __global__ void __launch_bounds__((4 * NG + kRoleWarps) * 32, 1)
             __syncwarp();
             if (lane == 0) bar_arrive(&hd.q_empty[g]);
             if (!d.valid) break;
-            const float sl2 = a.scale_log2[d.l];
+            float sl2h[kMaxGroup];  // softmax scale (log2 units) times the head's query divisor
+#pragma unroll
+            for (int h = 0; h < kMaxGroup; ++h) sl2h[h] = a.scale_log2[d.l] * d.qmul[h];
             const int n = d.n;
             bool alive = true;
             // ---- phase 1: logits of the item's K tiles, one token per thread
@@ -596,7 +614,7 @@ __global__ void __launch_bounds__((4 * NG + kRoleWarps) * 32, 1)
                 for (int h = 0; h < kMaxGroup; ++h) {
                     if (h < G) {
                         float s = fmaf(__uint_as_float(c[2 * G + h]), 0.00390625f, fmaf(__uint_as_float(c[G + h]), 0.0625f, __uint_as_float(c[h])));
-                        s = tok < n ? s * sl2 : -INFINITY;
+                        s = tok < n ? s * sl2h[h] : -INFINITY;
                         if (!SPILL || tok < cap_pad) park[(size_t)h * cap_pad + tok] = s;
                         else spill[(size_t)h * a.spill_tokens + (tok - cap_pad)] = s;
                         mx[h] = fmaxf(mx[h], s);

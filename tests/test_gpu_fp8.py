@@ -380,3 +380,28 @@ def test_quantised_automatic_choice_large_capacity(ctx, Hq, paged):
         kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
         vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
         _step(ctx, oc, gc, q, kn, vn, torch.arange(B, dtype=torch.int32) + 900 + step, scale, 0.97)
+
+
+@pytest.mark.parametrize("variant", [TENSOR_MEMORY, 0])
+def test_quantised_query_magnitudes(ctx, variant):
+    """Query rows far outside e4m3's range (the tensor-memory kernel feeds the queries to the MMAs as 8-bit terms):
+    heads whose rows are scaled by 2^12, 2^-20, 3e4 and 1e-7, with the softmax scale compensating so that the logits
+    stay ordinary; a head of zeros; one huge element in an otherwise ordinary row."""
+    L, B, Hq, Hkv, D, cap = 2, 3, 8, 2, 128, 416
+    g = torch.Generator().manual_seed(91)
+    lens = torch.randint(1, cap - 8, (L, B, Hkv), generator=g)
+    oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=17, k_scale=[0.37, 1.5], v_scale=[2.25, 0.6])
+    gc = to_device(oc)
+    ctx.set_tuning(variant, 0)
+    try:
+        for step, (mul, sc) in enumerate([(4096.0, 0.1 / 4096), (2.0 ** -20, 0.1 * 2.0 ** 20), (3.0e4, 0.08 / 3.0e4), (1.0e-7, 0.08e7)]):
+            q = torch.randn((L, B, Hq, D), generator=g) * mul
+            q[0, 0, 1] = 0.0                                         # a head of zeros: uniform attention
+            q[1, 1, 2, 5] = 40.0 * mul                               # one element far above the rest of its row
+            q = q.to(torch.bfloat16)
+            kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            scale = torch.tensor([sc, sc * 0.7], dtype=torch.float32)
+            _step(ctx, oc, gc, q, kn, vn, torch.arange(B, dtype=torch.int32) + 300 + step, scale, 0.95, want_lse=(step == 1))
+    finally:
+        ctx.set_tuning(0, 0)
