@@ -135,7 +135,9 @@ lethe_status lethe_poll_status(lethe_ctx *ctx, void *stream, int32_t *info);
  * beside a 64 KB tile ring; with more than five heads per KV head at least 0.4 of that, the rest overflows to
  * scratch; else LETHE_ERR_UNSUPPORTED).  Automatic (variant 0): for launches of at least two items per
  * SM the tensor-memory kernel where the cache fits it, else (e4m3, head_dim 128) the persistent kernel with shape (8,4);
- * otherwise, and for any other value, the clustered kernel with shape (4,4).
+ * otherwise (launches of few items, e.g. one layer at a time) the layer kernel described below for variants 44..49 in
+ * its byte-cache form (4 warps x 4 stages, head_dim 128; variant 44 forces it); for any other value, and for head_dim 64,
+ * the clustered kernel with shape (4,4).
  * 44..49 = the clustered kernel's six shapes for launches of one layer at a time (few items per launch): the CTAs of
  * an item merge by one-sided pushes through distributed shared memory (no cluster barriers), and — when variant 51
  * is also set — a launch fetches cached K / V tiles while the previous launch is still finishing.

@@ -23,6 +23,8 @@ size_t simt_smem_bytes(int D, int chunk_tokens, int GP);
 cudaError_t launch_attend_mma(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream);
 size_t mma_smem_bytes(int D, int shape, int chunk_tokens, int GP);
 cudaError_t launch_attend_layer(const AttendArgs& a, int D, int shape, bool paged, cudaStream_t stream);
+size_t kv8_layer_smem_bytes(int chunk_tokens, int GP);
+cudaError_t launch_attend_kv8_layer(const AttendArgs& a, bool paged, bool e5m2, cudaStream_t stream);
 size_t layer_smem_bytes(int D, int shape, int chunk_tokens, int GP);
 cudaError_t launch_attend_stream(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream);
 size_t stream_smem_bytes(int D, int shape, int chunk_tokens, int GP);
@@ -496,21 +498,27 @@ lethe_status lethe_decode_attend(lethe_ctx* ctx, const lethe_cache* c, int layer
             return LETHE_OK;
         }
         const int shape = want_clustered ? variant - 2 : 0;
+        // Few items per launch (one layer at a time): the layer kernel's byte-cache instance (one-sided merge, tiles
+        // fetched before the previous launch completes; variant 44 forces it), head_dim 128; else the clustered kernel.
+        const bool layer8 = (variant == 0 || variant == 44) && c->head_dim == 128;
         auto smem_for = [&](int S) -> size_t {
             const int chunk = ((cap_groups + S - 1) / S) * kGroupTokens;
-            return kv8_smem_bytes(c->head_dim, shape, chunk, a.GP);
+            return layer8 ? kv8_layer_smem_bytes(chunk, a.GP) : kv8_smem_bytes(c->head_dim, shape, chunk, a.GP);
         };
         int S = ctx->splits;
         if (S == 0) {
             S = 1;
             while (S < 16 && smem_for(S) > ctx->max_smem) S *= 2;
-            while (S < 8 && (long long)a.n_items * S < ctx->sm_count && cap_groups / (2 * S) >= 4) S *= 2;
+            while (S < 8 && ((long long)a.n_items * S < ctx->sm_count || (layer8 && a.n_items <= ctx->sm_count && S < 4)) &&
+                   cap_groups / (2 * S) >= 4)
+                S *= 2;
         }
         if (smem_for(S) > ctx->max_smem)
             return fail(ctx, LETHE_ERR_UNSUPPORTED, "capacity too large for the on-chip logit buffer at this split count");
         a.splits = S;
         a.chunk_tokens = ((cap_groups + S - 1) / S) * kGroupTokens;
-        const cudaError_t e8 = launch_attend_kv8(a, c->head_dim, shape, paged, c->dtype == LETHE_FP8_E5M2, (cudaStream_t)stream);
+        const cudaError_t e8 = layer8 ? launch_attend_kv8_layer(a, paged, c->dtype == LETHE_FP8_E5M2, (cudaStream_t)stream)
+                                      : launch_attend_kv8(a, c->head_dim, shape, paged, c->dtype == LETHE_FP8_E5M2, (cudaStream_t)stream);
         if (e8 != cudaSuccess) return cuda_fail(ctx, e8, "decode_attend launch (quantised cache)");
         return LETHE_OK;
     }

@@ -19,6 +19,7 @@
 //     which everything it needs is in its own shared memory.  Nobody reads a peer's memory, so a CTA may exit as
 //     soon as it has finished — no closing barrier.  The wait is bounded (LETHE_ERR_TIMEOUT).
 #include "common.cuh"
+#include "kv8_utils.cuh"
 #include "mma_utils.cuh"
 
 namespace lethe {
@@ -62,22 +63,33 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(unsigned long long* bar, u
 
 // GT: query heads per KV head when known at compile time (0 = from the arguments): the merge, output and relevance
 // loops over heads then carry no run-time bounds.
-template <int D, int NW, int NSTAGE, bool PAGED, int GT>
+// KV: 0 = bf16 cache; 1 / 2 = quantised cache (e4m3 / e5m2 bytes, one scale per layer): the same kernel around the
+// byte-cache group arithmetic (bytes -> f16 fragments, f16 MMAs; see attend_kv8.cu for the fragment layouts).
+template <int D, int NW, int NSTAGE, bool PAGED, int GT, int KV = 0>
 __global__ void __launch_bounds__(NW * 32) attend_layer_kernel(const __grid_constant__ AttendArgs a) {
-    using T = __nv_bfloat16;
+    using T = __nv_bfloat16;  // type of q, k_new, v_new, out (and of a bf16 cache)
+    constexpr bool BYTES = KV != 0, E5M2 = KV == 2;
     constexpr int NT = NW * 32;
-    constexpr int ROW_BYTES = D * 2;
+    constexpr int ROW_BYTES = BYTES ? D : D * 2;
     constexpr int CHUNKS = ROW_BYTES / 16;
+    constexpr int ROWS_PER_LINE = ROW_BYTES >= 128 ? 1 : 128 / ROW_BYTES;  // rows sharing a 128-byte line of shared memory
     constexpr int TILE_BYTES = kGroupTokens * ROW_BYTES;
     constexpr int STAGE_BYTES = 2 * TILE_BYTES;
     constexpr int WARP_BYTES = NSTAGE * STAGE_BYTES;
     constexpr int KS = D / 16;
+    constexpr int MT = D / 32;  // byte caches: 32-wide blocks of the output dimension
     static_assert(WARP_BYTES >= kMaxGroup * D * 4, "per-warp stage area doubles as the partial-output buffer");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     // layout: stages [NW][NSTAGE][K tile | V tile] | LayerSmem | lg [chunk_tokens][GP]
     unsigned char* stage_base = smem_raw;
     LayerSmem& ls = *reinterpret_cast<LayerSmem*>(smem_raw + (size_t)NW * WARP_BYTES);
     float* lg = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(&ls) + sizeof(LayerSmem));
+
+    // placement of 16-byte chunk c of row r in a tile: the eight rows an ldmatrix touches land in eight different chunk
+    // positions of their 128-byte lines
+    auto swz = [](int r, int c) -> uint32_t {
+        return (uint32_t)(r * ROW_BYTES + ((c ^ ((r / ROWS_PER_LINE) & (CHUNKS < 8 ? CHUNKS - 1 : 7))) << 4));
+    };
 
     const bool early = a.early_prefetch != 0;
     if (!early) asm volatile("griddepcontrol.wait;" ::: "memory");  // nothing is read before the previous kernel is done
@@ -133,7 +145,7 @@ __global__ void __launch_bounds__(NW * 32) attend_layer_kernel(const __grid_cons
             const int r = idx / CHUNKS, c = idx % CHUNKS;
             const bool valid = ok && (tok0 + r < n);
             const int soff = valid ? r * ROW_BYTES + c * 16 : 0;
-            const uint32_t doff = r * ROW_BYTES + ((c ^ (r & 7)) << 4);
+            const uint32_t doff = swz(r, c);
             cp_async16_hint(ks_u32 + doff, kb + soff, valid ? 16 : 0, stream_policy);
             cp_async16_hint(vs_u32 + doff, vb + soff, valid ? 16 : 0, stream_policy);
         }
@@ -171,15 +183,30 @@ __global__ void __launch_bounds__(NW * 32) attend_layer_kernel(const __grid_cons
         return;
     }
 
-    // Q^T fragments (B operand): b0 = Q[head gq][16 ks + 2 tq, +1], b1 = Q[head gq][16 ks + 8 + 2 tq, +1]
+    // Q^T fragments (B operand).  bf16 cache: b0 = Q[head gq][16 ks + 2 tq, +1], b1 = Q[head gq][16 ks + 8 + 2 tq, +1].
+    // Byte cache: f16, in the permuted order of the key bytes (b0 = Q[head gq][16 ks + 4 tq + {0, 1}], b1 = ... + {2, 3}),
+    // the row divided by the power of two qdiv first so that it fits f16 (the head's logits are multiplied back).
     uint32_t bq[KS][2];
-    {
+    float qdiv = 1.f;
+    if constexpr (!BYTES) {
         const uint32_t* qrow =
             reinterpret_cast<const uint32_t*>((const T*)a.q + ((size_t)(ic.li * a.B + ic.b) * a.Hq + ic.hkv * G + gq) * D);
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
             bq[ks][0] = (gq < G) ? qrow[8 * ks + tq] : 0u;
             bq[ks][1] = (gq < G) ? qrow[8 * ks + 4 + tq] : 0u;
+        }
+    } else {
+        const uint2* qrow =
+            reinterpret_cast<const uint2*>((const T*)a.q + ((size_t)(ic.li * a.B + ic.b) * a.Hq + ic.hkv * G + gq) * D);
+        uint2 w[KS];
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) w[ks] = gq < G ? qrow[4 * ks + tq] : make_uint2(0u, 0u);
+        const float inv = query_row_scale(w, qdiv);
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            bq[ks][0] = bf16x2_to_f16x2_scaled(w[ks].x, inv);
+            bq[ks][1] = bf16x2_to_f16x2_scaled(w[ks].y, inv);
         }
     }
     // Sec. 4.1: append the generated token's key / value; the CTA whose range holds slot n_old stores it.
@@ -188,15 +215,31 @@ __global__ void __launch_bounds__(NW * 32) attend_layer_kernel(const __grid_cons
         const size_t src = ((size_t)(ic.li * a.B + ic.b) * a.Hkv + ic.hkv) * ROW_BYTES;
         char* kd = const_cast<char*>(row_ptr<PAGED>(a, a.k, ic.item, n_old, ROW_BYTES, &bad_page));
         char* vd = const_cast<char*>(row_ptr<PAGED>(a, a.v, ic.item, n_old, ROW_BYTES, &bad_page));
-        if (kd && vd && lane * 16 < ROW_BYTES) {
-            *reinterpret_cast<uint4*>(kd + lane * 16) = *reinterpret_cast<const uint4*>((const char*)a.k_new + src + lane * 16);
-            *reinterpret_cast<uint4*>(vd + lane * 16) = *reinterpret_cast<const uint4*>((const char*)a.v_new + src + lane * 16);
+        if constexpr (!BYTES) {
+            if (kd && vd && lane * 16 < ROW_BYTES) {
+                *reinterpret_cast<uint4*>(kd + lane * 16) = *reinterpret_cast<const uint4*>((const char*)a.k_new + src + lane * 16);
+                *reinterpret_cast<uint4*>(vd + lane * 16) = *reinterpret_cast<const uint4*>((const char*)a.v_new + src + lane * 16);
+            }
+        } else if (kd && vd && lane * 4 < D) {  // quantised: x / scale in fp32, round to nearest even, saturate; four elements per lane
+            const float ks_l = a.k_scale[ic.l], vs_l = a.v_scale[ic.l];
+            const uint2 kw = *reinterpret_cast<const uint2*>((const T*)a.k_new + src + lane * 4);
+            const uint2 vw = *reinterpret_cast<const uint2*>((const T*)a.v_new + src + lane * 4);
+            auto quant4 = [](uint2 w, float sc) -> uint32_t {
+                const float x0 = __uint_as_float(w.x << 16), x1 = __uint_as_float(w.x & 0xffff0000u);
+                const float x2 = __uint_as_float(w.y << 16), x3 = __uint_as_float(w.y & 0xffff0000u);
+                return f32x2_to_fp8x2<E5M2>(__fdiv_rn(x0, sc), __fdiv_rn(x1, sc)) | (f32x2_to_fp8x2<E5M2>(__fdiv_rn(x2, sc), __fdiv_rn(x3, sc)) << 16);
+            };
+            *reinterpret_cast<uint32_t*>(kd + lane * 4) = quant4(kw, ks_l);
+            *reinterpret_cast<uint32_t*>(vd + lane * 4) = quant4(vw, vs_l);
         }
         if (lane == 0) a.pos[(size_t)ic.item * a.cap_tokens + n_old] = a.token_pos[ic.b];
     }
     if (i_append) __syncthreads();  // (uniform for the CTA) the appended row is in global memory before any warp streams it
 
-    const float sl2 = a.scale_log2[ic.l];
+    const float sl2 = a.scale_log2[ic.l];  // (byte caches: the key scale is folded in by the host)
+    // byte caches: this thread's two logit columns are heads 2 tq and 2 tq + 1, whose query divisors sit in the lanes with gq = head
+    const float sl2_0 = BYTES ? sl2 * __shfl_sync(0xffffffffu, qdiv, (2 * tq) * 4) : sl2;
+    const float sl2_1 = BYTES ? sl2 * __shfl_sync(0xffffffffu, qdiv, (2 * tq + 1) * 4) : sl2;
 #pragma unroll
     for (int s = 0; s < NSTAGE - 1; ++s) {
         if (s >= pre) {
@@ -220,11 +263,14 @@ __global__ void __launch_bounds__(NW * 32) attend_layer_kernel(const __grid_cons
 
     float m0 = -INFINITY, m1 = -INFINITY;
     float l0 = 0.f, l1 = 0.f;
+    // O^T fragments.  bf16: block mt covers d = 16 mt .. + 15 (rows gq, gq + 8).  Bytes: block mt / parity par covers
+    // d = 32 mt + 2 gq + par and d + 16; o8 aliases the same registers as [MT][2][4].
     float o[KS][4];
 #pragma unroll
     for (int mt = 0; mt < KS; ++mt)
 #pragma unroll
         for (int i = 0; i < 4; ++i) o[mt][i] = 0.f;
+    float (&o8)[MT][2][4] = reinterpret_cast<float (&)[MT][2][4]>(o);
 
     const int k_row = (lane & 7) + ((lane >> 3) & 1) * 8, k_chunk = lane >> 4;
     const int v_row = (lane & 7) + ((lane >> 4) & 1) * 8, v_chunk = (lane >> 3) & 1;
@@ -238,18 +284,32 @@ __global__ void __launch_bounds__(NW * 32) attend_layer_kernel(const __grid_cons
         const uint32_t vs_u32 = ks_u32 + TILE_BYTES;
 
         float ca[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f};
+        if constexpr (!BYTES) {
 #pragma unroll
-        for (int ks = 0; ks < KS; ++ks) {
-            uint32_t af[4];
-            ldmatrix_x4(ks_u32 + k_row * ROW_BYTES + (((2 * ks + k_chunk) ^ (k_row & 7)) << 4), af);
-            if (ks & 1) mma_bf16(cb, af, bq[ks][0], bq[ks][1]);
-            else mma_bf16(ca, af, bq[ks][0], bq[ks][1]);
+            for (int ks = 0; ks < KS; ++ks) {
+                uint32_t af[4];
+                ldmatrix_x4(ks_u32 + k_row * ROW_BYTES + (((2 * ks + k_chunk) ^ (k_row & 7)) << 4), af);
+                if (ks & 1) mma_bf16(cb, af, bq[ks][0], bq[ks][1]);
+                else mma_bf16(ca, af, bq[ks][0], bq[ks][1]);
+            }
+        } else {
+#pragma unroll
+            for (int pr = 0; pr < KS / 2; ++pr) {  // 32 bytes of every key row: two k-steps
+                uint32_t r[4];                     // rows gq | gq + 8 of bytes [32 pr, +16) | rows gq | gq + 8 of [32 pr + 16, +16)
+                ldmatrix_x4(ks_u32 + swz(k_row, 2 * pr + k_chunk), r);
+                const uint32_t a0[4] = {bytes_to_f16x2<E5M2, 0, 1>(r[0]), bytes_to_f16x2<E5M2, 0, 1>(r[1]),
+                                        bytes_to_f16x2<E5M2, 2, 3>(r[0]), bytes_to_f16x2<E5M2, 2, 3>(r[1])};
+                const uint32_t a1[4] = {bytes_to_f16x2<E5M2, 0, 1>(r[2]), bytes_to_f16x2<E5M2, 0, 1>(r[3]),
+                                        bytes_to_f16x2<E5M2, 2, 3>(r[2]), bytes_to_f16x2<E5M2, 2, 3>(r[3])};
+                mma_f16(ca, a0, bq[2 * pr][0], bq[2 * pr][1]);
+                mma_f16(cb, a1, bq[2 * pr + 1][0], bq[2 * pr + 1][1]);
+            }
         }
         const int tokA = grp * kGroupTokens + gq, tokB = tokA + 8;
-        float s00 = (tokA < n) ? (ca[0] + cb[0]) * sl2 : -INFINITY;
-        float s01 = (tokA < n) ? (ca[1] + cb[1]) * sl2 : -INFINITY;
-        float s10 = (tokB < n) ? (ca[2] + cb[2]) * sl2 : -INFINITY;
-        float s11 = (tokB < n) ? (ca[3] + cb[3]) * sl2 : -INFINITY;
+        float s00 = (tokA < n) ? (ca[0] + cb[0]) * sl2_0 : -INFINITY;
+        float s01 = (tokA < n) ? (ca[1] + cb[1]) * sl2_1 : -INFINITY;
+        float s10 = (tokB < n) ? (ca[2] + cb[2]) * sl2_0 : -INFINITY;
+        float s11 = (tokB < n) ? (ca[3] + cb[3]) * sl2_1 : -INFINITY;
         if (2 * tq < GP) {
             *reinterpret_cast<float2*>(lg + (size_t)(tokA - t0) * GP + 2 * tq) = make_float2(s00, s01);
             *reinterpret_cast<float2*>(lg + (size_t)(tokB - t0) * GP + 2 * tq) = make_float2(s10, s11);
@@ -277,13 +337,32 @@ __global__ void __launch_bounds__(NW * 32) attend_layer_kernel(const __grid_cons
         const float p10 = fast_exp2(s10 - m0), p11 = fast_exp2(s11 - m1);
         l0 += p00 + p10;
         l1 += p01 + p11;
-        const uint32_t pb0 = movmatrix_trans(pack_bf16(p00, p01));
-        const uint32_t pb1 = movmatrix_trans(pack_bf16(p10, p11));
+        if constexpr (!BYTES) {
+            const uint32_t pb0 = movmatrix_trans(pack_bf16(p00, p01));
+            const uint32_t pb1 = movmatrix_trans(pack_bf16(p10, p11));
 #pragma unroll
-        for (int mt = 0; mt < KS; ++mt) {
-            uint32_t af[4];
-            ldmatrix_x4_trans(vs_u32 + v_row * ROW_BYTES + (((2 * mt + v_chunk) ^ (v_row & 7)) << 4), af);
-            mma_bf16(o[mt], af, pb0, pb1);
+            for (int mt = 0; mt < KS; ++mt) {
+                uint32_t af[4];
+                ldmatrix_x4_trans(vs_u32 + v_row * ROW_BYTES + (((2 * mt + v_chunk) ^ (v_row & 7)) << 4), af);
+                mma_bf16(o[mt], af, pb0, pb1);
+            }
+        } else {
+            const uint32_t pb0 = movmatrix_trans(pack_f16(p00, p01));
+            const uint32_t pb1 = movmatrix_trans(pack_f16(p10, p11));
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                // per register: the byte pairs (d, d + 1) of two consecutive tokens; a byte permute separates even and odd d
+                uint32_t r[4];
+                ldmatrix_x4_trans(vs_u32 + swz(v_row, 2 * mt + v_chunk), r);
+                uint32_t ae[4], ao[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    ae[i] = bytes_to_f16x2<E5M2, 0, 2>(r[i]);
+                    ao[i] = bytes_to_f16x2<E5M2, 1, 3>(r[i]);
+                }
+                mma_f16(o8[mt][0], ae, pb0, pb1);
+                mma_f16(o8[mt][1], ao, pb0, pb1);
+            }
         }
         __syncwarp();
         const int nxt = it + NSTAGE - 1;
@@ -305,12 +384,26 @@ __global__ void __launch_bounds__(NW * 32) attend_layer_kernel(const __grid_cons
         ls.wstat[warp][2 * tq + 1] = make_float2(m1, l1);
     }
     float* wo = reinterpret_cast<float*>(my_stage);
+    if constexpr (!BYTES) {
 #pragma unroll
-    for (int mt = 0; mt < KS; ++mt) {
-        wo[(2 * tq) * D + 16 * mt + gq] = o[mt][0];
-        wo[(2 * tq + 1) * D + 16 * mt + gq] = o[mt][1];
-        wo[(2 * tq) * D + 16 * mt + gq + 8] = o[mt][2];
-        wo[(2 * tq + 1) * D + 16 * mt + gq + 8] = o[mt][3];
+        for (int mt = 0; mt < KS; ++mt) {
+            wo[(2 * tq) * D + 16 * mt + gq] = o[mt][0];
+            wo[(2 * tq + 1) * D + 16 * mt + gq] = o[mt][1];
+            wo[(2 * tq) * D + 16 * mt + gq + 8] = o[mt][2];
+            wo[(2 * tq + 1) * D + 16 * mt + gq + 8] = o[mt][3];
+        }
+    } else {
+        const float vs_l = a.v_scale[ic.l];  // a stored value byte x means v_scale * x
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int par = 0; par < 2; ++par) {
+                const int d = 32 * mt + 2 * gq + par;
+                wo[(2 * tq) * D + d] = o8[mt][par][0] * vs_l;
+                wo[(2 * tq + 1) * D + d] = o8[mt][par][1] * vs_l;
+                wo[(2 * tq) * D + d + 16] = o8[mt][par][2] * vs_l;
+                wo[(2 * tq + 1) * D + d + 16] = o8[mt][par][3] * vs_l;
+            }
     }
     __syncthreads();   // every warp's (max, sum) and partial output are in shared memory
     cluster_wait();    // every peer has initialised its barrier (they arrived at the top of the kernel)
@@ -437,15 +530,15 @@ __global__ void __launch_bounds__(NW * 32) attend_layer_kernel(const __grid_cons
     if (append_slot >= 0 && ic.rank == 0 && tid == 0) a.len[ic.item] = n;
 }
 
-template <int D, int NW, int NSTAGE>
+template <int D, int NW, int NSTAGE, int KV = 0>
 static size_t layer_smem(int chunk_tokens, int GP) {
-    return (size_t)NW * NSTAGE * 2 * kGroupTokens * D * 2 + sizeof(LayerSmem) + (size_t)chunk_tokens * GP * 4;
+    return (size_t)NW * NSTAGE * 2 * kGroupTokens * D * (KV ? 1 : 2) + sizeof(LayerSmem) + (size_t)chunk_tokens * GP * 4;
 }
 
-template <int D, int NW, int NSTAGE, bool PAGED, int GT>
+template <int D, int NW, int NSTAGE, bool PAGED, int GT, int KV = 0>
 static cudaError_t launch_layer_t(const AttendArgs& a, cudaStream_t stream) {
-    auto kern = attend_layer_kernel<D, NW, NSTAGE, PAGED, GT>;
-    const size_t smem = layer_smem<D, NW, NSTAGE>(a.chunk_tokens, a.GP);
+    auto kern = attend_layer_kernel<D, NW, NSTAGE, PAGED, GT, KV>;
+    const size_t smem = layer_smem<D, NW, NSTAGE, KV>(a.chunk_tokens, a.GP);
     cudaError_t e = prepare_kernel((const void*)kern, smem);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
@@ -491,6 +584,18 @@ cudaError_t launch_attend_layer(const AttendArgs& a, int D, int shape, bool page
     LETHE_LAYER_SHAPES(X, 64)
 #undef X
     return cudaErrorInvalidValue;
+}
+
+// Quantised caches: 4 warps x 4 stages (a stage is half the bytes of a bf16 one), head_dim 128.
+size_t kv8_layer_smem_bytes(int chunk_tokens, int GP) { return layer_smem<128, 4, 4, 1>(chunk_tokens, GP); }
+
+cudaError_t launch_attend_kv8_layer(const AttendArgs& a, bool paged, bool e5m2, cudaStream_t stream) {
+#define LETHE_L8(GT)                                                                                                   \
+    (paged ? (e5m2 ? launch_layer_t<128, 4, 4, true, GT, 2>(a, stream) : launch_layer_t<128, 4, 4, true, GT, 1>(a, stream))   \
+           : (e5m2 ? launch_layer_t<128, 4, 4, false, GT, 2>(a, stream) : launch_layer_t<128, 4, 4, false, GT, 1>(a, stream)))
+    if (a.G == 4) return LETHE_L8(4);
+    return LETHE_L8(0);
+#undef LETHE_L8
 }
 
 }  // namespace lethe
