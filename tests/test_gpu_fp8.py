@@ -405,3 +405,51 @@ def test_quantised_query_magnitudes(ctx, variant):
             _step(ctx, oc, gc, q, kn, vn, torch.arange(B, dtype=torch.int32) + 300 + step, scale, 0.95, want_lse=(step == 1))
     finally:
         ctx.set_tuning(0, 0)
+
+
+@pytest.mark.parametrize("fmt,paged,splits", [("e4m3", False, 0), ("e4m3", True, 4), ("e5m2", False, 2)])
+def test_quantised_layer_by_layer_with_pipelining(ctx, fmt, paged, splits):
+    """One launch per layer on a quantised cache, with the layer pipelining on (a launch fetches cached K / V tiles
+    before the previous layer's launch has completed), several appending steps, then the same layer twice in a row
+    (the second launch depends on the first one's append and must not take the early fetch)."""
+    L, B, Hq, Hkv, D, cap = 6, 3, 32, 8, 128, 352
+    g = torch.Generator().manual_seed(23 + paged)
+    lens = torch.randint(200, 330, (L, B, Hkv), generator=g)
+    lens[2, 1, 3] = 15; lens[4, 0, 0] = 1; lens[5, 2, 7] = 340
+    oc = fp8_cache(L, B, Hq, Hkv, D, cap, lens, seed=29, k_scale=[0.4, 0.6, 0.8, 0.5, 1.0, 0.7], v_scale=[1.0, 0.5, 2.0, 0.7, 0.9, 1.3],
+                   page_tokens=16 if paged else 0, fmt=fmt)
+    gc = to_device(oc)
+    dev = gc.device
+    scale = torch.tensor([0.1, 0.08, 0.12, 0.09, 0.1, 0.11], dtype=torch.float32)
+    ctx.set_tuning(44 if splits else 0, splits)
+    ctx.set_tuning(51, 0)
+    try:
+        for step in range(5):
+            q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+            kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            vn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            tp = torch.arange(B, dtype=torch.int32) + 400 + step
+            st, ref, _, _ = oracle.decode_attend(oc, 0, L, q, kn, vn, tp, scale, 0.97)
+            assert st == oracle.OK
+            out = torch.full_like(q, float("nan"), device=dev)
+            qd, kd, vd, td = q.to(dev), kn.to(dev), vn.to(dev), tp.to(dev)
+            for l in range(L):                                       # back to back, nothing in between
+                ctx.decode_attend(gc, l, l + 1, qd[l:l + 1], kd[l:l + 1], vd[l:l + 1], td, scale.tolist(), 0.97, out[l:l + 1])
+            assert ctx.poll_status()[0] == 0
+            d = (out.cpu().float() - ref.float()).abs()
+            assert bool((d <= 2e-2 + 2.0 ** -7 * ref.float().abs()).all()), f"attention output error {d.max().item()}"
+            assert_state_matches(gc, oc)
+        for rep in range(2):                                         # the same layer twice in a row
+            q = torch.randn((L, B, Hq, D), generator=g).to(torch.bfloat16)
+            kn = torch.randn((L, B, Hkv, D), generator=g).to(torch.bfloat16)
+            tp = torch.arange(B, dtype=torch.int32) + 500 + rep
+            st, ref, _, _ = oracle.decode_attend(oc, 3, 4, q[3:4], kn[3:4], kn[3:4], tp, scale, 0.97)
+            out = torch.zeros_like(q[3:4], device=dev)
+            ctx.decode_attend(gc, 3, 4, q[3:4].to(dev), kn[3:4].to(dev), kn[3:4].to(dev), tp.to(dev), scale.tolist(), 0.97, out)
+        assert ctx.poll_status()[0] == 0
+        d = (out.cpu().float() - ref.float()).abs()
+        assert bool((d <= 2e-2 + 2.0 ** -7 * ref.float().abs()).all())
+        assert_state_matches(gc, oc)
+    finally:
+        ctx.set_tuning(50, 0)
+        ctx.set_tuning(0, 0)
