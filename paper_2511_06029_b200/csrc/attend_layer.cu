@@ -30,7 +30,7 @@ struct LayerSmem {
     unsigned long long bar;             // one arrival per rank of the cluster, after that rank's pushes
     int abort;
     int pad;
-    float2 wstat[16][kMaxGroup];        // per warp, per head: (running max in log2 units, partial sum)
+    float2 wstat[8][kMaxGroup];         // per warp (at most 8 per CTA), per head: (running max in log2 units, partial sum)
     float2 peer_stat[16][kMaxGroup];    // pushed by rank r: its per-head (max, sum) over its whole token range
     alignas(16) float peer_o[kMaxGroup * 128 + 16]; // pushed by rank r: this CTA's slice of rank r's partial output, [S][per]
 };
@@ -79,6 +79,7 @@ __global__ void __launch_bounds__(NW * 32) attend_layer_kernel(const __grid_cons
     constexpr int KS = D / 16;
     constexpr int MT = D / 32;  // byte caches: 32-wide blocks of the output dimension
     static_assert(WARP_BYTES >= kMaxGroup * D * 4, "per-warp stage area doubles as the partial-output buffer");
+    static_assert(NW <= 8, "LayerSmem::wstat holds eight warps");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     // layout: stages [NW][NSTAGE][K tile | V tile] | LayerSmem | lg [chunk_tokens][GP]
     unsigned char* stage_base = smem_raw;
