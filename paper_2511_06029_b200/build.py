@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblethe.so")
-SOURCES = ["api.cu", "attend_simt.cu", "attend_mma.cu", "attend_layer.cu", "attend_stream.cu", "attend_async.cu", "attend_kv8.cu", "attend_kv8_tc.cu", "attend_kv8_tc_g4.cu", "attend_kv8_tc_g7.cu", "attend_kv8_tc_g8.cu", "attend_kv8_tc_n16.cu", "attend_kv8_tc_n32.cu", "attend_kv8_stream.cu", "prune.cu", "prefill.cu", "prefill_tc.cu"]
+SOURCES = ["api.cu", "attend_simt.cu", "attend_mma.cu", "attend_layer.cu", "attend_stream.cu", "attend_async.cu", "attend_kv8.cu", "attend_kv8_tc.cu", "attend_kv8_tc_g4.cu", "attend_kv8_tc_g5.cu", "attend_kv8_tc_g7.cu", "attend_kv8_tc_g8.cu", "attend_kv8_tc_n16.cu", "attend_kv8_tc_n32.cu", "attend_kv8_stream.cu", "prune.cu", "prefill.cu", "prefill_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-O2"]
 

@@ -804,8 +804,12 @@ cudaError_t launch_attend_async(const AttendArgs& a, int D, int shape, bool page
     TmaMaps none;
     memset(&none, 0, sizeof(none));
     const TmaMaps& m = (tma && maps) ? *reinterpret_cast<const TmaMaps*>(maps) : none;
-    // the default shape on the most common geometry (four query heads per KV head), group size compiled in
-    if (D == 128 && shape == 0 && !tma && a.G == 4) return dispatch_async<128, 8, 2, false, 4>(a, m, paged, grid, stream);
+    // the default shape on the common geometries (four, five or eight query heads per KV head), group size compiled in
+    if (D == 128 && shape == 0 && !tma) {
+        if (a.G == 4) return dispatch_async<128, 8, 2, false, 4>(a, m, paged, grid, stream);
+        if (a.G == 5) return dispatch_async<128, 8, 2, false, 5>(a, m, paged, grid, stream);
+        if (a.G == 8) return dispatch_async<128, 8, 2, false, 8>(a, m, paged, grid, stream);
+    }
 #define X(id, DD, NW, NS)                                                                            \
     if (shape == id && D == DD)                                                                      \
         return tma ? dispatch_async<DD, NW, NS, true>(a, m, paged, grid, stream) : dispatch_async<DD, NW, NS, false>(a, m, paged, grid, stream);

@@ -1,5 +1,5 @@
 // Host side of the tensor-memory kernel for quantised caches (attend_kv8_tc.cuh): shared-memory size, tensor maps,
-// and the choice of the instance: the group sizes of the common model geometries (4, 7 and 8 query heads per KV
+// and the choice of the instance: the group sizes of the common model geometries (4, 5, 7 and 8 query heads per KV
 // head) are compiled in, every other one runs the instances that read it from the arguments.
 #include "attend_kv8_tc.cuh"
 
@@ -41,6 +41,7 @@ bool build_kv8_tc_maps(void* encode, void* k, void* v, unsigned long long rows, 
 #define LETHE_KV8TC_DECL(name) \
     cudaError_t name(const AttendArgs& a, const void* maps, bool paged, bool e5m2, int nslot, int cap_pad, int grid, cudaStream_t stream)
 LETHE_KV8TC_DECL(launch_kv8_tc_g4);
+LETHE_KV8TC_DECL(launch_kv8_tc_g5);
 LETHE_KV8TC_DECL(launch_kv8_tc_g7);
 LETHE_KV8TC_DECL(launch_kv8_tc_g8);
 LETHE_KV8TC_DECL(launch_kv8_tc_n16);
@@ -53,6 +54,7 @@ cudaError_t launch_attend_kv8_tc(const AttendArgs& a, const void* maps, bool pag
     if (ng != 2) return cudaErrorInvalidValue;
     switch (a.G) {
         case 4: return launch_kv8_tc_g4(a, maps, paged, e5m2, nslot, cap_pad, grid, stream);
+        case 5: return launch_kv8_tc_g5(a, maps, paged, e5m2, nslot, cap_pad, grid, stream);
         case 7: return launch_kv8_tc_g7(a, maps, paged, e5m2, nslot, cap_pad, grid, stream);
         case 8: return launch_kv8_tc_g8(a, maps, paged, e5m2, nslot, cap_pad, grid, stream);
         default: break;

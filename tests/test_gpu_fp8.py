@@ -247,10 +247,10 @@ TENSOR_MEMORY = 14                                                   # lethe_set
 
 @pytest.mark.parametrize("fmt", ["e4m3", "e5m2"])
 @pytest.mark.parametrize("paged", [False, True])
-@pytest.mark.parametrize("Hq,Hkv", [(8, 2), (7, 1), (16, 2), (5, 5), (24, 4)])
+@pytest.mark.parametrize("Hq,Hkv", [(8, 2), (7, 1), (16, 2), (5, 5), (24, 4), (10, 2)])
 def test_quantised_tensor_memory_kernel(ctx, Hq, Hkv, paged, fmt):
     """The tcgen05 kernel (cache bytes straight into the MMAs, queries and probabilities as three e4m3 terms) on
-    G = 4, 7, 8, 1, 6: lengths around the 128-token tile (1, 127, 128, 129, 255, 256, 257), several tiles per item,
+    G = 4, 7, 8, 1, 6, 5: lengths around the 128-token tile (1, 127, 128, 129, 255, 256, 257), several tiles per item,
     appending and attend-only steps, a new token beyond the representable range, an empty and a full item."""
     L, B, D, cap = 2, 3, 128, 416
     g = torch.Generator().manual_seed(Hq * 10 + paged)

@@ -103,6 +103,8 @@ CASES = [
     (torch.bfloat16, 64, 8, 2, 300, 46, 2),
     (torch.bfloat16, 128, 28, 4, 700, 46, 4),            # seven query heads per KV head: the instance with the group size compiled in
     (torch.bfloat16, 128, 28, 4, 300, 8, 0),             # the same for the persistent kernel's automatic shape
+    (torch.bfloat16, 128, 40, 8, 300, 16, 0),            # five and eight heads per KV head: the asynchronous kernel's compiled-in sizes
+    (torch.bfloat16, 128, 64, 8, 300, 16, 0),
     (torch.bfloat16, 64, 10, 2, 500, 47, 4),
     (torch.bfloat16, 128, 32, 8, 300, 48, 0),
     (torch.bfloat16, 64, 16, 2, 300, 49, 2),
