@@ -100,7 +100,8 @@ __device__ __forceinline__ int opaque(int x) {
 
 }  // namespace
 
-template <int D, int NW, int NS, bool PAGED, bool SPILL>
+// GT: query heads per KV head when known at compile time (0 = from the arguments).
+template <int D, int NW, int NS, bool PAGED, bool SPILL, int GT = 0>
 __global__ void __launch_bounds__(NW * 32, 1) attend_kv8_stream_kernel(const __grid_constant__ AttendArgs a) {
     using T = __nv_bfloat16;
     constexpr int NT = NW * 32;
@@ -120,7 +121,7 @@ __global__ void __launch_bounds__(NW * 32, 1) attend_kv8_stream_kernel(const __g
     };
     extern __shared__ __align__(128) unsigned char smem_raw[];
     // layout: stages [NW][NS][K tile | V tile] | wo [NW][GP][D] fp32 | EpilogueSmem | lg [chunk_tokens][GP]
-    const int G = a.G, GP = a.GP;
+    const int G = GT ? GT : a.G, GP = GT ? ((GT + 1) & ~1) : a.GP;
     const int wo_stride = GP * D;
     float* wo_all = reinterpret_cast<float*>(smem_raw + (size_t)NW * WARP_BYTES);
     EpilogueSmem& es = *reinterpret_cast<EpilogueSmem*>(wo_all + (size_t)NW * wo_stride);
@@ -527,9 +528,9 @@ static size_t kv8s_smem(int chunk_tokens, int GP) {
            (size_t)chunk_tokens * GP * 4;
 }
 
-template <int D, int NW, int NS, bool PAGED, bool SPILL>
+template <int D, int NW, int NS, bool PAGED, bool SPILL, int GT = 0>
 static cudaError_t launch_kv8s_t(const AttendArgs& a, int grid, cudaStream_t stream) {
-    auto kern = attend_kv8_stream_kernel<D, NW, NS, PAGED, SPILL>;
+    auto kern = attend_kv8_stream_kernel<D, NW, NS, PAGED, SPILL, GT>;
     const size_t smem = kv8s_smem<D, NW, NS>(a.chunk_tokens, a.GP);
     cudaError_t e = prepare_kernel((const void*)kern, smem);
     if (e != cudaSuccess) return e;
@@ -537,11 +538,11 @@ static cudaError_t launch_kv8s_t(const AttendArgs& a, int grid, cudaStream_t str
     return cudaGetLastError();
 }
 
-template <int D, int NW, int NS>
+template <int D, int NW, int NS, int GT = 0>
 static cudaError_t dispatch_kv8s(const AttendArgs& a, bool paged, int grid, cudaStream_t stream) {
     const bool spill = a.spill != nullptr;
-    if (paged) return spill ? launch_kv8s_t<D, NW, NS, true, true>(a, grid, stream) : launch_kv8s_t<D, NW, NS, true, false>(a, grid, stream);
-    return spill ? launch_kv8s_t<D, NW, NS, false, true>(a, grid, stream) : launch_kv8s_t<D, NW, NS, false, false>(a, grid, stream);
+    if (paged) return spill ? launch_kv8s_t<D, NW, NS, true, true, GT>(a, grid, stream) : launch_kv8s_t<D, NW, NS, true, false, GT>(a, grid, stream);
+    return spill ? launch_kv8s_t<D, NW, NS, false, true, GT>(a, grid, stream) : launch_kv8s_t<D, NW, NS, false, false, GT>(a, grid, stream);
 }
 
 // Shapes of the persistent kernel: (warps per CTA, stages per warp); tiles are half the size of the bf16 kernel's
@@ -558,6 +559,8 @@ size_t kv8_stream_smem_bytes(int D, int shape, int chunk_tokens, int GP) {
 }
 
 cudaError_t launch_attend_kv8_stream(const AttendArgs& a, int D, int shape, bool paged, int grid, cudaStream_t stream) {
+    // the automatic fallback for wide groups at large capacities (seven query heads per KV head), group size compiled in
+    if (D == 128 && shape == 0 && a.G == 7) return dispatch_kv8s<128, 8, 4, 7>(a, paged, grid, stream);
 #define X(id, DD, NW, NS)                                                                                   \
     if (shape == id && D == DD)                                                                             \
         return dispatch_kv8s<DD, NW, NS>(a, paged, grid, stream);
