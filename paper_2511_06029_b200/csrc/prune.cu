@@ -132,15 +132,24 @@ __device__ __forceinline__ uint32_t score_key(float x) {
 
 constexpr int kPruneThreads = 512;
 
-__device__ __forceinline__ char* prune_row_ptr(const CacheView& c, void* base, size_t item, int slot, int row_bytes,
-                                               bool* bad) {
-    if (!c.paged) return (char*)base + (item * c.capacity + slot) * row_bytes;
-    const int page = c.page_table[item * c.capacity + slot / c.page_tokens];
+// Row index (in rows of the K / V arrays, which share it) of logical slot `slot` of an item, or -1 for a page id
+// outside the pool.  Pages of 16 tokens, the only size the tensor-core kernels take, are split with a shift.
+__device__ __forceinline__ long long prune_row_index(const CacheView& c, size_t item, int slot, bool* bad) {
+    if (!c.paged) return (long long)(item * c.capacity + slot);
+    int pg, within;
+    if (c.page_tokens == 16) {
+        pg = slot >> 4;
+        within = slot & 15;
+    } else {
+        pg = slot / c.page_tokens;
+        within = slot % c.page_tokens;
+    }
+    const int page = c.page_table[item * c.capacity + pg];
     if (page < 0 || page >= c.n_pages) {
         *bad = true;
-        return nullptr;
+        return -1;
     }
-    return (char*)base + ((size_t)page * c.page_tokens + slot % c.page_tokens) * row_bytes;
+    return (long long)page * c.page_tokens + within;
 }
 
 // Block-wide exclusive scan of one counter per thread (kPruneThreads threads): returns this thread's
@@ -282,8 +291,9 @@ __device__ __forceinline__ void move_wave_load(const CacheView& c, size_t item, 
         w.rv[r] = 0.f;
         w.pv[r] = 0;
         if (w.srcs[r] >= 0) {
-            const char* ks = prune_row_ptr(c, c.k, item, w.srcs[r], row_bytes, &bad);
-            const char* vs = prune_row_ptr(c, c.v, item, w.srcs[r], row_bytes, &bad);
+            const long long row = prune_row_index(c, item, w.srcs[r], &bad);  // K and V rows share the index
+            const char* ks = row < 0 ? nullptr : (const char*)c.k + (size_t)row * row_bytes;
+            const char* vs = row < 0 ? nullptr : (const char*)c.v + (size_t)row * row_bytes;
             if (ks && vs) {
                 w.kv[r] = *reinterpret_cast<const uint4*>(ks + piece * 16);
                 w.vv[r] = *reinterpret_cast<const uint4*>(vs + piece * 16);
@@ -302,8 +312,9 @@ __device__ __forceinline__ void move_wave_store(const CacheView& c, size_t item,
     for (int r = 0; r < RPT; ++r) {
         if (w.srcs[r] >= 0) {
             const int dst = w0 + r * slots + rslot;
-            char* kd = prune_row_ptr(c, c.k, item, dst, row_bytes, &bad);
-            char* vd = prune_row_ptr(c, c.v, item, dst, row_bytes, &bad);
+            const long long row = prune_row_index(c, item, dst, &bad);
+            char* kd = row < 0 ? nullptr : (char*)c.k + (size_t)row * row_bytes;
+            char* vd = row < 0 ? nullptr : (char*)c.v + (size_t)row * row_bytes;
             if (kd && vd) {
                 *reinterpret_cast<uint4*>(kd + piece * 16) = w.kv[r];
                 *reinterpret_cast<uint4*>(vd + piece * 16) = w.vv[r];
