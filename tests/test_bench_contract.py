@@ -55,3 +55,16 @@ def test_gpu_arm_prints_the_contract_line():
     assert wp["ms_per_step"] > c["attend_ms_per_step"] and 0.3 < wp["frac"] <= r["frac"]
     import bench
     assert set(c) == set(bench.CONFIG_KEYS)
+
+
+@pytest.mark.gpu
+def test_gpu_arm_on_a_quantised_cache():
+    """The same line for `--kv fp8`: 264 algorithmic bytes per token-head, the per-layer launch mode included."""
+    d = _run(["--kv", "fp8", "--steps", "8", "--warmup", "3", "--prep-rounds", "1", "--no-cpu-baseline"], timeout=900)
+    assert BASE_KEYS <= set(d) and d["dtype"].startswith("fp8") and d["steps"] == 8
+    r, c = d["roofline"], d["config"]
+    assert abs(r["achieved"] - c["token_heads_per_step"] * 264 / (c["attend_ms_per_step"] * 1e-3) / 1e9) < 1e-6 * r["achieved"]
+    assert 0.3 < r["frac"] < 1.2 and d["gpu_launches"] >= 8
+    pl = c["per_layer_launch"]
+    assert pl["ms_per_step"] > c["attend_ms_per_step"] and 0.05 < pl["frac"] < r["frac"]
+    assert c["prune_rounds_timed"] >= 3 and d["e2e"]["h2d_bytes_per_step"] > 0
