@@ -265,9 +265,9 @@ __device__ __forceinline__ int sweep_keep(PruneShared& sh, KeyAt key_at, int n, 
 
 // Rows of K, V, rel, pos move to their destinations in ascending waves: load wave -> barrier -> store wave.
 // Because a survivor's destination never exceeds its source and waves ascend, no unread source is overwritten.
-// The loads of wave w + 1 are issued before the stores of wave w (its sources lie above every destination of wave
-// w, so the order between them is free): reads and writes then overlap instead of alternating, which matters
-// most where only one CTA fits an SM (long items).
+// A wave carries RPT rows per thread slot in registers: 4 where two CTAs share an SM, 8 in the instance whose CTA has
+// the SM (and its registers) to itself; deeper waves beat overlapping a wave's stores with the next wave's loads at
+// the same register budget (ragged round: 3.97 ms against 4.52 ms).
 template <int RPT_>
 struct MoveWave {
     static constexpr int RPT = RPT_;  // rows each thread slot carries per wave
@@ -326,7 +326,7 @@ __device__ __forceinline__ void move_wave_store(const CacheView& c, size_t item,
         }
     }
 }
-template <int RPT, bool PIPELINED>
+template <int RPT>
 __device__ __forceinline__ void move_rows(const CacheView& c, size_t item, int keep_n, const int32_t* src_list, bool& bad) {
     const int tid = threadIdx.x;
     float* rel = c.rel + item * c.cap_tokens;
@@ -336,25 +336,12 @@ __device__ __forceinline__ void move_rows(const CacheView& c, size_t item, int k
     const int slots = kPruneThreads / lanes_per_row;     // row slots per pass
     const int rows_per_wave = slots * RPT;
     const int piece = tid % lanes_per_row, rslot = tid / lanes_per_row;
-    if (keep_n <= 0) return;
-    if (!PIPELINED) {  // two CTAs share the SM and cover each other's barriers: one wave in registers at a time
-        for (int w0 = 0; w0 < keep_n; w0 += rows_per_wave) {
-            MoveWave<RPT> cur;
-            move_wave_load(c, item, keep_n, src_list, w0, slots, rslot, piece, row_bytes, rel, pos, cur, bad);
-            __syncthreads();  // every source row of this wave has been read
-            move_wave_store(c, item, w0, slots, rslot, piece, row_bytes, rel, pos, cur, bad);
-            // no barrier needed here: the next wave's sources lie above every destination written so far
-        }
-        return;
-    }
-    MoveWave<RPT> cur, nxt;
-    move_wave_load(c, item, keep_n, src_list, 0, slots, rslot, piece, row_bytes, rel, pos, cur, bad);
     for (int w0 = 0; w0 < keep_n; w0 += rows_per_wave) {
-        __syncthreads();  // every source row of wave w0 has been read by every thread
-        const bool more = w0 + rows_per_wave < keep_n;
-        if (more) move_wave_load(c, item, keep_n, src_list, w0 + rows_per_wave, slots, rslot, piece, row_bytes, rel, pos, nxt, bad);
+        MoveWave<RPT> cur;
+        move_wave_load(c, item, keep_n, src_list, w0, slots, rslot, piece, row_bytes, rel, pos, cur, bad);
+        __syncthreads();  // every source row of this wave has been read
         move_wave_store(c, item, w0, slots, rslot, piece, row_bytes, rel, pos, cur, bad);
-        if (more) cur = nxt;
+        // no barrier needed here: the next wave's sources lie above every destination written so far
     }
 }
 
@@ -367,7 +354,7 @@ __device__ __forceinline__ void move_rows(const CacheView& c, size_t item, int k
  *  4. rows move in ascending waves.
  */
 // DEEP: the item's keys take more shared memory than half an SM has, so one CTA has the SM (and its registers) to
-// itself and keeps two waves of rows in registers (the next wave's loads overlap this wave's stores).
+// itself and carries twice the rows per wave.
 template <bool DEEP>
 __global__ void __launch_bounds__(kPruneThreads, DEEP ? 1 : 2) rasr_prune_kernel(CacheView c, const int32_t* __restrict__ budgets,
                                                                    int recent, int sink, int32_t* keep_idx, int max_k,
@@ -413,7 +400,7 @@ __global__ void __launch_bounds__(kPruneThreads, DEEP ? 1 : 2) rasr_prune_kernel
     int32_t* src_list = in_smem ? reinterpret_cast<int32_t*>(dyn) : list_scratch + item * c.cap_tokens;
     const int keep_n = sweep_keep(sh, key_at, n, cand_lo, cand_hi, cand_lo, cand_hi, take > 0, T, need_eq, src_list, kout, max_k);
     bool bad = false;
-    move_rows<4, DEEP>(c, item, keep_n, src_list, bad);
+    move_rows<DEEP ? 8 : 4>(c, item, keep_n, src_list, bad);
     // any thread may have met the bad page id (each carries its own row slots): reduce over the CTA
     if (__syncthreads_or(bad) && tid == 0) record_error(status, LETHE_ERR_PAGE, (int)item);
     if (tid == 0) c.len[item] = keep_n;
@@ -488,7 +475,7 @@ __global__ void __launch_bounds__(kPruneThreads, 2) segment_prune_kernel(CacheVi
     const int keep_n = sweep_keep(sh, key_at, n, min(sink, n), max(n - recent, 0), 0, n, breakpoint > 0, T, need_eq, src_list,
                                   kout, max_k);
     bool bad = false;
-    move_rows<4, false>(c, item, keep_n, src_list, bad);
+    move_rows<4>(c, item, keep_n, src_list, bad);
     if (__syncthreads_or(bad) && tid == 0) record_error(status, LETHE_ERR_PAGE, (int)item);
     if (tid == 0) {
         c.len[item] = keep_n;
@@ -607,7 +594,7 @@ __global__ void __launch_bounds__(kPruneThreads, 2) collapsed_move_kernel(CacheV
     const int keep_n = plan[group];
     if (keep_n < 0) return;
     bool bad = false;
-    move_rows<4, false>(c, item, keep_n, lists + group * c.cap_tokens, bad);
+    move_rows<4>(c, item, keep_n, lists + group * c.cap_tokens, bad);
     if (__syncthreads_or(bad) && threadIdx.x == 0) record_error(status, LETHE_ERR_PAGE, (int)item);
     if (threadIdx.x == 0) c.len[item] = keep_n;
 }
